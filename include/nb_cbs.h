@@ -1,0 +1,163 @@
+/*
+ * nb_cbs.h -- C ABI of the B200 (sm_100a) Conv2d -> BatchNorm(training-mode batch statistics) -> SiLU
+ * block: forward, data gradient, weight gradient, and the stand-alone batch statistics.
+ *
+ * Conventions follow the paper's description of its C ABI (Sec. 4): nb_* names, opaque caller-owned
+ * handles with explicit destructors, runtime dtype tags, status codes plus a thread-local error
+ * string, additive versioning (struct_size field).  The operators are the ones the paper's case
+ * study uses (Sec. 6: convolutions with SiLU activations; Sec. 3.2 and Table 2 row 2: batch
+ * normalisation kept in F32 while convolutions run in 16-bit).  The paper prints no formula for
+ * them; the definitions below are those of the works it cites for BN and SiLU.
+ *
+ * Shapes and layouts (all tensors dense, innermost dimension contiguous):
+ *   x      [N][H][W][Cin]        input activation, NHWC
+ *   w      [Cout][k][k][Cin]     filter, k in {1,3}, cross-correlation (no flip), zero pad P = k/2
+ *   y,a,g,dy [N][Ho][Wo][Cout]   Ho = (H + 2P - k)/stride + 1, likewise Wo;  M = N*Ho*Wo rows
+ *   dx     like x, dw like w (always fp32)
+ *   gamma, beta, mean, invstd, running_*, dgamma, dbeta: fp32 [Cout]
+ *
+ * Element types by mode:
+ *   NB_MODE_BF16_TC : x, w, a, g, dy, dx are bf16; the saved convolution output y is IEEE fp16
+ *                     (an internal tensor: same bytes as bf16, 8x finer, saturated at +-65504);
+ *                     accumulation and all BN/SiLU arithmetic in fp32; dw, dgamma, dbeta fp32.
+ *   NB_MODE_F32_REF : every tensor fp32, plain FMA arithmetic (no tensor cores, no TF32).
+ *
+ * Every pointer is a DEVICE pointer on the plan's device unless its name starts with `host_`; the
+ * caller owns all memory, including the workspace.  Tensor pointers must be 16-byte aligned.
+ * Compute calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ * and return without synchronising.  Outputs are overwritten, never accumulated into.  Calls on one
+ * plan must not run concurrently (they share the plan's status block and the workspace).
+ * On invalid arguments nothing is launched and a non-zero status is returned; nb_last_error()
+ * then describes the problem.
+ */
+#ifndef NB_CBS_H
+#define NB_CBS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NB_CBS_ABI_VERSION 1u
+
+typedef int32_t nb_status;
+enum {
+    NB_OK = 0,
+    NB_ERR_INVALID_ARG = 1, /* NULL pointer, non-positive extent, bad enum, struct_size mismatch */
+    NB_ERR_UNSUPPORTED = 2, /* shape outside what the mode supports (see nb_cbs_plan_create) */
+    NB_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than nb_cbs_workspace_bytes reports */
+    NB_ERR_ALIGNMENT = 4,   /* a tensor pointer is not 16-byte aligned */
+    NB_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (no device, launch error, ...) */
+    NB_ERR_ARCH = 6,        /* the device is not compute capability 10.x */
+    NB_ERR_TIMEOUT = 7,     /* a kernel gave up a bounded wait (reported by nb_cbs_poll_status) */
+    NB_ERR_INTERNAL = 8
+};
+
+typedef enum { NB_DTYPE_F32 = 0, NB_DTYPE_BF16 = 1, NB_DTYPE_F16 = 2 } nb_dtype;
+typedef enum { NB_MODE_BF16_TC = 0, NB_MODE_F32_REF = 1 } nb_mode;
+
+/* nb_cbs_desc.flags */
+#define NB_CBS_FLAG_FORCE_SIMT 1u /* BF16 mode: run the three convolutions on the CUDA-core kernels
+                                     (same arithmetic contract; for testing and as a cross-check) */
+
+typedef struct nb_cbs_desc {
+    uint32_t struct_size; /* = sizeof(nb_cbs_desc) */
+    int32_t n, h, w, c_in, c_out;
+    int32_t ksize;  /* 1 or 3; pad = ksize/2 */
+    int32_t stride; /* 1 or 2 */
+    float eps;      /* added to the biased batch variance; 1e-3 in every benchmark configuration */
+    float momentum; /* running-statistics momentum; read only when running_* pointers are given */
+    int32_t mode;   /* nb_mode */
+    uint32_t flags;
+} nb_cbs_desc;
+
+typedef struct nb_cbs_plan_s* nb_cbs_plan;
+
+/* ABI revision of the loaded library (NB_CBS_ABI_VERSION at build time). */
+uint32_t nb_abi_version(void);
+
+/* Description of the last failure on the calling thread ("" if none); valid until the next nb_* call
+ * on this thread. */
+const char* nb_last_error(void);
+
+/* Create a plan for one block shape on CUDA device `device`.  Allocates a small (<= 4 KB) device
+ * status block; all other memory is the caller's.  Requirements: all extents > 0; ksize in {1,3};
+ * stride in {1,2}; BF16 mode: c_out % 8 == 0; F32 mode: c_out % 4 == 0; N*Ho*Wo >= 2.
+ * Errors: NB_ERR_INVALID_ARG, NB_ERR_UNSUPPORTED, NB_ERR_CUDA (no usable device), NB_ERR_ARCH. */
+nb_status nb_cbs_plan_create(const nb_cbs_desc* desc, int device, nb_cbs_plan* out_plan);
+
+/* Free the plan and its status block.  NULL is accepted. */
+nb_status nb_cbs_plan_destroy(nb_cbs_plan plan);
+
+/* Output extents Ho, Wo of the plan's shape. */
+nb_status nb_cbs_out_shape(nb_cbs_plan plan, int32_t* ho, int32_t* wo);
+
+/* Minimum workspace sizes in bytes for the forward call (also enough for nb_bn_stats) and for the two
+ * backward calls.  The workspace needs no initialisation and may be shared between plans whose calls
+ * do not overlap on the device; it must be 256-byte aligned. */
+nb_status nb_cbs_workspace_bytes(nb_cbs_plan plan, size_t* fwd_bytes, size_t* bwd_bytes);
+
+/* Which implementation each convolution of this plan runs on: writes three ints (fprop, dgrad, wgrad),
+ * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel. */
+nb_status nb_cbs_plan_paths(nb_cbs_plan plan, int32_t* paths3);
+
+/* Synchronise `stream`, then report whether any kernel launched through this plan gave up a bounded
+ * wait (NB_ERR_TIMEOUT) or saturated an fp16 store (still NB_OK; see nb_last_error()).  Clears the
+ * status block. */
+nb_status nb_cbs_poll_status(nb_cbs_plan plan, void* stream);
+
+/* Forward (Sec. 6 operators; BN in fp32 per Sec. 3.2 / Table 2 row 2):
+ *   y[n,p,q,c'] = sum_{r,t,c} x[n, p*s-P+r, q*s-P+t, c] * w[c',r,t,c]        (zero outside the image)
+ *   mean_c = (1/M) sum y ; var_c = (1/M) sum (y-mean_c)^2 (biased) ; invstd_c = (var_c + eps)^-1/2
+ *   a = z * sigmoid(z),  z = gamma_c * (y - mean_c) * invstd_c + beta_c
+ *   optional: running_mean <- (1-m) running_mean + m mean ; running_var <- (1-m) running_var + m var*M/(M-1)
+ * x, w, gamma, beta: inputs.  running_mean/running_var: both NULL or both given (in/out).
+ * y_saved, save_mean, save_invstd: outputs that the backward calls need.  a_out: the block's output. */
+nb_status nb_conv_bn_silu_fwd(nb_cbs_plan plan, const void* x, const void* w, const float* gamma, const float* beta,
+                              float* running_mean, float* running_var, void* y_saved, float* save_mean,
+                              float* save_invstd, void* a_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Stand-alone training-mode batch statistics of a [M][Cout] tensor (M = N*Ho*Wo of the plan):
+ * mean and invstd as in the forward call; optionally also the raw per-channel sum and sum of squares.
+ * y_dtype: NB_DTYPE_F16 in BF16 mode (the saved y), NB_DTYPE_F32 in F32 mode; anything else is
+ * NB_ERR_UNSUPPORTED.  sum / sumsq may be NULL. */
+nb_status nb_bn_stats(nb_cbs_plan plan, const void* y, int32_t y_dtype, float* mean, float* invstd, float* sum,
+                      float* sumsq, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward with respect to the block's input, gamma and beta, given g = dL/da:
+ *   s = sigmoid(z) ; dz = g * s * (1 + z*(1-s))                               (z recomputed from y_saved)
+ *   dbeta_c = sum dz ; dgamma_c = sum dz*xhat,  xhat = (y-mean_c)*invstd_c
+ *   dy = gamma_c*invstd_c * (dz - dbeta_c/M - xhat*dgamma_c/M)                 -> dy_out (kept for bwd_weight)
+ *   dx[n,h,w,c] = sum over (p,q,r,t,c') with p*s-P+r = h, q*s-P+t = w of dy[n,p,q,c'] * w[c',r,t,c]
+ * dx may be NULL (first layer of a network): then only dy_out, dgamma and dbeta are produced. */
+nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan plan, const void* g, const void* y_saved, const float* save_mean,
+                                   const float* save_invstd, const float* gamma, const float* beta, const void* w,
+                                   void* dx, float* dgamma, float* dbeta, void* dy_out, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+/* Backward with respect to the filter:
+ *   dw[c',r,t,c] = sum_{n,p,q} dy[n,p,q,c'] * x[n, p*s-P+r, q*s-P+t, c]        (fp32 output)
+ * dy is the tensor nb_conv_bn_silu_bwd_data wrote to dy_out (ordering on the stream is the caller's). */
+nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan plan, const void* x, const void* dy, float* dw, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
+/* One whole training step of the block from HOST buffers (the end-to-end path of a caller whose data
+ * lives in host memory): copies host_x, host_w, host_gamma, host_beta, host_g to the device, runs the
+ * forward call and the two backward calls above, and copies a, dx (unless host_dx is NULL), dw, dgamma,
+ * dbeta back, all on `stream`; returns after enqueueing (host buffers should be pinned for the copies to
+ * be asynchronous, and must stay valid until the stream is synchronised).  device_scratch is a device
+ * buffer of at least nb_cbs_step_host_scratch_bytes() bytes, 256-byte aligned, owned by the caller; it
+ * holds the device copies, the saved tensors and the workspace.  The paper has no counterpart of this
+ * entry point; it exists so that the host-to-host cost of the path can be measured. */
+nb_status nb_cbs_step_host_scratch_bytes(nb_cbs_plan plan, size_t* bytes);
+nb_status nb_conv_bn_silu_step_host(nb_cbs_plan plan, const void* host_x, const void* host_w, const float* host_gamma,
+                                    const float* host_beta, const void* host_g, void* host_a, void* host_dx,
+                                    float* host_dw, float* host_dgamma, float* host_dbeta, void* device_scratch,
+                                    size_t scratch_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NB_CBS_H */

@@ -1,0 +1,197 @@
+"""ctypes binding of libnb_cbs.so: the same names as include/nb_cbs.h, argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels.  PyTorch appears only as the owner of
+device memory (``tensor.data_ptr()``) and streams.  There is no fallback: if the shared library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_size_t, c_uint32, c_void_p
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libnb_cbs.so")
+
+NB_OK = 0
+NB_ERR_INVALID_ARG, NB_ERR_UNSUPPORTED, NB_ERR_WORKSPACE, NB_ERR_ALIGNMENT = 1, 2, 3, 4
+NB_ERR_CUDA, NB_ERR_ARCH, NB_ERR_TIMEOUT, NB_ERR_INTERNAL = 5, 6, 7, 8
+NB_DTYPE_F32, NB_DTYPE_BF16, NB_DTYPE_F16 = 0, 1, 2
+NB_MODE_BF16_TC, NB_MODE_F32_REF = 0, 1
+NB_CBS_FLAG_FORCE_SIMT = 1
+
+EXPORTS = (
+    "nb_abi_version", "nb_last_error", "nb_cbs_plan_create", "nb_cbs_plan_destroy", "nb_cbs_out_shape",
+    "nb_cbs_workspace_bytes", "nb_cbs_plan_paths", "nb_cbs_poll_status", "nb_conv_bn_silu_fwd", "nb_bn_stats",
+    "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
+    "nb_conv_bn_silu_step_host",
+)
+
+
+class nb_cbs_desc(Structure):
+    _fields_ = [
+        ("struct_size", c_uint32), ("n", c_int32), ("h", c_int32), ("w", c_int32), ("c_in", c_int32), ("c_out", c_int32),
+        ("ksize", c_int32), ("stride", c_int32), ("eps", c_float), ("momentum", c_float), ("mode", c_int32), ("flags", c_uint32),
+    ]
+
+
+class NbError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"nb_cbs status {status}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the library (raises if it has not been built: there is no other implementation to fall back to)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2609_10632_b200.build` (nvcc, sm_100a)")
+        lib = ctypes.CDLL(LIB_PATH)
+        V = c_void_p
+        FP = c_void_p  # float* passed as raw addresses
+        lib.nb_abi_version.restype = c_uint32
+        lib.nb_abi_version.argtypes = []
+        lib.nb_last_error.restype = c_char_p
+        lib.nb_last_error.argtypes = []
+        lib.nb_cbs_plan_create.argtypes = [POINTER(nb_cbs_desc), c_int, POINTER(V)]
+        lib.nb_cbs_plan_destroy.argtypes = [V]
+        lib.nb_cbs_out_shape.argtypes = [V, POINTER(c_int32), POINTER(c_int32)]
+        lib.nb_cbs_workspace_bytes.argtypes = [V, POINTER(c_size_t), POINTER(c_size_t)]
+        lib.nb_cbs_plan_paths.argtypes = [V, POINTER(c_int32)]
+        lib.nb_cbs_poll_status.argtypes = [V, V]
+        lib.nb_conv_bn_silu_fwd.argtypes = [V, V, V, FP, FP, FP, FP, V, FP, FP, V, V, c_size_t, V]
+        lib.nb_bn_stats.argtypes = [V, V, c_int32, FP, FP, FP, FP, V, c_size_t, V]
+        lib.nb_conv_bn_silu_bwd_data.argtypes = [V, V, V, FP, FP, FP, FP, V, V, FP, FP, V, V, c_size_t, V]
+        lib.nb_conv_bn_silu_bwd_weight.argtypes = [V, V, V, FP, V, c_size_t, V]
+        lib.nb_cbs_step_host_scratch_bytes.argtypes = [V, POINTER(c_size_t)]
+        lib.nb_conv_bn_silu_step_host.argtypes = [V, V, V, FP, FP, V, V, V, FP, FP, FP, V, c_size_t, V]
+        for name in EXPORTS:
+            if name not in ("nb_abi_version", "nb_last_error"):
+                getattr(lib, name).restype = c_int32
+        _lib = lib
+    return _lib
+
+
+def nb_last_error() -> str:
+    return load().nb_last_error().decode()
+
+
+def _check(status: int):
+    if status != NB_OK:
+        raise NbError(status, nb_last_error())
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    if hasattr(t, "ctypes"):
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+def _nbytes(t) -> int:
+    if t is None:
+        return 0
+    if hasattr(t, "element_size"):
+        return t.numel() * t.element_size()
+    return t.nbytes
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def nb_abi_version() -> int:
+    return int(load().nb_abi_version())
+
+
+class Plan:
+    """Owner of one nb_cbs_plan handle."""
+
+    def __init__(self, n, h, w, c_in, c_out, ksize, stride, eps=1e-3, momentum=0.03, mode=NB_MODE_BF16_TC, flags=0, device=0):
+        self.desc = nb_cbs_desc(ctypes.sizeof(nb_cbs_desc), n, h, w, c_in, c_out, ksize, stride, eps, momentum, mode, flags)
+        self.handle = c_void_p()
+        self.device = device
+        _check(load().nb_cbs_plan_create(byref(self.desc), device, byref(self.handle)))
+        ho, wo = c_int32(), c_int32()
+        _check(load().nb_cbs_out_shape(self.handle, byref(ho), byref(wo)))
+        self.ho, self.wo = ho.value, wo.value
+        f, b = c_size_t(), c_size_t()
+        _check(load().nb_cbs_workspace_bytes(self.handle, byref(f), byref(b)))
+        self.fwd_bytes, self.bwd_bytes = f.value, b.value
+        p3 = (c_int32 * 3)()
+        _check(load().nb_cbs_plan_paths(self.handle, p3))
+        self.paths = {"fprop": p3[0], "dgrad": p3[1], "wgrad": p3[2]}
+
+    @classmethod
+    def for_shape(cls, s, **kw):
+        return cls(s.n, s.h, s.w, s.c_in, s.c_out, s.k, s.stride, **kw)
+
+    @property
+    def m(self):
+        return self.desc.n * self.ho * self.wo
+
+    def step_host_scratch_bytes(self) -> int:
+        b = c_size_t()
+        _check(load().nb_cbs_step_host_scratch_bytes(self.handle, byref(b)))
+        return b.value
+
+    def close(self):
+        if self.handle:
+            load().nb_cbs_plan_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def nb_cbs_poll_status(plan: Plan, stream=None):
+    _check(load().nb_cbs_poll_status(plan.handle, _stream(stream)))
+    return nb_last_error()
+
+
+def nb_conv_bn_silu_fwd(plan: Plan, x, w, gamma, beta, running_mean, running_var, y_saved, save_mean, save_invstd, a_out,
+                        workspace, stream=None):
+    _check(load().nb_conv_bn_silu_fwd(plan.handle, _ptr(x), _ptr(w), _ptr(gamma), _ptr(beta), _ptr(running_mean), _ptr(running_var),
+                                      _ptr(y_saved), _ptr(save_mean), _ptr(save_invstd), _ptr(a_out), _ptr(workspace),
+                                      _nbytes(workspace), _stream(stream)))
+
+
+def nb_bn_stats(plan: Plan, y, y_dtype, mean, invstd, sum_, sumsq, workspace, stream=None):
+    _check(load().nb_bn_stats(plan.handle, _ptr(y), y_dtype, _ptr(mean), _ptr(invstd), _ptr(sum_), _ptr(sumsq), _ptr(workspace),
+                              _nbytes(workspace), _stream(stream)))
+
+
+def nb_conv_bn_silu_bwd_data(plan: Plan, g, y_saved, save_mean, save_invstd, gamma, beta, w, dx, dgamma, dbeta, dy_out,
+                             workspace, stream=None):
+    _check(load().nb_conv_bn_silu_bwd_data(plan.handle, _ptr(g), _ptr(y_saved), _ptr(save_mean), _ptr(save_invstd), _ptr(gamma),
+                                           _ptr(beta), _ptr(w), _ptr(dx), _ptr(dgamma), _ptr(dbeta), _ptr(dy_out), _ptr(workspace),
+                                           _nbytes(workspace), _stream(stream)))
+
+
+def nb_conv_bn_silu_bwd_weight(plan: Plan, x, dy, dw, workspace, stream=None):
+    _check(load().nb_conv_bn_silu_bwd_weight(plan.handle, _ptr(x), _ptr(dy), _ptr(dw), _ptr(workspace), _nbytes(workspace),
+                                             _stream(stream)))
+
+
+def nb_conv_bn_silu_step_host(plan: Plan, host_x, host_w, host_gamma, host_beta, host_g, host_a, host_dx, host_dw, host_dgamma,
+                              host_dbeta, device_scratch, stream=None):
+    _check(load().nb_conv_bn_silu_step_host(plan.handle, _ptr(host_x), _ptr(host_w), _ptr(host_gamma), _ptr(host_beta), _ptr(host_g),
+                                            _ptr(host_a), _ptr(host_dx), _ptr(host_dw), _ptr(host_dgamma), _ptr(host_dbeta),
+                                            _ptr(device_scratch), _nbytes(device_scratch), _stream(stream)))

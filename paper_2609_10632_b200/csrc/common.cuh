@@ -1,0 +1,56 @@
+// Shared device/host helpers of the nb_cbs library: shape record, status block, small conversions.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nbcbs {
+
+// Geometry of one Conv(k, stride, pad k/2) block; plain ints so it can be passed by value to kernels.
+struct Geom {
+    int n, h, w, c_in, c_out, k, stride, pad, ho, wo;
+    long long m;  // n*ho*wo
+    int kdim;     // k*k*c_in
+};
+
+// Device status block owned by a plan (ints): [0] error code, [1] where, [2] detail, [3] fp16 saturation count.
+enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_WORDS = 16 };
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <> __device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+// fp16 stores saturate instead of producing inf (the saved conv output must stay finite for BN).
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) {
+    return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
+}
+
+// 16-byte vector of VT elements (8 x 16-bit or 4 x fp32).
+template <typename T> struct Vec16 {
+    static constexpr int N = 16 / sizeof(T);
+    T v[N];
+};
+template <typename T> __device__ __forceinline__ Vec16<T> ld16(const T* p) {
+    Vec16<T> r;
+    *reinterpret_cast<uint4*>(&r) = *reinterpret_cast<const uint4*>(p);
+    return r;
+}
+template <typename T> __device__ __forceinline__ void st16(T* p, const Vec16<T>& r) {
+    *reinterpret_cast<uint4*>(p) = *reinterpret_cast<const uint4*>(&r);
+}
+// Streaming variants: data touched once should not displace reusable lines in L1.
+template <typename T> __device__ __forceinline__ Vec16<T> ld16_stream(const T* p) {
+    Vec16<T> r;
+    *reinterpret_cast<uint4*>(&r) = __ldcs(reinterpret_cast<const uint4*>(p));
+    return r;
+}
+template <typename T> __device__ __forceinline__ void st16_stream(T* p, const Vec16<T>& r) {
+    __stcs(reinterpret_cast<uint4*>(p), *reinterpret_cast<const uint4*>(&r));
+}
+
+}  // namespace nbcbs

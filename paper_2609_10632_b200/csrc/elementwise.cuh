@@ -1,0 +1,246 @@
+// HBM-bound passes over [M][C] NHWC tensors: batch statistics, normalise+affine+SiLU, and their backward.
+// All of them walk the tensor as a flat array of 16-byte vectors with a stride that is a multiple of the
+// number of vectors per row, so a thread always sees the same channel group: per-channel parameters and
+// accumulators live in registers, loads are fully coalesced, and reductions have a fixed order
+// (bitwise reproducible run to run: no floating-point atomics anywhere).
+#pragma once
+#include "common.cuh"
+
+namespace nbcbs {
+
+template <bool FAST> __device__ __forceinline__ float sigmoid_f(float z) {
+    if (FAST) {
+        const float e = __expf(fminf(-z, 80.f));  // keeps 1+e far below 2^126, where __fdividef loses accuracy
+        return __fdividef(1.f, 1.f + e);
+    } else {
+        return 1.f / (1.f + expf(-z));
+    }
+}
+
+// ------------------------------------------------------------------ per-channel sum and sum of squares
+// partials layout: [gridDim.x][2][C]; blockDim.x = (C/V) * R.
+template <typename YT>
+__global__ void __launch_bounds__(1024) bn_stats_partial_kernel(const YT* __restrict__ y, long long total_vecs, int C,
+                                                                float* __restrict__ partials) {
+    constexpr int V = Vec16<YT>::N;
+    extern __shared__ float red[];  // [blockDim.x][V]
+    const int tid = threadIdx.x;
+    const int cgs = C / V;
+    float s[V], ss[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) s[i] = ss[i] = 0.f;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long v = (long long)blockIdx.x * blockDim.x + tid; v < total_vecs; v += stride) {
+        const Vec16<YT> q = ld16(y + v * V);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const float f = to_f32(q.v[i]);
+            s[i] += f;
+            ss[i] = fmaf(f, f, ss[i]);
+        }
+    }
+    const int R = blockDim.x / cgs;
+    for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) red[tid * V + i] = pass ? ss[i] : s[i];
+        __syncthreads();
+        for (int c = tid; c < C; c += blockDim.x) {
+            const int g = c / V, e = c % V;
+            float acc = 0.f;
+            for (int r = 0; r < R; ++r) acc += red[(r * cgs + g) * V + e];
+            partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;
+        }
+        __syncthreads();
+    }
+}
+
+// Combine partials [nparts][2][C] in fp64 (fixed order) and derive the per-channel quantities.
+// block (32,32): x = channel within a group of 32, y = slice of the partial list.
+// Outputs (any may be NULL): mean, invstd, scale = gamma*invstd, shift = beta - mean*scale, raw sums,
+// running statistics (in place; unbiased variance, momentum).
+__global__ void bn_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float eps,
+                                   float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
+                                   float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
+                                   float* sum_out, float* sumsq_out) {
+    __shared__ double sh_s[32][33], sh_q[32][33];
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double s = 0.0, q = 0.0;
+    if (c < C) {
+        for (int b = threadIdx.y; b < nparts; b += 32) {
+            s += (double)partials[((size_t)b * 2) * C + c];
+            q += (double)partials[((size_t)b * 2 + 1) * C + c];
+        }
+    }
+    sh_s[threadIdx.y][threadIdx.x] = s;
+    sh_q[threadIdx.y][threadIdx.x] = q;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        s = 0.0;
+        q = 0.0;
+        for (int j = 0; j < 32; ++j) {
+            s += sh_s[j][threadIdx.x];
+            q += sh_q[j][threadIdx.x];
+        }
+        const double mu = s / M;
+        double var = q / M - mu * mu;
+        if (var < 0.0) var = 0.0;
+        const double is = 1.0 / sqrt(var + (double)eps);
+        if (mean) mean[c] = (float)mu;
+        if (invstd) invstd[c] = (float)is;
+        if (scale) {
+            const double sc = (double)gamma[c] * is;
+            scale[c] = (float)sc;
+            shift[c] = (float)((double)beta[c] - mu * sc);
+        }
+        if (sum_out) sum_out[c] = (float)s;
+        if (sumsq_out) sumsq_out[c] = (float)q;
+        if (rmean) {
+            rmean[c] = (float)((1.0 - (double)momentum) * (double)rmean[c] + (double)momentum * mu);
+            rvar[c] = (float)((1.0 - (double)momentum) * (double)rvar[c] + (double)momentum * var * M / (M - 1.0));
+        }
+    }
+}
+
+// ------------------------------------------------------------------ a = SiLU(y*scale + shift)
+template <typename YT, typename AT, bool FAST>
+__global__ void __launch_bounds__(1024) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
+                                                             long long total_vecs, int C, const float* __restrict__ scale,
+                                                             const float* __restrict__ shift) {
+    constexpr int V = Vec16<YT>::N;
+    static_assert(V == Vec16<AT>::N, "y and a must have the same element size");
+    const int cg = threadIdx.x % (C / V);
+    float sc[V], sh[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        sc[i] = scale[cg * V + i];
+        sh[i] = shift[cg * V + i];
+    }
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+        const Vec16<YT> q = ld16(y + v * V);
+        Vec16<AT> o;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const float z = fmaf(to_f32(q.v[i]), sc[i], sh[i]);
+            o.v[i] = from_f32<AT>(z * sigmoid_f<FAST>(z));
+        }
+        st16(a + v * V, o);
+    }
+}
+
+// ------------------------------------------------------------------ backward reductions: sum dz, sum dz*xhat
+template <typename YT, typename AT, bool FAST>
+__global__ void __launch_bounds__(1024) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
+                                                                  long long total_vecs, int C, const float* __restrict__ mean,
+                                                                  const float* __restrict__ invstd, const float* __restrict__ gamma,
+                                                                  const float* __restrict__ beta, float* __restrict__ partials) {
+    constexpr int V = Vec16<YT>::N;
+    static_assert(V == Vec16<AT>::N, "g and y must have the same element size");
+    extern __shared__ float red[];
+    const int tid = threadIdx.x;
+    const int cgs = C / V;
+    const int cg = tid % cgs;
+    float mu[V], is[V], ga[V], be[V], sb[V], sg[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        mu[i] = mean[cg * V + i];
+        is[i] = invstd[cg * V + i];
+        ga[i] = gamma[cg * V + i];
+        be[i] = beta[cg * V + i];
+        sb[i] = sg[i] = 0.f;
+    }
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long v = (long long)blockIdx.x * blockDim.x + tid; v < total_vecs; v += stride) {
+        const Vec16<YT> qy = ld16(y + v * V);
+        const Vec16<AT> qg = ld16(g + v * V);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const float xhat = (to_f32(qy.v[i]) - mu[i]) * is[i];
+            const float z = fmaf(ga[i], xhat, be[i]);
+            const float s = sigmoid_f<FAST>(z);
+            const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
+            sb[i] += dz;
+            sg[i] = fmaf(dz, xhat, sg[i]);
+        }
+    }
+    const int R = blockDim.x / cgs;
+    for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) red[tid * V + i] = pass ? sg[i] : sb[i];
+        __syncthreads();
+        for (int c = tid; c < C; c += blockDim.x) {
+            const int gq = c / V, e = c % V;
+            float acc = 0.f;
+            for (int r = 0; r < R; ++r) acc += red[(r * cgs + gq) * V + e];
+            partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;  // pass 0: dbeta, pass 1: dgamma
+        }
+        __syncthreads();
+    }
+}
+
+// partials [nparts][2][C] -> dbeta, dgamma (fp32) and the two per-channel coefficients dbeta/M, dgamma/M.
+__global__ void bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float* dgamma,
+                                       float* dbeta, float* coef /*[2][C]*/) {
+    __shared__ double sh_s[32][33], sh_q[32][33];
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double s = 0.0, q = 0.0;
+    if (c < C) {
+        for (int b = threadIdx.y; b < nparts; b += 32) {
+            s += (double)partials[((size_t)b * 2) * C + c];
+            q += (double)partials[((size_t)b * 2 + 1) * C + c];
+        }
+    }
+    sh_s[threadIdx.y][threadIdx.x] = s;
+    sh_q[threadIdx.y][threadIdx.x] = q;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        s = 0.0;
+        q = 0.0;
+        for (int j = 0; j < 32; ++j) {
+            s += sh_s[j][threadIdx.x];
+            q += sh_q[j][threadIdx.x];
+        }
+        dbeta[c] = (float)s;
+        dgamma[c] = (float)q;
+        coef[c] = (float)(s / M);
+        coef[C + c] = (float)(q / M);
+    }
+}
+
+// ------------------------------------------------------------------ dy = gamma*invstd*(dz - dbeta/M - xhat*dgamma/M)
+template <typename YT, typename AT, bool FAST>
+__global__ void __launch_bounds__(1024) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
+                                                              AT* __restrict__ dy, long long total_vecs, int C,
+                                                              const float* __restrict__ mean, const float* __restrict__ invstd,
+                                                              const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                              const float* __restrict__ coef) {
+    constexpr int V = Vec16<YT>::N;
+    const int cg = threadIdx.x % (C / V);
+    float mu[V], is[V], ga[V], be[V], c1[V], c2[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        mu[i] = mean[cg * V + i];
+        is[i] = invstd[cg * V + i];
+        ga[i] = gamma[cg * V + i];
+        be[i] = beta[cg * V + i];
+        c1[i] = coef[cg * V + i];
+        c2[i] = coef[C + cg * V + i];
+    }
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+        const Vec16<YT> qy = ld16(y + v * V);
+        const Vec16<AT> qg = ld16(g + v * V);
+        Vec16<AT> o;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const float xhat = (to_f32(qy.v[i]) - mu[i]) * is[i];
+            const float z = fmaf(ga[i], xhat, be[i]);
+            const float s = sigmoid_f<FAST>(z);
+            const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
+            o.v[i] = from_f32<AT>(ga[i] * is[i] * (dz - c1[i] - xhat * c2[i]));
+        }
+        st16(dy + v * V, o);
+    }
+}
+
+}  // namespace nbcbs

@@ -1,0 +1,501 @@
+// C ABI of the Conv -> BN(train) -> SiLU block library (see include/nb_cbs.h): plans, validation, workspace
+// carving and kernel dispatch.  No device memory is allocated here except the plan's status block.
+#include "../../include/nb_cbs.h"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "simt_conv.cuh"
+#include "tc_conv.cuh"
+
+using namespace nbcbs;
+
+namespace {
+
+thread_local std::string g_err;
+
+nb_status fail(nb_status code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+#define NB_CUDA_CHECK(expr)                                                                         \
+    do {                                                                                            \
+        cudaError_t e__ = (expr);                                                                   \
+        if (e__ != cudaSuccess) return fail(NB_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct EwCfg {  // launch geometry of the [M][C] passes
+    int vec, cgs, tpb;
+    long long total_vecs;
+    int blocks_reduce, blocks_map;
+};
+
+}  // namespace
+
+struct nb_cbs_plan_s {
+    nb_cbs_desc desc;
+    Geom g;
+    int device;
+    int sm_count;
+    int* status;  // device, ST_WORDS ints
+    EwCfg ew;
+    int nparts;      // rows of the partial-sum buffers
+    int wg_splits;   // split-K slices of the CUDA-core wgrad
+    long long wg_chunk;
+    TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
+    size_t fwd_bytes, bwd_bytes;
+    // workspace offsets
+    size_t off_scale, off_shift, off_fpart;                  // forward
+    size_t off_coef, off_bpart, off_wt, off_wgpart;          // backward
+};
+
+namespace {
+
+bool is_f32(const nb_cbs_plan_s* p) { return p->desc.mode == NB_MODE_F32_REF; }
+
+nb_status check_ptr(const void* p, const char* name, bool nullable = false) {
+    if (!p) return nullable ? NB_OK : fail(NB_ERR_INVALID_ARG, "%s is NULL", name);
+    if (reinterpret_cast<uintptr_t>(p) & 15u) return fail(NB_ERR_ALIGNMENT, "%s is not 16-byte aligned", name);
+    return NB_OK;
+}
+#define NB_CHECK_PTR(p, ...)                                   \
+    do {                                                       \
+        nb_status s__ = check_ptr((p), #p, ##__VA_ARGS__);     \
+        if (s__ != NB_OK) return s__;                          \
+    } while (0)
+
+nb_status check_ws(const void* ws, size_t have, size_t need) {
+    if (need == 0) return NB_OK;
+    if (!ws) return fail(NB_ERR_WORKSPACE, "workspace is NULL (%zu bytes needed)", need);
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(NB_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+    if (have < need) return fail(NB_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", have, need);
+    return NB_OK;
+}
+
+nb_status launch_ok(const char* what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(NB_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+    return NB_OK;
+}
+#define NB_LAUNCH_OK(what)                    \
+    do {                                      \
+        nb_status s__ = launch_ok(what);      \
+        if (s__ != NB_OK) return s__;         \
+    } while (0)
+#define NB_TRY(expr)                          \
+    do {                                      \
+        nb_status s__ = (expr);               \
+        if (s__ != NB_OK) return s__;         \
+    } while (0)
+
+// ---------------------------------------------------------------- elementwise launch helpers
+template <typename YT> nb_status run_stats_partial(nb_cbs_plan_s* p, const void* y, float* partials, cudaStream_t st) {
+    const EwCfg& e = p->ew;
+    bn_stats_partial_kernel<YT><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+        static_cast<const YT*>(y), e.total_vecs, p->g.c_out, partials);
+    return launch_ok("bn_stats_partial");
+}
+
+nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, const float* gamma, const float* beta, float* mean,
+                       float* invstd, float* scale, float* shift, float* rmean, float* rvar, float* sum, float* sumsq,
+                       cudaStream_t st) {
+    const int C = p->g.c_out;
+    bn_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
+                                                              gamma, beta, mean, invstd, scale, shift, rmean, rvar, sum, sumsq);
+    return launch_ok("bn_finalize");
+}
+
+template <typename YT, typename AT, bool FAST>
+nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
+    const EwCfg& e = p->ew;
+    bn_silu_apply_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
+                                                                       p->g.c_out, scale, shift);
+    return launch_ok("bn_silu_apply");
+}
+
+template <typename YT, typename AT, bool FAST>
+nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, const float* mean, const float* invstd,
+                              const float* gamma, const float* beta, float* dgamma, float* dbeta, void* dy, float* partials,
+                              float* coef, cudaStream_t st) {
+    const EwCfg& e = p->ew;
+    const int C = p->g.c_out;
+    bn_silu_bwd_reduce_kernel<YT, AT, FAST><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+        static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials);
+    NB_LAUNCH_OK("bn_silu_bwd_reduce");
+    bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
+    NB_LAUNCH_OK("bn_bwd_finalize");
+    bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
+                                                                        static_cast<AT*>(dy), e.total_vecs, C, mean, invstd, gamma,
+                                                                        beta, coef);
+    return launch_ok("bn_silu_bwd_dy");
+}
+
+// ---------------------------------------------------------------- CUDA-core convolutions
+template <typename TIN, typename TOUT>
+nb_status run_simt_fprop(nb_cbs_plan_s* p, const void* x, const void* w, void* y, cudaStream_t st) {
+    FpropProblem<TIN, TIN> prob{static_cast<const TIN*>(x), static_cast<const TIN*>(w), p->g};
+    dim3 grid((unsigned)((p->g.m + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_out + SIMT_BN - 1) / SIMT_BN), 1);
+    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TOUT*>(y), (long long)p->g.kdim);
+    return launch_ok("simt fprop");
+}
+
+template <typename TIN>
+nb_status run_simt_dgrad(nb_cbs_plan_s* p, const void* dy, const void* w, void* dx, cudaStream_t st) {
+    DgradProblem<TIN, TIN> prob{static_cast<const TIN*>(dy), static_cast<const TIN*>(w), p->g};
+    const long long I = (long long)p->g.n * p->g.h * p->g.w;
+    dim3 grid((unsigned)((I + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_in + SIMT_BN - 1) / SIMT_BN), 1);
+    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TIN*>(dx), (long long)p->g.k * p->g.k * p->g.c_out);
+    return launch_ok("simt dgrad");
+}
+
+template <typename TIN>
+nb_status run_simt_wgrad(nb_cbs_plan_s* p, const void* x, const void* dy, float* dw, float* partial, cudaStream_t st) {
+    WgradProblem<TIN, TIN> prob{static_cast<const TIN*>(dy), static_cast<const TIN*>(x), p->g};
+    dim3 grid((unsigned)((p->g.c_out + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.kdim + SIMT_BN - 1) / SIMT_BN), (unsigned)p->wg_splits);
+    if (p->wg_splits == 1) {
+        simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, dw, p->g.m);
+        return launch_ok("simt wgrad");
+    }
+    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, partial, p->wg_chunk);
+    NB_LAUNCH_OK("simt wgrad (split-K)");
+    const size_t elems = (size_t)p->g.c_out * p->g.kdim;
+    splitk_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, p->wg_splits, elems, dw);
+    return launch_ok("splitk_reduce");
+}
+
+}  // namespace
+
+// ====================================================================================== exported functions
+extern "C" {
+
+uint32_t nb_abi_version(void) { return NB_CBS_ABI_VERSION; }
+
+const char* nb_last_error(void) { return g_err.c_str(); }
+
+nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out) {
+    g_err.clear();
+    if (!out) return fail(NB_ERR_INVALID_ARG, "out_plan is NULL");
+    *out = nullptr;
+    if (!d) return fail(NB_ERR_INVALID_ARG, "desc is NULL");
+    if (d->struct_size != sizeof(nb_cbs_desc))
+        return fail(NB_ERR_INVALID_ARG, "desc.struct_size is %u, this library expects %zu", d->struct_size, sizeof(nb_cbs_desc));
+    if (d->n <= 0 || d->h <= 0 || d->w <= 0 || d->c_in <= 0 || d->c_out <= 0)
+        return fail(NB_ERR_INVALID_ARG, "extents must be positive (n=%d h=%d w=%d c_in=%d c_out=%d)", d->n, d->h, d->w, d->c_in, d->c_out);
+    if (d->ksize != 1 && d->ksize != 3) return fail(NB_ERR_INVALID_ARG, "ksize must be 1 or 3, got %d", d->ksize);
+    if (d->stride != 1 && d->stride != 2) return fail(NB_ERR_INVALID_ARG, "stride must be 1 or 2, got %d", d->stride);
+    if (d->mode != NB_MODE_BF16_TC && d->mode != NB_MODE_F32_REF) return fail(NB_ERR_INVALID_ARG, "unknown mode %d", d->mode);
+    if (!(d->eps > 0.f)) return fail(NB_ERR_INVALID_ARG, "eps must be positive");
+    if (!(d->momentum >= 0.f && d->momentum <= 1.f)) return fail(NB_ERR_INVALID_ARG, "momentum must be in [0,1]");
+    const int vec = d->mode == NB_MODE_F32_REF ? 4 : 8;
+    if (d->c_out % vec) return fail(NB_ERR_UNSUPPORTED, "c_out=%d must be a multiple of %d in this mode", d->c_out, vec);
+    if (d->c_out / vec > 1024) return fail(NB_ERR_UNSUPPORTED, "c_out=%d is too large", d->c_out);
+
+    Geom g;
+    g.n = d->n; g.h = d->h; g.w = d->w; g.c_in = d->c_in; g.c_out = d->c_out; g.k = d->ksize; g.stride = d->stride;
+    g.pad = d->ksize / 2;
+    g.ho = (g.h + 2 * g.pad - g.k) / g.stride + 1;
+    g.wo = (g.w + 2 * g.pad - g.k) / g.stride + 1;
+    g.m = (long long)g.n * g.ho * g.wo;
+    g.kdim = g.k * g.k * g.c_in;
+    if (g.m < 2) return fail(NB_ERR_INVALID_ARG, "batch statistics need at least 2 rows (N*Ho*Wo=%lld)", g.m);
+    if ((double)g.m * g.c_out >= 9.0e18 || (long long)g.n * g.h * g.w * g.c_in < 0)
+        return fail(NB_ERR_UNSUPPORTED, "tensor too large");
+
+    int count = 0;
+    NB_CUDA_CHECK(cudaGetDeviceCount(&count));
+    if (device < 0 || device >= count) return fail(NB_ERR_INVALID_ARG, "device %d out of range (%d devices)", device, count);
+    cudaDeviceProp prop;
+    NB_CUDA_CHECK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return fail(NB_ERR_ARCH, "device %d is sm_%d%d; this library is built for sm_100a only", device, prop.major, prop.minor);
+
+    nb_cbs_plan_s* p = new (std::nothrow) nb_cbs_plan_s();
+    if (!p) return fail(NB_ERR_INTERNAL, "out of host memory");
+    p->desc = *d;
+    p->g = g;
+    p->device = device;
+    p->sm_count = prop.multiProcessorCount;
+
+    EwCfg& e = p->ew;
+    e.vec = vec;
+    e.cgs = g.c_out / vec;
+    const int R = e.cgs >= 256 ? 1 : 256 / e.cgs;
+    e.tpb = e.cgs * R;
+    e.total_vecs = g.m * e.cgs;
+    const long long max_blocks = (e.total_vecs + e.tpb - 1) / e.tpb;
+    e.blocks_reduce = (int)std::min<long long>(max_blocks, (long long)p->sm_count * 4);
+    e.blocks_map = (int)std::min<long long>(max_blocks, (long long)p->sm_count * 8);
+
+    // CUDA-core wgrad split-K: enough slices to fill the machine, at least 512 rows each.
+    {
+        const long long tiles = (long long)((g.c_out + SIMT_BM - 1) / SIMT_BM) * ((g.kdim + SIMT_BN - 1) / SIMT_BN);
+        long long splits = (4LL * p->sm_count + tiles - 1) / tiles;
+        const long long max_splits = std::max<long long>(1, g.m / 512);
+        splits = std::max<long long>(1, std::min(splits, max_splits));
+        long long chunk = (g.m + splits - 1) / splits;
+        chunk = (chunk + SIMT_BK - 1) / SIMT_BK * SIMT_BK;
+        splits = (g.m + chunk - 1) / chunk;
+        p->wg_splits = (int)splits;
+        p->wg_chunk = chunk;
+    }
+
+    int cur = 0;
+    NB_CUDA_CHECK(cudaGetDevice(&cur));
+    cudaError_t ce = cudaSetDevice(device);
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->status, ST_WORDS * sizeof(int));
+    if (ce == cudaSuccess) ce = cudaMemset(p->status, 0, ST_WORDS * sizeof(int));
+    nb_status tcs = NB_OK;
+    if (ce == cudaSuccess) tcs = tc_plan_init(&p->tc, g, d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT), p->sm_count, prop);
+    cudaSetDevice(cur);
+    if (ce != cudaSuccess || tcs != NB_OK) {
+        if (p->status) cudaFree(p->status);
+        delete p;
+        if (tcs != NB_OK) return fail(tcs, "tensor-core plan setup failed: %s", tc_last_error());
+        return fail(NB_ERR_CUDA, "status block allocation failed: %s", cudaGetErrorString(ce));
+    }
+
+    p->nparts = std::max(e.blocks_reduce, p->tc.fprop_parts);
+    const size_t C = (size_t)g.c_out;
+    size_t off = 0;
+    p->off_scale = off; off = align_up(off + C * 4, 256);
+    p->off_shift = off; off = align_up(off + C * 4, 256);
+    p->off_fpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
+    p->fwd_bytes = off;
+    off = 0;
+    p->off_coef = off; off = align_up(off + 2 * C * 4, 256);
+    p->off_bpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
+    p->off_wt = off; off = align_up(off + p->tc.wt_bytes, 256);
+    p->off_wgpart = off;
+    {
+        size_t simt = p->wg_splits > 1 ? (size_t)p->wg_splits * C * g.kdim * 4 : 0;
+        off = align_up(off + std::max(simt, p->tc.wgrad_partial_bytes), 256);
+    }
+    p->bwd_bytes = off;
+    *out = p;
+    return NB_OK;
+}
+
+nb_status nb_cbs_plan_destroy(nb_cbs_plan p) {
+    g_err.clear();
+    if (!p) return NB_OK;
+    if (p->status) {
+        int cur = 0;
+        cudaGetDevice(&cur);
+        cudaSetDevice(p->device);
+        cudaFree(p->status);
+        cudaSetDevice(cur);
+    }
+    delete p;
+    return NB_OK;
+}
+
+nb_status nb_cbs_out_shape(nb_cbs_plan p, int32_t* ho, int32_t* wo) {
+    g_err.clear();
+    if (!p || !ho || !wo) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    *ho = p->g.ho;
+    *wo = p->g.wo;
+    return NB_OK;
+}
+
+nb_status nb_cbs_workspace_bytes(nb_cbs_plan p, size_t* fwd, size_t* bwd) {
+    g_err.clear();
+    if (!p || !fwd || !bwd) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    *fwd = p->fwd_bytes;
+    *bwd = p->bwd_bytes;
+    return NB_OK;
+}
+
+nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
+    g_err.clear();
+    if (!p || !paths3) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    paths3[0] = p->tc.fprop ? 1 : 0;
+    paths3[1] = p->tc.dgrad ? 1 : 0;
+    paths3[2] = p->tc.wgrad ? 1 : 0;
+    return NB_OK;
+}
+
+nb_status nb_cbs_poll_status(nb_cbs_plan p, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int host[ST_WORDS];
+    NB_CUDA_CHECK(cudaStreamSynchronize(st));
+    NB_CUDA_CHECK(cudaMemcpy(host, p->status, sizeof host, cudaMemcpyDeviceToHost));
+    NB_CUDA_CHECK(cudaMemset(p->status, 0, sizeof host));
+    if (host[ST_ERR] != 0)
+        return fail((nb_status)host[ST_ERR], "device status: error %d at site %d (detail %d)", host[ST_ERR], host[ST_WHERE], host[ST_DETAIL]);
+    if (host[ST_SAT] != 0) {
+        char buf[96];
+        snprintf(buf, sizeof buf, "%d fp16 stores of the saved convolution output saturated", host[ST_SAT]);
+        g_err = buf;
+    }
+    return NB_OK;
+}
+
+nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const float* gamma, const float* beta,
+                              float* running_mean, float* running_var, void* y_saved, float* save_mean, float* save_invstd,
+                              void* a_out, void* workspace, size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta);
+    NB_CHECK_PTR(y_saved); NB_CHECK_PTR(save_mean); NB_CHECK_PTR(save_invstd); NB_CHECK_PTR(a_out);
+    if ((running_mean == nullptr) != (running_var == nullptr))
+        return fail(NB_ERR_INVALID_ARG, "running_mean and running_var must both be given or both be NULL");
+    NB_TRY(check_ws(workspace, workspace_bytes, p->fwd_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    float* scale = reinterpret_cast<float*>(ws + p->off_scale);
+    float* shift = reinterpret_cast<float*>(ws + p->off_shift);
+    float* part = reinterpret_cast<float*>(ws + p->off_fpart);
+    int nparts = p->ew.blocks_reduce;
+    if (is_f32(p)) {
+        NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
+        NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
+    } else if (p->tc.fprop) {
+        NB_TRY(tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st));  // writes y (fp16) and the partial sums
+        nparts = p->tc.fprop_parts;
+    } else {
+        NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y_saved, st)));
+        NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
+    }
+    NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
+    if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
+    return run_apply<__half, __nv_bfloat16, true>(p, y_saved, a_out, scale, shift, st);
+}
+
+nb_status nb_bn_stats(nb_cbs_plan p, const void* y, int32_t y_dtype, float* mean, float* invstd, float* sum, float* sumsq,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(y); NB_CHECK_PTR(mean); NB_CHECK_PTR(invstd);
+    NB_CHECK_PTR(sum, true); NB_CHECK_PTR(sumsq, true);
+    const int want = is_f32(p) ? NB_DTYPE_F32 : NB_DTYPE_F16;
+    if (y_dtype != want) return fail(NB_ERR_UNSUPPORTED, "y_dtype %d does not match the plan's mode (expected %d)", y_dtype, want);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->fwd_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* part = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_fpart);
+    if (is_f32(p)) NB_TRY(run_stats_partial<float>(p, y, part, st));
+    else NB_TRY(run_stats_partial<__half>(p, y, part, st));
+    return run_finalize(p, part, p->ew.blocks_reduce, nullptr, nullptr, mean, invstd, nullptr, nullptr, nullptr, nullptr, sum, sumsq, st);
+}
+
+nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_saved, const float* save_mean,
+                                   const float* save_invstd, const float* gamma, const float* beta, const void* w, void* dx,
+                                   float* dgamma, float* dbeta, void* dy_out, void* workspace, size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(g); NB_CHECK_PTR(y_saved); NB_CHECK_PTR(save_mean); NB_CHECK_PTR(save_invstd);
+    NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta); NB_CHECK_PTR(dgamma); NB_CHECK_PTR(dbeta); NB_CHECK_PTR(dy_out);
+    NB_CHECK_PTR(dx, true);
+    if (dx) NB_CHECK_PTR(w);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    float* coef = reinterpret_cast<float*>(ws + p->off_coef);
+    float* part = reinterpret_cast<float*>(ws + p->off_bpart);
+    if (is_f32(p)) {
+        NB_TRY((run_bwd_elementwise<float, float, false>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st)));
+        if (dx) NB_TRY(run_simt_dgrad<float>(p, dy_out, w, dx, st));
+        return NB_OK;
+    }
+    NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st)));
+    if (!dx) return NB_OK;
+    if (p->tc.dgrad) return tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st);
+    return run_simt_dgrad<__nv_bfloat16>(p, dy_out, w, dx, st);
+}
+
+nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* dy, float* dw, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(x); NB_CHECK_PTR(dy); NB_CHECK_PTR(dw);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_wgpart);
+    if (is_f32(p)) return run_simt_wgrad<float>(p, x, dy, dw, partial, st);
+    if (p->tc.wgrad) return tc_wgrad(&p->tc, p->g, x, dy, dw, partial, p->status, st);
+    return run_simt_wgrad<__nv_bfloat16>(p, x, dy, dw, partial, st);
+}
+
+// ---------------------------------------------------------------- host-buffer step
+namespace {
+struct StepLayout {
+    size_t x, w, gamma, beta, g, y, mean, invstd, a, dy, dx, dw, dgamma, dbeta, ws_fwd, ws_bwd, total;
+    size_t nx, nw, ny_act, ny_saved, ndw;  // byte counts
+};
+StepLayout step_layout(const nb_cbs_plan_s* p) {
+    StepLayout L;
+    const size_t act = is_f32(p) ? 4 : 2, ysz = is_f32(p) ? 4 : 2;
+    const Geom& g = p->g;
+    L.nx = (size_t)g.n * g.h * g.w * g.c_in * act;
+    L.nw = (size_t)g.c_out * g.kdim * act;
+    L.ny_act = (size_t)g.m * g.c_out * act;
+    L.ny_saved = (size_t)g.m * g.c_out * ysz;
+    L.ndw = (size_t)g.c_out * g.kdim * 4;
+    const size_t cb = (size_t)g.c_out * 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.x = take(L.nx); L.w = take(L.nw); L.gamma = take(cb); L.beta = take(cb); L.g = take(L.ny_act);
+    L.y = take(L.ny_saved); L.mean = take(cb); L.invstd = take(cb); L.a = take(L.ny_act); L.dy = take(L.ny_act);
+    L.dx = take(L.nx); L.dw = take(L.ndw); L.dgamma = take(cb); L.dbeta = take(cb);
+    L.ws_fwd = take(p->fwd_bytes); L.ws_bwd = take(p->bwd_bytes);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+nb_status nb_cbs_step_host_scratch_bytes(nb_cbs_plan p, size_t* bytes) {
+    g_err.clear();
+    if (!p || !bytes) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    *bytes = step_layout(p).total;
+    return NB_OK;
+}
+
+nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const void* host_w, const float* host_gamma,
+                                    const float* host_beta, const void* host_g, void* host_a, void* host_dx, float* host_dw,
+                                    float* host_dgamma, float* host_dbeta, void* device_scratch, size_t scratch_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    if (!host_x || !host_w || !host_gamma || !host_beta || !host_g || !host_a || !host_dw || !host_dgamma || !host_dbeta)
+        return fail(NB_ERR_INVALID_ARG, "a required host pointer is NULL");
+    const StepLayout L = step_layout(p);
+    NB_TRY(check_ws(device_scratch, scratch_bytes, L.total));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* d = static_cast<char*>(device_scratch);
+    const size_t cb = (size_t)p->g.c_out * 4;
+    NB_CUDA_CHECK(cudaMemcpyAsync(d + L.x, host_x, L.nx, cudaMemcpyHostToDevice, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(d + L.w, host_w, L.nw, cudaMemcpyHostToDevice, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(d + L.gamma, host_gamma, cb, cudaMemcpyHostToDevice, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(d + L.beta, host_beta, cb, cudaMemcpyHostToDevice, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(d + L.g, host_g, L.ny_act, cudaMemcpyHostToDevice, st));
+    float* gam = reinterpret_cast<float*>(d + L.gamma);
+    float* bet = reinterpret_cast<float*>(d + L.beta);
+    float* mean = reinterpret_cast<float*>(d + L.mean);
+    float* invstd = reinterpret_cast<float*>(d + L.invstd);
+    NB_TRY(nb_conv_bn_silu_fwd(p, d + L.x, d + L.w, gam, bet, nullptr, nullptr, d + L.y, mean, invstd, d + L.a, d + L.ws_fwd, p->fwd_bytes, stream));
+    NB_TRY(nb_conv_bn_silu_bwd_data(p, d + L.g, d + L.y, mean, invstd, gam, bet, d + L.w, host_dx ? d + L.dx : nullptr,
+                                    reinterpret_cast<float*>(d + L.dgamma), reinterpret_cast<float*>(d + L.dbeta), d + L.dy,
+                                    d + L.ws_bwd, p->bwd_bytes, stream));
+    NB_TRY(nb_conv_bn_silu_bwd_weight(p, d + L.x, d + L.dy, reinterpret_cast<float*>(d + L.dw), d + L.ws_bwd, p->bwd_bytes, stream));
+    NB_CUDA_CHECK(cudaMemcpyAsync(host_a, d + L.a, L.ny_act, cudaMemcpyDeviceToHost, st));
+    if (host_dx) NB_CUDA_CHECK(cudaMemcpyAsync(host_dx, d + L.dx, L.nx, cudaMemcpyDeviceToHost, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(host_dw, d + L.dw, L.ndw, cudaMemcpyDeviceToHost, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(host_dgamma, d + L.dgamma, cb, cudaMemcpyDeviceToHost, st));
+    NB_CUDA_CHECK(cudaMemcpyAsync(host_dbeta, d + L.dbeta, cb, cudaMemcpyDeviceToHost, st));
+    return NB_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,241 @@
+"""GPU results of the C-ABI calls against the fp64 CPU oracle, element by element, on seeded inputs.
+
+bf16 mode: relative L2 <= 5e-3 and per-element |err| <= 5e-2 * rms(ref) for a, dx, dw, dgamma, dbeta;
+fp32 reference mode: relative L2 <= 1e-5.  The oracle always computes end to end from (x, w, gamma, beta, g).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_10632_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-3
+
+
+def _run_block(shape, mode, cfg_id, layer_id=0, affine="init", flags=0, need_dx=True, running=False, momentum=0.03):
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    bf16 = mode == nb.NB_MODE_BF16_TC
+    inp = wl.make_inputs(shape, cfg_id, layer_id, bf16=bf16, affine=affine)
+    blk = CbsBlock(shape, mode=mode, eps=EPS, momentum=momentum, flags=flags, need_dx=need_dx, running_stats=running)
+    blk.upload(inp)
+    blk.step()
+    blk.poll()
+    return inp, blk, blk.download()
+
+
+def _oracle(inp, need_dx=True):
+    s = inp.shape
+    return oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, EPS, need_dx=need_dx)
+
+
+def _compare(out, ref, mode, need_dx=True, report=None):
+    tag = "bf16" if mode == 0 else "f32"
+    rep = {} if report is None else report
+    np.testing.assert_allclose(out["mean"], ref.mean, rtol=0, atol=(2e-3 if tag == "bf16" else 1e-5) * (np.abs(ref.mean).max() + np.sqrt(ref.var).max()))
+    np.testing.assert_allclose(out["invstd"], ref.invstd, rtol=2e-3 if tag == "bf16" else 1e-5)
+    parity.check("a", out["a"], ref.a, tag, rep)
+    parity.check("dgamma", out["dgamma"], ref.dgamma, tag, rep)
+    parity.check("dbeta", out["dbeta"], ref.dbeta, tag, rep)
+    parity.check("dw", out["dw"], ref.dw, tag, rep)
+    if need_dx:
+        parity.check("dx", out["dx"], ref.dx, tag, rep)
+    # diagnostics (internal tensors): same bars
+    parity.check("y", out["y"], ref.y, tag, rep)
+    parity.check("dy", out["dy"], ref.dy, tag, rep)
+    return rep
+
+
+def S(n, h, w, ci, co, k, s, img=False):
+    return wl.ConvShape(f"t{n}x{h}x{w}x{ci}->{co}k{k}s{s}", n, h, w, ci, co, k, s, img)
+
+
+SMALL_SHAPES = [
+    S(2, 32, 32, 16, 32, 3, 1),     # benchmark configuration 1
+    S(2, 7, 6, 3, 8, 3, 2),         # odd extents, stride 2, 3 input channels
+    S(1, 5, 5, 5, 8, 3, 2),
+    S(3, 9, 11, 24, 16, 3, 1),
+    S(2, 12, 10, 40, 24, 1, 1),
+    S(2, 13, 9, 16, 16, 1, 2),
+    S(1, 1, 3, 8, 8, 3, 1),         # fewer rows than any tile
+    S(2, 40, 40, 64, 64, 3, 1),     # several tiles and a ragged tail (3200 rows = 25 x 128)
+    S(2, 38, 42, 48, 96, 3, 1),     # 3192 rows: ragged last tile
+    S(2, 36, 36, 96, 192, 3, 2),
+    S(1, 64, 64, 3, 48, 3, 2, True),  # stem-like
+    S(2, 20, 20, 576, 64, 3, 1),
+    S(2, 20, 20, 288, 288, 1, 1),
+]
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES, ids=lambda s: s.name)
+@pytest.mark.parametrize("mode", [0, 1], ids=["bf16", "f32"])
+def test_block_matches_oracle(shape, mode):
+    if mode == 1 and shape.c_out % 4:
+        pytest.skip("fp32 mode needs c_out % 4 == 0")
+    inp, blk, out = _run_block(shape, mode, cfg_id=11, layer_id=SMALL_SHAPES.index(shape), affine="random")
+    ref = _oracle(inp)
+    _compare(out, ref, mode)
+
+
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[0], SMALL_SHAPES[7], SMALL_SHAPES[9]], ids=lambda s: s.name)
+def test_forced_cuda_core_path_matches_oracle(shape):
+    from paper_2609_10632_b200 import binding as nb
+
+    inp, blk, out = _run_block(shape, 0, cfg_id=12, flags=nb.NB_CBS_FLAG_FORCE_SIMT)
+    assert blk.plan.paths == {"fprop": 0, "dgrad": 0, "wgrad": 0}
+    _compare(out, _oracle(inp), 0)
+
+
+def test_config1_fresh_bn_both_modes():
+    shape, = wl.config_shapes(1)
+    for mode in (1, 0):
+        inp, blk, out = _run_block(shape, mode, cfg_id=1)
+        _compare(out, _oracle(inp), mode)
+
+
+def test_results_are_not_suspiciously_exact():
+    # bf16 outputs cannot be closer to the fp64 oracle than bf16 rounding allows; a much smaller error would mean
+    # the comparison is not comparing two implementations.
+    shape = SMALL_SHAPES[7]
+    inp, blk, out = _run_block(shape, 0, cfg_id=13)
+    ref = _oracle(inp)
+    assert parity.rel_l2(out["a"], ref.a) > 3e-4
+    assert parity.rel_l2(out["dx"], ref.dx) > 3e-4
+
+
+def test_first_layer_without_dx():
+    shape = SMALL_SHAPES[10]
+    inp, blk, out = _run_block(shape, 0, cfg_id=14, need_dx=False)
+    assert "dx" not in out
+    _compare(out, _oracle(inp, need_dx=False), 0, need_dx=False)
+
+
+def test_running_statistics_update():
+    shape = SMALL_SHAPES[3]
+    for mode in (0, 1):
+        inp, blk, out = _run_block(shape, mode, cfg_id=15, running=True, momentum=0.1)
+        rm, rv = np.zeros(shape.c_out), np.ones(shape.c_out)
+        oracle.cbs_fwd(inp.x, inp.w, inp.gamma, inp.beta, shape.stride, EPS, rm, rv, 0.1)
+        np.testing.assert_allclose(out["running_mean"], rm, rtol=0, atol=2e-3 if mode == 0 else 1e-6)
+        np.testing.assert_allclose(out["running_var"], rv, rtol=3e-3 if mode == 0 else 1e-5)
+
+
+def test_constant_channel_has_zero_variance():
+    # a filter of zeros makes one output channel constant: invstd = eps^-1/2, a = SiLU(beta)
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    shape = SMALL_SHAPES[3]
+    inp = wl.make_inputs(shape, 16, 0, affine="random")
+    inp.w[3] = 0.0
+    blk = CbsBlock(shape, mode=nb.NB_MODE_BF16_TC, eps=EPS)
+    blk.upload(inp)
+    blk.step()
+    blk.poll()
+    out = blk.download()
+    ref = _oracle(inp)
+    assert abs(out["invstd"][3] - EPS ** -0.5) < 1e-3 * EPS ** -0.5
+    _compare(out, ref, 0)
+
+
+def test_bn_stats_entry_point():
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    for mode, dt, tag in ((nb.NB_MODE_BF16_TC, torch.float16, nb.NB_DTYPE_F16), (nb.NB_MODE_F32_REF, torch.float32, nb.NB_DTYPE_F32)):
+        shape = S(2, 30, 34, 8, 48, 3, 1)
+        plan = nb.Plan.for_shape(shape, mode=mode)
+        rng = np.random.default_rng(5)
+        y = (rng.normal(size=(shape.m, shape.c_out)) * rng.uniform(0.5, 2, shape.c_out) + rng.normal(size=shape.c_out) * 3).astype(np.float32)
+        ty = torch.from_numpy(y).to(dt).cuda()
+        yq = ty.to(torch.float64).cpu().numpy()
+        mean, invstd, sm, sq = (torch.empty(shape.c_out, dtype=torch.float32, device="cuda") for _ in range(4))
+        ws = torch.empty(plan.fwd_bytes, dtype=torch.uint8, device="cuda")
+        nb.nb_bn_stats(plan, ty, tag, mean, invstd, sm, sq, ws)
+        torch.cuda.synchronize()
+        rmean, rvar, rinv = oracle.bn_stats(yq, EPS)
+        np.testing.assert_allclose(mean.cpu().numpy(), rmean, rtol=1e-5, atol=1e-6)
+        np.testing.assert_allclose(invstd.cpu().numpy(), rinv, rtol=1e-5)
+        np.testing.assert_allclose(sm.cpu().numpy(), yq.sum(0), rtol=1e-5, atol=1e-3)
+        np.testing.assert_allclose(sq.cpu().numpy(), (yq * yq).sum(0), rtol=1e-5)
+        with pytest.raises(nb.NbError) as ei:
+            nb.nb_bn_stats(plan, ty, nb.NB_DTYPE_BF16, mean, invstd, None, None, ws)
+        assert ei.value.status == nb.NB_ERR_UNSUPPORTED
+
+
+def test_bitwise_reproducible():
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    for shape in (SMALL_SHAPES[7], SMALL_SHAPES[9]):
+        inp = wl.make_inputs(shape, 17, 0, affine="random")
+        blk = CbsBlock(shape, mode=nb.NB_MODE_BF16_TC)
+        blk.upload(inp)
+        blk.step()
+        torch.cuda.synchronize()
+        first = {k: getattr(blk, k).clone() for k in ("a", "y", "dx", "dw", "dgamma", "dbeta", "mean", "invstd", "dy")}
+        for k in first:
+            getattr(blk, k).zero_()
+        blk.step()
+        torch.cuda.synchronize()
+        for k, v in first.items():
+            assert torch.equal(v.view(torch.uint8), getattr(blk, k).view(torch.uint8)), k
+
+
+def test_invalid_runtime_arguments_launch_nothing():
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    shape = SMALL_SHAPES[0]
+    blk = CbsBlock(shape)
+    blk.a.fill_(7.0)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(nb.NbError) as ei:
+        nb.nb_conv_bn_silu_fwd(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, None, None, blk.y, blk.mean, blk.invstd, blk.a, small)
+    assert ei.value.status == nb.NB_ERR_WORKSPACE
+    with pytest.raises(nb.NbError) as ei:
+        nb.nb_conv_bn_silu_fwd(blk.plan, blk.x.data_ptr() + 2, blk.w, blk.gamma, blk.beta, None, None, blk.y, blk.mean, blk.invstd, blk.a, blk.ws)
+    assert ei.value.status == nb.NB_ERR_ALIGNMENT
+    with pytest.raises(nb.NbError) as ei:
+        nb.nb_conv_bn_silu_fwd(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, blk.mean, None, blk.y, blk.mean, blk.invstd, blk.a, blk.ws)
+    assert ei.value.status == nb.NB_ERR_INVALID_ARG
+    with pytest.raises(nb.NbError) as ei:
+        nb.nb_conv_bn_silu_bwd_weight(blk.plan, blk.x, None, blk.dw, blk.ws)
+    assert ei.value.status == nb.NB_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert bool((blk.a == 7.0).all())
+
+
+def test_step_from_host_buffers():
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    shape = SMALL_SHAPES[8]
+    inp = wl.make_inputs(shape, 18, 0, affine="random")
+    plan = nb.Plan.for_shape(shape)
+    pin = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).pin_memory()
+    hx, hw, hg = pin(inp.x, torch.bfloat16), pin(inp.w, torch.bfloat16), pin(inp.g, torch.bfloat16)
+    hgam, hbet = pin(inp.gamma, torch.float32), pin(inp.beta, torch.float32)
+    ha = torch.empty(hg.shape, dtype=torch.bfloat16).pin_memory()
+    hdx = torch.empty(hx.shape, dtype=torch.bfloat16).pin_memory()
+    hdw = torch.empty(hw.shape, dtype=torch.float32).pin_memory()
+    hdg, hdb = torch.empty(shape.c_out).pin_memory(), torch.empty(shape.c_out).pin_memory()
+    scratch = torch.empty(plan.step_host_scratch_bytes(), dtype=torch.uint8, device="cuda")
+    nb.nb_conv_bn_silu_step_host(plan, hx, hw, hgam, hbet, hg, ha, hdx, hdw, hdg, hdb, scratch)
+    nb.nb_cbs_poll_status(plan)
+    ref = _oracle(inp)
+    parity.check("a", ha.double().numpy(), ref.a)
+    parity.check("dx", hdx.double().numpy(), ref.dx)
+    parity.check("dw", hdw.double().numpy(), ref.dw)
+    parity.check("dgamma", hdg.double().numpy(), ref.dgamma)
+    parity.check("dbeta", hdb.double().numpy(), ref.dbeta)
