@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the Conv-BN-SiLU forward + backward path on B200.
+
+A "step" is one forward call, one backward-data call and one backward-weight call of the C ABI for every
+Conv-BN-SiLU layer of the workload (default: the 77 layers of the YOLOv8m-class detector at batch 16,
+640 x 640; each layer on its own seeded synthetic tensors of the right shape).  One JSON line is printed:
+
+  value / ms_per_step : whole-job TFLOP/s (2*M*K*Cout per GEMM, three GEMMs per layer) and ms per step with all
+                        tensors resident in HBM, timed with CUDA events over exactly --steps steps;
+  e2e                 : the same through nb_conv_bn_silu_step_host from pinned host buffers, copies inside the timing;
+  roofline            : per-kernel-site device times from an instrumented pass (events around every launch) for the
+                        site that takes the largest share, against the measured peak;
+  cpu_baseline        : the fp64 CPU oracle timed on this host on a bounded sample of the same workload.
+
+`--impl reference` times the CPU oracle alone (the paper ships no code to install as a reference).
+Multi-GPU (`torchrun`): the path does not shard, so every rank runs an independent replica (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "conv_bn_silu_fwd_bwd_bf16_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def workload_layers(name: str):
+    from paper_2609_10632_b200 import workloads as wl
+
+    if name.startswith("cfg"):
+        return wl.config_shapes(int(name[3:]))
+    raise SystemExit(f"unknown workload {name}")
+
+
+def step_flops(layers) -> float:
+    return float(sum(3 * s.gemm_flops for s in layers))
+
+
+# ----------------------------------------------------------------------------- algorithmic work per kernel site
+def site_work(site: str, s):
+    """(flops, bytes) one launch of `site` must perform/move for layer shape s (bf16 activations, fp16 saved y)."""
+    out_e = s.m * s.c_out
+    in_b = 2 * s.n * s.h * s.w * s.c_in
+    w_b = 2 * s.kdim * s.c_out
+    if site == "conv_fprop":
+        return s.gemm_flops, in_b + w_b + 2 * out_e
+    if site == "conv_dgrad":
+        return s.gemm_flops, in_b + w_b + 2 * out_e
+    if site == "conv_wgrad":
+        return s.gemm_flops, in_b + 2 * out_e + 4 * s.kdim * s.c_out
+    if site == "bn_stats":
+        return 3 * out_e, 2 * out_e
+    if site == "bn_silu_apply":
+        return 10 * out_e, 4 * out_e
+    if site == "bn_silu_bwd_reduce":
+        return 15 * out_e, 4 * out_e
+    if site == "bn_silu_bwd_dy":
+        return 18 * out_e, 6 * out_e
+    if site == "dgrad_weight_transform":
+        return 0, 2 * w_b
+    return 0, 0
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+def time_oracle(layers, budget_s: float):
+    """Time the oracle (forward + backward of whole blocks) on a bounded sample: the layers at batch 1, and if that
+    is still over budget a prefix of the distinct shapes.  Returns (TFLOP/s, seconds, flops, cores, description)."""
+    import numpy as np
+
+    import oracle
+    from paper_2609_10632_b200 import workloads as wl
+
+    oracle.build()
+    cores = oracle.num_threads()
+    rate = 15e9  # conservative estimate of the oracle's flop rate, only used to size the sample
+    distinct = wl.distinct_shapes([s.with_batch(1) if s.n > 1 else s for s in layers])
+    chosen, est = [], 0.0
+    for s, mult in distinct:
+        f = 3 * s.gemm_flops
+        if chosen and est + f / rate > budget_s:
+            continue
+        chosen.append((s, mult))
+        est += f / rate
+    flops, secs = 0.0, 0.0
+    for i, (s, mult) in enumerate(chosen):
+        inp = wl.make_inputs(s, cfg_id=5, layer_id=i, bf16=True)
+        t0 = time.perf_counter()
+        oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, 1e-3)
+        secs += time.perf_counter() - t0
+        flops += 3 * s.gemm_flops
+    desc = f"{len(chosen)} of {len(distinct)} distinct layer shapes at batch {chosen[0][0].n}, one fwd+bwd each, fp64 direct loops"
+    return flops / secs / 1e12, secs, flops, cores, desc
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    layers = workload_layers(args.workload)
+    total = args.steps + args.warmup
+    budget = max(2.0, min(30.0, 150.0 / max(1, total)))
+    vals, secs_all = [], []
+    desc, cores = "", 0
+    for i in range(total):
+        v, secs, flops, cores, desc = time_oracle(layers, budget)
+        if i >= args.warmup:
+            vals.append(v)
+            secs_all.append(secs)
+    value = sum(vals) / len(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs_all) / len(secs_all), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "note": "fp64 CPU oracle on a bounded sample per step; ms_per_step is the sample's time"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="cfg5", help="cfg1..cfg5 (cfg5 = the detector's 77 Conv-BN-SiLU layers at batch 16)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--force-simt", action="store_true", help="run the convolutions on the CUDA-core kernels")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        print(f"note: warmup {args.warmup} < 3 breaks the timing rules", file=sys.stderr)
+
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200 import workloads as wl
+    from paper_2609_10632_b200.block import CbsBlock
+
+    nb.load()  # fails loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    layers = workload_layers(args.workload)
+    flags = nb.NB_CBS_FLAG_FORCE_SIMT if args.force_simt else 0
+    plans_probe = [nb.Plan.for_shape(s, flags=flags, device=local) for s in layers]
+    ws_bytes = max(max(p.fwd_bytes, p.bwd_bytes) for p in plans_probe)
+    del plans_probe
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    blocks = [CbsBlock(s, flags=flags, device=local, workspace=ws) for s in layers]
+    for i, b in enumerate(blocks):
+        b.fill_random(seed=1000 + i)
+    resident = sum(sum(t.numel() * t.element_size() for t in (b.x, b.w, b.g, b.y, b.a, b.dy, b.dx, b.dw)) for b in blocks)
+    flops = step_flops(layers)
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        for b in blocks:
+            b.step()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    for b in blocks:
+        b.poll()
+    barrier()
+    l0 = nb.nb_cbs_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        ev0.record(stream)
+        for _ in range(args.steps):
+            one_step()
+        ev1.record(stream)
+        barrier()
+    launches = nb.nb_cbs_launch_count() - l0
+    ms_total = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    peaks = load_peaks()
+
+    # ---------------- instrumented pass: per-site device times (events around every launch; calls wait for each kernel)
+    roofline, kernels = None, {}
+    if not args.no_profile:
+        for b in blocks:
+            nb.nb_cbs_profile_enable(b.plan, True)
+        prof_steps = max(1, min(args.steps, 3))
+        for _ in range(prof_steps):
+            one_step()
+        torch.cuda.synchronize()
+        agg = {}
+        for b in blocks:
+            for site, (ms, n) in nb.nb_cbs_profile_read(b.plan).items():
+                if n == 0:
+                    continue
+                f, by = site_work(site, b.shape)
+                a = agg.setdefault(site, {"ms": 0.0, "launches": 0, "flops": 0.0, "bytes": 0.0})
+                a["ms"] += ms
+                a["launches"] += n
+                a["flops"] += f * n
+                a["bytes"] += by * n
+            nb.nb_cbs_profile_enable(b.plan, False)
+        tot_ms = sum(a["ms"] for a in agg.values()) or 1.0
+        tensor_sites = {"conv_fprop", "conv_dgrad", "conv_wgrad"}
+        for site, a in agg.items():
+            sec = a["ms"] * 1e-3
+            k = {"launches": a["launches"], "ms_per_step": a["ms"] / prof_steps, "share": a["ms"] / tot_ms}
+            if site in tensor_sites:
+                k["tflops"] = a["flops"] / sec / 1e12
+                k["gbs_algorithmic"] = a["bytes"] / sec / 1e9
+            else:
+                k["gbs"] = a["bytes"] / sec / 1e9
+            kernels[site] = k
+        top = max(agg, key=lambda s: agg[s]["ms"])
+        a = agg[top]
+        sec = a["ms"] * 1e-3
+        if top in tensor_sites:
+            ach = a["flops"] / sec / 1e12
+            # a GEMM site that moves more bytes than its flops justify is HBM-bound (arithmetic intensity under the ridge)
+            ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+            if a["flops"] / max(a["bytes"], 1.0) >= ridge:
+                roofline = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+            else:
+                roofline = {"kernel": top, "bound": "hbm", "achieved": a["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roofline = {"kernel": top, "bound": "hbm", "achieved": a["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["traffic"] = None
+        roofline["peak_source"] = peaks["source"] + (" (burst figure: kernels timed one at a time)" if roofline["bound"] == "tensor" else "")
+        roofline["avg_launch_ms"] = a["ms"] / a["launches"]
+        roofline["share_of_step"] = a["ms"] / tot_ms
+
+    # ---------------- end to end from pinned host buffers through the C ABI
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, secs, fl, cores, desc = time_oracle(layers, args.cpu_budget)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": f"{desc}; {secs:.1f} s"}
+
+    if rank == 0:
+        paths = {"fprop": 0, "dgrad": 0, "wgrad": 0}
+        for b in blocks:
+            for k in paths:
+                paths[k] += b.plan.paths[k]
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": f"{args.workload}: {len(layers)} Conv-BN-SiLU layers, batch {layers[0].n}, fwd + bwd_data + bwd_weight per layer "
+                            f"(stem data gradient included), each layer on its own tensors",
+                "l2_policy": f"inputs larger than L2: {resident / 1e9:.2f} GB of tensors are touched per step",
+                "gflop_per_step": flops / 1e9, "multi_gpu": "replicas only", "tensor_core_layers": paths, "layers": len(layers),
+                "frac_of_nominal_bf16_peak": value / world / NOMINAL["bf16_tflops"],
+                "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
+            },
+            "clocks": clocks.summary(), "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
+            "kernels": kernels,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
+    """Whole steps through nb_conv_bn_silu_step_host: pinned host inputs -> device -> three calls -> pinned host outputs."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    host = {}  # per distinct shape: pinned input and output buffers (inputs filled from the device tensors)
+    scratch_bytes = 0
+    h2d = d2h = 0
+    for b in blocks:
+        s = b.shape
+        scratch_bytes = max(scratch_bytes, b.plan.step_host_scratch_bytes())
+        if s.key not in host:
+            pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
+            hin = {k: pin(getattr(b, k)) for k in ("x", "w", "gamma", "beta", "g")}
+            for k, t in hin.items():
+                t.copy_(getattr(b, k))
+            hout = {k: pin(getattr(b, k)) for k in ("a", "dx", "dw", "dgamma", "dbeta")}
+            host[s.key] = (hin, hout)
+        hin, hout = host[s.key]
+        h2d += sum(t.numel() * t.element_size() for t in hin.values())
+        d2h += sum(t.numel() * t.element_size() for t in hout.values())
+    # free the resident tensors of the device-timed arm before allocating the scratch
+    scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def one():
+        for b in blocks:
+            hin, hout = host[b.shape.key]
+            nb.nb_conv_bn_silu_step_host(b.plan, hin["x"], hin["w"], hin["gamma"], hin["beta"], hin["g"], hout["a"], hout["dx"],
+                                         hout["dw"], hout["dgamma"], hout["dbeta"], scratch)
+
+    steps = max(1, min(args.steps, 3))
+    one()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(steps):
+        one()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": world * flops / (ms / steps * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": ms / steps, "steps": steps}
+
+
+if __name__ == "__main__":
+    main()

@@ -108,6 +108,18 @@ nb_status nb_cbs_plan_paths(nb_cbs_plan plan, int32_t* paths3);
  * status block. */
 nb_status nb_cbs_poll_status(nb_cbs_plan plan, void* stream);
 
+/* Diagnostics (the paper has no counterpart; they exist for the benchmark's per-kernel roofline figures).
+ * nb_cbs_launch_count: number of CUDA kernels this library has launched in this process so far.
+ * nb_cbs_profile_enable(plan, 1): from now on every kernel site of calls on this plan is bracketed by CUDA
+ *   events and the call WAITS for the kernel, accumulating its device time; enable = 0 turns it off again;
+ *   either call clears the accumulators.  Not for use inside stream capture.
+ * nb_cbs_profile_site_name(i): name of kernel site i, NULL once i is past the last site.
+ * nb_cbs_profile_read: accumulated milliseconds and launch count of one site since the last enable call. */
+unsigned long long nb_cbs_launch_count(void);
+nb_status nb_cbs_profile_enable(nb_cbs_plan plan, int32_t enable);
+const char* nb_cbs_profile_site_name(int32_t site);
+nb_status nb_cbs_profile_read(nb_cbs_plan plan, int32_t site, double* total_ms, int64_t* launches);
+
 /* Forward (Sec. 6 operators; BN in fp32 per Sec. 3.2 / Table 2 row 2):
  *   y[n,p,q,c'] = sum_{r,t,c} x[n, p*s-P+r, q*s-P+t, c] * w[c',r,t,c]        (zero outside the image)
  *   mean_c = (1/M) sum y ; var_c = (1/M) sum (y-mean_c)^2 (biased) ; invstd_c = (var_c + eps)^-1/2

@@ -24,7 +24,8 @@ EXPORTS = (
     "nb_abi_version", "nb_last_error", "nb_cbs_plan_create", "nb_cbs_plan_destroy", "nb_cbs_out_shape",
     "nb_cbs_workspace_bytes", "nb_cbs_plan_paths", "nb_cbs_poll_status", "nb_conv_bn_silu_fwd", "nb_bn_stats",
     "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
-    "nb_conv_bn_silu_step_host",
+    "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
+    "nb_cbs_profile_read",
 )
 
 
@@ -69,8 +70,14 @@ def load() -> ctypes.CDLL:
         lib.nb_conv_bn_silu_bwd_weight.argtypes = [V, V, V, FP, V, c_size_t, V]
         lib.nb_cbs_step_host_scratch_bytes.argtypes = [V, POINTER(c_size_t)]
         lib.nb_conv_bn_silu_step_host.argtypes = [V, V, V, FP, FP, V, V, V, FP, FP, FP, V, c_size_t, V]
+        lib.nb_cbs_launch_count.argtypes = []
+        lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
+        lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
+        lib.nb_cbs_profile_site_name.argtypes = [c_int32]
+        lib.nb_cbs_profile_site_name.restype = c_char_p
+        lib.nb_cbs_profile_read.argtypes = [V, c_int32, POINTER(ctypes.c_double), POINTER(ctypes.c_int64)]
         for name in EXPORTS:
-            if name not in ("nb_abi_version", "nb_last_error"):
+            if name not in ("nb_abi_version", "nb_last_error", "nb_cbs_launch_count", "nb_cbs_profile_site_name"):
                 getattr(lib, name).restype = c_int32
         _lib = lib
     return _lib
@@ -159,6 +166,28 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+def nb_cbs_launch_count() -> int:
+    return int(load().nb_cbs_launch_count())
+
+
+def nb_cbs_profile_enable(plan: Plan, enable: bool):
+    _check(load().nb_cbs_profile_enable(plan.handle, 1 if enable else 0))
+
+
+def nb_cbs_profile_read(plan: Plan) -> dict:
+    """{site name: (total_ms, launches)} accumulated since profiling was enabled on this plan."""
+    out = {}
+    i = 0
+    while True:
+        name = load().nb_cbs_profile_site_name(i)
+        if name is None:
+            return out
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        _check(load().nb_cbs_profile_read(plan.handle, i, byref(ms), byref(n)))
+        out[name.decode()] = (ms.value, n.value)
+        i += 1
 
 
 def nb_cbs_poll_status(plan: Plan, stream=None):

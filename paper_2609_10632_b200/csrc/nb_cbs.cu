@@ -3,6 +3,7 @@
 #include "../../include/nb_cbs.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -38,6 +39,14 @@ nb_status fail(nb_status code, const char* fmt, ...) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+std::atomic<unsigned long long> g_launches{0};  // kernels launched by this library in this process
+
+enum Site { SITE_FPROP = 0, SITE_STATS, SITE_FINALIZE, SITE_APPLY, SITE_BWD_REDUCE, SITE_BWD_FINALIZE, SITE_BWD_DY,
+            SITE_WTRANSFORM, SITE_DGRAD, SITE_WGRAD, SITE_SPLITK_REDUCE, SITE_COUNT };
+const char* const kSiteNames[SITE_COUNT] = {"conv_fprop", "bn_stats", "bn_finalize", "bn_silu_apply", "bn_silu_bwd_reduce",
+                                            "bn_bwd_finalize", "bn_silu_bwd_dy", "dgrad_weight_transform", "conv_dgrad",
+                                            "conv_wgrad", "wgrad_splitk_reduce"};
+
 struct EwCfg {  // launch geometry of the [M][C] passes
     int vec, cgs, tpb;
     long long total_vecs;
@@ -57,6 +66,10 @@ struct nb_cbs_plan_s {
     int wg_splits;   // split-K slices of the CUDA-core wgrad
     long long wg_chunk;
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
+    bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    double prof_ms[SITE_COUNT] = {};
+    long long prof_n[SITE_COUNT] = {};
     size_t fwd_bytes, bwd_bytes;
     // workspace offsets
     size_t off_scale, off_shift, off_fpart;                  // forward
@@ -86,7 +99,27 @@ nb_status check_ws(const void* ws, size_t have, size_t need) {
     return NB_OK;
 }
 
+// Brackets one kernel site with events when the plan is in profiling mode (diagnostic; synchronises the stream).
+struct SiteTimer {
+    nb_cbs_plan_s* p;
+    int site;
+    cudaStream_t st;
+    SiteTimer(nb_cbs_plan_s* plan, int s, cudaStream_t stream) : p(plan), site(s), st(stream) {
+        if (p->profiling) cudaEventRecord(p->ev0, st);
+    }
+    ~SiteTimer() {
+        if (!p->profiling) return;
+        cudaEventRecord(p->ev1, st);
+        float ms = 0.f;
+        if (cudaEventSynchronize(p->ev1) == cudaSuccess && cudaEventElapsedTime(&ms, p->ev0, p->ev1) == cudaSuccess) {
+            p->prof_ms[site] += ms;
+            p->prof_n[site] += 1;
+        }
+    }
+};
+
 nb_status launch_ok(const char* what) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(NB_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
     return NB_OK;
@@ -105,6 +138,7 @@ nb_status launch_ok(const char* what) {
 // ---------------------------------------------------------------- elementwise launch helpers
 template <typename YT> nb_status run_stats_partial(nb_cbs_plan_s* p, const void* y, float* partials, cudaStream_t st) {
     const EwCfg& e = p->ew;
+    SiteTimer tm(p, SITE_STATS, st);
     bn_stats_partial_kernel<YT><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
         static_cast<const YT*>(y), e.total_vecs, p->g.c_out, partials);
     return launch_ok("bn_stats_partial");
@@ -114,6 +148,7 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
                        float* invstd, float* scale, float* shift, float* rmean, float* rvar, float* sum, float* sumsq,
                        cudaStream_t st) {
     const int C = p->g.c_out;
+    SiteTimer tm(p, SITE_FINALIZE, st);
     bn_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
                                                               gamma, beta, mean, invstd, scale, shift, rmean, rvar, sum, sumsq);
     return launch_ok("bn_finalize");
@@ -122,6 +157,7 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
 template <typename YT, typename AT, bool FAST>
 nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
     const EwCfg& e = p->ew;
+    SiteTimer tm(p, SITE_APPLY, st);
     bn_silu_apply_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
                                                                        p->g.c_out, scale, shift);
     return launch_ok("bn_silu_apply");
@@ -133,11 +169,18 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
                               float* coef, cudaStream_t st) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
-    bn_silu_bwd_reduce_kernel<YT, AT, FAST><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
-        static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials);
-    NB_LAUNCH_OK("bn_silu_bwd_reduce");
-    bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
-    NB_LAUNCH_OK("bn_bwd_finalize");
+    {
+        SiteTimer tm(p, SITE_BWD_REDUCE, st);
+        bn_silu_bwd_reduce_kernel<YT, AT, FAST><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials);
+        NB_LAUNCH_OK("bn_silu_bwd_reduce");
+    }
+    {
+        SiteTimer tm(p, SITE_BWD_FINALIZE, st);
+        bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
+        NB_LAUNCH_OK("bn_bwd_finalize");
+    }
+    SiteTimer tm(p, SITE_BWD_DY, st);
     bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
                                                                         static_cast<AT*>(dy), e.total_vecs, C, mean, invstd, gamma,
                                                                         beta, coef);
@@ -149,6 +192,7 @@ template <typename TIN, typename TOUT>
 nb_status run_simt_fprop(nb_cbs_plan_s* p, const void* x, const void* w, void* y, cudaStream_t st) {
     FpropProblem<TIN, TIN> prob{static_cast<const TIN*>(x), static_cast<const TIN*>(w), p->g};
     dim3 grid((unsigned)((p->g.m + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_out + SIMT_BN - 1) / SIMT_BN), 1);
+    SiteTimer tm(p, SITE_FPROP, st);
     simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TOUT*>(y), (long long)p->g.kdim);
     return launch_ok("simt fprop");
 }
@@ -158,6 +202,7 @@ nb_status run_simt_dgrad(nb_cbs_plan_s* p, const void* dy, const void* w, void* 
     DgradProblem<TIN, TIN> prob{static_cast<const TIN*>(dy), static_cast<const TIN*>(w), p->g};
     const long long I = (long long)p->g.n * p->g.h * p->g.w;
     dim3 grid((unsigned)((I + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_in + SIMT_BN - 1) / SIMT_BN), 1);
+    SiteTimer tm(p, SITE_DGRAD, st);
     simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TIN*>(dx), (long long)p->g.k * p->g.k * p->g.c_out);
     return launch_ok("simt dgrad");
 }
@@ -167,12 +212,17 @@ nb_status run_simt_wgrad(nb_cbs_plan_s* p, const void* x, const void* dy, float*
     WgradProblem<TIN, TIN> prob{static_cast<const TIN*>(dy), static_cast<const TIN*>(x), p->g};
     dim3 grid((unsigned)((p->g.c_out + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.kdim + SIMT_BN - 1) / SIMT_BN), (unsigned)p->wg_splits);
     if (p->wg_splits == 1) {
+        SiteTimer tm(p, SITE_WGRAD, st);
         simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, dw, p->g.m);
         return launch_ok("simt wgrad");
     }
-    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, partial, p->wg_chunk);
-    NB_LAUNCH_OK("simt wgrad (split-K)");
+    {
+        SiteTimer tm(p, SITE_WGRAD, st);
+        simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, partial, p->wg_chunk);
+        NB_LAUNCH_OK("simt wgrad (split-K)");
+    }
     const size_t elems = (size_t)p->g.c_out * p->g.kdim;
+    SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
     splitk_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, p->wg_splits, elems, dw);
     return launch_ok("splitk_reduce");
 }
@@ -296,6 +346,8 @@ nb_status nb_cbs_plan_destroy(nb_cbs_plan p) {
         cudaGetDevice(&cur);
         cudaSetDevice(p->device);
         cudaFree(p->status);
+        if (p->ev0) cudaEventDestroy(p->ev0);
+        if (p->ev1) cudaEventDestroy(p->ev1);
         cudaSetDevice(cur);
     }
     delete p;
@@ -324,6 +376,34 @@ nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
     paths3[0] = p->tc.fprop ? 1 : 0;
     paths3[1] = p->tc.dgrad ? 1 : 0;
     paths3[2] = p->tc.wgrad ? 1 : 0;
+    return NB_OK;
+}
+
+unsigned long long nb_cbs_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+nb_status nb_cbs_profile_enable(nb_cbs_plan p, int32_t enable) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    if (enable && !p->ev0) {
+        NB_CUDA_CHECK(cudaEventCreate(&p->ev0));
+        NB_CUDA_CHECK(cudaEventCreate(&p->ev1));
+    }
+    p->profiling = enable != 0;
+    for (int i = 0; i < SITE_COUNT; ++i) {
+        p->prof_ms[i] = 0.0;
+        p->prof_n[i] = 0;
+    }
+    return NB_OK;
+}
+
+const char* nb_cbs_profile_site_name(int32_t site) { return (site >= 0 && site < SITE_COUNT) ? kSiteNames[site] : nullptr; }
+
+nb_status nb_cbs_profile_read(nb_cbs_plan p, int32_t site, double* total_ms, int64_t* launches) {
+    g_err.clear();
+    if (!p || !total_ms || !launches) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    if (site < 0 || site >= SITE_COUNT) return fail(NB_ERR_INVALID_ARG, "site %d out of range", site);
+    *total_ms = p->prof_ms[site];
+    *launches = p->prof_n[site];
     return NB_OK;
 }
 
