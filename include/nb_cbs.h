@@ -155,6 +155,26 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan plan, const void* g, const void* 
 nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan plan, const void* x, const void* dy, float* dw, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
+/* Batch statistics for callers that cannot allocate device memory.  (The paper has no counterpart of this entry
+ * point.)  Some hosts of this library must not call cudaMalloc -- code running under a framework's caching allocator
+ * that forbids raw allocations, real-time or plug-in code with a fixed memory budget, or code that would have to size
+ * a workspace before it knows the tensor -- and nb_bn_stats needs both a plan (whose creation allocates a status
+ * block) and a caller-provided workspace.  This variant computes the same mean / invstd / sum / sumsq of a dense
+ * [m][c] tensor, with no plan and no workspace: its partial sums live in an array built into the library
+ * (2 MiB, file-scope device memory, held by every GPU that loads the library until the process exits).
+ *   Limits: c <= 1024 channels, c % 8 == 0 for NB_DTYPE_F16, c % 4 == 0 for NB_DTYPE_F32, m >= 2; anything beyond
+ *   returns NB_ERR_UNSUPPORTED (or NB_ERR_INVALID_ARG) with a message and launches nothing.
+ *   It runs on the CURRENT device.  The first call on each device looks up the array's device address (one
+ *   cudaGetSymbolAddress); make that first call before any stream capture begins.
+ *   It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   Every call on a device shares the one array, which keeps the previous call's contents; each call overwrites
+ *   every entry it later reads, so nothing needs clearing -- but two calls whose kernels overlap on the GPU
+ *   (different streams, no ordering between them) race on it and give wrong results.  Serialise such calls.
+ * y, mean, invstd (and sum, sumsq when not NULL) are device pointers, 16-byte aligned; results are written
+ * asynchronously on `stream`. */
+nb_status nb_bn_stats_static(const void* y, int32_t y_dtype, int64_t m, int32_t c, float eps, float* mean, float* invstd,
+                             float* sum, float* sumsq, void* stream);
+
 /* One whole training step of the block from HOST buffers (the end-to-end path of a caller whose data
  * lives in host memory): copies host_x, host_w, host_gamma, host_beta, host_g to the device, runs the
  * forward call and the two backward calls above, and copies a, dx (unless host_dx is NULL), dw, dgamma,

@@ -25,7 +25,7 @@ EXPORTS = (
     "nb_cbs_workspace_bytes", "nb_cbs_plan_paths", "nb_cbs_poll_status", "nb_conv_bn_silu_fwd", "nb_bn_stats",
     "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
-    "nb_cbs_profile_read",
+    "nb_cbs_profile_read", "nb_bn_stats_static",
 )
 
 
@@ -70,6 +70,7 @@ def load() -> ctypes.CDLL:
         lib.nb_conv_bn_silu_bwd_weight.argtypes = [V, V, V, FP, V, c_size_t, V]
         lib.nb_cbs_step_host_scratch_bytes.argtypes = [V, POINTER(c_size_t)]
         lib.nb_conv_bn_silu_step_host.argtypes = [V, V, V, FP, FP, V, V, V, FP, FP, FP, V, c_size_t, V]
+        lib.nb_bn_stats_static.argtypes = [V, c_int32, ctypes.c_int64, c_int32, c_float, FP, FP, FP, FP, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -205,6 +206,11 @@ def nb_conv_bn_silu_fwd(plan: Plan, x, w, gamma, beta, running_mean, running_var
 def nb_bn_stats(plan: Plan, y, y_dtype, mean, invstd, sum_, sumsq, workspace, stream=None):
     _check(load().nb_bn_stats(plan.handle, _ptr(y), y_dtype, _ptr(mean), _ptr(invstd), _ptr(sum_), _ptr(sumsq), _ptr(workspace),
                               _nbytes(workspace), _stream(stream)))
+
+
+def nb_bn_stats_static(y, y_dtype, m, c, eps, mean, invstd, sum_=None, sumsq=None, stream=None):
+    """Plan-free, workspace-free batch statistics on the current device (scratch is an array inside the library)."""
+    _check(load().nb_bn_stats_static(_ptr(y), y_dtype, m, c, eps, _ptr(mean), _ptr(invstd), _ptr(sum_), _ptr(sumsq), _stream(stream)))
 
 
 def nb_conv_bn_silu_bwd_data(plan: Plan, g, y_saved, save_mean, save_invstd, gamma, beta, w, dx, dgamma, dbeta, dy_out,

@@ -7,6 +7,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 
@@ -509,6 +510,84 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     if (p->tc.wgrad) return tc_wgrad(&p->tc, p->g, x, dy, dw, partial, p->status, st);
     return run_simt_wgrad<__nv_bfloat16>(p, x, dy, dw, partial, st);
 }
+
+}  // extern "C"
+
+// ---------------------------------------------------------------- batch statistics without any allocation
+// Scratch for nb_bn_stats_static: partial sums [kStaticParts][2][kStaticMaxC] floats = 2 MiB, resident on every
+// GPU that loads this library until the process exits.  In host code the name `g_static_partials` is only a
+// handle for the symbol, never a device address: the address comes from cudaGetSymbolAddress below.
+namespace {
+constexpr int kStaticParts = 256;
+constexpr int kStaticMaxC = 1024;
+constexpr int kStaticMaxDevices = 64;
+}  // namespace
+static __device__ __align__(256) float g_static_partials[(size_t)kStaticParts * 2 * kStaticMaxC];
+
+namespace {
+std::mutex g_static_mu;
+float* g_static_ptr[kStaticMaxDevices] = {};
+int g_static_sms[kStaticMaxDevices] = {};
+
+// Once per device, with that device current: resolve the device address of the static scratch array.
+nb_status static_scratch_for_current_device(float** out, int* sms) {
+    int dev = -1;
+    NB_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kStaticMaxDevices) return fail(NB_ERR_UNSUPPORTED, "device ordinal %d is beyond %d", dev, kStaticMaxDevices);
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        int major = 0, count = 0;
+        NB_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return fail(NB_ERR_ARCH, "device %d is not compute capability 10.x", dev);
+        NB_CUDA_CHECK(cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev));
+        void* ptr = nullptr;
+        NB_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_partials));
+        if (!ptr) return fail(NB_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_sms[dev] = count;
+        g_static_ptr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    *sms = g_static_sms[dev];
+    return NB_OK;
+}
+}  // namespace
+
+extern "C" nb_status nb_bn_stats_static(const void* y, int32_t y_dtype, int64_t m, int32_t c, float eps, float* mean, float* invstd,
+                                        float* sum, float* sumsq, void* stream) {
+    g_err.clear();
+    NB_CHECK_PTR(y); NB_CHECK_PTR(mean); NB_CHECK_PTR(invstd);
+    NB_CHECK_PTR(sum, true); NB_CHECK_PTR(sumsq, true);
+    if (y_dtype != NB_DTYPE_F16 && y_dtype != NB_DTYPE_F32) return fail(NB_ERR_UNSUPPORTED, "y_dtype %d: only F16 and F32 are supported", y_dtype);
+    if (m < 2 || c <= 0) return fail(NB_ERR_INVALID_ARG, "need m >= 2 rows and c > 0 channels (m=%lld c=%d)", (long long)m, c);
+    if (!(eps > 0.f)) return fail(NB_ERR_INVALID_ARG, "eps must be positive");
+    const int vec = y_dtype == NB_DTYPE_F32 ? 4 : 8;
+    if (c % vec) return fail(NB_ERR_UNSUPPORTED, "c=%d must be a multiple of %d for this dtype", c, vec);
+    if (c > kStaticMaxC)
+        return fail(NB_ERR_UNSUPPORTED, "c=%d exceeds the %d channels the built-in scratch array holds; use nb_bn_stats with a workspace", c, kStaticMaxC);
+    if ((double)m * c >= 9.0e18) return fail(NB_ERR_UNSUPPORTED, "tensor too large");
+    float* part = nullptr;
+    int sms = 0;
+    NB_TRY(static_scratch_for_current_device(&part, &sms));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int cgs = c / vec;
+    const int R = cgs >= 256 ? 1 : 256 / cgs;
+    const int tpb = cgs * R;
+    const long long total_vecs = (long long)m * cgs;
+    const long long max_blocks = (total_vecs + tpb - 1) / tpb;
+    const int blocks = (int)std::min<long long>(max_blocks, std::min(kStaticParts, std::max(1, sms)));
+    // Every partial that the second kernel reads is written by the first one in this same call, so nothing in the
+    // array has to start at zero and the previous call's contents do not matter.
+    if (y_dtype == NB_DTYPE_F32)
+        bn_stats_partial_kernel<float><<<blocks, tpb, (size_t)tpb * vec * sizeof(float), st>>>(static_cast<const float*>(y), total_vecs, c, part);
+    else
+        bn_stats_partial_kernel<__half><<<blocks, tpb, (size_t)tpb * vec * sizeof(float), st>>>(static_cast<const __half*>(y), total_vecs, c, part);
+    NB_LAUNCH_OK("bn_stats_partial (static scratch)");
+    bn_finalize_kernel<<<(c + 31) / 32, dim3(32, 32), 0, st>>>(part, blocks, c, (double)m, eps, 0.f, nullptr, nullptr, mean, invstd, nullptr,
+                                                              nullptr, nullptr, nullptr, sum, sumsq);
+    return launch_ok("bn_finalize (static scratch)");
+}
+
+extern "C" {
 
 // ---------------------------------------------------------------- host-buffer step
 namespace {
