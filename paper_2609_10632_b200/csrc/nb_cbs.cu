@@ -446,7 +446,11 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
     } else if (p->tc.fprop) {
-        NB_TRY(tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st));  // writes y (fp16) and the partial sums
+        SiteTimer tm(p, SITE_FPROP, st);
+        const long long l0 = p->tc.launches;
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st);  // writes y (fp16) and the partial sums
+        g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
+        if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
     } else {
         NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y_saved, st)));
@@ -494,7 +498,14 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     }
     NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st)));
     if (!dx) return NB_OK;
-    if (p->tc.dgrad) return tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st);
+    if (p->tc.dgrad) {
+        SiteTimer tm(p, SITE_DGRAD, st);
+        const long long l0 = p->tc.launches;
+        const nb_status ts = tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st);
+        g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
+        if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
+        return NB_OK;
+    }
     return run_simt_dgrad<__nv_bfloat16>(p, dy_out, w, dx, st);
 }
 
@@ -507,7 +518,14 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_wgpart);
     if (is_f32(p)) return run_simt_wgrad<float>(p, x, dy, dw, partial, st);
-    if (p->tc.wgrad) return tc_wgrad(&p->tc, p->g, x, dy, dw, partial, p->status, st);
+    if (p->tc.wgrad) {
+        SiteTimer tm(p, SITE_WGRAD, st);
+        const long long l0 = p->tc.launches;
+        const nb_status ts = tc_wgrad(&p->tc, p->g, x, dy, dw, partial, p->status, st);
+        g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
+        if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
+        return NB_OK;
+    }
     return run_simt_wgrad<__nv_bfloat16>(p, x, dy, dw, partial, st);
 }
 

@@ -1,25 +1,671 @@
-// Tensor-core (tcgen05 / TMEM / TMA) convolution kernels: plan record and entry points.
+// Tensor-core convolution kernels for sm_100a: an implicit GEMM whose A operand (activation pixels x channels of
+// one filter tap) is fetched by TMA in im2col mode, whose B operand (filter rows) is fetched by tiled TMA, whose
+// products are issued as tcgen05.mma by one thread with fp32 accumulators in TMEM, and whose epilogue (four warps)
+// reads the accumulators back with tcgen05.ld, converts, stages the tile in shared memory, takes per-channel sums
+// for the batch statistics and writes coalesced rows.  The same kernel computes fprop (A = x, B = w) and dgrad
+// (A = dy, B = the filter rearranged per output-parity class).  No multicast anywhere; every wait is bounded.
 #pragma once
-#include "common.cuh"
+#include <cuda.h>
+
+#include <algorithm>
+#include <cstring>
+#include <string>
+
 #include "../../include/nb_cbs.h"
+#include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace nbcbs {
 
-struct TcPlan {
-    bool fprop = false, dgrad = false, wgrad = false;
-    int fprop_parts = 0;             // rows of the [parts][2][Cout] partial-sum buffer the fprop epilogue writes
-    size_t wt_bytes = 0;             // rearranged filter for dgrad
-    size_t wgrad_partial_bytes = 0;  // split-K partial buffer of the wgrad kernel
+// ------------------------------------------------------------------------------------------ kernel parameters
+struct IgemmParams {
+    CUtensorMap tmA;  // im2col map over the activation [N][Hs][Ws][Ca]
+    CUtensorMap tmB;  // tiled map over the filter matrix [rowsB][ntaps*Ca], K contiguous
+    long long M;      // rows of the GEMM: n * Hq * Wq
+    int Hq, Wq;       // traversal grid per image
+    int ts;           // traversal stride (input pixels per grid step)
+    int lo_w, lo_h;   // input coordinate of grid position 0 for tap offset 0
+    int ntaps;
+    int Ca, KC, kc_per_tap;
+    int BN, n_tiles, m_tiles;
+    int stages, acc_stride, tmem_cols;
+    uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
+    int ldo;                     // channels per output pixel
+    int Hout, Wout, os, oa, ob;  // GEMM row (n,i,j) -> output pixel (n, i*os+oa, j*os+ob) of an Hout x Wout image
+    void* out;
+    float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
+    int* status;
+    uint16_t off_w[9], off_h[9];
 };
 
-inline const char* tc_last_error() { return ""; }
+constexpr int TC_BM = 128;
+constexpr int TC_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 
-inline nb_status tc_plan_init(TcPlan* tc, const Geom&, bool, int, const cudaDeviceProp&) {
-    *tc = TcPlan();
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded mbarrier wait: gives up after ~2 s (or as soon as another role has given up), records the site.
+__device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((i & 127u) == 127u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > 2000000000ull) {
+                *abort_flag = 1;
+                if (atomicCAS(status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
+                    status[ST_WHERE] = site;
+                    status[ST_DETAIL] = (int)blockIdx.x;
+                }
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the same decision.
+__device__ __forceinline__ bool epi_bar_and(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t"
+        "}\n"
+        : "=r"(r)
+        : "r"((uint32_t)ok)
+        : "memory");
+    return r != 0;
+}
+
+template <typename OutT> __device__ __forceinline__ uint32_t pack2(float a, float b, int* sat);
+template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b, int*) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, int* sat) {
+    if (fabsf(a) > 65504.f || fabsf(b) > 65504.f) {
+        *sat += 1;
+        a = fminf(fmaxf(a, -65504.f), 65504.f);
+        b = fminf(fmaxf(b, -65504.f), 65504.f);
+    }
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <typename OutT, bool STATS>
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = sA + (size_t)p.stages * p.a_stage_bytes;
+    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging tile [128][BN] of OutT, row pitch BN*2+16 bytes
+    const int pitch = p.BN * 2 + 16;
+    float* stat_sum = reinterpret_cast<float*>(stg + (size_t)TC_BM * pitch);  // [ldo]
+    float* stat_sq = stat_sum + p.ldo;                                        // [ldo]
+    float* wpart = stat_sq + p.ldo;                                           // [4][2][BN]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + 8 * p.BN);
+    uint64_t* full = bars;                // [stages]
+    uint64_t* empty = bars + p.stages;    // [stages]
+    uint64_t* tfull = empty + p.stages;   // [2]
+    uint64_t* tempty = tfull + 2;         // [2]
+    uint64_t* drain = tempty + 2;         // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int kblocks = p.ntaps * p.kc_per_tap;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(empty + s, 1);
+        }
+        ptx::mbar_init(tfull, 1);
+        ptx::mbar_init(tfull + 1, 1);
+        ptx::mbar_init(tempty, 128);
+        ptx::mbar_init(tempty + 1, 128);
+        ptx::mbar_init(drain, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (STATS) {
+        for (int c = threadIdx.x; c < 2 * p.ldo; c += TC_THREADS) stat_sum[c] = 0.f;
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (one thread)
+        if (lane == 0) {
+            ptx::prefetch_tmap(&p.tmA);
+            ptx::prefetch_tmap(&p.tmB);
+            int s = 0;
+            uint32_t ph = 0;
+            long long issued = 0;
+            bool ok = true;
+            const uint32_t tx_bytes = (uint32_t)(TC_BM * p.KC * 2 + p.BN * p.KC * 2);
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
+                const long long m0 = (long long)m_tile * TC_BM;
+                const int j0 = (int)(m0 % p.Wq);
+                const long long t1 = m0 / p.Wq;
+                const int i0 = (int)(t1 % p.Hq), n0 = (int)(t1 / p.Hq);
+                const int cw = p.lo_w + j0 * p.ts, ch = p.lo_h + i0 * p.ts;
+                for (int tap = 0; ok && tap < p.ntaps; ++tap) {
+                    for (int kc = 0; kc < p.kc_per_tap; ++kc) {
+                        if (!wait_bar(empty + s, ph ^ 1u, abort_flag, p.status, 1)) {
+                            ok = false;
+                            break;
+                        }
+                        ptx::mbar_expect_tx(full + s, tx_bytes);
+                        ptx::tma_load_im2col_4d(sA + (size_t)s * p.a_stage_bytes, &p.tmA, full + s, kc * p.KC, cw, ch, n0, p.off_w[tap],
+                                                p.off_h[tap]);
+                        ptx::tma_load_2d(sB + (size_t)s * p.b_stage_bytes, &p.tmB, full + s, tap * p.Ca + kc * p.KC, n_tile * p.BN);
+                        ++issued;
+                        if (++s == p.stages) {
+                            s = 0;
+                            ph ^= 1u;
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
+                const int back = issued < (long long)p.stages ? (int)issued : p.stages;
+                for (int b = 0; b < back; ++b) {
+                    s = (s == 0) ? p.stages - 1 : s - 1;
+                    if (s == p.stages - 1) ph ^= 1u;
+                    for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            int s = 0, acc = 0;
+            uint32_t ph = 0, acc_ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                if (!wait_bar(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.acc_stride);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!wait_bar(full + s, ph, abort_flag, p.status, 3)) {
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint64_t da = ptx::make_smem_desc(ptx::smem_u32(sA + (size_t)s * p.a_stage_bytes), 16, p.sbo, p.umma_swizzle);
+                    const uint64_t db = ptx::make_smem_desc(ptx::smem_u32(sB + (size_t)s * p.b_stage_bytes), 16, p.sbo, p.umma_swizzle);
+                    for (int k = 0; k < p.KC / 16; ++k)
+                        ptx::umma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), p.idesc, (kb | k) ? 1u : 0u);
+                    ptx::umma_commit(empty + s);
+                    if (++s == p.stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                ptx::umma_commit(tfull + acc);
+                acc ^= 1;
+                if (acc == 0) acc_ph ^= 1u;
+            }
+            // Make sure every MMA issued by this thread has retired before TMEM is released.
+            ptx::umma_commit(drain);
+            for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (128 threads)
+        const int et = threadIdx.x - 64;        // 0..127
+        const int lane_group = warp & 3;        // TMEM lanes this warp may read
+        const int row = lane_group * 32 + lane; // accumulator row == tile row
+        const int ew = warp - 2;                // 0..3
+        int acc = 0, sat = 0;
+        uint32_t acc_ph = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
+            const long long m0 = (long long)m_tile * TC_BM;
+            bool ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
+            ok = epi_bar_and(ok);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(acc * p.acc_stride);
+            uint8_t* my_row = stg + (size_t)row * pitch;
+            for (int c0 = 0; c0 < p.BN; c0 += 16) {
+                uint32_t r[16];
+                ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)c0, r);
+                ptx::tmem_ld_wait();
+                uint4 v0, v1;
+                v0.x = pack2<OutT>(__uint_as_float(r[0]), __uint_as_float(r[1]), &sat);
+                v0.y = pack2<OutT>(__uint_as_float(r[2]), __uint_as_float(r[3]), &sat);
+                v0.z = pack2<OutT>(__uint_as_float(r[4]), __uint_as_float(r[5]), &sat);
+                v0.w = pack2<OutT>(__uint_as_float(r[6]), __uint_as_float(r[7]), &sat);
+                v1.x = pack2<OutT>(__uint_as_float(r[8]), __uint_as_float(r[9]), &sat);
+                v1.y = pack2<OutT>(__uint_as_float(r[10]), __uint_as_float(r[11]), &sat);
+                v1.z = pack2<OutT>(__uint_as_float(r[12]), __uint_as_float(r[13]), &sat);
+                v1.w = pack2<OutT>(__uint_as_float(r[14]), __uint_as_float(r[15]), &sat);
+                *reinterpret_cast<uint4*>(my_row + c0 * 2) = v0;
+                *reinterpret_cast<uint4*>(my_row + c0 * 2 + 16) = v1;
+            }
+            // accumulator buffer is free for the MMA of the tile after next
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(tempty + acc);
+            epi_bar_sync();  // staging tile complete
+            if (STATS) {
+                // warp ew sums rows [32*ew, 32*ew+32) of every channel pair; rows past M hold zeros
+                for (int pc = lane; pc < p.BN / 2; pc += 32) {
+                    float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
+                    const uint8_t* col = stg + (size_t)(ew * 32) * pitch + pc * 4;
+#pragma unroll 8
+                    for (int rr = 0; rr < 32; ++rr) {
+                        const uint32_t u = *reinterpret_cast<const uint32_t*>(col + (size_t)rr * pitch);
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u));
+                        s0 += f.x;
+                        s1 += f.y;
+                        q0 = fmaf(f.x, f.x, q0);
+                        q1 = fmaf(f.y, f.y, q1);
+                    }
+                    wpart[(ew * 2 + 0) * p.BN + 2 * pc] = s0;
+                    wpart[(ew * 2 + 0) * p.BN + 2 * pc + 1] = s1;
+                    wpart[(ew * 2 + 1) * p.BN + 2 * pc] = q0;
+                    wpart[(ew * 2 + 1) * p.BN + 2 * pc + 1] = q1;
+                }
+            }
+            // coalesced row stores: consecutive threads write consecutive 16-byte pieces of a pixel's channel slice
+            {
+                const int cpr = p.BN / 8;  // 16-byte chunks per row
+                const int total = TC_BM * cpr;
+                uint8_t* outb = static_cast<uint8_t*>(p.out);
+                for (int chn = et; chn < total; chn += 128) {
+                    const int rr = chn / cpr, cc = chn - rr * cpr;
+                    const long long m = m0 + rr;
+                    if (m >= p.M) break;
+                    long long pix = m;
+                    if (p.os != 1) {
+                        const int j = (int)(m % p.Wq);
+                        const long long t1 = m / p.Wq;
+                        const int i = (int)(t1 % p.Hq);
+                        const long long n = t1 / p.Hq;
+                        pix = (n * p.Hout + (long long)i * p.os + p.oa) * p.Wout + (long long)j * p.os + p.ob;
+                    }
+                    const uint4 v = *reinterpret_cast<const uint4*>(stg + (size_t)rr * pitch + cc * 16);
+                    *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN) * 2 + (size_t)cc * 16) = v;
+                }
+            }
+            epi_bar_sync();  // staging tile and wpart fully consumed / produced
+            if (STATS) {
+                for (int c = et; c < p.BN; c += 128) {
+                    float s = 0.f, q = 0.f;
+#pragma unroll
+                    for (int w4 = 0; w4 < 4; ++w4) {
+                        s += wpart[(w4 * 2 + 0) * p.BN + c];
+                        q += wpart[(w4 * 2 + 1) * p.BN + c];
+                    }
+                    stat_sum[n_tile * p.BN + c] += s;
+                    stat_sq[n_tile * p.BN + c] += q;
+                }
+            }
+            acc ^= 1;
+            if (acc == 0) acc_ph ^= 1u;
+        }
+        if (STATS) {
+            epi_bar_sync();
+            float* dst = p.partials + (size_t)blockIdx.x * 2 * p.ldo;
+            for (int c = et; c < 2 * p.ldo; c += 128) dst[c] = stat_sum[c];
+        }
+        if (sat) atomicAdd(p.status + ST_SAT, sat);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+// Rearranged filter for dgrad: for parity class `cls` (a list of taps), wt[c][ti][c'] = w[c'][r_ti][t_ti][c].
+struct WtClass {
+    int ntaps;
+    int r[9], t[9];
+    size_t offset;  // element offset of this class's matrix in the output buffer
+};
+struct WtParams {
+    int c_in, c_out, k, nclasses;
+    WtClass cls[4];
+};
+__global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
+    // one thread per output element, output-contiguous (c' fastest)
+    size_t total = (size_t)P.c_in * P.k * P.k * P.c_out;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        int cls = 0;
+        while (cls + 1 < P.nclasses && e >= P.cls[cls + 1].offset) ++cls;
+        const WtClass& C = P.cls[cls];
+        size_t le = e - C.offset;
+        const int co = (int)(le % P.c_out);
+        le /= P.c_out;
+        const int ti = (int)(le % C.ntaps);
+        const int c = (int)(le / C.ntaps);
+        wt[e] = w[(((size_t)co * P.k + C.r[ti]) * P.k + C.t[ti]) * P.c_in + c];
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+struct IgemmCfg {
+    bool ok = false;
+    int Ca = 0, rowsB = 0, ntaps = 0;
+    int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0;
+    uint32_t a_stage = 0, b_stage = 0;
+    size_t smem_bytes = 0;
+    long long M = 0;
+};
+
+struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded for the pointers last seen
+    IgemmCfg cfg;
+    IgemmParams prm;
+    const void* a_ptr = nullptr;
+    const void* b_ptr = nullptr;
+};
+
+struct TcPlan {
+    bool fprop = false, dgrad = false, wgrad = false;
+    int fprop_parts = 0;
+    size_t wt_bytes = 0;
+    size_t wgrad_partial_bytes = 0;
+    int sm_count = 0;
+    long long launches = 0;  // kernels launched through this record
+    TcGemmSlot fp;
+    int dg_classes = 0;
+    TcGemmSlot dg[4];
+    WtParams wtp;
+};
+
+namespace tcdetail {
+
+inline std::string& err() {
+    static thread_local std::string e;
+    return e;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const int*, const int*,
+                                   cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+struct DriverFns {
+    EncodeTiledFn tiled = nullptr;
+    EncodeIm2colFn im2col = nullptr;
+    bool tried = false;
+};
+inline DriverFns& driver() {
+    static DriverFns d;
+    if (!d.tried) {
+        d.tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            d.tiled = reinterpret_cast<EncodeTiledFn>(f);
+        f = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            d.im2col = reinterpret_cast<EncodeIm2colFn>(f);
+    }
+    return d;
+}
+
+inline CUtensorMapSwizzle tma_swizzle_for(int KC) {
+    return KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : KC == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+}
+inline uint32_t umma_swizzle_for(int KC) { return KC == 64 ? (uint32_t)ptx::kSwizzle128 : KC == 32 ? (uint32_t)ptx::kSwizzle64 : (uint32_t)ptx::kSwizzle32; }
+
+constexpr size_t kMaxSmem = 232448;  // 227 KB opt-in limit per CTA
+
+// Tile configuration for a GEMM with M rows, `rowsB` output channels, `ntaps` taps of `Ca` channels each.
+inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count) {
+    IgemmCfg c;
+    c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
+    if (Ca % 16 || rowsB % 16 || M < 1) return c;
+    c.KC = (Ca % 64 == 0) ? 64 : (Ca % 32 == 0) ? 32 : 16;
+    c.m_tiles = (int)((M + TC_BM - 1) / TC_BM);
+    const double ksteps = (double)ntaps * Ca / 16.0;
+    double best = 1e30;
+    for (int bn = 16; bn <= 256 && bn <= rowsB; bn += 16) {
+        if (rowsB % bn) continue;
+        const long long tiles = (long long)c.m_tiles * (rowsB / bn);
+        const double waves = (double)((tiles + sm_count - 1) / sm_count);
+        const double per_tile = ksteps * std::max(bn, 32) / 2.0 + 400.0 + 6.0 * bn;
+        const double cost = waves * per_tile;
+        if (cost < best - 1e-9) {
+            best = cost;
+            c.BN = bn;
+        }
+    }
+    if (!c.BN) return c;
+    c.n_tiles = rowsB / c.BN;
+    c.acc_stride = c.BN <= 32 ? 32 : c.BN <= 64 ? 64 : c.BN <= 128 ? 128 : 256;
+    c.tmem_cols = 2 * c.acc_stride;
+    c.a_stage = (uint32_t)((TC_BM * c.KC * 2 + 1023) / 1024 * 1024);
+    c.b_stage = (uint32_t)((c.BN * c.KC * 2 + 1023) / 1024 * 1024);
+    const size_t fixed = 1024 /*alignment slack*/ + (size_t)TC_BM * (c.BN * 2 + 16) + (size_t)2 * ldo * 4 + (size_t)8 * c.BN * 4 + 512;
+    if (fixed + 2 * (size_t)(c.a_stage + c.b_stage) > kMaxSmem) return c;
+    c.stages = (int)std::min<size_t>(8, (kMaxSmem - fixed) / (c.a_stage + c.b_stage));
+    c.stages = std::max(2, std::min(c.stages, std::max(2, ntaps * (Ca / c.KC))));
+    c.smem_bytes = std::max<size_t>(fixed + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
+    c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count);
+    c.ok = true;
+    return c;
+}
+
+inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
+    P.M = c.M;
+    P.ntaps = c.ntaps;
+    P.Ca = c.Ca; P.KC = c.KC; P.kc_per_tap = c.Ca / c.KC;
+    P.BN = c.BN; P.n_tiles = c.n_tiles; P.m_tiles = c.m_tiles;
+    P.stages = c.stages; P.acc_stride = c.acc_stride; P.tmem_cols = c.tmem_cols;
+    P.umma_swizzle = umma_swizzle_for(c.KC);
+    P.sbo = (uint32_t)(8 * c.KC * 2);
+    P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
+    P.idesc = ptx::make_idesc_bf16(TC_BM, c.BN, 0, 0);
+}
+
+// im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
+inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W, int C, int lo, int up, int ts, int KC) {
+    DriverFns& d = driver();
+    if (!d.im2col) { err() = "cuTensorMapEncodeIm2col is not available from the driver"; return false; }
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    int lower[2] = {lo, lo}, upper[2] = {up, up};
+    cuuint32_t estr[4] = {1, (cuuint32_t)ts, (cuuint32_t)ts, 1};
+    CUresult r = d.im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower, upper, (cuuint32_t)KC, TC_BM, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, tma_swizzle_for(KC), CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeIm2col failed with code " + std::to_string((int)r); return false; }
+    return true;
+}
+
+// tiled map over a bf16 matrix [rows][cols] (cols contiguous), box = KC columns x box_rows rows.
+inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, long long cols, int KC, int box_rows) {
+    DriverFns& d = driver();
+    if (!d.tiled) { err() = "cuTensorMapEncodeTiled is not available from the driver"; return false; }
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)KC, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = d.tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         tma_swizzle_for(KC), CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return false; }
+    return true;
+}
+
+template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+            err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
+            return NB_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    tc_igemm_kernel<OutT, STATS><<<s.cfg.grid, TC_THREADS, s.cfg.smem_bytes, st>>>(s.prm);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
+        return NB_ERR_CUDA;
+    }
     return NB_OK;
 }
-inline nb_status tc_fprop(TcPlan*, const Geom&, const void*, const void*, void*, float*, int*, cudaStream_t) { return NB_ERR_INTERNAL; }
-inline nb_status tc_dgrad(TcPlan*, const Geom&, const void*, const void*, void*, void*, int*, cudaStream_t) { return NB_ERR_INTERNAL; }
-inline nb_status tc_wgrad(TcPlan*, const Geom&, const void*, const void*, float*, float*, int*, cudaStream_t) { return NB_ERR_INTERNAL; }
+
+}  // namespace tcdetail
+
+inline const char* tc_last_error() { return tcdetail::err().c_str(); }
+
+// Decide which convolutions of this shape run on the tensor-core kernels and size their scratch.
+inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&) {
+    using namespace tcdetail;
+    *tc = TcPlan();
+    tc->sm_count = sm_count;
+    if (!enable) return NB_OK;
+    DriverFns& d = driver();
+    if (!d.tiled || !d.im2col) return NB_OK;  // no TMA descriptors from this driver: stay on the CUDA-core kernels
+    const bool even = (g.h % 2 == 0) && (g.w % 2 == 0);
+    // ---- fprop: A = x (im2col), B = w [Cout][k*k*Cin]
+    if (g.c_in % 16 == 0 && g.c_out % 16 == 0) {
+        IgemmCfg c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count);
+        if (c.ok) {
+            tc->fp.cfg = c;
+            IgemmParams& P = tc->fp.prm;
+            memset(&P, 0, sizeof P);
+            fill_params(P, c);
+            P.Hq = g.ho; P.Wq = g.wo; P.ts = g.stride; P.lo_w = -g.pad; P.lo_h = -g.pad;
+            for (int r = 0; r < g.k; ++r)
+                for (int t = 0; t < g.k; ++t) {
+                    P.off_h[r * g.k + t] = (uint16_t)r;
+                    P.off_w[r * g.k + t] = (uint16_t)t;
+                }
+            P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1; P.oa = 0; P.ob = 0;
+            tc->fprop = true;
+            tc->fprop_parts = c.grid;
+        }
+    }
+    // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four parity classes
+    if (g.c_in % 16 == 0 && g.c_out % 16 == 0 && (g.stride == 1 || (g.k == 3 && even))) {
+        WtParams& W = tc->wtp;
+        memset(&W, 0, sizeof W);
+        W.c_in = g.c_in; W.c_out = g.c_out; W.k = g.k;
+        bool ok = true;
+        size_t off = 0;
+        const int ncls = g.stride == 1 ? 1 : 4;
+        for (int cls = 0; cls < ncls && ok; ++cls) {
+            const int pa = cls / 2, pb = cls % 2;  // output row / column parity (stride 2)
+            TcGemmSlot& S = tc->dg[cls];
+            IgemmParams& P = S.prm;
+            memset(&P, 0, sizeof P);
+            WtClass& C = W.cls[cls];
+            C.offset = off;
+            int nt = 0;
+            if (g.stride == 1) {
+                // dx[h][w] = sum_{r,t} dy[h+P-r][w+P-t] w[r][t]: traversal from -(k-1-P) with offsets r' = k-1-r
+                for (int ro = 0; ro < g.k; ++ro)
+                    for (int to = 0; to < g.k; ++to) {
+                        P.off_h[nt] = (uint16_t)ro; P.off_w[nt] = (uint16_t)to;
+                        C.r[nt] = g.k - 1 - ro; C.t[nt] = g.k - 1 - to;
+                        ++nt;
+                    }
+                P.Hq = g.h; P.Wq = g.w; P.ts = 1; P.lo_w = P.lo_h = -(g.k - 1 - g.pad);
+                P.Hout = g.h; P.Wout = g.w; P.os = 1; P.oa = 0; P.ob = 0;
+            } else {
+                // dx[2i+pa][2j+pb]: rows with pa=0 see tap r=1 at dy row i; pa=1 sees r=0 at dy row i+1 and r=2 at dy row i
+                int rs[2], ro[2], nr = 0, tsv[2], to[2], ntc = 0;
+                if (pa == 0) { rs[0] = 1; ro[0] = 0; nr = 1; } else { rs[0] = 2; ro[0] = 0; rs[1] = 0; ro[1] = 1; nr = 2; }
+                if (pb == 0) { tsv[0] = 1; to[0] = 0; ntc = 1; } else { tsv[0] = 2; to[0] = 0; tsv[1] = 0; to[1] = 1; ntc = 2; }
+                for (int a = 0; a < nr; ++a)
+                    for (int b = 0; b < ntc; ++b) {
+                        P.off_h[nt] = (uint16_t)ro[a]; P.off_w[nt] = (uint16_t)to[b];
+                        C.r[nt] = rs[a]; C.t[nt] = tsv[b];
+                        ++nt;
+                    }
+                P.Hq = g.h / 2; P.Wq = g.w / 2; P.ts = 1; P.lo_w = P.lo_h = 0;
+                P.Hout = g.h; P.Wout = g.w; P.os = 2; P.oa = pa; P.ob = pb;
+            }
+            C.ntaps = nt;
+            off += (size_t)g.c_in * nt * g.c_out;
+            IgemmCfg c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, nt, g.c_in, sm_count);
+            if (!c.ok) { ok = false; break; }
+            S.cfg = c;
+            fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
+            P.ldo = g.c_in;
+        }
+        if (ok) {
+            W.nclasses = ncls;
+            tc->dg_classes = ncls;
+            tc->wt_bytes = off * 2;
+            tc->dgrad = true;
+        }
+    }
+    return NB_OK;
+}
+
+inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st) {
+    using namespace tcdetail;
+    TcGemmSlot& S = tc->fp;
+    if (S.a_ptr != x || S.b_ptr != w) {
+        const int up = g.pad - (g.k - 1);
+        if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC)) return NB_ERR_CUDA;
+        if (!encode_tiled_2d(&S.prm.tmB, w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
+        S.a_ptr = x; S.b_ptr = w;
+    }
+    S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
+    tc->launches += 1;
+    return launch_igemm<__half, true>(S, st);
+}
+
+inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void* w, void* dx, void* wt, int* status, cudaStream_t st) {
+    using namespace tcdetail;
+    {
+        const size_t total = tc->wt_bytes / 2;
+        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)tc->sm_count * 8);
+        dgrad_weight_transform_kernel<<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), tc->wtp);
+        if (cudaGetLastError() != cudaSuccess) { err() = "launch of dgrad_weight_transform_kernel failed"; return NB_ERR_CUDA; }
+        tc->launches += 1;
+    }
+    for (int cls = 0; cls < tc->dg_classes; ++cls) {
+        TcGemmSlot& S = tc->dg[cls];
+        const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
+        if (S.a_ptr != dy || S.b_ptr != wcls) {
+            // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
+            const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
+            const int up = lo;
+            if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, up, 1, S.cfg.KC)) return NB_ERR_CUDA;
+            if (!encode_tiled_2d(&S.prm.tmB, wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
+            S.a_ptr = dy; S.b_ptr = wcls;
+        }
+        S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
+        nb_status r = launch_igemm<__nv_bfloat16, false>(S, st);
+        if (r != NB_OK) return r;
+        tc->launches += 1;
+    }
+    return NB_OK;
+}
+
+inline nb_status tc_wgrad(TcPlan*, const Geom&, const void*, const void*, float*, float*, int*, cudaStream_t) {
+    tcdetail::err() = "tensor-core wgrad is not available";
+    return NB_ERR_INTERNAL;
+}
 
 }  // namespace nbcbs
