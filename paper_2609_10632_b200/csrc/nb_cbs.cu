@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "simt_conv.cuh"
+#include "stem_conv.cuh"
 #include "tc_conv.cuh"
 
 using namespace nbcbs;
@@ -67,6 +68,8 @@ struct nb_cbs_plan_s {
     int wg_splits;   // split-K slices of the CUDA-core wgrad
     long long wg_chunk;
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
+    bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
+    int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     double prof_ms[SITE_COUNT] = {};
@@ -318,6 +321,9 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
         return fail(NB_ERR_CUDA, "status block allocation failed: %s", cudaGetErrorString(ce));
     }
 
+    p->stem = d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
+              g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0;
+    p->stem_blocks = (int)std::min<long long>((g.m + 255) / 256, (long long)p->sm_count * 8);
     p->nparts = std::max(e.blocks_reduce, p->tc.fprop_parts);
     const size_t C = (size_t)g.c_out;
     size_t off = 0;
@@ -332,7 +338,8 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->off_wgpart = off;
     {
         size_t simt = p->wg_splits > 1 ? (size_t)p->wg_splits * C * g.kdim * 4 : 0;
-        off = align_up(off + std::max(simt, p->tc.wgrad_partial_bytes), 256);
+        size_t stem = p->stem ? (size_t)p->stem_blocks * C * g.kdim * 4 : 0;
+        off = align_up(off + std::max(std::max(simt, stem), p->tc.wgrad_partial_bytes), 256);
     }
     p->bwd_bytes = off;
     *out = p;
@@ -445,6 +452,15 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
+    } else if (p->stem) {
+        {
+            SiteTimer tm(p, SITE_FPROP, st);
+            const int blocks = (int)std::min<long long>((p->g.m + 127) / 128, (long long)p->sm_count * 16);
+            stem_fprop_kernel<48><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
+                                                         static_cast<__half*>(y_saved), p->g);
+            NB_LAUNCH_OK("stem_fprop");
+        }
+        NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
@@ -498,6 +514,14 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     }
     NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st)));
     if (!dx) return NB_OK;
+    if (p->stem) {
+        SiteTimer tm(p, SITE_DGRAD, st);
+        const long long total = (long long)p->g.n * p->g.h * (p->g.w / 2);
+        const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
+        stem_dgrad_kernel<48><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
+                                                     static_cast<__nv_bfloat16*>(dx), p->g);
+        return launch_ok("stem_dgrad");
+    }
     if (p->tc.dgrad) {
         SiteTimer tm(p, SITE_DGRAD, st);
         const long long l0 = p->tc.launches;
@@ -518,6 +542,19 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_wgpart);
     if (is_f32(p)) return run_simt_wgrad<float>(p, x, dy, dw, partial, st);
+    if (p->stem) {
+        {
+            SiteTimer tm(p, SITE_WGRAD, st);
+            const long long per = (p->g.m + p->stem_blocks - 1) / p->stem_blocks;
+            stem_wgrad_kernel<48><<<p->stem_blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
+                                                                 partial, p->g, per);
+            NB_LAUNCH_OK("stem_wgrad");
+        }
+        const size_t elems = (size_t)p->g.c_out * p->g.kdim;
+        SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
+        splitk_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, p->stem_blocks, elems, dw);
+        return launch_ok("splitk_reduce");
+    }
     if (p->tc.wgrad) {
         SiteTimer tm(p, SITE_WGRAD, st);
         const long long l0 = p->tc.launches;

@@ -14,6 +14,7 @@
 #include "../../include/nb_cbs.h"
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "simt_conv.cuh"
 
 namespace nbcbs {
 
@@ -367,6 +368,10 @@ __global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ 
     }
 }
 
+}  // namespace nbcbs
+#include "tc_wgrad.cuh"
+namespace nbcbs {
+
 // ------------------------------------------------------------------------------------------ host side
 struct IgemmCfg {
     bool ok = false;
@@ -395,6 +400,12 @@ struct TcPlan {
     int dg_classes = 0;
     TcGemmSlot dg[4];
     WtParams wtp;
+    // wgrad
+    WgradParams wg;
+    int wg_grid = 0;
+    size_t wg_smem = 0;
+    const void* wg_a_ptr = nullptr;
+    const void* wg_b_ptr = nullptr;
 };
 
 namespace tcdetail {
@@ -486,14 +497,14 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
 }
 
 // im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
-inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W, int C, int lo, int up, int ts, int KC) {
+inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W, int C, int lo, int up, int ts, int KC, int pixels = TC_BM) {
     DriverFns& d = driver();
     if (!d.im2col) { err() = "cuTensorMapEncodeIm2col is not available from the driver"; return false; }
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
     int lower[2] = {lo, lo}, upper[2] = {up, up};
     cuuint32_t estr[4] = {1, (cuuint32_t)ts, (cuuint32_t)ts, 1};
-    CUresult r = d.im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower, upper, (cuuint32_t)KC, TC_BM, estr,
+    CUresult r = d.im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower, upper, (cuuint32_t)KC, (cuuint32_t)pixels, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, tma_swizzle_for(KC), CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeIm2col failed with code " + std::to_string((int)r); return false; }
     return true;
@@ -618,6 +629,53 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
             tc->dgrad = true;
         }
     }
+    // ---- wgrad: A = x (im2col, MN-major), B = dy (MN-major), reduction over pixels with split-K
+    if (g.c_in % 16 == 0 && g.c_out % 16 == 0) {
+        WgradParams& P = tc->wg;
+        memset(&P, 0, sizeof P);
+        P.M = g.m; P.Hq = g.ho; P.Wq = g.wo; P.ts = g.stride; P.lo_w = P.lo_h = -g.pad;
+        P.c_in = g.c_in; P.c_out = g.c_out; P.kdim = g.kdim;
+        for (int r = 0; r < g.k; ++r)
+            for (int t = 0; t < g.k; ++t) {
+                P.off_h[r * g.k + t] = (uint16_t)r;
+                P.off_w[r * g.k + t] = (uint16_t)t;
+            }
+        P.KCA = (g.c_in % 64 == 0) ? 64 : (g.c_in % 32 == 0) ? 32 : 16;
+        P.nblkA = 128 / P.KCA;
+        P.cblk_per_tap = g.c_in / P.KCA;
+        P.m_tiles = (g.kdim + 127) / 128;
+        double best = 1e30;
+        for (int bn = 16; bn <= 256 && bn <= g.c_out; bn += 16) {
+            if (g.c_out % bn) continue;
+            const double cost = (double)(g.c_out / bn) * (std::max(bn, 64) + 16);
+            if (cost < best - 1e-9 || (cost < best + 1e-9 && bn > P.BN)) {
+                best = cost;
+                P.BN = bn;
+            }
+        }
+        P.n_tiles = g.c_out / P.BN;
+        P.KCB = (P.BN % 64 == 0) ? 64 : (P.BN % 32 == 0) ? 32 : 16;
+        P.nblkB = P.BN / P.KCB;
+        P.total_chunks = (int)((g.m + WG_KP - 1) / WG_KP);
+        const int tiles = P.m_tiles * P.n_tiles;
+        int splits = std::max(1, (sm_count + tiles / 2) / tiles);
+        splits = std::min(splits, std::max(1, P.total_chunks / 8));
+        P.chunks_per_split = (P.total_chunks + splits - 1) / splits;
+        P.splits = (P.total_chunks + P.chunks_per_split - 1) / P.chunks_per_split;
+        P.a_stage_bytes = 128 * WG_KP * 2;
+        P.b_stage_bytes = (uint32_t)((P.BN * WG_KP * 2 + 1023) / 1024 * 1024);
+        P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
+        P.stages = std::max(2, std::min(P.stages, std::max(2, P.chunks_per_split)));
+        P.tmem_cols = P.BN <= 32 ? 32 : P.BN <= 64 ? 64 : P.BN <= 128 ? 128 : 256;
+        P.swzA = umma_swizzle_for(P.KCA); P.swzB = umma_swizzle_for(P.KCB);
+        P.sboA = (uint32_t)(8 * P.KCA * 2); P.sboB = (uint32_t)(8 * P.KCB * 2);
+        P.lboA = (uint32_t)(WG_KP * P.KCA * 2); P.lboB = (uint32_t)(WG_KP * P.KCB * 2);
+        P.idesc = ptx::make_idesc_bf16(128, P.BN, 1, 1);
+        tc->wg_smem = std::max<size_t>(2048 + (size_t)P.stages * (P.a_stage_bytes + P.b_stage_bytes), 120 * 1024);
+        tc->wg_grid = tiles * P.splits;
+        tc->wgrad_partial_bytes = P.splits > 1 ? (size_t)P.splits * g.c_out * g.kdim * 4 : 0;
+        tc->wgrad = true;
+    }
     return NB_OK;
 }
 
@@ -663,9 +721,37 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
     return NB_OK;
 }
 
-inline nb_status tc_wgrad(TcPlan*, const Geom&, const void*, const void*, float*, float*, int*, cudaStream_t) {
-    tcdetail::err() = "tensor-core wgrad is not available";
-    return NB_ERR_INTERNAL;
+inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* dy, float* dw, float* partial, int* status, cudaStream_t st) {
+    using namespace tcdetail;
+    WgradParams& P = tc->wg;
+    if (tc->wg_a_ptr != x || tc->wg_b_ptr != dy) {
+        const int up = g.pad - (g.k - 1);
+        if (!encode_im2col(&P.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, P.KCA, WG_KP)) return NB_ERR_CUDA;
+        if (!encode_tiled_2d(&P.tmB, dy, g.m, g.c_out, P.KCB, WG_KP)) return NB_ERR_CUDA;
+        tc->wg_a_ptr = x; tc->wg_b_ptr = dy;
+    }
+    P.out = P.splits > 1 ? partial : dw;
+    P.status = status;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+            err() = "cannot raise the dynamic shared memory limit of the wgrad kernel";
+            return NB_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    tc_wgrad_kernel<<<tc->wg_grid, TC_THREADS, tc->wg_smem, st>>>(P);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { err() = std::string("launch of tc_wgrad_kernel failed: ") + cudaGetErrorString(e); return NB_ERR_CUDA; }
+    tc->launches += 1;
+    if (P.splits > 1) {
+        const size_t elems = (size_t)g.c_out * g.kdim;
+        const int blocks = (int)std::min<size_t>((elems + 255) / 256, (size_t)tc->sm_count * 8);
+        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, P.splits, elems, dw);
+        if (cudaGetLastError() != cudaSuccess) { err() = "launch of splitk_reduce_kernel failed"; return NB_ERR_CUDA; }
+        tc->launches += 1;
+    }
+    return NB_OK;
 }
 
 }  // namespace nbcbs
