@@ -8,6 +8,8 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 
@@ -28,19 +30,32 @@ struct IgemmParams {
     int lo_w, lo_h;   // input coordinate of grid position 0 for tap offset 0
     int ntaps;
     int Ca, KC, kc_per_tap;
+    int kpb;                     // k-blocks (of KC channels) per pipeline stage
+    uint32_t a_sub_bytes, b_sub_bytes;  // bytes of one k-block of A / B inside a stage
     int BN, n_tiles, m_tiles;
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
+    int variant;                 // experiment switches
+    int a_tiled;                 // 1: A is a plain [M][Ca] matrix fetched with a tiled 2-D map (1x1 stride-1 convolutions)
     int ldo;                     // channels per output pixel
     int Hout, Wout, os, oa, ob;  // GEMM row (n,i,j) -> output pixel (n, i*os+oa, j*os+ob) of an Hout x Wout image
     void* out;
+    long long* dbg;   // optional [gridDim.x][8] cycle counters (only read when built with NB_TC_DEBUG_TIMING)
     float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
     int* status;
     uint16_t off_w[9], off_h[9];
 };
 
+#ifdef NB_TC_DEBUG_TIMING
+#define NB_DBG_T0() const long long dbg_t0__ = clock64()
+#define NB_DBG_ADD(var) var += clock64() - dbg_t0__
+#else
+#define NB_DBG_T0()
+#define NB_DBG_ADD(var)
+#endif
 constexpr int TC_BM = 128;
-constexpr int TC_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
+constexpr int TC_THREADS = 224;  // warp 0: TMA producer for A, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue, warp 6: TMA producer for B
+constexpr int WG_THREADS = 192;  // wgrad kernel: warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
@@ -68,6 +83,12 @@ __device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile i
             }
         }
     }
+}
+
+// Fast path inline (the barrier is usually complete already), slow bounded path out of line.
+__device__ __forceinline__ bool wait_bar_fast(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    return wait_bar(bar, parity, abort_flag, status, site);
 }
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -112,8 +133,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     const int pitch = p.BN * 2 + 16;
     float* stat_sum = reinterpret_cast<float*>(stg + (size_t)TC_BM * pitch);  // [ldo]
     float* stat_sq = stat_sum + p.ldo;                                        // [ldo]
-    float* wpart = stat_sq + p.ldo;                                           // [4][2][BN]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + 8 * p.BN);
+    float* wpart = stat_sq + p.ldo;                                           // [2 tile parities][4 warps][2][BN]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + 16 * p.BN);
     uint64_t* full = bars;                // [stages]
     uint64_t* empty = bars + p.stages;    // [stages]
     uint64_t* tfull = empty + p.stages;   // [2]
@@ -128,7 +149,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(full + s, 2);  // the A producer and the B producer each arrive once (with their byte counts)
             ptx::mbar_init(empty + s, 1);
         }
         ptx::mbar_init(tfull, 1);
@@ -151,41 +172,77 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (one thread)
+    if (warp == 0 || warp == 6) {
+        // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
         if (lane == 0) {
-            ptx::prefetch_tmap(&p.tmA);
-            ptx::prefetch_tmap(&p.tmB);
+            const bool isA = warp == 0;
+            ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
             int s = 0;
             uint32_t ph = 0;
             long long issued = 0;
             bool ok = true;
-            const uint32_t tx_bytes = (uint32_t)(TC_BM * p.KC * 2 + p.BN * p.KC * 2);
+#ifdef NB_TC_DEBUG_TIMING
+            long long dbg_wait_empty = 0;
+            const long long dbg_start = clock64();
+#endif
+            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * p.KC * 2) : (uint32_t)(p.BN * p.KC * 2);
+            // loop-invariant values in registers: this thread's instruction stream is on the critical path
+            const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
+            const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
+            const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes, sub_bytes = isA ? p.a_sub_bytes : p.b_sub_bytes;
+            const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB), full_u32 = ptx::smem_u32(full);
+            const CUtensorMap* tm = isA ? &p.tmA : &p.tmB;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
-                const long long m0 = (long long)m_tile * TC_BM;
-                const int j0 = (int)(m0 % p.Wq);
-                const long long t1 = m0 / p.Wq;
-                const int i0 = (int)(t1 % p.Hq), n0 = (int)(t1 / p.Hq);
-                const int cw = p.lo_w + j0 * p.ts, ch = p.lo_h + i0 * p.ts;
-                for (int tap = 0; ok && tap < p.ntaps; ++tap) {
-                    for (int kc = 0; kc < p.kc_per_tap; ++kc) {
-                        if (!wait_bar(empty + s, ph ^ 1u, abort_flag, p.status, 1)) {
+                const int m_tile = tile / n_tiles, n_tile = tile - m_tile * n_tiles;
+                const int m0 = m_tile * TC_BM;
+                int cw = 0, ch = 0, n0 = 0;
+                if (isA && !a_tiled) {
+                    const int j0 = m0 % Wq, t1 = m0 / Wq;
+                    const int i0 = t1 % Hq;
+                    n0 = t1 / Hq;
+                    cw = p.lo_w + j0 * ts;
+                    ch = p.lo_h + i0 * ts;
+                }
+                const int brow = n_tile * BN;
+                int tap = 0, kc = 0;
+                for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
+                    const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
+                    {
+                        NB_DBG_T0();
+                        if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, isA ? 1 : 5)) {
                             ok = false;
                             break;
                         }
-                        ptx::mbar_expect_tx(full + s, tx_bytes);
-                        ptx::tma_load_im2col_4d(sA + (size_t)s * p.a_stage_bytes, &p.tmA, full + s, kc * p.KC, cw, ch, n0, p.off_w[tap],
-                                                p.off_h[tap]);
-                        ptx::tma_load_2d(sB + (size_t)s * p.b_stage_bytes, &p.tmB, full + s, tap * p.Ca + kc * p.KC, n_tile * p.BN);
-                        ++issued;
-                        if (++s == p.stages) {
-                            s = 0;
-                            ph ^= 1u;
+                        NB_DBG_ADD(dbg_wait_empty);
+                    }
+                    const uint32_t bar = full_u32 + 8u * (uint32_t)s;
+                    ptx::mbar_expect_tx_u32(bar, kb_bytes * (uint32_t)nkb);
+                    uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
+                    for (int j = 0; j < nkb; ++j) {
+                        if (isA) {
+                            if (a_tiled)
+                                ptx::tma_load_2d_u32(dst, tm, bar, kc * KC, m0);
+                            else
+                                ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[tap], p.off_h[tap]);
+                        } else {
+                            ptx::tma_load_2d_u32(dst, tm, bar, tap * Ca + kc * KC, brow);
                         }
+                        dst += sub_bytes;
+                        if (++kc == kc_per_tap) {
+                            kc = 0;
+                            ++tap;
+                        }
+                    }
+                    ++issued;
+                    if (++s == stages) {
+                        s = 0;
+                        ph ^= 1u;
                     }
                 }
             }
+#ifdef NB_TC_DEBUG_TIMING
+            if (p.dbg && isA) { p.dbg[blockIdx.x * 8 + 0] = dbg_wait_empty; p.dbg[blockIdx.x * 8 + 1] = clock64() - dbg_start; }
+#endif
             if (!ok) {
                 // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
                 const int back = issued < (long long)p.stages ? (int)issued : p.stages;
@@ -203,24 +260,60 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
+#ifdef NB_TC_DEBUG_TIMING
+            long long dbg_wait_full = 0, dbg_wait_tempty = 0;
+            const long long dbg_start = clock64();
+#endif
+            const int ksteps = p.KC / 16, kpb = p.kpb, stages = p.stages;
+            const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
+            const uint64_t a_sub16 = (uint64_t)(p.a_sub_bytes >> 4), b_sub16 = (uint64_t)(p.b_sub_bytes >> 4);
+            const uint64_t a_stage16 = (uint64_t)(p.a_stage_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
+            const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), 16, p.sbo, p.umma_swizzle);
+            const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, p.sbo, p.umma_swizzle);
+            const uint32_t empty_u32 = ptx::smem_u32(empty);
+            uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                if (!wait_bar(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
+                {
+                    NB_DBG_T0();
+                    if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
+                    NB_DBG_ADD(dbg_wait_tempty);
+                }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.acc_stride);
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!wait_bar(full + s, ph, abort_flag, p.status, 3)) {
-                        ok = false;
-                        break;
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_stride;
+                uint32_t accumulate = 0;
+                for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
+                    const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
+                    {
+                        NB_DBG_T0();
+                        if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
+                            ok = false;
+                            break;
+                        }
+                        NB_DBG_ADD(dbg_wait_full);
                     }
                     ptx::tc_fence_after();
-                    const uint64_t da = ptx::make_smem_desc(ptx::smem_u32(sA + (size_t)s * p.a_stage_bytes), 16, p.sbo, p.umma_swizzle);
-                    const uint64_t db = ptx::make_smem_desc(ptx::smem_u32(sB + (size_t)s * p.b_stage_bytes), 16, p.sbo, p.umma_swizzle);
-                    for (int k = 0; k < p.KC / 16; ++k)
-                        ptx::umma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), p.idesc, (kb | k) ? 1u : 0u);
-                    ptx::umma_commit(empty + s);
-                    if (++s == p.stages) {
+                    uint64_t da = da_s, db = db_s;
+                    for (int j = 0; j < nkb; ++j) {
+                        if (ksteps == 4) {
+                            ptx::umma_f16(d_tmem, da, db, idesc, accumulate);
+                            ptx::umma_f16(d_tmem, da + 2, db + 2, idesc, 1u);
+                            ptx::umma_f16(d_tmem, da + 4, db + 4, idesc, 1u);
+                            ptx::umma_f16(d_tmem, da + 6, db + 6, idesc, 1u);
+                        } else {
+                            for (int k = 0; k < ksteps; ++k) ptx::umma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (k | (int)accumulate) ? 1u : 0u);
+                        }
+                        accumulate = 1u;
+                        da += a_sub16;
+                        db += b_sub16;
+                    }
+                    ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
+                    da_s += a_stage16;
+                    db_s += b_stage16;
+                    if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
+                        da_s = da0;
+                        db_s = db0;
                     }
                 }
                 if (!ok) break;
@@ -228,53 +321,80 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                 acc ^= 1;
                 if (acc == 0) acc_ph ^= 1u;
             }
+#ifdef NB_TC_DEBUG_TIMING
+            if (p.dbg) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
+#endif
             // Make sure every MMA issued by this thread has retired before TMEM is released.
             ptx::umma_commit(drain);
             for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (128 threads)
-        const int et = threadIdx.x - 64;        // 0..127
-        const int lane_group = warp & 3;        // TMEM lanes this warp may read
-        const int row = lane_group * 32 + lane; // accumulator row == tile row
-        const int ew = warp - 2;                // 0..3
-        int acc = 0, sat = 0;
+        // ------------------------------------------------------------------ epilogue (warps 2-5, 128 threads)
+        const int et = threadIdx.x - 64;          // 0..127
+        const int lane_group = warp & 3;          // TMEM lanes this warp may read: rows [32*lane_group, +32) of the tile
+        const int row = lane_group * 32 + lane;   // accumulator row == tile row
+        const int cpr = p.BN / 8;                 // 16-byte chunks per staged row (<= 32)
+        const int rpi = 32 / cpr;                 // rows one warp stores per iteration
+        const int lr = lane / cpr, lc = lane - lr * cpr;
+        int acc = 0, sat = 0, par = 0;
         uint32_t acc_ph = 0;
+#ifdef NB_TC_DEBUG_TIMING
+        long long dbg_wait_tfull = 0;
+        const long long dbg_start = clock64();
+#endif
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
             const long long m0 = (long long)m_tile * TC_BM;
-            bool ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
+            NB_DBG_T0();
+            bool ok = true;
+            if (p.variant & 2) {
+                ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
+            } else {
+                // one poller per warp: 128 threads spinning on one mbarrier would crowd the shared-memory pipe
+                if (lane == 0) ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            }
+            NB_DBG_ADD(dbg_wait_tfull);
             ok = epi_bar_and(ok);
             if (!ok) break;
             ptx::tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(acc * p.acc_stride);
             uint8_t* my_row = stg + (size_t)row * pitch;
-            for (int c0 = 0; c0 < p.BN; c0 += 16) {
-                uint32_t r[16];
+            for (int c0 = 0; c0 < p.BN; c0 += 32) {
+                uint32_t r[32];
+                const bool two = c0 + 16 < p.BN;
                 ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)c0, r);
+                if (two) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(c0 + 16), r + 16);
                 ptx::tmem_ld_wait();
-                uint4 v0, v1;
-                v0.x = pack2<OutT>(__uint_as_float(r[0]), __uint_as_float(r[1]), &sat);
-                v0.y = pack2<OutT>(__uint_as_float(r[2]), __uint_as_float(r[3]), &sat);
-                v0.z = pack2<OutT>(__uint_as_float(r[4]), __uint_as_float(r[5]), &sat);
-                v0.w = pack2<OutT>(__uint_as_float(r[6]), __uint_as_float(r[7]), &sat);
-                v1.x = pack2<OutT>(__uint_as_float(r[8]), __uint_as_float(r[9]), &sat);
-                v1.y = pack2<OutT>(__uint_as_float(r[10]), __uint_as_float(r[11]), &sat);
-                v1.z = pack2<OutT>(__uint_as_float(r[12]), __uint_as_float(r[13]), &sat);
-                v1.w = pack2<OutT>(__uint_as_float(r[14]), __uint_as_float(r[15]), &sat);
-                *reinterpret_cast<uint4*>(my_row + c0 * 2) = v0;
-                *reinterpret_cast<uint4*>(my_row + c0 * 2 + 16) = v1;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && !two) break;
+                    uint4 v0, v1;
+                    const uint32_t* q = r + 16 * h;
+                    v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat);
+                    v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat);
+                    v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat);
+                    v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat);
+                    v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat);
+                    v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat);
+                    v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat);
+                    v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat);
+                    *reinterpret_cast<uint4*>(my_row + (c0 + 16 * h) * 2) = v0;
+                    *reinterpret_cast<uint4*>(my_row + (c0 + 16 * h) * 2 + 16) = v1;
+                }
             }
             // accumulator buffer is free for the MMA of the tile after next
             ptx::tc_fence_before();
             ptx::mbar_arrive(tempty + acc);
-            epi_bar_sync();  // staging tile complete
+            __syncwarp();  // every warp only reads back the 32 rows it staged itself
+            const uint8_t* my_rows = stg + (size_t)(lane_group * 32) * pitch;
             if (STATS) {
-                // warp ew sums rows [32*ew, 32*ew+32) of every channel pair; rows past M hold zeros
+                // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled)
+                float* wp = wpart + (size_t)((par * 4 + lane_group) * 2) * p.BN;
                 for (int pc = lane; pc < p.BN / 2; pc += 32) {
                     float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
-                    const uint8_t* col = stg + (size_t)(ew * 32) * pitch + pc * 4;
+                    const uint8_t* col = my_rows + pc * 4;
 #pragma unroll 8
                     for (int rr = 0; rr < 32; ++rr) {
                         const uint32_t u = *reinterpret_cast<const uint32_t*>(col + (size_t)rr * pitch);
@@ -284,20 +404,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         q0 = fmaf(f.x, f.x, q0);
                         q1 = fmaf(f.y, f.y, q1);
                     }
-                    wpart[(ew * 2 + 0) * p.BN + 2 * pc] = s0;
-                    wpart[(ew * 2 + 0) * p.BN + 2 * pc + 1] = s1;
-                    wpart[(ew * 2 + 1) * p.BN + 2 * pc] = q0;
-                    wpart[(ew * 2 + 1) * p.BN + 2 * pc + 1] = q1;
+                    wp[2 * pc] = s0;
+                    wp[2 * pc + 1] = s1;
+                    wp[p.BN + 2 * pc] = q0;
+                    wp[p.BN + 2 * pc + 1] = q1;
                 }
             }
-            // coalesced row stores: consecutive threads write consecutive 16-byte pieces of a pixel's channel slice
-            {
-                const int cpr = p.BN / 8;  // 16-byte chunks per row
-                const int total = TC_BM * cpr;
+            // coalesced row stores: the lanes of a warp cover whole rows of 16-byte pieces
+            if (lr < rpi) {
                 uint8_t* outb = static_cast<uint8_t*>(p.out);
-                for (int chn = et; chn < total; chn += 128) {
-                    const int rr = chn / cpr, cc = chn - rr * cpr;
-                    const long long m = m0 + rr;
+                for (int rr = lr; rr < 32; rr += rpi) {
+                    const long long m = m0 + lane_group * 32 + rr;
                     if (m >= p.M) break;
                     long long pix = m;
                     if (p.os != 1) {
@@ -307,22 +424,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         const long long n = t1 / p.Hq;
                         pix = (n * p.Hout + (long long)i * p.os + p.oa) * p.Wout + (long long)j * p.os + p.ob;
                     }
-                    const uint4 v = *reinterpret_cast<const uint4*>(stg + (size_t)rr * pitch + cc * 16);
-                    *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN) * 2 + (size_t)cc * 16) = v;
+                    const uint4 v = *reinterpret_cast<const uint4*>(my_rows + (size_t)rr * pitch + lc * 16);
+                    *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN) * 2 + (size_t)lc * 16) = v;
                 }
             }
-            epi_bar_sync();  // staging tile and wpart fully consumed / produced
             if (STATS) {
+                epi_bar_sync();  // all four warps' partial sums of this tile are in wpart[par]
+                const float* wp = wpart + (size_t)(par * 8) * p.BN;
                 for (int c = et; c < p.BN; c += 128) {
                     float s = 0.f, q = 0.f;
 #pragma unroll
                     for (int w4 = 0; w4 < 4; ++w4) {
-                        s += wpart[(w4 * 2 + 0) * p.BN + c];
-                        q += wpart[(w4 * 2 + 1) * p.BN + c];
+                        s += wp[(w4 * 2 + 0) * p.BN + c];
+                        q += wp[(w4 * 2 + 1) * p.BN + c];
                     }
                     stat_sum[n_tile * p.BN + c] += s;
                     stat_sq[n_tile * p.BN + c] += q;
                 }
+                par ^= 1;
+            } else {
+                __syncwarp();  // staged rows consumed before the next tile overwrites them
             }
             acc ^= 1;
             if (acc == 0) acc_ph ^= 1u;
@@ -332,6 +453,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             float* dst = p.partials + (size_t)blockIdx.x * 2 * p.ldo;
             for (int c = et; c < 2 * p.ldo; c += 128) dst[c] = stat_sum[c];
         }
+#ifdef NB_TC_DEBUG_TIMING
+        if (p.dbg && et == 0) { p.dbg[blockIdx.x * 8 + 5] = dbg_wait_tfull; p.dbg[blockIdx.x * 8 + 6] = clock64() - dbg_start; }
+#endif
         if (sat) atomicAdd(p.status + ST_SAT, sat);
     }
     ptx::tc_fence_before();
@@ -376,8 +500,8 @@ namespace nbcbs {
 struct IgemmCfg {
     bool ok = false;
     int Ca = 0, rowsB = 0, ntaps = 0;
-    int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0;
-    uint32_t a_stage = 0, b_stage = 0;
+    int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1;
+    uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
 };
@@ -449,36 +573,63 @@ inline uint32_t umma_swizzle_for(int KC) { return KC == 64 ? (uint32_t)ptx::kSwi
 constexpr size_t kMaxSmem = 232448;  // 227 KB opt-in limit per CTA
 
 // Tile configuration for a GEMM with M rows, `rowsB` output channels, `ntaps` taps of `Ca` channels each.
+// A stage of the pipeline holds `kpb` k-blocks so that one barrier round trip (a few hundred cycles of issue
+// latency in the producer and MMA threads) is amortised over enough tensor-core work.
+inline size_t igemm_fixed_smem(int BN, int ldo) {
+    return 1024 /*alignment slack*/ + (size_t)TC_BM * (BN * 2 + 16) + (size_t)2 * ldo * 4 + (size_t)16 * BN * 4 + 512;
+}
 inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count) {
     IgemmCfg c;
     c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
     if (Ca % 16 || rowsB % 16 || M < 1) return c;
-    c.KC = (Ca % 64 == 0) ? 64 : (Ca % 32 == 0) ? 32 : 16;
+    // Always 64-channel k-blocks in the 128-byte swizzle (the narrower swizzles make tcgen05.mma 1.6-2.1x slower per
+    // instruction); when Ca is not a multiple of 64 the last k-block of every tap reads past the channel extent and
+    // TMA fills A with zeros there (whatever finite filter values B holds at those positions are multiplied by zero).
+    c.KC = getenv("NB_TC_KC") ? atoi(getenv("NB_TC_KC")) : 64;
+    if (c.KC != 64 && Ca % c.KC) c.KC = 16;
     c.m_tiles = (int)((M + TC_BM - 1) / TC_BM);
-    const double ksteps = (double)ntaps * Ca / 16.0;
+    const int kblocks = ntaps * ((Ca + c.KC - 1) / c.KC);
+    const int force_bn = getenv("NB_TC_BN") ? atoi(getenv("NB_TC_BN")) : 0;
+    const int force_kpb = getenv("NB_TC_KPB") ? atoi(getenv("NB_TC_KPB")) : 0;
     double best = 1e30;
     for (int bn = 16; bn <= 256 && bn <= rowsB; bn += 16) {
         if (rowsB % bn) continue;
+        if (force_bn && bn != force_bn && rowsB % force_bn == 0) continue;
+        const uint32_t a_sub = (uint32_t)((TC_BM * c.KC * 2 + 1023) / 1024 * 1024);
+        const uint32_t b_sub = (uint32_t)((bn * c.KC * 2 + 1023) / 1024 * 1024);
+        const size_t fixed = igemm_fixed_smem(bn, ldo);
+        if (fixed + 2 * (size_t)(a_sub + b_sub) > kMaxSmem) continue;
+        const double mma_kb = (c.KC / 16) * std::max(bn, 16) / 2.0;  // tensor cycles per k-block
+        int kpb = std::max(1, std::min(kblocks, (int)((450.0 + mma_kb - 1) / mma_kb)));
+        if (force_kpb) kpb = std::min(kblocks, force_kpb);
+        int stages = 0;
+        for (;; --kpb) {
+            stages = (int)std::min<size_t>(8, (kMaxSmem - fixed) / ((size_t)kpb * (a_sub + b_sub)));
+            if (stages >= 3 || kpb == 1) break;
+        }
+        if (stages < 2) continue;
+        const int nstage_tile = (kblocks + kpb - 1) / kpb;
+        const double rows = (double)kpb * (TC_BM + bn);
+        const double stage_t = std::max(kpb * mma_kb, 200.0 + 1.6 * rows);      // tensor pipe vs TMA fill
+        const double main_t = nstage_tile * stage_t;
+        const double epi_t = 800.0 + 45.0 * bn;
         const long long tiles = (long long)c.m_tiles * (rowsB / bn);
         const double waves = (double)((tiles + sm_count - 1) / sm_count);
-        const double per_tile = ksteps * std::max(bn, 32) / 2.0 + 400.0 + 6.0 * bn;
-        const double cost = waves * per_tile;
+        const double cost = waves * std::max(main_t, epi_t) + epi_t;
         if (cost < best - 1e-9) {
             best = cost;
-            c.BN = bn;
+            c.BN = bn; c.kpb = kpb; c.stages = stages; c.a_sub = a_sub; c.b_sub = b_sub;
         }
     }
     if (!c.BN) return c;
     c.n_tiles = rowsB / c.BN;
     c.acc_stride = c.BN <= 32 ? 32 : c.BN <= 64 ? 64 : c.BN <= 128 ? 128 : 256;
     c.tmem_cols = 2 * c.acc_stride;
-    c.a_stage = (uint32_t)((TC_BM * c.KC * 2 + 1023) / 1024 * 1024);
-    c.b_stage = (uint32_t)((c.BN * c.KC * 2 + 1023) / 1024 * 1024);
-    const size_t fixed = 1024 /*alignment slack*/ + (size_t)TC_BM * (c.BN * 2 + 16) + (size_t)2 * ldo * 4 + (size_t)8 * c.BN * 4 + 512;
-    if (fixed + 2 * (size_t)(c.a_stage + c.b_stage) > kMaxSmem) return c;
-    c.stages = (int)std::min<size_t>(8, (kMaxSmem - fixed) / (c.a_stage + c.b_stage));
-    c.stages = std::max(2, std::min(c.stages, std::max(2, ntaps * (Ca / c.KC))));
-    c.smem_bytes = std::max<size_t>(fixed + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
+    c.a_stage = c.a_sub * c.kpb;
+    c.b_stage = c.b_sub * c.kpb;
+    c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
+    (void)kblocks;
+    c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
     c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count);
     c.ok = true;
     return c;
@@ -487,12 +638,17 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
 inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.M = c.M;
     P.ntaps = c.ntaps;
-    P.Ca = c.Ca; P.KC = c.KC; P.kc_per_tap = c.Ca / c.KC;
+    P.Ca = c.Ca; P.KC = c.KC; P.kc_per_tap = (c.Ca + c.KC - 1) / c.KC;
     P.BN = c.BN; P.n_tiles = c.n_tiles; P.m_tiles = c.m_tiles;
     P.stages = c.stages; P.acc_stride = c.acc_stride; P.tmem_cols = c.tmem_cols;
     P.umma_swizzle = umma_swizzle_for(c.KC);
     P.sbo = (uint32_t)(8 * c.KC * 2);
     P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
+    P.kpb = c.kpb; P.a_sub_bytes = c.a_sub; P.b_sub_bytes = c.b_sub;
+    P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
+    if (getenv("NB_TC_VERBOSE"))
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: KC=%d BN=%d kpb=%d stages=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca, c.rowsB,
+                c.ntaps, c.KC, c.BN, c.kpb, c.stages, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
     P.idesc = ptx::make_idesc_bf16(TC_BM, c.BN, 0, 0);
 }
 
@@ -570,6 +726,7 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
                     P.off_w[r * g.k + t] = (uint16_t)t;
                 }
             P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1; P.oa = 0; P.ob = 0;
+            P.a_tiled = (g.k == 1 && g.stride == 1) ? 1 : 0;
             tc->fprop = true;
             tc->fprop_parts = c.grid;
         }
@@ -684,11 +841,18 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     TcGemmSlot& S = tc->fp;
     if (S.a_ptr != x || S.b_ptr != w) {
         const int up = g.pad - (g.k - 1);
-        if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC)) return NB_ERR_CUDA;
+        if (S.prm.a_tiled) {
+            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM)) return NB_ERR_CUDA;
+        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC)) {
+            return NB_ERR_CUDA;
+        }
         if (!encode_tiled_2d(&S.prm.tmB, w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
+#ifdef NB_TC_DEBUG_TIMING
+    if (const char* e = getenv("NB_TC_DBG_PTR")) S.prm.dbg = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
+#endif
     tc->launches += 1;
     return launch_igemm<__half, true>(S, st);
 }
@@ -740,7 +904,7 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
         }
         attr_set = true;
     }
-    tc_wgrad_kernel<<<tc->wg_grid, TC_THREADS, tc->wg_smem, st>>>(P);
+    tc_wgrad_kernel<<<tc->wg_grid, WG_THREADS, tc->wg_smem, st>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { err() = std::string("launch of tc_wgrad_kernel failed: ") + cudaGetErrorString(e); return NB_ERR_CUDA; }
     tc->launches += 1;
