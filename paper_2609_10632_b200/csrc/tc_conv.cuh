@@ -797,41 +797,64 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
                 P.off_h[r * g.k + t] = (uint16_t)r;
                 P.off_w[r * g.k + t] = (uint16_t)t;
             }
-        P.KCA = (g.c_in % 64 == 0) ? 64 : (g.c_in % 32 == 0) ? 32 : 16;
-        P.nblkA = 128 / P.KCA;
-        P.cblk_per_tap = g.c_in / P.KCA;
-        P.m_tiles = (g.kdim + 127) / 128;
+        P.cblk_per_tap = (g.c_in + 63) / 64;
+        P.nblk_total = g.k * g.k * P.cblk_per_tap;
+        P.m_tiles = (P.nblk_total + 1) / 2;
         double best = 1e30;
         for (int bn = 16; bn <= 256 && bn <= g.c_out; bn += 16) {
             if (g.c_out % bn) continue;
-            const double cost = (double)(g.c_out / bn) * (std::max(bn, 64) + 16);
+            const double cost = (double)(g.c_out / bn) * std::max(97.0, bn / 2.0);  // tensor cycles per K = 16 step
             if (cost < best - 1e-9 || (cost < best + 1e-9 && bn > P.BN)) {
                 best = cost;
                 P.BN = bn;
             }
         }
         P.n_tiles = g.c_out / P.BN;
-        P.KCB = (P.BN % 64 == 0) ? 64 : (P.BN % 32 == 0) ? 32 : 16;
-        P.nblkB = P.BN / P.KCB;
-        P.total_chunks = (int)((g.m + WG_KP - 1) / WG_KP);
+        P.nblkB = (P.BN + 63) / 64;
+        // 128 pixels per stage when at least three stages fit, else 64
+        P.KP = 128;
+        for (;;) {
+            P.blk_bytes = (uint32_t)(64 * 2 * P.KP);
+            P.a_stage_bytes = 2 * P.blk_bytes;
+            P.b_stage_bytes = (uint32_t)P.nblkB * P.blk_bytes;
+            P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
+            if (P.stages >= 3 || P.KP == 64) break;
+            P.KP = 64;
+        }
+        if (getenv("NB_WG_KP")) {
+            P.KP = atoi(getenv("NB_WG_KP"));
+            P.blk_bytes = (uint32_t)(64 * 2 * P.KP);
+            P.a_stage_bytes = 2 * P.blk_bytes;
+            P.b_stage_bytes = (uint32_t)P.nblkB * P.blk_bytes;
+            P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
+        }
+        P.total_chunks = (int)((g.m + P.KP - 1) / P.KP);
         const int tiles = P.m_tiles * P.n_tiles;
-        int splits = std::max(1, (sm_count + tiles / 2) / tiles);
-        splits = std::min(splits, std::max(1, P.total_chunks / 8));
-        P.chunks_per_split = (P.total_chunks + splits - 1) / splits;
+        // split-K factor: fewest waves of CTAs times chunks per CTA (plus a fixed prologue/epilogue of a few chunks)
+        int best_s = 1;
+        double best_c = 1e30;
+        const int max_s = std::max(1, std::min(64, P.total_chunks / 4));
+        for (int sp = 1; sp <= max_s; ++sp) {
+            const double waves = (double)(((long long)tiles * sp + sm_count - 1) / sm_count);
+            const double c = waves * ((P.total_chunks + sp - 1) / sp + 6.0) + 0.02 * sp;
+            if (c < best_c - 1e-9) {
+                best_c = c;
+                best_s = sp;
+            }
+        }
+        if (getenv("NB_WG_SPLITS")) best_s = std::max(1, std::min(max_s, atoi(getenv("NB_WG_SPLITS"))));
+        P.chunks_per_split = (P.total_chunks + best_s - 1) / best_s;
         P.splits = (P.total_chunks + P.chunks_per_split - 1) / P.chunks_per_split;
-        P.a_stage_bytes = 128 * WG_KP * 2;
-        P.b_stage_bytes = (uint32_t)((P.BN * WG_KP * 2 + 1023) / 1024 * 1024);
-        P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
         P.stages = std::max(2, std::min(P.stages, std::max(2, P.chunks_per_split)));
         P.tmem_cols = P.BN <= 32 ? 32 : P.BN <= 64 ? 64 : P.BN <= 128 ? 128 : 256;
-        P.swzA = umma_swizzle_for(P.KCA); P.swzB = umma_swizzle_for(P.KCB);
-        P.sboA = (uint32_t)(8 * P.KCA * 2); P.sboB = (uint32_t)(8 * P.KCB * 2);
-        P.lboA = (uint32_t)(WG_KP * P.KCA * 2); P.lboB = (uint32_t)(WG_KP * P.KCB * 2);
         P.idesc = ptx::make_idesc_bf16(128, P.BN, 1, 1);
         tc->wg_smem = std::max<size_t>(2048 + (size_t)P.stages * (P.a_stage_bytes + P.b_stage_bytes), 120 * 1024);
         tc->wg_grid = tiles * P.splits;
         tc->wgrad_partial_bytes = P.splits > 1 ? (size_t)P.splits * g.c_out * g.kdim * 4 : 0;
         tc->wgrad = true;
+        if (getenv("NB_TC_VERBOSE"))
+            fprintf(stderr, "[nb_cbs] wgrad M=%lld Cin=%d Cout=%d k=%d: BN=%d KP=%d stages=%d tiles=%dx%d splits=%d (chunks/split %d) grid=%d\n", (long long)g.m,
+                    g.c_in, g.c_out, g.k, P.BN, P.KP, P.stages, P.m_tiles, P.n_tiles, P.splits, P.chunks_per_split, tc->wg_grid);
     }
     return NB_OK;
 }
@@ -890,8 +913,8 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
     WgradParams& P = tc->wg;
     if (tc->wg_a_ptr != x || tc->wg_b_ptr != dy) {
         const int up = g.pad - (g.k - 1);
-        if (!encode_im2col(&P.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, P.KCA, WG_KP)) return NB_ERR_CUDA;
-        if (!encode_tiled_2d(&P.tmB, dy, g.m, g.c_out, P.KCB, WG_KP)) return NB_ERR_CUDA;
+        if (!encode_im2col(&P.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, 64, P.KP)) return NB_ERR_CUDA;
+        if (!encode_tiled_2d(&P.tmB, dy, g.m, g.c_out, 64, P.KP)) return NB_ERR_CUDA;
         tc->wg_a_ptr = x; tc->wg_b_ptr = dy;
     }
     P.out = P.splits > 1 ? partial : dw;
@@ -904,7 +927,7 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
         }
         attr_set = true;
     }
-    tc_wgrad_kernel<<<tc->wg_grid, WG_THREADS, tc->wg_smem, st>>>(P);
+    tc_wgrad_kernel<<<tc->wg_grid, TC_THREADS, tc->wg_smem, st>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { err() = std::string("launch of tc_wgrad_kernel failed: ") + cudaGetErrorString(e); return NB_ERR_CUDA; }
     tc->launches += 1;

@@ -1,7 +1,8 @@
 // Tensor-core weight gradient for sm_100a.  dw[c'][tap][c] = sum over pixels of dy[pixel][c'] * x_tap[pixel][c] is a
 // GEMM whose reduction index is the pixel.  Both operands are channel-contiguous, so both are fed to tcgen05.mma
-// as MN-major shared-memory tiles: A = im2col boxes of x (rows of the accumulator = positions in the flattened
-// (tap, c) axis of the filter, taken in blocks of KCA channels), B = boxes of dy (columns = output channels).
+// as MN-major shared-memory tiles in the 128-byte swizzle: A = im2col boxes of x, 64 channels of one filter tap by
+// KP pixels each (two boxes give the 128 accumulator rows; channels past Cin are zero-filled by TMA and never
+// stored), B = boxes of dy, 64 output channels by KP pixels (columns of the accumulator).
 // Each CTA owns one [128 x BN] tile of dw for one slice of the pixel range (split-K); slices are summed in a fixed
 // order by a second kernel, so the result is bitwise reproducible.
 // Included by tc_conv.cuh (uses its bounded-wait helpers).
@@ -10,25 +11,25 @@
 namespace nbcbs {
 
 struct WgradParams {
-    CUtensorMap tmA;  // im2col map over x [N][H][W][Cin], KCA channels x KP pixels per load
-    CUtensorMap tmB;  // tiled map over dy [M][Cout], KCB channels x KP pixels per load
+    CUtensorMap tmA;  // im2col map over x [N][H][W][Cin], 64 channels x KP pixels per load
+    CUtensorMap tmB;  // tiled map over dy [M][Cout], 64 channels x KP pixels per load
     long long M;      // pixels (reduction length)
     int Hq, Wq, ts, lo_w, lo_h;
     int c_in, c_out, kdim;
-    int KCA, KCB, nblkA, nblkB;  // channel-block widths and blocks per tile (128/KCA, BN/KCB)
-    int cblk_per_tap;            // c_in / KCA
+    int cblk_per_tap;  // ceil(c_in / 64): 64-channel blocks per tap along the accumulator rows
+    int nblk_total;    // taps * cblk_per_tap
+    int nblkB;         // ceil(BN / 64)
+    int KP;            // pixels per pipeline stage (64 or 128)
     int BN, n_tiles, m_tiles;
     int splits, chunks_per_split, total_chunks;
     int stages, tmem_cols;
-    uint32_t swzA, swzB, sboA, sboB, lboA, lboB, a_stage_bytes, b_stage_bytes, idesc;
+    uint32_t a_stage_bytes, b_stage_bytes, blk_bytes, idesc;
     float* out;  // [splits][c_out][kdim] (or dw itself when splits == 1)
     int* status;
     uint16_t off_w[9], off_h[9];
 };
 
-constexpr int WG_KP = 64;  // pixels per pipeline stage (four K = 16 MMA steps)
-
-__global__ void __launch_bounds__(WG_THREADS, 1) tc_wgrad_kernel(const __grid_constant__ WgradParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_constant__ WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
@@ -52,7 +53,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) tc_wgrad_kernel(const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(full + s, 2);  // the x producer and the dy producer each arrive once
             ptx::mbar_init(empty + s, 1);
         }
         ptx::mbar_init(tfull, 1);
@@ -69,73 +70,104 @@ __global__ void __launch_bounds__(WG_THREADS, 1) tc_wgrad_kernel(const __grid_co
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
+    if (warp == 0 || warp == 6) {
+        // ------------------------------------------------------------------ TMA producers: warp 0 feeds x, warp 6 feeds dy
         if (lane == 0 && nchunks > 0) {
-            ptx::prefetch_tmap(&p.tmA);
-            ptx::prefetch_tmap(&p.tmB);
+            const bool isA = warp == 0;
+            ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
             int s = 0, issued = 0;
             uint32_t ph = 0;
             bool ok = true;
-            const uint32_t blkA = (uint32_t)(WG_KP * p.KCA * 2), blkB = (uint32_t)(WG_KP * p.KCB * 2);
-            const uint32_t tx_bytes = (uint32_t)p.nblkA * blkA + (uint32_t)p.nblkB * blkB;
+            const int stages = p.stages, KP = p.KP, Wq = p.Wq, Hq = p.Hq, ts = p.ts;
+            const uint32_t blk = p.blk_bytes;
+            const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes;
+            const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB), full_u32 = ptx::smem_u32(full);
+            const CUtensorMap* tm = isA ? &p.tmA : &p.tmB;
+            const int nblk = isA ? 2 : p.nblkB;
+            // the two 64-channel blocks of x this tile owns (a block past the end of the filter is replaced by block 0:
+            // its accumulator rows are never stored)
+            int tapv[2], c0v[2];
+            for (int b = 0; b < 2; ++b) {
+                int fb = m_tile * 2 + b;
+                if (fb >= p.nblk_total) fb = 0;
+                tapv[b] = fb / p.cblk_per_tap;
+                c0v[b] = (fb - tapv[b] * p.cblk_per_tap) * 64;
+            }
+            const uint16_t ow0 = p.off_w[tapv[0]], oh0 = p.off_h[tapv[0]], ow1 = p.off_w[tapv[1]], oh1 = p.off_h[tapv[1]];
+            const int bcol = n_tile * p.BN;
             for (int ch = chunk0; ch < chunk1; ++ch) {
-                const long long m0 = (long long)ch * WG_KP;
-                const int j0 = (int)(m0 % p.Wq);
-                const long long t1 = m0 / p.Wq;
-                const int i0 = (int)(t1 % p.Hq), n0 = (int)(t1 / p.Hq);
-                const int cw = p.lo_w + j0 * p.ts, chh = p.lo_h + i0 * p.ts;
-                if (!wait_bar(empty + s, ph ^ 1u, abort_flag, p.status, 11)) {
+                const int m0 = ch * KP;
+                if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, isA ? 11 : 15)) {
                     ok = false;
                     break;
                 }
-                ptx::mbar_expect_tx(full + s, tx_bytes);
-                uint8_t* a = sA + (size_t)s * p.a_stage_bytes;
-                for (int b = 0; b < p.nblkA; ++b) {
-                    int fb = m_tile * p.nblkA + b;             // block index along the flattened (tap, c) axis
-                    if (fb * p.KCA >= p.kdim) fb = 0;           // past the end of the filter: any valid block (rows are not stored)
-                    const int tap = fb / p.cblk_per_tap, c0 = (fb - tap * p.cblk_per_tap) * p.KCA;
-                    ptx::tma_load_im2col_4d(a + (size_t)b * blkA, &p.tmA, full + s, c0, cw, chh, n0, p.off_w[tap], p.off_h[tap]);
+                const uint32_t bar = full_u32 + 8u * (uint32_t)s;
+                ptx::mbar_expect_tx_u32(bar, blk * (uint32_t)nblk);
+                const uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
+                if (isA) {
+                    const int j0 = m0 % Wq, t1 = m0 / Wq;
+                    const int i0 = t1 % Hq, n0 = t1 / Hq;
+                    const int cw = p.lo_w + j0 * ts, chh = p.lo_h + i0 * ts;
+                    ptx::tma_load_im2col_4d_u32(dst, tm, bar, c0v[0], cw, chh, n0, ow0, oh0);
+                    ptx::tma_load_im2col_4d_u32(dst + blk, tm, bar, c0v[1], cw, chh, n0, ow1, oh1);
+                } else {
+                    for (int b = 0; b < nblk; ++b) ptx::tma_load_2d_u32(dst + (uint32_t)b * blk, tm, bar, bcol + b * 64, m0);
                 }
-                uint8_t* bb = sB + (size_t)s * p.b_stage_bytes;
-                for (int b = 0; b < p.nblkB; ++b)
-                    ptx::tma_load_2d(bb + (size_t)b * blkB, &p.tmB, full + s, n_tile * p.BN + b * p.KCB, (int)m0);
                 ++issued;
-                if (++s == p.stages) {
+                if (++s == stages) {
                     s = 0;
                     ph ^= 1u;
                 }
             }
             if (!ok) {
                 // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
-                const int back = issued < p.stages ? issued : p.stages;
+                const int back = issued < stages ? issued : stages;
                 for (int b = 0; b < back; ++b) {
-                    s = (s == 0) ? p.stages - 1 : s - 1;
-                    if (s == p.stages - 1) ph ^= 1u;
+                    s = (s == 0) ? stages - 1 : s - 1;
+                    if (s == stages - 1) ph ^= 1u;
                     for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
                     }
                 }
             }
         }
     } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
         if (lane == 0 && nchunks > 0) {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            const int stages = p.stages, ksteps = p.KP / 16;
+            const uint32_t idesc = p.idesc;
+            // MN-major, 128-byte swizzle: 8 pixel rows of 128 bytes form one 1024-byte group (SBO); the next 64 channels
+            // start one block later (LBO); a K = 16 step advances by two row groups.
+            const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), p.blk_bytes, 1024, ptx::kSwizzle128);
+            const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), p.blk_bytes, 1024, ptx::kSwizzle128);
+            const uint64_t a_stage16 = (uint64_t)(p.a_stage_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
+            const uint32_t empty_u32 = ptx::smem_u32(empty);
+            uint64_t da_s = da0, db_s = db0;
+            uint32_t accumulate = 0;
             for (int ch = 0; ch < nchunks; ++ch) {
-                if (!wait_bar(full + s, ph, abort_flag, p.status, 12)) {
+                if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 12)) {
                     ok = false;
                     break;
                 }
                 ptx::tc_fence_after();
-                const uint64_t da = ptx::make_smem_desc(ptx::smem_u32(sA + (size_t)s * p.a_stage_bytes), p.lboA, p.sboA, p.swzA);
-                const uint64_t db = ptx::make_smem_desc(ptx::smem_u32(sB + (size_t)s * p.b_stage_bytes), p.lboB, p.sboB, p.swzB);
-                // one K = 16 step covers two 8-pixel row groups of every block
-                const uint64_t stepA = (uint64_t)((2 * p.sboA) >> 4), stepB = (uint64_t)((2 * p.sboB) >> 4);
-                for (int k = 0; k < WG_KP / 16; ++k) ptx::umma_f16(tmem_base, da + k * stepA, db + k * stepB, p.idesc, (ch | k) ? 1u : 0u);
-                ptx::umma_commit(empty + s);
-                if (++s == p.stages) {
+                uint64_t da = da_s, db = db_s;
+#pragma unroll 4
+                for (int k = 0; k < ksteps; ++k) {
+                    ptx::umma_f16(tmem_base, da, db, idesc, accumulate);
+                    accumulate = 1u;
+                    da += 128;  // 2048 bytes >> 4
+                    db += 128;
+                }
+                ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
+                da_s += a_stage16;
+                db_s += b_stage16;
+                if (++s == stages) {
                     s = 0;
                     ph ^= 1u;
+                    da_s = da0;
+                    db_s = db0;
                 }
             }
             if (ok) {
@@ -149,11 +181,18 @@ __global__ void __launch_bounds__(WG_THREADS, 1) tc_wgrad_kernel(const __grid_co
             }
         }
     } else {
+        // ------------------------------------------------------------------ epilogue (warps 2-5)
         const int lane_group = warp & 3;
         const int row = lane_group * 32 + lane;
-        const int kidx = m_tile * 128 + row;  // position along the flattened (tap, c) axis
+        // accumulator row -> (tap, channel): rows come in two blocks of 64 channels
+        const int fb = m_tile * 2 + (row >> 6);
+        const int tap = fb / p.cblk_per_tap;
+        const int c = (fb - tap * p.cblk_per_tap) * 64 + (row & 63);
+        const bool valid = fb < p.nblk_total && c < p.c_in;
+        const int kidx = tap * p.c_in + c;  // position inside dw[c'][:]
         bool ok = true;
-        if (nchunks > 0) ok = wait_bar(tfull, 0, abort_flag, p.status, 13);
+        if (nchunks > 0 && lane == 0) ok = wait_bar(tfull, 0, abort_flag, p.status, 13);
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         ok = epi_bar_and(ok);
         if (ok) {
             ptx::tc_fence_after();
@@ -168,7 +207,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) tc_wgrad_kernel(const __grid_co
 #pragma unroll
                     for (int j = 0; j < 16; ++j) r[j] = 0u;
                 }
-                if (kidx < p.kdim) {
+                if (valid) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) dst[(size_t)(n_tile * p.BN + c0 + j) * p.kdim + kidx] = __uint_as_float(r[j]);
                 }
