@@ -54,33 +54,41 @@ __global__ void __launch_bounds__(1024) bn_stats_partial_kernel(const YT* __rest
     }
 }
 
-// Combine partials [nparts][2][C] in fp64 (fixed order) and derive the per-channel quantities.
-// block (32,32): x = channel within a group of 32, y = slice of the partial list.
+// Sum partials[b][which][c] over b in fp64: lane l takes b = l, l+32, ... (independent loads in flight), then a
+// butterfly over the 32 lanes.  The order is fixed, so the result is bitwise reproducible.
+__device__ __forceinline__ double warp_sum_partials(const float* __restrict__ partials, int nparts, int C, int c, int which, int lane) {
+    double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
+    const float* base = partials + (size_t)which * C + c;
+    const size_t step = (size_t)2 * C;
+    int b = lane;
+    for (; b + 96 < nparts; b += 128) {
+        const float v0 = base[(size_t)b * step], v1 = base[(size_t)(b + 32) * step], v2 = base[(size_t)(b + 64) * step],
+                    v3 = base[(size_t)(b + 96) * step];
+        acc0 += (double)v0;
+        acc1 += (double)v1;
+        acc2 += (double)v2;
+        acc3 += (double)v3;
+    }
+    for (; b < nparts; b += 32) acc0 += (double)base[(size_t)b * step];
+    double s = (acc0 + acc1) + (acc2 + acc3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
+}
+
+// Combine partials [nparts][2][C] and derive the per-channel quantities.  One warp per channel, 8 channels per block.
 // Outputs (any may be NULL): mean, invstd, scale = gamma*invstd, shift = beta - mean*scale, raw sums,
 // running statistics (in place; unbiased variance, momentum).
-__global__ void bn_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float eps,
-                                   float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
-                                   float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
-                                   float* sum_out, float* sumsq_out) {
-    __shared__ double sh_s[32][33], sh_q[32][33];
-    const int c = blockIdx.x * 32 + threadIdx.x;
-    double s = 0.0, q = 0.0;
-    if (c < C) {
-        for (int b = threadIdx.y; b < nparts; b += 32) {
-            s += (double)partials[((size_t)b * 2) * C + c];
-            q += (double)partials[((size_t)b * 2 + 1) * C + c];
-        }
-    }
-    sh_s[threadIdx.y][threadIdx.x] = s;
-    sh_q[threadIdx.y][threadIdx.x] = q;
-    __syncthreads();
-    if (threadIdx.y == 0 && c < C) {
-        s = 0.0;
-        q = 0.0;
-        for (int j = 0; j < 32; ++j) {
-            s += sh_s[j][threadIdx.x];
-            q += sh_q[j][threadIdx.x];
-        }
+__global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float eps,
+                                                          float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                          float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
+                                                          float* sum_out, float* sumsq_out) {
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= C) return;
+    const double s = warp_sum_partials(partials, nparts, C, c, 0, lane);
+    const double q = warp_sum_partials(partials, nparts, C, c, 1, lane);
+    if (lane == 0) {
         const double mu = s / M;
         double var = q / M - mu * mu;
         if (var < 0.0) var = 0.0;
@@ -179,27 +187,14 @@ __global__ void __launch_bounds__(1024) bn_silu_bwd_reduce_kernel(const AT* __re
 }
 
 // partials [nparts][2][C] -> dbeta, dgamma (fp32) and the two per-channel coefficients dbeta/M, dgamma/M.
-__global__ void bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float* dgamma,
-                                       float* dbeta, float* coef /*[2][C]*/) {
-    __shared__ double sh_s[32][33], sh_q[32][33];
-    const int c = blockIdx.x * 32 + threadIdx.x;
-    double s = 0.0, q = 0.0;
-    if (c < C) {
-        for (int b = threadIdx.y; b < nparts; b += 32) {
-            s += (double)partials[((size_t)b * 2) * C + c];
-            q += (double)partials[((size_t)b * 2 + 1) * C + c];
-        }
-    }
-    sh_s[threadIdx.y][threadIdx.x] = s;
-    sh_q[threadIdx.y][threadIdx.x] = q;
-    __syncthreads();
-    if (threadIdx.y == 0 && c < C) {
-        s = 0.0;
-        q = 0.0;
-        for (int j = 0; j < 32; ++j) {
-            s += sh_s[j][threadIdx.x];
-            q += sh_q[j][threadIdx.x];
-        }
+__global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float* dgamma,
+                                                              float* dbeta, float* coef /*[2][C]*/) {
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= C) return;
+    const double s = warp_sum_partials(partials, nparts, C, c, 0, lane);
+    const double q = warp_sum_partials(partials, nparts, C, c, 1, lane);
+    if (lane == 0) {
         dbeta[c] = (float)s;
         dgamma[c] = (float)q;
         coef[c] = (float)(s / M);

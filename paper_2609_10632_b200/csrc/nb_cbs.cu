@@ -153,7 +153,7 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
                        cudaStream_t st) {
     const int C = p->g.c_out;
     SiteTimer tm(p, SITE_FINALIZE, st);
-    bn_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
+    bn_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
                                                               gamma, beta, mean, invstd, scale, shift, rmean, rvar, sum, sumsq);
     return launch_ok("bn_finalize");
 }
@@ -181,7 +181,7 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     }
     {
         SiteTimer tm(p, SITE_BWD_FINALIZE, st);
-        bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, 32), 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
+        bn_bwd_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
@@ -637,7 +637,7 @@ extern "C" nb_status nb_bn_stats_static(const void* y, int32_t y_dtype, int64_t 
     else
         bn_stats_partial_kernel<__half><<<blocks, tpb, (size_t)tpb * vec * sizeof(float), st>>>(static_cast<const __half*>(y), total_vecs, c, part);
     NB_LAUNCH_OK("bn_stats_partial (static scratch)");
-    bn_finalize_kernel<<<(c + 31) / 32, dim3(32, 32), 0, st>>>(part, blocks, c, (double)m, eps, 0.f, nullptr, nullptr, mean, invstd, nullptr,
+    bn_finalize_kernel<<<(c + 7) / 8, 256, 0, st>>>(part, blocks, c, (double)m, eps, 0.f, nullptr, nullptr, mean, invstd, nullptr,
                                                               nullptr, nullptr, nullptr, sum, sumsq);
     return launch_ok("bn_finalize (static scratch)");
 }

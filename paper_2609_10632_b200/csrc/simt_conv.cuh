@@ -155,12 +155,32 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(P prob, TO* __restrict__
     }
 }
 
-// out[e] = sum_z partial[z][e], summed in fp64 in slice order.
-__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int splits, size_t elems, float* __restrict__ out) {
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < elems; e += (size_t)gridDim.x * blockDim.x) {
-        double s = 0.0;
-        for (int z = 0; z < splits; ++z) s += (double)partial[(size_t)z * elems + e];
-        out[e] = (float)s;
+// out[e] = sum_z partial[z][e], summed in fp64 in slice order (four elements per thread when the count allows).
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partial, int splits, size_t elems, float* __restrict__ out) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    if ((elems & 3) == 0) {
+        const size_t nv = elems >> 2;
+        const float4* p4 = reinterpret_cast<const float4*>(partial);
+        for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
+            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+            int z = 0;
+            for (; z + 1 < splits; z += 2) {
+                const float4 a = p4[(size_t)z * nv + v], b = p4[(size_t)(z + 1) * nv + v];
+                s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
+                s0 += (double)b.x; s1 += (double)b.y; s2 += (double)b.z; s3 += (double)b.w;
+            }
+            if (z < splits) {
+                const float4 a = p4[(size_t)z * nv + v];
+                s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
+            }
+            reinterpret_cast<float4*>(out)[v] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
+        }
+    } else {
+        for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < elems; e += stride) {
+            double s = 0.0;
+            for (int z = 0; z < splits; ++z) s += (double)partial[(size_t)z * elems + e];
+            out[e] = (float)s;
+        }
     }
 }
 

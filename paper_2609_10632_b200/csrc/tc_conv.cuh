@@ -22,13 +22,17 @@ namespace nbcbs {
 
 // ------------------------------------------------------------------------------------------ kernel parameters
 struct IgemmParams {
-    CUtensorMap tmA;  // im2col map over the activation [N][Hs][Ws][Ca]
-    CUtensorMap tmB;  // tiled map over the filter matrix [rowsB][ntaps*Ca], K contiguous
+    CUtensorMap tmA;     // im2col map over the activation [N][Hs][Ws][Ca]
+    CUtensorMap tmB[4];  // per class: tiled map over the filter matrix [rowsB][ntaps*Ca], K contiguous
     long long M;      // rows of the GEMM: n * Hq * Wq
     int Hq, Wq;       // traversal grid per image
     int ts;           // traversal stride (input pixels per grid step)
     int lo_w, lo_h;   // input coordinate of grid position 0 for tap offset 0
-    int ntaps;
+    // A launch covers up to four "classes" that share A, the tiling and the output tensor but have their own filter
+    // matrix, tap list and output offset (the four output-parity classes of a stride-2 data gradient); tiles are
+    // numbered class by class, classes with more taps first.
+    int nclasses, tiles_per_class;
+    int cls_ntaps[4], cls_oa[4], cls_ob[4];
     int Ca, KC, kc_per_tap;
     int kpb;                     // k-blocks (of KC channels) per pipeline stage
     uint32_t a_sub_bytes, b_sub_bytes;  // bytes of one k-block of A / B inside a stage
@@ -38,12 +42,12 @@ struct IgemmParams {
     int variant;                 // experiment switches
     int a_tiled;                 // 1: A is a plain [M][Ca] matrix fetched with a tiled 2-D map (1x1 stride-1 convolutions)
     int ldo;                     // channels per output pixel
-    int Hout, Wout, os, oa, ob;  // GEMM row (n,i,j) -> output pixel (n, i*os+oa, j*os+ob) of an Hout x Wout image
+    int Hout, Wout, os;          // GEMM row (n,i,j) -> output pixel (n, i*os+oa, j*os+ob) of an Hout x Wout image
     void* out;
     long long* dbg;   // optional [gridDim.x][8] cycle counters (only read when built with NB_TC_DEBUG_TIMING)
     float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
     int* status;
-    uint16_t off_w[9], off_h[9];
+    uint16_t off_w[4][9], off_h[4][9];
 };
 
 #ifdef NB_TC_DEBUG_TIMING
@@ -144,8 +148,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = p.m_tiles * p.n_tiles;
-    const int kblocks = p.ntaps * p.kc_per_tap;
+    const int total_tiles = p.nclasses * p.tiles_per_class;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -176,7 +179,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
         if (lane == 0) {
             const bool isA = warp == 0;
-            ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
+            if (isA) {
+                ptx::prefetch_tmap(&p.tmA);
+            } else {
+                for (int c = 0; c < p.nclasses; ++c) ptx::prefetch_tmap(&p.tmB[c]);
+            }
             int s = 0;
             uint32_t ph = 0;
             long long issued = 0;
@@ -191,9 +198,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
             const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes, sub_bytes = isA ? p.a_sub_bytes : p.b_sub_bytes;
             const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB), full_u32 = ptx::smem_u32(full);
-            const CUtensorMap* tm = isA ? &p.tmA : &p.tmB;
+            const int tpc = p.tiles_per_class;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int m_tile = tile / n_tiles, n_tile = tile - m_tile * n_tiles;
+                const int cls = tile / tpc, lt = tile - cls * tpc;
+                const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
+                const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
+                const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
                 const int m0 = m_tile * TC_BM;
                 int cw = 0, ch = 0, n0 = 0;
                 if (isA && !a_tiled) {
@@ -223,7 +233,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                             if (a_tiled)
                                 ptx::tma_load_2d_u32(dst, tm, bar, kc * KC, m0);
                             else
-                                ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[tap], p.off_h[tap]);
+                                ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
                         } else {
                             ptx::tma_load_2d_u32(dst, tm, bar, tap * Ca + kc * KC, brow);
                         }
@@ -272,7 +282,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, p.sbo, p.umma_swizzle);
             const uint32_t empty_u32 = ptx::smem_u32(empty);
             uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
+            const int tpc = p.tiles_per_class, kc_per_tap = p.kc_per_tap;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const int kblocks = p.cls_ntaps[tile / tpc] * kc_per_tap;
                 {
                     NB_DBG_T0();
                     if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
@@ -344,7 +356,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         const long long dbg_start = clock64();
 #endif
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
+            const int cls = tile / p.tiles_per_class, lt = tile - cls * p.tiles_per_class;
+            const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
             const long long m0 = (long long)m_tile * TC_BM;
             NB_DBG_T0();
             bool ok = true;
@@ -422,7 +435,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         const long long t1 = m / p.Wq;
                         const int i = (int)(t1 % p.Hq);
                         const long long n = t1 / p.Hq;
-                        pix = (n * p.Hout + (long long)i * p.os + p.oa) * p.Wout + (long long)j * p.os + p.ob;
+                        pix = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
                     }
                     const uint4 v = *reinterpret_cast<const uint4*>(my_rows + (size_t)rr * pitch + lc * 16);
                     *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN) * 2 + (size_t)lc * 16) = v;
@@ -521,8 +534,7 @@ struct TcPlan {
     int sm_count = 0;
     long long launches = 0;  // kernels launched through this record
     TcGemmSlot fp;
-    int dg_classes = 0;
-    TcGemmSlot dg[4];
+    TcGemmSlot dg;  // one launch covers all output-parity classes
     WtParams wtp;
     // wgrad
     WgradParams wg;
@@ -578,7 +590,7 @@ constexpr size_t kMaxSmem = 232448;  // 227 KB opt-in limit per CTA
 inline size_t igemm_fixed_smem(int BN, int ldo) {
     return 1024 /*alignment slack*/ + (size_t)TC_BM * (BN * 2 + 16) + (size_t)2 * ldo * 4 + (size_t)16 * BN * 4 + 512;
 }
-inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count) {
+inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses) {
     IgemmCfg c;
     c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
     if (Ca % 16 || rowsB % 16 || M < 1) return c;
@@ -613,7 +625,7 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
         const double stage_t = std::max(kpb * mma_kb, 200.0 + 1.6 * rows);      // tensor pipe vs TMA fill
         const double main_t = nstage_tile * stage_t;
         const double epi_t = 800.0 + 45.0 * bn;
-        const long long tiles = (long long)c.m_tiles * (rowsB / bn);
+        const long long tiles = (long long)c.m_tiles * (rowsB / bn) * nclasses;
         const double waves = (double)((tiles + sm_count - 1) / sm_count);
         const double cost = waves * std::max(main_t, epi_t) + epi_t;
         if (cost < best - 1e-9) {
@@ -630,14 +642,13 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
     (void)kblocks;
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
-    c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count);
+    c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, sm_count);
     c.ok = true;
     return c;
 }
 
 inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.M = c.M;
-    P.ntaps = c.ntaps;
     P.Ca = c.Ca; P.KC = c.KC; P.kc_per_tap = (c.Ca + c.KC - 1) / c.KC;
     P.BN = c.BN; P.n_tiles = c.n_tiles; P.m_tiles = c.m_tiles;
     P.stages = c.stages; P.acc_stride = c.acc_stride; P.tmem_cols = c.tmem_cols;
@@ -713,75 +724,83 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
     const bool even = (g.h % 2 == 0) && (g.w % 2 == 0);
     // ---- fprop: A = x (im2col), B = w [Cout][k*k*Cin]
     if (g.c_in % 16 == 0 && g.c_out % 16 == 0) {
-        IgemmCfg c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count);
+        IgemmCfg c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count, 1);
         if (c.ok) {
             tc->fp.cfg = c;
             IgemmParams& P = tc->fp.prm;
             memset(&P, 0, sizeof P);
             fill_params(P, c);
             P.Hq = g.ho; P.Wq = g.wo; P.ts = g.stride; P.lo_w = -g.pad; P.lo_h = -g.pad;
+            P.nclasses = 1; P.tiles_per_class = c.m_tiles * c.n_tiles;
+            P.cls_ntaps[0] = g.k * g.k;
             for (int r = 0; r < g.k; ++r)
                 for (int t = 0; t < g.k; ++t) {
-                    P.off_h[r * g.k + t] = (uint16_t)r;
-                    P.off_w[r * g.k + t] = (uint16_t)t;
+                    P.off_h[0][r * g.k + t] = (uint16_t)r;
+                    P.off_w[0][r * g.k + t] = (uint16_t)t;
                 }
-            P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1; P.oa = 0; P.ob = 0;
+            P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1;
             P.a_tiled = (g.k == 1 && g.stride == 1) ? 1 : 0;
             tc->fprop = true;
             tc->fprop_parts = c.grid;
         }
     }
-    // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four parity classes
+    // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four output-parity
+    // classes, heaviest (four taps) first so that the static round-robin tile order approximates longest-first
     if (g.c_in % 16 == 0 && g.c_out % 16 == 0 && (g.stride == 1 || (g.k == 3 && even))) {
         WtParams& W = tc->wtp;
         memset(&W, 0, sizeof W);
         W.c_in = g.c_in; W.c_out = g.c_out; W.k = g.k;
-        bool ok = true;
-        size_t off = 0;
+        IgemmParams& P = tc->dg.prm;
+        memset(&P, 0, sizeof P);
         const int ncls = g.stride == 1 ? 1 : 4;
-        for (int cls = 0; cls < ncls && ok; ++cls) {
-            const int pa = cls / 2, pb = cls % 2;  // output row / column parity (stride 2)
-            TcGemmSlot& S = tc->dg[cls];
-            IgemmParams& P = S.prm;
-            memset(&P, 0, sizeof P);
+        size_t off = 0;
+        int max_taps = 0;
+        for (int cls = 0; cls < ncls; ++cls) {
             WtClass& C = W.cls[cls];
             C.offset = off;
             int nt = 0;
             if (g.stride == 1) {
-                // dx[h][w] = sum_{r,t} dy[h+P-r][w+P-t] w[r][t]: traversal from -(k-1-P) with offsets r' = k-1-r
+                // dx[h][w] = sum_{r,t} dy[h+P-r][w+P-t] w[r][t]: window start runs from -(k-1-P), tap offset ro pairs with r = k-1-ro
                 for (int ro = 0; ro < g.k; ++ro)
                     for (int to = 0; to < g.k; ++to) {
-                        P.off_h[nt] = (uint16_t)ro; P.off_w[nt] = (uint16_t)to;
+                        P.off_h[cls][nt] = (uint16_t)ro; P.off_w[cls][nt] = (uint16_t)to;
                         C.r[nt] = g.k - 1 - ro; C.t[nt] = g.k - 1 - to;
                         ++nt;
                     }
-                P.Hq = g.h; P.Wq = g.w; P.ts = 1; P.lo_w = P.lo_h = -(g.k - 1 - g.pad);
-                P.Hout = g.h; P.Wout = g.w; P.os = 1; P.oa = 0; P.ob = 0;
+                P.cls_oa[cls] = 0; P.cls_ob[cls] = 0;
             } else {
-                // dx[2i+pa][2j+pb]: rows with pa=0 see tap r=1 at dy row i; pa=1 sees r=0 at dy row i+1 and r=2 at dy row i
+                const int pa = 1 - cls / 2, pb = 1 - cls % 2;  // output row / column parity; class 0 = (odd, odd) = four taps
+                // dx[2i+pa][2j+pb]: even rows see tap r=1 at dy row i; odd rows see r=0 at dy row i+1 and r=2 at dy row i
                 int rs[2], ro[2], nr = 0, tsv[2], to[2], ntc = 0;
                 if (pa == 0) { rs[0] = 1; ro[0] = 0; nr = 1; } else { rs[0] = 2; ro[0] = 0; rs[1] = 0; ro[1] = 1; nr = 2; }
                 if (pb == 0) { tsv[0] = 1; to[0] = 0; ntc = 1; } else { tsv[0] = 2; to[0] = 0; tsv[1] = 0; to[1] = 1; ntc = 2; }
                 for (int a = 0; a < nr; ++a)
                     for (int b = 0; b < ntc; ++b) {
-                        P.off_h[nt] = (uint16_t)ro[a]; P.off_w[nt] = (uint16_t)to[b];
+                        P.off_h[cls][nt] = (uint16_t)ro[a]; P.off_w[cls][nt] = (uint16_t)to[b];
                         C.r[nt] = rs[a]; C.t[nt] = tsv[b];
                         ++nt;
                     }
-                P.Hq = g.h / 2; P.Wq = g.w / 2; P.ts = 1; P.lo_w = P.lo_h = 0;
-                P.Hout = g.h; P.Wout = g.w; P.os = 2; P.oa = pa; P.ob = pb;
+                P.cls_oa[cls] = pa; P.cls_ob[cls] = pb;
             }
             C.ntaps = nt;
+            P.cls_ntaps[cls] = nt;
+            max_taps = std::max(max_taps, nt);
             off += (size_t)g.c_in * nt * g.c_out;
-            IgemmCfg c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, nt, g.c_in, sm_count);
-            if (!c.ok) { ok = false; break; }
-            S.cfg = c;
-            fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
-            P.ldo = g.c_in;
         }
-        if (ok) {
+        if (g.stride == 1) {
+            P.Hq = g.h; P.Wq = g.w; P.ts = 1; P.lo_w = P.lo_h = -(g.k - 1 - g.pad);
+            P.Hout = g.h; P.Wout = g.w; P.os = 1;
+        } else {
+            P.Hq = g.h / 2; P.Wq = g.w / 2; P.ts = 1; P.lo_w = P.lo_h = 0;
+            P.Hout = g.h; P.Wout = g.w; P.os = 2;
+        }
+        IgemmCfg c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls);
+        if (c.ok) {
+            tc->dg.cfg = c;
+            fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
+            P.nclasses = ncls; P.tiles_per_class = c.m_tiles * c.n_tiles;
+            P.ldo = g.c_in;
             W.nclasses = ncls;
-            tc->dg_classes = ncls;
             tc->wt_bytes = off * 2;
             tc->dgrad = true;
         }
@@ -869,7 +888,7 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC)) {
             return NB_ERR_CUDA;
         }
-        if (!encode_tiled_2d(&S.prm.tmB, w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
+        if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
@@ -889,22 +908,21 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         if (cudaGetLastError() != cudaSuccess) { err() = "launch of dgrad_weight_transform_kernel failed"; return NB_ERR_CUDA; }
         tc->launches += 1;
     }
-    for (int cls = 0; cls < tc->dg_classes; ++cls) {
-        TcGemmSlot& S = tc->dg[cls];
-        const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
-        if (S.a_ptr != dy || S.b_ptr != wcls) {
-            // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
-            const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
-            const int up = lo;
-            if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, up, 1, S.cfg.KC)) return NB_ERR_CUDA;
-            if (!encode_tiled_2d(&S.prm.tmB, wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
-            S.a_ptr = dy; S.b_ptr = wcls;
+    TcGemmSlot& S = tc->dg;
+    if (S.a_ptr != dy || S.b_ptr != wt) {
+        // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
+        const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
+        if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC)) return NB_ERR_CUDA;
+        for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
+            const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
+            if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
         }
-        S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
-        nb_status r = launch_igemm<__nv_bfloat16, false>(S, st);
-        if (r != NB_OK) return r;
-        tc->launches += 1;
+        S.a_ptr = dy; S.b_ptr = wt;
     }
+    S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
+    nb_status r = launch_igemm<__nv_bfloat16, false>(S, st);
+    if (r != NB_OK) return r;
+    tc->launches += 1;
     return NB_OK;
 }
 
