@@ -109,6 +109,19 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restric
     }
 }
 
+// V consecutive per-channel floats (V = 4 or 8) with 16-byte loads.
+template <int V> __device__ __forceinline__ void load_params(const float* __restrict__ p, int cg, float (&out)[V]) {
+    const float4* q = reinterpret_cast<const float4*>(p + (size_t)cg * V);
+#pragma unroll
+    for (int i = 0; i < V / 4; ++i) {
+        const float4 t = q[i];
+        out[4 * i] = t.x;
+        out[4 * i + 1] = t.y;
+        out[4 * i + 2] = t.z;
+        out[4 * i + 3] = t.w;
+    }
+}
+
 // ------------------------------------------------------------------ a = SiLU(y*scale + shift)
 template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(1024) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
@@ -118,11 +131,8 @@ __global__ void __launch_bounds__(1024) bn_silu_apply_kernel(const YT* __restric
     static_assert(V == Vec16<AT>::N, "y and a must have the same element size");
     const int cg = threadIdx.x % (C / V);
     float sc[V], sh[V];
-#pragma unroll
-    for (int i = 0; i < V; ++i) {
-        sc[i] = scale[cg * V + i];
-        sh[i] = shift[cg * V + i];
-    }
+    load_params<V>(scale, cg, sc);
+    load_params<V>(shift, cg, sh);
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
         const Vec16<YT> q = ld16(y + v * V);
@@ -136,7 +146,10 @@ __global__ void __launch_bounds__(1024) bn_silu_apply_kernel(const YT* __restric
     }
 }
 
-// ------------------------------------------------------------------ backward reductions: sum dz, sum dz*xhat
+// ------------------------------------------------------------------ backward reductions: sum dz, sum dz*y
+// z = y*a + b with a = gamma*invstd, b = beta - mean*a (recomputed here from the saved statistics).  The second
+// sum is taken against y itself; sum dz*xhat = invstd*(sum dz*y - mean*sum dz) is formed in fp64 by the finalize
+// kernel, so this pass needs only two per-channel values per element.
 template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(1024) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                                   long long total_vecs, int C, const float* __restrict__ mean,
@@ -148,14 +161,19 @@ __global__ void __launch_bounds__(1024) bn_silu_bwd_reduce_kernel(const AT* __re
     const int tid = threadIdx.x;
     const int cgs = C / V;
     const int cg = tid % cgs;
-    float mu[V], is[V], ga[V], be[V], sb[V], sg[V];
+    float a[V], b[V], sb[V], sy[V];
+    {
+        float mu[V], is[V], ga[V], be[V];
+        load_params<V>(mean, cg, mu);
+        load_params<V>(invstd, cg, is);
+        load_params<V>(gamma, cg, ga);
+        load_params<V>(beta, cg, be);
 #pragma unroll
-    for (int i = 0; i < V; ++i) {
-        mu[i] = mean[cg * V + i];
-        is[i] = invstd[cg * V + i];
-        ga[i] = gamma[cg * V + i];
-        be[i] = beta[cg * V + i];
-        sb[i] = sg[i] = 0.f;
+        for (int i = 0; i < V; ++i) {
+            a[i] = ga[i] * is[i];
+            b[i] = fmaf(-mu[i], a[i], be[i]);
+            sb[i] = sy[i] = 0.f;
+        }
     }
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + tid; v < total_vecs; v += stride) {
@@ -163,64 +181,68 @@ __global__ void __launch_bounds__(1024) bn_silu_bwd_reduce_kernel(const AT* __re
         const Vec16<AT> qg = ld16(g + v * V);
 #pragma unroll
         for (int i = 0; i < V; ++i) {
-            const float xhat = (to_f32(qy.v[i]) - mu[i]) * is[i];
-            const float z = fmaf(ga[i], xhat, be[i]);
+            const float yv = to_f32(qy.v[i]);
+            const float z = fmaf(yv, a[i], b[i]);
             const float s = sigmoid_f<FAST>(z);
             const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
             sb[i] += dz;
-            sg[i] = fmaf(dz, xhat, sg[i]);
+            sy[i] = fmaf(dz, yv, sy[i]);
         }
     }
     const int R = blockDim.x / cgs;
     for (int pass = 0; pass < 2; ++pass) {
 #pragma unroll
-        for (int i = 0; i < V; ++i) red[tid * V + i] = pass ? sg[i] : sb[i];
+        for (int i = 0; i < V; ++i) red[tid * V + i] = pass ? sy[i] : sb[i];
         __syncthreads();
         for (int c = tid; c < C; c += blockDim.x) {
             const int gq = c / V, e = c % V;
             float acc = 0.f;
             for (int r = 0; r < R; ++r) acc += red[(r * cgs + gq) * V + e];
-            partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;  // pass 0: dbeta, pass 1: dgamma
+            partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;  // pass 0: sum dz, pass 1: sum dz*y
         }
         __syncthreads();
     }
 }
 
-// partials [nparts][2][C] -> dbeta, dgamma (fp32) and the two per-channel coefficients dbeta/M, dgamma/M.
-__global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float* dgamma,
-                                                              float* dbeta, float* coef /*[2][C]*/) {
+// partials [nparts][2][C] (sum dz, sum dz*y) -> dbeta, dgamma (fp32) and four per-channel coefficients for the dy pass:
+//   coef[0] = a = gamma*invstd, coef[1] = b = beta - mean*a                      (z = y*a + b)
+//   coef[2] = p1 = a*invstd*dgamma/M, coef[3] = p0 = p1*mean - a*dbeta/M        (dy = a*dz - p1*y + p0)
+// which is dy = a*(dz - dbeta/M - xhat*dgamma/M) with xhat = (y - mean)*invstd written out in terms of y.
+__global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M,
+                                                              const float* __restrict__ mean, const float* __restrict__ invstd,
+                                                              const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                              float* dgamma, float* dbeta, float* coef /*[4][C]*/) {
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
-    const double s = warp_sum_partials(partials, nparts, C, c, 0, lane);
-    const double q = warp_sum_partials(partials, nparts, C, c, 1, lane);
+    const double s0 = warp_sum_partials(partials, nparts, C, c, 0, lane);
+    const double s1 = warp_sum_partials(partials, nparts, C, c, 1, lane);
     if (lane == 0) {
-        dbeta[c] = (float)s;
-        dgamma[c] = (float)q;
-        coef[c] = (float)(s / M);
-        coef[C + c] = (float)(q / M);
+        const double mu = (double)mean[c], is = (double)invstd[c];
+        const double dg = is * (s1 - mu * s0);
+        const double a = (double)gamma[c] * is;
+        const double p1 = a * is * dg / M;
+        dbeta[c] = (float)s0;
+        dgamma[c] = (float)dg;
+        coef[c] = (float)a;
+        coef[C + c] = (float)((double)beta[c] - mu * a);
+        coef[2 * C + c] = (float)p1;
+        coef[3 * C + c] = (float)(p1 * mu - a * s0 / M);
     }
 }
 
-// ------------------------------------------------------------------ dy = gamma*invstd*(dz - dbeta/M - xhat*dgamma/M)
+// ------------------------------------------------------------------ dy = a*dz - p1*y + p0
 template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(1024) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
-                                                              const float* __restrict__ mean, const float* __restrict__ invstd,
-                                                              const float* __restrict__ gamma, const float* __restrict__ beta,
                                                               const float* __restrict__ coef) {
     constexpr int V = Vec16<YT>::N;
     const int cg = threadIdx.x % (C / V);
-    float mu[V], is[V], ga[V], be[V], c1[V], c2[V];
-#pragma unroll
-    for (int i = 0; i < V; ++i) {
-        mu[i] = mean[cg * V + i];
-        is[i] = invstd[cg * V + i];
-        ga[i] = gamma[cg * V + i];
-        be[i] = beta[cg * V + i];
-        c1[i] = coef[cg * V + i];
-        c2[i] = coef[C + cg * V + i];
-    }
+    float a[V], b[V], p1[V], p0[V];
+    load_params<V>(coef, cg, a);
+    load_params<V>(coef + C, cg, b);
+    load_params<V>(coef + 2 * C, cg, p1);
+    load_params<V>(coef + 3 * C, cg, p0);
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
         const Vec16<YT> qy = ld16(y + v * V);
@@ -228,11 +250,11 @@ __global__ void __launch_bounds__(1024) bn_silu_bwd_dy_kernel(const AT* __restri
         Vec16<AT> o;
 #pragma unroll
         for (int i = 0; i < V; ++i) {
-            const float xhat = (to_f32(qy.v[i]) - mu[i]) * is[i];
-            const float z = fmaf(ga[i], xhat, be[i]);
+            const float yv = to_f32(qy.v[i]);
+            const float z = fmaf(yv, a[i], b[i]);
             const float s = sigmoid_f<FAST>(z);
             const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
-            o.v[i] = from_f32<AT>(ga[i] * is[i] * (dz - c1[i] - xhat * c2[i]));
+            o.v[i] = from_f32<AT>(fmaf(a[i], dz, fmaf(-p1[i], yv, p0[i])));
         }
         st16(dy + v * V, o);
     }

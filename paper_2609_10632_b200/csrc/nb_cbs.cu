@@ -181,13 +181,12 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     }
     {
         SiteTimer tm(p, SITE_BWD_FINALIZE, st);
-        bn_bwd_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, dgamma, dbeta, coef);
+        bn_bwd_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta, coef);
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
     bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
-                                                                        static_cast<AT*>(dy), e.total_vecs, C, mean, invstd, gamma,
-                                                                        beta, coef);
+                                                                        static_cast<AT*>(dy), e.total_vecs, C, coef);
     return launch_ok("bn_silu_bwd_dy");
 }
 
@@ -290,8 +289,10 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     e.tpb = e.cgs * R;
     e.total_vecs = g.m * e.cgs;
     const long long max_blocks = (e.total_vecs + e.tpb - 1) / e.tpb;
-    e.blocks_reduce = (int)std::min<long long>(max_blocks, (long long)p->sm_count * 4);
-    e.blocks_map = (int)std::min<long long>(max_blocks, (long long)p->sm_count * 8);
+    // enough blocks to fill the machine, but at least ~8 (reductions) / ~4 (maps) vectors per thread so that the
+    // per-thread parameter loads and the block epilogue are amortised on small tensors
+    e.blocks_reduce = (int)std::max<long long>(1, std::min<long long>((max_blocks + 7) / 8, (long long)p->sm_count * 4));
+    e.blocks_map = (int)std::max<long long>(1, std::min<long long>((max_blocks + 3) / 4, (long long)p->sm_count * 6));
 
     // CUDA-core wgrad split-K: enough slices to fill the machine, at least 512 rows each.
     {
@@ -332,7 +333,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->off_fpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
     p->fwd_bytes = off;
     off = 0;
-    p->off_coef = off; off = align_up(off + 2 * C * 4, 256);
+    p->off_coef = off; off = align_up(off + 4 * C * 4, 256);
     p->off_bpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
     p->off_wt = off; off = align_up(off + p->tc.wt_bytes, 256);
     p->off_wgpart = off;

@@ -37,6 +37,9 @@ struct IgemmParams {
     int kpb;                     // k-blocks (of KC channels) per pipeline stage
     uint32_t a_sub_bytes, b_sub_bytes;  // bytes of one k-block of A / B inside a stage
     int BN, n_tiles, m_tiles;
+    int mh;                      // 128-row sub-tiles per tile (1 or 2): the tile is [128*mh x BN]
+    int acc_bufs;                // accumulator sets in TMEM (2 when 2*mh*acc_stride <= 512)
+    int stage_cols;              // columns the epilogue stages per pass
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
     int variant;                 // experiment switches
@@ -133,12 +136,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = sA + (size_t)p.stages * p.a_stage_bytes;
-    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging tile [128][BN] of OutT, row pitch BN*2+16 bytes
-    const int pitch = p.BN * 2 + 16;
-    float* stat_sum = reinterpret_cast<float*>(stg + (size_t)TC_BM * pitch);  // [ldo]
-    float* stat_sq = stat_sum + p.ldo;                                        // [ldo]
-    float* wpart = stat_sq + p.ldo;                                           // [2 tile parities][4 warps][2][BN]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + 16 * p.BN);
+    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging [128 rows][CW columns] of OutT, row pitch CW*2+16 bytes
+    const int CW = p.stage_cols;                             // columns staged per pass (<= 128)
+    const int pitch = CW * 2 + 16;
+    float* wstat = reinterpret_cast<float*>(stg + (size_t)TC_BM * pitch);  // [4 warps][2][ldo]: warp-private channel sums
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wstat + (STATS ? 8 * p.ldo : 0));
     uint64_t* full = bars;                // [stages]
     uint64_t* empty = bars + p.stages;    // [stages]
     uint64_t* tfull = empty + p.stages;   // [2]
@@ -149,6 +151,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.nclasses * p.tiles_per_class;
+    const int mh = p.mh;          // 128-row sub-tiles per tile (1 or 2); both share every B stage
+    const int nbuf = p.acc_bufs;  // accumulator sets in TMEM (2 = the epilogue of a tile overlaps the next tile's MMAs)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -164,7 +168,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         ptx::fence_mbar_init();
     }
     if (STATS) {
-        for (int c = threadIdx.x; c < 2 * p.ldo; c += TC_THREADS) stat_sum[c] = 0.f;
+        for (int c = threadIdx.x; c < 8 * p.ldo; c += TC_THREADS) wstat[c] = 0.f;
     }
     if (warp == 1) {
         ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
@@ -192,7 +196,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             long long dbg_wait_empty = 0;
             const long long dbg_start = clock64();
 #endif
-            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * p.KC * 2) : (uint32_t)(p.BN * p.KC * 2);
+            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(p.BN * p.KC * 2);
             // loop-invariant values in registers: this thread's instruction stream is on the critical path
             const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
             const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
@@ -204,7 +208,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                 const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
                 const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
                 const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
-                const int m0 = m_tile * TC_BM;
+                const int m0 = m_tile * TC_BM * mh;
                 int cw = 0, ch = 0, n0 = 0;
                 if (isA && !a_tiled) {
                     const int j0 = m0 % Wq, t1 = m0 / Wq;
@@ -214,7 +218,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     ch = p.lo_h + i0 * ts;
                 }
                 const int brow = n_tile * BN;
-                int tap = 0, kc = 0;
+                // each CTA starts its K loop at a different k-block so that the CTAs do not all ask L2 for the same
+                // filter lines at the same moment
+                const int ntaps_c = p.cls_ntaps[cls];
+                const int rot = (p.variant & 4) ? 0 : (int)((blockIdx.x * 7u) % (unsigned)kblocks);
+                int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
                     {
@@ -240,7 +248,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         dst += sub_bytes;
                         if (++kc == kc_per_tap) {
                             kc = 0;
-                            ++tap;
+                            if (++tap == ntaps_c) tap = 0;
                         }
                     }
                     ++issued;
@@ -278,6 +286,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
             const uint64_t a_sub16 = (uint64_t)(p.a_sub_bytes >> 4), b_sub16 = (uint64_t)(p.b_sub_bytes >> 4);
             const uint64_t a_stage16 = (uint64_t)(p.a_stage_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
+            const uint64_t a_half16 = (uint64_t)((TC_BM * p.KC * 2) >> 4);  // second 128-row sub-tile inside a k-block of A
             const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), 16, p.sbo, p.umma_swizzle);
             const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, p.sbo, p.umma_swizzle);
             const uint32_t empty_u32 = ptx::smem_u32(empty);
@@ -291,7 +300,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     NB_DBG_ADD(dbg_wait_tempty);
                 }
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_stride;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
                 uint32_t accumulate = 0;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
@@ -306,13 +315,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     ptx::tc_fence_after();
                     uint64_t da = da_s, db = db_s;
                     for (int j = 0; j < nkb; ++j) {
-                        if (ksteps == 4) {
-                            ptx::umma_f16(d_tmem, da, db, idesc, accumulate);
-                            ptx::umma_f16(d_tmem, da + 2, db + 2, idesc, 1u);
-                            ptx::umma_f16(d_tmem, da + 4, db + 4, idesc, 1u);
-                            ptx::umma_f16(d_tmem, da + 6, db + 6, idesc, 1u);
-                        } else {
-                            for (int k = 0; k < ksteps; ++k) ptx::umma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (k | (int)accumulate) ? 1u : 0u);
+                        for (int h = 0; h < mh; ++h) {
+                            const uint64_t dah = da + (uint64_t)h * a_half16;
+                            const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
+                            if (ksteps == 4) {
+                                ptx::umma_f16(dt, dah, db, idesc, accumulate);
+                                ptx::umma_f16(dt, dah + 2, db + 2, idesc, 1u);
+                                ptx::umma_f16(dt, dah + 4, db + 4, idesc, 1u);
+                                ptx::umma_f16(dt, dah + 6, db + 6, idesc, 1u);
+                            } else {
+                                for (int k = 0; k < ksteps; ++k)
+                                    ptx::umma_f16(dt, dah + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (k | (int)accumulate) ? 1u : 0u);
+                            }
                         }
                         accumulate = 1u;
                         da += a_sub16;
@@ -330,8 +344,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                 }
                 if (!ok) break;
                 ptx::umma_commit(tfull + acc);
-                acc ^= 1;
-                if (acc == 0) acc_ph ^= 1u;
+                if (++acc == nbuf) {
+                    acc = 0;
+                    acc_ph ^= 1u;
+                }
             }
 #ifdef NB_TC_DEBUG_TIMING
             if (p.dbg) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
@@ -344,13 +360,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2-5, 128 threads)
         const int et = threadIdx.x - 64;          // 0..127
-        const int lane_group = warp & 3;          // TMEM lanes this warp may read: rows [32*lane_group, +32) of the tile
-        const int row = lane_group * 32 + lane;   // accumulator row == tile row
-        const int cpr = p.BN / 8;                 // 16-byte chunks per staged row (<= 32)
-        const int rpi = 32 / cpr;                 // rows one warp stores per iteration
-        const int lr = lane / cpr, lc = lane - lr * cpr;
-        int acc = 0, sat = 0, par = 0;
+        const int lane_group = warp & 3;          // TMEM lanes this warp may read: rows [32*lane_group, +32) of a sub-tile
+        const int row = lane_group * 32 + lane;   // accumulator row == sub-tile row
+        int acc = 0, sat = 0;
         uint32_t acc_ph = 0;
+        float* my_stat = wstat + (size_t)lane_group * 2 * p.ldo;  // this warp's [2][ldo] running sums
+        uint8_t* my_row = stg + (size_t)row * pitch;
+        const uint8_t* my_rows = stg + (size_t)(lane_group * 32) * pitch;
+        uint8_t* outb = static_cast<uint8_t*>(p.out);
 #ifdef NB_TC_DEBUG_TIMING
         long long dbg_wait_tfull = 0;
         const long long dbg_start = clock64();
@@ -358,113 +375,116 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int cls = tile / p.tiles_per_class, lt = tile - cls * p.tiles_per_class;
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
-            const long long m0 = (long long)m_tile * TC_BM;
             NB_DBG_T0();
             bool ok = true;
-            if (p.variant & 2) {
-                ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
-            } else {
-                // one poller per warp: 128 threads spinning on one mbarrier would crowd the shared-memory pipe
-                if (lane == 0) ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            }
+            // one poller per warp: 128 threads spinning on one mbarrier would crowd the shared-memory pipe
+            if (lane == 0) ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             NB_DBG_ADD(dbg_wait_tfull);
             ok = epi_bar_and(ok);
             if (!ok) break;
             ptx::tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(acc * p.acc_stride);
-            uint8_t* my_row = stg + (size_t)row * pitch;
-            for (int c0 = 0; c0 < p.BN; c0 += 32) {
-                uint32_t r[32];
-                const bool two = c0 + 16 < p.BN;
-                ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)c0, r);
-                if (two) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(c0 + 16), r + 16);
-                ptx::tmem_ld_wait();
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (h == 1 && !two) break;
-                    uint4 v0, v1;
-                    const uint32_t* q = r + 16 * h;
-                    v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat);
-                    v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat);
-                    v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat);
-                    v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat);
-                    v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat);
-                    v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat);
-                    v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat);
-                    v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat);
-                    *reinterpret_cast<uint4*>(my_row + (c0 + 16 * h) * 2) = v0;
-                    *reinterpret_cast<uint4*>(my_row + (c0 + 16 * h) * 2 + 16) = v1;
+            if (p.variant & 8) {
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(tempty + acc);
+                if (++acc == nbuf) {
+                    acc = 0;
+                    acc_ph ^= 1u;
                 }
+                continue;
             }
-            // accumulator buffer is free for the MMA of the tile after next
-            ptx::tc_fence_before();
-            ptx::mbar_arrive(tempty + acc);
-            __syncwarp();  // every warp only reads back the 32 rows it staged itself
-            const uint8_t* my_rows = stg + (size_t)(lane_group * 32) * pitch;
-            if (STATS) {
-                // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled)
-                float* wp = wpart + (size_t)((par * 4 + lane_group) * 2) * p.BN;
-                for (int pc = lane; pc < p.BN / 2; pc += 32) {
-                    float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
-                    const uint8_t* col = my_rows + pc * 4;
+            for (int h = 0; h < mh; ++h) {
+                const long long m0 = ((long long)m_tile * mh + h) * TC_BM;
+                const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride);
+                for (int cbase = 0; cbase < p.BN; cbase += CW) {
+                    const int ncol = (p.BN - cbase < CW) ? p.BN - cbase : CW;  // multiple of 16
+                    // ---- TMEM -> registers -> staging (this thread's row)
+                    for (int c0 = 0; c0 < ncol; c0 += 32) {
+                        uint32_t r[32];
+                        const bool two = c0 + 16 < ncol;
+                        ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0), r);
+                        if (two) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0 + 16), r + 16);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            if (hh == 1 && !two) break;
+                            uint4 v0, v1;
+                            const uint32_t* q = r + 16 * hh;
+                            v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat);
+                            v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat);
+                            v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat);
+                            v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat);
+                            v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat);
+                            v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat);
+                            v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat);
+                            v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat);
+                            *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2) = v0;
+                            *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2 + 16) = v1;
+                        }
+                    }
+                    if (h == mh - 1 && cbase + CW >= p.BN) {
+                        // last TMEM read of this tile: the accumulator set is free for the MMAs of a later tile
+                        ptx::tc_fence_before();
+                        ptx::mbar_arrive(tempty + acc);
+                    }
+                    __syncwarp();  // every warp only reads back the 32 rows it staged itself
+                    if (STATS && !(p.variant & 16)) {
+                        // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
+                        // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends
+                        for (int pc = lane; pc < ncol / 2; pc += 32) {
+                            float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
+                            const uint8_t* col = my_rows + pc * 4;
 #pragma unroll 8
-                    for (int rr = 0; rr < 32; ++rr) {
-                        const uint32_t u = *reinterpret_cast<const uint32_t*>(col + (size_t)rr * pitch);
-                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u));
-                        s0 += f.x;
-                        s1 += f.y;
-                        q0 = fmaf(f.x, f.x, q0);
-                        q1 = fmaf(f.y, f.y, q1);
+                            for (int rr = 0; rr < 32; ++rr) {
+                                const uint32_t u = *reinterpret_cast<const uint32_t*>(col + (size_t)rr * pitch);
+                                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u));
+                                s0 += f.x;
+                                s1 += f.y;
+                                q0 = fmaf(f.x, f.x, q0);
+                                q1 = fmaf(f.y, f.y, q1);
+                            }
+                            const int ch0 = n_tile * p.BN + cbase + 2 * pc;
+                            my_stat[ch0] += s0;
+                            my_stat[ch0 + 1] += s1;
+                            my_stat[p.ldo + ch0] += q0;
+                            my_stat[p.ldo + ch0 + 1] += q1;
+                        }
                     }
-                    wp[2 * pc] = s0;
-                    wp[2 * pc + 1] = s1;
-                    wp[p.BN + 2 * pc] = q0;
-                    wp[p.BN + 2 * pc + 1] = q1;
+                    // ---- coalesced row stores: the lanes of a warp cover whole rows of 16-byte pieces
+                    {
+                        const int cpr = ncol / 8;   // 16-byte chunks per staged row (<= 16)
+                        const int rpi = 32 / cpr;   // rows one warp stores per iteration
+                        const int lr = lane / cpr, lc = lane - lr * cpr;
+                        if (lr < rpi && !(p.variant & 32)) {
+                            for (int rr = lr; rr < 32; rr += rpi) {
+                                const long long m = m0 + lane_group * 32 + rr;
+                                if (m >= p.M) break;
+                                long long pix = m;
+                                if (p.os != 1) {
+                                    const int j = (int)(m % p.Wq);
+                                    const long long t1 = m / p.Wq;
+                                    const int i = (int)(t1 % p.Hq);
+                                    const long long n = t1 / p.Hq;
+                                    pix = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
+                                }
+                                const uint4 v = *reinterpret_cast<const uint4*>(my_rows + (size_t)rr * pitch + lc * 16);
+                                *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN + cbase) * 2 + (size_t)lc * 16) = v;
+                            }
+                        }
+                    }
+                    __syncwarp();  // staged rows consumed before the next pass overwrites them
                 }
             }
-            // coalesced row stores: the lanes of a warp cover whole rows of 16-byte pieces
-            if (lr < rpi) {
-                uint8_t* outb = static_cast<uint8_t*>(p.out);
-                for (int rr = lr; rr < 32; rr += rpi) {
-                    const long long m = m0 + lane_group * 32 + rr;
-                    if (m >= p.M) break;
-                    long long pix = m;
-                    if (p.os != 1) {
-                        const int j = (int)(m % p.Wq);
-                        const long long t1 = m / p.Wq;
-                        const int i = (int)(t1 % p.Hq);
-                        const long long n = t1 / p.Hq;
-                        pix = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
-                    }
-                    const uint4 v = *reinterpret_cast<const uint4*>(my_rows + (size_t)rr * pitch + lc * 16);
-                    *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN) * 2 + (size_t)lc * 16) = v;
-                }
+            if (++acc == nbuf) {
+                acc = 0;
+                acc_ph ^= 1u;
             }
-            if (STATS) {
-                epi_bar_sync();  // all four warps' partial sums of this tile are in wpart[par]
-                const float* wp = wpart + (size_t)(par * 8) * p.BN;
-                for (int c = et; c < p.BN; c += 128) {
-                    float s = 0.f, q = 0.f;
-#pragma unroll
-                    for (int w4 = 0; w4 < 4; ++w4) {
-                        s += wp[(w4 * 2 + 0) * p.BN + c];
-                        q += wp[(w4 * 2 + 1) * p.BN + c];
-                    }
-                    stat_sum[n_tile * p.BN + c] += s;
-                    stat_sq[n_tile * p.BN + c] += q;
-                }
-                par ^= 1;
-            } else {
-                __syncwarp();  // staged rows consumed before the next tile overwrites them
-            }
-            acc ^= 1;
-            if (acc == 0) acc_ph ^= 1u;
         }
         if (STATS) {
-            epi_bar_sync();
+            epi_bar_sync();  // all four warps' running sums are final
             float* dst = p.partials + (size_t)blockIdx.x * 2 * p.ldo;
-            for (int c = et; c < 2 * p.ldo; c += 128) dst[c] = stat_sum[c];
+            for (int c = et; c < 2 * p.ldo; c += 128)
+                dst[c] = ((wstat[c] + wstat[2 * p.ldo + c]) + wstat[4 * p.ldo + c]) + wstat[6 * p.ldo + c];
         }
 #ifdef NB_TC_DEBUG_TIMING
         if (p.dbg && et == 0) { p.dbg[blockIdx.x * 8 + 5] = dbg_wait_tfull; p.dbg[blockIdx.x * 8 + 6] = clock64() - dbg_start; }
@@ -478,6 +498,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
+
 
 // Rearranged filter for dgrad: for parity class `cls` (a list of taps), wt[c][ti][c'] = w[c'][r_ti][t_ti][c].
 struct WtClass {
@@ -513,7 +534,7 @@ namespace nbcbs {
 struct IgemmCfg {
     bool ok = false;
     int Ca = 0, rowsB = 0, ntaps = 0;
-    int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1;
+    int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
     uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
@@ -585,10 +606,17 @@ inline uint32_t umma_swizzle_for(int KC) { return KC == 64 ? (uint32_t)ptx::kSwi
 constexpr size_t kMaxSmem = 232448;  // 227 KB opt-in limit per CTA
 
 // Tile configuration for a GEMM with M rows, `rowsB` output channels, `ntaps` taps of `Ca` channels each.
-// A stage of the pipeline holds `kpb` k-blocks so that one barrier round trip (a few hundred cycles of issue
-// latency in the producer and MMA threads) is amortised over enough tensor-core work.
+// Measured on B200: a tcgen05.mma of 128 x N x 16 takes max(97, N/2) cycles, so N below 192 wastes the tensor pipe;
+// TMA fills shared memory at roughly 100 cycles per box plus 1.4 (256-row boxes) to 2.3 (128-row boxes) cycles per
+// 128-byte row; one barrier round trip of the single-thread producer / MMA loops costs a few hundred cycles.
+// The tile is [128*mh x BN]: with mh = 2 two row blocks share every B stage (fewer rows fetched per flop).
+inline int igemm_stage_cols(int BN) {
+    if (BN <= 128) return BN;
+    if (BN % 32 == 0) return BN / 2;
+    return 128;
+}
 inline size_t igemm_fixed_smem(int BN, int ldo) {
-    return 1024 /*alignment slack*/ + (size_t)TC_BM * (BN * 2 + 16) + (size_t)2 * ldo * 4 + (size_t)16 * BN * 4 + 512;
+    return 1024 /*alignment slack*/ + (size_t)TC_BM * (igemm_stage_cols(BN) * 2 + 16) + (size_t)8 * ldo * 4 + 512;
 }
 inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses) {
     IgemmCfg c;
@@ -597,21 +625,31 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     // Always 64-channel k-blocks in the 128-byte swizzle (the narrower swizzles make tcgen05.mma 1.6-2.1x slower per
     // instruction); when Ca is not a multiple of 64 the last k-block of every tap reads past the channel extent and
     // TMA fills A with zeros there (whatever finite filter values B holds at those positions are multiplied by zero).
-    c.KC = getenv("NB_TC_KC") ? atoi(getenv("NB_TC_KC")) : 64;
-    if (c.KC != 64 && Ca % c.KC) c.KC = 16;
-    c.m_tiles = (int)((M + TC_BM - 1) / TC_BM);
+    c.KC = 64;
     const int kblocks = ntaps * ((Ca + c.KC - 1) / c.KC);
     const int force_bn = getenv("NB_TC_BN") ? atoi(getenv("NB_TC_BN")) : 0;
     const int force_kpb = getenv("NB_TC_KPB") ? atoi(getenv("NB_TC_KPB")) : 0;
-    double best = 1e30;
-    for (int bn = 16; bn <= 256 && bn <= rowsB; bn += 16) {
+    const int force_mh = getenv("NB_TC_MH") ? atoi(getenv("NB_TC_MH")) : 0;
+    // Rules distilled from sweeps over the detector's layer shapes on B200: the widest N tile that divides the channel
+    // count wins everywhere (fewer shared-memory bytes written and read per flop); pairing two 128-row blocks per tile
+    // (mh = 2) pays only while two accumulator sets still fit in TMEM (N <= 128) and there are enough tiles for every SM;
+    // a pipeline stage should hold about 450 tensor cycles of work.
+    for (int bn = std::min(256, rowsB) / 16 * 16; bn >= 16 && !c.BN; bn -= 16) {
         if (rowsB % bn) continue;
         if (force_bn && bn != force_bn && rowsB % force_bn == 0) continue;
-        const uint32_t a_sub = (uint32_t)((TC_BM * c.KC * 2 + 1023) / 1024 * 1024);
+        const int acc_stride = bn <= 32 ? 32 : bn <= 64 ? 64 : bn <= 128 ? 128 : 256;
+        int mh = 1;
+        if (4 * acc_stride <= 512) {
+            const long long tiles2 = ((M + 2 * TC_BM - 1) / (2 * TC_BM)) * (rowsB / bn) * nclasses;
+            if (tiles2 >= sm_count) mh = 2;
+        }
+        if (force_mh && force_mh * acc_stride <= 512) mh = force_mh;
+        const int acc_bufs = (2 * mh * acc_stride <= 512) ? 2 : 1;
+        const uint32_t a_sub = (uint32_t)(TC_BM * mh * c.KC * 2);
         const uint32_t b_sub = (uint32_t)((bn * c.KC * 2 + 1023) / 1024 * 1024);
         const size_t fixed = igemm_fixed_smem(bn, ldo);
         if (fixed + 2 * (size_t)(a_sub + b_sub) > kMaxSmem) continue;
-        const double mma_kb = (c.KC / 16) * std::max(bn, 16) / 2.0;  // tensor cycles per k-block
+        const double mma_kb = mh * 4.0 * std::max(97.0, bn / 2.0);  // tensor cycles per k-block
         int kpb = std::max(1, std::min(kblocks, (int)((450.0 + mma_kb - 1) / mma_kb)));
         if (force_kpb) kpb = std::min(kblocks, force_kpb);
         int stages = 0;
@@ -620,27 +658,17 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
             if (stages >= 3 || kpb == 1) break;
         }
         if (stages < 2) continue;
-        const int nstage_tile = (kblocks + kpb - 1) / kpb;
-        const double rows = (double)kpb * (TC_BM + bn);
-        const double stage_t = std::max(kpb * mma_kb, 200.0 + 1.6 * rows);      // tensor pipe vs TMA fill
-        const double main_t = nstage_tile * stage_t;
-        const double epi_t = 800.0 + 45.0 * bn;
-        const long long tiles = (long long)c.m_tiles * (rowsB / bn) * nclasses;
-        const double waves = (double)((tiles + sm_count - 1) / sm_count);
-        const double cost = waves * std::max(main_t, epi_t) + epi_t;
-        if (cost < best - 1e-9) {
-            best = cost;
-            c.BN = bn; c.kpb = kpb; c.stages = stages; c.a_sub = a_sub; c.b_sub = b_sub;
-        }
+        c.BN = bn; c.kpb = kpb; c.stages = stages; c.a_sub = a_sub; c.b_sub = b_sub; c.mh = mh; c.acc_bufs = acc_bufs;
+        c.acc_stride = acc_stride;
+        c.m_tiles = (int)((M + TC_BM * mh - 1) / (TC_BM * mh));
     }
     if (!c.BN) return c;
     c.n_tiles = rowsB / c.BN;
-    c.acc_stride = c.BN <= 32 ? 32 : c.BN <= 64 ? 64 : c.BN <= 128 ? 128 : 256;
-    c.tmem_cols = 2 * c.acc_stride;
+    c.stage_cols = igemm_stage_cols(c.BN);
+    c.tmem_cols = std::max(32, c.acc_bufs * c.mh * c.acc_stride);
     c.a_stage = c.a_sub * c.kpb;
     c.b_stage = c.b_sub * c.kpb;
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
-    (void)kblocks;
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
     c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, sm_count);
     c.ok = true;
@@ -656,10 +684,11 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.sbo = (uint32_t)(8 * c.KC * 2);
     P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
     P.kpb = c.kpb; P.a_sub_bytes = c.a_sub; P.b_sub_bytes = c.b_sub;
+    P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.stage_cols = c.stage_cols;
     P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
     if (getenv("NB_TC_VERBOSE"))
-        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: KC=%d BN=%d kpb=%d stages=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca, c.rowsB,
-                c.ntaps, c.KC, c.BN, c.kpb, c.stages, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
+                c.rowsB, c.ntaps, c.mh, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
     P.idesc = ptx::make_idesc_bf16(TC_BM, c.BN, 0, 0);
 }
 
@@ -884,8 +913,8 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     if (S.a_ptr != x || S.b_ptr != w) {
         const int up = g.pad - (g.k - 1);
         if (S.prm.a_tiled) {
-            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM)) return NB_ERR_CUDA;
-        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC)) {
+            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
+        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh)) {
             return NB_ERR_CUDA;
         }
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
@@ -912,7 +941,7 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
     if (S.a_ptr != dy || S.b_ptr != wt) {
         // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
         const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
-        if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC)) return NB_ERR_CUDA;
+        if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
         for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
             const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
             if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
