@@ -95,7 +95,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -138,32 +138,34 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- CPU oracle timing
 def time_oracle(layers, budget_s: float):
-    """Time the oracle (forward + backward of whole blocks) on a bounded sample: the layers at batch 1, and if that
-    is still over budget a prefix of the distinct shapes.  Returns (TFLOP/s, seconds, flops, cores, description)."""
-    import numpy as np
-
+    """Time the oracle (forward + backward of whole blocks) on a bounded sample of the workload: every distinct layer
+    shape once, at a reduced batch chosen so that the pass takes roughly `budget_s` seconds (batch 1 is timed first to
+    size it).  Returns (TFLOP/s, seconds, flops, cores, description)."""
     import oracle
     from paper_2609_10632_b200 import workloads as wl
 
     oracle.build()
     cores = oracle.num_threads()
-    rate = 15e9  # conservative estimate of the oracle's flop rate, only used to size the sample
-    distinct = wl.distinct_shapes([s.with_batch(1) if s.n > 1 else s for s in layers])
-    chosen, est = [], 0.0
-    for s, mult in distinct:
-        f = 3 * s.gemm_flops
-        if chosen and est + f / rate > budget_s:
-            continue
-        chosen.append((s, mult))
-        est += f / rate
-    flops, secs = 0.0, 0.0
-    for i, (s, mult) in enumerate(chosen):
-        inp = wl.make_inputs(s, cfg_id=5, layer_id=i, bf16=True)
-        t0 = time.perf_counter()
-        oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, 1e-3)
-        secs += time.perf_counter() - t0
-        flops += 3 * s.gemm_flops
-    desc = f"{len(chosen)} of {len(distinct)} distinct layer shapes at batch {chosen[0][0].n}, one fwd+bwd each, fp64 direct loops"
+
+    def one_pass(batch):
+        distinct = wl.distinct_shapes([s.with_batch(min(batch, s.n)) for s in layers])
+        flops, secs = 0.0, 0.0
+        for i, (s, _mult) in enumerate(distinct):
+            inp = wl.make_inputs(s, cfg_id=5, layer_id=i, bf16=True)
+            t0 = time.perf_counter()
+            oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, 1e-3)
+            secs += time.perf_counter() - t0
+            flops += 3 * s.gemm_flops
+        return flops, secs, len(distinct)
+
+    full_batch = max(s.n for s in layers)
+    flops, secs, nshapes = one_pass(1)
+    batch = 1
+    if full_batch > 1 and secs > 0:
+        batch = int(max(1, min(full_batch, budget_s / secs)))
+        if batch > 1:
+            flops, secs, nshapes = one_pass(batch)
+    desc = f"{nshapes} distinct layer shapes at batch {batch} (of {full_batch}), one fwd+bwd each, fp64 direct loops"
     return flops / secs / 1e12, secs, flops, cores, desc
 
 
@@ -173,7 +175,7 @@ def run_reference(args):
         return
     layers = workload_layers(args.workload)
     total = args.steps + args.warmup
-    budget = max(2.0, min(30.0, 150.0 / max(1, total)))
+    budget = max(1.0, min(30.0, 120.0 / max(1, total)))
     vals, secs_all = [], []
     desc, cores = "", 0
     for i in range(total):
@@ -197,7 +199,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg5", help="cfg1..cfg5 (cfg5 = the detector's 77 Conv-BN-SiLU layers at batch 16)")
@@ -206,6 +208,7 @@ def main():
     ap.add_argument("--no-profile", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--force-simt", action="store_true", help="run the convolutions on the CUDA-core kernels")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph of one step")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -258,15 +261,41 @@ def main():
     for b in blocks:
         b.poll()
     barrier()
+    # The step is launch-bound on its small layers (about 770 kernels): capture one step of C-ABI calls into a CUDA
+    # graph and replay it.  Every call only enqueues kernels on the current stream, so the capture holds exactly the
+    # kernels an eager step launches.
+    l0 = nb.nb_cbs_launch_count()
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            one_step()
+        torch.cuda.current_stream().wait_stream(side)
+        l0 = nb.nb_cbs_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_step()
+        launches_per_step = nb.nb_cbs_launch_count() - l0
+        run_step = graph.replay
+        for _ in range(2):
+            run_step()
+    else:
+        run_step = one_step
+        launches_per_step = None
+    barrier()
+    stream = torch.cuda.current_stream()
     l0 = nb.nb_cbs_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         ev0.record(stream)
         for _ in range(args.steps):
-            one_step()
+            run_step()
         ev1.record(stream)
         barrier()
-    launches = nb.nb_cbs_launch_count() - l0
+    launches = launches_per_step * args.steps if launches_per_step is not None else nb.nb_cbs_launch_count() - l0
+    for b in blocks:
+        b.poll()
     ms_total = ev0.elapsed_time(ev1)
     if dist is not None:
         t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
@@ -349,7 +378,7 @@ def main():
                 "workload": f"{args.workload}: {len(layers)} Conv-BN-SiLU layers, batch {layers[0].n}, fwd + bwd_data + bwd_weight per layer "
                             f"(stem data gradient included), each layer on its own tensors",
                 "l2_policy": f"inputs larger than L2: {resident / 1e9:.2f} GB of tensors are touched per step",
-                "gflop_per_step": flops / 1e9, "multi_gpu": "replicas only", "tensor_core_layers": paths, "layers": len(layers),
+                "gflop_per_step": flops / 1e9, "multi_gpu": "replicas only", "cuda_graph": graph is not None, "tensor_core_layers": paths, "layers": len(layers),
                 "frac_of_nominal_bf16_peak": value / world / NOMINAL["bf16_tflops"],
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },

@@ -52,7 +52,8 @@ const char* const kSiteNames[SITE_COUNT] = {"conv_fprop", "bn_stats", "bn_finali
 struct EwCfg {  // launch geometry of the [M][C] passes
     int vec, cgs, tpb;
     long long total_vecs;
-    int blocks_reduce, blocks_map;
+    int blocks_reduce, blocks_map;  // stats / backward-reduce grids (they size the partial buffers) and apply / dy grids
+    int blocks_stats, blocks_apply, blocks_dy;
 };
 
 }  // namespace
@@ -143,7 +144,7 @@ nb_status launch_ok(const char* what) {
 template <typename YT> nb_status run_stats_partial(nb_cbs_plan_s* p, const void* y, float* partials, cudaStream_t st) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_STATS, st);
-    bn_stats_partial_kernel<YT><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+    bn_stats_partial_kernel<YT><<<e.blocks_stats, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
         static_cast<const YT*>(y), e.total_vecs, p->g.c_out, partials);
     return launch_ok("bn_stats_partial");
 }
@@ -162,7 +163,7 @@ template <typename YT, typename AT, bool FAST>
 nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_APPLY, st);
-    bn_silu_apply_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
+    bn_silu_apply_kernel<YT, AT, FAST><<<e.blocks_apply, e.tpb, 0, st>>>(static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
                                                                        p->g.c_out, scale, shift);
     return launch_ok("bn_silu_apply");
 }
@@ -185,7 +186,7 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
-    bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_map, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
+    bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_dy, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
                                                                         static_cast<AT*>(dy), e.total_vecs, C, coef);
     return launch_ok("bn_silu_bwd_dy");
 }
@@ -255,7 +256,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     if (!(d->momentum >= 0.f && d->momentum <= 1.f)) return fail(NB_ERR_INVALID_ARG, "momentum must be in [0,1]");
     const int vec = d->mode == NB_MODE_F32_REF ? 4 : 8;
     if (d->c_out % vec) return fail(NB_ERR_UNSUPPORTED, "c_out=%d must be a multiple of %d in this mode", d->c_out, vec);
-    if (d->c_out / vec > 1024) return fail(NB_ERR_UNSUPPORTED, "c_out=%d is too large", d->c_out);
+    if (d->c_out / vec > 288) return fail(NB_ERR_UNSUPPORTED, "c_out=%d is too large (at most %d channels in this mode)", d->c_out, 288 * vec);
 
     Geom g;
     g.n = d->n; g.h = d->h; g.w = d->w; g.c_in = d->c_in; g.c_out = d->c_out; g.k = d->ksize; g.stride = d->stride;
@@ -291,8 +292,29 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     const long long max_blocks = (e.total_vecs + e.tpb - 1) / e.tpb;
     // enough blocks to fill the machine, but at least ~8 (reductions) / ~4 (maps) vectors per thread so that the
     // per-thread parameter loads and the block epilogue are amortised on small tensors
-    e.blocks_reduce = (int)std::max<long long>(1, std::min<long long>((max_blocks + 7) / 8, (long long)p->sm_count * 4));
-    e.blocks_map = (int)std::max<long long>(1, std::min<long long>((max_blocks + 3) / 4, (long long)p->sm_count * 6));
+    // Grids are one wave of resident blocks (occupancy queried per kernel), but never so many that a thread sees fewer
+    // than ~8 (reductions) / ~4 (maps) vectors: the per-thread parameter loads and block epilogues must be amortised.
+    {
+        auto wave = [&](const void* fn, size_t dyn_smem, int min_vecs) {
+            int occ = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, e.tpb, dyn_smem) != cudaSuccess || occ < 1) occ = 2;
+            const long long cap = (long long)p->sm_count * occ;
+            return (int)std::max<long long>(1, std::min<long long>((max_blocks + min_vecs - 1) / min_vecs, cap));
+        };
+        const size_t red_smem = (size_t)e.tpb * vec * sizeof(float);
+        if (d->mode == NB_MODE_F32_REF) {
+            e.blocks_stats = wave((const void*)bn_stats_partial_kernel<float>, red_smem, 8);
+            e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<float, float, false>, red_smem, 8);
+            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<float, float, false>, 0, 4);
+            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<float, float, false>, 0, 4);
+        } else {
+            e.blocks_stats = wave((const void*)bn_stats_partial_kernel<__half>, red_smem, 8);
+            e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<__half, __nv_bfloat16, true>, red_smem, 8);
+            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __nv_bfloat16, true>, 0, 4);
+            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __nv_bfloat16, true>, 0, 4);
+        }
+        e.blocks_map = std::max(e.blocks_apply, e.blocks_dy);
+    }
 
     // CUDA-core wgrad split-K: enough slices to fill the machine, at least 512 rows each.
     {
@@ -325,7 +347,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->stem = d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
               g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0;
     p->stem_blocks = (int)std::min<long long>((g.m + 255) / 256, (long long)p->sm_count * 8);
-    p->nparts = std::max(e.blocks_reduce, p->tc.fprop_parts);
+    p->nparts = std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts);
     const size_t C = (size_t)g.c_out;
     size_t off = 0;
     p->off_scale = off; off = align_up(off + C * 4, 256);
@@ -449,7 +471,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
     float* shift = reinterpret_cast<float*>(ws + p->off_shift);
     float* part = reinterpret_cast<float*>(ws + p->off_fpart);
-    int nparts = p->ew.blocks_reduce;
+    int nparts = p->ew.blocks_stats;
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
@@ -491,7 +513,7 @@ nb_status nb_bn_stats(nb_cbs_plan p, const void* y, int32_t y_dtype, float* mean
     float* part = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_fpart);
     if (is_f32(p)) NB_TRY(run_stats_partial<float>(p, y, part, st));
     else NB_TRY(run_stats_partial<__half>(p, y, part, st));
-    return run_finalize(p, part, p->ew.blocks_reduce, nullptr, nullptr, mean, invstd, nullptr, nullptr, nullptr, nullptr, sum, sumsq, st);
+    return run_finalize(p, part, p->ew.blocks_stats, nullptr, nullptr, mean, invstd, nullptr, nullptr, nullptr, nullptr, sum, sumsq, st);
 }
 
 nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_saved, const float* save_mean,
