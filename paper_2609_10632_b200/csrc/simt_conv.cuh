@@ -156,6 +156,8 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(P prob, TO* __restrict__
 }
 
 // out[e] = sum_z partial[z][e], summed in fp64 in slice order (four elements per thread when the count allows).
+// Eight slices are loaded before any is added so that a thread keeps eight independent 16-byte loads in flight:
+// the kernel is tiny and otherwise bound by one memory latency per slice.
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partial, int splits, size_t elems, float* __restrict__ out) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     if ((elems & 3) == 0) {
@@ -163,15 +165,19 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
         const float4* p4 = reinterpret_cast<const float4*>(partial);
         for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
             double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-            int z = 0;
-            for (; z + 1 < splits; z += 2) {
-                const float4 a = p4[(size_t)z * nv + v], b = p4[(size_t)(z + 1) * nv + v];
-                s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
-                s0 += (double)b.x; s1 += (double)b.y; s2 += (double)b.z; s3 += (double)b.w;
-            }
-            if (z < splits) {
-                const float4 a = p4[(size_t)z * nv + v];
-                s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
+            for (int z0 = 0; z0 < splits; z0 += 8) {
+                float4 a[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (z0 + u < splits) a[u] = p4[(size_t)(z0 + u) * nv + v];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (z0 + u < splits) {
+                        s0 += (double)a[u].x;
+                        s1 += (double)a[u].y;
+                        s2 += (double)a[u].z;
+                        s3 += (double)a[u].w;
+                    }
             }
             reinterpret_cast<float4*>(out)[v] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
         }

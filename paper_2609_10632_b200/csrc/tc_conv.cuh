@@ -980,8 +980,8 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
     tc->launches += 1;
     if (P.splits > 1) {
         const size_t elems = (size_t)g.c_out * g.kdim;
-        const int blocks = (int)std::min<size_t>((elems + 255) / 256, (size_t)tc->sm_count * 8);
-        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, P.splits, elems, dw);
+        const int blocks = (int)std::min<size_t>((elems / 4 + 127) / 128 + 1, (size_t)tc->sm_count * 8);
+        splitk_reduce_kernel<<<blocks, 128, 0, st>>>(partial, P.splits, elems, dw);
         if (cudaGetLastError() != cudaSuccess) { err() = "launch of splitk_reduce_kernel failed"; return NB_ERR_CUDA; }
         tc->launches += 1;
     }
