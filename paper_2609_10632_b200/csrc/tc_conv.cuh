@@ -430,45 +430,58 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     __syncwarp();  // every warp only reads back the 32 rows it staged itself
                     if (STATS && !(p.variant & 16)) {
                         // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
-                        // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends
-                        for (int pc = lane; pc < ncol / 2; pc += 32) {
-                            float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
-                            const uint8_t* col = my_rows + pc * 4;
+                        // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends.
+                        // A lane owns four adjacent channels (ncol <= 128, so one pass covers the chunk).
+                        if (lane < ncol / 4) {
+                            float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
+                            const uint8_t* col = my_rows + lane * 8;
 #pragma unroll 8
                             for (int rr = 0; rr < 32; ++rr) {
-                                const uint32_t u = *reinterpret_cast<const uint32_t*>(col + (size_t)rr * pitch);
-                                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u));
-                                s0 += f.x;
-                                s1 += f.y;
-                                q0 = fmaf(f.x, f.x, q0);
-                                q1 = fmaf(f.y, f.y, q1);
+                                const uint2 u = *reinterpret_cast<const uint2*>(col + (size_t)rr * pitch);
+                                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
+                                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+                                s4[0] += f0.x; s4[1] += f0.y; s4[2] += f1.x; s4[3] += f1.y;
+                                q4[0] = fmaf(f0.x, f0.x, q4[0]); q4[1] = fmaf(f0.y, f0.y, q4[1]);
+                                q4[2] = fmaf(f1.x, f1.x, q4[2]); q4[3] = fmaf(f1.y, f1.y, q4[3]);
                             }
-                            const int ch0 = n_tile * p.BN + cbase + 2 * pc;
-                            my_stat[ch0] += s0;
-                            my_stat[ch0 + 1] += s1;
-                            my_stat[p.ldo + ch0] += q0;
-                            my_stat[p.ldo + ch0 + 1] += q1;
+                            float4* ps = reinterpret_cast<float4*>(my_stat + n_tile * p.BN + cbase + 4 * lane);
+                            float4* pq = reinterpret_cast<float4*>(my_stat + p.ldo + n_tile * p.BN + cbase + 4 * lane);
+                            float4 a4 = *ps, b4 = *pq;
+                            a4.x += s4[0]; a4.y += s4[1]; a4.z += s4[2]; a4.w += s4[3];
+                            b4.x += q4[0]; b4.y += q4[1]; b4.z += q4[2]; b4.w += q4[3];
+                            *ps = a4;
+                            *pq = b4;
                         }
                     }
-                    // ---- coalesced row stores: the lanes of a warp cover whole rows of 16-byte pieces
-                    {
-                        const int cpr = ncol / 8;   // 16-byte chunks per staged row (<= 16)
-                        const int rpi = 32 / cpr;   // rows one warp stores per iteration
-                        const int lr = lane / cpr, lc = lane - lr * cpr;
-                        if (lr < rpi && !(p.variant & 32)) {
-                            for (int rr = lr; rr < 32; rr += rpi) {
-                                const long long m = m0 + lane_group * 32 + rr;
-                                if (m >= p.M) break;
-                                long long pix = m;
-                                if (p.os != 1) {
-                                    const int j = (int)(m % p.Wq);
-                                    const long long t1 = m / p.Wq;
-                                    const int i = (int)(t1 % p.Hq);
-                                    const long long n = t1 / p.Hq;
-                                    pix = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
-                                }
-                                const uint4 v = *reinterpret_cast<const uint4*>(my_rows + (size_t)rr * pitch + lc * 16);
-                                *reinterpret_cast<uint4*>(outb + ((size_t)pix * p.ldo + (size_t)n_tile * p.BN + cbase) * 2 + (size_t)lc * 16) = v;
+                    // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
+                    // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
+                    // output pixel of row r, the others fetch it by shuffle
+                    if (!(p.variant & 32)) {
+                        const int cpr = ncol / 8;  // 16-byte pieces per staged row (<= 16)
+                        long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
+                        if (pixrow >= p.M) {
+                            pixrow = -1;
+                        } else if (p.os != 1) {
+                            const int j = (int)(pixrow % p.Wq);
+                            const long long t1 = pixrow / p.Wq;
+                            const int i = (int)(t1 % p.Hq);
+                            const long long n = t1 / p.Hq;
+                            pixrow = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
+                        }
+                        const int col_off = (n_tile * p.BN + cbase) * 2;
+                        const int step_r = 32 / cpr, step_c = 32 - step_r * cpr;
+                        int rr = lane / cpr, cc = lane - rr * cpr;
+                        for (int it = 0; it < cpr; ++it) {
+                            const long long pix = __shfl_sync(0xffffffffu, pixrow, rr);
+                            if (pix >= 0) {
+                                const uint4 v = *reinterpret_cast<const uint4*>(my_rows + rr * pitch + cc * 16);
+                                *reinterpret_cast<uint4*>(outb + (size_t)pix * (size_t)(p.ldo * 2) + col_off + cc * 16) = v;
+                            }
+                            rr += step_r;
+                            cc += step_c;
+                            if (cc >= cpr) {
+                                cc -= cpr;
+                                ++rr;
                             }
                         }
                     }
