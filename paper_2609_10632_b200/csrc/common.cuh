@@ -4,6 +4,8 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
 
 namespace nbcbs {
 
@@ -51,6 +53,46 @@ template <typename T> __device__ __forceinline__ Vec16<T> ld16_stream(const T* p
 }
 template <typename T> __device__ __forceinline__ void st16_stream(T* p, const Vec16<T>& r) {
     __stcs(reinterpret_cast<uint4*>(p), *reinterpret_cast<const uint4*>(&r));
+}
+
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_launch_dependents() and executes pdl_wait()
+// before its first access to global memory: the next kernel in the stream may then become resident and run its prologue
+// (barrier set-up, TMEM allocation, descriptor prefetch) while this one drains, and still sees all of its results.
+// Because every kernel waits before it finishes, completion of the previous kernel implies completion of all earlier ones.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+inline bool pdl_enabled() {
+    static const bool on = !(getenv("NB_PDL") && atoi(getenv("NB_PDL")) == 0);
+    return on;
+}
+
+// Launches `kernel` on `st` with the programmatic-serialization attribute (and a cluster of `cluster_x` CTAs when > 1).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x, Args&&... args) {
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof lc);
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute at[2];
+    unsigned n = 0;
+    if (pdl_enabled()) {
+        at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster_x > 1) {
+        at[n].id = cudaLaunchAttributeClusterDimension;
+        at[n].val.clusterDim.x = (unsigned)cluster_x;
+        at[n].val.clusterDim.y = 1;
+        at[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    lc.attrs = at;
+    lc.numAttrs = n;
+    return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace nbcbs

@@ -26,6 +26,8 @@ template <bool FAST> __device__ __forceinline__ float sigmoid_f(float z) {
 template <typename YT>
 __global__ void __launch_bounds__(288, 3) bn_stats_partial_kernel(const YT* __restrict__ y, long long total_vecs, int C,
                                                                 float* __restrict__ partials) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int V = Vec16<YT>::N;
     extern __shared__ float red[];  // [blockDim.x][V]
     const int tid = threadIdx.x;
@@ -87,6 +89,8 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restric
                                                           float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
                                                           float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
                                                           float* sum_out, float* sumsq_out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
@@ -131,6 +135,8 @@ template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
                                                              long long total_vecs, int C, const float* __restrict__ scale,
                                                              const float* __restrict__ shift) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "y and a must have the same element size");
     const int cg = threadIdx.x % (C / V);
@@ -159,6 +165,8 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
                                                                   long long total_vecs, int C, const float* __restrict__ mean,
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
                                                                   const float* __restrict__ beta, float* __restrict__ partials) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "g and y must have the same element size");
     extern __shared__ float red[];
@@ -216,6 +224,8 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __res
                                                               const float* __restrict__ mean, const float* __restrict__ invstd,
                                                               const float* __restrict__ gamma, const float* __restrict__ beta,
                                                               float* dgamma, float* dbeta, float* coef /*[4][C]*/) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
@@ -240,6 +250,8 @@ template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
                                                               const float* __restrict__ coef) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int V = Vec16<YT>::N;
     const int cg = threadIdx.x % (C / V);
     float a[V], b[V], p1[V], p0[V];

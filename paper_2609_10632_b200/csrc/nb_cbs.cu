@@ -144,7 +144,7 @@ nb_status launch_ok(const char* what) {
 template <typename YT> nb_status run_stats_partial(nb_cbs_plan_s* p, const void* y, float* partials, cudaStream_t st) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_STATS, st);
-    bn_stats_partial_kernel<YT><<<e.blocks_stats, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+    launch_k(bn_stats_partial_kernel<YT>, dim3(e.blocks_stats), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
         static_cast<const YT*>(y), e.total_vecs, p->g.c_out, partials);
     return launch_ok("bn_stats_partial");
 }
@@ -154,7 +154,7 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
                        cudaStream_t st) {
     const int C = p->g.c_out;
     SiteTimer tm(p, SITE_FINALIZE, st);
-    bn_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
+    launch_k(bn_finalize_kernel, dim3((C + 7) / 8), dim3(256), 0, st, 1, partials, nparts, C, (double)p->g.m, p->desc.eps, p->desc.momentum,
                                                               gamma, beta, mean, invstd, scale, shift, rmean, rvar, sum, sumsq);
     return launch_ok("bn_finalize");
 }
@@ -163,7 +163,7 @@ template <typename YT, typename AT, bool FAST>
 nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_APPLY, st);
-    bn_silu_apply_kernel<YT, AT, FAST><<<e.blocks_apply, e.tpb, 0, st>>>(static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
+    launch_k(bn_silu_apply_kernel<YT, AT, FAST>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
                                                                        p->g.c_out, scale, shift);
     return launch_ok("bn_silu_apply");
 }
@@ -176,17 +176,17 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     const int C = p->g.c_out;
     {
         SiteTimer tm(p, SITE_BWD_REDUCE, st);
-        bn_silu_bwd_reduce_kernel<YT, AT, FAST><<<e.blocks_reduce, e.tpb, (size_t)e.tpb * e.vec * sizeof(float), st>>>(
+        launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
             static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials);
         NB_LAUNCH_OK("bn_silu_bwd_reduce");
     }
     {
         SiteTimer tm(p, SITE_BWD_FINALIZE, st);
-        bn_bwd_finalize_kernel<<<(C + 7) / 8, 256, 0, st>>>(partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta, coef);
+        launch_k(bn_bwd_finalize_kernel, dim3((C + 7) / 8), dim3(256), 0, st, 1, partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta, coef);
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
-    bn_silu_bwd_dy_kernel<YT, AT, FAST><<<e.blocks_dy, e.tpb, 0, st>>>(static_cast<const AT*>(g), static_cast<const YT*>(y),
+    launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
                                                                         static_cast<AT*>(dy), e.total_vecs, C, coef);
     return launch_ok("bn_silu_bwd_dy");
 }
@@ -197,7 +197,7 @@ nb_status run_simt_fprop(nb_cbs_plan_s* p, const void* x, const void* w, void* y
     FpropProblem<TIN, TIN> prob{static_cast<const TIN*>(x), static_cast<const TIN*>(w), p->g};
     dim3 grid((unsigned)((p->g.m + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_out + SIMT_BN - 1) / SIMT_BN), 1);
     SiteTimer tm(p, SITE_FPROP, st);
-    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TOUT*>(y), (long long)p->g.kdim);
+    launch_k(simt_gemm_kernel<FpropProblem<TIN, TIN>, TOUT>, grid, dim3(256), 0, st, 1, prob, static_cast<TOUT*>(y), (long long)p->g.kdim);
     return launch_ok("simt fprop");
 }
 
@@ -207,7 +207,7 @@ nb_status run_simt_dgrad(nb_cbs_plan_s* p, const void* dy, const void* w, void* 
     const long long I = (long long)p->g.n * p->g.h * p->g.w;
     dim3 grid((unsigned)((I + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.c_in + SIMT_BN - 1) / SIMT_BN), 1);
     SiteTimer tm(p, SITE_DGRAD, st);
-    simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, static_cast<TIN*>(dx), (long long)p->g.k * p->g.k * p->g.c_out);
+    launch_k(simt_gemm_kernel<DgradProblem<TIN, TIN>, TIN>, grid, dim3(256), 0, st, 1, prob, static_cast<TIN*>(dx), (long long)p->g.k * p->g.k * p->g.c_out);
     return launch_ok("simt dgrad");
 }
 
@@ -217,17 +217,17 @@ nb_status run_simt_wgrad(nb_cbs_plan_s* p, const void* x, const void* dy, float*
     dim3 grid((unsigned)((p->g.c_out + SIMT_BM - 1) / SIMT_BM), (unsigned)((p->g.kdim + SIMT_BN - 1) / SIMT_BN), (unsigned)p->wg_splits);
     if (p->wg_splits == 1) {
         SiteTimer tm(p, SITE_WGRAD, st);
-        simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, dw, p->g.m);
+        launch_k(simt_gemm_kernel<WgradProblem<TIN, TIN>, float>, grid, dim3(256), 0, st, 1, prob, dw, p->g.m);
         return launch_ok("simt wgrad");
     }
     {
         SiteTimer tm(p, SITE_WGRAD, st);
-        simt_gemm_kernel<<<grid, 256, 0, st>>>(prob, partial, p->wg_chunk);
+        launch_k(simt_gemm_kernel<WgradProblem<TIN, TIN>, float>, grid, dim3(256), 0, st, 1, prob, partial, p->wg_chunk);
         NB_LAUNCH_OK("simt wgrad (split-K)");
     }
     const size_t elems = (size_t)p->g.c_out * p->g.kdim;
     SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
-    splitk_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, p->wg_splits, elems, dw);
+    launch_k(splitk_reduce_kernel, dim3((unsigned)((elems + 255) / 256)), dim3(256), 0, st, 1, partial, p->wg_splits, elems, dw);
     return launch_ok("splitk_reduce");
 }
 
@@ -479,7 +479,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         {
             SiteTimer tm(p, SITE_FPROP, st);
             const int blocks = (int)std::min<long long>((p->g.m + 127) / 128, (long long)p->sm_count * 16);
-            stem_fprop_kernel<48><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
+            launch_k(stem_fprop_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
                                                          static_cast<__half*>(y_saved), p->g);
             NB_LAUNCH_OK("stem_fprop");
         }
@@ -541,7 +541,7 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
         SiteTimer tm(p, SITE_DGRAD, st);
         const long long total = (long long)p->g.n * p->g.h * (p->g.w / 2);
         const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-        stem_dgrad_kernel<48><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
+        launch_k(stem_dgrad_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
                                                      static_cast<__nv_bfloat16*>(dx), p->g);
         return launch_ok("stem_dgrad");
     }
@@ -569,13 +569,13 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
         {
             SiteTimer tm(p, SITE_WGRAD, st);
             const long long per = (p->g.m + p->stem_blocks - 1) / p->stem_blocks;
-            stem_wgrad_kernel<48><<<p->stem_blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
+            launch_k(stem_wgrad_kernel<48>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
                                                                  partial, p->g, per);
             NB_LAUNCH_OK("stem_wgrad");
         }
         const size_t elems = (size_t)p->g.c_out * p->g.kdim;
         SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
-        splitk_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, p->stem_blocks, elems, dw);
+        launch_k(splitk_reduce_kernel, dim3((unsigned)((elems + 255) / 256)), dim3(256), 0, st, 1, partial, p->stem_blocks, elems, dw);
         return launch_ok("splitk_reduce");
     }
     if (p->tc.wgrad) {
@@ -656,11 +656,11 @@ extern "C" nb_status nb_bn_stats_static(const void* y, int32_t y_dtype, int64_t 
     // Every partial that the second kernel reads is written by the first one in this same call, so nothing in the
     // array has to start at zero and the previous call's contents do not matter.
     if (y_dtype == NB_DTYPE_F32)
-        bn_stats_partial_kernel<float><<<blocks, tpb, (size_t)tpb * vec * sizeof(float), st>>>(static_cast<const float*>(y), total_vecs, c, part);
+        launch_k(bn_stats_partial_kernel<float>, dim3(blocks), dim3(tpb), (size_t)tpb * vec * sizeof(float), st, 1, static_cast<const float*>(y), total_vecs, c, part);
     else
-        bn_stats_partial_kernel<__half><<<blocks, tpb, (size_t)tpb * vec * sizeof(float), st>>>(static_cast<const __half*>(y), total_vecs, c, part);
+        launch_k(bn_stats_partial_kernel<__half>, dim3(blocks), dim3(tpb), (size_t)tpb * vec * sizeof(float), st, 1, static_cast<const __half*>(y), total_vecs, c, part);
     NB_LAUNCH_OK("bn_stats_partial (static scratch)");
-    bn_finalize_kernel<<<(c + 7) / 8, 256, 0, st>>>(part, blocks, c, (double)m, eps, 0.f, nullptr, nullptr, mean, invstd, nullptr,
+    launch_k(bn_finalize_kernel, dim3((c + 7) / 8), dim3(256), 0, st, 1, part, blocks, c, (double)m, eps, 0.f, nullptr, nullptr, mean, invstd, nullptr,
                                                               nullptr, nullptr, nullptr, sum, sumsq);
     return launch_ok("bn_finalize (static scratch)");
 }

@@ -85,6 +85,8 @@ constexpr int SIMT_BM = 64, SIMT_BN = 64, SIMT_BK = 16, SIMT_FLUSH = 64;
 // [splits][I][J] and slice z covers kk in [z*kchunk, (z+1)*kchunk).
 template <class P, typename TO>
 __global__ void __launch_bounds__(256) simt_gemm_kernel(P prob, TO* __restrict__ out, long long kchunk) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ float As[SIMT_BK][SIMT_BM + 4];
     __shared__ float Bs[SIMT_BK][SIMT_BN + 4];
     const long long I = prob.I();
@@ -159,6 +161,8 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(P prob, TO* __restrict__
 // Eight slices are loaded before any is added so that a thread keeps eight independent 16-byte loads in flight:
 // the kernel is tiny and otherwise bound by one memory latency per slice.
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partial, int splits, size_t elems, float* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     if ((elems & 3) == 0) {
         const size_t nv = elems >> 2;

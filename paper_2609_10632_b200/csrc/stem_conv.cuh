@@ -14,6 +14,8 @@ constexpr int STEM_CIN = 3, STEM_K = 3, STEM_TAPS = 9, STEM_KDIM = 27;
 template <int COUT>
 __global__ void __launch_bounds__(128) stem_fprop_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                                                          __half* __restrict__ y, Geom g) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ __align__(16) float ws[STEM_KDIM][COUT];  // ws[k][c'] = w[c'][k]
     for (int e = threadIdx.x; e < STEM_KDIM * COUT; e += blockDim.x) {
         const int co = e / STEM_KDIM, k = e % STEM_KDIM;
@@ -70,6 +72,8 @@ __global__ void __launch_bounds__(128) stem_fprop_kernel(const __nv_bfloat16* __
 template <int COUT>
 __global__ void __launch_bounds__(128) stem_dgrad_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ w,
                                                          __nv_bfloat16* __restrict__ dx, Geom g) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ __align__(16) float ws[STEM_TAPS][COUT][4];  // ws[tap][c'][c], c padded to 4
     for (int e = threadIdx.x; e < STEM_TAPS * COUT; e += blockDim.x) {
         const int tap = e / COUT, co = e % COUT;
@@ -133,6 +137,8 @@ __global__ void __launch_bounds__(128) stem_dgrad_kernel(const __nv_bfloat16* __
 template <int COUT>
 __global__ void __launch_bounds__(128) stem_wgrad_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
                                                          float* __restrict__ partial, Geom g, long long pix_per_block) {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int P = 32;  // pixels per staged chunk
     constexpr int NCG = COUT / 4;
     __shared__ __align__(16) float dys[P][COUT];

@@ -130,7 +130,10 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <typename OutT, bool STATS>
+// CG2 = the CTAs run as pairs (clusters of two): rank 0 issues tcgen05.mma.cta_group::2 with M = 256; each CTA owns 128
+// of the rows (its own A tile, accumulator and epilogue) and fetches half of the B tile, which halves the filter
+// bytes written to and read from each SM's shared memory.
+template <typename OutT, bool STATS, bool CG2>
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -149,20 +152,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.nclasses * p.tiles_per_class;
     const int mh = p.mh;          // 128-row sub-tiles per tile (1 or 2); both share every B stage
     const int nbuf = p.acc_bufs;  // accumulator sets in TMEM (2 = the epilogue of a tile overlaps the next tile's MMAs)
+    const uint32_t rank = CG2 ? ptx::cluster_ctarank() : 0u;                  // position in the CTA pair
+    const int worker = CG2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;        // tile-loop start
+    const int nworkers = CG2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;        // tile-loop stride
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, 2);  // the A producer and the B producer each arrive once (with their byte counts)
+            ptx::mbar_init(full + s, 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
+                                          // producers announce the bytes of both CTAs, the peer only issues its loads)
             ptx::mbar_init(empty + s, 1);
         }
         ptx::mbar_init(tfull, 1);
         ptx::mbar_init(tfull + 1, 1);
-        ptx::mbar_init(tempty, 128);
-        ptx::mbar_init(tempty + 1, 128);
+        ptx::mbar_init(tempty, CG2 ? 8 : 128);  // pairs: one arrival per epilogue warp of both CTAs
+        ptx::mbar_init(tempty + 1, CG2 ? 8 : 128);
         ptx::mbar_init(drain, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -171,13 +179,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         for (int c = threadIdx.x; c < 8 * p.ldo; c += TC_THREADS) wstat[c] = 0.f;
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
-        ptx::tmem_relinquish();
+        if (CG2) {
+            ptx::tmem_alloc_cg2(tmem_slot, (uint32_t)p.tmem_cols);
+            ptx::tmem_relinquish_cg2();
+        } else {
+            ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG2) ptx::cluster_sync_all(); else __syncthreads();  // barriers of both CTAs are initialised before any remote arrive
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // everything above touched only shared memory, TMEM and kernel parameters
 
     if (warp == 0 || warp == 6) {
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
@@ -196,19 +210,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             long long dbg_wait_empty = 0;
             const long long dbg_start = clock64();
 #endif
-            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(p.BN * p.KC * 2);
+            const int bn_own = CG2 ? p.BN / 2 : p.BN;  // rows of the B tile this CTA fetches
+            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(bn_own * p.KC * 2);
             // loop-invariant values in registers: this thread's instruction stream is on the critical path
             const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
             const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
             const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes, sub_bytes = isA ? p.a_sub_bytes : p.b_sub_bytes;
-            const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB), full_u32 = ptx::smem_u32(full);
+            // pairs: loads of both CTAs are counted on the rank-0 CTA's full barriers (the MMA issuer waits there)
+            const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB);
+            const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
             const int tpc = p.tiles_per_class;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 const int cls = tile / tpc, lt = tile - cls * tpc;
                 const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
                 const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
                 const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
-                const int m0 = m_tile * TC_BM * mh;
+                const int m0 = (CG2 ? m_tile * 2 + (int)rank : m_tile) * TC_BM * mh;
                 int cw = 0, ch = 0, n0 = 0;
                 if (isA && !a_tiled) {
                     const int j0 = m0 % Wq, t1 = m0 / Wq;
@@ -217,11 +234,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     cw = p.lo_w + j0 * ts;
                     ch = p.lo_h + i0 * ts;
                 }
-                const int brow = n_tile * BN;
+                const int brow = n_tile * BN + (CG2 ? (int)rank * bn_own : 0);
                 // each CTA starts its K loop at a different k-block so that the CTAs do not all ask L2 for the same
                 // filter lines at the same moment
                 const int ntaps_c = p.cls_ntaps[cls];
-                const int rot = (p.variant & 4) ? 0 : (int)((blockIdx.x * 7u) % (unsigned)kblocks);
+                const int rot = (p.variant & 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
                 int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
@@ -234,16 +251,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         NB_DBG_ADD(dbg_wait_empty);
                     }
                     const uint32_t bar = full_u32 + 8u * (uint32_t)s;
-                    ptx::mbar_expect_tx_u32(bar, kb_bytes * (uint32_t)nkb);
+                    if (!CG2) ptx::mbar_expect_tx_u32(bar, kb_bytes * (uint32_t)nkb);
+                    else if (rank == 0) ptx::mbar_expect_tx_u32(ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
                     uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
                     for (int j = 0; j < nkb; ++j) {
                         if (isA) {
-                            if (a_tiled)
-                                ptx::tma_load_2d_u32(dst, tm, bar, kc * KC, m0);
-                            else
-                                ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                            if (a_tiled) {
+                                if (CG2) ptx::tma_load_2d_cg2(dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32(dst, tm, bar, kc * KC, m0);
+                            } else {
+                                if (CG2)
+                                    ptx::tma_load_im2col_4d_cg2(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                                else
+                                    ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                            }
                         } else {
-                            ptx::tma_load_2d_u32(dst, tm, bar, tap * Ca + kc * KC, brow);
+                            if (CG2) ptx::tma_load_2d_cg2(dst, tm, bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32(dst, tm, bar, tap * Ca + kc * KC, brow);
                         }
                         dst += sub_bytes;
                         if (++kc == kc_per_tap) {
@@ -273,8 +295,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (one thread)
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (one thread; in a pair only rank 0)
+        if (lane == 0 && rank == 0) {
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
@@ -292,7 +314,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint32_t empty_u32 = ptx::smem_u32(empty);
             uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
             const int tpc = p.tiles_per_class, kc_per_tap = p.kc_per_tap;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            const uint32_t tfull_u32 = ptx::smem_u32(tfull);
+            for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 const int kblocks = p.cls_ntaps[tile / tpc] * kc_per_tap;
                 {
                     NB_DBG_T0();
@@ -318,7 +341,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         for (int h = 0; h < mh; ++h) {
                             const uint64_t dah = da + (uint64_t)h * a_half16;
                             const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
-                            if (ksteps == 4) {
+                            if (CG2) {
+                                ptx::umma_f16_cg2(dt, dah, db, idesc, accumulate);
+                                ptx::umma_f16_cg2(dt, dah + 2, db + 2, idesc, 1u);
+                                ptx::umma_f16_cg2(dt, dah + 4, db + 4, idesc, 1u);
+                                ptx::umma_f16_cg2(dt, dah + 6, db + 6, idesc, 1u);
+                            } else if (ksteps == 4) {
                                 ptx::umma_f16(dt, dah, db, idesc, accumulate);
                                 ptx::umma_f16(dt, dah + 2, db + 2, idesc, 1u);
                                 ptx::umma_f16(dt, dah + 4, db + 4, idesc, 1u);
@@ -332,7 +360,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         da += a_sub16;
                         db += b_sub16;
                     }
-                    ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
+                    if (CG2) ptx::umma_commit_cg2_mc(empty_u32 + 8u * (uint32_t)s, 3); else ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
                     da_s += a_stage16;
                     db_s += b_stage16;
                     if (++s == stages) {
@@ -343,7 +371,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     }
                 }
                 if (!ok) break;
-                ptx::umma_commit(tfull + acc);
+                if (CG2) ptx::umma_commit_cg2_mc(tfull_u32 + 8u * (uint32_t)acc, 3); else ptx::umma_commit(tfull + acc);
                 if (++acc == nbuf) {
                     acc = 0;
                     acc_ph ^= 1u;
@@ -353,7 +381,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             if (p.dbg) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
 #endif
             // Make sure every MMA issued by this thread has retired before TMEM is released.
-            ptx::umma_commit(drain);
+            if (CG2) ptx::umma_commit_cg2(ptx::smem_u32(drain)); else ptx::umma_commit(drain);
             for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
             }
         }
@@ -372,7 +400,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         long long dbg_wait_tfull = 0;
         const long long dbg_start = clock64();
 #endif
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
+        for (int tile = worker; tile < total_tiles; tile += nworkers) {
             const int cls = tile / p.tiles_per_class, lt = tile - cls * p.tiles_per_class;
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
             NB_DBG_T0();
@@ -386,7 +415,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             ptx::tc_fence_after();
             if (p.variant & 8) {
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(tempty + acc);
+                if (CG2) {
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
+                } else {
+                    ptx::mbar_arrive(tempty + acc);
+                }
                 if (++acc == nbuf) {
                     acc = 0;
                     acc_ph ^= 1u;
@@ -394,7 +428,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                 continue;
             }
             for (int h = 0; h < mh; ++h) {
-                const long long m0 = ((long long)m_tile * mh + h) * TC_BM;
+                const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
                 const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride);
                 for (int cbase = 0; cbase < p.BN; cbase += CW) {
                     const int ncol = (p.BN - cbase < CW) ? p.BN - cbase : CW;  // multiple of 16
@@ -425,7 +459,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     if (h == mh - 1 && cbase + CW >= p.BN) {
                         // last TMEM read of this tile: the accumulator set is free for the MMAs of a later tile
                         ptx::tc_fence_before();
-                        ptx::mbar_arrive(tempty + acc);
+                        if (CG2) {
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
+                        } else {
+                            ptx::mbar_arrive(tempty + acc);
+                        }
                     }
                     __syncwarp();  // every warp only reads back the 32 rows it staged itself
                     if (STATS && !(p.variant & 16)) {
@@ -505,10 +544,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         if (sat) atomicAdd(p.status + ST_SAT, sat);
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG2) ptx::cluster_sync_all(); else __syncthreads();  // pairs: neither CTA may leave while the other still uses its memory
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+        if (CG2) ptx::tmem_dealloc_cg2(tmem_base, (uint32_t)p.tmem_cols); else ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
 
@@ -524,6 +563,8 @@ struct WtParams {
     WtClass cls[4];
 };
 __global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
+    pdl_launch_dependents();
+    pdl_wait();
     // one thread per output element, output-contiguous (c' fastest)
     size_t total = (size_t)P.c_in * P.k * P.k * P.c_out;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
@@ -548,6 +589,7 @@ struct IgemmCfg {
     bool ok = false;
     int Ca = 0, rowsB = 0, ntaps = 0;
     int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
+    bool cg2 = false;  // CTA pairs (tcgen05 cta_group::2)
     uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
@@ -651,15 +693,24 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
         if (rowsB % bn) continue;
         if (force_bn && bn != force_bn && rowsB % force_bn == 0) continue;
         const int acc_stride = bn <= 32 ? 32 : bn <= 64 ? 64 : bn <= 128 ? 128 : 256;
+        // CTA pairs (one tcgen05.mma over 256 rows whose B tile is split between two CTAs): a pair's MMA of 256 x N x 16
+        // runs at N/2 cycles even for small N where a single CTA's 128 x N x 16 never drops below 97, and each CTA reads
+        // and writes only half of B in shared memory.  Measured per layer on B200: 3x3 layers with at least 96 reduction
+        // channels gain 5-15 %; 1x1 layers (one k-block group per tile, epilogue-bound) lose 5-10 % to the extra
+        // cluster synchronisation, as do 3x3 layers with one k-block per tap and the stride-2 data gradients (1-4 taps
+        // per parity class) below 384 channels.
+        const bool pair_pays = ntaps > 1 && Ca >= 96 && (nclasses == 1 || Ca >= 384);
+        const bool cg2 = bn % 32 == 0 && (getenv("NB_TC_CG2") ? atoi(getenv("NB_TC_CG2")) != 0 : pair_pays);
         int mh = 1;
         if (4 * acc_stride <= 512) {
-            const long long tiles2 = ((M + 2 * TC_BM - 1) / (2 * TC_BM)) * (rowsB / bn) * nclasses;
-            if (tiles2 >= sm_count) mh = 2;
+            const long long rows_tile = 2LL * TC_BM * (cg2 ? 2 : 1);
+            const long long tiles2 = ((M + rows_tile - 1) / rows_tile) * (rowsB / bn) * nclasses;
+            if (tiles2 >= (cg2 ? sm_count / 2 : sm_count)) mh = 2;
         }
         if (force_mh && force_mh * acc_stride <= 512) mh = force_mh;
         const int acc_bufs = (2 * mh * acc_stride <= 512) ? 2 : 1;
         const uint32_t a_sub = (uint32_t)(TC_BM * mh * c.KC * 2);
-        const uint32_t b_sub = (uint32_t)((bn * c.KC * 2 + 1023) / 1024 * 1024);
+        const uint32_t b_sub = (uint32_t)(((cg2 ? bn / 2 : bn) * c.KC * 2 + 1023) / 1024 * 1024);
         const size_t fixed = igemm_fixed_smem(bn, ldo);
         if (fixed + 2 * (size_t)(a_sub + b_sub) > kMaxSmem) continue;
         const double mma_kb = mh * 4.0 * std::max(97.0, bn / 2.0);  // tensor cycles per k-block
@@ -673,7 +724,8 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
         if (stages < 2) continue;
         c.BN = bn; c.kpb = kpb; c.stages = stages; c.a_sub = a_sub; c.b_sub = b_sub; c.mh = mh; c.acc_bufs = acc_bufs;
         c.acc_stride = acc_stride;
-        c.m_tiles = (int)((M + TC_BM * mh - 1) / (TC_BM * mh));
+        c.cg2 = cg2;
+        c.m_tiles = (int)((M + TC_BM * mh * (cg2 ? 2 : 1) - 1) / (TC_BM * mh * (cg2 ? 2 : 1)));
     }
     if (!c.BN) return c;
     c.n_tiles = rowsB / c.BN;
@@ -683,7 +735,8 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     c.b_stage = c.b_sub * c.kpb;
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
-    c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, sm_count);
+    c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, c.cg2 ? sm_count / 2 : sm_count);
+    if (c.cg2) c.grid *= 2;  // two CTAs per pair
     c.ok = true;
     return c;
 }
@@ -700,9 +753,9 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.stage_cols = c.stage_cols;
     P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
     if (getenv("NB_TC_VERBOSE"))
-        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
-                c.rowsB, c.ntaps, c.mh, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
-    P.idesc = ptx::make_idesc_bf16(TC_BM, c.BN, 0, 0);
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
+                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
+    P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
 }
 
 // im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
@@ -733,22 +786,24 @@ inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, lo
     return true;
 }
 
-template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
+template <typename OutT, bool STATS, bool CG2> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
         attr_set = true;
     }
-    tc_igemm_kernel<OutT, STATS><<<s.cfg.grid, TC_THREADS, s.cfg.smem_bytes, st>>>(s.prm);
-    cudaError_t e = cudaGetLastError();
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2>, dim3((unsigned)s.cfg.grid), dim3(TC_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
     }
     return NB_OK;
+}
+template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
+    return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true>(s, st) : launch_igemm_impl<OutT, STATS, false>(s, st);
 }
 
 }  // namespace tcdetail
@@ -930,7 +985,7 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh)) {
             return NB_ERR_CUDA;
         }
-        if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
+        if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
@@ -946,7 +1001,7 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
     {
         const size_t total = tc->wt_bytes / 2;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)tc->sm_count * 8);
-        dgrad_weight_transform_kernel<<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), tc->wtp);
+        launch_k(dgrad_weight_transform_kernel, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), tc->wtp);
         if (cudaGetLastError() != cudaSuccess) { err() = "launch of dgrad_weight_transform_kernel failed"; return NB_ERR_CUDA; }
         tc->launches += 1;
     }
@@ -957,7 +1012,7 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
         for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
             const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
-            if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.BN)) return NB_ERR_CUDA;
+            if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         }
         S.a_ptr = dy; S.b_ptr = wt;
     }
@@ -987,14 +1042,14 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
         }
         attr_set = true;
     }
-    tc_wgrad_kernel<<<tc->wg_grid, TC_THREADS, tc->wg_smem, st>>>(P);
+    launch_k(tc_wgrad_kernel, dim3(tc->wg_grid), dim3(TC_THREADS), tc->wg_smem, st, 1, P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { err() = std::string("launch of tc_wgrad_kernel failed: ") + cudaGetErrorString(e); return NB_ERR_CUDA; }
     tc->launches += 1;
     if (P.splits > 1) {
         const size_t elems = (size_t)g.c_out * g.kdim;
         const int blocks = (int)std::min<size_t>((elems / 4 + 127) / 128 + 1, (size_t)tc->sm_count * 8);
-        splitk_reduce_kernel<<<blocks, 128, 0, st>>>(partial, P.splits, elems, dw);
+        launch_k(splitk_reduce_kernel, dim3(blocks), dim3(128), 0, st, 1, partial, P.splits, elems, dw);
         if (cudaGetLastError() != cudaSuccess) { err() = "launch of splitk_reduce_kernel failed"; return NB_ERR_CUDA; }
         tc->launches += 1;
     }

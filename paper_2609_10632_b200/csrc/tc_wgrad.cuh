@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // tile = (m_tile, n_tile, split), split fastest so that CTAs sharing a pixel range run together
     const int split = blockIdx.x % p.splits;
@@ -69,6 +70,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // everything above touched only shared memory, TMEM and kernel parameters
 
     if (warp == 0 || warp == 6) {
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds x, warp 6 feeds dy
