@@ -100,7 +100,9 @@ nb_status nb_cbs_out_shape(nb_cbs_plan plan, int32_t* ho, int32_t* wo);
 nb_status nb_cbs_workspace_bytes(nb_cbs_plan plan, size_t* fwd_bytes, size_t* bwd_bytes);
 
 /* Which implementation each convolution of this plan runs on: writes three ints (fprop, dgrad, wgrad),
- * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel. */
+ * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel, 2 = the tap-reuse variant of the tensor-core kernel
+ * (3x3 stride-1 layers only; an experiment that is chosen only when the environment variable NB_TC_HALO is 1
+ * at plan creation). */
 nb_status nb_cbs_plan_paths(nb_cbs_plan plan, int32_t* paths3);
 
 /* Synchronise `stream`, then report whether any kernel launched through this plan gave up a bounded

@@ -404,8 +404,8 @@ nb_status nb_cbs_workspace_bytes(nb_cbs_plan p, size_t* fwd, size_t* bwd) {
 nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
     g_err.clear();
     if (!p || !paths3) return fail(NB_ERR_INVALID_ARG, "NULL argument");
-    paths3[0] = p->tc.fprop ? 1 : 0;
-    paths3[1] = p->tc.dgrad ? 1 : 0;
+    paths3[0] = p->tc.fprop ? (p->tc.fp.cfg.halo ? 2 : 1) : 0;
+    paths3[1] = p->tc.dgrad ? (p->tc.dg.cfg.halo ? 2 : 1) : 0;
     paths3[2] = p->tc.wgrad ? 1 : 0;
     return NB_OK;
 }

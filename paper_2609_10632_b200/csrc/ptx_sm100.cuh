@@ -244,6 +244,71 @@ __device__ __forceinline__ void umma_commit_cg2(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ------------------------------------------------------------------ warp-uniform issue
+// The producer and MMA loops are executed by a whole converged warp and only the asynchronous instruction itself is
+// predicated on an elected lane.  Measured on B200: a loop run by a single thread behind `if (lane == 0)` spends 80-100
+// cycles per tcgen05.mma on issue alone, the converged form 41-50, so narrow tiles (N < 192) run twice as fast.
+#define NB_PRED_OPEN "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %0, 0;\n\t"
+__device__ __forceinline__ void mbar_expect_tx_u32_if(uint32_t issue, uint32_t bar, uint32_t bytes) {
+    asm volatile(NB_PRED_OPEN "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t}\n" ::"r"(issue), "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_u32_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
+    asm volatile(NB_PRED_OPEN "@q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2, {%4, %5}], [%3];\n\t}\n" ::"r"(issue),
+                 "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_u32_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c, int w, int h, int n,
+                                                          uint16_t off_w, uint16_t off_h) {
+    asm volatile(NB_PRED_OPEN
+                 "@q cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%1], [%2, {%4, %5, %6, %7}], [%3], {%8, %9};\n\t}\n" ::"r"(
+                     issue),
+                 "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_cg2_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
+    asm volatile(NB_PRED_OPEN
+                 "@q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2, {%4, %5}], [%3];\n\t}\n" ::"r"(issue),
+                 "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_cg2_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c, int w, int h, int n,
+                                                          uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        NB_PRED_OPEN
+        "@q cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2, {%4, %5, %6, %7}], [%3], {%8, %9};\n\t}\n" ::"r"(
+            issue),
+        "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void umma_f16_if(uint32_t issue, uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(NB_PRED_OPEN
+                 ".reg .pred p;\n\t"
+                 "setp.ne.b32 p, %5, 0;\n\t"
+                 "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t}\n" ::"r"(issue),
+                 "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_f16_cg2_if(uint32_t issue, uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(NB_PRED_OPEN
+                 ".reg .pred p;\n\t"
+                 "setp.ne.b32 p, %5, 0;\n\t"
+                 "@q tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %4, p;\n\t}\n" ::"r"(issue),
+                 "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit_u32_if(uint32_t issue, uint32_t bar) {
+    asm volatile(NB_PRED_OPEN "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}\n" ::"r"(issue), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_commit_cg2_mc_if(uint32_t issue, uint32_t bar, uint16_t mask) {
+    asm volatile(NB_PRED_OPEN "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t}\n" ::"r"(issue),
+                 "r"(bar), "h"(mask)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit_cg2_if(uint32_t issue, uint32_t bar) {
+    asm volatile(NB_PRED_OPEN "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}\n" ::"r"(issue), "r"(bar) : "memory");
+}
+#undef NB_PRED_OPEN
+
 // 32 lanes x 32 consecutive columns of 32-bit values: thread i of the warp gets lane (base lane + i), r[j] = column j.
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t* r) {
     asm volatile(

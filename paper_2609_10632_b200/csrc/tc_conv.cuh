@@ -51,6 +51,13 @@ struct IgemmParams {
     float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
     int* status;
     uint16_t off_w[4][9], off_h[4][9];
+    // Halo mode (3x3, stride 1): the GEMM rows are the positions of the zero-padded raster [N][H+2][W+2]; one slab of
+    // 128*mh + 2*(W+2) + 2 consecutive positions x 64 channels serves all nine taps (tap (r,t) starts r*(W+2)+t rows in).
+    int halo, Wp, Hp, Hin, Win, Nimg;
+    int slab_boxes, box_pix, a_slots;
+    uint32_t slab_bytes;
+    long long npos;            // N*(H+2)*(W+2)
+    uint32_t tap_off16[9];     // start of tap t inside the slab, in 16-byte units
 };
 
 #ifdef NB_TC_DEBUG_TIMING
@@ -93,9 +100,11 @@ __device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile i
 }
 
 // Fast path inline (the barrier is usually complete already), slow bounded path out of line.
+// Called by all 32 lanes of a producer or MMA warp; the lanes leave together with the same answer.
 __device__ __forceinline__ bool wait_bar_fast(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    return wait_bar(bar, parity, abort_flag, status, site);
+    bool ok = ptx::mbar_try_wait(bar, parity);
+    if (!ok) ok = wait_bar(bar, parity, abort_flag, status, site);
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -133,12 +142,17 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
 // CG2 = the CTAs run as pairs (clusters of two): rank 0 issues tcgen05.mma.cta_group::2 with M = 256; each CTA owns 128
 // of the rows (its own A tile, accumulator and epilogue) and fetches half of the B tile, which halves the filter
 // bytes written to and read from each SM's shared memory.
-template <typename OutT, bool STATS, bool CG2>
+// HALO = the tap-reuse variant for 3x3 stride-1 convolutions (always CTA pairs): A is fetched once per 64-channel block
+// as a slab of padded-raster positions and the nine taps are nine row offsets into it, so the activation bytes written to
+// shared memory drop from 9 x 128*mh rows to 128*mh + 2*(W+2) + 2 rows per block.  Rows that fall on the padding ring
+// are computed and discarded.
+template <typename OutT, bool STATS, bool CG2, bool HALO>
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
+    static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
-    uint8_t* sB = sA + (size_t)p.stages * p.a_stage_bytes;
+    uint8_t* sB = sA + (HALO ? (size_t)p.a_slots * p.slab_bytes : (size_t)p.stages * p.a_stage_bytes);
     uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging [128 rows][CW columns] of OutT, row pitch CW*2+16 bytes
     const int CW = p.stage_cols;                             // columns staged per pass (<= 128)
     const int pitch = CW * 2 + 16;
@@ -149,21 +163,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint64_t* tfull = empty + p.stages;   // [2]
     uint64_t* tempty = tfull + 2;         // [2]
     uint64_t* drain = tempty + 2;         // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    uint64_t* fullA = drain + 1;          // [4] halo mode: the slab ring has its own barriers
+    uint64_t* emptyA = fullA + 4;         // [4]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(emptyA + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     pdl_launch_dependents();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // warp index in a form the compiler knows to be uniform
     const int total_tiles = p.nclasses * p.tiles_per_class;
     const int mh = p.mh;          // 128-row sub-tiles per tile (1 or 2); both share every B stage
     const int nbuf = p.acc_bufs;  // accumulator sets in TMEM (2 = the epilogue of a tile overlaps the next tile's MMAs)
-    const uint32_t rank = CG2 ? ptx::cluster_ctarank() : 0u;                  // position in the CTA pair
+    const uint32_t rank = CG2 ? (blockIdx.x & 1u) : 0u;                       // position in the CTA pair (clusters are (2,1,1))
     const int worker = CG2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;        // tile-loop start
     const int nworkers = CG2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;        // tile-loop stride
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
+            ptx::mbar_init(full + s, HALO ? 1 : 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
                                           // producers announce the bytes of both CTAs, the peer only issues its loads)
             ptx::mbar_init(empty + s, 1);
         }
@@ -172,6 +188,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         ptx::mbar_init(tempty, CG2 ? 8 : 128);  // pairs: one arrival per epilogue warp of both CTAs
         ptx::mbar_init(tempty + 1, CG2 ? 8 : 128);
         ptx::mbar_init(drain, 1);
+        for (int s = 0; s < 4; ++s) {
+            ptx::mbar_init(fullA + s, 1);
+            ptx::mbar_init(emptyA + s, 1);
+        }
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -195,12 +215,111 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
 
     if (warp == 0 || warp == 6) {
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
-        if (lane == 0) {
+        // Both producer warps run their loops converged; `leader` predicates the instructions that must be issued once.
+        const uint32_t leader = ptx::elect_one() ? 1u : 0u;
+        if (HALO) {
+            {
+                const bool isA = warp == 0;
+                if (leader) ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB[0]);
+                const int n_tiles = p.n_tiles, cbs = p.kc_per_tap, bn_own = p.BN / 2;
+                bool ok = true;
+                int issued = 0;
+                if (isA) {
+                    const int a_slots = p.a_slots, boxes = p.slab_boxes, box_pix = p.box_pix, Wp = p.Wp, HpWp = p.Hp * p.Wp;
+                    const uint32_t slab_bytes = p.slab_bytes, box_bytes = (uint32_t)box_pix * 128u;
+                    const uint32_t base_u32 = ptx::smem_u32(sA), fullA_local = ptx::smem_u32(fullA);
+                    const uint32_t fullA0 = ptx::mapa_u32(fullA_local, 0u);
+                    const int npos = (int)p.npos, rows_cta = TC_BM * mh;
+                    int sa = 0;
+                    uint32_t pha = 0;
+                    for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
+                        const int m_tile = tile / n_tiles;
+                        const int s0 = (m_tile * 2 + (int)rank) * rows_cta;  // first padded-raster position of this CTA's slab
+                        for (int cb = 0; cb < cbs; ++cb) {
+                            if (!wait_bar_fast(emptyA + sa, pha ^ 1u, abort_flag, p.status, 1)) {
+                                ok = false;
+                                break;
+                            }
+                            if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, fullA_local + 8u * (uint32_t)sa, 2u * slab_bytes);
+                            const uint32_t bar = fullA0 + 8u * (uint32_t)sa;
+                            uint32_t dst = base_u32 + (uint32_t)sa * slab_bytes;
+                            for (int b = 0; b < boxes; ++b) {
+                                // a box that would start past the last position feeds discarded rows only: fetch position 0 instead
+                                int q = s0 + b * box_pix;
+                                if (q >= npos) q = 0;
+                                const int n = q / HpWp, r = q - n * HpWp;
+                                const int hp = r / Wp, wp = r - hp * Wp;
+                                ptx::tma_load_im2col_4d_cg2_if(leader, dst, &p.tmA, bar, cb * 64, wp - 1, hp - 1, n, 0, 0);
+                                dst += box_bytes;
+                            }
+                            ++issued;
+                            if (++sa == a_slots) {
+                                sa = 0;
+                                pha ^= 1u;
+                            }
+                        }
+                    }
+                    if (!ok) {
+                        // gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited
+                        const int back = issued < a_slots ? issued : a_slots;
+                        for (int b = 0; b < back; ++b) {
+                            sa = (sa == 0) ? a_slots - 1 : sa - 1;
+                            if (sa == a_slots - 1) pha ^= 1u;
+                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(fullA + sa, pha); ++i) {
+                            }
+                        }
+                    }
+                } else {
+                    const int kpb = p.kpb, stages = p.stages, Ca = p.Ca, BN = p.BN, ntaps = p.cls_ntaps[0];
+                    const uint32_t b_sub = p.b_sub_bytes, stage_bytes = p.b_stage_bytes;
+                    const uint32_t tx = 2u * (uint32_t)kpb * (uint32_t)(bn_own * 128);
+                    const uint32_t base_u32 = ptx::smem_u32(sB), full_local = ptx::smem_u32(full);
+                    const uint32_t full0 = ptx::mapa_u32(full_local, 0u);
+                    int s = 0;
+                    uint32_t ph = 0;
+                    for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
+                        const int n_tile = tile % n_tiles;
+                        const int brow = n_tile * BN + (int)rank * bn_own;
+                        for (int cb = 0; ok && cb < cbs; ++cb) {
+                            for (int tap0 = 0; tap0 < ntaps; tap0 += kpb) {
+                                if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, 5)) {
+                                    ok = false;
+                                    break;
+                                }
+                                if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, full_local + 8u * (uint32_t)s, tx);
+                                const uint32_t bar = full0 + 8u * (uint32_t)s;
+                                uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
+                                for (int j = 0; j < kpb; ++j) {
+                                    ptx::tma_load_2d_cg2_if(leader, dst, &p.tmB[0], bar, (tap0 + j) * Ca + cb * 64, brow);
+                                    dst += b_sub;
+                                }
+                                ++issued;
+                                if (++s == stages) {
+                                    s = 0;
+                                    ph ^= 1u;
+                                }
+                            }
+                        }
+                    }
+                    if (!ok) {
+                        const int back = issued < stages ? issued : stages;
+                        for (int b = 0; b < back; ++b) {
+                            s = (s == 0) ? stages - 1 : s - 1;
+                            if (s == stages - 1) ph ^= 1u;
+                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
+                            }
+                        }
+                    }
+                }
+            }
+        } else {
             const bool isA = warp == 0;
-            if (isA) {
-                ptx::prefetch_tmap(&p.tmA);
-            } else {
-                for (int c = 0; c < p.nclasses; ++c) ptx::prefetch_tmap(&p.tmB[c]);
+            if (leader) {
+                if (isA) {
+                    ptx::prefetch_tmap(&p.tmA);
+                } else {
+                    for (int c = 0; c < p.nclasses; ++c) ptx::prefetch_tmap(&p.tmB[c]);
+                }
             }
             int s = 0;
             uint32_t ph = 0;
@@ -251,21 +370,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         NB_DBG_ADD(dbg_wait_empty);
                     }
                     const uint32_t bar = full_u32 + 8u * (uint32_t)s;
-                    if (!CG2) ptx::mbar_expect_tx_u32(bar, kb_bytes * (uint32_t)nkb);
-                    else if (rank == 0) ptx::mbar_expect_tx_u32(ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
+                    if (!CG2) ptx::mbar_expect_tx_u32_if(leader, bar, kb_bytes * (uint32_t)nkb);
+                    else if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
                     uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
                     for (int j = 0; j < nkb; ++j) {
                         if (isA) {
                             if (a_tiled) {
-                                if (CG2) ptx::tma_load_2d_cg2(dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32(dst, tm, bar, kc * KC, m0);
+                                if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, kc * KC, m0);
                             } else {
                                 if (CG2)
-                                    ptx::tma_load_im2col_4d_cg2(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                                    ptx::tma_load_im2col_4d_cg2_if(leader, dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
                                 else
-                                    ptx::tma_load_im2col_4d_u32(dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                                    ptx::tma_load_im2col_4d_u32_if(leader, dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
                             }
                         } else {
-                            if (CG2) ptx::tma_load_2d_cg2(dst, tm, bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32(dst, tm, bar, tap * Ca + kc * KC, brow);
+                            if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow);
                         }
                         dst += sub_bytes;
                         if (++kc == kc_per_tap) {
@@ -281,7 +400,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                 }
             }
 #ifdef NB_TC_DEBUG_TIMING
-            if (p.dbg && isA) { p.dbg[blockIdx.x * 8 + 0] = dbg_wait_empty; p.dbg[blockIdx.x * 8 + 1] = clock64() - dbg_start; }
+            if (p.dbg && isA && leader) { p.dbg[blockIdx.x * 8 + 0] = dbg_wait_empty; p.dbg[blockIdx.x * 8 + 1] = clock64() - dbg_start; }
 #endif
             if (!ok) {
                 // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
@@ -296,12 +415,103 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (one thread; in a pair only rank 0)
-        if (lane == 0 && rank == 0) {
+        const uint32_t leader = ptx::elect_one() ? 1u : 0u;  // the whole warp runs the loop, this lane issues
+        if (HALO) {
+            if (rank == 0) {
+                int s = 0, sa = 0, acc = 0;
+                uint32_t ph = 0, pha = 0, acc_ph = 0;
+                bool ok = true;
+#ifdef NB_TC_DEBUG_TIMING
+                long long dbg_wait_full = 0, dbg_wait_tempty = 0;
+                const long long dbg_start = clock64();
+#endif
+                const int kpb = p.kpb, stages = p.stages, a_slots = p.a_slots, cbs = p.kc_per_tap, ntaps = p.cls_ntaps[0];
+                const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
+                const uint64_t b_sub16 = (uint64_t)(p.b_sub_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
+                const uint64_t slab16 = (uint64_t)(p.slab_bytes >> 4);
+                const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), 16, 1024, ptx::kSwizzle128);
+                const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, 1024, ptx::kSwizzle128);
+                const uint32_t empty_u32 = ptx::smem_u32(empty), emptyA_u32 = ptx::smem_u32(emptyA), tfull_u32 = ptx::smem_u32(tfull);
+                for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
+                    {
+                        NB_DBG_T0();
+                        if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
+                        NB_DBG_ADD(dbg_wait_tempty);
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
+                    uint32_t accumulate = 0;
+                    for (int cb = 0; ok && cb < cbs; ++cb) {
+                        {
+                            NB_DBG_T0();
+                            if (!wait_bar_fast(fullA + sa, pha, abort_flag, p.status, 6)) {
+                                ok = false;
+                                break;
+                            }
+                            NB_DBG_ADD(dbg_wait_full);
+                        }
+                        ptx::tc_fence_after();
+                        const uint64_t da_slab = da0 + (uint64_t)sa * slab16;
+                        for (int tap0 = 0; tap0 < ntaps; tap0 += kpb) {
+                            {
+                                NB_DBG_T0();
+                                if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
+                                    ok = false;
+                                    break;
+                                }
+                                NB_DBG_ADD(dbg_wait_full);
+                            }
+                            ptx::tc_fence_after();
+                            uint64_t db = db0 + (uint64_t)s * b_stage16;
+                            for (int j = 0; j < kpb; ++j) {
+                                const uint64_t da_tap = da_slab + (uint64_t)p.tap_off16[tap0 + j];
+                                for (int h = 0; h < mh; ++h) {
+                                    const uint64_t dah = da_tap + (uint64_t)h * (uint64_t)((TC_BM * 128) >> 4);
+                                    // the rows of a tap start anywhere inside an 8-row swizzle group; the pattern itself stays
+                                    // anchored at 1024-byte boundaries of shared memory, where TMA put it, so the descriptor's
+                                    // base-offset field stays zero (measured: setting it to the row phase gives wrong sums)
+                                    const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
+                                    ptx::umma_f16_cg2_if(leader, dt, dah, db, idesc, accumulate);
+                                    ptx::umma_f16_cg2_if(leader, dt, dah + 2, db + 2, idesc, 1u);
+                                    ptx::umma_f16_cg2_if(leader, dt, dah + 4, db + 4, idesc, 1u);
+                                    ptx::umma_f16_cg2_if(leader, dt, dah + 6, db + 6, idesc, 1u);
+                                }
+                                accumulate = 1u;
+                                db += b_sub16;
+                            }
+                            ptx::umma_commit_cg2_mc_if(leader, empty_u32 + 8u * (uint32_t)s, 3);
+                            if (++s == stages) {
+                                s = 0;
+                                ph ^= 1u;
+                            }
+                        }
+                        if (!ok) break;
+                        ptx::umma_commit_cg2_mc_if(leader, emptyA_u32 + 8u * (uint32_t)sa, 3);
+                        if (++sa == a_slots) {
+                            sa = 0;
+                            pha ^= 1u;
+                        }
+                    }
+                    if (!ok) break;
+                    ptx::umma_commit_cg2_mc_if(leader, tfull_u32 + 8u * (uint32_t)acc, 3);
+                    if (++acc == nbuf) {
+                        acc = 0;
+                        acc_ph ^= 1u;
+                    }
+                }
+#ifdef NB_TC_DEBUG_TIMING
+                if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
+#endif
+                ptx::umma_commit_cg2_if(leader, ptx::smem_u32(drain));
+                for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
+                }
+            }
+        } else if (rank == 0) {
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
 #ifdef NB_TC_DEBUG_TIMING
-            long long dbg_wait_full = 0, dbg_wait_tempty = 0;
+            long long dbg_wait_full = 0, dbg_wait_tempty = 0, dbg_wait_first = 0;
             const long long dbg_start = clock64();
 #endif
             const int ksteps = p.KC / 16, kpb = p.kpb, stages = p.stages;
@@ -333,7 +543,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                             ok = false;
                             break;
                         }
-                        NB_DBG_ADD(dbg_wait_full);
+                        if (kb0 == 0) { NB_DBG_ADD(dbg_wait_first); } else { NB_DBG_ADD(dbg_wait_full); }
                     }
                     ptx::tc_fence_after();
                     uint64_t da = da_s, db = db_s;
@@ -342,25 +552,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                             const uint64_t dah = da + (uint64_t)h * a_half16;
                             const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
                             if (CG2) {
-                                ptx::umma_f16_cg2(dt, dah, db, idesc, accumulate);
-                                ptx::umma_f16_cg2(dt, dah + 2, db + 2, idesc, 1u);
-                                ptx::umma_f16_cg2(dt, dah + 4, db + 4, idesc, 1u);
-                                ptx::umma_f16_cg2(dt, dah + 6, db + 6, idesc, 1u);
+                                ptx::umma_f16_cg2_if(leader, dt, dah, db, idesc, accumulate);
+                                ptx::umma_f16_cg2_if(leader, dt, dah + 2, db + 2, idesc, 1u);
+                                ptx::umma_f16_cg2_if(leader, dt, dah + 4, db + 4, idesc, 1u);
+                                ptx::umma_f16_cg2_if(leader, dt, dah + 6, db + 6, idesc, 1u);
                             } else if (ksteps == 4) {
-                                ptx::umma_f16(dt, dah, db, idesc, accumulate);
-                                ptx::umma_f16(dt, dah + 2, db + 2, idesc, 1u);
-                                ptx::umma_f16(dt, dah + 4, db + 4, idesc, 1u);
-                                ptx::umma_f16(dt, dah + 6, db + 6, idesc, 1u);
+                                ptx::umma_f16_if(leader, dt, dah, db, idesc, accumulate);
+                                ptx::umma_f16_if(leader, dt, dah + 2, db + 2, idesc, 1u);
+                                ptx::umma_f16_if(leader, dt, dah + 4, db + 4, idesc, 1u);
+                                ptx::umma_f16_if(leader, dt, dah + 6, db + 6, idesc, 1u);
                             } else {
                                 for (int k = 0; k < ksteps; ++k)
-                                    ptx::umma_f16(dt, dah + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (k | (int)accumulate) ? 1u : 0u);
+                                    ptx::umma_f16_if(leader, dt, dah + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (k | (int)accumulate) ? 1u : 0u);
                             }
                         }
                         accumulate = 1u;
                         da += a_sub16;
                         db += b_sub16;
                     }
-                    if (CG2) ptx::umma_commit_cg2_mc(empty_u32 + 8u * (uint32_t)s, 3); else ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
+                    if (CG2) ptx::umma_commit_cg2_mc_if(leader, empty_u32 + 8u * (uint32_t)s, 3); else ptx::umma_commit_u32_if(leader, empty_u32 + 8u * (uint32_t)s);
                     da_s += a_stage16;
                     db_s += b_stage16;
                     if (++s == stages) {
@@ -371,17 +581,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     }
                 }
                 if (!ok) break;
-                if (CG2) ptx::umma_commit_cg2_mc(tfull_u32 + 8u * (uint32_t)acc, 3); else ptx::umma_commit(tfull + acc);
+                if (CG2) ptx::umma_commit_cg2_mc_if(leader, tfull_u32 + 8u * (uint32_t)acc, 3); else ptx::umma_commit_u32_if(leader, tfull_u32 + 8u * (uint32_t)acc);
                 if (++acc == nbuf) {
                     acc = 0;
                     acc_ph ^= 1u;
                 }
             }
 #ifdef NB_TC_DEBUG_TIMING
-            if (p.dbg) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
+            if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; p.dbg[blockIdx.x * 8 + 7] = dbg_wait_first; }
 #endif
             // Make sure every MMA issued by this thread has retired before TMEM is released.
-            if (CG2) ptx::umma_commit_cg2(ptx::smem_u32(drain)); else ptx::umma_commit(drain);
+            if (CG2) ptx::umma_commit_cg2_if(leader, ptx::smem_u32(drain)); else ptx::umma_commit_u32_if(leader, ptx::smem_u32(drain));
             for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
             }
         }
@@ -430,6 +640,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             for (int h = 0; h < mh; ++h) {
                 const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
                 const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride);
+                long long halo_pix = -1;  // halo mode: output pixel of this thread's row, -1 on the padding ring / past the end
+                if (HALO) {
+                    const long long pos = m0 + row + p.Wp + 1;  // output tiles start one padded row and one pixel in
+                    if (pos < p.npos) {
+                        const int HpWp = p.Hp * p.Wp;
+                        const int n = (int)(pos / HpWp), r = (int)(pos - (long long)n * HpWp);
+                        const int hp = r / p.Wp, wp = r - hp * p.Wp;
+                        if (hp >= 1 && hp <= p.Hin && wp >= 1 && wp <= p.Win) halo_pix = ((long long)n * p.Hin + (hp - 1)) * p.Win + (wp - 1);
+                    }
+                }
                 for (int cbase = 0; cbase < p.BN; cbase += CW) {
                     const int ncol = (p.BN - cbase < CW) ? p.BN - cbase : CW;  // multiple of 16
                     // ---- TMEM -> registers -> staging (this thread's row)
@@ -439,6 +659,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0), r);
                         if (two) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0 + 16), r + 16);
                         ptx::tmem_ld_wait();
+                        const int sat_before = sat;
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
                             if (hh == 1 && !two) break;
@@ -452,6 +673,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                             v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat);
                             v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat);
                             v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat);
+                            if (HALO && halo_pix < 0) {  // discarded row: zeros keep the channel sums exact
+                                v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
+                                sat = sat_before;
+                            }
                             *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2) = v0;
                             *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2 + 16) = v1;
                         }
@@ -498,7 +723,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                     if (!(p.variant & 32)) {
                         const int cpr = ncol / 8;  // 16-byte pieces per staged row (<= 16)
                         long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
-                        if (pixrow >= p.M) {
+                        if (HALO) {
+                            pixrow = halo_pix;
+                        } else if (pixrow >= p.M) {
                             pixrow = -1;
                         } else if (p.os != 1) {
                             const int j = (int)(pixrow % p.Wq);
@@ -590,6 +817,10 @@ struct IgemmCfg {
     int Ca = 0, rowsB = 0, ntaps = 0;
     int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
     bool cg2 = false;  // CTA pairs (tcgen05 cta_group::2)
+    bool halo = false;  // tap-reuse variant (3x3, stride 1)
+    int Wp = 0, Hp = 0, Hin = 0, Win = 0, Nimg = 0, slab_boxes = 0, box_pix = 0, a_slots = 0;
+    uint32_t slab_bytes = 0;
+    long long npos = 0;
     uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
@@ -741,6 +972,72 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     return c;
 }
 
+// Tile configuration of the tap-reuse variant for a 3x3 stride-1 convolution over [N][H][W][Ca] with rowsB output channels.
+// Rows of the GEMM are padded-raster positions; CTA t of the launch order owns positions [W+3 + t*128*mh, +128*mh) and
+// fetches the slab [t*128*mh, +128*mh + 2*(W+2) + 2).
+inline IgemmCfg halo_configure(int N, int H, int W, int Ca, int rowsB, int ldo, int sm_count) {
+    IgemmCfg c;
+    c.Ca = Ca; c.rowsB = rowsB; c.ntaps = 9; c.KC = 64;
+    c.M = (long long)N * H * W;
+    // Off unless NB_TC_HALO=1.  Measured on B200 over the detector's 3x3 layers: the slab cuts the bytes TMA writes to
+    // shared memory by 1.3-1.9x, but a tap whose first row is not a multiple of eight rows into the slab makes every
+    // tcgen05.mma read its A operand ~1.2x slower (119 instead of 92-96 cycles per 256 x 192 x 16 MMA), and 5-17 % of the
+    // rows are padding; only the 20 x 20 layers with 288 channels gained (10 %), the others lost 5-20 %.
+    if (!(getenv("NB_TC_HALO") && atoi(getenv("NB_TC_HALO")) == 1)) return c;
+    if (Ca % 16 || rowsB % 16) return c;
+    const int Wp = W + 2, Hp = H + 2;
+    const long long npos = (long long)N * Hp * Wp;
+    if (npos >= (1LL << 30)) return c;
+    const int force_bn = getenv("NB_TC_BN") ? atoi(getenv("NB_TC_BN")) : 0;
+    const int force_mh = getenv("NB_TC_MH") ? atoi(getenv("NB_TC_MH")) : 0;
+    const int force_kpb = getenv("NB_TC_KPB") ? atoi(getenv("NB_TC_KPB")) : 0;
+    const long long span = npos - 2LL * (Wp + 1);  // positions from the first to the last real output
+    for (int bn = std::min(256, rowsB) / 16 * 16; bn >= 16 && !c.BN; bn -= 16) {
+        if (rowsB % bn) continue;
+        if (force_bn && bn != force_bn && rowsB % force_bn == 0) continue;
+        const int acc_stride = bn <= 32 ? 32 : bn <= 64 ? 64 : bn <= 128 ? 128 : 256;
+        for (int mh = (4 * acc_stride <= 512) ? 2 : 1; mh >= 1 && !c.BN; --mh) {
+            if (force_mh && mh != force_mh && force_mh * acc_stride <= 512) continue;
+            const int rows_cta = TC_BM * mh;
+            const long long cta_tiles = (span + rows_cta - 1) / rows_cta;
+            const long long pair_tiles = (cta_tiles + 1) / 2;
+            // two row blocks per CTA only while every pair still gets a tile
+            if (mh == 2 && !force_mh && pair_tiles * (rowsB / bn) < sm_count / 2) continue;
+            const int R = rows_cta + 2 * Wp + 2;
+            const int boxes = (R + 255) / 256;
+            const int box_pix = ((R + boxes - 1) / boxes + 7) / 8 * 8;
+            const uint32_t slab = (uint32_t)boxes * (uint32_t)box_pix * 128u;
+            const uint32_t b_sub = (uint32_t)((bn / 2 * 128 + 1023) / 1024 * 1024);
+            const size_t fixed = igemm_fixed_smem(bn, ldo);
+            const double tap_cycles = 4.0 * mh * std::max(32.0, bn / 2.0);  // tensor cycles per tap of one 64-channel block
+            int kpb = tap_cycles < 300.0 ? 3 : 1;
+            if (force_kpb == 1 || force_kpb == 3 || force_kpb == 9) kpb = force_kpb;
+            int a_slots = 2, stages = 0;
+            for (;;) {
+                if (fixed + (size_t)a_slots * slab < kMaxSmem) stages = (int)std::min<size_t>(8, (kMaxSmem - fixed - (size_t)a_slots * slab) / ((size_t)kpb * b_sub));
+                if (stages >= 3 || kpb == 1) break;
+                kpb = 1;
+            }
+            if (stages < 2) continue;
+            c.BN = bn; c.mh = mh; c.kpb = kpb; c.stages = stages; c.acc_stride = acc_stride;
+            c.acc_bufs = (2 * mh * acc_stride <= 512) ? 2 : 1;
+            c.a_sub = 0; c.b_sub = b_sub; c.a_stage = slab; c.b_stage = b_sub * (uint32_t)kpb;
+            c.cg2 = true; c.halo = true;
+            c.Wp = Wp; c.Hp = Hp; c.Hin = H; c.Win = W; c.Nimg = N;
+            c.slab_boxes = boxes; c.box_pix = box_pix; c.a_slots = a_slots; c.slab_bytes = slab; c.npos = npos;
+            c.m_tiles = (int)pair_tiles;
+        }
+    }
+    if (!c.BN) return c;
+    c.n_tiles = rowsB / c.BN;
+    c.stage_cols = igemm_stage_cols(c.BN);
+    c.tmem_cols = std::max(32, c.acc_bufs * c.mh * c.acc_stride);
+    c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.a_slots * c.slab_bytes + (size_t)c.stages * c.b_stage, 120 * 1024);
+    c.grid = 2 * (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count / 2);
+    c.ok = true;
+    return c;
+}
+
 inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.M = c.M;
     P.Ca = c.Ca; P.KC = c.KC; P.kc_per_tap = (c.Ca + c.KC - 1) / c.KC;
@@ -756,6 +1053,18 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
         fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
                 c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
     P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
+    P.halo = c.halo ? 1 : 0;
+    if (c.halo) {
+        P.Wp = c.Wp; P.Hp = c.Hp; P.Hin = c.Hin; P.Win = c.Win; P.Nimg = c.Nimg;
+        P.slab_boxes = c.slab_boxes; P.box_pix = c.box_pix; P.a_slots = c.a_slots; P.slab_bytes = c.slab_bytes; P.npos = c.npos;
+        if (getenv("NB_TC_VERBOSE"))
+            fprintf(stderr, "[nb_cbs]   halo: Wp=%d slab=%d boxes x %d positions (%u bytes) x %d slots, taps per B stage %d\n", c.Wp, c.slab_boxes, c.box_pix,
+                    c.slab_bytes, c.a_slots, c.kpb);
+    }
+}
+// Start of tap t inside a slab: off_h rows of the padded raster down, off_w positions right (16-byte units, 8 per position).
+inline void fill_halo_taps(IgemmParams& P) {
+    for (int t = 0; t < 9; ++t) P.tap_off16[t] = (uint32_t)((int)P.off_h[0][t] * P.Wp + (int)P.off_w[0][t]) * 8u;
 }
 
 // im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
@@ -786,16 +1095,16 @@ inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, lo
     return true;
 }
 
-template <typename OutT, bool STATS, bool CG2> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+template <typename OutT, bool STATS, bool CG2, bool HALO> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
         attr_set = true;
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2>, dim3((unsigned)s.cfg.grid), dim3(TC_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO>, dim3((unsigned)s.cfg.grid), dim3(TC_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
@@ -803,7 +1112,8 @@ template <typename OutT, bool STATS, bool CG2> inline nb_status launch_igemm_imp
     return NB_OK;
 }
 template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
-    return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true>(s, st) : launch_igemm_impl<OutT, STATS, false>(s, st);
+    if (s.cfg.halo) return launch_igemm_impl<OutT, STATS, true, true>(s, st);
+    return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true, false>(s, st) : launch_igemm_impl<OutT, STATS, false, false>(s, st);
 }
 
 }  // namespace tcdetail
@@ -821,7 +1131,9 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
     const bool even = (g.h % 2 == 0) && (g.w % 2 == 0);
     // ---- fprop: A = x (im2col), B = w [Cout][k*k*Cin]
     if (g.c_in % 16 == 0 && g.c_out % 16 == 0) {
-        IgemmCfg c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count, 1);
+        IgemmCfg c;
+        if (g.k == 3 && g.stride == 1 && g.pad == 1) c = halo_configure(g.n, g.h, g.w, g.c_in, g.c_out, g.c_out, sm_count);
+        if (!c.ok) c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count, 1);
         if (c.ok) {
             tc->fp.cfg = c;
             IgemmParams& P = tc->fp.prm;
@@ -837,6 +1149,7 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
                 }
             P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1;
             P.a_tiled = (g.k == 1 && g.stride == 1) ? 1 : 0;
+            if (c.halo) fill_halo_taps(P);
             tc->fprop = true;
             tc->fprop_parts = c.grid;
         }
@@ -891,10 +1204,13 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
             P.Hq = g.h / 2; P.Wq = g.w / 2; P.ts = 1; P.lo_w = P.lo_h = 0;
             P.Hout = g.h; P.Wout = g.w; P.os = 2;
         }
-        IgemmCfg c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls);
+        IgemmCfg c;
+        if (g.k == 3 && g.stride == 1 && g.pad == 1) c = halo_configure(g.n, g.h, g.w, g.c_out, g.c_in, g.c_in, sm_count);
+        if (!c.ok) c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls);
         if (c.ok) {
             tc->dg.cfg = c;
             fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
+            if (c.halo) fill_halo_taps(P);
             P.nclasses = ncls; P.tiles_per_class = c.m_tiles * c.n_tiles;
             P.ldo = g.c_in;
             W.nclasses = ncls;
@@ -980,7 +1296,10 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     TcGemmSlot& S = tc->fp;
     if (S.a_ptr != x || S.b_ptr != w) {
         const int up = g.pad - (g.k - 1);
-        if (S.prm.a_tiled) {
+        if (S.cfg.halo) {
+            // traversal over the padded raster: window start from -1 to W (one past each edge), tap offsets always zero
+            if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -1, 1, 1, 64, S.cfg.box_pix)) return NB_ERR_CUDA;
+        } else if (S.prm.a_tiled) {
             if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
         } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh)) {
             return NB_ERR_CUDA;
@@ -1009,7 +1328,11 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
     if (S.a_ptr != dy || S.b_ptr != wt) {
         // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
         const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
-        if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
+        if (S.cfg.halo) {
+            if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, -1, 1, 1, 64, S.cfg.box_pix)) return NB_ERR_CUDA;
+        } else if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) {
+            return NB_ERR_CUDA;
+        }
         for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
             const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
             if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;

@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     pdl_launch_dependents();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     // tile = (m_tile, n_tile, split), split fastest so that CTAs sharing a pixel range run together
     const int split = blockIdx.x % p.splits;
     const int tn = blockIdx.x / p.splits;
@@ -74,9 +74,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 
     if (warp == 0 || warp == 6) {
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds x, warp 6 feeds dy
-        if (lane == 0 && nchunks > 0) {
+        // the whole warp runs the loop converged; `leader` predicates the instructions that must be issued once
+        const uint32_t leader = ptx::elect_one() ? 1u : 0u;
+        if (nchunks > 0) {
             const bool isA = warp == 0;
-            ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
+            if (leader) ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
             int s = 0, issued = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -104,16 +106,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                     break;
                 }
                 const uint32_t bar = full_u32 + 8u * (uint32_t)s;
-                ptx::mbar_expect_tx_u32(bar, blk * (uint32_t)nblk);
+                ptx::mbar_expect_tx_u32_if(leader, bar, blk * (uint32_t)nblk);
                 const uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
                 if (isA) {
                     const int j0 = m0 % Wq, t1 = m0 / Wq;
                     const int i0 = t1 % Hq, n0 = t1 / Hq;
                     const int cw = p.lo_w + j0 * ts, chh = p.lo_h + i0 * ts;
-                    ptx::tma_load_im2col_4d_u32(dst, tm, bar, c0v[0], cw, chh, n0, ow0, oh0);
-                    ptx::tma_load_im2col_4d_u32(dst + blk, tm, bar, c0v[1], cw, chh, n0, ow1, oh1);
+                    ptx::tma_load_im2col_4d_u32_if(leader, dst, tm, bar, c0v[0], cw, chh, n0, ow0, oh0);
+                    ptx::tma_load_im2col_4d_u32_if(leader, dst + blk, tm, bar, c0v[1], cw, chh, n0, ow1, oh1);
                 } else {
-                    for (int b = 0; b < nblk; ++b) ptx::tma_load_2d_u32(dst + (uint32_t)b * blk, tm, bar, bcol + b * 64, m0);
+                    for (int b = 0; b < nblk; ++b) ptx::tma_load_2d_u32_if(leader, dst + (uint32_t)b * blk, tm, bar, bcol + b * 64, m0);
                 }
                 ++issued;
                 if (++s == stages) {
@@ -134,7 +136,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (one thread)
-        if (lane == 0 && nchunks > 0) {
+        const uint32_t leader = ptx::elect_one() ? 1u : 0u;
+        if (nchunks > 0) {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -157,12 +160,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                 uint64_t da = da_s, db = db_s;
 #pragma unroll 4
                 for (int k = 0; k < ksteps; ++k) {
-                    ptx::umma_f16(tmem_base, da, db, idesc, accumulate);
+                    ptx::umma_f16_if(leader, tmem_base, da, db, idesc, accumulate);
                     accumulate = 1u;
                     da += 128;  // 2048 bytes >> 4
                     db += 128;
                 }
-                ptx::umma_commit_u32(empty_u32 + 8u * (uint32_t)s);
+                ptx::umma_commit_u32_if(leader, empty_u32 + 8u * (uint32_t)s);
                 da_s += a_stage16;
                 db_s += b_stage16;
                 if (++s == stages) {
@@ -173,11 +176,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                 }
             }
             if (ok) {
-                ptx::umma_commit(tfull);
+                ptx::umma_commit_u32_if(leader, ptx::smem_u32(tfull));
             } else {
                 // tfull is never signalled (the epilogue's bounded wait sees the abort flag); make sure the MMAs already
                 // issued have retired before TMEM is released
-                ptx::umma_commit(drain);
+                ptx::umma_commit_u32_if(leader, ptx::smem_u32(drain));
                 for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
                 }
             }

@@ -90,6 +90,18 @@ def test_forced_cuda_core_path_matches_oracle(shape):
     _compare(out, _oracle(inp), 0)
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[11], S(3, 9, 11, 32, 16, 3, 1), S(2, 24, 24, 96, 192, 3, 1)],
+                         ids=lambda s: s.name)
+def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
+    """The slab variant of the 3x3 stride-1 kernels (rows = positions of the zero-padded raster, nine taps = nine row
+    offsets into one slab) is off by default; it must stay correct: images meet inside tiles, the padding ring is
+    discarded and excluded from the statistics."""
+    monkeypatch.setenv("NB_TC_HALO", "1")
+    inp, blk, out = _run_block(shape, 0, cfg_id=13, affine="random")
+    assert blk.plan.paths["fprop"] == 2 and blk.plan.paths["dgrad"] == 2
+    _compare(out, _oracle(inp), 0)
+
+
 def test_config1_fresh_bn_both_modes():
     shape, = wl.config_shapes(1)
     for mode in (1, 0):
