@@ -39,7 +39,8 @@ struct IgemmParams {
     int BN, n_tiles, m_tiles;
     int mh;                      // 128-row sub-tiles per tile (1 or 2): the tile is [128*mh x BN]
     int acc_bufs;                // accumulator sets in TMEM (2 when 2*mh*acc_stride <= 512)
-    int stage_cols;              // columns the epilogue stages per pass
+    int ncol_a;                  // columns of a tile that epilogue team 0 handles (team 1: the other BN - ncol_a)
+    int stage_cw;                // columns per staging pass of a team (<= 64)
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
     int variant;                 // experiment switches
@@ -63,11 +64,14 @@ struct IgemmParams {
 #ifdef NB_TC_DEBUG_TIMING
 #define NB_DBG_T0() const long long dbg_t0__ = clock64()
 #define NB_DBG_ADD(var) var += clock64() - dbg_t0__
+#define NB_DBG_PHASE(var) { const long long dbg_now__ = clock64(); var += dbg_now__ - dbg_ph__; dbg_ph__ = dbg_now__; }
 #else
 #define NB_DBG_T0()
 #define NB_DBG_ADD(var)
+#define NB_DBG_PHASE(var)
 #endif
 constexpr int TC_BM = 128;
+constexpr int IG_THREADS = 352;  // implicit-GEMM kernel: the roles below plus a second epilogue team in warps 7-10
 constexpr int TC_THREADS = 224;  // warp 0: TMA producer for A, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue, warp 6: TMA producer for B
 constexpr int WG_THREADS = 192;  // wgrad kernel: warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 
@@ -81,7 +85,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 __device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
     uint64_t t0 = 0;
     for (uint32_t i = 0;; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (ptx::mbar_try_wait_parked(bar, parity, 4000u)) return true;
         if ((i & 127u) == 127u) {
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
@@ -108,6 +112,22 @@ __device__ __forceinline__ bool wait_bar_fast(uint64_t* bar, uint32_t parity, vo
 }
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// The same over the 256 threads of the implicit-GEMM kernel's two epilogue teams.
+__device__ __forceinline__ void epi2_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool epi2_bar_and(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 256, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t"
+        "}\n"
+        : "=r"(r)
+        : "r"((uint32_t)ok)
+        : "memory");
+    return r != 0;
+}
 // Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the same decision.
 __device__ __forceinline__ bool epi_bar_and(bool ok) {
     uint32_t r;
@@ -129,14 +149,13 @@ template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, fl
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// fp16 stores saturate to the largest finite value; `sat` collects, per 16-bit half, a flag bit (bit 15 / 31) that is set
+// when a stored magnitude is 65504 (0x7bff) or an exceptional pattern above it.
 template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, int* sat) {
-    if (fabsf(a) > 65504.f || fabsf(b) > 65504.f) {
-        *sat += 1;
-        a = fminf(fmaxf(a, -65504.f), 65504.f);
-        b = fminf(fmaxf(b, -65504.f), 65504.f);
-    }
-    __half2 v = __floats2half2_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&v);
+    uint32_t v;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(v) : "f"(b), "f"(a));
+    *sat |= (int)((v & 0x7fff7fffu) + 0x04010401u);
+    return v;
 }
 
 // CG2 = the CTAs run as pairs (clusters of two): rank 0 issues tcgen05.mma.cta_group::2 with M = 256; each CTA owns 128
@@ -147,16 +166,16 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
 // shared memory drop from 9 x 128*mh rows to 128*mh + 2*(W+2) + 2 rows per block.  Rows that fall on the padding ring
 // are computed and discarded.
 template <typename OutT, bool STATS, bool CG2, bool HALO>
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
+__global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
     static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = sA + (HALO ? (size_t)p.a_slots * p.slab_bytes : (size_t)p.stages * p.a_stage_bytes);
-    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging [128 rows][CW columns] of OutT, row pitch CW*2+16 bytes
-    const int CW = p.stage_cols;                             // columns staged per pass (<= 128)
-    const int pitch = CW * 2 + 16;
-    float* wstat = reinterpret_cast<float*>(stg + (size_t)TC_BM * pitch);  // [4 warps][2][ldo]: warp-private channel sums
+    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
+    const int cw = p.stage_cw;  // columns per staging pass (<= 64)
+    const int pitch = cw * 2 + 16;
+    float* wstat = reinterpret_cast<float*>(stg + (size_t)2 * TC_BM * pitch);  // per team [4 warps][2][its columns of every n-tile]: warp-private channel sums
     uint64_t* bars = reinterpret_cast<uint64_t*>(wstat + (STATS ? 8 * p.ldo : 0));
     uint64_t* full = bars;                // [stages]
     uint64_t* empty = bars + p.stages;    // [stages]
@@ -185,8 +204,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         }
         ptx::mbar_init(tfull, 1);
         ptx::mbar_init(tfull + 1, 1);
-        ptx::mbar_init(tempty, CG2 ? 8 : 128);  // pairs: one arrival per epilogue warp of both CTAs
-        ptx::mbar_init(tempty + 1, CG2 ? 8 : 128);
+        ptx::mbar_init(tempty, CG2 ? 16 : 256);  // pairs: one arrival per epilogue warp of both CTAs
+        ptx::mbar_init(tempty + 1, CG2 ? 16 : 256);
         ptx::mbar_init(drain, 1);
         for (int s = 0; s < 4; ++s) {
             ptx::mbar_init(fullA + s, 1);
@@ -196,7 +215,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
         ptx::fence_mbar_init();
     }
     if (STATS) {
-        for (int c = threadIdx.x; c < 8 * p.ldo; c += TC_THREADS) wstat[c] = 0.f;
+        for (int c = threadIdx.x; c < 8 * p.ldo; c += IG_THREADS) wstat[c] = 0.f;
     }
     if (warp == 1) {
         if (CG2) {
@@ -596,18 +615,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2-5, 128 threads)
-        const int et = threadIdx.x - 64;          // 0..127
+        // ------------------------------------------------------------------ epilogue: two teams of four warps (warps 2-5 and 7-10)
+        // Every tile's columns are split between the teams (team 0: the first ncol_a columns, team 1: the rest), each team
+        // has its own staging buffer and running sums, and inside a team warp q owns accumulator rows [32q, 32q+32).
+        // The epilogue is bound by the latency of its own instruction stream (one warp per scheduler), so a second team
+        // nearly halves the time per tile.
+        const int team = warp >= 7 ? 1 : 0;
         const int lane_group = warp & 3;          // TMEM lanes this warp may read: rows [32*lane_group, +32) of a sub-tile
         const int row = lane_group * 32 + lane;   // accumulator row == sub-tile row
+        const int c_lo = team ? p.ncol_a : 0;     // first column (within the tile) and number of columns of this team
+        const int ncol = team ? p.BN - p.ncol_a : p.ncol_a;
+        const int st_ld = p.n_tiles * ncol;       // row length of this team's running sums: its columns of every n-tile
         int acc = 0, sat = 0;
         uint32_t acc_ph = 0;
-        float* my_stat = wstat + (size_t)lane_group * 2 * p.ldo;  // this warp's [2][ldo] running sums
-        uint8_t* my_row = stg + (size_t)row * pitch;
-        const uint8_t* my_rows = stg + (size_t)(lane_group * 32) * pitch;
+        float* team_stat = wstat + (team ? (size_t)8 * p.n_tiles * p.ncol_a : 0);  // [4 warps][2][st_ld]
+        float* my_stat = team_stat + (size_t)lane_group * 2 * st_ld;
+        uint8_t* stg_t = stg + (size_t)team * TC_BM * pitch;
+        uint8_t* my_row = stg_t + (size_t)row * pitch;
+        const uint8_t* my_rows = stg_t + (size_t)(lane_group * 32) * pitch;
         uint8_t* outb = static_cast<uint8_t*>(p.out);
 #ifdef NB_TC_DEBUG_TIMING
-        long long dbg_wait_tfull = 0;
+        long long dbg_wait_tfull = 0, dbg_ld = 0, dbg_pack = 0, dbg_stats = 0, dbg_store = 0, dbg_ph__ = 0;
         const long long dbg_start = clock64();
 #endif
         const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
@@ -616,14 +644,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
             NB_DBG_T0();
             bool ok = true;
-            // one poller per warp: 128 threads spinning on one mbarrier would crowd the shared-memory pipe
+            // one poller per warp: 256 threads spinning on one mbarrier would crowd the shared-memory pipe
             if (lane == 0) ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             NB_DBG_ADD(dbg_wait_tfull);
-            ok = epi_bar_and(ok);
+            ok = epi2_bar_and(ok);
             if (!ok) break;
             ptx::tc_fence_after();
-            if (p.variant & 8) {
+            if ((p.variant & 8) || ncol == 0) {
                 ptx::tc_fence_before();
                 if (CG2) {
                     __syncwarp();
@@ -639,7 +667,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             }
             for (int h = 0; h < mh; ++h) {
                 const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
-                const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride);
+                const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride) + (uint32_t)c_lo;
                 long long halo_pix = -1;  // halo mode: output pixel of this thread's row, -1 on the padding ring / past the end
                 if (HALO) {
                     const long long pos = m0 + row + p.Wp + 1;  // output tiles start one padded row and one pixel in
@@ -650,108 +678,148 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
                         if (hp >= 1 && hp <= p.Hin && wp >= 1 && wp <= p.Win) halo_pix = ((long long)n * p.Hin + (hp - 1)) * p.Win + (wp - 1);
                     }
                 }
-                for (int cbase = 0; cbase < p.BN; cbase += CW) {
-                    const int ncol = (p.BN - cbase < CW) ? p.BN - cbase : CW;  // multiple of 16
-                    // ---- TMEM -> registers -> staging (this thread's row)
-                    for (int c0 = 0; c0 < ncol; c0 += 32) {
-                        uint32_t r[32];
-                        const bool two = c0 + 16 < ncol;
-                        ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0), r);
-                        if (two) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cbase + c0 + 16), r + 16);
-                        ptx::tmem_ld_wait();
-                        const int sat_before = sat;
+                // The team's columns go through the staging buffer in passes of at most cw (<= 64) columns.
+                for (int cb = 0; cb < ncol; cb += cw) {
+                const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
+                // ---- TMEM -> registers -> staging (this thread's row); up to four 16-column loads are in flight before the
+                // one wait: a TMEM load has a long latency
+                {
+                    uint32_t r[64];
+                    const int nld = npass / 16;
+#ifdef NB_TC_DEBUG_TIMING
+                    dbg_ph__ = clock64();
+#endif
 #pragma unroll
-                        for (int hh = 0; hh < 2; ++hh) {
-                            if (hh == 1 && !two) break;
-                            uint4 v0, v1;
-                            const uint32_t* q = r + 16 * hh;
-                            v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat);
-                            v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat);
-                            v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat);
-                            v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat);
-                            v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat);
-                            v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat);
-                            v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat);
-                            v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat);
-                            if (HALO && halo_pix < 0) {  // discarded row: zeros keep the channel sums exact
-                                v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
-                                sat = sat_before;
-                            }
-                            *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2) = v0;
-                            *reinterpret_cast<uint4*>(my_row + (c0 + 16 * hh) * 2 + 16) = v1;
+                    for (int hh = 0; hh < 4; ++hh)
+                        if (hh < nld) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cb + 16 * hh), r + 16 * hh);
+                    ptx::tmem_ld_wait();
+                    NB_DBG_PHASE(dbg_ld);
+                    int sat_bits = 0;
+#pragma unroll
+                    for (int hh = 0; hh < 4; ++hh) {
+                        if (hh >= nld) break;
+                        uint4 v0, v1;
+                        const uint32_t* q = r + 16 * hh;
+                        v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat_bits);
+                        v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat_bits);
+                        v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat_bits);
+                        v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat_bits);
+                        v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat_bits);
+                        v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat_bits);
+                        v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat_bits);
+                        v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat_bits);
+                        if (HALO && halo_pix < 0) {  // discarded row: zeros keep the channel sums exact
+                            v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
+                            sat_bits = 0;
                         }
+                        *reinterpret_cast<uint4*>(my_row + (16 * hh) * 2) = v0;
+                        *reinterpret_cast<uint4*>(my_row + (16 * hh) * 2 + 16) = v1;
                     }
-                    if (h == mh - 1 && cbase + CW >= p.BN) {
-                        // last TMEM read of this tile: the accumulator set is free for the MMAs of a later tile
-                        ptx::tc_fence_before();
-                        if (CG2) {
-                            __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
-                        } else {
-                            ptx::mbar_arrive(tempty + acc);
-                        }
+                    if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
+                }
+                if (h == mh - 1 && cb + cw >= ncol) {
+                    // last TMEM read of this tile: the accumulator set is free for the MMAs of a later tile
+                    ptx::tc_fence_before();
+                    if (CG2) {
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
+                    } else {
+                        ptx::mbar_arrive(tempty + acc);
                     }
-                    __syncwarp();  // every warp only reads back the 32 rows it staged itself
-                    if (STATS && !(p.variant & 16)) {
-                        // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
-                        // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends.
-                        // A lane owns four adjacent channels (ncol <= 128, so one pass covers the chunk).
-                        if (lane < ncol / 4) {
-                            float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
-                            const uint8_t* col = my_rows + lane * 8;
+                }
+                __syncwarp();  // every warp only reads back the 32 rows it staged itself
+                NB_DBG_PHASE(dbg_pack);
+                if (STATS && !(p.variant & 16)) {
+                    // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
+                    // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends.
+                    // A lane owns two adjacent channels (a pass has at most 64), two rows per step for independent chains.
+                    if (lane < npass / 2) {
+                        float2 sa = make_float2(0.f, 0.f), sb = sa, qa = sa, qb = sa;
+                        const uint8_t* col = my_rows + lane * 4;
 #pragma unroll 8
-                            for (int rr = 0; rr < 32; ++rr) {
-                                const uint2 u = *reinterpret_cast<const uint2*>(col + (size_t)rr * pitch);
-                                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
-                                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
-                                s4[0] += f0.x; s4[1] += f0.y; s4[2] += f1.x; s4[3] += f1.y;
-                                q4[0] = fmaf(f0.x, f0.x, q4[0]); q4[1] = fmaf(f0.y, f0.y, q4[1]);
-                                q4[2] = fmaf(f1.x, f1.x, q4[2]); q4[3] = fmaf(f1.y, f1.y, q4[3]);
-                            }
-                            float4* ps = reinterpret_cast<float4*>(my_stat + n_tile * p.BN + cbase + 4 * lane);
-                            float4* pq = reinterpret_cast<float4*>(my_stat + p.ldo + n_tile * p.BN + cbase + 4 * lane);
-                            float4 a4 = *ps, b4 = *pq;
-                            a4.x += s4[0]; a4.y += s4[1]; a4.z += s4[2]; a4.w += s4[3];
-                            b4.x += q4[0]; b4.y += q4[1]; b4.z += q4[2]; b4.w += q4[3];
-                            *ps = a4;
-                            *pq = b4;
+                        for (int rr = 0; rr < 32; rr += 2) {
+                            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(col + (size_t)rr * pitch));
+                            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(col + (size_t)(rr + 1) * pitch));
+                            sa.x += f0.x; sa.y += f0.y;
+                            sb.x += f1.x; sb.y += f1.y;
+                            qa.x = fmaf(f0.x, f0.x, qa.x); qa.y = fmaf(f0.y, f0.y, qa.y);
+                            qb.x = fmaf(f1.x, f1.x, qb.x); qb.y = fmaf(f1.y, f1.y, qb.y);
                         }
+                        float2* ps = reinterpret_cast<float2*>(my_stat + n_tile * ncol + cb + 2 * lane);
+                        float2* pq = reinterpret_cast<float2*>(my_stat + st_ld + n_tile * ncol + cb + 2 * lane);
+                        float2 a2 = *ps, b2 = *pq;
+                        a2.x += sa.x + sb.x; a2.y += sa.y + sb.y;
+                        b2.x += qa.x + qb.x; b2.y += qa.y + qb.y;
+                        *ps = a2;
+                        *pq = b2;
                     }
-                    // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
-                    // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
-                    // output pixel of row r, the others fetch it by shuffle
-                    if (!(p.variant & 32)) {
-                        const int cpr = ncol / 8;  // 16-byte pieces per staged row (<= 16)
-                        long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
-                        if (HALO) {
-                            pixrow = halo_pix;
-                        } else if (pixrow >= p.M) {
-                            pixrow = -1;
-                        } else if (p.os != 1) {
-                            const int j = (int)(pixrow % p.Wq);
-                            const long long t1 = pixrow / p.Wq;
-                            const int i = (int)(t1 % p.Hq);
-                            const long long n = t1 / p.Hq;
-                            pixrow = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
-                        }
-                        const int col_off = (n_tile * p.BN + cbase) * 2;
-                        const int step_r = 32 / cpr, step_c = 32 - step_r * cpr;
-                        int rr = lane / cpr, cc = lane - rr * cpr;
-                        for (int it = 0; it < cpr; ++it) {
-                            const long long pix = __shfl_sync(0xffffffffu, pixrow, rr);
-                            if (pix >= 0) {
-                                const uint4 v = *reinterpret_cast<const uint4*>(my_rows + rr * pitch + cc * 16);
-                                *reinterpret_cast<uint4*>(outb + (size_t)pix * (size_t)(p.ldo * 2) + col_off + cc * 16) = v;
-                            }
-                            rr += step_r;
-                            cc += step_c;
-                            if (cc >= cpr) {
-                                cc -= cpr;
-                                ++rr;
-                            }
-                        }
+                }
+                NB_DBG_PHASE(dbg_stats);
+                // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
+                // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
+                // output offset of row r, the others fetch it by shuffle
+                if (!(p.variant & 32)) {
+                    const int cpr = npass / 8;  // 16-byte pieces per staged row (<= 8)
+                    long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
+                    if (HALO) {
+                        pixrow = halo_pix;
+                    } else if (pixrow >= p.M) {
+                        pixrow = -1;
+                    } else if (p.os != 1) {
+                        const int j = (int)(pixrow % p.Wq);
+                        const long long t1 = pixrow / p.Wq;
+                        const int i = (int)(t1 % p.Hq);
+                        const long long n = t1 / p.Hq;
+                        pixrow = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
                     }
-                    __syncwarp();  // staged rows consumed before the next pass overwrites them
+                    // byte offset of staged row `lane` in the output (-1: not stored); pieces are handled four (or two) at
+                    // a time so that their shuffle -> shared load -> global store chains overlap
+                    const long long rowbyte = pixrow < 0 ? -1 : pixrow * (long long)(p.ldo * 2) + (n_tile * p.BN + c_lo + cb) * 2;
+                    const int step_r = 32 / cpr, step_c = 32 - step_r * cpr;
+                    int rr = lane / cpr, cc = lane - rr * cpr;
+                    auto advance = [&](int& r_, int& c_) {
+                        r_ += step_r;
+                        c_ += step_c;
+                        if (c_ >= cpr) {
+                            c_ -= cpr;
+                            ++r_;
+                        }
+                    };
+                    int it = 0;
+                    for (; it + 4 <= cpr; it += 4) {
+                        int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
+                        advance(r1, c1);
+                        int r2 = r1, c2 = c1;
+                        advance(r2, c2);
+                        int r3 = r2, c3 = c2;
+                        advance(r3, c3);
+                        rr = r3; cc = c3;
+                        advance(rr, cc);
+                        const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
+                        const long long o2 = __shfl_sync(0xffffffffu, rowbyte, r2), o3 = __shfl_sync(0xffffffffu, rowbyte, r3);
+                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * pitch + c0 * 16);
+                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * pitch + c1 * 16);
+                        const uint4 v2 = *reinterpret_cast<const uint4*>(my_rows + r2 * pitch + c2 * 16);
+                        const uint4 v3 = *reinterpret_cast<const uint4*>(my_rows + r3 * pitch + c3 * 16);
+                        if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
+                        if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
+                        if (o2 >= 0) *reinterpret_cast<uint4*>(outb + o2 + c2 * 16) = v2;
+                        if (o3 >= 0) *reinterpret_cast<uint4*>(outb + o3 + c3 * 16) = v3;
+                    }
+                    for (; it < cpr; it += 2) {  // cpr is even
+                        int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
+                        advance(r1, c1);
+                        rr = r1; cc = c1;
+                        advance(rr, cc);
+                        const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
+                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * pitch + c0 * 16);
+                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * pitch + c1 * 16);
+                        if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
+                        if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
+                    }
+                }
+                __syncwarp();  // staged rows consumed before the next pass overwrites them
+                NB_DBG_PHASE(dbg_store);
                 }
             }
             if (++acc == nbuf) {
@@ -760,13 +828,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_igemm_kernel(const __grid_co
             }
         }
         if (STATS) {
-            epi_bar_sync();  // all four warps' running sums are final
+            epi2_bar_sync();  // all eight warps' running sums are final
+            // channel c of the layer sits in team (c % BN >= ncol_a) at index (c / BN) * (team's columns) + its column there
             float* dst = p.partials + (size_t)blockIdx.x * 2 * p.ldo;
-            for (int c = et; c < 2 * p.ldo; c += 128)
-                dst[c] = ((wstat[c] + wstat[2 * p.ldo + c]) + wstat[4 * p.ldo + c]) + wstat[6 * p.ldo + c];
+            const int et = (warp >= 7 ? warp - 3 : warp - 2) * 32 + lane;  // 0..255
+            const int ncb = p.BN - p.ncol_a;
+            for (int e = et; e < 2 * p.ldo; e += 256) {
+                const int which = e >= p.ldo ? 1 : 0, c = e - which * p.ldo;
+                const int nt = c / p.BN, cc = c - nt * p.BN;
+                const int tm = cc >= p.ncol_a ? 1 : 0;
+                const int ld = p.n_tiles * (tm ? ncb : p.ncol_a);
+                const float* base = wstat + (tm ? (size_t)8 * p.n_tiles * p.ncol_a : 0) + (size_t)which * ld + nt * (tm ? ncb : p.ncol_a) + (cc - (tm ? p.ncol_a : 0));
+                dst[e] = ((base[0] + base[2 * ld]) + base[4 * ld]) + base[6 * ld];
+            }
         }
 #ifdef NB_TC_DEBUG_TIMING
-        if (p.dbg && et == 0) { p.dbg[blockIdx.x * 8 + 5] = dbg_wait_tfull; p.dbg[blockIdx.x * 8 + 6] = clock64() - dbg_start; }
+        if (p.dbg && warp == 2 && lane == 0) {
+            p.dbg[blockIdx.x * 8 + 5] = dbg_wait_tfull; p.dbg[blockIdx.x * 8 + 6] = clock64() - dbg_start;
+            long long* ph = p.dbg + (size_t)gridDim.x * 8 + blockIdx.x * 4;
+            ph[0] = dbg_ld; ph[1] = dbg_pack; ph[2] = dbg_stats; ph[3] = dbg_store;
+        }
 #endif
         if (sat) atomicAdd(p.status + ST_SAT, sat);
     }
@@ -896,13 +977,15 @@ constexpr size_t kMaxSmem = 232448;  // 227 KB opt-in limit per CTA
 // TMA fills shared memory at roughly 100 cycles per box plus 1.4 (256-row boxes) to 2.3 (128-row boxes) cycles per
 // 128-byte row; one barrier round trip of the single-thread producer / MMA loops costs a few hundred cycles.
 // The tile is [128*mh x BN]: with mh = 2 two row blocks share every B stage (fewer rows fetched per flop).
-inline int igemm_stage_cols(int BN) {
-    if (BN <= 128) return BN;
-    if (BN % 32 == 0) return BN / 2;
-    return 128;
+// Columns of a [128 x BN] tile that the first epilogue team takes: half of them, rounded up to a multiple of 16.
+inline int igemm_team_cols(int BN) { return (BN / 16 + 1) / 2 * 16; }
+// Columns per staging pass: the team's columns in the fewest passes of at most 64, balanced.
+inline int igemm_stage_cw(int BN) {
+    const int nc = igemm_team_cols(BN), passes = (nc + 63) / 64;
+    return ((nc + passes - 1) / passes + 15) / 16 * 16;
 }
 inline size_t igemm_fixed_smem(int BN, int ldo) {
-    return 1024 /*alignment slack*/ + (size_t)TC_BM * (igemm_stage_cols(BN) * 2 + 16) + (size_t)8 * ldo * 4 + 512;
+    return 1024 /*alignment slack*/ + (size_t)2 * TC_BM * (igemm_stage_cw(BN) * 2 + 16) + (size_t)8 * ldo * 4 + 512;
 }
 inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses) {
     IgemmCfg c;
@@ -960,7 +1043,7 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     }
     if (!c.BN) return c;
     c.n_tiles = rowsB / c.BN;
-    c.stage_cols = igemm_stage_cols(c.BN);
+    c.stage_cols = igemm_team_cols(c.BN);
     c.tmem_cols = std::max(32, c.acc_bufs * c.mh * c.acc_stride);
     c.a_stage = c.a_sub * c.kpb;
     c.b_stage = c.b_sub * c.kpb;
@@ -1030,7 +1113,7 @@ inline IgemmCfg halo_configure(int N, int H, int W, int Ca, int rowsB, int ldo, 
     }
     if (!c.BN) return c;
     c.n_tiles = rowsB / c.BN;
-    c.stage_cols = igemm_stage_cols(c.BN);
+    c.stage_cols = igemm_team_cols(c.BN);
     c.tmem_cols = std::max(32, c.acc_bufs * c.mh * c.acc_stride);
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.a_slots * c.slab_bytes + (size_t)c.stages * c.b_stage, 120 * 1024);
     c.grid = 2 * (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count / 2);
@@ -1047,7 +1130,7 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.sbo = (uint32_t)(8 * c.KC * 2);
     P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
     P.kpb = c.kpb; P.a_sub_bytes = c.a_sub; P.b_sub_bytes = c.b_sub;
-    P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.stage_cols = c.stage_cols;
+    P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.ncol_a = c.stage_cols; P.stage_cw = igemm_stage_cw(c.BN);
     P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
     if (getenv("NB_TC_VERBOSE"))
         fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
@@ -1104,7 +1187,7 @@ template <typename OutT, bool STATS, bool CG2, bool HALO> inline nb_status launc
         }
         attr_set = true;
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO>, dim3((unsigned)s.cfg.grid), dim3(TC_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
