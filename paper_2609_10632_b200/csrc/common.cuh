@@ -95,4 +95,36 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
+// Rearranged filter for dgrad: for parity class `cls` (a list of taps), wt[c][ti][c'] = w[c'][r_ti][t_ti][c].
+struct WtClass {
+    int ntaps;
+    int r[9], t[9];
+    size_t offset;  // element offset of this class's matrix in the output buffer
+};
+struct WtParams {
+    int c_in, c_out, k, nclasses;
+    WtClass cls[4];
+};
+// One thread per output element, output-contiguous (c' fastest); `block` of `nblocks` blocks of blockDim.x threads.
+__device__ __forceinline__ void wt_transform_blocks(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, const WtParams& P, int block,
+                                                    int nblocks) {
+    const size_t total = (size_t)P.c_in * P.k * P.k * P.c_out;
+    for (size_t e = (size_t)block * blockDim.x + threadIdx.x; e < total; e += (size_t)nblocks * blockDim.x) {
+        int cls = 0;
+        while (cls + 1 < P.nclasses && e >= P.cls[cls + 1].offset) ++cls;
+        const WtClass& C = P.cls[cls];
+        size_t le = e - C.offset;
+        const int co = (int)(le % P.c_out);
+        le /= P.c_out;
+        const int ti = (int)(le % C.ntaps);
+        const int c = (int)(le / C.ntaps);
+        wt[e] = w[(((size_t)co * P.k + C.r[ti]) * P.k + C.t[ti]) * P.c_in + c];
+    }
+}
+__global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
+    pdl_launch_dependents();
+    pdl_wait();
+    wt_transform_blocks(w, wt, P, (int)blockIdx.x, (int)gridDim.x);
+}
+
 }  // namespace nbcbs

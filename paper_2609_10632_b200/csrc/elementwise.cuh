@@ -60,26 +60,34 @@ __global__ void __launch_bounds__(288, 3) bn_stats_partial_kernel(const YT* __re
     }
 }
 
-// Sum partials[b][which][c] over b in fp64: lane l takes b = l, l+32, ... (independent loads in flight), then a
-// butterfly over the 32 lanes.  The order is fixed, so the result is bitwise reproducible.
-__device__ __forceinline__ double warp_sum_partials(const float* __restrict__ partials, int nparts, int C, int c, int which, int lane) {
-    double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
-    const float* base = partials + (size_t)which * C + c;
+// Both sums of channel c at once: s0 = sum over b of partials[b][0][c], s1 = the same for [b][1][c].  Lane l takes
+// b = l, l+32, ... (all loads of a step are issued before any is used), then a butterfly over the 32 lanes, in fp64.
+// The order is fixed, so the result is bitwise reproducible.
+__device__ __forceinline__ void warp_sum_partials2(const float* __restrict__ partials, int nparts, int C, int c, int lane, double& s0, double& s1) {
+    double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
+    const float* base = partials + c;
     const size_t step = (size_t)2 * C;
     int b = lane;
-    for (; b + 96 < nparts; b += 128) {
-        const float v0 = base[(size_t)b * step], v1 = base[(size_t)(b + 32) * step], v2 = base[(size_t)(b + 64) * step],
-                    v3 = base[(size_t)(b + 96) * step];
-        acc0 += (double)v0;
-        acc1 += (double)v1;
-        acc2 += (double)v2;
-        acc3 += (double)v3;
+    for (; b + 32 < nparts; b += 64) {
+        const float u0 = base[(size_t)b * step], v0 = base[(size_t)b * step + C];
+        const float u1 = base[(size_t)(b + 32) * step], v1 = base[(size_t)(b + 32) * step + C];
+        a0 += (double)u0;
+        b0 += (double)v0;
+        a1 += (double)u1;
+        b1 += (double)v1;
     }
-    for (; b < nparts; b += 32) acc0 += (double)base[(size_t)b * step];
-    double s = (acc0 + acc1) + (acc2 + acc3);
+    if (b < nparts) {
+        a0 += (double)base[(size_t)b * step];
+        b0 += (double)base[(size_t)b * step + C];
+    }
+    double s = a0 + a1, q = b0 + b1;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return s;
+    for (int o = 16; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+    }
+    s0 = s;
+    s1 = q;
 }
 
 // Combine partials [nparts][2][C] and derive the per-channel quantities.  One warp per channel, 8 channels per block.
@@ -94,8 +102,11 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restric
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
-    const double s = warp_sum_partials(partials, nparts, C, c, 0, lane);
-    const double q = warp_sum_partials(partials, nparts, C, c, 1, lane);
+    // the per-channel inputs of the last step are requested first so that they arrive while the partials are summed
+    const float ga = scale ? gamma[c] : 0.f, be = scale ? beta[c] : 0.f;
+    const float rm = rmean ? rmean[c] : 0.f, rv = rmean ? rvar[c] : 0.f;
+    double s, q;
+    warp_sum_partials2(partials, nparts, C, c, lane, s, q);
     if (lane == 0) {
         const double mu = s / M;
         double var = q / M - mu * mu;
@@ -104,15 +115,15 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restric
         if (mean) mean[c] = (float)mu;
         if (invstd) invstd[c] = (float)is;
         if (scale) {
-            const double sc = (double)gamma[c] * is;
+            const double sc = (double)ga * is;
             scale[c] = (float)sc;
-            shift[c] = (float)((double)beta[c] - mu * sc);
+            shift[c] = (float)((double)be - mu * sc);
         }
         if (sum_out) sum_out[c] = (float)s;
         if (sumsq_out) sumsq_out[c] = (float)q;
         if (rmean) {
-            rmean[c] = (float)((1.0 - (double)momentum) * (double)rmean[c] + (double)momentum * mu);
-            rvar[c] = (float)((1.0 - (double)momentum) * (double)rvar[c] + (double)momentum * var * M / (M - 1.0));
+            rmean[c] = (float)((1.0 - (double)momentum) * (double)rm + (double)momentum * mu);
+            rvar[c] = (float)((1.0 - (double)momentum) * (double)rv + (double)momentum * var * M / (M - 1.0));
         }
     }
 }
@@ -223,23 +234,31 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
 __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M,
                                                               const float* __restrict__ mean, const float* __restrict__ invstd,
                                                               const float* __restrict__ gamma, const float* __restrict__ beta,
-                                                              float* dgamma, float* dbeta, float* coef /*[4][C]*/) {
+                                                              float* dgamma, float* dbeta, float* coef /*[4][C]*/, int fin_blocks,
+                                                              const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams wtp) {
     pdl_launch_dependents();
     pdl_wait();
+    // Blocks past the first `fin_blocks` rearrange the filter for the data-gradient GEMM that follows this call's dy pass
+    // (independent work that fills the otherwise idle GPU while the short finalize chain runs).
+    if ((int)blockIdx.x >= fin_blocks) {
+        wt_transform_blocks(w, wt, wtp, (int)blockIdx.x - fin_blocks, (int)gridDim.x - fin_blocks);
+        return;
+    }
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
-    const double s0 = warp_sum_partials(partials, nparts, C, c, 0, lane);
-    const double s1 = warp_sum_partials(partials, nparts, C, c, 1, lane);
+    const float mu_f = mean[c], is_f = invstd[c], ga = gamma[c], be = beta[c];  // requested before the partials are summed
+    double s0, s1;
+    warp_sum_partials2(partials, nparts, C, c, lane, s0, s1);
     if (lane == 0) {
-        const double mu = (double)mean[c], is = (double)invstd[c];
+        const double mu = (double)mu_f, is = (double)is_f;
         const double dg = is * (s1 - mu * s0);
-        const double a = (double)gamma[c] * is;
+        const double a = (double)ga * is;
         const double p1 = a * is * dg / M;
         dbeta[c] = (float)s0;
         dgamma[c] = (float)dg;
         coef[c] = (float)a;
-        coef[C + c] = (float)((double)beta[c] - mu * a);
+        coef[C + c] = (float)((double)be - mu * a);
         coef[2 * C + c] = (float)p1;
         coef[3 * C + c] = (float)(p1 * mu - a * s0 / M);
     }

@@ -171,7 +171,7 @@ nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale
 template <typename YT, typename AT, bool FAST>
 nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, const float* mean, const float* invstd,
                               const float* gamma, const float* beta, float* dgamma, float* dbeta, void* dy, float* partials,
-                              float* coef, cudaStream_t st) {
+                              float* coef, cudaStream_t st, const void* w = nullptr, void* wt = nullptr, const WtParams* wtp = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
     {
@@ -182,7 +182,17 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     }
     {
         SiteTimer tm(p, SITE_BWD_FINALIZE, st);
-        launch_k(bn_bwd_finalize_kernel, dim3((C + 7) / 8), dim3(256), 0, st, 1, partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta, coef);
+        const int fin_blocks = (C + 7) / 8;
+        int wt_blocks = 0;
+        WtParams none;
+        if (wtp) {
+            const size_t total = (size_t)wtp->c_in * wtp->k * wtp->k * wtp->c_out;
+            wt_blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)p->sm_count * 8);
+        } else {
+            memset(&none, 0, sizeof none);
+        }
+        launch_k(bn_bwd_finalize_kernel, dim3(fin_blocks + wt_blocks), dim3(256), 0, st, 1, partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta,
+                 dgamma, dbeta, coef, fin_blocks, static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), wtp ? *wtp : none);
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
@@ -535,7 +545,9 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
         if (dx) NB_TRY(run_simt_dgrad<float>(p, dy_out, w, dx, st));
         return NB_OK;
     }
-    NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st)));
+    const bool tc_dg = dx && !p->stem && p->tc.dgrad;  // the finalize kernel also rearranges the filter for the tensor-core dgrad
+    NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st,
+                                                             tc_dg ? w : nullptr, tc_dg ? ws + p->off_wt : nullptr, tc_dg ? &p->tc.wtp : nullptr)));
     if (!dx) return NB_OK;
     if (p->stem) {
         SiteTimer tm(p, SITE_DGRAD, st);
@@ -548,7 +560,7 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     if (p->tc.dgrad) {
         SiteTimer tm(p, SITE_DGRAD, st);
         const long long l0 = p->tc.launches;
-        const nb_status ts = tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st);
+        const nb_status ts = tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st, true);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         return NB_OK;

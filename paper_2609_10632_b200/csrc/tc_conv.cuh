@@ -860,34 +860,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
 }
 
 
-// Rearranged filter for dgrad: for parity class `cls` (a list of taps), wt[c][ti][c'] = w[c'][r_ti][t_ti][c].
-struct WtClass {
-    int ntaps;
-    int r[9], t[9];
-    size_t offset;  // element offset of this class's matrix in the output buffer
-};
-struct WtParams {
-    int c_in, c_out, k, nclasses;
-    WtClass cls[4];
-};
-__global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
-    pdl_launch_dependents();
-    pdl_wait();
-    // one thread per output element, output-contiguous (c' fastest)
-    size_t total = (size_t)P.c_in * P.k * P.k * P.c_out;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-        int cls = 0;
-        while (cls + 1 < P.nclasses && e >= P.cls[cls + 1].offset) ++cls;
-        const WtClass& C = P.cls[cls];
-        size_t le = e - C.offset;
-        const int co = (int)(le % P.c_out);
-        le /= P.c_out;
-        const int ti = (int)(le % C.ntaps);
-        const int c = (int)(le / C.ntaps);
-        wt[e] = w[(((size_t)co * P.k + C.r[ti]) * P.k + C.t[ti]) * P.c_in + c];
-    }
-}
-
 }  // namespace nbcbs
 #include "tc_wgrad.cuh"
 namespace nbcbs {
@@ -1398,9 +1370,11 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     return launch_igemm<__half, true>(S, st);
 }
 
-inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void* w, void* dx, void* wt, int* status, cudaStream_t st) {
+// `wt_ready`: the rearranged filter was already written by an earlier kernel of this call (the BN backward finalize kernel
+// carries that work in extra blocks, where it costs nothing: the GPU is almost empty while the finalize chain runs).
+inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void* w, void* dx, void* wt, int* status, cudaStream_t st, bool wt_ready) {
     using namespace tcdetail;
-    {
+    if (!wt_ready) {
         const size_t total = tc->wt_bytes / 2;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)tc->sm_count * 8);
         launch_k(dgrad_weight_transform_kernel, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), tc->wtp);
