@@ -41,6 +41,11 @@ struct IgemmParams {
     int acc_bufs;                // accumulator sets in TMEM (2 when 2*mh*acc_stride <= 512)
     int ncol_a;                  // columns of a tile that epilogue team 0 handles (team 1: the other BN - ncol_a)
     int stage_cw;                // columns per staging pass of a team (<= 64)
+    // When GEMM row == output row (not a stride-2 dgrad, not the halo variant) a warp hands each staged [32 x width] piece
+    // to TMA: tmOut[i] is a tiled map over the output [M][ldo] with box {out_w[i], 32}; clipping at M is the map's.
+    int tma_store;
+    int out_w[3];
+    CUtensorMap tmOut[3];
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
     int variant;                 // experiment switches
@@ -630,9 +635,11 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         uint32_t acc_ph = 0;
         float* team_stat = wstat + (team ? (size_t)8 * p.n_tiles * p.ncol_a : 0);  // [4 warps][2][st_ld]
         float* my_stat = team_stat + (size_t)lane_group * 2 * st_ld;
+        const bool tma_out = !HALO && p.tma_store != 0;
+        // staging of this warp's 32 rows: padded rows for the store loop, dense rows (the TMA box) for TMA stores
         uint8_t* stg_t = stg + (size_t)team * TC_BM * pitch;
-        uint8_t* my_row = stg_t + (size_t)row * pitch;
-        const uint8_t* my_rows = stg_t + (size_t)(lane_group * 32) * pitch;
+        uint8_t* const wrows = tma_out ? stg + (size_t)((team * 4 + lane_group) * 32) * (cw * 2) : stg_t + (size_t)(lane_group * 32) * pitch;
+        bool store_pending = false;
         uint8_t* outb = static_cast<uint8_t*>(p.out);
 #ifdef NB_TC_DEBUG_TIMING
         long long dbg_wait_tfull = 0, dbg_ld = 0, dbg_pack = 0, dbg_stats = 0, dbg_store = 0, dbg_ph__ = 0;
@@ -681,6 +688,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // The team's columns go through the staging buffer in passes of at most cw (<= 64) columns.
                 for (int cb = 0; cb < ncol; cb += cw) {
                 const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
+                const int rpitch = tma_out ? npass * 2 : pitch;       // bytes between staged rows of this pass
+                const bool swz = tma_out && npass == 64;              // 128-byte rows: 16-byte chunk j of row r sits at j ^ (r & 7)
+                uint8_t* const my_row = wrows + (size_t)lane * rpitch;
+                const uint8_t* const my_rows = wrows;
                 // ---- TMEM -> registers -> staging (this thread's row); up to four 16-column loads are in flight before the
                 // one wait: a TMEM load has a long latency
                 {
@@ -694,6 +705,11 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                         if (hh < nld) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cb + 16 * hh), r + 16 * hh);
                     ptx::tmem_ld_wait();
                     NB_DBG_PHASE(dbg_ld);
+                    if (store_pending) {  // the previous TMA store must have read the staging rows before they are overwritten
+                        if (lane == 0) ptx::tma_store_wait_read<0>();
+                        __syncwarp();
+                        store_pending = false;
+                    }
                     int sat_bits = 0;
 #pragma unroll
                     for (int hh = 0; hh < 4; ++hh) {
@@ -712,8 +728,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                             v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
                             sat_bits = 0;
                         }
-                        *reinterpret_cast<uint4*>(my_row + (16 * hh) * 2) = v0;
-                        *reinterpret_cast<uint4*>(my_row + (16 * hh) * 2 + 16) = v1;
+                        const int j0 = swz ? ((2 * hh) ^ (lane & 7)) : 2 * hh, j1 = swz ? ((2 * hh + 1) ^ (lane & 7)) : 2 * hh + 1;
+                        *reinterpret_cast<uint4*>(my_row + j0 * 16) = v0;
+                        *reinterpret_cast<uint4*>(my_row + j1 * 16) = v1;
                     }
                     if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
                 }
@@ -727,7 +744,19 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                         ptx::mbar_arrive(tempty + acc);
                     }
                 }
-                __syncwarp();  // every warp only reads back the 32 rows it staged itself
+                if (tma_out) {
+                    // hand the staged rows to TMA: writes made visible to the async proxy, then one lane issues the store
+                    ptx::fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut[0] : npass == p.out_w[1] ? &p.tmOut[1] : &p.tmOut[2];
+                        ptx::tma_store_2d(tm, wrows, n_tile * p.BN + c_lo + cb, (int)(m0 + lane_group * 32));
+                        ptx::tma_store_commit();
+                    }
+                    store_pending = true;
+                } else {
+                    __syncwarp();  // every warp only reads back the 32 rows it staged itself
+                }
                 NB_DBG_PHASE(dbg_pack);
                 if (STATS && !(p.variant & 16)) {
                     // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
@@ -735,11 +764,12 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     // A lane owns two adjacent channels (a pass has at most 64), two rows per step for independent chains.
                     if (lane < npass / 2) {
                         float2 sa = make_float2(0.f, 0.f), sb = sa, qa = sa, qb = sa;
-                        const uint8_t* col = my_rows + lane * 4;
+                        const int cj = lane >> 2, cw4 = (lane & 3) * 4;  // 16-byte chunk and offset inside it of this lane's channels
 #pragma unroll 8
                         for (int rr = 0; rr < 32; rr += 2) {
-                            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(col + (size_t)rr * pitch));
-                            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(col + (size_t)(rr + 1) * pitch));
+                            const int ja = swz ? (cj ^ (rr & 7)) : cj, jb = swz ? (cj ^ ((rr + 1) & 7)) : cj;
+                            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(my_rows + (size_t)rr * rpitch + ja * 16 + cw4));
+                            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(my_rows + (size_t)(rr + 1) * rpitch + jb * 16 + cw4));
                             sa.x += f0.x; sa.y += f0.y;
                             sb.x += f1.x; sb.y += f1.y;
                             qa.x = fmaf(f0.x, f0.x, qa.x); qa.y = fmaf(f0.y, f0.y, qa.y);
@@ -758,7 +788,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
                 // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
                 // output offset of row r, the others fetch it by shuffle
-                if (!(p.variant & 32)) {
+                if (!tma_out && !(p.variant & 32)) {
                     const int cpr = npass / 8;  // 16-byte pieces per staged row (<= 8)
                     long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
                     if (HALO) {
@@ -797,10 +827,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                         advance(rr, cc);
                         const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
                         const long long o2 = __shfl_sync(0xffffffffu, rowbyte, r2), o3 = __shfl_sync(0xffffffffu, rowbyte, r3);
-                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * pitch + c0 * 16);
-                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * pitch + c1 * 16);
-                        const uint4 v2 = *reinterpret_cast<const uint4*>(my_rows + r2 * pitch + c2 * 16);
-                        const uint4 v3 = *reinterpret_cast<const uint4*>(my_rows + r3 * pitch + c3 * 16);
+                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * rpitch + c0 * 16);
+                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * rpitch + c1 * 16);
+                        const uint4 v2 = *reinterpret_cast<const uint4*>(my_rows + r2 * rpitch + c2 * 16);
+                        const uint4 v3 = *reinterpret_cast<const uint4*>(my_rows + r3 * rpitch + c3 * 16);
                         if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
                         if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
                         if (o2 >= 0) *reinterpret_cast<uint4*>(outb + o2 + c2 * 16) = v2;
@@ -812,8 +842,8 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                         rr = r1; cc = c1;
                         advance(rr, cc);
                         const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
-                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * pitch + c0 * 16);
-                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * pitch + c1 * 16);
+                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * rpitch + c0 * 16);
+                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * rpitch + c1 * 16);
                         if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
                         if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
                     }
@@ -827,6 +857,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 acc_ph ^= 1u;
             }
         }
+        if (store_pending && lane == 0) ptx::tma_store_wait_all<0>();  // the stores are complete before the kernel ends
         if (STATS) {
             epi2_bar_sync();  // all eight warps' running sums are final
             // channel c of the layer sits in team (c % BN >= ncol_a) at index (c / BN) * (team's columns) + its column there
@@ -884,6 +915,7 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
     IgemmParams prm;
     const void* a_ptr = nullptr;
     const void* b_ptr = nullptr;
+    const void* out_ptr = nullptr;
 };
 
 struct TcPlan {
@@ -1150,6 +1182,29 @@ inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, lo
     return true;
 }
 
+// Tiled maps over the output matrix [rows][ldo] (16-bit elements) for the epilogue's TMA stores: one per distinct pass width.
+inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long long rows) {
+    DriverFns& d = driver();
+    const int na = c.stage_cols, nb = c.BN - c.stage_cols, cw = P.stage_cw;
+    const int cand[3] = {cw, na % cw, nb % cw};  // full passes, team 0's last pass, team 1's last pass
+    int n = 0;
+    P.out_w[0] = P.out_w[1] = P.out_w[2] = 0;
+    for (int i = 0; i < 3; ++i) {
+        const int wv = cand[i];
+        if (wv == 0 || (n > 0 && P.out_w[0] == wv) || (n > 1 && P.out_w[1] == wv)) continue;
+        cuuint64_t dims[2] = {(cuuint64_t)P.ldo, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)P.ldo * 2};
+        cuuint32_t box[2] = {(cuuint32_t)wv, 32};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = d.tiled(&P.tmOut[n], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             wv == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeTiled (output) failed with code " + std::to_string((int)r); return false; }
+        P.out_w[n++] = wv;
+    }
+    return true;
+}
+
 template <typename OutT, bool STATS, bool CG2, bool HALO> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
@@ -1362,6 +1417,11 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
+    S.prm.tma_store = (!S.cfg.halo && !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0)) ? 1 : 0;
+    if (S.prm.tma_store && S.out_ptr != y) {
+        if (!encode_out_maps(S.prm, S.cfg, y, g.m)) return NB_ERR_CUDA;
+        S.out_ptr = y;
+    }
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
 #ifdef NB_TC_DEBUG_TIMING
     if (const char* e = getenv("NB_TC_DBG_PTR")) S.prm.dbg = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
@@ -1395,6 +1455,11 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
             if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         }
         S.a_ptr = dy; S.b_ptr = wt;
+    }
+    S.prm.tma_store = (g.stride == 1 && !S.cfg.halo && !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0)) ? 1 : 0;
+    if (S.prm.tma_store && S.out_ptr != dx) {
+        if (!encode_out_maps(S.prm, S.cfg, dx, (long long)g.n * g.h * g.w)) return NB_ERR_CUDA;
+        S.out_ptr = dx;
     }
     S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
     nb_status r = launch_igemm<__nv_bfloat16, false>(S, st);
