@@ -17,7 +17,9 @@ struct Geom {
 };
 
 // Device status block owned by a plan (ints): [0] error code, [1] where, [2] detail, [3] fp16 saturation count.
-enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_WORDS = 16 };
+// Words 8-13 are three arrive/depart counter pairs of the in-kernel grid barriers (forward finalize, backward finalize,
+// split-K reduce); each pair is zero whenever no kernel of the plan is running.
+enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_BAR_FWD = 8, ST_BAR_BWD = 10, ST_BAR_WG = 12, ST_WORDS = 16 };
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
@@ -53,6 +55,40 @@ template <typename T> __device__ __forceinline__ Vec16<T> ld16_stream(const T* p
 }
 template <typename T> __device__ __forceinline__ void st16_stream(T* p, const Vec16<T>& r) {
     __stcs(reinterpret_cast<uint4*>(p), *reinterpret_cast<const uint4*>(&r));
+}
+
+// Grid-wide barrier for kernels whose CTAs are all resident at once (grids of at most one wave, nothing the CTAs wait for
+// runs behind them).  ctr[0] counts arrivals, ctr[1] departures; the last CTA to leave zeroes both, so the pair is ready
+// for the next launch.  All calls are made by ONE thread of the CTA, bracketed by CTA-level barriers; data written before
+// grid_arrive_wait by any CTA may be read (from L2: __ldcg) after it.  The wait is bounded (about 2 s): false = gave up.
+__device__ __forceinline__ void grid_arrive(int* ctr) {
+    __threadfence();
+    atomicAdd(ctr, 1);
+}
+__device__ __forceinline__ bool grid_wait(int* ctr, int nblocks) {
+    unsigned long long t0 = 0;
+    for (unsigned i = 0;; ++i) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= nblocks) return true;
+        if ((i & 255u) == 255u) {
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ull) return false;
+        }
+    }
+}
+__device__ __forceinline__ bool grid_arrive_wait(int* ctr, int nblocks) {
+    grid_arrive(ctr);
+    return grid_wait(ctr, nblocks);
+}
+__device__ __forceinline__ void grid_depart(int* ctr, int nblocks) {
+    if (atomicAdd(ctr + 1, 1) == nblocks - 1) {
+        ctr[1] = 0;
+        ctr[0] = 0;
+        __threadfence();
+    }
 }
 
 // Programmatic dependent launch.  Every kernel of the library starts with pdl_launch_dependents() and executes pdl_wait()
@@ -105,20 +141,70 @@ struct WtParams {
     int c_in, c_out, k, nclasses;
     WtClass cls[4];
 };
-// One thread per output element, output-contiguous (c' fastest); `block` of `nblocks` blocks of blockDim.x threads.
+// Tiled transpose through shared memory: per (class, tap) the [c_out][c_in] slice of the filter (c_in contiguous) becomes
+// [c_in][c_out] (c_out contiguous).  A tile is 32 c_out rows x 64 c_in columns; it is fetched with 16-byte cp.async copies
+// (no registers held, so a kernel can start the fetch, do its own work and finish the tile later) and written back as
+// 16-byte vectors of eight c_out values.  Channel counts are multiples of 8 on this path.
+constexpr int WT_PITCH = 72;  // elements per shared-memory row of a tile (64 + padding, rows stay 16-byte aligned)
+typedef __nv_bfloat16 WtTileBuf[32][WT_PITCH];
+struct WtTile {
+    int cls, tap, r0, c0;
+};
+__device__ __forceinline__ int wt_num_tiles(const WtParams& P) {
+    int taps = 0;
+    for (int cls = 0; cls < P.nclasses; ++cls) taps += P.cls[cls].ntaps;
+    return taps * ((P.c_out + 31) / 32) * ((P.c_in + 63) / 64);
+}
+__device__ __forceinline__ WtTile wt_tile_decode(const WtParams& P, int t) {
+    const int tc = (P.c_in + 63) / 64, per_tap = ((P.c_out + 31) / 32) * tc;
+    WtTile T;
+    T.tap = t / per_tap;
+    const int rem = t - T.tap * per_tap;
+    T.r0 = (rem / tc) * 32;
+    T.c0 = (rem - (rem / tc) * tc) * 64;
+    T.cls = 0;
+    while (T.tap >= P.cls[T.cls].ntaps) T.tap -= P.cls[T.cls++].ntaps;
+    return T;
+}
+// Starts the copies of one tile (all threads of the block take part); complete them with wt_async_wait() + __syncthreads().
+__device__ __forceinline__ void wt_tile_load_async(const __nv_bfloat16* __restrict__ w, const WtParams& P, const WtTile& T, WtTileBuf& tile) {
+    const WtClass& C = P.cls[T.cls];
+    const int src_tap = C.r[T.tap] * P.k + C.t[T.tap], kk = P.k * P.k;
+    for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+        const int i = e >> 3, v = e & 7;  // row (c_out) and 16-byte vector (eight c_in) within the tile
+        const bool ok = T.r0 + i < P.c_out && T.c0 + v * 8 < P.c_in;
+        const __nv_bfloat16* src = ok ? w + ((size_t)(T.r0 + i) * kk + src_tap) * P.c_in + T.c0 + v * 8 : w;
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(&tile[i][v * 8]);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(ok ? 16 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void wt_async_wait() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// Writes one fetched tile transposed (call after the copies have landed and the block has synchronised).
+__device__ __forceinline__ void wt_tile_store(__nv_bfloat16* __restrict__ wt, const WtParams& P, const WtTile& T, const WtTileBuf& tile) {
+    const WtClass& C = P.cls[T.cls];
+    for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+        const int j = e >> 2, v = e & 3;  // column (c_in) within the tile and vector of eight c_out rows
+        if (T.c0 + j < P.c_in && T.r0 + v * 8 < P.c_out) {
+            Vec16<__nv_bfloat16> o;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o.v[i] = tile[v * 8 + i][j];
+            st16(wt + C.offset + ((size_t)(T.c0 + j) * C.ntaps + T.tap) * P.c_out + T.r0 + v * 8, o);
+        }
+    }
+}
+// The whole rearrangement by `nblocks` blocks, tiles dealt round-robin (all threads of a block take part).
 __device__ __forceinline__ void wt_transform_blocks(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, const WtParams& P, int block,
-                                                    int nblocks) {
-    const size_t total = (size_t)P.c_in * P.k * P.k * P.c_out;
-    for (size_t e = (size_t)block * blockDim.x + threadIdx.x; e < total; e += (size_t)nblocks * blockDim.x) {
-        int cls = 0;
-        while (cls + 1 < P.nclasses && e >= P.cls[cls + 1].offset) ++cls;
-        const WtClass& C = P.cls[cls];
-        size_t le = e - C.offset;
-        const int co = (int)(le % P.c_out);
-        le /= P.c_out;
-        const int ti = (int)(le % C.ntaps);
-        const int c = (int)(le / C.ntaps);
-        wt[e] = w[(((size_t)co * P.k + C.r[ti]) * P.k + C.t[ti]) * P.c_in + c];
+                                                    int nblocks, int first_round = 0) {
+    __shared__ __align__(16) WtTileBuf tile;
+    const int ntiles = wt_num_tiles(P);
+    for (int t = block + first_round * nblocks; t < ntiles; t += nblocks) {
+        const WtTile T = wt_tile_decode(P, t);
+        wt_tile_load_async(w, P, T, tile);
+        wt_async_wait();
+        __syncthreads();
+        wt_tile_store(wt, P, T, tile);
+        __syncthreads();
     }
 }
 __global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {

@@ -63,22 +63,30 @@ __global__ void __launch_bounds__(288, 3) bn_stats_partial_kernel(const YT* __re
 // Both sums of channel c at once: s0 = sum over b of partials[b][0][c], s1 = the same for [b][1][c].  Lane l takes
 // b = l, l+32, ... (all loads of a step are issued before any is used), then a butterfly over the 32 lanes, in fp64.
 // The order is fixed, so the result is bitwise reproducible.
+// L2 = read around L1 (the partials were written by other CTAs of the same launch).
+// Sixteen loads (eight slices x two quantities) are issued before the first is used, so up to 256 slices cost one
+// memory round trip; the fused finalize steps at the tail of other kernels sit on the critical path.
+template <bool L2 = false>
 __device__ __forceinline__ void warp_sum_partials2(const float* __restrict__ partials, int nparts, int C, int c, int lane, double& s0, double& s1) {
     double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
     const float* base = partials + c;
     const size_t step = (size_t)2 * C;
-    int b = lane;
-    for (; b + 32 < nparts; b += 64) {
-        const float u0 = base[(size_t)b * step], v0 = base[(size_t)b * step + C];
-        const float u1 = base[(size_t)(b + 32) * step], v1 = base[(size_t)(b + 32) * step + C];
-        a0 += (double)u0;
-        b0 += (double)v0;
-        a1 += (double)u1;
-        b1 += (double)v1;
-    }
-    if (b < nparts) {
-        a0 += (double)base[(size_t)b * step];
-        b0 += (double)base[(size_t)b * step + C];
+    for (int b = lane; b < nparts; b += 256) {
+        float u[8], v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int bk = b + 32 * k;
+            const float* q = base + (size_t)bk * step;
+            u[k] = bk < nparts ? (L2 ? __ldcg(q) : *q) : 0.f;
+            v[k] = bk < nparts ? (L2 ? __ldcg(q + C) : q[C]) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; k += 2) {
+            a0 += (double)u[k];
+            b0 += (double)v[k];
+            a1 += (double)u[k + 1];
+            b1 += (double)v[k + 1];
+        }
     }
     double s = a0 + a1, q = b0 + b1;
 #pragma unroll
@@ -90,23 +98,17 @@ __device__ __forceinline__ void warp_sum_partials2(const float* __restrict__ par
     s1 = q;
 }
 
-// Combine partials [nparts][2][C] and derive the per-channel quantities.  One warp per channel, 8 channels per block.
-// Outputs (any may be NULL): mean, invstd, scale = gamma*invstd, shift = beta - mean*scale, raw sums,
-// running statistics (in place; unbiased variance, momentum).
-__global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float eps,
-                                                          float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
-                                                          float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
-                                                          float* sum_out, float* sumsq_out) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (c >= C) return;
+// The finalize of one channel by one warp (also called from the tail of the tensor-core forward kernel).
+template <bool L2>
+__device__ __forceinline__ void bn_finalize_channel(const float* __restrict__ partials, int nparts, int C, int c, int lane, double M, float eps,
+                                                    float momentum, const float* __restrict__ gamma, const float* __restrict__ beta, float* mean,
+                                                    float* invstd, float* scale, float* shift, float* rmean, float* rvar, float* sum_out,
+                                                    float* sumsq_out) {
     // the per-channel inputs of the last step are requested first so that they arrive while the partials are summed
     const float ga = scale ? gamma[c] : 0.f, be = scale ? beta[c] : 0.f;
     const float rm = rmean ? rmean[c] : 0.f, rv = rmean ? rvar[c] : 0.f;
     double s, q;
-    warp_sum_partials2(partials, nparts, C, c, lane, s, q);
+    warp_sum_partials2<L2>(partials, nparts, C, c, lane, s, q);
     if (lane == 0) {
         const double mu = s / M;
         double var = q / M - mu * mu;
@@ -126,6 +128,21 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restric
             rvar[c] = (float)((1.0 - (double)momentum) * (double)rv + (double)momentum * var * M / (M - 1.0));
         }
     }
+}
+
+// Combine partials [nparts][2][C] and derive the per-channel quantities.  One warp per channel, 8 channels per block.
+// Outputs (any may be NULL): mean, invstd, scale = gamma*invstd, shift = beta - mean*scale, raw sums,
+// running statistics (in place; unbiased variance, momentum).
+__global__ void __launch_bounds__(256) bn_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M, float eps,
+                                                          float momentum, const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                          float* mean, float* invstd, float* scale, float* shift, float* rmean, float* rvar,
+                                                          float* sum_out, float* sumsq_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= C) return;
+    bn_finalize_channel<false>(partials, nparts, C, c, lane, M, eps, momentum, gamma, beta, mean, invstd, scale, shift, rmean, rvar, sum_out, sumsq_out);
 }
 
 // V consecutive per-channel floats (V = 4 or 8) with 16-byte loads.
@@ -167,15 +184,52 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
     }
 }
 
+// partials [nparts][2][C] (sum dz, sum dz*y) -> dbeta, dgamma (fp32) and four per-channel coefficients for the dy pass:
+//   coef[0] = a = gamma*invstd, coef[1] = b = beta - mean*a                      (z = y*a + b)
+//   coef[2] = p1 = a*invstd*dgamma/M, coef[3] = p0 = p1*mean - a*dbeta/M        (dy = a*dz - p1*y + p0)
+// which is dy = a*(dz - dbeta/M - xhat*dgamma/M) with xhat = (y - mean)*invstd written out in terms of y.
+template <bool L2>
+__device__ __forceinline__ void bn_bwd_finalize_channel(const float* __restrict__ partials, int nparts, int C, int c, int lane, double M,
+                                                        const float* __restrict__ mean, const float* __restrict__ invstd,
+                                                        const float* __restrict__ gamma, const float* __restrict__ beta, float* dgamma, float* dbeta,
+                                                        float* coef /*[4][C]*/) {
+    const float mu_f = mean[c], is_f = invstd[c], ga = gamma[c], be = beta[c];  // requested before the partials are summed
+    double s0, s1;
+    warp_sum_partials2<L2>(partials, nparts, C, c, lane, s0, s1);
+    if (lane == 0) {
+        const double mu = (double)mu_f, is = (double)is_f;
+        const double dg = is * (s1 - mu * s0);
+        const double a = (double)ga * is;
+        const double p1 = a * is * dg / M;
+        dbeta[c] = (float)s0;
+        dgamma[c] = (float)dg;
+        coef[c] = (float)a;
+        coef[C + c] = (float)((double)be - mu * a);
+        coef[2 * C + c] = (float)p1;
+        coef[3 * C + c] = (float)(p1 * mu - a * s0 / M);
+    }
+}
+
 // ------------------------------------------------------------------ backward reductions: sum dz, sum dz*y
 // z = y*a + b with a = gamma*invstd, b = beta - mean*a (recomputed here from the saved statistics).  The second
 // sum is taken against y itself; sum dz*xhat = invstd*(sum dz*y - mean*sum dz) is formed in fp64 by the finalize
 // kernel, so this pass needs only two per-channel values per element.
+// What the reduce kernel needs to finalize by itself (on = 0: it only writes the partial sums).
+struct BwdFused {
+    int on;
+    int* ctr;     // arrive/depart counters of the grid barrier
+    int* status;  // the plan's status block
+    double M;
+    float *dgamma, *dbeta, *coef;
+    const __nv_bfloat16* w;  // filter and its rearranged copy for the data-gradient GEMM (wt = NULL: nothing to rearrange)
+    __nv_bfloat16* wt;
+};
 template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                                   long long total_vecs, int C, const float* __restrict__ mean,
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
-                                                                  const float* __restrict__ beta, float* __restrict__ partials) {
+                                                                  const float* __restrict__ beta, float* __restrict__ partials, BwdFused fb,
+                                                                  WtParams wtp) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -184,6 +238,17 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
     const int tid = threadIdx.x;
     const int cgs = C / V;
     const int cg = tid % cgs;
+    // Fused mode: the first two filter tiles of this block (for the data-gradient GEMM's rearranged filter) are requested
+    // now with cp.async and written back after the streaming loop, so their memory latency costs nothing.
+    __shared__ __align__(16) WtTileBuf wtile[2];
+    const int wt_tiles = (fb.on && fb.wt) ? wt_num_tiles(wtp) : 0;
+    if (wt_tiles > 0) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int t = (int)blockIdx.x + k * (int)gridDim.x;
+            if (t < wt_tiles) wt_tile_load_async(fb.w, wtp, wt_tile_decode(wtp, t), wtile[k]);
+        }
+    }
     float a[V], b[V], sb[V], sy[V];
     {
         float mu[V], is[V], ga[V], be[V];
@@ -225,12 +290,37 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
         }
         __syncthreads();
     }
+    if (fb.on) {
+        // Fused finalize: the grid is one wave of resident blocks, so a grid-wide barrier is safe.  Between arriving and
+        // waiting the block writes back its filter tiles; afterwards block b finalizes channels b, b + gridDim.x, ...
+        // with one warp per channel.
+        __shared__ int ok;
+        if (tid == 0) grid_arrive(fb.ctr);
+        if (wt_tiles > 0) {
+            wt_async_wait();
+            __syncthreads();
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int t = (int)blockIdx.x + k * (int)gridDim.x;
+                if (t < wt_tiles) wt_tile_store(fb.wt, wtp, wt_tile_decode(wtp, t), wtile[k]);
+            }
+            if (wt_tiles > 2 * (int)gridDim.x) wt_transform_blocks(fb.w, fb.wt, wtp, (int)blockIdx.x, (int)gridDim.x, 2);  // rare: very large filters
+        }
+        if (tid == 0) ok = grid_wait(fb.ctr, (int)gridDim.x) ? 1 : 0;
+        __syncthreads();
+        if (ok) {
+            const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+            for (int c = (int)blockIdx.x + (int)gridDim.x * warp; c < C; c += (int)gridDim.x * nwarps)
+                bn_bwd_finalize_channel<true>(partials, (int)gridDim.x, C, c, lane, fb.M, mean, invstd, gamma, beta, fb.dgamma, fb.dbeta, fb.coef);
+        } else if (tid == 0 && atomicCAS(fb.status + ST_ERR, 0, 2 /* NB_ERR_TIMEOUT */) == 0) {
+            fb.status[ST_WHERE] = 21;
+            fb.status[ST_DETAIL] = (int)blockIdx.x;
+        }
+        __syncthreads();
+        if (tid == 0) grid_depart(fb.ctr, (int)gridDim.x);
+    }
 }
 
-// partials [nparts][2][C] (sum dz, sum dz*y) -> dbeta, dgamma (fp32) and four per-channel coefficients for the dy pass:
-//   coef[0] = a = gamma*invstd, coef[1] = b = beta - mean*a                      (z = y*a + b)
-//   coef[2] = p1 = a*invstd*dgamma/M, coef[3] = p0 = p1*mean - a*dbeta/M        (dy = a*dz - p1*y + p0)
-// which is dy = a*(dz - dbeta/M - xhat*dgamma/M) with xhat = (y - mean)*invstd written out in terms of y.
 __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __restrict__ partials, int nparts, int C, double M,
                                                               const float* __restrict__ mean, const float* __restrict__ invstd,
                                                               const float* __restrict__ gamma, const float* __restrict__ beta,
@@ -247,21 +337,7 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __res
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c >= C) return;
-    const float mu_f = mean[c], is_f = invstd[c], ga = gamma[c], be = beta[c];  // requested before the partials are summed
-    double s0, s1;
-    warp_sum_partials2(partials, nparts, C, c, lane, s0, s1);
-    if (lane == 0) {
-        const double mu = (double)mu_f, is = (double)is_f;
-        const double dg = is * (s1 - mu * s0);
-        const double a = (double)ga * is;
-        const double p1 = a * is * dg / M;
-        dbeta[c] = (float)s0;
-        dgamma[c] = (float)dg;
-        coef[c] = (float)a;
-        coef[C + c] = (float)((double)be - mu * a);
-        coef[2 * C + c] = (float)p1;
-        coef[3 * C + c] = (float)(p1 * mu - a * s0 / M);
-    }
+    bn_bwd_finalize_channel<false>(partials, nparts, C, c, lane, M, mean, invstd, gamma, beta, dgamma, dbeta, coef);
 }
 
 // ------------------------------------------------------------------ dy = a*dz - p1*y + p0

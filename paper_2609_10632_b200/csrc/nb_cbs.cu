@@ -174,22 +174,30 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
                               float* coef, cudaStream_t st, const void* w = nullptr, void* wt = nullptr, const WtParams* wtp = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
+    const bool fuse = !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+    WtParams none;
+    if (!wtp) memset(&none, 0, sizeof none);
     {
+        // one wave of resident blocks: the kernel finalizes behind a grid-wide barrier and rearranges the dgrad filter meanwhile
         SiteTimer tm(p, SITE_BWD_REDUCE, st);
+        BwdFused fb;
+        memset(&fb, 0, sizeof fb);
+        if (fuse) {
+            fb.on = 1; fb.ctr = p->status + ST_BAR_BWD; fb.status = p->status; fb.M = (double)p->g.m;
+            fb.dgamma = dgamma; fb.dbeta = dbeta; fb.coef = coef;
+            fb.w = static_cast<const __nv_bfloat16*>(w); fb.wt = wtp ? static_cast<__nv_bfloat16*>(wt) : nullptr;
+        }
         launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
-            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials);
+            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none);
         NB_LAUNCH_OK("bn_silu_bwd_reduce");
     }
-    {
+    if (!fuse) {
         SiteTimer tm(p, SITE_BWD_FINALIZE, st);
         const int fin_blocks = (C + 7) / 8;
         int wt_blocks = 0;
-        WtParams none;
         if (wtp) {
             const size_t total = (size_t)wtp->c_in * wtp->k * wtp->k * wtp->c_out;
             wt_blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)p->sm_count * 8);
-        } else {
-            memset(&none, 0, sizeof none);
         }
         launch_k(bn_bwd_finalize_kernel, dim3(fin_blocks + wt_blocks), dim3(256), 0, st, 1, partials, e.blocks_reduce, C, (double)p->g.m, mean, invstd, gamma, beta,
                  dgamma, dbeta, coef, fin_blocks, static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(wt), wtp ? *wtp : none);
@@ -482,6 +490,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     float* shift = reinterpret_cast<float*>(ws + p->off_shift);
     float* part = reinterpret_cast<float*>(ws + p->off_fpart);
     int nparts = p->ew.blocks_stats;
+    bool finalized = false;
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
@@ -497,15 +506,20 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
-        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st);  // writes y (fp16) and the partial sums
+        // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
+        const bool fuse = !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+        const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
+        finalized = fuse;
     } else {
         NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
     }
-    NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
+    if (!finalized)
+        NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
     return run_apply<__half, __nv_bfloat16, true>(p, y_saved, a_out, scale, shift, st);
 }

@@ -46,6 +46,14 @@ struct IgemmParams {
     int tma_store;
     int out_w[3];
     CUtensorMap tmOut[3];
+    // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
+    // b, b + gridDim.x, ...: sums the per-CTA partials in fp64 and writes mean, invstd, scale, shift and the running
+    // statistics, which saves the separate finalize launch between this kernel and the apply pass.
+    int fin_on;
+    float fin_eps, fin_momentum;
+    double fin_count;
+    const float *fin_gamma, *fin_beta;
+    float *fin_mean, *fin_invstd, *fin_scale, *fin_shift, *fin_rmean, *fin_rvar;
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
     int variant;                 // experiment switches
@@ -872,6 +880,24 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 const float* base = wstat + (tm ? (size_t)8 * p.n_tiles * p.ncol_a : 0) + (size_t)which * ld + nt * (tm ? ncb : p.ncol_a) + (cc - (tm ? p.ncol_a : 0));
                 dst[e] = ((base[0] + base[2 * ld]) + base[4 * ld]) + base[6 * ld];
             }
+            if (p.fin_on) {
+                int* ctr = p.status + ST_BAR_FWD;
+                volatile int* fin_ok = abort_flag + 1;  // (the kernel uses all of the opt-in shared memory as dynamic: no static variables)
+                epi2_bar_sync();  // this CTA's partial sums are written
+                if (et == 0) *fin_ok = grid_arrive_wait(ctr, (int)gridDim.x) ? 1 : 0;
+                epi2_bar_sync();
+                if (*fin_ok) {
+                    const int ew = et >> 5;
+                    for (int c = (int)blockIdx.x + (int)gridDim.x * ew; c < p.ldo; c += (int)gridDim.x * 8)
+                        bn_finalize_channel<true>(p.partials, (int)gridDim.x, p.ldo, c, lane, p.fin_count, p.fin_eps, p.fin_momentum, p.fin_gamma, p.fin_beta,
+                                                  p.fin_mean, p.fin_invstd, p.fin_scale, p.fin_shift, p.fin_rmean, p.fin_rvar, nullptr, nullptr);
+                } else if (et == 0 && atomicCAS(p.status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
+                    p.status[ST_WHERE] = 20;
+                    p.status[ST_DETAIL] = (int)blockIdx.x;
+                }
+                epi2_bar_sync();  // every warp is past its reads of the partial sums
+                if (et == 0) grid_depart(ctr, (int)gridDim.x);
+            }
         }
 #ifdef NB_TC_DEBUG_TIMING
         if (p.dbg && warp == 2 && lane == 0) {
@@ -1401,7 +1427,13 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
     return NB_OK;
 }
 
-inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st) {
+struct FwdFinalize {  // inputs and outputs of the BatchNorm finalize that the forward kernel performs itself
+    float eps, momentum;
+    const float *gamma, *beta;
+    float *mean, *invstd, *scale, *shift, *rmean, *rvar;
+};
+inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st,
+                          const FwdFinalize* fin) {
     using namespace tcdetail;
     TcGemmSlot& S = tc->fp;
     if (S.a_ptr != x || S.b_ptr != w) {
@@ -1421,6 +1453,13 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     if (S.prm.tma_store && S.out_ptr != y) {
         if (!encode_out_maps(S.prm, S.cfg, y, g.m)) return NB_ERR_CUDA;
         S.out_ptr = y;
+    }
+    S.prm.fin_on = fin ? 1 : 0;
+    if (fin) {
+        S.prm.fin_eps = fin->eps; S.prm.fin_momentum = fin->momentum; S.prm.fin_count = (double)g.m;
+        S.prm.fin_gamma = fin->gamma; S.prm.fin_beta = fin->beta;
+        S.prm.fin_mean = fin->mean; S.prm.fin_invstd = fin->invstd; S.prm.fin_scale = fin->scale; S.prm.fin_shift = fin->shift;
+        S.prm.fin_rmean = fin->rmean; S.prm.fin_rvar = fin->rvar;
     }
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
 #ifdef NB_TC_DEBUG_TIMING
