@@ -61,6 +61,13 @@ typedef enum { NB_MODE_BF16_TC = 0, NB_MODE_F32_REF = 1 } nb_mode;
 /* nb_cbs_desc.flags */
 #define NB_CBS_FLAG_FORCE_SIMT 1u /* BF16 mode: run the three convolutions on the CUDA-core kernels
                                      (same arithmetic contract; for testing and as a cross-check) */
+#define NB_CBS_FLAG_SHARED_GPU 2u /* kernels of this plan may run at the same time as other kernels (other streams,
+                                     other processes).  By default the forward kernel and the backward reduce kernel
+                                     finish the BatchNorm statistics themselves behind a grid-wide barrier, which needs
+                                     all of their blocks resident at once: two such kernels that each hold half of the
+                                     GPU would wait for each other until the bounded waits give up (NB_ERR_TIMEOUT).
+                                     With this flag the finalize steps run as separate small kernels instead
+                                     (same results, a few microseconds more per call). */
 
 typedef struct nb_cbs_desc {
     uint32_t struct_size; /* = sizeof(nb_cbs_desc) */

@@ -19,6 +19,7 @@ NB_ERR_CUDA, NB_ERR_ARCH, NB_ERR_TIMEOUT, NB_ERR_INTERNAL = 5, 6, 7, 8
 NB_DTYPE_F32, NB_DTYPE_BF16, NB_DTYPE_F16 = 0, 1, 2
 NB_MODE_BF16_TC, NB_MODE_F32_REF = 0, 1
 NB_CBS_FLAG_FORCE_SIMT = 1
+NB_CBS_FLAG_SHARED_GPU = 2
 
 EXPORTS = (
     "nb_abi_version", "nb_last_error", "nb_cbs_plan_create", "nb_cbs_plan_destroy", "nb_cbs_out_shape",

@@ -174,7 +174,7 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
                               float* coef, cudaStream_t st, const void* w = nullptr, void* wt = nullptr, const WtParams* wtp = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
-    const bool fuse = !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+    const bool fuse = !(p->desc.flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
     WtParams none;
     if (!wtp) memset(&none, 0, sizeof none);
     {
@@ -507,7 +507,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
         // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
-        const bool fuse = !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+        const bool fuse = !(p->desc.flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
         const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
         const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);

@@ -171,6 +171,70 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
     return v;
 }
 
+// One epilogue pass of NP columns (16, 32, 48 or 64) by one warp when the output goes through TMA: this thread's
+// accumulator row segment travels TMEM -> registers -> dense staging rows (row pitch NP*2 bytes; 128-byte rows in the
+// 128-byte swizzle), `release` is called as soon as the registers hold the data (the accumulator may be reused), lane 0
+// hands the 32 x NP piece to TMA, and with STATS the warp adds the piece's per-channel sums of the rounded values to its
+// running sums (a lane owns two adjacent channels).  Everything is unrolled on NP: constant offsets, no predicates.
+template <typename OutT, bool STATS, int NP, class Release>
+__device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int lane, bool& store_pending, int& sat, const CUtensorMap* tm, int col,
+                                             int grow, float* stat_s, float* stat_q, Release release) {
+    constexpr bool SWZ = NP == 64;
+    constexpr int PITCH = NP * 2;
+    uint32_t r[NP];
+#pragma unroll
+    for (int hh = 0; hh < NP / 16; ++hh) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(16 * hh), r + 16 * hh);
+    ptx::tmem_ld_wait();
+    release();
+    if (store_pending) {  // the previous TMA store must have read the staging rows before they are overwritten
+        if (lane == 0) ptx::tma_store_wait_read<0>();
+        __syncwarp();
+    }
+    uint8_t* const my_row = wrows + lane * PITCH;
+    int sat_bits = 0;
+#pragma unroll
+    for (int j = 0; j < NP / 8; ++j) {
+        uint4 v;
+        v.x = pack2<OutT>(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]), &sat_bits);
+        v.y = pack2<OutT>(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]), &sat_bits);
+        v.z = pack2<OutT>(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]), &sat_bits);
+        v.w = pack2<OutT>(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]), &sat_bits);
+        *reinterpret_cast<uint4*>(my_row + (SWZ ? (j ^ (lane & 7)) : j) * 16) = v;
+    }
+    if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
+    ptx::fence_async_smem();  // writes visible to the async proxy before the store is issued
+    __syncwarp();
+    if (lane == 0) {
+        ptx::tma_store_2d(tm, wrows, col, grow);
+        ptx::tma_store_commit();
+    }
+    store_pending = true;
+    if (STATS) {
+        if (lane < NP / 2) {
+            float2 sa = make_float2(0.f, 0.f), sb = sa, qa = sa, qb = sa;
+            const int cj = lane >> 2;
+            const uint8_t* base = wrows + (lane & 3) * 4;
+#pragma unroll
+            for (int rr = 0; rr < 32; rr += 2) {
+                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(base + rr * PITCH + (SWZ ? (cj ^ (rr & 7)) : cj) * 16));
+                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(base + (rr + 1) * PITCH + (SWZ ? (cj ^ ((rr + 1) & 7)) : cj) * 16));
+                sa.x += f0.x; sa.y += f0.y;
+                sb.x += f1.x; sb.y += f1.y;
+                qa.x = fmaf(f0.x, f0.x, qa.x); qa.y = fmaf(f0.y, f0.y, qa.y);
+                qb.x = fmaf(f1.x, f1.x, qb.x); qb.y = fmaf(f1.y, f1.y, qb.y);
+            }
+            float2* ps = reinterpret_cast<float2*>(stat_s + 2 * lane);
+            float2* pq = reinterpret_cast<float2*>(stat_q + 2 * lane);
+            float2 a2 = *ps, b2 = *pq;
+            a2.x += sa.x + sb.x; a2.y += sa.y + sb.y;
+            b2.x += qa.x + qb.x; b2.y += qa.y + qb.y;
+            *ps = a2;
+            *pq = b2;
+        }
+        __syncwarp();  // staged rows read before the next pass overwrites them
+    }
+}
+
 // CG2 = the CTAs run as pairs (clusters of two): rank 0 issues tcgen05.mma.cta_group::2 with M = 256; each CTA owns 128
 // of the rows (its own A tile, accumulator and epilogue) and fetches half of the B tile, which halves the filter
 // bytes written to and read from each SM's shared memory.
@@ -696,6 +760,30 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // The team's columns go through the staging buffer in passes of at most cw (<= 64) columns.
                 for (int cb = 0; cb < ncol; cb += cw) {
                 const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
+                if (tma_out && !(p.variant & (16 | 32))) {
+                    const bool last = h == mh - 1 && cb + cw >= ncol;  // last TMEM read of this tile: the accumulator set becomes free
+                    auto release = [&]() {
+                        if (last) {
+                            ptx::tc_fence_before();
+                            if (CG2) {
+                                __syncwarp();
+                                if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
+                            } else {
+                                ptx::mbar_arrive(tempty + acc);
+                            }
+                        }
+                    };
+                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut[0] : npass == p.out_w[1] ? &p.tmOut[1] : &p.tmOut[2];
+                    const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
+                    float* ss = my_stat + n_tile * ncol + cb;
+                    float* sq = ss + st_ld;
+                    const uint32_t ta = taddr + (uint32_t)cb;
+                    if (npass == 64) epi_pass_tma<OutT, STATS, 64>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
+                    else if (npass == 48) epi_pass_tma<OutT, STATS, 48>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
+                    else if (npass == 32) epi_pass_tma<OutT, STATS, 32>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
+                    else epi_pass_tma<OutT, STATS, 16>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
+                    continue;
+                }
                 const int rpitch = tma_out ? npass * 2 : pitch;       // bytes between staged rows of this pass
                 const bool swz = tma_out && npass == 64;              // 128-byte rows: 16-byte chunk j of row r sits at j ^ (r & 7)
                 uint8_t* const my_row = wrows + (size_t)lane * rpitch;

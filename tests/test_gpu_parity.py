@@ -90,6 +90,15 @@ def test_forced_cuda_core_path_matches_oracle(shape):
     _compare(out, _oracle(inp), 0)
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[9], SMALL_SHAPES[12]], ids=lambda s: s.name)
+def test_separate_finalize_kernels_match_oracle(shape):
+    """NB_CBS_FLAG_SHARED_GPU: the finalize steps run as separate kernels instead of behind in-kernel grid barriers."""
+    from paper_2609_10632_b200 import binding as nb
+
+    inp, blk, out = _run_block(shape, 0, cfg_id=14, affine="random", flags=nb.NB_CBS_FLAG_SHARED_GPU, running=True)
+    _compare(out, _oracle(inp), 0)
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[11], S(3, 9, 11, 32, 16, 3, 1), S(2, 24, 24, 96, 192, 3, 1)],
                          ids=lambda s: s.name)
 def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
