@@ -1467,50 +1467,65 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
         }
         P.n_tiles = g.c_out / P.BN;
         P.nblkB = (P.BN + 63) / 64;
-        // 128 pixels per stage when at least three stages fit, else 64
-        P.KP = 128;
-        for (;;) {
-            P.blk_bytes = (uint32_t)(64 * 2 * P.KP);
-            P.a_stage_bytes = 2 * P.blk_bytes;
-            P.b_stage_bytes = (uint32_t)P.nblkB * P.blk_bytes;
-            P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
-            if (P.stages >= 3 || P.KP == 64) break;
-            P.KP = 64;
-        }
-        if (getenv("NB_WG_KP")) {
-            P.KP = atoi(getenv("NB_WG_KP"));
-            P.blk_bytes = (uint32_t)(64 * 2 * P.KP);
-            P.a_stage_bytes = 2 * P.blk_bytes;
-            P.b_stage_bytes = (uint32_t)P.nblkB * P.blk_bytes;
-            P.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (P.a_stage_bytes + P.b_stage_bytes));
-        }
-        P.total_chunks = (int)((g.m + P.KP - 1) / P.KP);
-        const int tiles = P.m_tiles * P.n_tiles;
-        // split-K factor: fewest waves of CTAs times chunks per CTA (plus a fixed prologue/epilogue of a few chunks)
-        int best_s = 1;
-        double best_c = 1e30;
-        const int max_s = std::max(1, std::min(64, P.total_chunks / 4));
-        for (int sp = 1; sp <= max_s; ++sp) {
-            const double waves = (double)(((long long)tiles * sp + sm_count - 1) / sm_count);
-            const double c = waves * ((P.total_chunks + sp - 1) / sp + 6.0) + 0.02 * sp;
-            if (c < best_c - 1e-9) {
-                best_c = c;
-                best_s = sp;
+        // One or two 128-row accumulator blocks per CTA.  With two, four x boxes share every dy stage (a third less
+        // shared-memory traffic per MMA: measured 1.6x the time of a one-block stage for twice the work) but there are half
+        // as many tiles, hence more split-K slices with fewer pixels each.  Both are planned and the cheaper one is kept;
+        // cost = waves x (stage time x stages per CTA + a fixed prologue/epilogue), in units of a 128-pixel one-block stage.
+        P.acc_stride = P.BN <= 32 ? 32 : P.BN <= 64 ? 64 : P.BN <= 128 ? 128 : 256;
+        double best_cost = 1e30;
+        WgradParams bestP = P;
+        const int force_mh = getenv("NB_WG_MH") ? atoi(getenv("NB_WG_MH")) : 0;
+        for (int mh = 1; mh <= 2; ++mh) {
+            if (mh == 2 && (P.nblk_total < 4 || 2 * P.acc_stride > 512)) continue;
+            if (force_mh && mh != force_mh && !(force_mh == 2 && (P.nblk_total < 4 || 2 * P.acc_stride > 512))) continue;
+            WgradParams Q = P;
+            Q.mh = mh;
+            Q.m_tiles = (Q.nblk_total + 2 * mh - 1) / (2 * mh);
+            // 128 pixels per stage when at least three stages fit, else 64
+            Q.KP = getenv("NB_WG_KP") ? atoi(getenv("NB_WG_KP")) : 128;
+            for (;;) {
+                Q.blk_bytes = (uint32_t)(64 * 2 * Q.KP);
+                Q.a_stage_bytes = 2 * mh * Q.blk_bytes;
+                Q.b_stage_bytes = (uint32_t)Q.nblkB * Q.blk_bytes;
+                Q.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (Q.a_stage_bytes + Q.b_stage_bytes));
+                if (Q.stages >= 3 || Q.KP == 64 || getenv("NB_WG_KP")) break;
+                Q.KP = 64;
+            }
+            if (Q.stages < 2) continue;
+            Q.total_chunks = (int)((g.m + Q.KP - 1) / Q.KP);
+            const int tiles = Q.m_tiles * Q.n_tiles;
+            const double stage_time = (Q.KP / 128.0) * (mh == 2 ? 1.6 : 1.0), fixed = mh == 2 ? 10.0 : 6.0;
+            int best_s = 1;
+            double best_c = 1e30;
+            const int max_s = std::max(1, std::min(64, Q.total_chunks / 4));
+            for (int sp = 1; sp <= max_s; ++sp) {
+                const double waves = (double)(((long long)tiles * sp + sm_count - 1) / sm_count);
+                const double c = waves * (((Q.total_chunks + sp - 1) / sp) * stage_time + fixed) + 0.02 * sp;
+                if (c < best_c - 1e-9) {
+                    best_c = c;
+                    best_s = sp;
+                }
+            }
+            if (getenv("NB_WG_SPLITS")) best_s = std::max(1, std::min(max_s, atoi(getenv("NB_WG_SPLITS"))));
+            Q.chunks_per_split = (Q.total_chunks + best_s - 1) / best_s;
+            Q.splits = (Q.total_chunks + Q.chunks_per_split - 1) / Q.chunks_per_split;
+            Q.stages = std::max(2, std::min(Q.stages, std::max(2, Q.chunks_per_split)));
+            if (best_c < best_cost - 1e-9) {
+                best_cost = best_c;
+                bestP = Q;
             }
         }
-        if (getenv("NB_WG_SPLITS")) best_s = std::max(1, std::min(max_s, atoi(getenv("NB_WG_SPLITS"))));
-        P.chunks_per_split = (P.total_chunks + best_s - 1) / best_s;
-        P.splits = (P.total_chunks + P.chunks_per_split - 1) / P.chunks_per_split;
-        P.stages = std::max(2, std::min(P.stages, std::max(2, P.chunks_per_split)));
-        P.tmem_cols = P.BN <= 32 ? 32 : P.BN <= 64 ? 64 : P.BN <= 128 ? 128 : 256;
+        P = bestP;
+        const int tiles = P.m_tiles * P.n_tiles;
+        P.tmem_cols = P.mh * P.acc_stride;
         P.idesc = ptx::make_idesc_bf16(128, P.BN, 1, 1);
         tc->wg_smem = std::max<size_t>(2048 + (size_t)P.stages * (P.a_stage_bytes + P.b_stage_bytes), 120 * 1024);
         tc->wg_grid = tiles * P.splits;
         tc->wgrad_partial_bytes = P.splits > 1 ? (size_t)P.splits * g.c_out * g.kdim * 4 : 0;
         tc->wgrad = true;
         if (getenv("NB_TC_VERBOSE"))
-            fprintf(stderr, "[nb_cbs] wgrad M=%lld Cin=%d Cout=%d k=%d: BN=%d KP=%d stages=%d tiles=%dx%d splits=%d (chunks/split %d) grid=%d\n", (long long)g.m,
-                    g.c_in, g.c_out, g.k, P.BN, P.KP, P.stages, P.m_tiles, P.n_tiles, P.splits, P.chunks_per_split, tc->wg_grid);
+            fprintf(stderr, "[nb_cbs] wgrad M=%lld Cin=%d Cout=%d k=%d: BN=%d mh=%d KP=%d stages=%d tiles=%dx%d splits=%d (chunks/split %d) grid=%d\n", (long long)g.m,
+                    g.c_in, g.c_out, g.k, P.BN, P.mh, P.KP, P.stages, P.m_tiles, P.n_tiles, P.splits, P.chunks_per_split, tc->wg_grid);
     }
     return NB_OK;
 }

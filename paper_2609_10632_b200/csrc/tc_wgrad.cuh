@@ -20,6 +20,8 @@ struct WgradParams {
     int nblk_total;    // taps * cblk_per_tap
     int nblkB;         // ceil(BN / 64)
     int KP;            // pixels per pipeline stage (64 or 128)
+    int mh;            // 128-row accumulator blocks per CTA (1 or 2): with 2, four x boxes share every dy stage
+    int acc_stride;    // TMEM columns between the accumulator blocks
     int BN, n_tiles, m_tiles;
     int splits, chunks_per_split, total_chunks;
     int stages, tmem_cols;
@@ -87,17 +89,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes;
             const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB), full_u32 = ptx::smem_u32(full);
             const CUtensorMap* tm = isA ? &p.tmA : &p.tmB;
-            const int nblk = isA ? 2 : p.nblkB;
-            // the two 64-channel blocks of x this tile owns (a block past the end of the filter is replaced by block 0:
+            const int nblkA = 2 * p.mh;
+            const int nblk = isA ? nblkA : p.nblkB;
+            // the 64-channel blocks of x this tile owns (a block past the end of the filter is replaced by block 0:
             // its accumulator rows are never stored)
-            int tapv[2], c0v[2];
-            for (int b = 0; b < 2; ++b) {
-                int fb = m_tile * 2 + b;
-                if (fb >= p.nblk_total) fb = 0;
-                tapv[b] = fb / p.cblk_per_tap;
-                c0v[b] = (fb - tapv[b] * p.cblk_per_tap) * 64;
+            int c0v[4];
+            uint16_t owv[4], ohv[4];
+            for (int b = 0; b < 4; ++b) {
+                int fb = m_tile * nblkA + b;
+                if (b >= nblkA || fb >= p.nblk_total) fb = 0;
+                const int tap = fb / p.cblk_per_tap;
+                c0v[b] = (fb - tap * p.cblk_per_tap) * 64;
+                owv[b] = p.off_w[tap];
+                ohv[b] = p.off_h[tap];
             }
-            const uint16_t ow0 = p.off_w[tapv[0]], oh0 = p.off_h[tapv[0]], ow1 = p.off_w[tapv[1]], oh1 = p.off_h[tapv[1]];
             const int bcol = n_tile * p.BN;
             for (int ch = chunk0; ch < chunk1; ++ch) {
                 const int m0 = ch * KP;
@@ -112,8 +117,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                     const int j0 = m0 % Wq, t1 = m0 / Wq;
                     const int i0 = t1 % Hq, n0 = t1 / Hq;
                     const int cw = p.lo_w + j0 * ts, chh = p.lo_h + i0 * ts;
-                    ptx::tma_load_im2col_4d_u32_if(leader, dst, tm, bar, c0v[0], cw, chh, n0, ow0, oh0);
-                    ptx::tma_load_im2col_4d_u32_if(leader, dst + blk, tm, bar, c0v[1], cw, chh, n0, ow1, oh1);
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if (b < nblkA) ptx::tma_load_im2col_4d_u32_if(leader, dst + (uint32_t)b * blk, tm, bar, c0v[b], cw, chh, n0, owv[b], ohv[b]);
                 } else {
                     for (int b = 0; b < nblk; ++b) ptx::tma_load_2d_u32_if(leader, dst + (uint32_t)b * blk, tm, bar, bcol + b * 64, m0);
                 }
@@ -141,8 +147,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            const int stages = p.stages, ksteps = p.KP / 16;
-            const uint32_t idesc = p.idesc;
+            const int stages = p.stages, ksteps = p.KP / 16, mh = p.mh;
+            const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
+            const uint64_t a_half16 = (uint64_t)((2 * p.blk_bytes) >> 4);  // the second pair of x blocks inside a stage
             // MN-major, 128-byte swizzle: 8 pixel rows of 128 bytes form one 1024-byte group (SBO); the next 64 channels
             // start one block later (LBO); a K = 16 step advances by two row groups.
             const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), p.blk_bytes, 1024, ptx::kSwizzle128);
@@ -161,6 +168,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 #pragma unroll 4
                 for (int k = 0; k < ksteps; ++k) {
                     ptx::umma_f16_if(leader, tmem_base, da, db, idesc, accumulate);
+                    if (mh == 2) ptx::umma_f16_if(leader, tmem_base + acc_stride, da + a_half16, db, idesc, accumulate);
                     accumulate = 1u;
                     da += 128;  // 2048 bytes >> 4
                     db += 128;
@@ -189,19 +197,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         // ------------------------------------------------------------------ epilogue (warps 2-5)
         const int lane_group = warp & 3;
         const int row = lane_group * 32 + lane;
-        // accumulator row -> (tap, channel): rows come in two blocks of 64 channels
-        const int fb = m_tile * 2 + (row >> 6);
-        const int tap = fb / p.cblk_per_tap;
-        const int c = (fb - tap * p.cblk_per_tap) * 64 + (row & 63);
-        const bool valid = fb < p.nblk_total && c < p.c_in;
-        const int kidx = tap * p.c_in + c;  // position inside dw[c'][:]
         bool ok = true;
         if (nchunks > 0 && lane == 0) ok = wait_bar(tfull, 0, abort_flag, p.status, 13);
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         ok = epi_bar_and(ok);
-        if (ok) {
-            ptx::tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16);
+        if (ok) ptx::tc_fence_after();
+        for (int h = 0; ok && h < p.mh; ++h) {
+            // accumulator row -> (tap, channel): rows come in blocks of 64 channels
+            const int fb = (m_tile * p.mh + h) * 2 + (row >> 6);
+            const int tap = fb / p.cblk_per_tap;
+            const int c = (fb - tap * p.cblk_per_tap) * 64 + (row & 63);
+            const bool valid = fb < p.nblk_total && c < p.c_in;
+            const int kidx = tap * p.c_in + c;  // position inside dw[c'][:]
+            const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(h * p.acc_stride);
             float* dst = p.out + (size_t)split * p.c_out * p.kdim;
             for (int c0 = 0; c0 < p.BN; c0 += 16) {
                 uint32_t r[16];
