@@ -363,7 +363,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     }
 
     p->stem = d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
-              g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0;
+              g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0 && g.m < (1LL << 31) && (long long)g.n * g.h * g.w * 3 < (1LL << 31);
     p->stem_blocks = (int)std::min<long long>((g.m + 255) / 256, (long long)p->sm_count * 8);
     p->nparts = std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts);
     const size_t C = (size_t)g.c_out;
@@ -497,9 +497,9 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     } else if (p->stem) {
         {
             SiteTimer tm(p, SITE_FPROP, st);
-            const int blocks = (int)std::min<long long>((p->g.m + 127) / 128, (long long)p->sm_count * 16);
-            launch_k(stem_fprop_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
-                                                         static_cast<__half*>(y_saved), p->g);
+            const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
+            launch_k(stem_fprop_mma_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
+                         static_cast<__half*>(y_saved), p->g);
             NB_LAUNCH_OK("stem_fprop");
         }
         NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
@@ -565,10 +565,12 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     if (!dx) return NB_OK;
     if (p->stem) {
         SiteTimer tm(p, SITE_DGRAD, st);
-        const long long total = (long long)p->g.n * p->g.h * (p->g.w / 2);
-        const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-        launch_k(stem_dgrad_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
-                                                     static_cast<__nv_bfloat16*>(dx), p->g);
+        {
+            const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
+            const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
+            launch_k(stem_dgrad_tiled_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
+                     static_cast<__nv_bfloat16*>(dx), p->g);
+        }
         return launch_ok("stem_dgrad");
     }
     if (p->tc.dgrad) {
@@ -595,7 +597,7 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
         {
             SiteTimer tm(p, SITE_WGRAD, st);
             const long long per = (p->g.m + p->stem_blocks - 1) / p->stem_blocks;
-            launch_k(stem_wgrad_kernel<48>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
+            launch_k(stem_wgrad_mma_kernel<48>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
                                                                  partial, p->g, per);
             NB_LAUNCH_OK("stem_wgrad");
         }

@@ -1,8 +1,8 @@
-// Direct CUDA-core kernels for the network's first layer: 3 input channels, 3x3, stride 2, pad 1.
-// A 3-channel bf16 pixel is 6 bytes, which no TMA descriptor can address (strides must be multiples of 16 bytes),
-// and with K = 27 the layer is bound by HBM traffic, not by arithmetic: these kernels keep the filter in shared
-// memory as fp32, one thread per output pixel (fprop), per pair of input pixels (dgrad), or per 4x3 patch of the
-// filter gradient (wgrad).  COUT is a template parameter (48 for the detector's stem).
+// Kernels for the network's first layer: 3 input channels, 3x3, stride 2, pad 1.
+// A 3-channel bf16 pixel is 6 bytes, which no TMA descriptor can address (strides must be multiples of 16 bytes), and
+// K = 27 is far too short for the tcgen05 pipeline: the forward and the weight gradient run on warp-level mma.sync tiles of
+// 16 pixels, the data gradient (3 output channels) on register-tiled CUDA-core FMAs.  COUT is a template parameter
+// (48 for the detector's stem).
 #pragma once
 #include "common.cuh"
 
@@ -10,203 +10,289 @@ namespace nbcbs {
 
 constexpr int STEM_CIN = 3, STEM_K = 3, STEM_TAPS = 9, STEM_KDIM = 27;
 
-// y[n,p,q,:] = sum_{r,t,c} x[n,2p-1+r,2q-1+t,c] * w[:,r,t,c]   (fp16 output, fp32 accumulate)
+// ---- tensor-core forward for the stem.  K = 27 is far too short for the tcgen05 pipeline (and a 6-byte pixel cannot be
+// fetched by TMA), so this kernel uses warp-level mma.sync (m16n8k16, bf16 -> fp32): a warp computes 16 consecutive output
+// pixels x COUT channels with K padded to 32.  The filter fragments stay in registers for the whole kernel; a thread
+// gathers the 2 x 8 input values of its fragment rows with 2-byte loads (the 3 x 3 x 3 patch of a pixel is three runs of 9
+// contiguous values, L1-resident across neighbouring pixels) and writes its accumulator pairs as fp16.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 template <int COUT>
-__global__ void __launch_bounds__(128) stem_fprop_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
-                                                         __half* __restrict__ y, Geom g) {
+__global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+                                                             __half* __restrict__ y, Geom g) {
     pdl_launch_dependents();
     pdl_wait();
-    __shared__ __align__(16) float ws[STEM_KDIM][COUT];  // ws[k][c'] = w[c'][k]
-    for (int e = threadIdx.x; e < STEM_KDIM * COUT; e += blockDim.x) {
-        const int co = e / STEM_KDIM, k = e % STEM_KDIM;
-        ws[k][co] = __bfloat162float(w[e]);
-    }
-    __syncthreads();
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < g.m; m += stride) {
-        const int q = (int)(m % g.wo);
-        const long long t1 = m / g.wo;
-        const int p = (int)(t1 % g.ho), n = (int)(t1 / g.ho);
-        float xin[STEM_KDIM];
+    static_assert(COUT % 8 == 0, "whole n-blocks");
+    constexpr int NB = COUT / 8;
+    const int lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
+    const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
+    const unsigned short* wsrc = reinterpret_cast<const unsigned short*>(w);
+    // the eight K indices of this lane's A / B fragment elements: k-step s, register half j, element e
+    int koff[8];   // element offset of K index k inside the input relative to the patch origin, or -1 for the padding (k >= 27)
+    int kr[8], kt[8];  // filter row and column of k (bounds checks)
+    uint32_t bfrag[2][NB][2];
 #pragma unroll
-        for (int r = 0; r < 3; ++r) {
-            const int h = 2 * p - 1 + r;
+    for (int s2 = 0; s2 < 2; ++s2)
 #pragma unroll
-            for (int t = 0; t < 3; ++t) {
-                const int ww = 2 * q - 1 + t;
-                const bool ok = h >= 0 && h < g.h && ww >= 0 && ww < g.w;
-                const __nv_bfloat16* px = x + (((size_t)n * g.h + (ok ? h : 0)) * g.w + (ok ? ww : 0)) * 3;
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-                for (int c = 0; c < 3; ++c) xin[(r * 3 + t) * 3 + c] = ok ? __bfloat162float(px[c]) : 0.f;
+            for (int e = 0; e < 2; ++e) {
+                const int k = s2 * 16 + j * 8 + tq * 2 + e, i = s2 * 4 + j * 2 + e;
+                const int r = k / 9, kp = k - r * 9;
+                kr[i] = r;
+                kt[i] = kp / 3;
+                koff[i] = k < STEM_KDIM ? r * g.w * 3 + kp : -1;
             }
-        }
-        float acc[COUT];
 #pragma unroll
-        for (int c = 0; c < COUT; ++c) acc[c] = 0.f;
+    for (int s2 = 0; s2 < 2; ++s2)
 #pragma unroll
-        for (int k = 0; k < STEM_KDIM; ++k) {
-            const float xv = xin[k];
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-            for (int c = 0; c < COUT; c += 4) {
-                const float4 wv = *reinterpret_cast<const float4*>(&ws[k][c]);
-                acc[c] = fmaf(xv, wv.x, acc[c]);
-                acc[c + 1] = fmaf(xv, wv.y, acc[c + 1]);
-                acc[c + 2] = fmaf(xv, wv.z, acc[c + 2]);
-                acc[c + 3] = fmaf(xv, wv.w, acc[c + 3]);
+            for (int j = 0; j < 2; ++j) {
+                const int k = s2 * 16 + j * 8 + tq * 2, n = nb * 8 + gq;
+                const uint32_t lo = k < STEM_KDIM ? wsrc[n * STEM_KDIM + k] : 0u, hi = k + 1 < STEM_KDIM ? wsrc[n * STEM_KDIM + k + 1] : 0u;
+                bfrag[s2][nb][j] = lo | (hi << 16);
             }
-        }
-        __half* yo = y + (size_t)m * COUT;
+    __shared__ __align__(16) __half stage[4][16 * COUT];
+    const long long ntiles = (g.m + 15) / 16;
+    const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < ntiles; tile += wstride) {
+        const long long m0 = tile * 16;
+        uint32_t a[2][4];
 #pragma unroll
-        for (int c = 0; c < COUT; c += 8) {
-            Vec16<__half> v;
+        for (int half = 0; half < 2; ++half) {  // fragment rows gq and gq + 8
+            const long long m = m0 + gq + half * 8;
+            const bool row_ok = m < g.m;
+            const unsigned mm = row_ok ? (unsigned)m : 0u;  // the stem has fewer than 2^31 output pixels: 32-bit divisions
+            const unsigned t1 = mm / (unsigned)g.wo;
+            const int q = (int)(mm - t1 * (unsigned)g.wo);
+            const int n = (int)(t1 / (unsigned)g.ho), p = (int)(t1 - (unsigned)n * (unsigned)g.ho);
+            const int h0 = 2 * p - 1, w0 = 2 * q - 1;
+            const long long origin = (((long long)n * g.h + h0) * g.w + w0) * 3;  // may point before the image; only used when in bounds
+            unsigned short v[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v.v[i] = from_f32<__half>(acc[c + i]);
-            st16(yo + c, v);
+            for (int i = 0; i < 8; ++i) {
+                const int h = h0 + kr[i], ww = w0 + kt[i];
+                const bool ok = row_ok && koff[i] >= 0 && h >= 0 && h < g.h && ww >= 0 && ww < g.w;
+                v[i] = ok ? xs[origin + koff[i]] : (unsigned short)0;
+            }
+            // registers of m16n8k16 A: a0 = (row g, k 2t..2t+1), a1 = (row g+8, same k), a2 = (row g, k 2t+8..), a3 = (row g+8, k 2t+8..)
+            a[0][half] = (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+            a[0][2 + half] = (uint32_t)v[2] | ((uint32_t)v[3] << 16);
+            a[1][half] = (uint32_t)v[4] | ((uint32_t)v[5] << 16);
+            a[1][2 + half] = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
         }
+        float acc[NB][4];
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+            acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
+            mma_bf16_16816(acc[nb], a[0], bfrag[0][nb][0], bfrag[0][nb][1]);
+            mma_bf16_16816(acc[nb], a[1], bfrag[1][nb][0], bfrag[1][nb][1]);
+        }
+        // accumulator registers: c0, c1 = (row g, columns 2t, 2t+1), c2, c3 = (row g+8, same columns).  The 16 x COUT tile is one
+        // contiguous run of the output, so it is staged in shared memory and written with coalesced 16-byte stores.
+        __half* st = stage[threadIdx.x >> 5];
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+                *reinterpret_cast<__half2*>(st + (gq + half * 8) * COUT + nb * 8 + tq * 2) =
+                    __halves2half2(from_f32<__half>(acc[nb][2 * half]), from_f32<__half>(acc[nb][2 * half + 1]));
+        __syncwarp();
+        const long long rows_left = g.m - m0;
+        const int nvec = (int)(rows_left >= 16 ? 16 : rows_left) * COUT / 8;  // 16-byte pieces of the tile that exist
+        for (int v = lane; v < nvec; v += 32) st16(y + (size_t)m0 * COUT + v * 8, ld16(st + v * 8));
+        __syncwarp();
     }
 }
 
-// dx for two horizontally adjacent input pixels (w = 2*w2, 2*w2+1) per thread; H and W even.
-// Input column 2*w2 sees filter column t=1 at output column w2; column 2*w2+1 sees t=0 at w2+1 and t=2 at w2.
-// Input row h even sees filter row r=1 at output row h/2; h odd sees r=0 at (h+1)/2 and r=2 at (h-1)/2.
+// Data gradient, register-tiled: a thread produces the 2 x 4 input pixels (rows 2i, 2i+1, columns 4jp .. 4jp+3) that the
+// six dy pixels (rows i, i+1, columns 2jp .. 2jp+2) feed, so one broadcast read of a channel's 27 filter values serves
+// 54 FMAs (a one-pair-per-thread version read three float4 per nine FMAs and was bound by shared-memory reads: 246 us
+// against 175 us on the 16 x 640 x 640 stem).
+// With pixel (2i+a, 2j+b): (0,0) <- dy[i][j] w11;  (0,1) <- dy[i][j+1] w10 + dy[i][j] w12;  (1,0) <- dy[i+1][j] w01 + dy[i][j] w21;
+// (1,1) <- dy[i+1][j+1] w00 + dy[i+1][j] w02 + dy[i][j+1] w20 + dy[i][j] w22   (w_rt = filter tap (r,t); H and W even).
 template <int COUT>
-__global__ void __launch_bounds__(128) stem_dgrad_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ w,
-                                                         __nv_bfloat16* __restrict__ dx, Geom g) {
+__global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ w,
+                                                               __nv_bfloat16* __restrict__ dx, Geom g) {
     pdl_launch_dependents();
     pdl_wait();
-    __shared__ __align__(16) float ws[STEM_TAPS][COUT][4];  // ws[tap][c'][c], c padded to 4
-    for (int e = threadIdx.x; e < STEM_TAPS * COUT; e += blockDim.x) {
-        const int tap = e / COUT, co = e % COUT;
-#pragma unroll
-        for (int c = 0; c < 3; ++c) ws[tap][co][c] = __bfloat162float(w[((size_t)co * STEM_TAPS + tap) * 3 + c]);
-        ws[tap][co][3] = 0.f;
-    }
+    __shared__ __align__(16) float ws[COUT][28];  // ws[c'][tap*3 + c]
+    for (int e = threadIdx.x; e < COUT * STEM_KDIM; e += blockDim.x) ws[e / STEM_KDIM][e % STEM_KDIM] = __bfloat162float(w[e]);
     __syncthreads();
-    const int w2n = g.w / 2;
-    const long long total = (long long)g.n * g.h * w2n;
+    const int npair = (g.wo + 1) / 2;
+    const long long total = (long long)g.n * g.ho * npair;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += stride) {
-        const int w2 = (int)(idx % w2n);
-        const long long t1 = idx / w2n;
-        const int h = (int)(t1 % g.h), n = (int)(t1 / g.h);
-        float e0 = 0.f, e1 = 0.f, e2 = 0.f;  // pixel (h, 2*w2)
-        float o0 = 0.f, o1 = 0.f, o2 = 0.f;  // pixel (h, 2*w2+1)
-        const int nrows = (h & 1) ? 2 : 1;
-        for (int ri = 0; ri < nrows; ++ri) {
-            int r, p;
-            if (h & 1) {
-                r = ri == 0 ? 0 : 2;
-                p = ri == 0 ? (h + 1) / 2 : (h - 1) / 2;
-            } else {
-                r = 1;
-                p = h / 2;
-            }
-            if (p >= g.ho) continue;
-            const __nv_bfloat16* row = dy + (((size_t)n * g.ho + p) * g.wo) * COUT;
-            const __nv_bfloat16* dA = row + (size_t)w2 * COUT;  // output column w2
-            const bool hasB = w2 + 1 < g.wo;
-            const __nv_bfloat16* dB = row + (size_t)(hasB ? w2 + 1 : w2) * COUT;  // output column w2+1
+        const int jp = (int)(idx % npair);
+        const long long t1 = idx / npair;
+        const int i = (int)(t1 % g.ho), n = (int)(t1 / g.ho);
+        const int j = 2 * jp;
+        const bool row1 = i + 1 < g.ho, col1 = j + 1 < g.wo, col2 = j + 2 < g.wo;
+        const __nv_bfloat16* r0 = dy + (((size_t)n * g.ho + i) * g.wo + j) * COUT;
+        const __nv_bfloat16* r1 = r0 + (size_t)g.wo * COUT;
+        float acc[2][4][3];  // [row a][column 0..3 of the 4 produced][channel]
 #pragma unroll
-            for (int c0 = 0; c0 < COUT; c0 += 8) {
-                const Vec16<__nv_bfloat16> va = ld16(dA + c0);
-                const Vec16<__nv_bfloat16> vb = ld16(dB + c0);
+        for (int a = 0; a < 2; ++a)
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float a = __bfloat162float(va.v[i]);
-                    const float b = hasB ? __bfloat162float(vb.v[i]) : 0.f;
-                    const float4 w1 = *reinterpret_cast<const float4*>(ws[r * 3 + 1][c0 + i]);  // t = 1
-                    const float4 w0 = *reinterpret_cast<const float4*>(ws[r * 3 + 0][c0 + i]);  // t = 0
-                    const float4 w2v = *reinterpret_cast<const float4*>(ws[r * 3 + 2][c0 + i]); // t = 2
-                    e0 = fmaf(a, w1.x, e0); e1 = fmaf(a, w1.y, e1); e2 = fmaf(a, w1.z, e2);
-                    o0 = fmaf(b, w0.x, o0); o1 = fmaf(b, w0.y, o1); o2 = fmaf(b, w0.z, o2);
-                    o0 = fmaf(a, w2v.x, o0); o1 = fmaf(a, w2v.y, o1); o2 = fmaf(a, w2v.z, o2);
+            for (int b = 0; b < 4; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = 0.f;
+        Vec16<__nv_bfloat16> zero;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) zero.v[e] = __float2bfloat16_rn(0.f);
+#pragma unroll 1
+        for (int c0 = 0; c0 < COUT; c0 += 8) {
+            const Vec16<__nv_bfloat16> v00 = ld16(r0 + c0);
+            const Vec16<__nv_bfloat16> v01 = col1 ? ld16(r0 + COUT + c0) : zero;
+            const Vec16<__nv_bfloat16> v02 = col2 ? ld16(r0 + 2 * COUT + c0) : zero;
+            const Vec16<__nv_bfloat16> v10 = row1 ? ld16(r1 + c0) : zero;
+            const Vec16<__nv_bfloat16> v11 = (row1 && col1) ? ld16(r1 + COUT + c0) : zero;
+            const Vec16<__nv_bfloat16> v12 = (row1 && col2) ? ld16(r1 + 2 * COUT + c0) : zero;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float d00 = __bfloat162float(v00.v[e]), d01 = __bfloat162float(v01.v[e]), d02 = __bfloat162float(v02.v[e]);
+                const float d10 = __bfloat162float(v10.v[e]), d11 = __bfloat162float(v11.v[e]), d12 = __bfloat162float(v12.v[e]);
+                float wv[28];
+#pragma unroll
+                for (int q = 0; q < 7; ++q) *reinterpret_cast<float4*>(wv + 4 * q) = *reinterpret_cast<const float4*>(&ws[c0 + e][4 * q]);
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const float w00 = wv[0 + c], w01 = wv[3 + c], w02 = wv[6 + c], w10 = wv[9 + c], w11 = wv[12 + c], w12 = wv[15 + c];
+                    const float w20 = wv[18 + c], w21 = wv[21 + c], w22 = wv[24 + c];
+                    // first 2 x 2 group (dy column j), second (dy column j+1)
+                    acc[0][0][c] = fmaf(d00, w11, acc[0][0][c]);
+                    acc[0][1][c] = fmaf(d01, w10, fmaf(d00, w12, acc[0][1][c]));
+                    acc[1][0][c] = fmaf(d10, w01, fmaf(d00, w21, acc[1][0][c]));
+                    acc[1][1][c] = fmaf(d11, w00, fmaf(d10, w02, fmaf(d01, w20, fmaf(d00, w22, acc[1][1][c]))));
+                    acc[0][2][c] = fmaf(d01, w11, acc[0][2][c]);
+                    acc[0][3][c] = fmaf(d02, w10, fmaf(d01, w12, acc[0][3][c]));
+                    acc[1][2][c] = fmaf(d11, w01, fmaf(d01, w21, acc[1][2][c]));
+                    acc[1][3][c] = fmaf(d12, w00, fmaf(d11, w02, fmaf(d02, w20, fmaf(d01, w22, acc[1][3][c]))));
                 }
             }
         }
-        // six consecutive bf16 values (12 bytes) at a 4-byte aligned address
-        __nv_bfloat16* o = dx + (((size_t)n * g.h + h) * g.w + 2 * (size_t)w2) * 3;
-        __nv_bfloat162* o2p = reinterpret_cast<__nv_bfloat162*>(o);
-        o2p[0] = __floats2bfloat162_rn(e0, e1);
-        o2p[1] = __floats2bfloat162_rn(e2, o0);
-        o2p[2] = __floats2bfloat162_rn(o1, o2);
+        // rows 2i and 2i+1, columns 4jp .. 4jp+3 (the last two only when dy column j+1 exists): 12 bf16 = 24 bytes per row, 8-byte aligned
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+            __nv_bfloat16* o = dx + (((size_t)n * g.h + 2 * i + a) * g.w + 4 * (size_t)jp) * 3;
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(o);
+            o2[0] = __floats2bfloat162_rn(acc[a][0][0], acc[a][0][1]);
+            o2[1] = __floats2bfloat162_rn(acc[a][0][2], acc[a][1][0]);
+            o2[2] = __floats2bfloat162_rn(acc[a][1][1], acc[a][1][2]);
+            if (col1) {
+                o2[3] = __floats2bfloat162_rn(acc[a][2][0], acc[a][2][1]);
+                o2[4] = __floats2bfloat162_rn(acc[a][2][2], acc[a][3][0]);
+                o2[5] = __floats2bfloat162_rn(acc[a][3][1], acc[a][3][2]);
+            }
+        }
     }
 }
 
-// dw partials: block b accumulates dw over its pixel range; thread (cg, tap) owns dw[4*cg .. 4*cg+3][tap][0..2].
-// partial layout [gridDim.x][COUT][27].
+// ---- tensor-core weight gradient for the stem: dw[c'][k] = sum over pixels of dy[pixel][c'] * patch[pixel][k] as
+// mma.sync tiles of 16 pixels (the reduction index): A = dy^T (the 16 x COUT piece of dy is one contiguous run: staged in
+// shared memory with 16-byte loads and read back transposed with ldmatrix), B = the pixels' patch values (gathered like
+// in the forward kernel).  A block sums its pixel range; its four warps are combined in a fixed order into the block's
+// slice of `partial` [gridDim.x][COUT][27].
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
 template <int COUT>
-__global__ void __launch_bounds__(128) stem_wgrad_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
-                                                         float* __restrict__ partial, Geom g, long long pix_per_block) {
+__global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
+                                                             float* __restrict__ partial, Geom g, long long pix_per_block) {
     pdl_launch_dependents();
     pdl_wait();
-    constexpr int P = 32;  // pixels per staged chunk
-    constexpr int NCG = COUT / 4;
-    __shared__ __align__(16) float dys[P][COUT];
-    __shared__ float xs[P][STEM_KDIM + 1];
-    const int tid = threadIdx.x;
-    const int cg = tid / STEM_TAPS, tap = tid % STEM_TAPS;
-    const bool compute = tid < NCG * STEM_TAPS;
-    float acc[4][3];
+    static_assert(COUT % 16 == 0, "whole m-blocks");
+    constexpr int MB = COUT / 16, NBK = 4;  // accumulator blocks: MB x 16 channels by NBK x 8 filter positions (27 padded to 32)
+    __shared__ __align__(16) __nv_bfloat16 dys[4][16 * COUT];
+    __shared__ float red[4][COUT][33];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
+    const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
+    // B fragment element (k = pixel 2t.., n = 8*nb + g): filter position n of the pixel's patch
+    int koff[NBK], kr[NBK], kt[NBK];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int nb = 0; nb < NBK; ++nb) {
+        const int k = nb * 8 + gq, r = k / 9, kp = k - r * 9;
+        kr[nb] = r;
+        kt[nb] = kp / 3;
+        koff[nb] = k < STEM_KDIM ? r * g.w * 3 + kp : -1;
+    }
+    float acc[MB][NBK][4];
 #pragma unroll
-        for (int c = 0; c < 3; ++c) acc[a][c] = 0.f;
+    for (int a = 0; a < MB; ++a)
+#pragma unroll
+        for (int b = 0; b < NBK; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = acc[a][b][3] = 0.f;
     const long long m_begin = (long long)blockIdx.x * pix_per_block;
     const long long m_end = (m_begin + pix_per_block < g.m) ? m_begin + pix_per_block : g.m;
-    for (long long m0 = m_begin; m0 < m_end; m0 += P) {
-        const int np = (int)((m_end - m0 < P) ? (m_end - m0) : P);
-        // stage dy (COUT/8 vectors per pixel) and the 27 input values of every pixel
-        for (int e = tid; e < P * (COUT / 8); e += blockDim.x) {
-            const int pi = e / (COUT / 8), v = e % (COUT / 8);
-            if (pi < np) {
-                const Vec16<__nv_bfloat16> q = ld16(dy + (size_t)(m0 + pi) * COUT + v * 8);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) dys[pi][v * 8 + i] = __bfloat162float(q.v[i]);
+    __nv_bfloat16* st = dys[warp];
+    for (long long m0 = m_begin + warp * 16; m0 < m_end; m0 += 64) {
+        const int np = (int)((m_end - m0 < 16) ? (m_end - m0) : 16);  // pixels of this tile inside the block's range
+        // stage dy[m0 .. m0+15][:] (zeros past the range)
+        for (int v = lane; v < 16 * COUT / 8; v += 32) {
+            Vec16<__nv_bfloat16> q;
+            if (v * 8 < np * COUT) {
+                q = ld16(dy + (size_t)m0 * COUT + v * 8);
             } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) dys[pi][v * 8 + i] = 0.f;
+                for (int i = 0; i < 8; ++i) q.v[i] = __float2bfloat16_rn(0.f);
+            }
+            st16(st + v * 8, q);
+        }
+        // B fragments: four pixels of the tile (2t, 2t+1, 2t+8, 2t+9) x NBK filter positions
+        uint32_t bfr[NBK][2];
+        unsigned short v4[4][NBK];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int pl = tq * 2 + (j & 1) + (j >> 1) * 8;
+            const bool row_ok = pl < np;
+            const unsigned mm = row_ok ? (unsigned)(m0 + pl) : 0u;
+            const unsigned t1 = mm / (unsigned)g.wo;
+            const int q = (int)(mm - t1 * (unsigned)g.wo);
+            const int n = (int)(t1 / (unsigned)g.ho), p = (int)(t1 - (unsigned)n * (unsigned)g.ho);
+            const int h0 = 2 * p - 1, w0 = 2 * q - 1;
+            const long long origin = (((long long)n * g.h + h0) * g.w + w0) * 3;
+#pragma unroll
+            for (int nb = 0; nb < NBK; ++nb) {
+                const int h = h0 + kr[nb], ww = w0 + kt[nb];
+                const bool ok = row_ok && koff[nb] >= 0 && h >= 0 && h < g.h && ww >= 0 && ww < g.w;
+                v4[j][nb] = ok ? xs[origin + koff[nb]] : (unsigned short)0;
             }
         }
-        for (int e = tid; e < P * STEM_TAPS; e += blockDim.x) {
-            const int pi = e / STEM_TAPS, tp = e % STEM_TAPS;
-            float v0 = 0.f, v1 = 0.f, v2 = 0.f;
-            if (pi < np) {
-                const long long m = m0 + pi;
-                const int q = (int)(m % g.wo);
-                const long long t1 = m / g.wo;
-                const int p = (int)(t1 % g.ho), n = (int)(t1 / g.ho);
-                const int h = 2 * p - 1 + tp / 3, ww = 2 * q - 1 + tp % 3;
-                if (h >= 0 && h < g.h && ww >= 0 && ww < g.w) {
-                    const __nv_bfloat16* px = x + (((size_t)n * g.h + h) * g.w + ww) * 3;
-                    v0 = __bfloat162float(px[0]);
-                    v1 = __bfloat162float(px[1]);
-                    v2 = __bfloat162float(px[2]);
-                }
-            }
-            xs[pi][tp * 3] = v0;
-            xs[pi][tp * 3 + 1] = v1;
-            xs[pi][tp * 3 + 2] = v2;
+#pragma unroll
+        for (int nb = 0; nb < NBK; ++nb) {
+            bfr[nb][0] = (uint32_t)v4[0][nb] | ((uint32_t)v4[1][nb] << 16);
+            bfr[nb][1] = (uint32_t)v4[2][nb] | ((uint32_t)v4[3][nb] << 16);
         }
-        __syncthreads();
-        if (compute) {
-#pragma unroll 8
-            for (int pi = 0; pi < P; ++pi) {
-                const float4 d = *reinterpret_cast<const float4*>(&dys[pi][cg * 4]);
-                const float x0 = xs[pi][tap * 3], x1 = xs[pi][tap * 3 + 1], x2 = xs[pi][tap * 3 + 2];
-                acc[0][0] = fmaf(d.x, x0, acc[0][0]); acc[0][1] = fmaf(d.x, x1, acc[0][1]); acc[0][2] = fmaf(d.x, x2, acc[0][2]);
-                acc[1][0] = fmaf(d.y, x0, acc[1][0]); acc[1][1] = fmaf(d.y, x1, acc[1][1]); acc[1][2] = fmaf(d.y, x2, acc[1][2]);
-                acc[2][0] = fmaf(d.z, x0, acc[2][0]); acc[2][1] = fmaf(d.z, x1, acc[2][1]); acc[2][2] = fmaf(d.z, x2, acc[2][2]);
-                acc[3][0] = fmaf(d.w, x0, acc[3][0]); acc[3][1] = fmaf(d.w, x1, acc[3][1]); acc[3][2] = fmaf(d.w, x2, acc[3][2]);
-            }
+        __syncwarp();  // the staged dy rows are complete
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) {
+            // A = dy^T: matrix i of the x4 load is [8 pixels][8 channels] of the staged tile, read transposed:
+            // i = 0: pixels 0-7, channels 16mb+0..7 (a0), 1: pixels 0-7, channels +8 (a1), 2: pixels 8-15, channels +0 (a2), 3: pixels 8-15, +8 (a3)
+            uint32_t afr[4];
+            const int mi = lane >> 3, mr = lane & 7;
+            ldmatrix_x4_trans(afr, st + (mr + (mi >> 1) * 8) * COUT + mb * 16 + (mi & 1) * 8);
+#pragma unroll
+            for (int nb = 0; nb < NBK; ++nb) mma_bf16_16816(acc[mb][nb], afr, bfr[nb][0], bfr[nb][1]);
         }
-        __syncthreads();
+        __syncwarp();  // before the next tile overwrites the staged rows
     }
-    if (compute) {
-        float* o = partial + (size_t)blockIdx.x * COUT * STEM_KDIM;
+    // accumulator registers: c0, c1 = (channel 16mb+g, positions 8nb+2t, +1), c2, c3 = (channel 16mb+g+8, same positions)
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+    for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
-            for (int c = 0; c < 3; ++c) o[(size_t)(cg * 4 + a) * STEM_KDIM + tap * 3 + c] = acc[a][c];
+        for (int nb = 0; nb < NBK; ++nb) {
+            red[warp][mb * 16 + gq][nb * 8 + tq * 2] = acc[mb][nb][0];
+            red[warp][mb * 16 + gq][nb * 8 + tq * 2 + 1] = acc[mb][nb][1];
+            red[warp][mb * 16 + gq + 8][nb * 8 + tq * 2] = acc[mb][nb][2];
+            red[warp][mb * 16 + gq + 8][nb * 8 + tq * 2 + 1] = acc[mb][nb][3];
+        }
+    __syncthreads();
+    float* o = partial + (size_t)blockIdx.x * COUT * STEM_KDIM;
+    for (int e = threadIdx.x; e < COUT * STEM_KDIM; e += blockDim.x) {
+        const int c = e / STEM_KDIM, k = e - c * STEM_KDIM;
+        o[e] = ((red[0][c][k] + red[1][c][k]) + red[2][c][k]) + red[3][c][k];
     }
 }
 
