@@ -35,6 +35,19 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the 77 launches of a site in one step
+# of the cfg5 workload) from the ncu capture summarised in profiles/launch_list_cfg5_step.md (warm caches, as in a real
+# step: most layers' tensors stay in the 126 MB L2, so the traffic is well below the algorithmic bytes).
+NCU_DRAM_BYTES_PER_LAUNCH_CFG5 = {
+    "conv_fprop": (807 + 1283 + 39 + 654 + 641 + 149) * 1e6 / 77,
+    "conv_dgrad": (623 + 25 + 156 + 1169 + 505 + 52) * 1e6 / 77,
+    "conv_wgrad": (2237 + 185 + 1402 + 19) * 1e6 / 77,
+    "bn_silu_apply": (436 + 770) * 1e6 / 77,
+    "bn_silu_bwd_reduce": (1981 + 820) * 1e6 / 77,
+    "bn_silu_bwd_dy": (1107 + 880) * 1e6 / 77,
+}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -351,7 +364,9 @@ def main():
         else:
             roofline = {"kernel": top, "bound": "hbm", "achieved": a["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        roofline["traffic"] = None
+        roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH_CFG5.get(top) if args.workload == "cfg5" else None
+        roofline["traffic_note"] = ("bytes per launch, average of the site's launches in one step, from the committed ncu launch list "
+                                    "(profiles/launch_list_cfg5_step.md); algorithmic bytes per launch: %.3g" % (a["bytes"] / a["launches"]))
         roofline["peak_source"] = peaks["source"] + (" (burst figure: kernels timed one at a time)" if roofline["bound"] == "tensor" else "")
         roofline["avg_launch_ms"] = a["ms"] / a["launches"]
         roofline["share_of_step"] = a["ms"] / tot_ms
