@@ -217,6 +217,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg5", help="cfg1..cfg5 (cfg5 = the detector's 77 Conv-BN-SiLU layers at batch 16)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-streams", type=int, default=6, help="streams of the end-to-end arm (1 = no overlap of copies and compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
@@ -427,26 +428,54 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
         hin, hout = host[s.key]
         h2d += sum(t.numel() * t.element_size() for t in hin.values())
         d2h += sum(t.numel() * t.element_size() for t in hout.values())
-    # free the resident tensors of the device-timed arm before allocating the scratch
-    scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
+    # Three streams, each with its own device scratch, take the layers round-robin: while one layer computes, the next
+    # layer's inputs arrive over PCIe and the previous layer's results leave (the two copy directions run concurrently).
+    # Kernels of different layers may then share the GPU, so the plans of this arm are created with NB_CBS_FLAG_SHARED_GPU
+    # (separate finalize kernels instead of in-kernel grid barriers).
+    nstreams = max(1, args.e2e_streams)
+    plans = {}
+    for b in blocks:
+        if b.shape.key not in plans:
+            plans[b.shape.key] = nb.Plan.for_shape(b.shape, flags=flags | (nb.NB_CBS_FLAG_SHARED_GPU if nstreams > 1 else 0), device=local)
+    scratches = [torch.empty(scratch_bytes, dtype=torch.uint8, device=dev) for _ in range(nstreams)]
+    main = torch.cuda.current_stream()
+    streams = [main] if nstreams == 1 else [torch.cuda.Stream(device=dev) for _ in range(nstreams)]
 
     def one():
-        for b in blocks:
+        for i, b in enumerate(blocks):
             hin, hout = host[b.shape.key]
-            nb.nb_conv_bn_silu_step_host(b.plan, hin["x"], hin["w"], hin["gamma"], hin["beta"], hin["g"], hout["a"], hout["dx"],
-                                         hout["dw"], hout["dgamma"], hout["dbeta"], scratch)
+            k = i % nstreams
+            nb.nb_conv_bn_silu_step_host(plans[b.shape.key], hin["x"], hin["w"], hin["gamma"], hin["beta"], hin["g"], hout["a"], hout["dx"],
+                                         hout["dw"], hout["dgamma"], hout["dbeta"], scratches[k], stream=streams[k])
+
+    def fork():  # the side streams start after everything already queued on the main stream
+        if nstreams > 1:
+            e = torch.cuda.Event()
+            e.record(main)
+            for st in streams:
+                st.wait_event(e)
+
+    def join():  # the main stream continues after all side streams
+        if nstreams > 1:
+            for st in streams:
+                e = torch.cuda.Event()
+                e.record(st)
+                main.wait_event(e)
 
     steps = max(1, min(args.steps, 3))
+    fork()
     one()
+    join()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
+    ev0.record(main)
+    fork()
     for _ in range(steps):
         one()
-    ev1.record(stream)
+    join()
+    ev1.record(main)
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1)
     if dist is not None:
@@ -454,7 +483,7 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     return {"value": world * flops / (ms / steps * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "ms_per_step": ms / steps, "steps": steps}
+            "ms_per_step": ms / steps, "steps": steps, "streams": nstreams}
 
 
 if __name__ == "__main__":
