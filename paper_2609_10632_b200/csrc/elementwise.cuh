@@ -173,6 +173,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
     load_params<V>(shift, cg, sh);
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+        if (v + 2 * stride < total_vecs) asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));  // see the reduce kernel
         const Vec16<YT> q = ld16(y + v * V);
         Vec16<AT> o;
 #pragma unroll
@@ -265,6 +266,12 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
     }
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + tid; v < total_vecs; v += stride) {
+        // ask L2 for the lines this thread reads two iterations from now: more DRAM requests in flight without holding
+        // registers (measured on 157 MB tensors: 93 -> 79 us; no effect on tensors that already sit in L2)
+        if (v + 2 * stride < total_vecs) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + (v + 2 * stride) * V));
+        }
         const Vec16<YT> qy = ld16(y + v * V);
         const Vec16<AT> qg = ld16(g + v * V);
 #pragma unroll
@@ -356,6 +363,10 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
     load_params<V>(coef + 3 * C, cg, p0);
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+        if (v + 2 * stride < total_vecs) {  // L2 prefetch two iterations ahead (see the reduce kernel)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + (v + 2 * stride) * V));
+        }
         const Vec16<YT> qy = ld16(y + v * V);
         const Vec16<AT> qg = ld16(g + v * V);
         Vec16<AT> o;

@@ -603,7 +603,7 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
         }
         const size_t elems = (size_t)p->g.c_out * p->g.kdim;
         SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
-        launch_k(splitk_reduce_kernel, dim3((unsigned)((elems + 255) / 256)), dim3(256), 0, st, 1, partial, p->stem_blocks, elems, dw);
+        launch_k(splitk_reduce_tall_kernel, dim3((unsigned)((elems + 31) / 32)), dim3(1024), 0, st, 1, partial, p->stem_blocks, elems, dw);
         return launch_ok("splitk_reduce");
     }
     if (p->tc.wgrad) {

@@ -194,4 +194,33 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     }
 }
 
+// The same sum for many slices of few elements (the first layer's weight gradient: ~1200 slices of 1296 values): a block of
+// 32 x 32 threads takes 32 consecutive elements; thread (e, zg) adds slices zg, zg + 32, ... in that order in fp64 (coalesced
+// 128-byte rows, eight loads in flight), and the 32 partial sums of an element are combined in the order of zg.
+__global__ void __launch_bounds__(1024) splitk_reduce_tall_kernel(const float* __restrict__ partial, int splits, size_t elems, float* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ double red[32][33];
+    const int ex = threadIdx.x & 31, zg = threadIdx.x >> 5;
+    const size_t e = (size_t)blockIdx.x * 32 + ex;
+    double acc = 0.0;
+    if (e < elems) {
+        for (int z0 = zg; z0 < splits; z0 += 256) {
+            float a[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] = z0 + 32 * u < splits ? partial[(size_t)(z0 + 32 * u) * elems + e] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += (double)a[u];
+        }
+    }
+    red[zg][ex] = acc;
+    __syncthreads();
+    if (zg == 0 && e < elems) {
+        double s = 0.0;
+#pragma unroll 8
+        for (int k = 0; k < 32; ++k) s += red[k][ex];
+        out[e] = (float)s;
+    }
+}
+
 }  // namespace nbcbs
