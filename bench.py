@@ -48,6 +48,35 @@ NCU_DRAM_BYTES_PER_LAUNCH_CFG5 = {
 }
 
 
+def write_per_layer(path, blocks, per_shape, peaks):
+    """Markdown table: per distinct layer shape, the instrumented device time of each kernel site per launch and what it
+    means against the measured peaks (the times include a few microseconds of launch latency per kernel)."""
+    counts = {}
+    for b in blocks:
+        counts[b.shape.key] = counts.get(b.shape.key, 0) + 1
+    lines = ["| layer shape (Cin, Cout, k, stride, H) | layers | fprop us (TFLOP/s, % of peak) | dgrad us | wgrad+reduce us | apply us (GB/s) | bwd reduce us (GB/s) | dy us (GB/s) |",
+             "|---|---|---|---|---|---|---|---|"]
+    for key, rec in per_shape.items():
+        s, st = rec["shape"], rec["sites"]
+        us = lambda site: (st[site][0] / st[site][1] * 1e3) if site in st else 0.0
+        def gemm(site, extra=None):
+            t = us(site) + (us(extra) if extra else 0.0)
+            if t <= 0:
+                return "-"
+            tf = s.gemm_flops / (t * 1e-6) / 1e12
+            return "%.1f (%.0f, %.0f %%)" % (t, tf, 100.0 * tf / peaks["bf16_tflops"])
+        def ew(site):
+            t = us(site)
+            if t <= 0:
+                return "-"
+            return "%.1f (%.0f)" % (t, site_work(site, s)[1] / (t * 1e-6) / 1e9)
+        lines.append("| (%d, %d, %d, %d, %d) | %d | %s | %s | %s | %s | %s | %s |" % (
+            s.c_in, s.c_out, s.k, s.stride, s.h, counts[key], gemm("conv_fprop"), gemm("conv_dgrad"), gemm("conv_wgrad", "wgrad_splitk_reduce"),
+            ew("bn_silu_apply"), ew("bn_silu_bwd_reduce"), ew("bn_silu_bwd_dy")))
+    with open(path, "w") as f:
+        f.write("\n".join(lines) + "\n")
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -216,6 +245,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg5", help="cfg1..cfg5 (cfg5 = the detector's 77 Conv-BN-SiLU layers at batch 16)")
+    ap.add_argument("--per-layer", default=None, help="write a per-layer-shape table of the instrumented kernel times to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=6, help="streams of the end-to-end arm (1 = no overlap of copies and compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -329,10 +359,14 @@ def main():
             one_step()
         torch.cuda.synchronize()
         agg = {}
+        per_shape = {}  # distinct layer shape -> site -> [ms, launches]
         for b in blocks:
             for site, (ms, n) in nb.nb_cbs_profile_read(b.plan).items():
                 if n == 0:
                     continue
+                ps = per_shape.setdefault(b.shape.key, {"shape": b.shape, "count": 0, "sites": {}})["sites"].setdefault(site, [0.0, 0])
+                ps[0] += ms
+                ps[1] += n
                 f, by = site_work(site, b.shape)
                 a = agg.setdefault(site, {"ms": 0.0, "launches": 0, "flops": 0.0, "bytes": 0.0})
                 a["ms"] += ms
@@ -342,6 +376,8 @@ def main():
             nb.nb_cbs_profile_enable(b.plan, False)
         tot_ms = sum(a["ms"] for a in agg.values()) or 1.0
         tensor_sites = {"conv_fprop", "conv_dgrad", "conv_wgrad"}
+        if args.per_layer and rank == 0:
+            write_per_layer(args.per_layer, blocks, per_shape, peaks)
         for site, a in agg.items():
             sec = a["ms"] * 1e-3
             k = {"launches": a["launches"], "ms_per_step": a["ms"] / prof_steps, "share": a["ms"] / tot_ms}
