@@ -237,6 +237,23 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The step time of a multi-process run is the slowest rank's (replicas only: no data-path collective, the only
+    communication of the benchmark is this reduction and the barriers around the timed region)."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, flops_per_replica: float, ms_step: float) -> float:
+    """TFLOP/s of all replicas together: every rank does the same work (weak scaling) in the slowest rank's time."""
+    return world * flops_per_replica / (ms_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -341,12 +358,9 @@ def main():
     for b in blocks:
         b.poll()
     ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
     ms_step = ms_total / args.steps
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(world, flops, ms_step)
     peaks = load_peaks()
 
     # ---------------- instrumented pass: per-site device times (events around every launch; calls wait for each kernel)
@@ -514,11 +528,8 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
     ev1.record(main)
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return {"value": world * flops / (ms / steps * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+    ms = max_over_ranks(ms, dist, dev)
+    return {"value": whole_job_value(world, flops, ms / steps), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "ms_per_step": ms / steps, "steps": steps, "streams": nstreams}
 
 
