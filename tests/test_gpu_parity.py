@@ -99,6 +99,29 @@ def test_separate_finalize_kernels_match_oracle(shape):
     _compare(out, _oracle(inp), 0)
 
 
+def test_two_plans_on_two_streams_with_the_shared_gpu_flag():
+    """Calls of different plans may overlap on the GPU when both plans carry NB_CBS_FLAG_SHARED_GPU (no grid barriers)."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    shapes = [SMALL_SHAPES[7], SMALL_SHAPES[9]]
+    inps = [wl.make_inputs(s, 16, i, bf16=True, affine="random") for i, s in enumerate(shapes)]
+    blks = [CbsBlock(s, eps=EPS, flags=nb.NB_CBS_FLAG_SHARED_GPU) for s in shapes]
+    for b, inp in zip(blks, inps):
+        b.upload(inp)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in blks]
+    for _ in range(3):  # interleave the launches of the two plans
+        for b, st in zip(blks, streams):
+            b.step(stream=st)
+    torch.cuda.synchronize()
+    for b, inp in zip(blks, inps):
+        b.poll()
+        _compare(b.download(), _oracle(inp), 0)
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[11], S(3, 9, 11, 32, 16, 3, 1), S(2, 24, 24, 96, 192, 3, 1)],
                          ids=lambda s: s.name)
 def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
