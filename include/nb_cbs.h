@@ -25,8 +25,10 @@
  * Every pointer is a DEVICE pointer on the plan's device unless its name starts with `host_`; the
  * caller owns all memory, including the workspace.  Tensor pointers must be 16-byte aligned.
  * Compute calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
- * and return without synchronising.  Outputs are overwritten, never accumulated into.  Calls on one
- * plan must not run concurrently (they share the plan's status block and the workspace).
+ * and return without synchronising; they make the plan's device current while they run and restore the
+ * caller's current device before returning (`stream` must belong to the plan's device).  Outputs are
+ * overwritten, never accumulated into.  Calls on one plan must not run concurrently, neither on the host
+ * (they share the plan's cached tensor maps) nor on the device (its status block and the workspace).
  * On invalid arguments nothing is launched and a non-zero status is returned; nb_last_error()
  * then describes the problem.
  */

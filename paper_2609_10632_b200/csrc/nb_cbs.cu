@@ -123,6 +123,18 @@ struct SiteTimer {
     }
 };
 
+// Makes the plan's device current for the duration of a compute call and restores the caller's device afterwards.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int device) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != device) switched = cudaSetDevice(device) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
 nb_status launch_ok(const char* what) {
     g_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t e = cudaGetLastError();
@@ -484,6 +496,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     if ((running_mean == nullptr) != (running_var == nullptr))
         return fail(NB_ERR_INVALID_ARG, "running_mean and running_var must both be given or both be NULL");
     NB_TRY(check_ws(workspace, workspace_bytes, p->fwd_bytes));
+    DeviceGuard on_device(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
@@ -533,6 +546,7 @@ nb_status nb_bn_stats(nb_cbs_plan p, const void* y, int32_t y_dtype, float* mean
     const int want = is_f32(p) ? NB_DTYPE_F32 : NB_DTYPE_F16;
     if (y_dtype != want) return fail(NB_ERR_UNSUPPORTED, "y_dtype %d does not match the plan's mode (expected %d)", y_dtype, want);
     NB_TRY(check_ws(workspace, workspace_bytes, p->fwd_bytes));
+    DeviceGuard on_device(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* part = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_fpart);
     if (is_f32(p)) NB_TRY(run_stats_partial<float>(p, y, part, st));
@@ -550,6 +564,7 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     NB_CHECK_PTR(dx, true);
     if (dx) NB_CHECK_PTR(w);
     NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
+    DeviceGuard on_device(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     float* coef = reinterpret_cast<float*>(ws + p->off_coef);
@@ -590,6 +605,7 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(dy); NB_CHECK_PTR(dw);
     NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
+    DeviceGuard on_device(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + p->off_wgpart);
     if (is_f32(p)) return run_simt_wgrad<float>(p, x, dy, dw, partial, st);
@@ -738,6 +754,7 @@ nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const voi
         return fail(NB_ERR_INVALID_ARG, "a required host pointer is NULL");
     const StepLayout L = step_layout(p);
     NB_TRY(check_ws(device_scratch, scratch_bytes, L.total));
+    DeviceGuard on_device(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* d = static_cast<char*>(device_scratch);
     const size_t cb = (size_t)p->g.c_out * 4;

@@ -5,6 +5,7 @@
 // for the batch statistics and writes coalesced rows.  The same kernel computes fprop (A = x, B = w) and dgrad
 // (A = dy, B = the filter rearranged per output-parity class).  No multicast anywhere; every wait is bounded.
 #pragma once
+#include <atomic>
 #include <cuda.h>
 
 #include <algorithm>
@@ -1320,13 +1321,17 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
 }
 
 template <typename OutT, bool STATS, bool CG2, bool HALO> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the (function, device) pair: one bit per device ordinal that already has it
+    static std::atomic<unsigned long long> attr_set{0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(attr_set.load(std::memory_order_acquire) & bit)) {
         if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
-        attr_set = true;
+        attr_set.fetch_or(bit, std::memory_order_release);
     }
     const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
@@ -1621,13 +1626,16 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
     }
     P.out = P.splits > 1 ? partial : dw;
     P.status = status;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static std::atomic<unsigned long long> attr_set{0};  // one bit per device ordinal (see launch_igemm_impl)
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(attr_set.load(std::memory_order_acquire) & bit)) {
         if (cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the wgrad kernel";
             return NB_ERR_CUDA;
         }
-        attr_set = true;
+        attr_set.fetch_or(bit, std::memory_order_release);
     }
     launch_k(tc_wgrad_kernel, dim3(tc->wg_grid), dim3(TC_THREADS), tc->wg_smem, st, 1, P);
     cudaError_t e = cudaGetLastError();
