@@ -292,6 +292,15 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
+    // the tensor maps live in the kernel's parameters: their fetch can run while this kernel still waits for its predecessor
+    if (lane == 0) {
+        if (warp == 0) ptx::prefetch_tmap(&p.tmA);
+        if (warp == 6)
+            for (int c = 0; c < p.nclasses; ++c) ptx::prefetch_tmap(&p.tmB[c]);
+        if (warp == 2 && p.tma_store)
+            for (int i = 0; i < 3; ++i)
+                if (p.out_w[i]) ptx::prefetch_tmap(&p.tmOut[i]);
+    }
     if (STATS) {
         for (int c = threadIdx.x; c < 8 * p.ldo; c += IG_THREADS) wstat[c] = 0.f;
     }
@@ -317,7 +326,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         if (HALO) {
             {
                 const bool isA = warp == 0;
-                if (leader) ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB[0]);
                 const int n_tiles = p.n_tiles, cbs = p.kc_per_tap, bn_own = p.BN / 2;
                 bool ok = true;
                 int issued = 0;
@@ -411,13 +419,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             }
         } else {
             const bool isA = warp == 0;
-            if (leader) {
-                if (isA) {
-                    ptx::prefetch_tmap(&p.tmA);
-                } else {
-                    for (int c = 0; c < p.nclasses; ++c) ptx::prefetch_tmap(&p.tmB[c]);
-                }
-            }
             int s = 0;
             uint32_t ph = 0;
             long long issued = 0;
@@ -954,7 +955,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 acc_ph ^= 1u;
             }
         }
-        if (store_pending && lane == 0) ptx::tma_store_wait_all<0>();  // the stores are complete before the kernel ends
+        // the staging rows must have been read before this CTA's shared memory is released; the writes themselves are
+        // complete when the grid is (a kernel boundary orders them like any other store)
+        if (store_pending && lane == 0) ptx::tma_store_wait_read<0>();
         if (STATS) {
             epi2_bar_sync();  // all eight warps' running sums are final
             // channel c of the layer sits in team (c % BN >= ncol_a) at index (c / BN) * (team's columns) + its column there

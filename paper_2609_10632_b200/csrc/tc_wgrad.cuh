@@ -64,6 +64,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
+    if (lane == 0 && (warp == 0 || warp == 6)) ptx::prefetch_tmap(warp == 0 ? &p.tmA : &p.tmB);  // before the wait for the predecessor
     if (warp == 1) {
         ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
         ptx::tmem_relinquish();
@@ -80,7 +81,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         const uint32_t leader = ptx::elect_one() ? 1u : 0u;
         if (nchunks > 0) {
             const bool isA = warp == 0;
-            if (leader) ptx::prefetch_tmap(isA ? &p.tmA : &p.tmB);
             int s = 0, issued = 0;
             uint32_t ph = 0;
             bool ok = true;
