@@ -269,6 +269,7 @@ def main():
     ap.add_argument("--no-profile", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--force-simt", action="store_true", help="run the convolutions on the CUDA-core kernels")
+    ap.add_argument("--no-wgrad-stream", action="store_true", help="queue the weight gradients on the main stream instead of a second stream")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph of one step")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -308,9 +309,21 @@ def main():
     flops = step_flops(layers)
     stream = torch.cuda.current_stream()
 
+    # The weight gradient of a layer depends only on dy and x, so it goes to a second stream (with a workspace of its
+    # own) and overlaps the kernels that follow on the main stream; the step ends when both streams have finished.
+    wgrad_stream = None if args.no_wgrad_stream else torch.cuda.Stream(device=dev)
+    wgrad_ws = None if args.no_wgrad_stream else torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
     def one_step():
+        if wgrad_stream is None:
+            for b in blocks:
+                b.step()
+            return
+        main = torch.cuda.current_stream()
+        wgrad_stream.wait_stream(main)
         for b in blocks:
-            b.step()
+            b.step(wgrad_stream=wgrad_stream, wgrad_workspace=wgrad_ws)
+        main.wait_stream(wgrad_stream)
 
     def barrier():
         if dist is not None:
@@ -444,7 +457,7 @@ def main():
                 "workload": f"{args.workload}: {len(layers)} Conv-BN-SiLU layers, batch {layers[0].n}, fwd + bwd_data + bwd_weight per layer "
                             f"(stem data gradient included), each layer on its own tensors",
                 "l2_policy": f"inputs larger than L2: {resident / 1e9:.2f} GB of tensors are touched per step",
-                "gflop_per_step": flops / 1e9, "multi_gpu": "replicas only", "cuda_graph": graph is not None, "tensor_core_layers": paths, "layers": len(layers),
+                "gflop_per_step": flops / 1e9, "multi_gpu": "replicas only", "cuda_graph": graph is not None, "wgrad_on_second_stream": wgrad_stream is not None, "tensor_core_layers": paths, "layers": len(layers),
                 "frac_of_nominal_bf16_peak": value / world / NOMINAL["bf16_tflops"],
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },

@@ -29,6 +29,9 @@
  * caller's current device before returning (`stream` must belong to the plan's device).  Outputs are
  * overwritten, never accumulated into.  Calls on one plan must not run concurrently, neither on the host
  * (they share the plan's cached tensor maps) nor on the device (its status block and the workspace).
+ * One exception on the device: nb_conv_bn_silu_bwd_weight uses no grid barrier and of the status block only
+ * its atomic error words, so on a stream of its own, with a workspace of its own and ordered after the call
+ * that produced dy, it may overlap any other call of this or another plan (default flags included).
  * On invalid arguments nothing is launched and a non-zero status is returned; nb_last_error()
  * then describes the problem.
  */

@@ -74,13 +74,23 @@ class CbsBlock:
         nb.nb_conv_bn_silu_bwd_data(self.plan, self.g, self.y, self.mean, self.invstd, self.gamma, self.beta, self.w, self.dx,
                                     self.dgamma, self.dbeta, self.dy, self.ws, stream)
 
-    def backward_weight(self, stream=None):
-        nb.nb_conv_bn_silu_bwd_weight(self.plan, self.x, self.dy, self.dw, self.ws, stream)
+    def backward_weight(self, stream=None, workspace=None):
+        nb.nb_conv_bn_silu_bwd_weight(self.plan, self.x, self.dy, self.dw, self.ws if workspace is None else workspace, stream)
 
-    def step(self, stream=None):
+    def step(self, stream=None, wgrad_stream=None, wgrad_workspace=None):
+        """Forward, data gradient, weight gradient.  With `wgrad_stream` (and a workspace of its own) the weight gradient
+        is queued on that stream behind an event that follows the data-gradient call, so it overlaps whatever the caller
+        queues next on `stream`; the caller joins the two streams."""
         self.forward(stream)
         self.backward_data(stream)
-        self.backward_weight(stream)
+        if wgrad_stream is None:
+            self.backward_weight(stream)
+            return
+        assert wgrad_workspace is not None and wgrad_workspace.numel() >= self.plan.bwd_bytes
+        ev = torch.cuda.Event()
+        ev.record(torch.cuda.current_stream(self.dev) if stream is None else stream)
+        wgrad_stream.wait_event(ev)
+        self.backward_weight(wgrad_stream, wgrad_workspace)
 
     def poll(self):
         return nb.nb_cbs_poll_status(self.plan)

@@ -122,6 +122,37 @@ def test_two_plans_on_two_streams_with_the_shared_gpu_flag():
         _compare(b.download(), _oracle(inp), 0)
 
 
+def test_weight_gradient_on_a_second_stream_overlaps_the_next_layers():
+    """The step bench.py times: each layer's weight gradient runs on a second stream with a workspace of its own while
+    the main stream goes on with the next layer (default plans: the grid-barrier kernels stay on the main stream)."""
+    import torch
+
+    from paper_2609_10632_b200.block import CbsBlock
+
+    shapes = [SMALL_SHAPES[7], SMALL_SHAPES[9], SMALL_SHAPES[11], SMALL_SHAPES[0]]
+    inps = [wl.make_inputs(s, 17, i, bf16=True, affine="random") for i, s in enumerate(shapes)]
+    need = 0
+    blks = []
+    for s in shapes:
+        blks.append(CbsBlock(s, eps=EPS))
+        need = max(need, blks[-1].plan.bwd_bytes)
+    for b, inp in zip(blks, inps):
+        b.upload(inp)
+    side_ws = torch.empty(need, dtype=torch.uint8, device=blks[0].dev)
+    side = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        side.wait_stream(main)
+        for b in blks:
+            b.step(wgrad_stream=side, wgrad_workspace=side_ws)
+        main.wait_stream(side)
+    torch.cuda.synchronize()
+    for b, inp in zip(blks, inps):
+        b.poll()
+        _compare(b.download(), _oracle(inp), 0)
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[11], S(3, 9, 11, 32, 16, 3, 1), S(2, 24, 24, 96, 192, 3, 1)],
                          ids=lambda s: s.name)
 def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
