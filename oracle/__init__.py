@@ -52,6 +52,13 @@ def _load():
         lib.oracle_bn_silu_fwd.restype = None
         lib.oracle_bn_silu_bwd.argtypes = [dp, dp, ctypes.c_longlong, ci, dp, dp, dp, dp, dp, dp, dp]
         lib.oracle_bn_silu_bwd.restype = None
+        dbl = ctypes.c_double
+        lib.oracle_bn_eval_act.argtypes = [dp, ctypes.c_longlong, ci, dp, dp, dp, dp, dbl, ci, dp]
+        lib.oracle_bn_eval_act.restype = None
+        lib.oracle_bias_act.argtypes = [dp, ctypes.c_longlong, ci, dp, ci, dp]
+        lib.oracle_bias_act.restype = None
+        lib.oracle_bn_fold.argtypes = [dp, ci, ctypes.c_longlong, dp, dp, dp, dp, dbl, dp, dp]
+        lib.oracle_bn_fold.restype = None
         lib.oracle_out_extent.argtypes = [ci, ci, ci]
         lib.oracle_out_extent.restype = ci
         lib.oracle_num_threads.argtypes = []
@@ -170,3 +177,42 @@ def cbs_fwd_bwd(x, w, gamma, beta, g, stride: int, eps: float, need_dx: bool = T
         res.dx = conv_dgrad(res.dy, w, np.shape(x), stride)
     res.dw = conv_wgrad(x, res.dy, k, stride)
     return res
+
+
+# ------------------------------------------------------------------ evaluation-mode and plain variants
+def bn_eval_act(y, gamma, beta, running_mean, running_var, eps: float, act: bool = True):
+    """Evaluation-mode BN (running statistics, Table 2 row 9) then SiLU when `act`."""
+    y = _f64(y)
+    C = y.shape[-1]
+    a = np.empty_like(y)
+    _load().oracle_bn_eval_act(_p(y), y.size // C, C, _p(_f64(gamma)), _p(_f64(beta)), _p(_f64(running_mean)), _p(_f64(running_var)),
+                               float(eps), int(bool(act)), _p(a))
+    return a
+
+
+def bias_act(y, bias, act: bool):
+    y = _f64(y)
+    C = y.shape[-1]
+    out = np.empty_like(y)
+    _load().oracle_bias_act(_p(y), y.size // C, C, _p(_f64(bias)) if bias is not None else None, int(bool(act)), _p(out))
+    return out
+
+
+def bn_fold(w, gamma, beta, running_mean, running_var, eps: float):
+    """Filter and bias of the convolution that equals conv -> evaluation-mode BN."""
+    w = _f64(w)
+    Cout = w.shape[0]
+    wf, bf = np.empty_like(w), np.empty(Cout, dtype=np.float64)
+    _load().oracle_bn_fold(_p(w), Cout, w.size // Cout, _p(_f64(gamma)), _p(_f64(beta)), _p(_f64(running_mean)), _p(_f64(running_var)),
+                           float(eps), _p(wf), _p(bf))
+    return wf, bf
+
+
+def cbs_infer(x, w, gamma, beta, running_mean, running_var, stride: int, eps: float, act: bool = True):
+    """Evaluation-mode block from (x, w, gamma, beta, running statistics): conv -> BN(running) -> SiLU."""
+    return bn_eval_act(conv_fwd(x, w, stride), gamma, beta, running_mean, running_var, eps, act)
+
+
+def conv_bias_act(x, w, bias, stride: int, act: bool = False):
+    """Convolution with a per-channel bias and no normalisation (the head's output layers, Table 2 row 3)."""
+    return bias_act(conv_fwd(x, w, stride), bias, act)

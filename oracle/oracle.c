@@ -18,7 +18,11 @@
  * all-ones closed form; brute-force re-derivation on tiny tensors; adjoint identities
  * <conv(x,w),g> = <x,dgrad(g,w)> = <w,wgrad(x,g)>; BN zero-mean / mean(xhat^2) = 1-eps*invstd^2;
  * SiLU closed-form values; central finite differences of the whole block; sum(dy)=0 and
- * sum(dy*xhat) = gamma*dgamma*eps*invstd^3 per channel.  No function here is "parity unpinned".
+ * sum(dy*xhat) = gamma*dgamma*eps*invstd^3 per channel.  Evaluation-mode and plain variants (end of
+ * the file): a hand-worked value; running statistics set to the batch statistics reproduce the
+ * training-mode forward; gamma = 0 and huge-variance limits; conv + bias against a library
+ * correlation; folded filter + bias reproduces the unfolded evaluation-mode block.
+ * No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stddef.h>
@@ -208,4 +212,51 @@ void oracle_bn_silu_bwd(const double* g, const double* y, long long M, int C,
             const double dz = g[(size_t)i * C + c] * s * (1.0 + z * (1.0 - s));
             dy[(size_t)i * C + c] = gamma[c] * invstd[c] * (dz - dbeta[c] / (double)M - xhat * dgamma[c] / (double)M);
         }
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Evaluation-mode and plain variants (the paper's Table 2 row 9 fix: validation must normalise
+ * with the running statistics, not with batch statistics; Table 2 row 3: the detection head's
+ * output convolutions carry a bias and no normalisation).
+ * ------------------------------------------------------------------------------------------- */
+
+/* Evaluation-mode BN then optional SiLU: the stored running mean and running variance take the
+ * place of the batch statistics; nothing is updated.
+ *   z = gamma*(y - rmean)/sqrt(rvar + eps) + beta ;  a = act ? z*sigmoid(z) : z. */
+void oracle_bn_eval_act(const double* y, long long M, int C,
+                        const double* gamma, const double* beta, const double* rmean, const double* rvar,
+                        double eps, int act, double* a)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < M; ++i)
+        for (int c = 0; c < C; ++c) {
+            const double xhat = (y[(size_t)i * C + c] - rmean[c]) / sqrt(rvar[c] + eps);
+            const double z = gamma[c] * xhat + beta[c];
+            a[(size_t)i * C + c] = act ? z * sigmoid(z) : z;
+        }
+}
+
+/* Per-channel bias then optional SiLU:  z = y + bias[c] ;  out = act ? z*sigmoid(z) : z.  bias may be NULL (zero). */
+void oracle_bias_act(const double* y, long long M, int C, const double* bias, int act, double* out)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < M; ++i)
+        for (int c = 0; c < C; ++c) {
+            const double z = y[(size_t)i * C + c] + (bias ? bias[c] : 0.0);
+            out[(size_t)i * C + c] = act ? z * sigmoid(z) : z;
+        }
+}
+
+/* Folding evaluation-mode BN into the convolution that feeds it: with s_c = gamma_c/sqrt(rvar_c + eps),
+ *   w'[c',r,t,c] = s_c' * w[c',r,t,c] ;  bias'[c'] = beta_c' - rmean_c' * s_c',
+ * so that conv(x, w') + bias' equals the BN output for every x.  K = k*k*Cin filter taps per output channel. */
+void oracle_bn_fold(const double* w, int Cout, long long K,
+                    const double* gamma, const double* beta, const double* rmean, const double* rvar, double eps,
+                    double* w_folded, double* bias_folded)
+{
+    for (int co = 0; co < Cout; ++co) {
+        const double s = gamma[co] / sqrt(rvar[co] + eps);
+        for (long long t = 0; t < K; ++t) w_folded[(size_t)co * K + t] = s * w[(size_t)co * K + t];
+        bias_folded[co] = beta[co] - rmean[co] * s;
+    }
 }
