@@ -45,7 +45,7 @@
 extern "C" {
 #endif
 
-#define NB_CBS_ABI_VERSION 1u
+#define NB_CBS_ABI_VERSION 2u /* 2: adds the evaluation-mode / plain calls (additive) */
 
 typedef int32_t nb_status;
 enum {
@@ -168,6 +168,38 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan plan, const void* g, const void* 
  * dy is the tensor nb_conv_bn_silu_bwd_data wrote to dy_out (ordering on the stream is the caller's). */
 nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan plan, const void* x, const void* dy, float* dw, void* workspace,
                                      size_t workspace_bytes, void* stream);
+
+/* ---- Evaluation-mode and plain variants of the block (inference; nothing is saved, nothing is updated) ----
+ * The paper's reproduction protocol found that validation must normalise with the RUNNING statistics (Table 2 row 9),
+ * and its detector's head ends in convolutions that carry a bias and no normalisation (Table 2 row 3).
+ *
+ * Workspace size of the three calls below and whether they run as ONE kernel: `*fused` (may be NULL) is 1 when the
+ * convolution runs on the tensor-core kernel with the per-channel scale/shift and the activation applied to the fp32
+ * accumulators in its epilogue (BF16 mode, c_in % 16 == 0, c_out % 16 == 0); 0 when the plan falls back to
+ * convolution -> coefficient kernel -> elementwise pass, whose workspace also holds the convolution output. */
+nb_status nb_cbs_infer_workspace_bytes(nb_cbs_plan plan, size_t* bytes, int32_t* fused);
+
+/* Evaluation-mode forward:
+ *   y = conv(x, w) as in nb_conv_bn_silu_fwd
+ *   z = gamma_c * (y - running_mean_c) / sqrt(running_var_c + eps) + beta_c ;  a = z * sigmoid(z)  -> a_out
+ * The per-channel scale gamma/sqrt(var+eps) and shift beta - mean*scale are formed in fp64 and applied in fp32.
+ * Layouts and dtypes as in the training forward (a_out bf16 in BF16 mode, fp32 in F32 mode). */
+nb_status nb_conv_bn_silu_infer(nb_cbs_plan plan, const void* x, const void* w, const float* gamma, const float* beta,
+                                const float* running_mean, const float* running_var, void* a_out, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
+/* Convolution with a per-channel bias and no normalisation:
+ *   z = conv(x, w) + bias_c (bias may be NULL: zero) ;  out = act ? z * sigmoid(z) : z     (act: 0 = none, 1 = SiLU)
+ * With the outputs of nb_bn_fold as (w, bias) and act = 1 this is the evaluation-mode block with BN folded away. */
+nb_status nb_conv_bias_act(nb_cbs_plan plan, const void* x, const void* w, const float* bias, int32_t act, void* out,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Fold evaluation-mode BN into the filter that feeds it: with s_c' = gamma_c' / sqrt(running_var_c' + eps),
+ *   w_folded[c',r,t,c] = s_c' * w[c',r,t,c]   (the plan's activation dtype, rounded once)
+ *   bias_folded[c']    = beta_c' - running_mean_c' * s_c'                                   (fp32)
+ * No workspace.  w_folded may not alias w. */
+nb_status nb_bn_fold(nb_cbs_plan plan, const void* w, const float* gamma, const float* beta, const float* running_mean,
+                     const float* running_var, void* w_folded, float* bias_folded, void* stream);
 
 /* Batch statistics for callers that cannot allocate device memory.  (The paper has no counterpart of this entry
  * point.)  Some hosts of this library must not call cudaMalloc -- code running under a framework's caching allocator

@@ -26,7 +26,8 @@ EXPORTS = (
     "nb_cbs_workspace_bytes", "nb_cbs_plan_paths", "nb_cbs_poll_status", "nb_conv_bn_silu_fwd", "nb_bn_stats",
     "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
-    "nb_cbs_profile_read", "nb_bn_stats_static",
+    "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
+    "nb_bn_fold",
 )
 
 
@@ -72,6 +73,10 @@ def load() -> ctypes.CDLL:
         lib.nb_cbs_step_host_scratch_bytes.argtypes = [V, POINTER(c_size_t)]
         lib.nb_conv_bn_silu_step_host.argtypes = [V, V, V, FP, FP, V, V, V, FP, FP, FP, V, c_size_t, V]
         lib.nb_bn_stats_static.argtypes = [V, c_int32, ctypes.c_int64, c_int32, c_float, FP, FP, FP, FP, V]
+        lib.nb_cbs_infer_workspace_bytes.argtypes = [V, POINTER(c_size_t), POINTER(c_int32)]
+        lib.nb_conv_bn_silu_infer.argtypes = [V, V, V, FP, FP, FP, FP, V, V, c_size_t, V]
+        lib.nb_conv_bias_act.argtypes = [V, V, V, FP, c_int32, V, V, c_size_t, V]
+        lib.nb_bn_fold.argtypes = [V, V, FP, FP, FP, FP, V, FP, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -144,6 +149,9 @@ class Plan:
         p3 = (c_int32 * 3)()
         _check(load().nb_cbs_plan_paths(self.handle, p3))
         self.paths = {"fprop": p3[0], "dgrad": p3[1], "wgrad": p3[2]}
+        ib, fused = c_size_t(), c_int32()
+        _check(load().nb_cbs_infer_workspace_bytes(self.handle, byref(ib), byref(fused)))
+        self.infer_bytes, self.infer_fused = ib.value, bool(fused.value)
 
     @classmethod
     def for_shape(cls, s, **kw):
@@ -224,6 +232,21 @@ def nb_conv_bn_silu_bwd_data(plan: Plan, g, y_saved, save_mean, save_invstd, gam
 def nb_conv_bn_silu_bwd_weight(plan: Plan, x, dy, dw, workspace, stream=None):
     _check(load().nb_conv_bn_silu_bwd_weight(plan.handle, _ptr(x), _ptr(dy), _ptr(dw), _ptr(workspace), _nbytes(workspace),
                                              _stream(stream)))
+
+
+def nb_conv_bn_silu_infer(plan: Plan, x, w, gamma, beta, running_mean, running_var, a_out, workspace, stream=None):
+    _check(load().nb_conv_bn_silu_infer(plan.handle, _ptr(x), _ptr(w), _ptr(gamma), _ptr(beta), _ptr(running_mean), _ptr(running_var),
+                                        _ptr(a_out), _ptr(workspace), _nbytes(workspace), _stream(stream)))
+
+
+def nb_conv_bias_act(plan: Plan, x, w, bias, act, out, workspace, stream=None):
+    _check(load().nb_conv_bias_act(plan.handle, _ptr(x), _ptr(w), _ptr(bias), int(act), _ptr(out), _ptr(workspace), _nbytes(workspace),
+                                   _stream(stream)))
+
+
+def nb_bn_fold(plan: Plan, w, gamma, beta, running_mean, running_var, w_folded, bias_folded, stream=None):
+    _check(load().nb_bn_fold(plan.handle, _ptr(w), _ptr(gamma), _ptr(beta), _ptr(running_mean), _ptr(running_var), _ptr(w_folded),
+                             _ptr(bias_folded), _stream(stream)))
 
 
 def nb_conv_bn_silu_step_host(plan: Plan, host_x, host_w, host_gamma, host_beta, host_g, host_a, host_dx, host_dw, host_dgamma,

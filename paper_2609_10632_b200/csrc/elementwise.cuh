@@ -158,8 +158,8 @@ template <int V> __device__ __forceinline__ void load_params(const float* __rest
     }
 }
 
-// ------------------------------------------------------------------ a = SiLU(y*scale + shift)
-template <typename YT, typename AT, bool FAST>
+// ------------------------------------------------------------------ a = SiLU(y*scale + shift)  (ACT = false: no SiLU)
+template <typename YT, typename AT, bool FAST, bool ACT = true>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
                                                              long long total_vecs, int C, const float* __restrict__ scale,
                                                              const float* __restrict__ shift) {
@@ -179,9 +179,50 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const float z = fmaf(to_f32(q.v[i]), sc[i], sh[i]);
-            o.v[i] = from_f32<AT>(z * sigmoid_f<FAST>(z));
+            o.v[i] = from_f32<AT>(ACT ? z * sigmoid_f<FAST>(z) : z);
         }
         st16(a + v * V, o);
+    }
+}
+
+// ------------------------------------------------------------------ evaluation-mode coefficients and BN folding
+// scale_c = gamma_c / sqrt(rvar_c + eps), shift_c = beta_c - rmean_c*scale_c (fp64 arithmetic, like the training-mode
+// finalize).  gamma NULL: scale 1; rmean NULL: no normalisation (shift = beta, or 0 when beta is NULL too).
+__device__ __forceinline__ void bn_eval_coef(const float* gamma, const float* beta, const float* rmean, const float* rvar, float eps, int c, double& sc,
+                                             double& sh) {
+    sc = gamma ? (double)gamma[c] : 1.0;
+    sh = beta ? (double)beta[c] : 0.0;
+    if (rmean) {
+        sc /= sqrt((double)rvar[c] + (double)eps);
+        sh -= (double)rmean[c] * sc;
+    }
+}
+__global__ void __launch_bounds__(256) bn_eval_coef_kernel(const float* __restrict__ gamma, const float* __restrict__ beta, const float* __restrict__ rmean,
+                                                           const float* __restrict__ rvar, float eps, int C, float* __restrict__ scale,
+                                                           float* __restrict__ shift) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double sc, sh;
+    bn_eval_coef(gamma, beta, rmean, rvar, eps, c, sc, sh);
+    scale[c] = (float)sc;
+    shift[c] = (float)sh;
+}
+// Folded filter w'[co][t] = scale_co * w[co][t] (rounded to WT once) and bias'[co] = shift_co; K = taps per output channel.
+template <typename WT>
+__global__ void __launch_bounds__(256) bn_fold_kernel(const WT* __restrict__ w, long long K, int C, const float* __restrict__ gamma,
+                                                      const float* __restrict__ beta, const float* __restrict__ rmean, const float* __restrict__ rvar,
+                                                      float eps, WT* __restrict__ w_folded, float* __restrict__ bias_folded) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long total = (long long)C * K;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int co = (int)(i / K);
+        double sc, sh;
+        bn_eval_coef(gamma, beta, rmean, rvar, eps, co, sc, sh);
+        w_folded[i] = from_f32<WT>((float)((double)to_f32(w[i]) * sc));
+        if (i - (long long)co * K == 0) bias_folded[co] = (float)sh;
     }
 }
 

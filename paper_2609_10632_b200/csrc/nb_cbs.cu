@@ -44,10 +44,10 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 std::atomic<unsigned long long> g_launches{0};  // kernels launched by this library in this process
 
 enum Site { SITE_FPROP = 0, SITE_STATS, SITE_FINALIZE, SITE_APPLY, SITE_BWD_REDUCE, SITE_BWD_FINALIZE, SITE_BWD_DY,
-            SITE_WTRANSFORM, SITE_DGRAD, SITE_WGRAD, SITE_SPLITK_REDUCE, SITE_COUNT };
+            SITE_WTRANSFORM, SITE_DGRAD, SITE_WGRAD, SITE_SPLITK_REDUCE, SITE_INFER, SITE_EVAL_COEF, SITE_FOLD, SITE_COUNT };
 const char* const kSiteNames[SITE_COUNT] = {"conv_fprop", "bn_stats", "bn_finalize", "bn_silu_apply", "bn_silu_bwd_reduce",
                                             "bn_bwd_finalize", "bn_silu_bwd_dy", "dgrad_weight_transform", "conv_dgrad",
-                                            "conv_wgrad", "wgrad_splitk_reduce"};
+                                            "conv_wgrad", "wgrad_splitk_reduce", "conv_infer_fused", "bn_eval_coef", "bn_fold"};
 
 struct EwCfg {  // launch geometry of the [M][C] passes
     int vec, cgs, tpb;
@@ -76,6 +76,7 @@ struct nb_cbs_plan_s {
     double prof_ms[SITE_COUNT] = {};
     long long prof_n[SITE_COUNT] = {};
     size_t fwd_bytes, bwd_bytes;
+    size_t infer_bytes, off_iy;  // evaluation-mode forward: scale and shift at the forward offsets, then the convolution output when not fused
     // workspace offsets
     size_t off_scale, off_shift, off_fpart;                  // forward
     size_t off_coef, off_bpart, off_wt, off_wgpart;          // backward
@@ -84,6 +85,8 @@ struct nb_cbs_plan_s {
 namespace {
 
 bool is_f32(const nb_cbs_plan_s* p) { return p->desc.mode == NB_MODE_F32_REF; }
+// the evaluation-mode forward is one tensor-core kernel with the per-channel epilogue fused
+bool infer_fused(const nb_cbs_plan_s* p) { return !is_f32(p) && !p->stem && p->tc.infer; }
 
 nb_status check_ptr(const void* p, const char* name, bool nullable = false) {
     if (!p) return nullable ? NB_OK : fail(NB_ERR_INVALID_ARG, "%s is NULL", name);
@@ -171,11 +174,11 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
     return launch_ok("bn_finalize");
 }
 
-template <typename YT, typename AT, bool FAST>
+template <typename YT, typename AT, bool FAST, bool ACT = true>
 nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_APPLY, st);
-    launch_k(bn_silu_apply_kernel<YT, AT, FAST>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
+    launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
                                                                        p->g.c_out, scale, shift);
     return launch_ok("bn_silu_apply");
 }
@@ -384,6 +387,8 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->off_shift = off; off = align_up(off + C * 4, 256);
     p->off_fpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
     p->fwd_bytes = off;
+    p->off_iy = p->off_fpart;
+    p->infer_bytes = infer_fused(p) ? p->off_fpart : align_up(p->off_iy + (size_t)g.m * C * (is_f32(p) ? 4 : 2), 256);
     off = 0;
     p->off_coef = off; off = align_up(off + 4 * C * 4, 256);
     p->off_bpart = off; off = align_up(off + (size_t)p->nparts * 2 * C * 4, 256);
@@ -535,6 +540,93 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
     return run_apply<__half, __nv_bfloat16, true>(p, y_saved, a_out, scale, shift, st);
+}
+
+namespace {
+// conv -> out = act(conv*scale_c + shift_c) with (scale, shift) from evaluation-mode BN or a bias (see bn_eval_coef)
+nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float* gamma, const float* beta, const float* rmean, const float* rvar,
+                    int act, void* out, char* ws, cudaStream_t st) {
+    if (infer_fused(p)) {
+        SiteTimer tm(p, SITE_INFER, st);
+        const long long l0 = p->tc.launches;
+        const EpiAffine e{gamma, beta, rmean, rvar, p->desc.eps, act};
+        const nb_status ts = tc_infer(&p->tc, p->g, x, w, out, e, p->status, st);
+        g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
+        if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
+        return NB_OK;
+    }
+    float* scale = reinterpret_cast<float*>(ws + p->off_scale);
+    float* shift = reinterpret_cast<float*>(ws + p->off_shift);
+    void* y = ws + p->off_iy;
+    if (is_f32(p)) {
+        NB_TRY((run_simt_fprop<float, float>(p, x, w, y, st)));
+    } else if (p->stem) {
+        SiteTimer tm(p, SITE_FPROP, st);
+        const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
+        launch_k(stem_fprop_mma_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
+                 static_cast<__half*>(y), p->g);
+        NB_LAUNCH_OK("stem_fprop");
+    } else {
+        NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y, st)));
+    }
+    {
+        SiteTimer tm(p, SITE_EVAL_COEF, st);
+        launch_k(bn_eval_coef_kernel, dim3((unsigned)((p->g.c_out + 255) / 256)), dim3(256), 0, st, 1, gamma, beta, rmean, rvar, p->desc.eps, p->g.c_out, scale, shift);
+        NB_LAUNCH_OK("bn_eval_coef");
+    }
+    if (is_f32(p)) return act ? run_apply<float, float, false, true>(p, y, out, scale, shift, st) : run_apply<float, float, false, false>(p, y, out, scale, shift, st);
+    return act ? run_apply<__half, __nv_bfloat16, true, true>(p, y, out, scale, shift, st) : run_apply<__half, __nv_bfloat16, true, false>(p, y, out, scale, shift, st);
+}
+}  // namespace
+
+nb_status nb_cbs_infer_workspace_bytes(nb_cbs_plan p, size_t* bytes, int32_t* fused) {
+    g_err.clear();
+    if (!p || !bytes) return fail(NB_ERR_INVALID_ARG, "NULL argument");
+    *bytes = p->infer_bytes;
+    if (fused) *fused = infer_fused(p) ? 1 : 0;
+    return NB_OK;
+}
+
+nb_status nb_conv_bn_silu_infer(nb_cbs_plan p, const void* x, const void* w, const float* gamma, const float* beta, const float* running_mean,
+                                const float* running_var, void* a_out, void* workspace, size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta); NB_CHECK_PTR(running_mean); NB_CHECK_PTR(running_var);
+    NB_CHECK_PTR(a_out);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
+    DeviceGuard on_device(p->device);
+    return run_infer(p, x, w, gamma, beta, running_mean, running_var, 1, a_out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
+}
+
+nb_status nb_conv_bias_act(nb_cbs_plan p, const void* x, const void* w, const float* bias, int32_t act, void* out, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(bias, true); NB_CHECK_PTR(out);
+    if (act != 0 && act != 1) return fail(NB_ERR_INVALID_ARG, "act must be 0 (none) or 1 (SiLU), got %d", act);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
+    DeviceGuard on_device(p->device);
+    return run_infer(p, x, w, nullptr, bias, nullptr, nullptr, act, out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
+}
+
+nb_status nb_bn_fold(nb_cbs_plan p, const void* w, const float* gamma, const float* beta, const float* running_mean, const float* running_var,
+                     void* w_folded, float* bias_folded, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(w); NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta); NB_CHECK_PTR(running_mean); NB_CHECK_PTR(running_var);
+    NB_CHECK_PTR(w_folded); NB_CHECK_PTR(bias_folded);
+    DeviceGuard on_device(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long K = p->g.kdim, total = K * p->g.c_out;
+    const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, (long long)p->sm_count * 8);
+    SiteTimer tm(p, SITE_FOLD, st);
+    if (is_f32(p))
+        launch_k(bn_fold_kernel<float>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const float*>(w), K, p->g.c_out, gamma, beta, running_mean, running_var,
+                 p->desc.eps, static_cast<float*>(w_folded), bias_folded);
+    else
+        launch_k(bn_fold_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(w), K, p->g.c_out, gamma, beta, running_mean,
+                 running_var, p->desc.eps, static_cast<__nv_bfloat16*>(w_folded), bias_folded);
+    return launch_ok("bn_fold");
 }
 
 nb_status nb_bn_stats(nb_cbs_plan p, const void* y, int32_t y_dtype, float* mean, float* invstd, float* sum, float* sumsq,

@@ -55,6 +55,10 @@ struct IgemmParams {
     double fin_count;
     const float *fin_gamma, *fin_beta;
     float *fin_mean, *fin_invstd, *fin_scale, *fin_shift, *fin_rmean, *fin_rvar;
+    // Fused per-channel epilogue (EPI variant: evaluation-mode BN or a bias, then optionally SiLU, applied to the fp32
+    // accumulators before they are rounded): out = act(acc*scale_c + shift_c).  The CTA derives the coefficients itself
+    // from fin_gamma / fin_beta / fin_rmean / fin_rvar / fin_eps (gamma NULL: scale 1; rmean NULL: shift = beta or 0).
+    int epi_act;
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
     int variant;                 // experiment switches
@@ -177,9 +181,11 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
 // 128-byte swizzle), `release` is called as soon as the registers hold the data (the accumulator may be reused), lane 0
 // hands the 32 x NP piece to TMA, and with STATS the warp adds the piece's per-channel sums of the rounded values to its
 // running sums (a lane owns two adjacent channels).  Everything is unrolled on NP: constant offsets, no predicates.
-template <typename OutT, bool STATS, int NP, class Release>
+// With EPI the accumulators first become act(acc*scale + shift) with the pass's per-channel (scale, shift) pairs read
+// from shared memory (`coef`, the same address in every lane: a broadcast).
+template <typename OutT, bool STATS, int NP, int EPI, class Release>
 __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int lane, bool& store_pending, int& sat, const CUtensorMap* tm, int col,
-                                             int grow, float* stat_s, float* stat_q, Release release) {
+                                             int grow, float* stat_s, float* stat_q, const float2* coef, int act, Release release) {
     constexpr bool SWZ = NP == 64;
     constexpr int PITCH = NP * 2;
     uint32_t r[NP];
@@ -187,6 +193,24 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
     for (int hh = 0; hh < NP / 16; ++hh) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(16 * hh), r + 16 * hh);
     ptx::tmem_ld_wait();
     release();
+    if (EPI) {
+        if (act) {
+#pragma unroll
+            for (int j = 0; j < NP; j += 2) {
+                const float4 cf = *reinterpret_cast<const float4*>(coef + j);
+                const float z0 = fmaf(__uint_as_float(r[j]), cf.x, cf.y), z1 = fmaf(__uint_as_float(r[j + 1]), cf.z, cf.w);
+                r[j] = __float_as_uint(z0 * sigmoid_f<true>(z0));
+                r[j + 1] = __float_as_uint(z1 * sigmoid_f<true>(z1));
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NP; j += 2) {
+                const float4 cf = *reinterpret_cast<const float4*>(coef + j);
+                r[j] = __float_as_uint(fmaf(__uint_as_float(r[j]), cf.x, cf.y));
+                r[j + 1] = __float_as_uint(fmaf(__uint_as_float(r[j + 1]), cf.z, cf.w));
+            }
+        }
+    }
     if (store_pending) {  // the previous TMA store must have read the staging rows before they are overwritten
         if (lane == 0) ptx::tma_store_wait_read<0>();
         __syncwarp();
@@ -243,9 +267,12 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 // as a slab of padded-raster positions and the nine taps are nine row offsets into it, so the activation bytes written to
 // shared memory drop from 9 x 128*mh rows to 128*mh + 2*(W+2) + 2 rows per block.  Rows that fall on the padding ring
 // are computed and discarded.
-template <typename OutT, bool STATS, bool CG2, bool HALO>
+// EPI = 1: the epilogue applies a per-channel scale and shift (evaluation-mode BN or a bias) and optionally SiLU to the
+// accumulators, so the kernel writes the block's final activations (no statistics, no second pass); TMA stores only.
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0>
 __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
     static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
+    static_assert(!EPI || (!STATS && !HALO), "the fused per-channel epilogue is a forward-only variant without statistics");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
@@ -254,7 +281,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     const int cw = p.stage_cw;  // columns per staging pass (<= 64)
     const int pitch = cw * 2 + 16;
     float* wstat = reinterpret_cast<float*>(stg + (size_t)2 * TC_BM * pitch);  // per team [4 warps][2][its columns of every n-tile]: warp-private channel sums
-    uint64_t* bars = reinterpret_cast<uint64_t*>(wstat + (STATS ? 8 * p.ldo : 0));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wstat + ((STATS || EPI) ? 8 * p.ldo : 0));  // EPI: wstat holds [ldo] (scale, shift) pairs
     uint64_t* full = bars;                // [stages]
     uint64_t* empty = bars + p.stages;    // [stages]
     uint64_t* tfull = empty + p.stages;   // [2]
@@ -318,6 +345,16 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();  // everything above touched only shared memory, TMEM and kernel parameters
+    if (EPI) {
+        // per-channel coefficients of the fused epilogue, in fp64 like the training-mode finalize
+        float2* coef = reinterpret_cast<float2*>(wstat);
+        for (int c = threadIdx.x; c < p.ldo; c += IG_THREADS) {
+            double sc, sh;
+            bn_eval_coef(p.fin_gamma, p.fin_beta, p.fin_rmean, p.fin_rvar, p.fin_eps, c, sc, sh);
+            coef[c] = make_float2((float)sc, (float)sh);
+        }
+        __syncthreads();
+    }
 
     if (warp == 0 || warp == 6) {
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
@@ -780,10 +817,11 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     float* ss = my_stat + n_tile * ncol + cb;
                     float* sq = ss + st_ld;
                     const uint32_t ta = taddr + (uint32_t)cb;
-                    if (npass == 64) epi_pass_tma<OutT, STATS, 64>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
-                    else if (npass == 48) epi_pass_tma<OutT, STATS, 48>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
-                    else if (npass == 32) epi_pass_tma<OutT, STATS, 32>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
-                    else epi_pass_tma<OutT, STATS, 16>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, release);
+                    const float2* cf = reinterpret_cast<const float2*>(wstat) + col;  // read only by the EPI variant
+                    if (npass == 64) epi_pass_tma<OutT, STATS, 64, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                    else if (npass == 48) epi_pass_tma<OutT, STATS, 48, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                    else if (npass == 32) epi_pass_tma<OutT, STATS, 32, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                    else epi_pass_tma<OutT, STATS, 16, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
                     continue;
                 }
                 const int rpitch = tma_out ? npass * 2 : pitch;       // bytes between staged rows of this pass
@@ -1044,6 +1082,8 @@ struct TcPlan {
     int sm_count = 0;
     long long launches = 0;  // kernels launched through this record
     TcGemmSlot fp;
+    bool infer = false;  // the forward configuration also runs with the fused per-channel epilogue (its own slot: own output maps)
+    TcGemmSlot inf;
     TcGemmSlot dg;  // one launch covers all output-parity classes
     WtParams wtp;
     // wgrad
@@ -1323,20 +1363,20 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
     return true;
 }
 
-template <typename OutT, bool STATS, bool CG2, bool HALO> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     // the attribute belongs to the (function, device) pair: one bit per device ordinal that already has it
     static std::atomic<unsigned long long> attr_set{0};
     int dev = 0;
     cudaGetDevice(&dev);
     const unsigned long long bit = 1ull << (dev & 63);
     if (!(attr_set.load(std::memory_order_acquire) & bit)) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
         attr_set.fetch_or(bit, std::memory_order_release);
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
@@ -1384,6 +1424,10 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
             if (c.halo) fill_halo_taps(P);
             tc->fprop = true;
             tc->fprop_parts = c.grid;
+            if (!c.halo) {
+                tc->inf = tc->fp;
+                tc->infer = true;
+            }
         }
     }
     // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four output-parity
@@ -1578,6 +1622,40 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
 #endif
     tc->launches += 1;
     return launch_igemm<__half, true>(S, st);
+}
+
+// Forward convolution whose epilogue applies out = act(acc*scale_c + shift_c) and writes bf16: evaluation-mode BN
+// (gamma, beta, running statistics) or a plain bias (gamma = rmean = rvar = NULL, beta = bias or NULL).
+struct EpiAffine {
+    const float *gamma, *beta, *rmean, *rvar;
+    float eps;
+    int act;  // 1: SiLU
+};
+inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* w, void* out, const EpiAffine& e, int* status, cudaStream_t st) {
+    using namespace tcdetail;
+    TcGemmSlot& S = tc->inf;
+    if (S.a_ptr != x || S.b_ptr != w) {
+        if (S.prm.a_tiled) {
+            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
+        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, g.pad - (g.k - 1), g.stride, S.cfg.KC, TC_BM * S.cfg.mh)) {
+            return NB_ERR_CUDA;
+        }
+        if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+        S.a_ptr = x; S.b_ptr = w;
+    }
+    S.prm.tma_store = 1;  // the fused epilogue exists only on the TMA-store path
+    if (S.out_ptr != out) {
+        if (!encode_out_maps(S.prm, S.cfg, out, g.m)) return NB_ERR_CUDA;
+        S.out_ptr = out;
+    }
+    S.prm.fin_on = 0;
+    S.prm.fin_gamma = e.gamma; S.prm.fin_beta = e.beta;
+    S.prm.fin_rmean = const_cast<float*>(e.rmean); S.prm.fin_rvar = const_cast<float*>(e.rvar);  // only read
+    S.prm.fin_eps = e.eps; S.prm.epi_act = e.act;
+    S.prm.variant = 0;
+    S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
+    tc->launches += 1;
+    return S.cfg.cg2 ? launch_igemm_impl<__nv_bfloat16, false, true, false, 1>(S, st) : launch_igemm_impl<__nv_bfloat16, false, false, false, 1>(S, st);
 }
 
 // `wt_ready`: the rearranged filter was already written by an earlier kernel of this call (the BN backward finalize kernel

@@ -165,7 +165,7 @@ def round_to_bf16(a: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------- generators
-_ROLES = {"x": 0, "w": 1, "gamma": 2, "beta": 3, "g": 4, "rm": 5, "rv": 6}
+_ROLES = {"x": 0, "w": 1, "gamma": 2, "beta": 3, "g": 4, "rm": 5, "rv": 6, "bias": 7}
 
 
 def _rng(cfg_id: int, layer_id: int, role: str) -> np.random.Generator:
@@ -212,3 +212,16 @@ def make_inputs(shape: ConvShape, cfg_id: int = 0, layer_id: int = 0, bf16: bool
     if bf16:
         x, w, g = round_to_bf16(x), round_to_bf16(w), round_to_bf16(g)
     return BlockInputs(s, x, w, gamma, beta, g, {"cfg_id": cfg_id, "layer_id": layer_id, "bf16": bf16, "affine": affine})
+
+
+def make_eval_stats(shape: ConvShape, cfg_id: int = 0, layer_id: int = 0):
+    """Running statistics and a bias for the evaluation-mode / plain variants of one block (fp32 [c_out] each).
+
+    A unit-variance input through a filter drawn as in make_inputs gives a convolution output of variance 1/3, so the
+    running variance is U[0.25, 0.75), the running mean 0.2 * N(0,1); the bias of a plain layer is 0.5 * N(0,1).
+    """
+    c = shape.c_out
+    rm = (0.2 * _rng(cfg_id, layer_id, "rm").standard_normal(c, dtype=np.float32)).astype(np.float32)
+    rv = (0.25 + 0.5 * _rng(cfg_id, layer_id, "rv").random(c, dtype=np.float32)).astype(np.float32)
+    bias = (0.5 * _rng(cfg_id, layer_id, "bias").standard_normal(c, dtype=np.float32)).astype(np.float32)
+    return rm, rv, bias
