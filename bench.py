@@ -266,6 +266,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=6, help="streams of the end-to-end arm (1 = no overlap of copies and compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-eval-forward", action="store_true", help="skip the evaluation-mode forward measurement (extra object of the JSON line)")
     ap.add_argument("--no-profile", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--force-simt", action="store_true", help="run the convolutions on the CUDA-core kernels")
@@ -435,6 +436,11 @@ def main():
         roofline["avg_launch_ms"] = a["ms"] / a["launches"]
         roofline["share_of_step"] = a["ms"] / tot_ms
 
+    # ---------------- the evaluation-mode forward (running statistics; one fused kernel per tensor-core layer)
+    eval_fwd = None
+    if not args.no_eval_forward:
+        eval_fwd = run_eval_forward(args, blocks, dev, flops / 3.0, peaks, kernels)
+
     # ---------------- end to end from pinned host buffers through the C ABI
     e2e = None
     if not args.no_e2e:
@@ -462,11 +468,57 @@ def main():
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },
             "clocks": clocks.summary(), "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernels,
+            "kernels": kernels, "eval_forward": eval_fwd,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_eval_forward(args, blocks, dev, fwd_flops, peaks, kernels):
+    """The evaluation-mode forward of every layer (nb_conv_bn_silu_infer: running statistics, no saved tensors) as a
+    CUDA-graph replay on this rank; reported beside the training step, not part of `value`."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4242)
+    ws = torch.empty(max(max(b.plan.infer_bytes for b in blocks), 256), dtype=torch.uint8, device=dev)
+    stats = []
+    for b in blocks:
+        c = b.shape.c_out
+        stats.append((0.2 * torch.randn(c, generator=gen, device=dev), 0.25 + 0.5 * torch.rand(c, generator=gen, device=dev)))
+
+    def fwd_all():
+        for b, (rm, rv) in zip(blocks, stats):
+            nb.nb_conv_bn_silu_infer(b.plan, b.x, b.w, b.gamma, b.beta, rm, rv, b.a, ws)
+
+    for _ in range(max(3, args.warmup)):
+        fwd_all()
+    torch.cuda.synchronize()
+    l0 = nb.nb_cbs_launch_count()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fwd_all()
+    launches = nb.nb_cbs_launch_count() - l0
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    for b in blocks:
+        b.poll()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    train_fwd = sum(kernels[k]["ms_per_step"] for k in ("conv_fprop", "bn_stats", "bn_finalize", "bn_silu_apply") if k in kernels) if kernels else None
+    tf = fwd_flops / (ms * 1e-3) / 1e12
+    return {"call": "nb_conv_bn_silu_infer", "ms_per_pass": ms, "tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"],
+            "launches_per_pass": int(launches), "fused_layers": sum(1 for b in blocks if b.plan.infer_fused), "layers": len(blocks),
+            "training_forward_kernels_ms": train_fwd, "cuda_graph": True}
 
 
 def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):

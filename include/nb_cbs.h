@@ -175,7 +175,8 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan plan, const void* x, const void
  *
  * Workspace size of the three calls below and whether they run as ONE kernel: `*fused` (may be NULL) is 1 when the
  * convolution runs on the tensor-core kernel with the per-channel scale/shift and the activation applied to the fp32
- * accumulators in its epilogue (BF16 mode, c_in % 16 == 0, c_out % 16 == 0); 0 when the plan falls back to
+ * accumulators in its epilogue (BF16 mode, c_in % 16 == 0, c_out % 16 == 0; also the 3 -> 48 channel 3x3 stride-2
+ * first layer, whose own kernel has the same epilogue); 0 when the plan falls back to
  * convolution -> coefficient kernel -> elementwise pass, whose workspace also holds the convolution output. */
 nb_status nb_cbs_infer_workspace_bytes(nb_cbs_plan plan, size_t* bytes, int32_t* fused);
 

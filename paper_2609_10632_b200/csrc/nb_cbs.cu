@@ -86,7 +86,7 @@ namespace {
 
 bool is_f32(const nb_cbs_plan_s* p) { return p->desc.mode == NB_MODE_F32_REF; }
 // the evaluation-mode forward is one tensor-core kernel with the per-channel epilogue fused
-bool infer_fused(const nb_cbs_plan_s* p) { return !is_f32(p) && !p->stem && p->tc.infer; }
+bool infer_fused(const nb_cbs_plan_s* p) { return !is_f32(p) && (p->stem || p->tc.infer); }
 
 nb_status check_ptr(const void* p, const char* name, bool nullable = false) {
     if (!p) return nullable ? NB_OK : fail(NB_ERR_INVALID_ARG, "%s is NULL", name);
@@ -517,7 +517,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
             SiteTimer tm(p, SITE_FPROP, st);
             const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
             launch_k(stem_fprop_mma_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
-                         static_cast<__half*>(y_saved), p->g);
+                         static_cast<__half*>(y_saved), p->g, StemEpi{});
             NB_LAUNCH_OK("stem_fprop");
         }
         NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
@@ -546,7 +546,7 @@ namespace {
 // conv -> out = act(conv*scale_c + shift_c) with (scale, shift) from evaluation-mode BN or a bias (see bn_eval_coef)
 nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float* gamma, const float* beta, const float* rmean, const float* rvar,
                     int act, void* out, char* ws, cudaStream_t st) {
-    if (infer_fused(p)) {
+    if (infer_fused(p) && !p->stem) {
         SiteTimer tm(p, SITE_INFER, st);
         const long long l0 = p->tc.launches;
         const EpiAffine e{gamma, beta, rmean, rvar, p->desc.eps, act};
@@ -555,17 +555,18 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         return NB_OK;
     }
+    if (!is_f32(p) && p->stem) {  // the first layer's own kernel applies the coefficients and the activation itself
+        SiteTimer tm(p, SITE_INFER, st);
+        const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
+        launch_k(stem_fprop_mma_kernel<48, __nv_bfloat16, true>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x),
+                 static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act});
+        return launch_ok("stem_fprop (fused epilogue)");
+    }
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
     float* shift = reinterpret_cast<float*>(ws + p->off_shift);
     void* y = ws + p->off_iy;
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y, st)));
-    } else if (p->stem) {
-        SiteTimer tm(p, SITE_FPROP, st);
-        const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
-        launch_k(stem_fprop_mma_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
-                 static_cast<__half*>(y), p->g);
-        NB_LAUNCH_OK("stem_fprop");
     } else {
         NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y, st)));
     }

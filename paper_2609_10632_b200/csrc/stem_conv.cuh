@@ -20,9 +20,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-template <int COUT>
+// Per-channel epilogue of the evaluation-mode / plain forward: out = act(acc*scale_c + shift_c), coefficients as bn_eval_coef.
+struct StemEpi {
+    const float *gamma, *beta, *rmean, *rvar;
+    float eps;
+    int act;
+};
+// EPI = false: y = the convolution output in fp16 (training forward).  EPI = true: OutT = bf16 activations, see StemEpi.
+template <int COUT, typename OutT = __half, bool EPI = false>
 __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
-                                                             __half* __restrict__ y, Geom g) {
+                                                             OutT* __restrict__ y, Geom g, StemEpi ep) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 8 == 0, "whole n-blocks");
@@ -56,7 +63,20 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16
                 const uint32_t lo = k < STEM_KDIM ? wsrc[n * STEM_KDIM + k] : 0u, hi = k + 1 < STEM_KDIM ? wsrc[n * STEM_KDIM + k + 1] : 0u;
                 bfrag[s2][nb][j] = lo | (hi << 16);
             }
-    __shared__ __align__(16) __half stage[4][16 * COUT];
+    // this lane's accumulator columns are nb*8 + 2*tq and the next one: their (scale, shift) pairs stay in registers
+    float esc[EPI ? NB : 1][2], esh[EPI ? NB : 1][2];
+    if (EPI) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                double sc, sh;
+                bn_eval_coef(ep.gamma, ep.beta, ep.rmean, ep.rvar, ep.eps, nb * 8 + tq * 2 + e, sc, sh);
+                esc[nb][e] = (float)sc;
+                esh[nb][e] = (float)sh;
+            }
+    }
+    __shared__ __align__(16) OutT stage[4][16 * COUT];
     const long long ntiles = (g.m + 15) / 16;
     const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
     for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < ntiles; tile += wstride) {
@@ -94,13 +114,24 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16
         }
         // accumulator registers: c0, c1 = (row g, columns 2t, 2t+1), c2, c3 = (row g+8, same columns).  The 16 x COUT tile is one
         // contiguous run of the output, so it is staged in shared memory and written with coalesced 16-byte stores.
-        __half* st = stage[threadIdx.x >> 5];
+        OutT* st = stage[threadIdx.x >> 5];
 #pragma unroll
         for (int half = 0; half < 2; ++half)
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb)
-                *reinterpret_cast<__half2*>(st + (gq + half * 8) * COUT + nb * 8 + tq * 2) =
-                    __halves2half2(from_f32<__half>(acc[nb][2 * half]), from_f32<__half>(acc[nb][2 * half + 1]));
+            for (int nb = 0; nb < NB; ++nb) {
+                float v0 = acc[nb][2 * half], v1 = acc[nb][2 * half + 1];
+                if (EPI) {
+                    v0 = fmaf(v0, esc[nb][0], esh[nb][0]);
+                    v1 = fmaf(v1, esc[nb][1], esh[nb][1]);
+                    if (ep.act) {
+                        v0 *= sigmoid_f<true>(v0);
+                        v1 *= sigmoid_f<true>(v1);
+                    }
+                }
+                OutT* dst = st + (gq + half * 8) * COUT + nb * 8 + tq * 2;
+                dst[0] = from_f32<OutT>(v0);
+                dst[1] = from_f32<OutT>(v1);
+            }
         __syncwarp();
         const long long rows_left = g.m - m0;
         const int nvec = (int)(rows_left >= 16 ? 16 : rows_left) * COUT / 8;  // 16-byte pieces of the tile that exist

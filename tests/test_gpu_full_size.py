@@ -35,8 +35,20 @@ def test_full_size_block_matches_oracle(shape, label, layer_id):
     msg = blk.poll()
     assert "saturated" not in msg
     out = blk.download()
-    del blk
+    # the evaluation-mode forward of the same layer (running statistics from the seeded generator), same launch as bench.py's
+    import torch
+
+    rm, rv, _ = wl.make_eval_stats(shape, cfg_id=5, layer_id=layer_id)
+    a_eval = torch.empty_like(blk.a)
+    ws = torch.empty(max(blk.plan.infer_bytes, 256), dtype=torch.uint8, device=blk.dev)
+    nb.nb_conv_bn_silu_infer(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, torch.from_numpy(rm).to(blk.dev), torch.from_numpy(rv).to(blk.dev), a_eval, ws)
+    torch.cuda.synchronize()
+    blk.poll()
+    a_eval = a_eval.to(torch.float64).cpu().numpy()
+    del blk, ws
     ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, shape.stride, EPS)
+    # oracle stage applied to the oracle's own convolution output of the same (x, w)
+    parity.check("a_eval", a_eval, oracle.bn_eval_act(ref.y, inp.gamma, inp.beta, rm, rv, EPS), "bf16")
     rep = {}
     for name in ("a", "dx", "dw", "dgamma", "dbeta", "y", "dy"):
         parity.check(name, out[name], getattr(ref, name), "bf16", rep)
