@@ -27,7 +27,7 @@ EXPORTS = (
     "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
-    "nb_bn_fold",
+    "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step",
 )
 
 
@@ -36,6 +36,16 @@ class nb_cbs_desc(Structure):
         ("struct_size", c_uint32), ("n", c_int32), ("h", c_int32), ("w", c_int32), ("c_in", c_int32), ("c_out", c_int32),
         ("ksize", c_int32), ("stride", c_int32), ("eps", c_float), ("momentum", c_float), ("mode", c_int32), ("flags", c_uint32),
     ]
+
+
+class nb_sgd_tensor(Structure):
+    _fields_ = [("grad", c_void_p), ("param", c_void_p), ("momentum", c_void_p), ("param_bf16", c_void_p), ("numel", ctypes.c_int64),
+                ("group", c_int32), ("reserved", c_int32)]
+
+
+class nb_sgd_hyper(Structure):
+    _fields_ = [("struct_size", c_uint32), ("momentum", c_float), ("max_norm", c_float), ("lr", c_float * 3), ("weight_decay", c_float * 3),
+                ("first_step", c_int32)]
 
 
 class NbError(RuntimeError):
@@ -77,6 +87,11 @@ def load() -> ctypes.CDLL:
         lib.nb_conv_bn_silu_infer.argtypes = [V, V, V, FP, FP, FP, FP, V, V, c_size_t, V]
         lib.nb_conv_bias_act.argtypes = [V, V, V, FP, c_int32, V, V, c_size_t, V]
         lib.nb_bn_fold.argtypes = [V, V, FP, FP, FP, FP, V, FP, V]
+        lib.nb_sgd_plan_create.argtypes = [POINTER(nb_sgd_tensor), c_int32, c_int, POINTER(V)]
+        lib.nb_sgd_plan_destroy.argtypes = [V]
+        lib.nb_sgd_workspace_bytes.argtypes = [V, POINTER(c_size_t)]
+        lib.nb_sgd_upload.argtypes = [V, V, c_size_t, V]
+        lib.nb_sgd_clip_nesterov_step.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), FP, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -254,3 +269,40 @@ def nb_conv_bn_silu_step_host(plan: Plan, host_x, host_w, host_gamma, host_beta,
     _check(load().nb_conv_bn_silu_step_host(plan.handle, _ptr(host_x), _ptr(host_w), _ptr(host_gamma), _ptr(host_beta), _ptr(host_g),
                                             _ptr(host_a), _ptr(host_dx), _ptr(host_dw), _ptr(host_dgamma), _ptr(host_dbeta),
                                             _ptr(device_scratch), _nbytes(device_scratch), _stream(stream)))
+
+
+class SgdPlan:
+    """Owner of one nb_sgd_plan handle.  `tensors`: iterable of (grad, param, momentum, param_bf16 or None, group), each a
+    device tensor (or a raw address with an explicit numel as a sixth item)."""
+
+    def __init__(self, tensors, device=0):
+        items = list(tensors)
+        arr = (nb_sgd_tensor * max(len(items), 1))()
+        for i, it in enumerate(items):
+            grad, param, mom, lp, group = it[:5]
+            numel = it[5] if len(it) > 5 else param.numel()
+            arr[i] = nb_sgd_tensor(_ptr(grad), _ptr(param), _ptr(mom), _ptr(lp), int(numel), int(group), 0)
+        self.count = len(items)
+        self.handle = c_void_p()
+        _check(load().nb_sgd_plan_create(arr, self.count, device, byref(self.handle)))
+        b = c_size_t()
+        _check(load().nb_sgd_workspace_bytes(self.handle, byref(b)))
+        self.workspace_bytes = b.value
+
+    def upload(self, workspace, stream=None):
+        _check(load().nb_sgd_upload(self.handle, _ptr(workspace), _nbytes(workspace), _stream(stream)))
+
+    def step(self, workspace, lr, weight_decay, momentum, max_norm, first_step, total_norm=None, stream=None):
+        h = nb_sgd_hyper(ctypes.sizeof(nb_sgd_hyper), momentum, max_norm, (c_float * 3)(*lr), (c_float * 3)(*weight_decay), 1 if first_step else 0)
+        _check(load().nb_sgd_clip_nesterov_step(self.handle, _ptr(workspace), _nbytes(workspace), byref(h), _ptr(total_norm), _stream(stream)))
+
+    def close(self):
+        if self.handle:
+            load().nb_sgd_plan_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

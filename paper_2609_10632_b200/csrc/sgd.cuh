@@ -1,0 +1,137 @@
+// Fused optimiser step: global-norm clipping over a list of gradient tensors, then SGD with Nesterov momentum
+// (see include/nb_sgd.h for the arithmetic).  Two kernels for any number of tensors: the elements of all tensors are
+// cut into chunks of SGD_CHUNK elements, chunk i belongs to block i % gridDim.x, and both kernels walk the same table.
+#pragma once
+#include "../../include/nb_sgd.h"
+#include "common.cuh"
+
+namespace nbcbs {
+
+constexpr int SGD_CHUNK = 4096;    // elements per chunk (a multiple of 4: chunks start 16-byte aligned)
+constexpr int SGD_THREADS = 256;
+constexpr int SGD_MAX_BLOCKS = 2048;
+constexpr uint32_t SGD_MAGIC = 0x6e627367u;
+
+struct SgdChunk {
+    int32_t tensor;
+    int32_t len;     // elements of this chunk (<= SGD_CHUNK)
+    int64_t start;   // first element inside the tensor
+};
+struct SgdHeader {  // first 256 bytes of the workspace
+    uint32_t magic;
+    int32_t count, nchunks, grid;
+    uint64_t off_tensors, off_chunks, off_partials, total_bytes;
+};
+
+__device__ __forceinline__ double block_sum_fixed_order(double v, double* red /*[SGD_THREADS/32]*/) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < SGD_THREADS / 32; ++w) t += red[w];
+    return t;  // valid in thread 0
+}
+
+// partials[b] = sum of g^2 over the chunks of block b (fp32 per thread over at most a few hundred elements, fp64 above).
+__global__ void __launch_bounds__(SGD_THREADS) sgd_sqnorm_kernel(const uint8_t* __restrict__ ws) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const SgdHeader& H = *reinterpret_cast<const SgdHeader*>(ws);
+    const nb_sgd_tensor* T = reinterpret_cast<const nb_sgd_tensor*>(ws + H.off_tensors);
+    const SgdChunk* C = reinterpret_cast<const SgdChunk*>(ws + H.off_chunks);
+    double* partials = reinterpret_cast<double*>(const_cast<uint8_t*>(ws) + H.off_partials);
+    __shared__ double red[SGD_THREADS / 32];
+    double acc = 0.0;
+    for (int c = blockIdx.x; c < H.nchunks; c += gridDim.x) {
+        const SgdChunk ch = C[c];
+        const float* g = T[ch.tensor].grad + ch.start;
+        const int n4 = ch.len >> 2;
+        float s = 0.f;
+        for (int i = threadIdx.x; i < n4; i += SGD_THREADS) {
+            const float4 v = reinterpret_cast<const float4*>(g)[i];
+            s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); s = fmaf(v.z, v.z, s); s = fmaf(v.w, v.w, s);
+        }
+        for (int i = (n4 << 2) + threadIdx.x; i < ch.len; i += SGD_THREADS) s = fmaf(g[i], g[i], s);
+        acc += (double)s;
+    }
+    const double t = block_sum_fixed_order(acc, red);
+    if (threadIdx.x == 0) partials[blockIdx.x] = t;
+}
+
+struct SgdScalars {
+    float momentum, max_norm;
+    float lr[NB_SGD_GROUPS], wd[NB_SGD_GROUPS];
+    int first_step;
+};
+
+__device__ __forceinline__ void sgd_one(float g, float& p, float& b, float coef, float lr, float wd, float mom, bool first) {
+    const float d = fmaf(wd, p, g * coef);
+    b = first ? d : fmaf(mom, b, d);
+    p = fmaf(-lr, fmaf(mom, b, d), p);
+}
+
+__global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* __restrict__ ws, SgdScalars hs, float* __restrict__ total_norm_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const SgdHeader& H = *reinterpret_cast<const SgdHeader*>(ws);
+    const nb_sgd_tensor* T = reinterpret_cast<const nb_sgd_tensor*>(ws + H.off_tensors);
+    const SgdChunk* C = reinterpret_cast<const SgdChunk*>(ws + H.off_chunks);
+    const double* partials = reinterpret_cast<const double*>(ws + H.off_partials);
+    // every block forms the clip coefficient itself from the norm kernel's partial sums, in one fixed order
+    __shared__ double red[SGD_THREADS / 32];
+    __shared__ float s_coef;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < H.grid; i += SGD_THREADS) acc += partials[i];
+    const double t = block_sum_fixed_order(acc, red);
+    if (threadIdx.x == 0) {
+        const double total = sqrt(t);
+        double c = 1.0;
+        if (hs.max_norm > 0.f && hs.max_norm < __int_as_float(0x7f800000)) c = fmin((double)hs.max_norm / (total + 1e-6), 1.0);
+        s_coef = (float)c;
+        if (blockIdx.x == 0 && total_norm_out) *total_norm_out = (float)total;
+    }
+    __syncthreads();
+    const float coef = s_coef, mom = hs.momentum;
+    const bool first = hs.first_step != 0;
+    for (int c = blockIdx.x; c < H.nchunks; c += gridDim.x) {
+        const SgdChunk ch = C[c];
+        const nb_sgd_tensor t_ = T[ch.tensor];
+        const int grp = t_.group;  // selects, not indexing: the scalars stay in the parameter bank
+        const float lr = grp == 0 ? hs.lr[0] : grp == 1 ? hs.lr[1] : hs.lr[2];
+        const float wd = grp == 0 ? hs.wd[0] : grp == 1 ? hs.wd[1] : hs.wd[2];
+        const float* g = t_.grad + ch.start;
+        float* p = t_.param + ch.start;
+        float* b = t_.momentum + ch.start;
+        __nv_bfloat16* lp = t_.param_bf16 ? static_cast<__nv_bfloat16*>(t_.param_bf16) + ch.start : nullptr;
+        const int n4 = ch.len >> 2;
+        for (int i = threadIdx.x; i < n4; i += SGD_THREADS) {
+            const float4 gv = reinterpret_cast<const float4*>(g)[i];
+            float4 pv = reinterpret_cast<const float4*>(p)[i];
+            float4 bv = first ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(b)[i];
+            sgd_one(gv.x, pv.x, bv.x, coef, lr, wd, mom, first);
+            sgd_one(gv.y, pv.y, bv.y, coef, lr, wd, mom, first);
+            sgd_one(gv.z, pv.z, bv.z, coef, lr, wd, mom, first);
+            sgd_one(gv.w, pv.w, bv.w, coef, lr, wd, mom, first);
+            reinterpret_cast<float4*>(p)[i] = pv;
+            reinterpret_cast<float4*>(b)[i] = bv;
+            if (lp) {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(pv.x, pv.y), hi = __floats2bfloat162_rn(pv.z, pv.w);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t*>(&lo);
+                o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                reinterpret_cast<uint2*>(lp)[i] = o;
+            }
+        }
+        for (int i = (n4 << 2) + threadIdx.x; i < ch.len; i += SGD_THREADS) {
+            float pv = p[i], bv = first ? 0.f : b[i];
+            sgd_one(g[i], pv, bv, coef, lr, wd, mom, first);
+            p[i] = pv;
+            b[i] = bv;
+            if (lp) lp[i] = __float2bfloat16_rn(pv);
+        }
+    }
+}
+
+}  // namespace nbcbs

@@ -121,6 +121,21 @@ def detector_plain_head_convs():
     return [(64, 64), (192, 80)] * 3
 
 
+def detector_parameter_tensors():
+    """[(name, numel, group)] of the detector's trainable tensors in network order: per Conv-BN-SiLU layer the filter
+    (group 0: decayed weights), the BN gain (group 1) and the BN shift (group 2: biases); per plain head convolution its
+    filter (group 0) and bias (group 2).  243 tensors, about 25.9 M elements (Sec. 3.2 / Sec. 6; pinned in tests)."""
+    out = []
+    for s in detector_layers():
+        out.append((f"{s.name}.w", s.c_out * s.k * s.k * s.c_in, 0))
+        out.append((f"{s.name}.gamma", s.c_out, 1))
+        out.append((f"{s.name}.beta", s.c_out, 2))
+    for i, (cin, cout) in enumerate(detector_plain_head_convs()):
+        out.append((f"h22.out{i}.w", cout * cin, 0))
+        out.append((f"h22.out{i}.bias", cout, 2))
+    return out
+
+
 def distinct_shapes(layers):
     """[(shape, multiplicity)] in first-appearance order."""
     seen: dict = {}
@@ -225,3 +240,16 @@ def make_eval_stats(shape: ConvShape, cfg_id: int = 0, layer_id: int = 0):
     rv = (0.25 + 0.5 * _rng(cfg_id, layer_id, "rv").random(c, dtype=np.float32)).astype(np.float32)
     bias = (0.5 * _rng(cfg_id, layer_id, "bias").standard_normal(c, dtype=np.float32)).astype(np.float32)
     return rm, rv, bias
+
+
+def make_optimizer_inputs(sizes, cfg_id: int, step: int, grad_scale: float = 1.0):
+    """Seeded fp32 gradients for optimiser step `step` over tensors of the given sizes, plus (for step 0) parameters.
+
+    Parameters: 0.05 * N(0,1); gradients: grad_scale * N(0,1).  Returns (params or None, grads) as lists of fp32 arrays.
+    """
+    params = None
+    if step == 0:
+        params = [(0.05 * _rng(cfg_id, i, "w").standard_normal(n, dtype=np.float32)).astype(np.float32) for i, n in enumerate(sizes)]
+    grads = [(np.float32(grad_scale) * _rng(cfg_id + 1000 * (step + 1), i, "g").standard_normal(n, dtype=np.float32)).astype(np.float32)
+             for i, n in enumerate(sizes)]
+    return params, grads

@@ -95,3 +95,21 @@ def test_plan_create_without_a_device_fails_loudly(lib):
     assert st == nb.NB_ERR_CUDA and msg
     with pytest.raises(nb.NbError):
         nb.Plan(2, 8, 8, 16, 32, 3, 1)
+
+
+def test_sgd_plan_rejects_bad_lists_before_any_cuda_call(lib):
+    h = ctypes.c_void_p()
+    assert lib.nb_sgd_plan_create(None, 1, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
+    arr = (nb.nb_sgd_tensor * 1)()
+    arr[0] = nb.nb_sgd_tensor(0x1000, 0x2000, 0x3000, None, 16, 0, 0)
+    assert lib.nb_sgd_plan_create(arr, 0, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
+    arr[0].numel = 0
+    assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
+    arr[0].numel = 16
+    arr[0].group = 3
+    assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
+    assert "group" in nb.nb_last_error()
+    arr[0].group = 0
+    arr[0].grad = 0x1004
+    assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_ALIGNMENT
+    assert ctypes.sizeof(nb.nb_sgd_tensor) == 48 and ctypes.sizeof(nb.nb_sgd_hyper) == 40

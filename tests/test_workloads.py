@@ -30,6 +30,9 @@ def test_layer_table_matches_paper_counts():
     assert round(total / 1e6, 1) == gold["params_millions"]
     # trainable tensors: weight + gamma + beta per Conv-BN-SiLU layer, weight + bias per plain head conv
     assert 3 * len(layers) + 2 * len(wl.detector_plain_head_convs()) == int(gold["gradient_tensors"])
+    tensors = wl.detector_parameter_tensors()  # the optimiser's tensor list
+    assert len(tensors) == int(gold["gradient_tensors"]) and sum(n for _, n, _ in tensors) == total
+    assert [sum(1 for t in tensors if t[2] == g) for g in (0, 1, 2)] == [83, 77, 83]  # decayed weights, BN gains, biases
     # head levels
     heads = [s for s in layers if s.name.startswith("h22.cls") and s.name.endswith(".0")]
     assert sum(s.ho * s.wo for s in heads) == int(gold["candidate_locations"])
