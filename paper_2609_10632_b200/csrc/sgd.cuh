@@ -9,6 +9,7 @@ namespace nbcbs {
 
 constexpr int SGD_CHUNK = 4096;    // elements per chunk (a multiple of 4: chunks start 16-byte aligned)
 constexpr int SGD_THREADS = 256;
+constexpr int SGD_VPT = SGD_CHUNK / 4 / SGD_THREADS;  // 16-byte vectors per thread and chunk
 constexpr int SGD_MAX_BLOCKS = 2048;
 constexpr uint32_t SGD_MAGIC = 0x6e627367u;
 
@@ -49,9 +50,16 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_sqnorm_kernel(const uint8_t* 
         const float* g = T[ch.tensor].grad + ch.start;
         const int n4 = ch.len >> 2;
         float s = 0.f;
-        for (int i = threadIdx.x; i < n4; i += SGD_THREADS) {
-            const float4 v = reinterpret_cast<const float4*>(g)[i];
-            s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); s = fmaf(v.z, v.z, s); s = fmaf(v.w, v.w, s);
+        // a chunk is at most SGD_VPT vectors per thread: all of them are requested before the first is used
+        float4 v[SGD_VPT];
+#pragma unroll
+        for (int k = 0; k < SGD_VPT; ++k) {
+            const int i = threadIdx.x + k * SGD_THREADS;
+            v[k] = i < n4 ? reinterpret_cast<const float4*>(g)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < SGD_VPT; ++k) {
+            s = fmaf(v[k].x, v[k].x, s); s = fmaf(v[k].y, v[k].y, s); s = fmaf(v[k].z, v[k].z, s); s = fmaf(v[k].w, v[k].w, s);
         }
         for (int i = (n4 << 2) + threadIdx.x; i < ch.len; i += SGD_THREADS) s = fmaf(g[i], g[i], s);
         acc += (double)s;
@@ -106,18 +114,29 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
         float* b = t_.momentum + ch.start;
         __nv_bfloat16* lp = t_.param_bf16 ? static_cast<__nv_bfloat16*>(t_.param_bf16) + ch.start : nullptr;
         const int n4 = ch.len >> 2;
-        for (int i = threadIdx.x; i < n4; i += SGD_THREADS) {
-            const float4 gv = reinterpret_cast<const float4*>(g)[i];
-            float4 pv = reinterpret_cast<const float4*>(p)[i];
-            float4 bv = first ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<const float4*>(b)[i];
-            sgd_one(gv.x, pv.x, bv.x, coef, lr, wd, mom, first);
-            sgd_one(gv.y, pv.y, bv.y, coef, lr, wd, mom, first);
-            sgd_one(gv.z, pv.z, bv.z, coef, lr, wd, mom, first);
-            sgd_one(gv.w, pv.w, bv.w, coef, lr, wd, mom, first);
-            reinterpret_cast<float4*>(p)[i] = pv;
-            reinterpret_cast<float4*>(b)[i] = bv;
+        // all loads of the chunk first (up to 3 x SGD_VPT vectors in flight per thread), then the arithmetic and the stores
+        float4 gv[SGD_VPT], pv[SGD_VPT], bv[SGD_VPT];
+        const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < SGD_VPT; ++k) {
+            const int i = threadIdx.x + k * SGD_THREADS;
+            const bool in = i < n4;
+            gv[k] = in ? reinterpret_cast<const float4*>(g)[i] : zero4;
+            pv[k] = in ? reinterpret_cast<const float4*>(p)[i] : zero4;
+            bv[k] = (in && !first) ? reinterpret_cast<const float4*>(b)[i] : zero4;
+        }
+#pragma unroll
+        for (int k = 0; k < SGD_VPT; ++k) {
+            const int i = threadIdx.x + k * SGD_THREADS;
+            if (i >= n4) break;
+            sgd_one(gv[k].x, pv[k].x, bv[k].x, coef, lr, wd, mom, first);
+            sgd_one(gv[k].y, pv[k].y, bv[k].y, coef, lr, wd, mom, first);
+            sgd_one(gv[k].z, pv[k].z, bv[k].z, coef, lr, wd, mom, first);
+            sgd_one(gv[k].w, pv[k].w, bv[k].w, coef, lr, wd, mom, first);
+            reinterpret_cast<float4*>(p)[i] = pv[k];
+            reinterpret_cast<float4*>(b)[i] = bv[k];
             if (lp) {
-                const __nv_bfloat162 lo = __floats2bfloat162_rn(pv.x, pv.y), hi = __floats2bfloat162_rn(pv.z, pv.w);
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(pv[k].x, pv[k].y), hi = __floats2bfloat162_rn(pv[k].z, pv[k].w);
                 uint2 o;
                 o.x = *reinterpret_cast<const uint32_t*>(&lo);
                 o.y = *reinterpret_cast<const uint32_t*>(&hi);
