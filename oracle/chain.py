@@ -1,0 +1,79 @@
+"""fp64 CPU oracle of a CHAINED group of Conv-BN-SiLU blocks: the C2f unit of the paper's detector (Sec. 6), forward and
+backward, composed from the single-block stage functions of this package and plain numpy slicing.
+
+TEST INFRASTRUCTURE ONLY (same rules as the rest of this package).
+
+C2f(c1 -> c2, n bottlenecks, shortcut): with c = c2 / 2
+    a0 = CBS_1x1(x)                      [.., 2c]
+    parts = [a0[.., :c], a0[.., c:]]
+    for i < n:  t = parts[-1];  v = CBS_3x3(CBS_3x3(t));  parts.append(t + v if shortcut else v)
+    out = CBS_1x1(concat(parts))         [.., c2]
+Every CBS is conv -> BN(batch statistics) -> SiLU.  In the backward pass a tensor with several consumers receives the
+sum of their gradients (a part feeds the concatenation, the next bottleneck and, with the shortcut, that bottleneck's sum).
+
+Pins (tests/test_oracle_pins_chain.py): central finite differences of the whole unit with respect to inputs and filters,
+n = 0 reducing to two blocks in sequence, and the shortcut's effect on a linearised case.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+import oracle
+
+
+@dataclass
+class BlockParams:
+    w: np.ndarray
+    gamma: np.ndarray
+    beta: np.ndarray
+
+
+@dataclass
+class C2fResult:
+    out: np.ndarray
+    parts: list
+    dx: np.ndarray | None = None
+    grads: list = field(default_factory=list)  # per block, in layer order: (dw, dgamma, dbeta)
+
+
+def _block_bwd(x_in, prm: BlockParams, fwd, g, stride=1):
+    dy, dgamma, dbeta = oracle.bn_silu_bwd(g, fwd.y, fwd.mean, fwd.invstd, prm.gamma, prm.beta)
+    dx = oracle.conv_dgrad(dy, prm.w, np.shape(x_in), stride)
+    dw = oracle.conv_wgrad(x_in, dy, np.shape(prm.w)[1], stride)
+    return dx, (dw, dgamma, dbeta)
+
+
+def c2f_fwd_bwd(x, params, n: int, shortcut: bool, eps: float, g_out=None) -> C2fResult:
+    """params: BlockParams in layer order cv1, m0.cv1, m0.cv2, ..., cv2.  g_out = dL/d out (None: forward only)."""
+    assert len(params) == 2 + 2 * n
+    x = np.asarray(x, dtype=np.float64)
+    f_cv1 = oracle.cbs_fwd(x, params[0].w, params[0].gamma, params[0].beta, 1, eps)
+    c = f_cv1.a.shape[-1] // 2
+    parts = [f_cv1.a[..., :c], f_cv1.a[..., c:]]
+    inner = []  # per bottleneck: (input t, fwd of cv1, fwd of cv2)
+    for i in range(n):
+        t = parts[-1]
+        f1 = oracle.cbs_fwd(t, params[1 + 2 * i].w, params[1 + 2 * i].gamma, params[1 + 2 * i].beta, 1, eps)
+        f2 = oracle.cbs_fwd(f1.a, params[2 + 2 * i].w, params[2 + 2 * i].gamma, params[2 + 2 * i].beta, 1, eps)
+        inner.append((t, f1, f2))
+        parts.append(t + f2.a if shortcut else f2.a)
+    cat = np.concatenate(parts, axis=-1)
+    f_cv2 = oracle.cbs_fwd(cat, params[-1].w, params[-1].gamma, params[-1].beta, 1, eps)
+    res = C2fResult(out=f_cv2.a, parts=parts)
+    if g_out is None:
+        return res
+    grads = [None] * len(params)
+    dcat, grads[-1] = _block_bwd(cat, params[-1], f_cv2, np.asarray(g_out, dtype=np.float64))
+    dparts = [dcat[..., j * c:(j + 1) * c].copy() for j in range(2 + n)]
+    for i in reversed(range(n)):
+        t, f1, f2 = inner[i]
+        dv = dparts[2 + i]  # complete: the concatenation's share plus whatever bottleneck i+1 added
+        du, grads[2 + 2 * i] = _block_bwd(f1.a, params[2 + 2 * i], f2, dv)
+        dt, grads[1 + 2 * i] = _block_bwd(t, params[1 + 2 * i], f1, du)
+        dparts[1 + i] = dparts[1 + i] + dt + (dv if shortcut else 0.0)
+    da0 = np.concatenate(dparts[:2], axis=-1)
+    res.dx, grads[0] = _block_bwd(x, params[0], f_cv1, da0)
+    res.grads = grads
+    return res

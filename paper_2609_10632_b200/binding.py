@@ -28,6 +28,7 @@ EXPORTS = (
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step",
+    "nb_slice_add",
 )
 
 
@@ -92,6 +93,7 @@ def load() -> ctypes.CDLL:
         lib.nb_sgd_workspace_bytes.argtypes = [V, POINTER(c_size_t)]
         lib.nb_sgd_upload.argtypes = [V, V, c_size_t, V]
         lib.nb_sgd_clip_nesterov_step.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), FP, V]
+        lib.nb_slice_add.argtypes = [c_int32, ctypes.c_int64, c_int32, V, ctypes.c_int64, V, ctypes.c_int64, V, ctypes.c_int64, c_int32, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -269,6 +271,12 @@ def nb_conv_bn_silu_step_host(plan: Plan, host_x, host_w, host_gamma, host_beta,
     _check(load().nb_conv_bn_silu_step_host(plan.handle, _ptr(host_x), _ptr(host_w), _ptr(host_gamma), _ptr(host_beta), _ptr(host_g),
                                             _ptr(host_a), _ptr(host_dx), _ptr(host_dw), _ptr(host_dgamma), _ptr(host_dbeta),
                                             _ptr(device_scratch), _nbytes(device_scratch), _stream(stream)))
+
+
+def nb_slice_add(dtype, rows, channels, out, ld_out, a, ld_a, b=None, ld_b=0, accumulate=False, stream=None):
+    """out/a/b: raw device addresses (ints) of the slices' first elements, or tensors whose data_ptr is that address."""
+    _check(load().nb_slice_add(int(dtype), int(rows), int(channels), _ptr(out), int(ld_out), _ptr(a), int(ld_a), _ptr(b), int(ld_b),
+                               1 if accumulate else 0, _stream(stream)))
 
 
 class SgdPlan:

@@ -18,6 +18,7 @@
 #include "stem_conv.cuh"
 #include "tc_conv.cuh"
 #include "sgd.cuh"
+#include "glue.cuh"
 
 using namespace nbcbs;
 
@@ -981,3 +982,44 @@ nb_status nb_sgd_clip_nesterov_step(nb_sgd_plan p, void* workspace, size_t works
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- glue between chained blocks (include/nb_glue.h)
+namespace {
+template <typename T>
+nb_status run_slice_add(void* out, long long ld_out, const void* a, long long ld_a, const void* b, long long ld_b, long long rows, int channels,
+                        int accumulate, cudaStream_t st) {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool vec = channels % V == 0 && ld_out % V == 0 && ld_a % V == 0 && (!b || ld_b % V == 0) &&
+                     !((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) & 15u);
+    const long long total = rows * (vec ? channels / V : channels);
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 8));
+    if (vec)
+        launch_k(slice_add_kernel<T, true>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a,
+                 static_cast<const T*>(b), ld_b, rows, channels, accumulate);
+    else
+        launch_k(slice_add_kernel<T, false>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a,
+                 static_cast<const T*>(b), ld_b, rows, channels, accumulate);
+    return launch_ok("slice_add");
+}
+}  // namespace
+
+extern "C" nb_status nb_slice_add(int32_t dtype, int64_t rows, int32_t channels, void* out, int64_t ld_out, const void* a, int64_t ld_a,
+                                  const void* b, int64_t ld_b, int32_t accumulate, void* stream) {
+    g_err.clear();
+    if (!out || !a) return fail(NB_ERR_INVALID_ARG, "out and a must not be NULL");
+    if (rows <= 0 || channels <= 0) return fail(NB_ERR_INVALID_ARG, "rows and channels must be positive");
+    if (ld_out < channels || ld_a < channels || (b && ld_b < channels)) return fail(NB_ERR_INVALID_ARG, "a row pitch is smaller than the channel count");
+    const size_t es = dtype == NB_DTYPE_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) & (es - 1))
+        return fail(NB_ERR_ALIGNMENT, "a pointer is not aligned to its element size");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (dtype) {
+        case NB_DTYPE_F32: return run_slice_add<float>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
+        case NB_DTYPE_BF16: return run_slice_add<__nv_bfloat16>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
+        case NB_DTYPE_F16: return run_slice_add<__half>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
+        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    }
+}

@@ -1,0 +1,68 @@
+"""Pins of the chained-block oracle (CPU only): the C2f unit's forward and backward, composed from the single-block
+oracle (pinned elsewhere) with numpy slicing.  What can go wrong here is the wiring: which part feeds which block, the
+shortcut, and the accumulation of gradients where a tensor has several consumers -- central finite differences of the
+whole unit catch all of it."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import chain
+
+RNG = np.random.default_rng(20261127)
+EPS = 1e-3
+
+
+def _params(c1, c2, n):
+    c = c2 // 2
+    shapes = [(2 * c, 1, 1, c1)] + [(c, 3, 3, c)] * (2 * n) + [(c2, 1, 1, (2 + n) * c)]
+    return [chain.BlockParams(RNG.normal(size=s) * 0.5, RNG.uniform(0.5, 1.5, s[0]), RNG.normal(size=s[0]) * 0.1) for s in shapes]
+
+
+@pytest.mark.parametrize("n,shortcut", [(1, True), (2, True), (2, False)])
+def test_whole_unit_finite_differences(n, shortcut):
+    x = RNG.normal(size=(2, 4, 3, 4))
+    prm = _params(4, 4, n)
+    G = RNG.normal(size=(2, 4, 3, 4))
+    res = chain.c2f_fwd_bwd(x, prm, n, shortcut, EPS, G)
+    loss = lambda xx, pp: float((chain.c2f_fwd_bwd(xx, pp, n, shortcut, EPS).out * G).sum())
+    h = 1e-5
+    for idx in [(0, 0, 0, 0), (1, 3, 2, 3), (0, 2, 1, 1)]:
+        xp, xm = x.copy(), x.copy()
+        xp[idx] += h
+        xm[idx] -= h
+        fd = (loss(xp, prm) - loss(xm, prm)) / (2 * h)
+        assert res.dx[idx] == pytest.approx(fd, rel=2e-5, abs=1e-7)
+    # one filter tap, one gain and one shift of every block
+    for b in range(len(prm)):
+        for name, slot in (("w", 0), ("gamma", 1), ("beta", 2)):
+            arr = getattr(prm[b], name)
+            idx = tuple(int(RNG.integers(0, d)) for d in arr.shape)
+            saved = arr[idx]
+            arr[idx] = saved + h
+            lp = loss(x, prm)
+            arr[idx] = saved - h
+            lm = loss(x, prm)
+            arr[idx] = saved
+            assert res.grads[b][slot][idx] == pytest.approx((lp - lm) / (2 * h), rel=2e-5, abs=1e-7), (b, name)
+
+
+def test_no_bottlenecks_is_two_blocks_in_sequence():
+    x = RNG.normal(size=(2, 5, 4, 6))
+    prm = _params(6, 8, 0)
+    G = RNG.normal(size=(2, 5, 4, 8))
+    res = chain.c2f_fwd_bwd(x, prm, 0, True, EPS, G)
+    first = oracle.cbs_fwd(x, prm[0].w, prm[0].gamma, prm[0].beta, 1, EPS)
+    second = oracle.cbs_fwd_bwd(first.a, prm[1].w, prm[1].gamma, prm[1].beta, G, 1, EPS)
+    np.testing.assert_allclose(res.out, second.a, rtol=1e-13)
+    np.testing.assert_allclose(res.grads[1][0], second.dw, rtol=1e-12, atol=1e-14)
+    back = oracle.bn_silu_bwd(second.dx, first.y, first.mean, first.invstd, prm[0].gamma, prm[0].beta)
+    np.testing.assert_allclose(res.dx, oracle.conv_dgrad(back[0], prm[0].w, x.shape, 1), rtol=1e-11, atol=1e-13)
+
+
+def test_shortcut_adds_the_bottleneck_input():
+    x = RNG.normal(size=(1, 4, 4, 4))
+    prm = _params(4, 4, 1)
+    with_sc = chain.c2f_fwd_bwd(x, prm, 1, True, EPS)
+    without = chain.c2f_fwd_bwd(x, prm, 1, False, EPS)
+    np.testing.assert_allclose(with_sc.parts[2] - without.parts[2], with_sc.parts[1], rtol=1e-13, atol=1e-15)
+    assert len(with_sc.parts) == 3 and with_sc.parts[0].shape[-1] == 2
