@@ -266,6 +266,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=6, help="streams of the end-to-end arm (1 = no overlap of copies and compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chain", action="store_true", help="skip the chained C2f units measurement (extra object of the JSON line)")
     ap.add_argument("--no-optimizer", action="store_true", help="skip the fused clip + SGD-Nesterov step measurement (extra object of the JSON line)")
     ap.add_argument("--no-eval-forward", action="store_true", help="skip the evaluation-mode forward measurement (extra object of the JSON line)")
     ap.add_argument("--no-profile", action="store_true")
@@ -447,6 +448,11 @@ def main():
     if not args.no_optimizer and args.workload == "cfg5":
         opt_step = run_optimizer_step(args, blocks, dev, local, peaks)
 
+    # ---------------- the backbone's four C2f units as chained blocks (split / add / concat glue included)
+    chain = None
+    if not args.no_chain and args.workload == "cfg5":
+        chain = run_c2f_chains(args, dev, local, peaks)
+
     # ---------------- end to end from pinned host buffers through the C ABI
     e2e = None
     if not args.no_e2e:
@@ -474,7 +480,7 @@ def main():
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },
             "clocks": clocks.summary(), "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernels, "eval_forward": eval_fwd, "optimizer_step": opt_step,
+            "kernels": kernels, "eval_forward": eval_fwd, "optimizer_step": opt_step, "c2f_chain": chain,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -525,6 +531,56 @@ def run_eval_forward(args, blocks, dev, fwd_flops, peaks, kernels):
     return {"call": "nb_conv_bn_silu_infer", "ms_per_pass": ms, "tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"],
             "launches_per_pass": int(launches), "fused_layers": sum(1 for b in blocks if b.plan.infer_fused), "layers": len(blocks),
             "training_forward_kernels_ms": train_fwd, "cuda_graph": True}
+
+
+def run_c2f_chains(args, dev, local, peaks):
+    """The four C2f units of the backbone (96/192/384/576 channels at 160/80/40/20 pixels, 2/4/4/2 bottlenecks with
+    shortcut) run as CHAINS: each block consumes the previous block's activations and gradients, joined by nb_slice_add
+    (split, residual add, concat, gradient accumulation).  Forward + backward of all four as one CUDA-graph replay."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.c2f import C2fChain
+
+    units = [C2fChain(16, h, h, c, c, n, True, device=local) for c, h, n in ((96, 160, 2), (192, 80, 4), (384, 40, 4), (576, 20, 2))]
+    flops = 0.0
+    for u in units:
+        for i, b in enumerate(u.blocks):
+            b.fill_random(seed=5000 + i)
+            flops += 3.0 * b.shape.gemm_flops
+        u.cv2.g.normal_()
+
+    def step():
+        for u in units:
+            u.forward()
+            u.backward()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    for u in units:
+        u.poll()
+    l0 = nb.nb_cbs_launch_count()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    launches = nb.nb_cbs_launch_count() - l0
+    graph.replay()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    for u in units:
+        u.poll()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    nblocks = sum(len(u.blocks) for u in units)
+    glue = sum(2 + 4 * u.n for u in units)  # forward: 1 + 2n, backward: 2n + 1
+    return {"units": "backbone C2f x4 (96@160 n2, 192@80 n4, 384@40 n4, 576@20 n2), batch 16, shortcut", "conv_bn_silu_blocks": nblocks,
+            "glue_launches": glue, "launches_per_step": int(launches), "ms_per_step": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+            "frac_of_measured_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "cuda_graph": True}
 
 
 def run_optimizer_step(args, blocks, dev, local, peaks):
