@@ -77,3 +77,44 @@ def c2f_fwd_bwd(x, params, n: int, shortcut: bool, eps: float, g_out=None) -> C2
     res.dx, grads[0] = _block_bwd(x, params[0], f_cv1, da0)
     res.grads = grads
     return res
+
+
+# ------------------------------------------------------------------ the other glue of the detector (Sec. 6): SPPF, upsampling
+def maxpool5(x):
+    """5x5 max-pool, stride 1, padding 2 (padding never wins), NHWC.  Returns (y, idx) with idx = r*5 + t of the FIRST
+    maximum of the window in row-major order (r, t = offsets 0..4 from the window's top-left corner at (p-2, q-2))."""
+    x = np.asarray(x, dtype=np.float64)
+    N, H, W, C = x.shape
+    y = np.full_like(x, -np.inf)
+    idx = np.zeros(x.shape, dtype=np.int64)
+    for r in range(5):
+        for t in range(5):
+            shifted = np.full_like(x, -np.inf)
+            h0, h1 = max(0, 2 - r), min(H, H + 2 - r)  # output rows p with 0 <= p - 2 + r < H
+            w0, w1 = max(0, 2 - t), min(W, W + 2 - t)
+            shifted[:, h0:h1, w0:w1, :] = x[:, h0 - 2 + r:h1 - 2 + r, w0 - 2 + t:w1 - 2 + t, :]
+            better = shifted > y  # strict: an equal later element does not replace the first maximum
+            y = np.where(better, shifted, y)
+            idx = np.where(better, r * 5 + t, idx)
+    return y, idx
+
+
+def maxpool5_bwd(g, idx):
+    """Gradient of maxpool5: every output's gradient goes to the input element its window's first maximum came from."""
+    g = np.asarray(g, dtype=np.float64)
+    N, H, W, C = g.shape
+    dx = np.zeros_like(g)
+    n, p, q, c = np.meshgrid(np.arange(N), np.arange(H), np.arange(W), np.arange(C), indexing="ij")
+    np.add.at(dx, (n, p - 2 + idx // 5, q - 2 + idx % 5, c), g)
+    return dx
+
+
+def upsample2(x):
+    """Nearest-neighbour 2x upsampling, NHWC: y[n, 2h+a, 2w+b, c] = x[n, h, w, c]."""
+    return np.repeat(np.repeat(np.asarray(x, dtype=np.float64), 2, axis=1), 2, axis=2)
+
+
+def upsample2_bwd(g):
+    g = np.asarray(g, dtype=np.float64)
+    N, H2, W2, C = g.shape
+    return g.reshape(N, H2 // 2, 2, W2 // 2, 2, C).sum(axis=(2, 4))

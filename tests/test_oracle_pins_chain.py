@@ -66,3 +66,49 @@ def test_shortcut_adds_the_bottleneck_input():
     without = chain.c2f_fwd_bwd(x, prm, 1, False, EPS)
     np.testing.assert_allclose(with_sc.parts[2] - without.parts[2], with_sc.parts[1], rtol=1e-13, atol=1e-15)
     assert len(with_sc.parts) == 3 and with_sc.parts[0].shape[-1] == 2
+
+
+def test_maxpool5_against_brute_force_and_library_filter():
+    from scipy.ndimage import maximum_filter
+
+    x = RNG.normal(size=(2, 7, 6, 3))
+    y, idx = chain.maxpool5(x)
+    # library routine: a 5x5 maximum filter over H and W with -inf outside
+    want = maximum_filter(x, size=(1, 5, 5, 1), mode="constant", cval=-np.inf)
+    np.testing.assert_array_equal(y, want)
+    # brute force incl. the index convention
+    for n, p, q, c in [(0, 0, 0, 0), (1, 6, 5, 2), (0, 3, 2, 1), (1, 0, 5, 0)]:
+        best, bi = -np.inf, -1
+        for r in range(5):
+            for t in range(5):
+                h, w = p - 2 + r, q - 2 + t
+                if 0 <= h < 7 and 0 <= w < 6 and x[n, h, w, c] > best:
+                    best, bi = x[n, h, w, c], r * 5 + t
+        assert y[n, p, q, c] == best and idx[n, p, q, c] == bi
+
+
+def test_maxpool5_ties_go_to_the_first_element_and_gradient_is_the_adjoint():
+    x = np.zeros((1, 5, 5, 1))  # all equal: every window's first in-bounds element wins
+    y, idx = chain.maxpool5(x)
+    assert idx[0, 2, 2, 0] == 0 and idx[0, 0, 0, 0] == 2 * 5 + 2
+    g = RNG.normal(size=(2, 6, 5, 4))
+    x = RNG.normal(size=(2, 6, 5, 4))
+    y, idx = chain.maxpool5(x)
+    dx = chain.maxpool5_bwd(g, idx)
+    assert dx.sum() == pytest.approx(g.sum(), rel=1e-12)
+    # directional derivative: moving x by a small v changes sum(y*g) by <dx, v> (no ties in random data)
+    v = RNG.normal(size=x.shape)
+    h = 1e-7
+    fd = ((chain.maxpool5(x + h * v)[0] - chain.maxpool5(x - h * v)[0]) * g).sum() / (2 * h)
+    assert (dx * v).sum() == pytest.approx(fd, rel=1e-6)
+
+
+def test_upsample2_and_its_adjoint():
+    x = RNG.normal(size=(2, 3, 4, 5))
+    y = chain.upsample2(x)
+    assert y.shape == (2, 6, 8, 5)
+    for a in (0, 1):
+        for b in (0, 1):
+            np.testing.assert_array_equal(y[:, a::2, b::2, :], x)
+    g = RNG.normal(size=y.shape)
+    assert (chain.upsample2_bwd(g) * x).sum() == pytest.approx((g * y).sum(), rel=1e-12)
