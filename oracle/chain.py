@@ -118,3 +118,40 @@ def upsample2_bwd(g):
     g = np.asarray(g, dtype=np.float64)
     N, H2, W2, C = g.shape
     return g.reshape(N, H2 // 2, 2, W2 // 2, 2, C).sum(axis=(2, 4))
+
+
+def round_bf16(a):
+    """Round fp64 values to the nearest bf16 (ties to even), returned as fp64: the storage precision of activations."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    bits = f.view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return bits.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(a))
+
+
+def sppf_fwd_bwd(x, params, eps: float, g_out=None, pool_in_bf16: bool = False):
+    """SPPF unit (Sec. 6): a0 = CBS_1x1(x); p1 = pool(a0); p2 = pool(p1); p3 = pool(p2); out = CBS_1x1(concat(a0, p1, p2, p3)).
+    Returns (out, parts, dx, grads) with grads per block (cv1, cv2) = (dw, dgamma, dbeta); dx, grads None without g_out.
+
+    pool_in_bf16: which element of a window is the maximum is an integer decision taken on floating-point values; a
+    16-bit implementation takes it on bf16-rounded activations, where near-equal candidates become exact ties (first
+    one wins).  With this flag the first block's activations are rounded to bf16 before the pools, so that both sides
+    decide in the same precision; everything else stays fp64."""
+    assert len(params) == 2
+    x = np.asarray(x, dtype=np.float64)
+    f1 = oracle.cbs_fwd(x, params[0].w, params[0].gamma, params[0].beta, 1, eps)
+    parts, idxs = [round_bf16(f1.a) if pool_in_bf16 else f1.a], []
+    for _ in range(3):
+        y, idx = maxpool5(parts[-1])
+        parts.append(y)
+        idxs.append(idx)
+    cat = np.concatenate(parts, axis=-1)
+    f2 = oracle.cbs_fwd(cat, params[1].w, params[1].gamma, params[1].beta, 1, eps)
+    if g_out is None:
+        return f2.a, parts, None, None
+    c = f1.a.shape[-1]
+    dcat, g2 = _block_bwd(cat, params[1], f2, np.asarray(g_out, dtype=np.float64))
+    d = [dcat[..., j * c:(j + 1) * c].copy() for j in range(4)]
+    for j in (3, 2, 1):  # part j = pool(part j-1): its complete gradient flows back into part j-1
+        d[j - 1] += maxpool5_bwd(d[j], idxs[j - 1])
+    dx, g1 = _block_bwd(x, params[0], f1, d[0])
+    return f2.a, parts, dx, [g1, g2]

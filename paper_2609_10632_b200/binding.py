@@ -28,7 +28,7 @@ EXPORTS = (
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step",
-    "nb_slice_add",
+    "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2",
 )
 
 
@@ -94,6 +94,9 @@ def load() -> ctypes.CDLL:
         lib.nb_sgd_upload.argtypes = [V, V, c_size_t, V]
         lib.nb_sgd_clip_nesterov_step.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), FP, V]
         lib.nb_slice_add.argtypes = [c_int32, ctypes.c_int64, c_int32, V, ctypes.c_int64, V, ctypes.c_int64, V, ctypes.c_int64, c_int32, V]
+        lib.nb_maxpool5_fwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, V]
+        lib.nb_maxpool5_bwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, c_int32, V]
+        lib.nb_upsample2.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, c_int32, c_int32, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -277,6 +280,19 @@ def nb_slice_add(dtype, rows, channels, out, ld_out, a, ld_a, b=None, ld_b=0, ac
     """out/a/b: raw device addresses (ints) of the slices' first elements, or tensors whose data_ptr is that address."""
     _check(load().nb_slice_add(int(dtype), int(rows), int(channels), _ptr(out), int(ld_out), _ptr(a), int(ld_a), _ptr(b), int(ld_b),
                                1 if accumulate else 0, _stream(stream)))
+
+
+def nb_maxpool5_fwd(dtype, n, h, w, c, x, y, idx=None, stream=None):
+    _check(load().nb_maxpool5_fwd(int(dtype), n, h, w, c, _ptr(x), _ptr(y), _ptr(idx), _stream(stream)))
+
+
+def nb_maxpool5_bwd(dtype, n, h, w, c, g, idx, dx, accumulate=False, stream=None):
+    _check(load().nb_maxpool5_bwd(int(dtype), n, h, w, c, _ptr(g), _ptr(idx), _ptr(dx), 1 if accumulate else 0, _stream(stream)))
+
+
+def nb_upsample2(dtype, n, h, w, c, src, dst, backward=False, accumulate=False, stream=None):
+    """(n, h, w, c) are the extents of the SMALL tensor."""
+    _check(load().nb_upsample2(int(dtype), n, h, w, c, _ptr(src), _ptr(dst), 1 if backward else 0, 1 if accumulate else 0, _stream(stream)))
 
 
 class SgdPlan:

@@ -85,3 +85,56 @@ class C2fChain:
     def poll(self):
         for b in self.blocks:
             b.poll()
+
+
+class SppfChain:
+    """The SPPF unit: 1x1 block, three chained 5x5 max-pools, concatenation of the four parts, 1x1 block; forward and
+    backward.  Each pool writes a dense part buffer (the pool kernels take dense tensors); nb_slice_add moves the parts
+    into, and the gradients out of, the concatenation buffer."""
+
+    def __init__(self, batch, h, w, c1, c2, eps=1e-3, device=0):
+        c = c1 // 2
+        self.c, self.dims = c, (batch, h, w, c)
+        shape = lambda name, ci, co: wl.ConvShape(name, batch, h, w, ci, co, 1, 1)
+        self.cv1 = CbsBlock(shape("cv1", c1, c), eps=eps, device=device)
+        self.cv2 = CbsBlock(shape("cv2", 4 * c, c2), eps=eps, device=device)
+        self.rows = batch * h * w
+        dev = self.cv1.dev
+        self.pool = [torch.empty(batch, h, w, c, dtype=torch.bfloat16, device=dev) for _ in range(3)]
+        self.idx = [torch.empty(batch, h, w, c, dtype=torch.uint8, device=dev) for _ in range(3)]
+        self.dpart = [torch.empty(batch, h, w, c, dtype=torch.bfloat16, device=dev) for _ in range(4)]  # dense gradients of the parts
+        self.cat, self.dcat = self.cv2.x, self.cv2.dx
+
+    @property
+    def blocks(self):
+        return [self.cv1, self.cv2]
+
+    def _slice(self, t, first_channel):
+        return t.data_ptr() + first_channel * t.element_size()
+
+    def forward(self, stream=None):
+        n, h, w, c = self.dims
+        self.cv1.forward(stream)
+        src = self.cv1.a
+        nb.nb_slice_add(nb.NB_DTYPE_BF16, self.rows, c, self._slice(self.cat, 0), 4 * c, src, c, stream=stream)
+        for j in range(3):
+            nb.nb_maxpool5_fwd(nb.NB_DTYPE_BF16, n, h, w, c, src, self.pool[j], self.idx[j], stream)
+            nb.nb_slice_add(nb.NB_DTYPE_BF16, self.rows, c, self._slice(self.cat, (1 + j) * c), 4 * c, self.pool[j], c, stream=stream)
+            src = self.pool[j]
+        self.cv2.forward(stream)
+
+    def backward(self, stream=None):
+        n, h, w, c = self.dims
+        self.cv2.backward_data(stream)
+        self.cv2.backward_weight(stream)
+        for j in range(4):
+            nb.nb_slice_add(nb.NB_DTYPE_BF16, self.rows, c, self.dpart[j], c, self._slice(self.dcat, j * c), 4 * c, stream=stream)
+        for j in (3, 2, 1):  # part j = pool(part j-1)
+            nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, self.dpart[j], self.idx[j - 1], self.dpart[j - 1], True, stream)
+        self.cv1.g = self.dpart[0]
+        self.cv1.backward_data(stream)
+        self.cv1.backward_weight(stream)
+
+    def poll(self):
+        for b in self.blocks:
+            b.poll()

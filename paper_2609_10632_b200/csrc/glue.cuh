@@ -42,3 +42,119 @@ __global__ void __launch_bounds__(256) slice_add_kernel(T* __restrict__ out, lon
 }
 
 }  // namespace nbcbs
+
+namespace nbcbs {
+
+// 5x5 max-pool, stride 1, padding 2 over NHWC (the SPPF unit chains three of them).  One thread per 8-channel (16-byte)
+// vector of an output pixel, or per element when C % 8 != 0.  idx (optional, one byte per element) = r*5 + t of the FIRST
+// maximum of the window in row-major order: comparisons are strict, elements outside the image never win.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, uint8_t* __restrict__ idx, int N, int H, int W, int C) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int cv = C / V;
+    const long long total = (long long)N * H * W * cv;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % cv) * V;
+        long long t1 = i / cv;
+        const int q = (int)(t1 % W);
+        t1 /= W;
+        const int p = (int)(t1 % H);
+        const long long n = t1 / H;
+        float best[V];
+        int bi[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            best[k] = -__int_as_float(0x7f800000);
+            bi[k] = 0;
+        }
+        for (int r = 0; r < 5; ++r) {
+            const int h = p - 2 + r;
+            if (h < 0 || h >= H) continue;
+            for (int t = 0; t < 5; ++t) {
+                const int w = q - 2 + t;
+                if (w < 0 || w >= W) continue;
+                const T* src = x + (((n * H + h) * W + w) * (long long)C + c);
+                T v[V];
+                if (V == 8) *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(src); else v[0] = src[0];
+#pragma unroll
+                for (int k = 0; k < V; ++k) {
+                    const float f = to_f32(v[k]);
+                    if (f > best[k]) {
+                        best[k] = f;
+                        bi[k] = r * 5 + t;
+                    }
+                }
+            }
+        }
+        const long long o = ((n * H + p) * W + q) * (long long)C + c;
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            y[o + k] = from_f32<T>(best[k]);  // the maximum of stored values is itself a stored value: exact
+            if (idx) idx[o + k] = (uint8_t)bi[k];
+        }
+    }
+}
+
+// dx[n][h][w][c] = sum of g over the (at most 25) windows whose recorded maximum is this element; fp32 sum in fixed
+// (row-major window) order, one rounding.  accumulate != 0 adds the result to dx instead of overwriting it.
+template <typename T>
+__global__ void __launch_bounds__(256) maxpool5_bwd_kernel(const T* __restrict__ g, const uint8_t* __restrict__ idx, T* __restrict__ dx, int N, int H, int W,
+                                                           int C, int accumulate) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long total = (long long)N * H * W * C;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C);
+        long long t1 = i / C;
+        const int w = (int)(t1 % W);
+        t1 /= W;
+        const int h = (int)(t1 % H);
+        const long long n = t1 / H;
+        float s = 0.f;
+        for (int r = 4; r >= 0; --r) {      // window at output row p = h + 2 - r sees this element at offset r
+            const int p = h + 2 - r;
+            if (p < 0 || p >= H) continue;
+            for (int t = 4; t >= 0; --t) {
+                const int q = w + 2 - t;
+                if (q < 0 || q >= W) continue;
+                const long long o = ((n * H + p) * W + q) * (long long)C + c;
+                if (idx[o] == r * 5 + t) s += to_f32(g[o]);
+            }
+        }
+        if (accumulate) s += to_f32(dx[i]);
+        dx[i] = from_f32<T>(s);
+    }
+}
+
+// Nearest-neighbour 2x upsampling y[n][2h+a][2w+b][c] = x[n][h][w][c] (BWD = false), and its adjoint
+// dx[n][h][w][c] = sum of the four g (BWD = true; fp32 sum, one rounding; accumulate adds to dx).  x / dx is [N][H][W][C].
+template <typename T, bool BWD>
+__global__ void __launch_bounds__(256) upsample2_kernel(const T* __restrict__ src, T* __restrict__ dst, int N, int H, int W, int C, int accumulate) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long total = (long long)N * H * W * C;
+    const long long row2 = 2LL * W * C;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C);
+        long long t1 = i / C;
+        const int w = (int)(t1 % W);
+        t1 /= W;
+        const int h = (int)(t1 % H);
+        const long long n = t1 / H;
+        const long long o = ((n * 2 * H + 2 * h) * 2 * W + 2 * w) * (long long)C + c;  // (2h, 2w) in the large tensor
+        if (BWD) {
+            float s = (to_f32(src[o]) + to_f32(src[o + C])) + (to_f32(src[o + row2]) + to_f32(src[o + row2 + C]));
+            if (accumulate) s += to_f32(dst[i]);
+            dst[i] = from_f32<T>(s);
+        } else {
+            const T v = src[i];
+            dst[o] = v;
+            dst[o + C] = v;
+            dst[o + row2] = v;
+            dst[o + row2 + C] = v;
+        }
+    }
+}
+
+}  // namespace nbcbs

@@ -1023,3 +1023,83 @@ extern "C" nb_status nb_slice_add(int32_t dtype, int64_t rows, int32_t channels,
         default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     }
 }
+
+namespace {
+unsigned glue_blocks(long long total) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 8));
+}
+nb_status check_nhwc(int32_t n, int32_t h, int32_t w, int32_t c) {
+    if (n <= 0 || h <= 0 || w <= 0 || c <= 0) return fail(NB_ERR_INVALID_ARG, "extents must be positive");
+    return NB_OK;
+}
+template <typename T>
+nb_status run_maxpool_fwd(const void* x, void* y, uint8_t* idx, int n, int h, int w, int c, cudaStream_t st) {
+    const bool vec = sizeof(T) == 2 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u);
+    if (vec) {
+        const long long total = (long long)n * h * w * (c / 8);
+        launch_k(maxpool5_fwd_kernel<T, 8>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
+    } else {
+        const long long total = (long long)n * h * w * c;
+        launch_k(maxpool5_fwd_kernel<T, 1>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
+    }
+    return launch_ok("maxpool5_fwd");
+}
+}  // namespace
+
+extern "C" {
+
+nb_status nb_maxpool5_fwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* x, void* y, uint8_t* idx, void* stream) {
+    g_err.clear();
+    if (!x || !y) return fail(NB_ERR_INVALID_ARG, "x and y must not be NULL");
+    NB_TRY(check_nhwc(n, h, w, c));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (dtype) {
+        case NB_DTYPE_F32: return run_maxpool_fwd<float>(x, y, idx, n, h, w, c, st);
+        case NB_DTYPE_BF16: return run_maxpool_fwd<__nv_bfloat16>(x, y, idx, n, h, w, c, st);
+        case NB_DTYPE_F16: return run_maxpool_fwd<__half>(x, y, idx, n, h, w, c, st);
+        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    }
+}
+
+nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* g, const uint8_t* idx, void* dx, int32_t accumulate,
+                          void* stream) {
+    g_err.clear();
+    if (!g || !idx || !dx) return fail(NB_ERR_INVALID_ARG, "g, idx and dx must not be NULL");
+    NB_TRY(check_nhwc(n, h, w, c));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned blocks = glue_blocks((long long)n * h * w * c);
+    switch (dtype) {
+        case NB_DTYPE_F32: launch_k(maxpool5_bwd_kernel<float>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const float*>(g), idx, static_cast<float*>(dx), n, h, w, c, accumulate != 0); break;
+        case NB_DTYPE_BF16: launch_k(maxpool5_bwd_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(g), idx, static_cast<__nv_bfloat16*>(dx), n, h, w, c, accumulate != 0); break;
+        case NB_DTYPE_F16: launch_k(maxpool5_bwd_kernel<__half>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __half*>(g), idx, static_cast<__half*>(dx), n, h, w, c, accumulate != 0); break;
+        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    }
+    return launch_ok("maxpool5_bwd");
+}
+
+nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* src, void* dst, int32_t backward, int32_t accumulate,
+                       void* stream) {
+    g_err.clear();
+    if (!src || !dst) return fail(NB_ERR_INVALID_ARG, "src and dst must not be NULL");
+    NB_TRY(check_nhwc(n, h, w, c));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned blocks = glue_blocks((long long)n * h * w * c);
+#define NB_UPS(T)                                                                                                                              \
+    do {                                                                                                                                       \
+        if (backward) launch_k(upsample2_kernel<T, true>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0); \
+        else launch_k(upsample2_kernel<T, false>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, 0);                    \
+    } while (0)
+    switch (dtype) {
+        case NB_DTYPE_F32: NB_UPS(float); break;
+        case NB_DTYPE_BF16: NB_UPS(__nv_bfloat16); break;
+        case NB_DTYPE_F16: NB_UPS(__half); break;
+        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    }
+#undef NB_UPS
+    return launch_ok("upsample2");
+}
+
+}  // extern "C"

@@ -102,3 +102,120 @@ def test_c2f_unit_matches_chained_oracle(n, shortcut, c1, c2):
         _check(f"block{i}.dgamma", f64(blk.dgamma), dgamma, report)
         _check(f"block{i}.dbeta", f64(blk.dbeta), dbeta, report)
     print("\n".join(report))
+
+
+@pytest.mark.parametrize("dtype_name,n,h,w,c", [("bfloat16", 2, 9, 7, 16), ("bfloat16", 1, 5, 6, 3), ("float32", 2, 6, 6, 5), ("float16", 1, 20, 20, 8)])
+def test_maxpool5_forward_backward(dtype_name, n, h, w, c):
+    """Values and recorded positions bit-exact (bf16 data has many ties: the first maximum must win on both sides);
+    gradient within one rounding of the exact scatter-sum."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    dt = getattr(torch, dtype_name)
+    code = {"float32": nb.NB_DTYPE_F32, "bfloat16": nb.NB_DTYPE_BF16, "float16": nb.NB_DTYPE_F16}[dtype_name]
+    rng = np.random.Generator(np.random.Philox(key=[42, n * 100 + c]))
+    dev = torch.device("cuda", 0)
+    x = torch.from_numpy(rng.standard_normal((n, h, w, c)).astype(np.float32)).to(dt)
+    if dtype_name == "bfloat16":
+        x = (x.float() * 4).round().div(4).to(dt)  # quarter steps: plenty of exact ties
+    g = torch.from_numpy(rng.standard_normal((n, h, w, c)).astype(np.float32)).to(dt)
+    xd, gd = x.to(dev), g.to(dev)
+    y, idx, dx = torch.empty_like(xd), torch.empty(n, h, w, c, dtype=torch.uint8, device=dev), torch.empty_like(xd)
+    nb.nb_maxpool5_fwd(code, n, h, w, c, xd, y, idx)
+    nb.nb_maxpool5_bwd(code, n, h, w, c, gd, idx, dx)
+    torch.cuda.synchronize()
+    ref_y, ref_idx = chain.maxpool5(x.double().numpy())
+    np.testing.assert_array_equal(y.double().cpu().numpy(), ref_y)
+    np.testing.assert_array_equal(idx.cpu().numpy().astype(np.int64), ref_idx)
+    ref_dx = chain.maxpool5_bwd(g.double().numpy(), ref_idx)
+    ulp = {"float32": 2.0 ** -23, "bfloat16": 2.0 ** -8, "float16": 2.0 ** -10}[dtype_name]
+    # up to 25 terms: in fp32 the running sum rounds after every term (error <= 25 ulp of the largest partial sum);
+    # 16-bit terms add exactly in fp32, so those results are one rounding away from the exact sum
+    atol = 25 * ulp * float(np.abs(g.double().numpy()).max()) * 5 if dtype_name == "float32" else ulp * 1e-3
+    np.testing.assert_allclose(dx.double().cpu().numpy(), ref_dx, rtol=ulp, atol=atol)
+    # accumulate: dx += the same gradient again
+    nb.nb_maxpool5_bwd(code, n, h, w, c, gd, idx, dx, accumulate=True)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(dx.double().cpu().numpy(), 2 * ref_dx, rtol=4 * ulp, atol=2 * atol)
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float32"])
+def test_upsample2_forward_and_adjoint(dtype_name):
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    dt = getattr(torch, dtype_name)
+    code = {"float32": nb.NB_DTYPE_F32, "bfloat16": nb.NB_DTYPE_BF16}[dtype_name]
+    n, h, w, c = 2, 5, 7, 12
+    rng = np.random.Generator(np.random.Philox(key=[43, 1]))
+    dev = torch.device("cuda", 0)
+    x = torch.from_numpy(rng.standard_normal((n, h, w, c)).astype(np.float32)).to(dt).to(dev)
+    g = torch.from_numpy(rng.standard_normal((n, 2 * h, 2 * w, c)).astype(np.float32)).to(dt).to(dev)
+    y, dx = torch.empty(n, 2 * h, 2 * w, c, dtype=dt, device=dev), torch.empty_like(x)
+    nb.nb_upsample2(code, n, h, w, c, x, y)
+    nb.nb_upsample2(code, n, h, w, c, g, dx, backward=True)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(y.double().cpu().numpy(), chain.upsample2(x.double().cpu().numpy()))
+    ref = chain.upsample2_bwd(g.double().cpu().numpy())
+    if dtype_name == "bfloat16":  # four 16-bit values sum exactly in fp32: the result is the correctly rounded exact sum
+        assert torch.equal(dx, torch.from_numpy(ref).to(dt).to(dev))
+    else:
+        np.testing.assert_allclose(dx.double().cpu().numpy(), ref, rtol=1e-6, atol=2e-6)  # three fp32 additions with cancellation
+
+
+def test_sppf_unit_matches_chained_oracle():
+    import torch
+
+    from paper_2609_10632_b200.c2f import SppfChain
+
+    ch = SppfChain(2, 20, 20, 64, 64, eps=EPS)
+    params, inputs = [], []
+    for i, blk in enumerate(ch.blocks):
+        inp = wl.make_inputs(blk.shape, 52, i, bf16=True, affine="random")
+        inputs.append(inp)
+        params.append(chain.BlockParams(inp.w, inp.gamma, inp.beta))
+        for name in ("w", "gamma", "beta"):
+            dst = getattr(blk, name)
+            dst.copy_(torch.from_numpy(np.ascontiguousarray(getattr(inp, name))).to(dst.dtype))
+    x, g_out = inputs[0].x, inputs[1].g
+    ch.cv1.x.copy_(torch.from_numpy(x).to(torch.bfloat16))
+    ch.cv2.g.copy_(torch.from_numpy(g_out).to(torch.bfloat16))
+    ch.forward()
+    ch.backward()
+    torch.cuda.synchronize()
+    ch.poll()
+    # which window element is the maximum is decided on bf16 activations on the GPU: the oracle decides in the same precision
+    out, parts, dx, grads = chain.sppf_fwd_bwd(x, params, EPS, g_out, pool_in_bf16=True)
+    f64 = lambda t: t.detach().double().cpu().numpy()
+    report = []
+    # unique results: the forward and everything of the backward that does not pass through a pool
+    _check("out", f64(ch.cv2.a), out, report)
+    cat = f64(ch.cat)
+    for j, part in enumerate(parts):
+        _check(f"part{j}", cat[..., j * ch.c:(j + 1) * ch.c], part, report)
+    _check("cv2.dw", f64(ch.cv2.dw), grads[1][0], report)
+    _check("cv2.dgamma", f64(ch.cv2.dgamma), grads[1][1], report)
+    _check("cv2.dbeta", f64(ch.cv2.dbeta), grads[1][2], report)
+    # The gradient behind the pools is NOT unique: the GPU's activations differ from the oracle's by a bf16 ulp in many
+    # elements (they pass through the fp16 convolution output), so a few per cent of the windows have a different, equally
+    # valid maximum position and their gradient lands on a neighbouring pixel.  Checked instead: (1) every recorded
+    # position IS the first maximum of the GPU's own window (the decision is valid), (2) the pools' gradient routing
+    # conserves the gradient mass per channel, (3) the results stay close to the oracle's (loose bar).
+    src = f64(ch.cv1.a)
+    for j in range(3):
+        want_y, want_idx = chain.maxpool5(src)
+        np.testing.assert_array_equal(f64(ch.pool[j]), want_y)
+        np.testing.assert_array_equal(ch.idx[j].cpu().numpy().astype(np.int64), want_idx)
+        src = want_y
+    dcat = f64(ch.dcat)
+    mass = sum(dcat[..., j * ch.c:(j + 1) * ch.c].sum(axis=(0, 1, 2)) for j in range(4))
+    l1 = sum(np.abs(dcat[..., j * ch.c:(j + 1) * ch.c]).sum(axis=(0, 1, 2)) for j in range(4))
+    # every stored gradient value carries a bf16 rounding (2^-9 relative), three accumulations deep
+    np.testing.assert_allclose(f64(ch.dpart[0]).sum(axis=(0, 1, 2)), mass, rtol=0, atol=float((4 * 2.0 ** -9 * l1).max()))
+    for name, got, ref in (("dx", ch.cv1.dx, dx), ("cv1.dw", ch.cv1.dw, grads[0][0]), ("cv1.dgamma", ch.cv1.dgamma, grads[0][1]), ("cv1.dbeta", ch.cv1.dbeta, grads[0][2])):
+        r = parity.rel_l2(f64(got), ref)
+        report.append(f"{name} (behind the pools): rel_l2={r:.2e}")
+        assert r <= 0.1, name
+    print("\n".join(report))

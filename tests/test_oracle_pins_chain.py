@@ -112,3 +112,36 @@ def test_upsample2_and_its_adjoint():
             np.testing.assert_array_equal(y[:, a::2, b::2, :], x)
     g = RNG.normal(size=y.shape)
     assert (chain.upsample2_bwd(g) * x).sum() == pytest.approx((g * y).sum(), rel=1e-12)
+
+
+def test_sppf_unit_finite_differences():
+    x = RNG.normal(size=(1, 6, 6, 4))
+    prm = [chain.BlockParams(RNG.normal(size=(2, 1, 1, 4)) * 0.7, RNG.uniform(0.5, 1.5, 2), RNG.normal(size=2) * 0.1),
+           chain.BlockParams(RNG.normal(size=(4, 1, 1, 8)) * 0.5, RNG.uniform(0.5, 1.5, 4), RNG.normal(size=4) * 0.1)]
+    G = RNG.normal(size=(1, 6, 6, 4))
+    out, parts, dx, grads = chain.sppf_fwd_bwd(x, prm, EPS, G)
+    assert len(parts) == 4 and out.shape == G.shape
+    loss = lambda xx: float((chain.sppf_fwd_bwd(xx, prm, EPS)[0] * G).sum())
+    h = 1e-6
+    for idx in [(0, 0, 0, 0), (0, 3, 2, 1), (0, 5, 5, 3)]:
+        xp, xm = x.copy(), x.copy()
+        xp[idx] += h
+        xm[idx] -= h
+        assert dx[idx] == pytest.approx((loss(xp) - loss(xm)) / (2 * h), rel=1e-4, abs=1e-7)
+    w = prm[0].w
+    saved = w[1, 0, 0, 2]
+    w[1, 0, 0, 2] = saved + h
+    lp = loss(x)
+    w[1, 0, 0, 2] = saved - h
+    lm = loss(x)
+    w[1, 0, 0, 2] = saved
+    assert grads[0][0][1, 0, 0, 2] == pytest.approx((lp - lm) / (2 * h), rel=1e-4, abs=1e-7)
+
+
+def test_round_bf16_is_nearest_even_on_known_values():
+    # 1 + 2^-8 lies halfway between 1 and 1 + 2^-7: ties go to the even mantissa (1.0); 1 + 3*2^-8 goes up to 1 + 2^-6
+    vals = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -2.5, 0.0, 3.0e-5])
+    got = chain.round_bf16(vals)
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == 1.0 + 2.0 ** -6 and got[3] == 1.0 + 2.0 ** -7 and got[4] == -2.5 and got[5] == 0.0
+    assert abs(got[6] - 3.0e-5) <= 3.0e-5 * 2.0 ** -8
+    assert np.array_equal(chain.round_bf16(got), got)
