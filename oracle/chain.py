@@ -155,3 +155,73 @@ def sppf_fwd_bwd(x, params, eps: float, g_out=None, pool_in_bf16: bool = False):
         d[j - 1] += maxpool5_bwd(d[j], idxs[j - 1])
     dx, g1 = _block_bwd(x, params[0], f1, d[0])
     return f2.a, parts, dx, [g1, g2]
+
+
+# ------------------------------------------------------------------ a whole dataflow graph of blocks and glue
+def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf16: bool = False):
+    """Interpret a dataflow description (a list of op dicts: "cbs" with a layer index, "slice", "add", "concat", "maxpool",
+    "upsample"; see the detector's description in the workload module) forwards and, given gradients for some tensors,
+    backwards.  layers[k] gives block k's stride; params[k] its BlockParams.  A tensor with several consumers receives
+    the sum of their gradients.  Returns (tensors, grads, block_grads): dicts name -> array, and per layer (dw, dgamma, dbeta).
+    pool_in_bf16: inputs of max-pools are rounded to bf16 first (see sppf_fwd_bwd)."""
+    T = {"img": np.asarray(x, dtype=np.float64)}
+    saved = {}
+    for o in ops:
+        ins = [T[i] for i in o["ins"]]
+        kind = o["op"]
+        if kind == "cbs":
+            k = o["layer"]
+            f = oracle.cbs_fwd(ins[0], params[k].w, params[k].gamma, params[k].beta, layers[k].stride, eps)
+            saved[o["out"]] = f
+            T[o["out"]] = f.a
+        elif kind == "slice":
+            T[o["out"]] = ins[0][..., o["c0"]:o["c1"]]
+        elif kind == "add":
+            T[o["out"]] = ins[0] + ins[1]
+        elif kind == "concat":
+            T[o["out"]] = np.concatenate(ins, axis=-1)
+        elif kind == "maxpool":
+            src = round_bf16(ins[0]) if pool_in_bf16 else ins[0]
+            T[o["out"]], saved[o["out"]] = maxpool5(src)
+        elif kind == "upsample":
+            T[o["out"]] = upsample2(ins[0])
+        else:
+            raise ValueError(kind)
+    if out_grads is None:
+        return T, None, None
+    G = {k: np.asarray(v, dtype=np.float64).copy() for k, v in out_grads.items()}
+
+    def give(name, g):
+        if name == "img":
+            G["img"] = G.get("img", 0.0) + g
+        else:
+            G[name] = G[name] + g if name in G else g.copy()
+
+    block_grads = [None] * len(layers)
+    for o in reversed(ops):
+        if o["out"] not in G:
+            continue  # nothing downstream needs this tensor
+        g = G[o["out"]]
+        kind = o["op"]
+        if kind == "cbs":
+            k = o["layer"]
+            dx, block_grads[k] = _block_bwd(T[o["ins"][0]], params[k], saved[o["out"]], g, layers[k].stride)
+            give(o["ins"][0], dx)
+        elif kind == "slice":
+            full = np.zeros_like(T[o["ins"][0]])
+            full[..., o["c0"]:o["c1"]] = g
+            give(o["ins"][0], full)
+        elif kind == "add":
+            give(o["ins"][0], g)
+            give(o["ins"][1], g)
+        elif kind == "concat":
+            c0 = 0
+            for name in o["ins"]:
+                c = T[name].shape[-1]
+                give(name, g[..., c0:c0 + c])
+                c0 += c
+        elif kind == "maxpool":
+            give(o["ins"][0], maxpool5_bwd(g, saved[o["out"]]))
+        elif kind == "upsample":
+            give(o["ins"][0], upsample2_bwd(g))
+    return T, G, block_grads

@@ -121,6 +121,68 @@ def detector_plain_head_convs():
     return [(64, 64), (192, 80)] * 3
 
 
+def detector_graph(batch: int = 16, image: int = 640):
+    """The detector's dataflow up to the last Conv-BN-SiLU block of every head branch, as a list of primitive operations
+    over named tensors (a description only: no arithmetic here, both the GPU runner and the CPU oracle interpret it).
+
+    Returns (ops, layers, outputs): `layers` = detector_layers(batch, image); every op is a dict with "out", "op" and
+    "ins": op "cbs" (+ "layer": index into layers), "slice" (+ "c0", "c1": channel range), "add", "concat", "maxpool"
+    (5x5, stride 1), "upsample" (nearest 2x); tensor "img" is the input image batch; `outputs` names the six head tensors
+    (box and class branch of the three levels), which feed the plain output convolutions and the loss (not part of this).
+    Backbone C2f units have the residual shortcut, neck units do not.
+    """
+    layers = detector_layers(batch, image)
+    index = {s.name: i for i, s in enumerate(layers)}
+    ops = []
+
+    def cbs(name, src):
+        ops.append({"out": name, "op": "cbs", "ins": [src], "layer": index[name]})
+        return name
+
+    def c2f(name, src, n, shortcut):
+        c = layers[index[f"{name}.cv1"]].c_out // 2
+        a0 = cbs(f"{name}.cv1", src)
+        parts = []
+        for j in range(2):
+            ops.append({"out": f"{name}.p{j}", "op": "slice", "ins": [a0], "c0": j * c, "c1": (j + 1) * c})
+            parts.append(f"{name}.p{j}")
+        for i in range(n):
+            v = cbs(f"{name}.m{i}.cv2", cbs(f"{name}.m{i}.cv1", parts[-1]))
+            if shortcut:
+                ops.append({"out": f"{name}.p{2 + i}", "op": "add", "ins": [parts[-1], v]})
+                v = f"{name}.p{2 + i}"
+            parts.append(v)
+        ops.append({"out": f"{name}.cat", "op": "concat", "ins": list(parts)})
+        return cbs(f"{name}.cv2", f"{name}.cat")
+
+    def cat(name, srcs):
+        ops.append({"out": name, "op": "concat", "ins": list(srcs)})
+        return name
+
+    t = cbs("b1.down", cbs("b0.stem", "img"))
+    t = cbs("b3.down", c2f("b2.c2f", t, 2, True))
+    p3 = c2f("b4.c2f", t, 4, True)
+    p4 = c2f("b6.c2f", cbs("b5.down", p3), 4, True)
+    t = c2f("b8.c2f", cbs("b7.down", p4), 2, True)
+    a0 = cbs("b9.sppf.cv1", t)
+    pools = [a0]
+    for j in range(3):
+        ops.append({"out": f"b9.sppf.pool{j}", "op": "maxpool", "ins": [pools[-1]]})
+        pools.append(f"b9.sppf.pool{j}")
+    p5 = cbs("b9.sppf.cv2", cat("b9.sppf.cat", pools))
+    ops.append({"out": "n10.up", "op": "upsample", "ins": [p5]})
+    n12 = c2f("n12.c2f", cat("n11.cat", ["n10.up", p4]), 2, False)
+    ops.append({"out": "n13.up", "op": "upsample", "ins": [n12]})
+    n15 = c2f("n15.c2f", cat("n14.cat", ["n13.up", p3]), 2, False)
+    n18 = c2f("n18.c2f", cat("n17.cat", [cbs("n16.down", n15), n12]), 2, False)
+    n21 = c2f("n21.c2f", cat("n20.cat", [cbs("n19.down", n18), p5]), 2, False)
+    outputs = []
+    for lvl, src in enumerate([n15, n18, n21]):
+        outputs.append(cbs(f"h22.box{lvl}.1", cbs(f"h22.box{lvl}.0", src)))
+        outputs.append(cbs(f"h22.cls{lvl}.1", cbs(f"h22.cls{lvl}.0", src)))
+    return ops, layers, outputs
+
+
 def detector_parameter_tensors():
     """[(name, numel, group)] of the detector's trainable tensors in network order: per Conv-BN-SiLU layer the filter
     (group 0: decayed weights), the BN gain (group 1) and the BN shift (group 2: biases); per plain head convolution its

@@ -145,3 +145,73 @@ def test_round_bf16_is_nearest_even_on_known_values():
     assert got[0] == 1.0 and got[1] == 1.0 and got[2] == 1.0 + 2.0 ** -6 and got[3] == 1.0 + 2.0 ** -7 and got[4] == -2.5 and got[5] == 0.0
     assert abs(got[6] - 3.0e-5) <= 3.0e-5 * 2.0 ** -8
     assert np.array_equal(chain.round_bf16(got), got)
+
+
+def _detector_params(layers):
+    return [chain.BlockParams(RNG.uniform(-1, 1, (s.c_out, s.k, s.k, s.c_in)) / np.sqrt(s.c_in * s.k * s.k) * 1.7,
+                              RNG.uniform(0.5, 1.5, s.c_out), RNG.normal(size=s.c_out) * 0.1) for s in layers]
+
+
+def test_graph_interpreter_reproduces_the_c2f_unit():
+    # the same unit written twice: once by hand (c2f_fwd_bwd, pinned by finite differences above), once as a graph
+    from paper_2609_10632_b200 import workloads as wl
+
+    c, n = 2, 2
+    layers = [wl.ConvShape("cv1", 2, 4, 3, 4, 2 * c, 1, 1)] + [wl.ConvShape(f"m{i}", 2, 4, 3, c, c, 3, 1) for i in range(2 * n)]
+    layers.append(wl.ConvShape("cv2", 2, 4, 3, (2 + n) * c, 4, 1, 1))
+    ops = [{"out": "a0", "op": "cbs", "ins": ["img"], "layer": 0},
+           {"out": "p0", "op": "slice", "ins": ["a0"], "c0": 0, "c1": c}, {"out": "p1", "op": "slice", "ins": ["a0"], "c0": c, "c1": 2 * c}]
+    parts = ["p0", "p1"]
+    for i in range(n):
+        ops += [{"out": f"u{i}", "op": "cbs", "ins": [parts[-1]], "layer": 1 + 2 * i}, {"out": f"v{i}", "op": "cbs", "ins": [f"u{i}"], "layer": 2 + 2 * i},
+                {"out": f"p{2 + i}", "op": "add", "ins": [parts[-1], f"v{i}"]}]
+        parts.append(f"p{2 + i}")
+    ops += [{"out": "cat", "op": "concat", "ins": parts}, {"out": "out", "op": "cbs", "ins": ["cat"], "layer": 1 + 2 * n}]
+    prm = _params(4, 4, n)
+    x, G = RNG.normal(size=(2, 4, 3, 4)), RNG.normal(size=(2, 4, 3, 4))
+    want = chain.c2f_fwd_bwd(x, prm, n, True, EPS, G)
+    T, grads, bg = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, {"out": G})
+    np.testing.assert_allclose(T["out"], want.out, rtol=1e-13)
+    np.testing.assert_allclose(grads["img"], want.dx, rtol=1e-11, atol=1e-13)
+    for k in range(len(prm)):
+        for a, b in zip(bg[k], want.grads[k]):
+            np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-13)
+
+
+def test_detector_graph_finite_differences_at_a_tiny_size():
+    """The whole detector dataflow (77 blocks, splits, adds, concats, three pools, two upsamplings) at batch 2, 64 x 64
+    (the coarsest level is then 2 x 2: batch statistics over 8 values; over the 2 values of a 32 x 32 image BN degenerates
+    to a sign function and finite differences stop being meaningful):
+    directional derivative with respect to the image and single-entry derivatives of a few filters in different places
+    (backbone behind the pools, neck, head) against central differences of sum(outputs * G)."""
+    from paper_2609_10632_b200 import workloads as wl
+
+    ops, layers, outs = wl.detector_graph(2, 64)
+    prm = _detector_params(layers)
+    x = RNG.uniform(0, 1, (2, 64, 64, 3))
+    T, _, _ = chain.graph_fwd_bwd(ops, layers, prm, x, EPS)
+    Gs = {name: RNG.normal(size=T[name].shape) for name in outs}
+    T, grads, bg = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, Gs)
+    assert all(g is not None for g in bg)
+
+    def loss(xx):
+        TT, _, _ = chain.graph_fwd_bwd(ops, layers, prm, xx, EPS)
+        return float(sum((TT[n] * Gs[n]).sum() for n in outs))
+
+    v = RNG.normal(size=x.shape)
+    h = 1e-6
+    fd = (loss(x + h * v) - loss(x - h * v)) / (2 * h)
+    assert float((grads["img"] * v).sum()) == pytest.approx(fd, rel=2e-4)
+    names = [s.name for s in layers]
+    for lname in ("b2.c2f.m1.cv1", "b8.c2f.cv2", "b9.sppf.cv1", "n12.c2f.m0.cv2", "n18.c2f.cv1", "h22.cls1.0"):
+        k = names.index(lname)
+        w = prm[k].w
+        idx = tuple(int(RNG.integers(0, d)) for d in w.shape)
+        saved = w[idx]
+        hh = 1e-5
+        w[idx] = saved + hh
+        lp = loss(x)
+        w[idx] = saved - hh
+        lm = loss(x)
+        w[idx] = saved
+        assert bg[k][0][idx] == pytest.approx((lp - lm) / (2 * hh), rel=5e-4, abs=1e-6), lname
