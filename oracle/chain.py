@@ -158,12 +158,20 @@ def sppf_fwd_bwd(x, params, eps: float, g_out=None, pool_in_bf16: bool = False):
 
 
 # ------------------------------------------------------------------ a whole dataflow graph of blocks and glue
-def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf16: bool = False):
+def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf16: bool = False, storage_16bit: bool = False):
     """Interpret a dataflow description (a list of op dicts: "cbs" with a layer index, "slice", "add", "concat", "maxpool",
     "upsample"; see the detector's description in the workload module) forwards and, given gradients for some tensors,
     backwards.  layers[k] gives block k's stride; params[k] its BlockParams.  A tensor with several consumers receives
     the sum of their gradients.  Returns (tensors, grads, block_grads): dicts name -> array, and per layer (dw, dgamma, dbeta).
-    pool_in_bf16: inputs of max-pools are rounded to bf16 first (see sppf_fwd_bwd)."""
+    pool_in_bf16: inputs of max-pools are rounded to bf16 first (see sppf_fwd_bwd).
+
+    storage_16bit: model the STORAGE precision the benchmark spec fixes for a chained run -- activations, upstream gradients,
+    dy and dx are bf16 tensors, the saved convolution output is fp16 -- by rounding exactly where a tensor is stored
+    (after the convolution: fp16; after SiLU, after a residual add, after dy, after dx, after every accumulation into a
+    gradient: bf16), while all arithmetic in between stays fp64.  A deep randomly initialised network amplifies
+    perturbations from layer to layer, so two runs that round at different points drift apart geometrically; with the
+    same rounding points the remaining differences are the arithmetic's alone."""
+    r16 = round_bf16 if storage_16bit else (lambda a: a)
     T = {"img": np.asarray(x, dtype=np.float64)}
     saved = {}
     for o in ops:
@@ -171,13 +179,19 @@ def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf
         kind = o["op"]
         if kind == "cbs":
             k = o["layer"]
-            f = oracle.cbs_fwd(ins[0], params[k].w, params[k].gamma, params[k].beta, layers[k].stride, eps)
+            if storage_16bit:
+                y = oracle.conv_fwd(ins[0], params[k].w, layers[k].stride).astype(np.float16).astype(np.float64)
+                mean, var, invstd = oracle.bn_stats(y, eps)
+                f = oracle.BlockResult(y=y, mean=mean, var=var, invstd=invstd,
+                                       a=round_bf16(oracle.bn_silu_fwd(y, mean, invstd, params[k].gamma, params[k].beta)))
+            else:
+                f = oracle.cbs_fwd(ins[0], params[k].w, params[k].gamma, params[k].beta, layers[k].stride, eps)
             saved[o["out"]] = f
             T[o["out"]] = f.a
         elif kind == "slice":
             T[o["out"]] = ins[0][..., o["c0"]:o["c1"]]
         elif kind == "add":
-            T[o["out"]] = ins[0] + ins[1]
+            T[o["out"]] = r16(ins[0] + ins[1])
         elif kind == "concat":
             T[o["out"]] = np.concatenate(ins, axis=-1)
         elif kind == "maxpool":
@@ -192,10 +206,7 @@ def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf
     G = {k: np.asarray(v, dtype=np.float64).copy() for k, v in out_grads.items()}
 
     def give(name, g):
-        if name == "img":
-            G["img"] = G.get("img", 0.0) + g
-        else:
-            G[name] = G[name] + g if name in G else g.copy()
+        G[name] = r16(G[name] + g) if name in G else r16(g)
 
     block_grads = [None] * len(layers)
     for o in reversed(ops):
@@ -205,7 +216,14 @@ def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf
         kind = o["op"]
         if kind == "cbs":
             k = o["layer"]
-            dx, block_grads[k] = _block_bwd(T[o["ins"][0]], params[k], saved[o["out"]], g, layers[k].stride)
+            if storage_16bit:
+                f, prm = saved[o["out"]], params[k]
+                dy, dgamma, dbeta = oracle.bn_silu_bwd(g, f.y, f.mean, f.invstd, prm.gamma, prm.beta)
+                dy = round_bf16(dy)
+                dx = round_bf16(oracle.conv_dgrad(dy, prm.w, np.shape(T[o["ins"][0]]), layers[k].stride))
+                block_grads[k] = (oracle.conv_wgrad(T[o["ins"][0]], dy, np.shape(prm.w)[1], layers[k].stride), dgamma, dbeta)
+            else:
+                dx, block_grads[k] = _block_bwd(T[o["ins"][0]], params[k], saved[o["out"]], g, layers[k].stride)
             give(o["ins"][0], dx)
         elif kind == "slice":
             full = np.zeros_like(T[o["ins"][0]])

@@ -1,0 +1,158 @@
+"""Run a dataflow description of chained Conv-BN-SiLU blocks and glue (workloads.detector_graph: the paper's detector,
+Sec. 6, up to the last block of every head branch) on the GPU, forward and backward.
+
+Only wiring happens here: every arithmetic step is a C-ABI call (block calls of nb_cbs.h, glue calls of nb_glue.h);
+torch allocates the buffers, zeroes gradient accumulators and owns the stream.
+
+Every named tensor is a dense NHWC bf16 buffer.  A block reads its input tensor's buffer directly and writes its
+activations into its output tensor's buffer.  Gradients: a tensor whose only consumer is a block takes that block's dx
+buffer as its gradient (no copy); every other tensor owns a gradient buffer that is zeroed when the backward pass
+starts and to which each consumer ADDS its share (several consumers: the sum of their gradients).
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as nb
+from .block import CbsBlock
+
+
+class GraphRunner:
+    def __init__(self, ops, layers, outputs, eps=1e-3, device=0):
+        self.ops, self.layers, self.outputs = ops, layers, list(outputs)
+        self.dev = torch.device("cuda", device)
+        s0 = layers[0]
+        self.shape = {"img": (s0.n, s0.h, s0.w, s0.c_in)}
+        self.buf = {"img": torch.empty(self.shape["img"], dtype=torch.bfloat16, device=self.dev)}
+        self.blocks = [None] * len(layers)
+        self.idx = {}
+        consumers = {}
+        for o in ops:
+            for name in o["ins"]:
+                consumers.setdefault(name, []).append(o)
+        # ---- forward buffers
+        for o in ops:
+            ins = [self.shape[i] for i in o["ins"]]
+            kind = o["op"]
+            if kind == "cbs":
+                s = layers[o["layer"]]
+                assert ins[0] == (s.n, s.h, s.w, s.c_in), (o["out"], ins[0])
+                blk = CbsBlock(s, eps=eps, device=device)
+                blk.x = self.buf[o["ins"][0]]
+                self.blocks[o["layer"]] = blk
+                shp, buf = (s.n, s.ho, s.wo, s.c_out), blk.a
+            else:
+                n, h, w, c = ins[0]
+                if kind == "slice":
+                    shp = (n, h, w, o["c1"] - o["c0"])
+                elif kind == "add" or kind == "maxpool":
+                    shp = ins[0]
+                elif kind == "concat":
+                    shp = (n, h, w, sum(i[3] for i in ins))
+                elif kind == "upsample":
+                    shp = (n, 2 * h, 2 * w, c)
+                else:
+                    raise ValueError(kind)
+                buf = torch.empty(shp, dtype=torch.bfloat16, device=self.dev)
+                if kind == "maxpool":
+                    self.idx[o["out"]] = torch.empty(shp, dtype=torch.uint8, device=self.dev)
+            self.shape[o["out"]], self.buf[o["out"]] = shp, buf
+        # ---- gradient buffers
+        self.grad, self.owned = {}, []
+        by_out = {o["out"]: o for o in ops}
+        for name in list(self.buf):
+            cons = consumers.get(name, [])
+            if len(cons) == 1 and cons[0]["op"] == "cbs":
+                self.grad[name] = self.blocks[cons[0]["layer"]].dx
+            else:
+                self.grad[name] = torch.zeros(self.shape[name], dtype=torch.bfloat16, device=self.dev)
+                if name not in self.outputs:
+                    self.owned.append(name)
+        for o in ops:
+            if o["op"] == "cbs":
+                self.blocks[o["layer"]].g = self.grad[o["out"]]
+        self.aliased = {name for name in self.buf if name not in self.owned and name not in self.outputs}
+
+    # ------------------------------------------------------------------ helpers
+    def _rows(self, name):
+        n, h, w, _ = self.shape[name]
+        return n * h * w
+
+    @staticmethod
+    def _at(t, channel):
+        return t.data_ptr() + channel * t.element_size()
+
+    def _copy(self, out, ld_out, a, ld_a, rows, channels, b=None, ld_b=0, accumulate=False, stream=None):
+        nb.nb_slice_add(nb.NB_DTYPE_BF16, rows, channels, out, ld_out, a, ld_a, b, ld_b, accumulate, stream)
+
+    # ------------------------------------------------------------------ passes
+    def forward(self, stream=None):
+        B = self.buf
+        for o in self.ops:
+            kind, out, ins = o["op"], o["out"], o["ins"]
+            rows = self._rows(out)
+            c_out = self.shape[out][3]
+            if kind == "cbs":
+                self.blocks[o["layer"]].forward(stream)
+            elif kind == "slice":
+                self._copy(B[out], c_out, self._at(B[ins[0]], o["c0"]), self.shape[ins[0]][3], rows, c_out, stream=stream)
+            elif kind == "add":
+                self._copy(B[out], c_out, B[ins[0]], c_out, rows, c_out, b=B[ins[1]], ld_b=c_out, stream=stream)
+            elif kind == "concat":
+                c0 = 0
+                for name in ins:
+                    c = self.shape[name][3]
+                    self._copy(self._at(B[out], c0), c_out, B[name], c, rows, c, stream=stream)
+                    c0 += c
+            elif kind == "maxpool":
+                n, h, w, c = self.shape[out]
+                nb.nb_maxpool5_fwd(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], self.idx[out], stream)
+            elif kind == "upsample":
+                n, h, w, c = self.shape[ins[0]]
+                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], stream=stream)
+
+    def backward(self, stream=None):
+        """Expects the gradients of the output tensors in self.grad[name]; leaves dL/d img in self.grad['img'] and every
+        block's dw, dgamma, dbeta in the block."""
+        G = self.grad
+        for name in self.owned:
+            G[name].zero_()
+        for o in reversed(self.ops):
+            kind, out, ins = o["op"], o["out"], o["ins"]
+            c_out = self.shape[out][3]
+            if kind == "cbs":
+                blk = self.blocks[o["layer"]]
+                blk.backward_data(stream)
+                blk.backward_weight(stream)
+                src = ins[0]
+                if G[src] is not blk.dx:
+                    c = self.shape[src][3]
+                    self._copy(G[src], c, blk.dx, c, self._rows(src), c, accumulate=True, stream=stream)
+            elif kind == "slice":
+                src = ins[0]
+                self._copy(self._at(G[src], o["c0"]), self.shape[src][3], G[out], c_out, self._rows(out), c_out, accumulate=True, stream=stream)
+            elif kind == "add":
+                for src in ins:
+                    self._copy(G[src], c_out, G[out], c_out, self._rows(out), c_out, accumulate=True, stream=stream)
+            elif kind == "concat":
+                c0 = 0
+                for src in ins:
+                    c = self.shape[src][3]
+                    self._copy(G[src], c, self._at(G[out], c0), c_out, self._rows(out), c, accumulate=True, stream=stream)
+                    c0 += c
+            elif kind == "maxpool":
+                n, h, w, c = self.shape[out]
+                nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, G[out], self.idx[out], G[ins[0]], True, stream)
+            elif kind == "upsample":
+                n, h, w, c = self.shape[ins[0]]
+                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, G[out], G[ins[0]], backward=True, accumulate=True, stream=stream)
+
+    def poll(self):
+        for b in self.blocks:
+            b.poll()
+
+    def glue_launches(self):
+        fwd = sum(len(o["ins"]) if o["op"] == "concat" else 1 for o in self.ops if o["op"] != "cbs")
+        bwd = sum(len(o["ins"]) if o["op"] in ("concat", "add") else 1 for o in self.ops if o["op"] != "cbs")
+        bwd += sum(1 for o in self.ops if o["op"] == "cbs" and self.grad[o["ins"][0]] is not self.blocks[o["layer"]].dx)
+        return fwd, bwd

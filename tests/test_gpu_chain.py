@@ -219,3 +219,62 @@ def test_sppf_unit_matches_chained_oracle():
         report.append(f"{name} (behind the pools): rel_l2={r:.2e}")
         assert r <= 0.1, name
     print("\n".join(report))
+
+
+def test_detector_dataflow_matches_graph_oracle():
+    """All 77 blocks chained as the detector's dataflow (batch 2, 256 x 256 image: the coarsest level is 8 x 8) against the
+    oracle's interpretation of the same description.
+
+    A deep randomly initialised BN network amplifies perturbations from block to block: in the oracle alone, rounding the
+    stored tensors to 16 bits (its storage mode) moves the results away from the exact fp64 graph by 2e-3 after the first
+    block, 2e-2 after the third C2f unit and 0.2 at the heads, and two 16-bit runs that round slightly differently drift
+    apart just as much.  No fixed small tolerance is meaningful at that depth, so the oracle's own drift is the
+    yardstick: for every tensor of the forward pass and every block's dw, dgamma, dbeta the GPU's distance from the exact
+    graph must stay within TWICE the distance of the oracle's 16-bit storage run from the exact graph (+ 5e-3).  A wiring
+    mistake (a missing shortcut, a wrong slice, a dropped gradient contribution) is an O(1) error from the first
+    affected tensor on, where the yardstick is still a few 1e-3.  The yardstick also absorbs the non-uniqueness of the
+    gradients behind the max-pools (see the SPPF test), because the storage run's pools flip in the same way."""
+    import torch
+
+    from paper_2609_10632_b200.detector import GraphRunner
+
+    ops, layers, outs = wl.detector_graph(2, 256)
+    run = GraphRunner(ops, layers, outs, eps=EPS)
+    params = []
+    for k, blk in enumerate(run.blocks):
+        inp = wl.make_inputs(layers[k], 53, k, bf16=True, affine="random")
+        params.append(chain.BlockParams(inp.w, inp.gamma, inp.beta))
+        for name in ("w", "gamma", "beta"):
+            dst = getattr(blk, name)
+            dst.copy_(torch.from_numpy(np.ascontiguousarray(getattr(inp, name))).to(dst.dtype))
+    x = wl.make_inputs(layers[0], 53, 0, bf16=True).x
+    run.buf["img"].copy_(torch.from_numpy(x).to(torch.bfloat16))
+    gouts = {}
+    for j, name in enumerate(outs):
+        rng = np.random.Generator(np.random.Philox(key=[53, 5000 + j]))
+        g = wl.round_to_bf16(rng.standard_normal(run.shape[name], dtype=np.float32))
+        gouts[name] = g
+        run.grad[name].copy_(torch.from_numpy(g).to(torch.bfloat16))
+    run.forward()
+    run.backward()
+    torch.cuda.synchronize()
+    run.poll()
+    f64 = lambda t: t.detach().double().cpu().numpy()
+    T0, G0, b0 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts)                      # exact
+    T1, G1, b1 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts, storage_16bit=True)  # the yardstick
+    worst = {"ratio": 0.0, "gpu": 0.0, "yardstick": 0.0}
+
+    def held(name, got, exact, stored):
+        e, y = parity.rel_l2(got, exact), parity.rel_l2(stored, exact)
+        assert np.isfinite(got).all(), name
+        worst["ratio"], worst["gpu"], worst["yardstick"] = max(worst["ratio"], e / (y + 2.5e-3)), max(worst["gpu"], e), max(worst["yardstick"], y)
+        assert e <= 2 * y + 5e-3, (name, e, y)
+
+    for name in T0:
+        if name != "img":
+            held(name, f64(run.buf[name]), T0[name], T1[name])
+    held("d img", f64(run.grad["img"]), G0["img"], G1["img"])
+    for k, blk in enumerate(run.blocks):
+        for slot, t in enumerate((blk.dw, blk.dgamma, blk.dbeta)):
+            held(f"{layers[k].name}.{('dw', 'dgamma', 'dbeta')[slot]}", f64(t), b0[k][slot], b1[k][slot])
+    print("worst:", {k: f"{v:.2e}" for k, v in worst.items()}, "glue launches fwd/bwd:", run.glue_launches())

@@ -215,3 +215,30 @@ def test_detector_graph_finite_differences_at_a_tiny_size():
         lm = loss(x)
         w[idx] = saved
         assert bg[k][0][idx] == pytest.approx((lp - lm) / (2 * hh), rel=5e-4, abs=1e-6), lname
+
+
+def test_storage_rounding_mode_stays_close_to_the_exact_graph_on_a_shallow_unit():
+    # the 16-bit storage mode only rounds stored tensors: on one C2f unit it must agree with the exact graph to bf16 accuracy,
+    # every stored activation must be exactly representable in bf16, and the exact mode must be untouched by the flag's code
+    from paper_2609_10632_b200 import workloads as wl
+
+    c, n = 4, 1
+    layers = [wl.ConvShape("cv1", 2, 6, 5, 8, 2 * c, 1, 1), wl.ConvShape("m0", 2, 6, 5, c, c, 3, 1), wl.ConvShape("m1", 2, 6, 5, c, c, 3, 1),
+              wl.ConvShape("cv2", 2, 6, 5, 3 * c, 8, 1, 1)]
+    ops = [{"out": "a0", "op": "cbs", "ins": ["img"], "layer": 0},
+           {"out": "p0", "op": "slice", "ins": ["a0"], "c0": 0, "c1": c}, {"out": "p1", "op": "slice", "ins": ["a0"], "c0": c, "c1": 2 * c},
+           {"out": "u", "op": "cbs", "ins": ["p1"], "layer": 1}, {"out": "v", "op": "cbs", "ins": ["u"], "layer": 2},
+           {"out": "p2", "op": "add", "ins": ["p1", "v"]}, {"out": "cat", "op": "concat", "ins": ["p0", "p1", "p2"]},
+           {"out": "out", "op": "cbs", "ins": ["cat"], "layer": 3}]
+    prm = _params(8, 8, n)
+    x = chain.round_bf16(RNG.normal(size=(2, 6, 5, 8)))
+    G = chain.round_bf16(RNG.normal(size=(2, 6, 5, 8)))
+    T0, G0, b0 = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, {"out": G})
+    T1, G1, b1 = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, {"out": G}, storage_16bit=True)
+    for name in ("a0", "v", "p2", "out"):
+        assert np.array_equal(chain.round_bf16(T1[name]), T1[name]), name
+        assert np.linalg.norm(T1[name] - T0[name]) <= 1e-2 * np.linalg.norm(T0[name]), name
+    assert np.array_equal(chain.round_bf16(G1["img"]), G1["img"])
+    assert np.linalg.norm(G1["img"] - G0["img"]) <= 3e-2 * np.linalg.norm(G0["img"])
+    for k in range(4):
+        assert np.linalg.norm(b1[k][0] - b0[k][0]) <= 3e-2 * np.linalg.norm(b0[k][0])
