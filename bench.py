@@ -448,10 +448,10 @@ def main():
     if not args.no_optimizer and args.workload == "cfg5":
         opt_step = run_optimizer_step(args, blocks, dev, local, peaks)
 
-    # ---------------- the backbone's four C2f units as chained blocks (split / add / concat glue included)
+    # ---------------- the whole detector as CHAINED blocks (split / add / concat / pool / upsample glue included)
     chain = None
     if not args.no_chain and args.workload == "cfg5":
-        chain = run_c2f_chains(args, dev, local, peaks)
+        chain = run_detector_chain(args, dev, local, peaks, flops)
 
     # ---------------- end to end from pinned host buffers through the C ABI
     e2e = None
@@ -480,7 +480,7 @@ def main():
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },
             "clocks": clocks.summary(), "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernels, "eval_forward": eval_fwd, "optimizer_step": opt_step, "c2f_chain": chain,
+            "kernels": kernels, "eval_forward": eval_fwd, "optimizer_step": opt_step, "detector_chain": chain,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -533,33 +533,42 @@ def run_eval_forward(args, blocks, dev, fwd_flops, peaks, kernels):
             "training_forward_kernels_ms": train_fwd, "cuda_graph": True}
 
 
-def run_c2f_chains(args, dev, local, peaks):
-    """The four C2f units of the backbone (96/192/384/576 channels at 160/80/40/20 pixels, 2/4/4/2 bottlenecks with
-    shortcut) run as CHAINS: each block consumes the previous block's activations and gradients, joined by nb_slice_add
-    (split, residual add, concat, gradient accumulation).  Forward + backward of all four as one CUDA-graph replay."""
+def run_detector_chain(args, dev, local, peaks, step_flops_value):
+    """The 77 blocks run as the detector's dataflow (workloads.detector_graph): every block consumes the previous blocks'
+    activations and gradients, joined by the glue calls (channel split / concat, residual add, 5x5 max-pools, 2x
+    upsampling, gradient accumulation at fan-out).  Forward + backward from a uniform[0,1] image batch and random
+    gradients at the six head tensors, as one CUDA-graph replay.  Same convolution work as the per-layer step."""
     import torch
 
     from paper_2609_10632_b200 import binding as nb
-    from paper_2609_10632_b200.c2f import C2fChain
+    from paper_2609_10632_b200 import workloads as wl
+    from paper_2609_10632_b200.detector import GraphRunner
 
-    units = [C2fChain(16, h, h, c, c, n, True, device=local) for c, h, n in ((96, 160, 2), (192, 80, 4), (384, 40, 4), (576, 20, 2))]
-    flops = 0.0
-    for u in units:
-        for i, b in enumerate(u.blocks):
-            b.fill_random(seed=5000 + i)
-            flops += 3.0 * b.shape.gemm_flops
-        u.cv2.g.normal_()
+    ops, layers, outs = wl.detector_graph(16, 640)
+    run = GraphRunner(ops, layers, outs, device=local)
+    for i, b in enumerate(run.blocks):
+        b.fill_random(seed=7000 + i)  # (fills the block's own scratch x / g as well; the chained buffers are set below)
+    run.buf["img"].uniform_(0.0, 1.0)
+    for name in outs:
+        run.grad[name].normal_()
+
+    side = None if args.no_wgrad_stream else torch.cuda.Stream(device=dev)
+    side_ws = None if side is None else torch.empty(max(b.plan.bwd_bytes for b in run.blocks), dtype=torch.uint8, device=dev)
 
     def step():
-        for u in units:
-            u.forward()
-            u.backward()
+        run.forward()
+        if side is None:
+            run.backward()
+        else:
+            main = torch.cuda.current_stream()
+            side.wait_stream(main)
+            run.backward(wgrad_stream=side, wgrad_workspace=side_ws)
+            main.wait_stream(side)
 
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
-    for u in units:
-        u.poll()
+    run.poll()
     l0 = nb.nb_cbs_launch_count()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
@@ -573,14 +582,13 @@ def run_c2f_chains(args, dev, local, peaks):
         graph.replay()
     ev1.record()
     torch.cuda.synchronize()
-    for u in units:
-        u.poll()
+    run.poll()
     ms = ev0.elapsed_time(ev1) / args.steps
-    nblocks = sum(len(u.blocks) for u in units)
-    glue = sum(2 + 4 * u.n for u in units)  # forward: 1 + 2n, backward: 2n + 1
-    return {"units": "backbone C2f x4 (96@160 n2, 192@80 n4, 384@40 n4, 576@20 n2), batch 16, shortcut", "conv_bn_silu_blocks": nblocks,
-            "glue_launches": glue, "launches_per_step": int(launches), "ms_per_step": ms, "tflops": flops / (ms * 1e-3) / 1e12,
-            "frac_of_measured_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "cuda_graph": True}
+    gf, gb = run.glue_launches()
+    tf = step_flops_value / (ms * 1e-3) / 1e12
+    return {"what": "77 chained Conv-BN-SiLU blocks + glue, fwd + bwd, batch 16, 640 x 640", "wgrad_on_second_stream": side is not None, "ms_per_step": ms, "tflops": tf,
+            "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "launches_per_step": int(launches), "glue_launches_fwd_bwd": [gf, gb],
+            "cuda_graph": True}
 
 
 def run_optimizer_step(args, blocks, dev, local, peaks):

@@ -111,9 +111,11 @@ class GraphRunner:
                 n, h, w, c = self.shape[ins[0]]
                 nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], stream=stream)
 
-    def backward(self, stream=None):
+    def backward(self, stream=None, wgrad_stream=None, wgrad_workspace=None):
         """Expects the gradients of the output tensors in self.grad[name]; leaves dL/d img in self.grad['img'] and every
-        block's dw, dgamma, dbeta in the block."""
+        block's dw, dgamma, dbeta in the block.  With wgrad_stream (and a workspace for it) every weight gradient is queued
+        on that stream behind an event that follows the block's data-gradient call (it only reads the block's input
+        activations and dy, which nothing overwrites during the backward pass); the caller joins the streams."""
         G = self.grad
         for name in self.owned:
             G[name].zero_()
@@ -123,7 +125,13 @@ class GraphRunner:
             if kind == "cbs":
                 blk = self.blocks[o["layer"]]
                 blk.backward_data(stream)
-                blk.backward_weight(stream)
+                if wgrad_stream is None:
+                    blk.backward_weight(stream)
+                else:
+                    ev = torch.cuda.Event()
+                    ev.record(torch.cuda.current_stream(self.dev) if stream is None else stream)
+                    wgrad_stream.wait_event(ev)
+                    blk.backward_weight(wgrad_stream, wgrad_workspace)
                 src = ins[0]
                 if G[src] is not blk.dx:
                     c = self.shape[src][3]
