@@ -6,8 +6,10 @@ torch allocates the buffers, zeroes gradient accumulators and owns the stream.
 
 Every named tensor is a dense NHWC bf16 buffer.  A block reads its input tensor's buffer directly and writes its
 activations into its output tensor's buffer.  Gradients: a tensor whose only consumer is a block takes that block's dx
-buffer as its gradient (no copy); every other tensor owns a gradient buffer that is zeroed when the backward pass
-starts and to which each consumer ADDS its share (several consumers: the sum of their gradients).
+buffer as its gradient (no copy); every other tensor owns a gradient buffer to which each consumer contributes its share
+(several consumers: the sum of their gradients).  The first contribution to a channel range OVERWRITES it and later ones
+add to it (decided once, from the order of the backward pass); a buffer is zeroed beforehand only if the overwriting
+contributions do not cover all of its channels.
 """
 from __future__ import annotations
 
@@ -72,6 +74,33 @@ class GraphRunner:
             if o["op"] == "cbs":
                 self.blocks[o["layer"]].g = self.grad[o["out"]]
         self.aliased = {name for name in self.buf if name not in self.owned and name not in self.outputs}
+        # ---- which contributions overwrite and which add: walk the backward order once
+        covered = {name: [] for name in self.owned}  # channel intervals already written
+        self.acc = {}                                  # (op index, input position) -> accumulate?
+        for oi in reversed(range(len(ops))):
+            o = ops[oi]
+            for pos, src in enumerate(o["ins"]):
+                if src not in covered:
+                    continue  # aliased to a block's dx, or the block writes there directly
+                c = self.shape[src][3]
+                lo, hi = (o["c0"], o["c1"]) if o["op"] == "slice" else (0, c)
+                inside = any(a <= lo and hi <= b for a, b in covered[src])
+                disjoint = all(hi <= a or b <= lo for a, b in covered[src])
+                if inside:
+                    self.acc[(oi, pos)] = True
+                elif disjoint:
+                    self.acc[(oi, pos)] = False
+                    covered[src].append((lo, hi))
+                else:  # partial overlap: give up on this tensor, zero it and add everything
+                    covered[src] = [(0, 0)]
+                    self.acc[(oi, pos)] = True
+        self.zeroed = []
+        for name, iv in covered.items():
+            full = sorted(iv) and sum(b - a for a, b in iv) == self.shape[name][3] and (0, 0) not in iv
+            if not full:
+                self.zeroed.append(name)
+                for key in [k for k in self.acc if ops[k[0]]["ins"][k[1]] == name]:
+                    self.acc[key] = True
 
     # ------------------------------------------------------------------ helpers
     def _rows(self, name):
@@ -117,9 +146,10 @@ class GraphRunner:
         on that stream behind an event that follows the block's data-gradient call (it only reads the block's input
         activations and dy, which nothing overwrites during the backward pass); the caller joins the streams."""
         G = self.grad
-        for name in self.owned:
+        for name in self.zeroed:
             G[name].zero_()
-        for o in reversed(self.ops):
+        for oi in reversed(range(len(self.ops))):
+            o = self.ops[oi]
             kind, out, ins = o["op"], o["out"], o["ins"]
             c_out = self.shape[out][3]
             if kind == "cbs":
@@ -135,25 +165,25 @@ class GraphRunner:
                 src = ins[0]
                 if G[src] is not blk.dx:
                     c = self.shape[src][3]
-                    self._copy(G[src], c, blk.dx, c, self._rows(src), c, accumulate=True, stream=stream)
+                    self._copy(G[src], c, blk.dx, c, self._rows(src), c, accumulate=self.acc[(oi, 0)], stream=stream)
             elif kind == "slice":
                 src = ins[0]
-                self._copy(self._at(G[src], o["c0"]), self.shape[src][3], G[out], c_out, self._rows(out), c_out, accumulate=True, stream=stream)
+                self._copy(self._at(G[src], o["c0"]), self.shape[src][3], G[out], c_out, self._rows(out), c_out, accumulate=self.acc[(oi, 0)], stream=stream)
             elif kind == "add":
-                for src in ins:
-                    self._copy(G[src], c_out, G[out], c_out, self._rows(out), c_out, accumulate=True, stream=stream)
+                for pos, src in enumerate(ins):
+                    self._copy(G[src], c_out, G[out], c_out, self._rows(out), c_out, accumulate=self.acc[(oi, pos)], stream=stream)
             elif kind == "concat":
                 c0 = 0
-                for src in ins:
+                for pos, src in enumerate(ins):
                     c = self.shape[src][3]
-                    self._copy(G[src], c, self._at(G[out], c0), c_out, self._rows(out), c, accumulate=True, stream=stream)
+                    self._copy(G[src], c, self._at(G[out], c0), c_out, self._rows(out), c, accumulate=self.acc[(oi, pos)], stream=stream)
                     c0 += c
             elif kind == "maxpool":
                 n, h, w, c = self.shape[out]
-                nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, G[out], self.idx[out], G[ins[0]], True, stream)
+                nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, G[out], self.idx[out], G[ins[0]], self.acc[(oi, 0)], stream)
             elif kind == "upsample":
                 n, h, w, c = self.shape[ins[0]]
-                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, G[out], G[ins[0]], backward=True, accumulate=True, stream=stream)
+                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, G[out], G[ins[0]], backward=True, accumulate=self.acc[(oi, 0)], stream=stream)
 
     def poll(self):
         for b in self.blocks:
