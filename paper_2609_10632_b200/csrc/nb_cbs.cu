@@ -995,13 +995,16 @@ nb_status run_slice_add(void* out, long long ld_out, const void* a, long long ld
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 8));
-    if (vec)
-        launch_k(slice_add_kernel<T, true>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a,
-                 static_cast<const T*>(b), ld_b, rows, channels, accumulate);
-    else
-        launch_k(slice_add_kernel<T, false>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a,
-                 static_cast<const T*>(b), ld_b, rows, channels, accumulate);
+    const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 16));
+    const bool small = total + 256LL * blocks < (1LL << 32);  // indices (one grid stride past the end included) fit 32 bits
+#define NB_SLICE_LAUNCH(VECF, IDX)                                                                                                         \
+    launch_k(slice_add_kernel<T, VECF, IDX>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a, \
+             static_cast<const T*>(b), ld_b, rows, channels, accumulate)
+    if (vec && small) NB_SLICE_LAUNCH(true, unsigned);
+    else if (vec) NB_SLICE_LAUNCH(true, long long);
+    else if (small) NB_SLICE_LAUNCH(false, unsigned);
+    else NB_SLICE_LAUNCH(false, long long);
+#undef NB_SLICE_LAUNCH
     return launch_ok("slice_add");
 }
 }  // namespace
@@ -1069,14 +1072,23 @@ nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_
     g_err.clear();
     if (!g || !idx || !dx) return fail(NB_ERR_INVALID_ARG, "g, idx and dx must not be NULL");
     NB_TRY(check_nhwc(n, h, w, c));
+    if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const unsigned blocks = glue_blocks((long long)n * h * w * c);
+    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 &&
+                     !((reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(dx)) & 15u) && !(reinterpret_cast<uintptr_t>(idx) & 7u);
+    const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
+#define NB_POOLB(T)                                                                                                                               \
+    do {                                                                                                                                          \
+        if (vec) launch_k(maxpool5_bwd_kernel<T, 8>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0); \
+        else launch_k(maxpool5_bwd_kernel<T, 1>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0);     \
+    } while (0)
     switch (dtype) {
-        case NB_DTYPE_F32: launch_k(maxpool5_bwd_kernel<float>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const float*>(g), idx, static_cast<float*>(dx), n, h, w, c, accumulate != 0); break;
-        case NB_DTYPE_BF16: launch_k(maxpool5_bwd_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(g), idx, static_cast<__nv_bfloat16*>(dx), n, h, w, c, accumulate != 0); break;
-        case NB_DTYPE_F16: launch_k(maxpool5_bwd_kernel<__half>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __half*>(g), idx, static_cast<__half*>(dx), n, h, w, c, accumulate != 0); break;
+        case NB_DTYPE_F32: NB_POOLB(float); break;
+        case NB_DTYPE_BF16: NB_POOLB(__nv_bfloat16); break;
+        case NB_DTYPE_F16: NB_POOLB(__half); break;
         default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     }
+#undef NB_POOLB
     return launch_ok("maxpool5_bwd");
 }
 
@@ -1085,12 +1097,17 @@ nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c
     g_err.clear();
     if (!src || !dst) return fail(NB_ERR_INVALID_ARG, "src and dst must not be NULL");
     NB_TRY(check_nhwc(n, h, w, c));
+    if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const unsigned blocks = glue_blocks((long long)n * h * w * c);
-#define NB_UPS(T)                                                                                                                              \
-    do {                                                                                                                                       \
-        if (backward) launch_k(upsample2_kernel<T, true>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0); \
-        else launch_k(upsample2_kernel<T, false>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, 0);                    \
+    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u);
+    const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
+#define NB_UPS1(T, BW, VV) launch_k(upsample2_kernel<T, BW, VV>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0)
+#define NB_UPS(T)                                   \
+    do {                                            \
+        if (backward && vec) NB_UPS1(T, true, 8);   \
+        else if (backward) NB_UPS1(T, true, 1);     \
+        else if (vec) NB_UPS1(T, false, 8);         \
+        else NB_UPS1(T, false, 1);                  \
     } while (0)
     switch (dtype) {
         case NB_DTYPE_F32: NB_UPS(float); break;
@@ -1099,6 +1116,7 @@ nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c
         default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     }
 #undef NB_UPS
+#undef NB_UPS1
     return launch_ok("upsample2");
 }
 

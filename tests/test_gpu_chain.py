@@ -278,3 +278,61 @@ def test_detector_dataflow_matches_graph_oracle():
         for slot, t in enumerate((blk.dw, blk.dgamma, blk.dbeta)):
             held(f"{layers[k].name}.{('dw', 'dgamma', 'dbeta')[slot]}", f64(t), b0[k][slot], b1[k][slot])
     print("worst:", {k: f"{v:.2e}" for k, v in worst.items()}, "glue launches fwd/bwd:", run.glue_launches())
+
+
+def test_chained_detector_in_the_benchmarks_launch_configuration_is_bitwise_the_plain_run():
+    """bench.py replays the chained detector as a CUDA graph with the weight gradients on a second stream: that launch
+    configuration must give bit for bit what the plain single-stream eager run (checked against the oracle above) gives."""
+    import torch
+
+    from paper_2609_10632_b200.detector import GraphRunner
+
+    ops, layers, outs = wl.detector_graph(2, 128)
+    run = GraphRunner(ops, layers, outs, eps=EPS)
+    gen = torch.Generator(device=run.dev)
+    gen.manual_seed(7)
+    for i, b in enumerate(run.blocks):
+        b.fill_random(seed=100 + i)
+    img = torch.rand(run.shape["img"], generator=gen, device=run.dev).to(torch.bfloat16)
+    gout = {n: torch.randn(run.shape[n], generator=gen, device=run.dev).to(torch.bfloat16) for n in outs}
+
+    def load():
+        run.buf["img"].copy_(img)
+        for n in outs:
+            run.grad[n].copy_(gout[n])
+
+    load()
+    run.forward()
+    run.backward()
+    torch.cuda.synchronize()
+    want = [(b.dw.clone(), b.dgamma.clone(), b.dbeta.clone()) for b in run.blocks]
+    want_dimg = run.grad["img"].clone()
+    side = torch.cuda.Stream()
+    side_ws = torch.empty(max(b.plan.bwd_bytes for b in run.blocks), dtype=torch.uint8, device=run.dev)
+
+    def step():
+        main = torch.cuda.current_stream()
+        run.forward()
+        side.wait_stream(main)
+        run.backward(wgrad_stream=side, wgrad_workspace=side_ws)
+        main.wait_stream(side)
+
+    load()
+    step()  # eager, two streams
+    torch.cuda.synchronize()
+    for b in run.blocks:
+        b.dw.zero_()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(cap):
+        with torch.cuda.graph(graph, stream=cap):
+            step()
+    torch.cuda.current_stream().wait_stream(cap)
+    load()
+    graph.replay()
+    torch.cuda.synchronize()
+    run.poll()
+    for b, (dw, dgamma, dbeta) in zip(run.blocks, want):
+        assert torch.equal(b.dw, dw) and torch.equal(b.dgamma, dgamma) and torch.equal(b.dbeta, dbeta), b.shape.name
+    assert torch.equal(run.grad["img"], want_dimg)
