@@ -195,6 +195,12 @@ nb_status nb_conv_bn_silu_infer(nb_cbs_plan plan, const void* x, const void* w, 
 nb_status nb_conv_bias_act(nb_cbs_plan plan, const void* x, const void* w, const float* bias, int32_t act, void* out,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* Backward of the plain convolution with bias (act = 0), given dout = dL/d out:
+ *   dx = conv^T(dout, w) (may be NULL), dw[c',r,t,c] = sum_{n,p,q} dout[n,p,q,c'] * x[...] (fp32), dbias_c' = sum dout (may be NULL).
+ * The same data-gradient and weight-gradient kernels as the block's backward calls; workspace of the backward size. */
+nb_status nb_conv_bias_bwd(nb_cbs_plan plan, const void* x, const void* w, const void* dout, void* dx, float* dw,
+                           float* dbias, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Fold evaluation-mode BN into the filter that feeds it: with s_c' = gamma_c' / sqrt(running_var_c' + eps),
  *   w_folded[c',r,t,c] = s_c' * w[c',r,t,c]   (the plan's activation dtype, rounded once)
  *   bias_folded[c']    = beta_c' - running_mean_c' * s_c'                                   (fp32)

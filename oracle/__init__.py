@@ -216,3 +216,10 @@ def cbs_infer(x, w, gamma, beta, running_mean, running_var, stride: int, eps: fl
 def conv_bias_act(x, w, bias, stride: int, act: bool = False):
     """Convolution with a per-channel bias and no normalisation (the head's output layers, Table 2 row 3)."""
     return bias_act(conv_fwd(x, w, stride), bias, act)
+
+
+def conv_bias_bwd(x, w, g, stride: int):
+    """Backward of conv_bias_act(act=False) given g = dL/d out: (dx, dw, dbias) with dbias_c = sum of g over all pixels."""
+    g = _f64(g)
+    k = np.shape(w)[1]
+    return conv_dgrad(g, w, np.shape(x), stride), conv_wgrad(x, g, k, stride), g.reshape(-1, g.shape[-1]).sum(axis=0)

@@ -28,7 +28,7 @@ EXPORTS = (
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step",
-    "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2",
+    "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd",
 )
 
 
@@ -88,6 +88,7 @@ def load() -> ctypes.CDLL:
         lib.nb_conv_bn_silu_infer.argtypes = [V, V, V, FP, FP, FP, FP, V, V, c_size_t, V]
         lib.nb_conv_bias_act.argtypes = [V, V, V, FP, c_int32, V, V, c_size_t, V]
         lib.nb_bn_fold.argtypes = [V, V, FP, FP, FP, FP, V, FP, V]
+        lib.nb_conv_bias_bwd.argtypes = [V, V, V, V, V, FP, FP, V, c_size_t, V]
         lib.nb_sgd_plan_create.argtypes = [POINTER(nb_sgd_tensor), c_int32, c_int, POINTER(V)]
         lib.nb_sgd_plan_destroy.argtypes = [V]
         lib.nb_sgd_workspace_bytes.argtypes = [V, POINTER(c_size_t)]
@@ -261,6 +262,11 @@ def nb_conv_bn_silu_infer(plan: Plan, x, w, gamma, beta, running_mean, running_v
 
 def nb_conv_bias_act(plan: Plan, x, w, bias, act, out, workspace, stream=None):
     _check(load().nb_conv_bias_act(plan.handle, _ptr(x), _ptr(w), _ptr(bias), int(act), _ptr(out), _ptr(workspace), _nbytes(workspace),
+                                   _stream(stream)))
+
+
+def nb_conv_bias_bwd(plan: Plan, x, w, dout, dx, dw, dbias, workspace, stream=None):
+    _check(load().nb_conv_bias_bwd(plan.handle, _ptr(x), _ptr(w), _ptr(dout), _ptr(dx), _ptr(dw), _ptr(dbias), _ptr(workspace), _nbytes(workspace),
                                    _stream(stream)))
 
 

@@ -695,6 +695,47 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     return run_simt_dgrad<__nv_bfloat16>(p, dy_out, w, dx, st);
 }
 
+nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const void* dout, void* dx, float* dw, float* dbias, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(x); NB_CHECK_PTR(dout); NB_CHECK_PTR(dw); NB_CHECK_PTR(dx, true); NB_CHECK_PTR(dbias, true);
+    if (dx) NB_CHECK_PTR(w);
+    NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
+    {
+        DeviceGuard on_device(p->device);
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        char* ws = static_cast<char*>(workspace);
+        if (dbias) {  // column sums of dout: the statistics kernels with only the raw sum requested
+            float* part = reinterpret_cast<float*>(ws + p->off_bpart);
+            if (is_f32(p)) NB_TRY(run_stats_partial<float>(p, dout, part, st));
+            else NB_TRY(run_stats_partial<__nv_bfloat16>(p, dout, part, st));
+            NB_TRY(run_finalize(p, part, p->ew.blocks_stats, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, dbias, nullptr, st));
+        }
+        if (dx) {
+            if (is_f32(p)) {
+                NB_TRY(run_simt_dgrad<float>(p, dout, w, dx, st));
+            } else if (p->stem) {
+                SiteTimer tm(p, SITE_DGRAD, st);
+                const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
+                const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
+                launch_k(stem_dgrad_tiled_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(w),
+                         static_cast<__nv_bfloat16*>(dx), p->g);
+                NB_LAUNCH_OK("stem_dgrad");
+            } else if (p->tc.dgrad) {
+                SiteTimer tm(p, SITE_DGRAD, st);
+                const long long l0 = p->tc.launches;
+                const nb_status ts = tc_dgrad(&p->tc, p->g, dout, w, dx, ws + p->off_wt, p->status, st, false);  // rearranges the filter itself
+                g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
+                if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
+            } else {
+                NB_TRY(run_simt_dgrad<__nv_bfloat16>(p, dout, w, dx, st));
+            }
+        }
+    }
+    return nb_conv_bn_silu_bwd_weight(p, x, dout, dw, workspace, workspace_bytes, stream);
+}
+
 nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* dy, float* dw, void* workspace,
                                      size_t workspace_bytes, void* stream) {
     g_err.clear();

@@ -168,3 +168,31 @@ def test_infer_argument_checks():
     with pytest.raises(nb.NbError) as e:
         nb.nb_conv_bn_silu_infer(d2.plan, d2.x, d2.w, d2.gamma, d2.beta, d2.d_rm, d2.d_rv, d2.out, d2.ws[:256])
     assert e.value.status == nb.NB_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("shape", [SHAPES[6], SHAPES[1], SHAPES[3], SHAPES[8]], ids=lambda s: s.name)
+@pytest.mark.parametrize("mode", [0, 1], ids=["bf16", "f32"])
+def test_conv_bias_backward_matches_oracle(shape, mode):
+    d = Dev(shape, mode, cfg_id=27, layer_id=SHAPES.index(shape))
+    torch = d.torch
+    act = torch.float32 if d.f32 else torch.bfloat16
+    g = d.inp.g  # seeded upstream gradient of the output's shape (bf16-representable in bf16 mode)
+    dev = d.x.device
+    dout = torch.from_numpy(np.ascontiguousarray(g)).to(act).to(dev)
+    dx = torch.empty_like(d.x)
+    dw = torch.empty(d.w.shape, dtype=torch.float32, device=dev)
+    db = torch.empty(shape.c_out, dtype=torch.float32, device=dev)
+    ws = torch.empty(d.plan.bwd_bytes, dtype=torch.uint8, device=dev)
+    d.nb.nb_conv_bias_bwd(d.plan, d.x, d.w, dout, dx, dw, db, ws)
+    torch.cuda.synchronize()
+    d.nb.nb_cbs_poll_status(d.plan)
+    rdx, rdw, rdb = oracle.conv_bias_bwd(d.inp.x, d.inp.w, g, shape.stride)
+    tag = _tag(mode)
+    parity.check("dx", dx.double().cpu().numpy(), rdx, tag)
+    parity.check("dw", dw.double().cpu().numpy(), rdw, tag)
+    parity.check("dbias", db.double().cpu().numpy(), rdb, tag)
+    # dx and dbias are optional
+    dw2 = torch.empty_like(dw)
+    d.nb.nb_conv_bias_bwd(d.plan, d.x, d.w, dout, None, dw2, None, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(dw, dw2)

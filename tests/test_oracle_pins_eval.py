@@ -108,3 +108,23 @@ def test_folded_convolution_equals_the_evaluation_mode_block(k, stride):
     wf, bf = oracle.bn_fold(w, gamma, beta, rm, rv, eps=1e-3)
     got = oracle.conv_bias_act(x, wf, bf, stride, act=True)
     np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+
+
+def test_conv_bias_backward_is_the_adjoint_of_the_forward():
+    x = RNG.normal(size=(2, 6, 5, 3))
+    w = RNG.normal(size=(4, 3, 3, 3))
+    bias = RNG.normal(size=4)
+    g = RNG.normal(size=(2, 3, 3, 4))
+    dx, dw, db = oracle.conv_bias_bwd(x, w, g, 2)
+    loss = lambda xx, ww, bb: float((oracle.conv_bias_act(xx, ww, bb, 2) * g).sum())
+    h = 1e-6
+    for arr, grad in ((x, dx), (w, dw), (bias, db)):
+        idx = tuple(int(RNG.integers(0, d)) for d in arr.shape)
+        saved = arr[idx]
+        arr[idx] = saved + h
+        lp = loss(x, w, bias)
+        arr[idx] = saved - h
+        lm = loss(x, w, bias)
+        arr[idx] = saved
+        assert grad[idx] == pytest.approx((lp - lm) / (2 * h), rel=1e-7, abs=1e-9)
+    np.testing.assert_allclose(db, g.sum(axis=(0, 1, 2)), rtol=1e-14)
