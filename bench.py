@@ -544,10 +544,13 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
     from paper_2609_10632_b200 import workloads as wl
     from paper_2609_10632_b200.detector import GraphRunner
 
-    ops, layers, outs = wl.detector_graph(16, 640)
-    run = GraphRunner(ops, layers, outs, device=local)
+    ops, layers, outs, plain = wl.detector_graph(16, 640, plain_head=True)  # up to the six raw head outputs
+    run = GraphRunner(ops, layers, outs, device=local, plain_layers=plain)
     for i, b in enumerate(run.blocks):
         b.fill_random(seed=7000 + i)  # (fills the block's own scratch x / g as well; the chained buffers are set below)
+    for pl in run.plain:
+        pl["w"].normal_(0.0, 0.05)
+        pl["bias"].normal_(0.0, 0.5)
     run.buf["img"].uniform_(0.0, 1.0)
     for name in outs:
         run.grad[name].normal_()
@@ -586,7 +589,7 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
     ms = ev0.elapsed_time(ev1) / args.steps
     gf, gb = run.glue_launches()
     tf = step_flops_value / (ms * 1e-3) / 1e12
-    return {"what": "77 chained Conv-BN-SiLU blocks + glue, fwd + bwd, batch 16, 640 x 640", "wgrad_on_second_stream": side is not None, "ms_per_step": ms, "tflops": tf,
+    return {"what": "77 chained Conv-BN-SiLU blocks + 6 plain head convolutions + glue, image -> raw head outputs, fwd + bwd, batch 16, 640 x 640", "wgrad_on_second_stream": side is not None, "ms_per_step": ms, "tflops": tf,
             "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "launches_per_step": int(launches), "glue_launches_fwd_bwd": [gf, gb],
             "cuda_graph": True}
 

@@ -158,12 +158,15 @@ def sppf_fwd_bwd(x, params, eps: float, g_out=None, pool_in_bf16: bool = False):
 
 
 # ------------------------------------------------------------------ a whole dataflow graph of blocks and glue
-def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf16: bool = False, storage_16bit: bool = False):
+def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf16: bool = False, storage_16bit: bool = False,
+                  plain_layers=None, plain_params=None):
     """Interpret a dataflow description (a list of op dicts: "cbs" with a layer index, "slice", "add", "concat", "maxpool",
     "upsample"; see the detector's description in the workload module) forwards and, given gradients for some tensors,
     backwards.  layers[k] gives block k's stride; params[k] its BlockParams.  A tensor with several consumers receives
     the sum of their gradients.  Returns (tensors, grads, block_grads): dicts name -> array, and per layer (dw, dgamma, dbeta).
     pool_in_bf16: inputs of max-pools are rounded to bf16 first (see sppf_fwd_bwd).
+    Op "plain" (convolution + bias, no BN, no activation) takes its shape from plain_layers[k] and (w, bias) from
+    plain_params[k]; its gradients (dw, dbias) are returned in a fourth value when plain_layers is given.
 
     storage_16bit: model the STORAGE precision the benchmark spec fixes for a chained run -- activations, upstream gradients,
     dy and dx are bf16 tensors, the saved convolution output is fp16 -- by rounding exactly where a tensor is stored
@@ -199,16 +202,20 @@ def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf
             T[o["out"]], saved[o["out"]] = maxpool5(src)
         elif kind == "upsample":
             T[o["out"]] = upsample2(ins[0])
+        elif kind == "plain":
+            w, bias = plain_params[o["layer"]]
+            T[o["out"]] = r16(oracle.conv_bias_act(ins[0], w, bias, plain_layers[o["layer"]].stride))
         else:
             raise ValueError(kind)
     if out_grads is None:
-        return T, None, None
+        return (T, None, None) if plain_layers is None else (T, None, None, None)
     G = {k: np.asarray(v, dtype=np.float64).copy() for k, v in out_grads.items()}
 
     def give(name, g):
         G[name] = r16(G[name] + g) if name in G else r16(g)
 
     block_grads = [None] * len(layers)
+    plain_grads = [None] * (len(plain_layers) if plain_layers is not None else 0)
     for o in reversed(ops):
         if o["out"] not in G:
             continue  # nothing downstream needs this tensor
@@ -242,4 +249,9 @@ def graph_fwd_bwd(ops, layers, params, x, eps: float, out_grads=None, pool_in_bf
             give(o["ins"][0], maxpool5_bwd(g, saved[o["out"]]))
         elif kind == "upsample":
             give(o["ins"][0], upsample2_bwd(g))
-    return T, G, block_grads
+        elif kind == "plain":
+            k = o["layer"]
+            dx, dw, db = oracle.conv_bias_bwd(T[o["ins"][0]], plain_params[k][0], g, plain_layers[k].stride)
+            plain_grads[k] = (dw, db)
+            give(o["ins"][0], r16(dx))
+    return (T, G, block_grads) if plain_layers is None else (T, G, block_grads, plain_grads)

@@ -20,8 +20,11 @@ from .block import CbsBlock
 
 
 class GraphRunner:
-    def __init__(self, ops, layers, outputs, eps=1e-3, device=0):
+    def __init__(self, ops, layers, outputs, eps=1e-3, device=0, plain_layers=None):
+        """plain_layers: shapes of the plain convolutions (bias, no BN, no activation) that "plain" ops refer to; their
+        parameters and gradients live in self.plain[k] (dict with plan, w, bias, dw, dbias, dx, ws)."""
         self.ops, self.layers, self.outputs = ops, layers, list(outputs)
+        self.plain = []
         self.dev = torch.device("cuda", device)
         s0 = layers[0]
         self.shape = {"img": (s0.n, s0.h, s0.w, s0.c_in)}
@@ -43,6 +46,17 @@ class GraphRunner:
                 blk.x = self.buf[o["ins"][0]]
                 self.blocks[o["layer"]] = blk
                 shp, buf = (s.n, s.ho, s.wo, s.c_out), blk.a
+            elif kind == "plain":
+                s = plain_layers[o["layer"]]
+                assert o["layer"] == len(self.plain) and ins[0] == (s.n, s.h, s.w, s.c_in), o["out"]
+                plan = nb.Plan.for_shape(s, eps=eps, device=device)
+                e = lambda *sz, dtype: torch.empty(*sz, dtype=dtype, device=self.dev)
+                shp = (s.n, s.ho, s.wo, s.c_out)
+                buf = e(shp, dtype=torch.bfloat16)
+                self.plain.append({"plan": plan, "shape": s, "w": e(s.c_out, s.k, s.k, s.c_in, dtype=torch.bfloat16), "bias": e(s.c_out, dtype=torch.float32),
+                                   "dw": e(s.c_out, s.k, s.k, s.c_in, dtype=torch.float32), "dbias": e(s.c_out, dtype=torch.float32),
+                                   "dx": e(s.n, s.h, s.w, s.c_in, dtype=torch.bfloat16),
+                                   "ws": e(max(plan.infer_bytes, plan.bwd_bytes, 256), dtype=torch.uint8)})
             else:
                 n, h, w, c = ins[0]
                 if kind == "slice":
@@ -64,7 +78,9 @@ class GraphRunner:
         by_out = {o["out"]: o for o in ops}
         for name in list(self.buf):
             cons = consumers.get(name, [])
-            if len(cons) == 1 and cons[0]["op"] == "cbs":
+            if len(cons) == 1 and cons[0]["op"] == "plain":
+                self.grad[name] = self.plain[cons[0]["layer"]]["dx"]
+            elif len(cons) == 1 and cons[0]["op"] == "cbs":
                 self.grad[name] = self.blocks[cons[0]["layer"]].dx
             else:
                 self.grad[name] = torch.zeros(self.shape[name], dtype=torch.bfloat16, device=self.dev)
@@ -123,6 +139,9 @@ class GraphRunner:
             c_out = self.shape[out][3]
             if kind == "cbs":
                 self.blocks[o["layer"]].forward(stream)
+            elif kind == "plain":
+                pl = self.plain[o["layer"]]
+                nb.nb_conv_bias_act(pl["plan"], B[ins[0]], pl["w"], pl["bias"], 0, B[out], pl["ws"], stream)
             elif kind == "slice":
                 self._copy(B[out], c_out, self._at(B[ins[0]], o["c0"]), self.shape[ins[0]][3], rows, c_out, stream=stream)
             elif kind == "add":
@@ -166,6 +185,10 @@ class GraphRunner:
                 if G[src] is not blk.dx:
                     c = self.shape[src][3]
                     self._copy(G[src], c, blk.dx, c, self._rows(src), c, accumulate=self.acc[(oi, 0)], stream=stream)
+            elif kind == "plain":
+                pl = self.plain[o["layer"]]
+                nb.nb_conv_bias_bwd(pl["plan"], self.buf[ins[0]], pl["w"], G[out], pl["dx"], pl["dw"], pl["dbias"], pl["ws"], stream)
+                assert G[ins[0]] is pl["dx"]  # a plain convolution is the only consumer of its input in this dataflow
             elif kind == "slice":
                 src = ins[0]
                 self._copy(self._at(G[src], o["c0"]), self.shape[src][3], G[out], c_out, self._rows(out), c_out, accumulate=self.acc[(oi, 0)], stream=stream)
@@ -190,7 +213,8 @@ class GraphRunner:
             b.poll()
 
     def glue_launches(self):
-        fwd = sum(len(o["ins"]) if o["op"] == "concat" else 1 for o in self.ops if o["op"] != "cbs")
-        bwd = sum(len(o["ins"]) if o["op"] in ("concat", "add") else 1 for o in self.ops if o["op"] != "cbs")
+        glue = [o for o in self.ops if o["op"] not in ("cbs", "plain")]
+        fwd = sum(len(o["ins"]) if o["op"] == "concat" else 1 for o in glue)
+        bwd = sum(len(o["ins"]) if o["op"] in ("concat", "add") else 1 for o in glue)
         bwd += sum(1 for o in self.ops if o["op"] == "cbs" and self.grad[o["ins"][0]] is not self.blocks[o["layer"]].dx)
         return fwd, bwd

@@ -121,15 +121,19 @@ def detector_plain_head_convs():
     return [(64, 64), (192, 80)] * 3
 
 
-def detector_graph(batch: int = 16, image: int = 640):
+def detector_graph(batch: int = 16, image: int = 640, plain_head: bool = False):
     """The detector's dataflow up to the last Conv-BN-SiLU block of every head branch, as a list of primitive operations
     over named tensors (a description only: no arithmetic here, both the GPU runner and the CPU oracle interpret it).
 
     Returns (ops, layers, outputs): `layers` = detector_layers(batch, image); every op is a dict with "out", "op" and
     "ins": op "cbs" (+ "layer": index into layers), "slice" (+ "c0", "c1": channel range), "add", "concat", "maxpool"
     (5x5, stride 1), "upsample" (nearest 2x); tensor "img" is the input image batch; `outputs` names the six head tensors
-    (box and class branch of the three levels), which feed the plain output convolutions and the loss (not part of this).
+    (box and class branch of the three levels), which feed the plain output convolutions and the loss.
     Backbone C2f units have the residual shortcut, neck units do not.
+
+    plain_head=True appends the six plain 1x1 output convolutions (bias, no BN, no activation): op "plain" with "layer" =
+    index into a fourth return value, the list of their ConvShapes; `outputs` then names the six raw head outputs
+    (64 box-distribution channels and 80 class logits per level).
     """
     layers = detector_layers(batch, image)
     index = {s.name: i for i, s in enumerate(layers)}
@@ -180,7 +184,17 @@ def detector_graph(batch: int = 16, image: int = 640):
     for lvl, src in enumerate([n15, n18, n21]):
         outputs.append(cbs(f"h22.box{lvl}.1", cbs(f"h22.box{lvl}.0", src)))
         outputs.append(cbs(f"h22.cls{lvl}.1", cbs(f"h22.cls{lvl}.0", src)))
-    return ops, layers, outputs
+    if not plain_head:
+        return ops, layers, outputs
+    plain, raw = [], []
+    for j, (src, (cin, cout)) in enumerate(zip(outputs, detector_plain_head_convs())):
+        s = layers[index[src]]
+        assert s.c_out == cin
+        name = src.replace(".1", ".out")
+        plain.append(ConvShape(name, batch, s.ho, s.wo, cin, cout, 1, 1))
+        ops.append({"out": name, "op": "plain", "ins": [src], "layer": j})
+        raw.append(name)
+    return ops, layers, raw, plain
 
 
 def detector_parameter_tensors():

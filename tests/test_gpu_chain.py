@@ -238,8 +238,16 @@ def test_detector_dataflow_matches_graph_oracle():
 
     from paper_2609_10632_b200.detector import GraphRunner
 
-    ops, layers, outs = wl.detector_graph(2, 256)
-    run = GraphRunner(ops, layers, outs, eps=EPS)
+    ops, layers, outs, plain = wl.detector_graph(2, 256, plain_head=True)  # up to the six raw head outputs
+    run = GraphRunner(ops, layers, outs, eps=EPS, plain_layers=plain)
+    pparams = []
+    for j, pl in enumerate(run.plain):
+        w = wl.make_inputs(plain[j], 54, j, bf16=True).w
+        bias = wl.make_eval_stats(plain[j], 54, j)[2]
+        pparams.append((w, bias))
+        pl["w"].copy_(torch.from_numpy(w).to(torch.bfloat16))
+        pl["bias"].copy_(torch.from_numpy(bias))
+    kw = dict(plain_layers=plain, plain_params=pparams)
     params = []
     for k, blk in enumerate(run.blocks):
         inp = wl.make_inputs(layers[k], 53, k, bf16=True, affine="random")
@@ -260,8 +268,8 @@ def test_detector_dataflow_matches_graph_oracle():
     torch.cuda.synchronize()
     run.poll()
     f64 = lambda t: t.detach().double().cpu().numpy()
-    T0, G0, b0 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts)                      # exact
-    T1, G1, b1 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts, storage_16bit=True)  # the yardstick
+    T0, G0, b0, q0 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts, **kw)                      # exact
+    T1, G1, b1, q1 = chain.graph_fwd_bwd(ops, layers, params, x, EPS, gouts, storage_16bit=True, **kw)  # the yardstick
     worst = {"ratio": 0.0, "gpu": 0.0, "yardstick": 0.0}
 
     def held(name, got, exact, stored):
@@ -277,6 +285,9 @@ def test_detector_dataflow_matches_graph_oracle():
     for k, blk in enumerate(run.blocks):
         for slot, t in enumerate((blk.dw, blk.dgamma, blk.dbeta)):
             held(f"{layers[k].name}.{('dw', 'dgamma', 'dbeta')[slot]}", f64(t), b0[k][slot], b1[k][slot])
+    for j, pl in enumerate(run.plain):
+        held(f"{plain[j].name}.dw", f64(pl["dw"]), q0[j][0], q1[j][0])
+        held(f"{plain[j].name}.dbias", f64(pl["dbias"]), q0[j][1], q1[j][1])
     print("worst:", {k: f"{v:.2e}" for k, v in worst.items()}, "glue launches fwd/bwd:", run.glue_launches())
 
 

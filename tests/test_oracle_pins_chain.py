@@ -186,16 +186,18 @@ def test_detector_graph_finite_differences_at_a_tiny_size():
     (backbone behind the pools, neck, head) against central differences of sum(outputs * G)."""
     from paper_2609_10632_b200 import workloads as wl
 
-    ops, layers, outs = wl.detector_graph(2, 64)
+    ops, layers, outs, plain = wl.detector_graph(2, 64, plain_head=True)  # up to the raw head outputs
     prm = _detector_params(layers)
+    pprm = [(RNG.uniform(-1, 1, (s.c_out, 1, 1, s.c_in)) / np.sqrt(s.c_in), RNG.normal(size=s.c_out) * 0.5) for s in plain]
+    kw = dict(plain_layers=plain, plain_params=pprm)
     x = RNG.uniform(0, 1, (2, 64, 64, 3))
-    T, _, _ = chain.graph_fwd_bwd(ops, layers, prm, x, EPS)
+    T = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, **kw)[0]
     Gs = {name: RNG.normal(size=T[name].shape) for name in outs}
-    T, grads, bg = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, Gs)
-    assert all(g is not None for g in bg)
+    T, grads, bg, pg = chain.graph_fwd_bwd(ops, layers, prm, x, EPS, Gs, **kw)
+    assert all(g is not None for g in bg) and all(g is not None for g in pg)
 
     def loss(xx):
-        TT, _, _ = chain.graph_fwd_bwd(ops, layers, prm, xx, EPS)
+        TT = chain.graph_fwd_bwd(ops, layers, prm, xx, EPS, **kw)[0]
         return float(sum((TT[n] * Gs[n]).sum() for n in outs))
 
     v = RNG.normal(size=x.shape)
@@ -215,6 +217,17 @@ def test_detector_graph_finite_differences_at_a_tiny_size():
         lm = loss(x)
         w[idx] = saved
         assert bg[k][0][idx] == pytest.approx((lp - lm) / (2 * hh), rel=5e-4, abs=1e-6), lname
+
+    # a plain head convolution: one filter entry and one bias entry
+    w, b = pprm[3]
+    for arr, grad, idx in ((w, pg[3][0], (5, 0, 0, 7)), (b, pg[3][1], (11,))):
+        saved = arr[idx]
+        arr[idx] = saved + 1e-5
+        lp = loss(x)
+        arr[idx] = saved - 1e-5
+        lm = loss(x)
+        arr[idx] = saved
+        assert grad[idx] == pytest.approx((lp - lm) / 2e-5, rel=5e-4, abs=1e-6)
 
 
 def test_storage_rounding_mode_stays_close_to_the_exact_graph_on_a_shallow_unit():
