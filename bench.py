@@ -557,8 +557,22 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
 
     side = None if args.no_wgrad_stream else torch.cuda.Stream(device=dev)
     side_ws = None if side is None else torch.empty(max(b.plan.bwd_bytes for b in run.blocks), dtype=torch.uint8, device=dev)
+    # the optimiser step over the chain's 243 gradient tensors: fp32 masters and momentum here, the blocks' bf16 filters are
+    # the working copies it rewrites; BN gains / shifts and the plain biases are fp32 parameters updated in place
+    items = []
+    for b in run.blocks:
+        items.append((b.dw, b.w.float().reshape(-1).clone(), torch.zeros(b.w.numel(), dtype=torch.float32, device=dev), b.w, 0))
+        items.append((b.dgamma, b.gamma, torch.zeros_like(b.gamma), None, 1))
+        items.append((b.dbeta, b.beta, torch.zeros_like(b.beta), None, 2))
+    for pl in run.plain:
+        items.append((pl["dw"], pl["w"].float().reshape(-1).clone(), torch.zeros(pl["w"].numel(), dtype=torch.float32, device=dev), pl["w"], 0))
+        items.append((pl["dbias"], pl["bias"], torch.zeros_like(pl["bias"]), None, 2))
+    sgd = nb.SgdPlan(items, device=local)
+    sgd_ws = torch.empty(sgd.workspace_bytes, dtype=torch.uint8, device=dev)
+    sgd.upload(sgd_ws)
+    hyper = dict(lr=[1e-4, 1e-4, 1e-4], weight_decay=[3.75e-4, 0.0, 0.0], momentum=0.937, max_norm=10.0)  # Table 1 (small lr: random gradients)
 
-    def step():
+    def step(with_update=False):
         run.forward()
         if side is None:
             run.backward()
@@ -567,6 +581,8 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
             side.wait_stream(main)
             run.backward(wgrad_stream=side, wgrad_workspace=side_ws)
             main.wait_stream(side)
+        if with_update:
+            sgd.step(sgd_ws, first_step=False, **hyper)
 
     for _ in range(max(3, args.warmup)):
         step()
@@ -587,11 +603,27 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
     torch.cuda.synchronize()
     run.poll()
     ms = ev0.elapsed_time(ev1) / args.steps
+    # the same with the clip + SGD-Nesterov update of all 243 tensors behind it: one training iteration minus the loss
+    sgd.step(sgd_ws, first_step=True, **hyper)
+    torch.cuda.synchronize()
+    graph2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph2):
+        step(with_update=True)
+    graph2.replay()
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(args.steps):
+        graph2.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    run.poll()
+    ms_upd = ev0.elapsed_time(ev1) / args.steps
+    finite = all(bool(torch.isfinite(b.w.float()).all()) for b in run.blocks[:3])
     gf, gb = run.glue_launches()
     tf = step_flops_value / (ms * 1e-3) / 1e12
     return {"what": "77 chained Conv-BN-SiLU blocks + 6 plain head convolutions + glue, image -> raw head outputs, fwd + bwd, batch 16, 640 x 640", "wgrad_on_second_stream": side is not None, "ms_per_step": ms, "tflops": tf,
             "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "launches_per_step": int(launches), "glue_launches_fwd_bwd": [gf, gb],
-            "cuda_graph": True}
+            "ms_per_step_with_optimizer_update": ms_upd, "optimizer_tensors": len(items), "weights_finite_after_updates": finite, "cuda_graph": True}
 
 
 def run_optimizer_step(args, blocks, dev, local, peaks):
