@@ -63,3 +63,29 @@ def clip_sgd_step(params, grads, bufs, groups, lr, weight_decay, momentum: float
         new_p.append(q)
         new_b.append(nb_)
     return new_p, new_b, total
+
+
+# ------------------------------------------------------------------ dynamic loss scaling (Sec. 3.2 "Mixed precision", Table 1, Table 2 row 4)
+def scaled_clip_sgd_step(params, grads, bufs, groups, lr, weight_decay, momentum: float, max_norm: float, first_step: bool,
+                         scale: float, growth_tracker: int, growth_factor: float = 2.0, backoff_factor: float = 0.5,
+                         growth_interval: int = 2000, floor: float = 0.0):
+    """One optimiser step when the gradients arrive multiplied by the loss scale (the paper's recipe: initial scale 2^16,
+    dynamic, with a FLOOR -- Table 2 row 4: without it per-rank overflows drove the scale towards zero).  The dominant
+    framework's scaler semantics, which the paper keeps:
+
+      unscale: g <- g / scale;  if any gradient element is inf or NaN the step is SKIPPED (parameters and momentum
+      untouched), scale <- max(scale * backoff_factor, floor), growth_tracker <- 0;
+      otherwise clip + update as clip_sgd_step on the unscaled gradients, growth_tracker += 1, and after growth_interval
+      consecutive good steps scale <- scale * growth_factor, growth_tracker <- 0.
+
+    Returns (params, bufs, total_norm of the unscaled gradients or inf/nan, scale, growth_tracker, skipped)."""
+    inv = 1.0 / float(scale)
+    unscaled = [np.asarray(g, dtype=np.float64) * inv for g in grads]
+    finite = all(bool(np.isfinite(g).all()) for g in unscaled)
+    if not finite:
+        return list(params), list(bufs), float("nan"), max(float(scale) * backoff_factor, float(floor)), 0, True
+    new_p, new_b, total = clip_sgd_step(params, unscaled, bufs, groups, lr, weight_decay, momentum, max_norm, first_step)
+    growth_tracker += 1
+    if growth_tracker == growth_interval:
+        scale, growth_tracker = float(scale) * growth_factor, 0
+    return new_p, new_b, total, float(scale), growth_tracker, False

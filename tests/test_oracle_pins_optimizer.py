@@ -67,3 +67,46 @@ def test_against_the_frameworks_cpu_optimiser_in_float64():
         assert total == pytest.approx(tn, rel=1e-12)
         for p, tp in zip(params, tparams):
             np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_loss_scaler_against_the_frameworks_cpu_scaler():
+    torch = pytest.importorskip("torch")
+    shapes, groups = [(6, 4), (6,)], [0, 2]
+    lr, wd, mom, max_norm = [0.05, 0.1, 0.1], [1e-3, 0.0, 0.0], 0.9, 1.0
+    params = [RNG.normal(size=s) for s in shapes]
+    tparams = [torch.tensor(p, dtype=torch.float64, requires_grad=True) for p in params]
+    sgd = torch.optim.SGD([{"params": [tparams[0]], "lr": lr[0], "weight_decay": wd[0]}, {"params": [tparams[1]], "lr": lr[2], "weight_decay": wd[2]}],
+                          lr=0.1, momentum=mom, nesterov=True)
+    scaler = torch.amp.GradScaler("cpu", init_scale=1024.0, growth_factor=2.0, backoff_factor=0.5, growth_interval=2)
+    scale, tracker, bufs, first = 1024.0, 0, [None, None], True
+    for step in range(7):
+        grads = [RNG.normal(size=s) * scale for s in shapes]  # what the backward pass of a scaled loss delivers
+        if step in (1, 4):
+            grads[0][2, 1] = np.inf if step == 1 else np.nan
+        scaler.scale(torch.tensor(1.0))
+        for tp, g in zip(tparams, grads):
+            tp.grad = torch.tensor(g, dtype=torch.float64)
+        scaler.unscale_(sgd)
+        torch.nn.utils.clip_grad_norm_(tparams, max_norm)
+        scaler.step(sgd)
+        scaler.update()
+        params, bufs, total, scale, tracker, skipped = opt.scaled_clip_sgd_step(params, grads, bufs, groups, lr, wd, mom, max_norm, first, scale, tracker,
+                                                                                 2.0, 0.5, 2, floor=0.0)
+        if not skipped:
+            first = False
+        assert skipped == (step in (1, 4))
+        assert scale == scaler.get_scale() and tracker == int(scaler._growth_tracker)
+        for p, tp in zip(params, tparams):
+            np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_loss_scaler_floor_and_hand_sequence():
+    p, g = [np.array([1.0])], [np.array([np.inf])]
+    scale, tracker = 4.0, 1
+    for want in (2.0, 1.5, 1.5):  # halves until the floor 1.5 holds it
+        p2, _, total, scale, tracker, skipped = opt.scaled_clip_sgd_step(p, g, [None], [0], [0.1] * 3, [0.0] * 3, 0.9, 10.0, True, scale, tracker, floor=1.5)
+        assert skipped and scale == want and tracker == 0 and p2[0][0] == 1.0 and not np.isfinite(total)
+    # a good step with scale 8: gradient 16 means 2; lr 0.1, no momentum history: p = 1 - 0.1*(2 + 0.9*2) = 0.62
+    p2, b2, total, scale, tracker, skipped = opt.scaled_clip_sgd_step([np.array([1.0])], [np.array([16.0])], [None], [0], [0.1] * 3, [0.0] * 3, 0.9, 10.0, True,
+                                                                      8.0, 0, growth_interval=1)
+    assert not skipped and total == pytest.approx(2.0) and p2[0][0] == pytest.approx(0.62) and scale == 16.0 and tracker == 0
