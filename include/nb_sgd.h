@@ -54,6 +54,24 @@ typedef struct nb_sgd_hyper {
     int32_t first_step;   /* non-zero: the momentum buffers hold nothing yet */
 } nb_sgd_hyper;
 
+/* Dynamic loss scaling (Sec. 3.2 "Mixed precision"; Table 1: initial scale 2^16; Table 2 row 4: a FLOOR keeps repeated
+ * overflows from driving the scale towards zero).  The state lives in DEVICE memory and never visits the host:
+ * the gradients handed to the step are the gradients of (scale * loss). */
+typedef struct nb_loss_scaler {
+    float scale;            /* current loss scale; initialise (e.g. 65536) before the first step */
+    int32_t growth_tracker; /* consecutive good steps since the last change; initialise to 0 */
+    int32_t skipped;        /* written by every step: 1 if it was skipped because a gradient was inf or NaN */
+    int32_t reserved;
+} nb_loss_scaler;
+
+typedef struct nb_scaler_hyper {
+    uint32_t struct_size;  /* = sizeof(nb_scaler_hyper) */
+    float growth_factor;   /* 2.0 */
+    float backoff_factor;  /* 0.5 */
+    float floor_scale;     /* the scale never drops below this (0 = no floor) */
+    int32_t growth_interval; /* good steps before the scale grows (2000) */
+} nb_scaler_hyper;
+
 typedef struct nb_sgd_plan_s* nb_sgd_plan; /* opaque, caller-owned, host memory only */
 
 /* Validate a tensor list (a HOST array of `count` entries holding DEVICE pointers on device `device`) and build
@@ -80,6 +98,16 @@ nb_status nb_sgd_upload(nb_sgd_plan plan, void* workspace, size_t workspace_byte
  * Errors: NB_ERR_INVALID_ARG (NULL, struct_size mismatch), NB_ERR_WORKSPACE, NB_ERR_ALIGNMENT, NB_ERR_CUDA. */
 nb_status nb_sgd_clip_nesterov_step(nb_sgd_plan plan, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper,
                                     float* total_norm, void* stream);
+
+/* The same step for gradients that arrive multiplied by state->scale: they are unscaled (g / scale) on the fly, the
+ * clip threshold applies to the unscaled norm (which total_norm receives), and if any gradient element is inf or NaN
+ * the step is SKIPPED: parameters, momentum and working copies stay untouched.  Then the state is advanced:
+ *   skipped:  scale = max(scale * backoff_factor, floor_scale), growth_tracker = 0, skipped = 1
+ *   otherwise growth_tracker += 1; when it reaches growth_interval: scale *= growth_factor, growth_tracker = 0; skipped = 0
+ * Three launches (norm partials; clip + update; scaler state), no host readback; `state` is a device pointer, 16-byte
+ * aligned.  Errors as nb_sgd_clip_nesterov_step, plus NB_ERR_INVALID_ARG for a NULL state or scaler. */
+nb_status nb_sgd_clip_nesterov_step_scaled(nb_sgd_plan plan, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper,
+                                           const nb_scaler_hyper* scaler, nb_loss_scaler* state, float* total_norm, void* stream);
 
 #ifdef __cplusplus
 }

@@ -27,7 +27,7 @@ EXPORTS = (
     "nb_conv_bn_silu_bwd_data", "nb_conv_bn_silu_bwd_weight", "nb_cbs_step_host_scratch_bytes",
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
-    "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step",
+    "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step", "nb_sgd_clip_nesterov_step_scaled",
     "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd",
 )
 
@@ -47,6 +47,10 @@ class nb_sgd_tensor(Structure):
 class nb_sgd_hyper(Structure):
     _fields_ = [("struct_size", c_uint32), ("momentum", c_float), ("max_norm", c_float), ("lr", c_float * 3), ("weight_decay", c_float * 3),
                 ("first_step", c_int32)]
+
+
+class nb_scaler_hyper(Structure):
+    _fields_ = [("struct_size", c_uint32), ("growth_factor", c_float), ("backoff_factor", c_float), ("floor_scale", c_float), ("growth_interval", c_int32)]
 
 
 class NbError(RuntimeError):
@@ -94,6 +98,7 @@ def load() -> ctypes.CDLL:
         lib.nb_sgd_workspace_bytes.argtypes = [V, POINTER(c_size_t)]
         lib.nb_sgd_upload.argtypes = [V, V, c_size_t, V]
         lib.nb_sgd_clip_nesterov_step.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), FP, V]
+        lib.nb_sgd_clip_nesterov_step_scaled.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), POINTER(nb_scaler_hyper), V, FP, V]
         lib.nb_slice_add.argtypes = [c_int32, ctypes.c_int64, c_int32, V, ctypes.c_int64, V, ctypes.c_int64, V, ctypes.c_int64, c_int32, V]
         lib.nb_maxpool5_fwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, V]
         lib.nb_maxpool5_bwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, c_int32, V]
@@ -325,6 +330,14 @@ class SgdPlan:
     def step(self, workspace, lr, weight_decay, momentum, max_norm, first_step, total_norm=None, stream=None):
         h = nb_sgd_hyper(ctypes.sizeof(nb_sgd_hyper), momentum, max_norm, (c_float * 3)(*lr), (c_float * 3)(*weight_decay), 1 if first_step else 0)
         _check(load().nb_sgd_clip_nesterov_step(self.handle, _ptr(workspace), _nbytes(workspace), byref(h), _ptr(total_norm), _stream(stream)))
+
+    def step_scaled(self, workspace, state, lr, weight_decay, momentum, max_norm, first_step, growth_factor=2.0, backoff_factor=0.5, floor_scale=0.0,
+                    growth_interval=2000, total_norm=None, stream=None):
+        """`state`: a 16-byte device buffer laid out as nb_loss_scaler (float scale, int32 growth_tracker, int32 skipped, int32 reserved)."""
+        h = nb_sgd_hyper(ctypes.sizeof(nb_sgd_hyper), momentum, max_norm, (c_float * 3)(*lr), (c_float * 3)(*weight_decay), 1 if first_step else 0)
+        sc = nb_scaler_hyper(ctypes.sizeof(nb_scaler_hyper), growth_factor, backoff_factor, floor_scale, growth_interval)
+        _check(load().nb_sgd_clip_nesterov_step_scaled(self.handle, _ptr(workspace), _nbytes(workspace), byref(h), byref(sc), _ptr(state), _ptr(total_norm),
+                                                       _stream(stream)))
 
     def close(self):
         if self.handle:

@@ -1001,9 +1001,31 @@ nb_status nb_sgd_upload(nb_sgd_plan p, void* workspace, size_t workspace_bytes, 
     return NB_OK;
 }
 
+namespace {
+nb_status sgd_step_impl(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc, nb_loss_scaler* state,
+                        float* total_norm, void* stream);
+}
 nb_status nb_sgd_clip_nesterov_step(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, float* total_norm,
                                     void* stream) {
     g_err.clear();
+    return sgd_step_impl(p, workspace, workspace_bytes, hyper, nullptr, nullptr, total_norm, stream);
+}
+
+nb_status nb_sgd_clip_nesterov_step_scaled(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc,
+                                           nb_loss_scaler* state, float* total_norm, void* stream) {
+    g_err.clear();
+    if (!sc || !state) return fail(NB_ERR_INVALID_ARG, "scaler and state must not be NULL");
+    if (sc->struct_size != sizeof(nb_scaler_hyper)) return fail(NB_ERR_INVALID_ARG, "nb_scaler_hyper.struct_size is %u, expected %zu", sc->struct_size, sizeof(nb_scaler_hyper));
+    if (reinterpret_cast<uintptr_t>(state) & 15u) return fail(NB_ERR_ALIGNMENT, "state is not 16-byte aligned");
+    if (!(sc->growth_factor > 0.f) || !(sc->backoff_factor > 0.f) || sc->growth_interval < 1) return fail(NB_ERR_INVALID_ARG, "scaler factors must be positive, growth_interval >= 1");
+    return sgd_step_impl(p, workspace, workspace_bytes, hyper, sc, state, total_norm, stream);
+}
+
+}  // extern "C"
+
+namespace {
+nb_status sgd_step_impl(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc, nb_loss_scaler* state,
+                        float* total_norm, void* stream) {
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     if (!hyper) return fail(NB_ERR_INVALID_ARG, "hyper is NULL");
     if (hyper->struct_size != sizeof(nb_sgd_hyper))
@@ -1014,15 +1036,20 @@ nb_status nb_sgd_clip_nesterov_step(nb_sgd_plan p, void* workspace, size_t works
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SgdScalars s;
     s.momentum = hyper->momentum; s.max_norm = hyper->max_norm; s.first_step = hyper->first_step;
+    s.scaler = state;
     for (int i = 0; i < NB_SGD_GROUPS; ++i) { s.lr[i] = hyper->lr[i]; s.wd[i] = hyper->weight_decay[i]; }
     const uint8_t* ws = static_cast<const uint8_t*>(workspace);
     launch_k(sgd_sqnorm_kernel, dim3((unsigned)p->h.grid), dim3(SGD_THREADS), 0, st, 1, ws);
     NB_LAUNCH_OK("sgd_sqnorm");
     launch_k(sgd_update_kernel, dim3((unsigned)p->h.grid), dim3(SGD_THREADS), 0, st, 1, ws, s, total_norm);
-    return launch_ok("sgd_update");
+    NB_LAUNCH_OK("sgd_update");
+    if (state) {
+        launch_k(sgd_scaler_kernel, dim3(1), dim3(32), 0, st, 1, ws, state, sc->growth_factor, sc->backoff_factor, sc->floor_scale, (int)sc->growth_interval);
+        NB_LAUNCH_OK("sgd_scaler");
+    }
+    return NB_OK;
 }
-
-}  // extern "C"
+}  // namespace
 
 // ---------------------------------------------------------------- glue between chained blocks (include/nb_glue.h)
 namespace {

@@ -72,6 +72,8 @@ struct SgdScalars {
     float momentum, max_norm;
     float lr[NB_SGD_GROUPS], wd[NB_SGD_GROUPS];
     int first_step;
+    // dynamic loss scaling (scaler == NULL: gradients are unscaled): the gradients arrive multiplied by scaler->scale
+    const nb_loss_scaler* scaler;
 };
 
 __device__ __forceinline__ void sgd_one(float g, float& p, float& b, float coef, float lr, float wd, float mom, bool first) {
@@ -93,14 +95,19 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
     double acc = 0.0;
     for (int i = threadIdx.x; i < H.grid; i += SGD_THREADS) acc += partials[i];
     const double t = block_sum_fixed_order(acc, red);
+    __shared__ int s_skip;
     if (threadIdx.x == 0) {
-        const double total = sqrt(t);
+        // the state is read here and rewritten only by the scaler kernel that runs after this one
+        const double inv = hs.scaler ? 1.0 / (double)hs.scaler->scale : 1.0;
+        const double total = sqrt(t) * inv;  // norm of the unscaled gradients; inf or NaN if any gradient element is
         double c = 1.0;
         if (hs.max_norm > 0.f && hs.max_norm < __int_as_float(0x7f800000)) c = fmin((double)hs.max_norm / (total + 1e-6), 1.0);
-        s_coef = (float)c;
+        s_coef = (float)(c * inv);
+        s_skip = (hs.scaler && !isfinite(t)) ? 1 : 0;
         if (blockIdx.x == 0 && total_norm_out) *total_norm_out = (float)total;
     }
     __syncthreads();
+    if (s_skip) return;  // overflow under loss scaling: parameters and momentum stay as they are
     const float coef = s_coef, mom = hs.momentum;
     const bool first = hs.first_step != 0;
     for (int c = blockIdx.x; c < H.nchunks; c += gridDim.x) {
@@ -149,6 +156,30 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
             p[i] = pv;
             b[i] = bv;
             if (lp) lp[i] = __float2bfloat16_rn(pv);
+        }
+    }
+}
+
+// After the update kernel: the scaler's state for the next step (one thread).  found_inf is recomputed from the same
+// partial sums in the same order.
+__global__ void sgd_scaler_kernel(const uint8_t* __restrict__ ws, nb_loss_scaler* state, float growth_factor, float backoff_factor, float floor_scale,
+                                  int growth_interval) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const SgdHeader& H = *reinterpret_cast<const SgdHeader*>(ws);
+    const double* partials = reinterpret_cast<const double*>(ws + H.off_partials);
+    double t = 0.0;
+    for (int i = 0; i < H.grid; ++i) t += partials[i];
+    if (!isfinite(t)) {
+        state->scale = fmaxf(state->scale * backoff_factor, floor_scale);
+        state->growth_tracker = 0;
+        state->skipped = 1;
+    } else {
+        state->skipped = 0;
+        if (++state->growth_tracker >= growth_interval) {
+            state->scale *= growth_factor;
+            state->growth_tracker = 0;
         }
     }
 }

@@ -138,3 +138,48 @@ def test_argument_checks():
     with pytest.raises(nb.NbError) as e:
         plan.upload(ws[:256])
     assert e.value.status == nb.NB_ERR_WORKSPACE
+
+
+def test_loss_scaled_steps_skip_on_overflow_and_follow_the_scaler_dynamics():
+    """Gradients arrive multiplied by the loss scale; steps 1 and 4 carry an inf / a NaN and must be skipped (parameters,
+    momentum and bf16 copies untouched, scale halved down to the floor); after two good steps in a row the scale doubles.
+    Parameters against the oracle at the fp32 bar, scaler state exactly."""
+    import struct
+
+    import torch
+
+    sizes, groups = [5000, 64, 4097], [0, 1, 2]
+    st = State(sizes, groups, cfg_id=35)
+    dev = st.p[0].device
+    state = torch.zeros(4, dtype=torch.int32, device=dev)
+    state[0] = struct.unpack("i", struct.pack("f", 1024.0))[0]
+    scale, tracker, first = 1024.0, 0, True
+    read = lambda: (struct.unpack("f", struct.pack("i", int(state[0].item())))[0], int(state[1].item()), int(state[2].item()))
+    for k in range(7):
+        _, grads = wl.make_optimizer_inputs(sizes, 35, k, 0.3)
+        grads = [(g * np.float32(scale)).astype(np.float32) for g in grads]
+        if k == 1:
+            grads[0][123] = np.inf
+        if k == 4:
+            grads[2][4096] = np.nan
+        for d, h in zip(st.g, grads):
+            d.copy_(torch.from_numpy(h))
+        before = [p.clone() for p in st.p], [m.clone() for m in st.m], [None if l is None else l.clone() for l in st.lp]
+        st.plan.step_scaled(st.ws, state, LR, WD, MOM, 1.0, first_step=first, growth_interval=2, floor_scale=300.0, total_norm=st.norm)
+        torch.cuda.synchronize()
+        st.h_params, st.h_bufs, total, scale, tracker, skipped = opt.scaled_clip_sgd_step(st.h_params, grads, st.h_bufs, groups, LR, WD, MOM, 1.0, first, scale,
+                                                                                          tracker, 2.0, 0.5, 2, floor=300.0)
+        assert read() == (scale, tracker, int(skipped)), (k, read(), scale, tracker, skipped)
+        if skipped:
+            assert k in (1, 4)
+            for i in range(len(sizes)):
+                assert torch.equal(st.p[i], before[0][i]) and (first or torch.equal(st.m[i], before[1][i]))
+                assert st.lp[i] is None or torch.equal(st.lp[i], before[2][i])
+            assert not np.isfinite(float(st.norm.item()))
+        else:
+            first = False
+            assert float(st.norm.item()) == pytest.approx(total, rel=2e-6)
+            for i in range(len(sizes)):
+                parity.check(f"param[{i}]", st.p[i].double().cpu().numpy(), st.h_params[i], "f32")
+                parity.check(f"momentum[{i}]", st.m[i].double().cpu().numpy(), st.h_bufs[i], "f32")
+    assert scale == 1024.0  # 1024 -> 512 (skip) -> 1024 (two good steps) -> 512 (skip) -> 1024 (two good steps)
