@@ -266,6 +266,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=6, help="streams of the end-to-end arm (1 = no overlap of copies and compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--f16", action="store_true", help="run the per-layer step in NB_MODE_F16_TC (fp16 operands, the paper's own 16-bit format) "
+                    "instead of bf16; the chained-detector and end-to-end objects are skipped")
     ap.add_argument("--no-chain", action="store_true", help="skip the chained C2f units measurement (extra object of the JSON line)")
     ap.add_argument("--no-optimizer", action="store_true", help="skip the fused clip + SGD-Nesterov step measurement (extra object of the JSON line)")
     ap.add_argument("--no-eval-forward", action="store_true", help="skip the evaluation-mode forward measurement (extra object of the JSON line)")
@@ -305,7 +307,10 @@ def main():
     ws_bytes = max(max(p.fwd_bytes, p.bwd_bytes) for p in plans_probe)
     del plans_probe
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    blocks = [CbsBlock(s, flags=flags, device=local, workspace=ws) for s in layers]
+    mode = nb.NB_MODE_F16_TC if args.f16 else nb.NB_MODE_BF16_TC
+    if args.f16:
+        args.no_chain = args.no_e2e = True
+    blocks = [CbsBlock(s, mode=mode, flags=flags, device=local, workspace=ws) for s in layers]
     for i, b in enumerate(blocks):
         b.fill_random(seed=1000 + i)
     resident = sum(sum(t.numel() * t.element_size() for t in (b.x, b.w, b.g, b.y, b.a, b.dy, b.dx, b.dw)) for b in blocks)
@@ -470,7 +475,7 @@ def main():
                 paths[k] += b.plan.paths[k]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16" if args.f16 else "bf16", "data": "synthetic",
             "config": {
                 "workload": f"{args.workload}: {len(layers)} Conv-BN-SiLU layers, batch {layers[0].n}, fwd + bwd_data + bwd_weight per layer "
                             f"(stem data gradient included), each layer on its own tensors",

@@ -21,6 +21,11 @@
  *                     (an internal tensor: same bytes as bf16, 8x finer, saturated at +-65504);
  *                     accumulation and all BN/SiLU arithmetic in fp32; dw, dgamma, dbeta fp32.
  *   NB_MODE_F32_REF : every tensor fp32, plain FMA arithmetic (no tensor cores, no TF32).
+ *   NB_MODE_F16_TC  : as NB_MODE_BF16_TC with IEEE fp16 in place of bf16 for x, w, a, g, dy, dx (the paper's own
+ *                     mixed-precision policy, Sec. 3.2: F16 convolutions, F32 BN, dynamic loss scaling -- the scaler
+ *                     is nb_sgd_clip_nesterov_step_scaled).  Same tensor-core kernels with fp16 operand formats;
+ *                     16-bit stores saturate at +-65504 and the tensor-core epilogues count saturations in the
+ *                     status block.
  *
  * Every pointer is a DEVICE pointer on the plan's device unless its name starts with `host_`; the
  * caller owns all memory, including the workspace.  Tensor pointers must be 16-byte aligned.
@@ -61,7 +66,7 @@ enum {
 };
 
 typedef enum { NB_DTYPE_F32 = 0, NB_DTYPE_BF16 = 1, NB_DTYPE_F16 = 2 } nb_dtype;
-typedef enum { NB_MODE_BF16_TC = 0, NB_MODE_F32_REF = 1 } nb_mode;
+typedef enum { NB_MODE_BF16_TC = 0, NB_MODE_F32_REF = 1, NB_MODE_F16_TC = 2 } nb_mode;
 
 /* nb_cbs_desc.flags */
 #define NB_CBS_FLAG_FORCE_SIMT 1u /* BF16 mode: run the three convolutions on the CUDA-core kernels

@@ -39,10 +39,10 @@ typedef struct nb_sgd_tensor {
     const float* grad; /* [numel] gradient (dw, dgamma, dbeta of the block calls); read only */
     float* param;      /* [numel] fp32 master parameter, updated in place */
     float* momentum;   /* [numel] momentum buffer, updated in place */
-    void* param_bf16;  /* NULL, or [numel] bf16 working copy (what the convolution calls read), rewritten */
+    void* param_bf16;  /* NULL, or [numel] 16-bit working copy (what the convolution calls read), rewritten */
     int64_t numel;     /* > 0 */
     int32_t group;     /* 0 .. NB_SGD_GROUPS-1 */
-    int32_t reserved;  /* 0 */
+    int32_t copy_dtype; /* type of the working copy: 0 or NB_DTYPE_BF16 = bf16, NB_DTYPE_F16 = IEEE fp16 (saturating) */
 } nb_sgd_tensor;
 
 typedef struct nb_sgd_hyper {

@@ -17,7 +17,7 @@ NB_OK = 0
 NB_ERR_INVALID_ARG, NB_ERR_UNSUPPORTED, NB_ERR_WORKSPACE, NB_ERR_ALIGNMENT = 1, 2, 3, 4
 NB_ERR_CUDA, NB_ERR_ARCH, NB_ERR_TIMEOUT, NB_ERR_INTERNAL = 5, 6, 7, 8
 NB_DTYPE_F32, NB_DTYPE_BF16, NB_DTYPE_F16 = 0, 1, 2
-NB_MODE_BF16_TC, NB_MODE_F32_REF = 0, 1
+NB_MODE_BF16_TC, NB_MODE_F32_REF, NB_MODE_F16_TC = 0, 1, 2
 NB_CBS_FLAG_FORCE_SIMT = 1
 NB_CBS_FLAG_SHARED_GPU = 2
 
@@ -41,7 +41,7 @@ class nb_cbs_desc(Structure):
 
 class nb_sgd_tensor(Structure):
     _fields_ = [("grad", c_void_p), ("param", c_void_p), ("momentum", c_void_p), ("param_bf16", c_void_p), ("numel", ctypes.c_int64),
-                ("group", c_int32), ("reserved", c_int32)]
+                ("group", c_int32), ("copy_dtype", c_int32)]
 
 
 class nb_sgd_hyper(Structure):
@@ -316,7 +316,8 @@ class SgdPlan:
         for i, it in enumerate(items):
             grad, param, mom, lp, group = it[:5]
             numel = it[5] if len(it) > 5 else param.numel()
-            arr[i] = nb_sgd_tensor(_ptr(grad), _ptr(param), _ptr(mom), _ptr(lp), int(numel), int(group), 0)
+            copy_dtype = NB_DTYPE_F16 if (lp is not None and hasattr(lp, "dtype") and "float16" in str(lp.dtype) and "bfloat16" not in str(lp.dtype)) else 0
+            arr[i] = nb_sgd_tensor(_ptr(grad), _ptr(param), _ptr(mom), _ptr(lp), int(numel), int(group), copy_dtype)
         self.count = len(items)
         self.handle = c_void_p()
         _check(load().nb_sgd_plan_create(arr, self.count, device, byref(self.handle)))

@@ -20,7 +20,7 @@ class CbsBlock:
         self.dev = torch.device("cuda", device)
         self.plan = nb.Plan.for_shape(s, eps=eps, momentum=momentum, mode=mode, flags=flags, device=device)
         f32 = mode == nb.NB_MODE_F32_REF
-        self.act_dtype = torch.float32 if f32 else torch.bfloat16
+        self.act_dtype = torch.float32 if f32 else (torch.float16 if mode == nb.NB_MODE_F16_TC else torch.bfloat16)
         self.y_dtype = torch.float32 if f32 else torch.float16
         e = lambda *sz, dtype: torch.empty(*sz, dtype=dtype, device=self.dev)
         self.x = e(s.n, s.h, s.w, s.c_in, dtype=self.act_dtype)

@@ -88,6 +88,9 @@ struct nb_cbs_plan_s {
 namespace {
 
 bool is_f32(const nb_cbs_plan_s* p) { return p->desc.mode == NB_MODE_F32_REF; }
+bool is_f16(const nb_cbs_plan_s* p) { return p->desc.mode == NB_MODE_F16_TC; }
+// Run an expression with AT = the plan's 16-bit activation type (bf16, or IEEE fp16 in NB_MODE_F16_TC).
+#define NB_WITH_AT(p, ...) (is_f16(p) ? ([&]() { using AT = __half; return __VA_ARGS__; })() : ([&]() { using AT = __nv_bfloat16; return __VA_ARGS__; })())
 // the evaluation-mode forward is one tensor-core kernel with the per-channel epilogue fused
 bool infer_fused(const nb_cbs_plan_s* p) { return !is_f32(p) && (p->stem || p->tc.infer); }
 
@@ -287,7 +290,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
         return fail(NB_ERR_INVALID_ARG, "extents must be positive (n=%d h=%d w=%d c_in=%d c_out=%d)", d->n, d->h, d->w, d->c_in, d->c_out);
     if (d->ksize != 1 && d->ksize != 3) return fail(NB_ERR_INVALID_ARG, "ksize must be 1 or 3, got %d", d->ksize);
     if (d->stride != 1 && d->stride != 2) return fail(NB_ERR_INVALID_ARG, "stride must be 1 or 2, got %d", d->stride);
-    if (d->mode != NB_MODE_BF16_TC && d->mode != NB_MODE_F32_REF) return fail(NB_ERR_INVALID_ARG, "unknown mode %d", d->mode);
+    if (d->mode != NB_MODE_BF16_TC && d->mode != NB_MODE_F32_REF && d->mode != NB_MODE_F16_TC) return fail(NB_ERR_INVALID_ARG, "unknown mode %d", d->mode);
     if (!(d->eps > 0.f)) return fail(NB_ERR_INVALID_ARG, "eps must be positive");
     if (!(d->momentum >= 0.f && d->momentum <= 1.f)) return fail(NB_ERR_INVALID_ARG, "momentum must be in [0,1]");
     const int vec = d->mode == NB_MODE_F32_REF ? 4 : 8;
@@ -343,6 +346,11 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
             e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<float, float, false>, red_smem, 8);
             e.blocks_apply = wave((const void*)bn_silu_apply_kernel<float, float, false>, 0, 4);
             e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<float, float, false>, 0, 4);
+        } else if (d->mode == NB_MODE_F16_TC) {
+            e.blocks_stats = wave((const void*)bn_stats_partial_kernel<__half>, red_smem, 8);
+            e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<__half, __half, true>, red_smem, 8);
+            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __half, true>, 0, 4);
+            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __half, true>, 0, 4);
         } else {
             e.blocks_stats = wave((const void*)bn_stats_partial_kernel<__half>, red_smem, 8);
             e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<__half, __nv_bfloat16, true>, red_smem, 8);
@@ -371,7 +379,8 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     if (ce == cudaSuccess) ce = cudaMalloc(&p->status, ST_WORDS * sizeof(int));
     if (ce == cudaSuccess) ce = cudaMemset(p->status, 0, ST_WORDS * sizeof(int));
     nb_status tcs = NB_OK;
-    if (ce == cudaSuccess) tcs = tc_plan_init(&p->tc, g, d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT), p->sm_count, prop);
+    if (ce == cudaSuccess)
+        tcs = tc_plan_init(&p->tc, g, d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT), p->sm_count, prop, d->mode == NB_MODE_F16_TC);
     cudaSetDevice(cur);
     if (ce != cudaSuccess || tcs != NB_OK) {
         if (p->status) cudaFree(p->status);
@@ -380,7 +389,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
         return fail(NB_ERR_CUDA, "status block allocation failed: %s", cudaGetErrorString(ce));
     }
 
-    p->stem = d->mode == NB_MODE_BF16_TC && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
+    p->stem = d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
               g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0 && g.m < (1LL << 31) && (long long)g.n * g.h * g.w * 3 < (1LL << 31);
     p->stem_blocks = (int)std::min<long long>((g.m + 255) / 256, (long long)p->sm_count * 8);
     p->nparts = std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts);
@@ -519,8 +528,8 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         {
             SiteTimer tm(p, SITE_FPROP, st);
             const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
-            launch_k(stem_fprop_mma_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
-                         static_cast<__half*>(y_saved), p->g, StemEpi{});
+            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
+                                   static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}));
             NB_LAUNCH_OK("stem_fprop");
         }
         NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
@@ -536,13 +545,13 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         nparts = p->tc.fprop_parts;
         finalized = fuse;
     } else {
-        NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y_saved, st)));
+        NB_TRY(NB_WITH_AT(p, run_simt_fprop<AT, __half>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
     }
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
-    return run_apply<__half, __nv_bfloat16, true>(p, y_saved, a_out, scale, shift, st);
+    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st));
 }
 
 namespace {
@@ -561,8 +570,8 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
     if (!is_f32(p) && p->stem) {  // the first layer's own kernel applies the coefficients and the activation itself
         SiteTimer tm(p, SITE_INFER, st);
         const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
-        launch_k(stem_fprop_mma_kernel<48, __nv_bfloat16, true>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x),
-                 static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act});
+        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(w),
+                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}));
         return launch_ok("stem_fprop (fused epilogue)");
     }
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
@@ -571,7 +580,7 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y, st)));
     } else {
-        NB_TRY((run_simt_fprop<__nv_bfloat16, __half>(p, x, w, y, st)));
+        NB_TRY(NB_WITH_AT(p, run_simt_fprop<AT, __half>(p, x, w, y, st)));
     }
     {
         SiteTimer tm(p, SITE_EVAL_COEF, st);
@@ -579,7 +588,7 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
         NB_LAUNCH_OK("bn_eval_coef");
     }
     if (is_f32(p)) return act ? run_apply<float, float, false, true>(p, y, out, scale, shift, st) : run_apply<float, float, false, false>(p, y, out, scale, shift, st);
-    return act ? run_apply<__half, __nv_bfloat16, true, true>(p, y, out, scale, shift, st) : run_apply<__half, __nv_bfloat16, true, false>(p, y, out, scale, shift, st);
+    return NB_WITH_AT(p, act ? run_apply<__half, AT, true, true>(p, y, out, scale, shift, st) : run_apply<__half, AT, true, false>(p, y, out, scale, shift, st));
 }
 }  // namespace
 
@@ -627,6 +636,9 @@ nb_status nb_bn_fold(nb_cbs_plan p, const void* w, const float* gamma, const flo
     if (is_f32(p))
         launch_k(bn_fold_kernel<float>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const float*>(w), K, p->g.c_out, gamma, beta, running_mean, running_var,
                  p->desc.eps, static_cast<float*>(w_folded), bias_folded);
+    else if (is_f16(p))
+        launch_k(bn_fold_kernel<__half>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __half*>(w), K, p->g.c_out, gamma, beta, running_mean, running_var,
+                 p->desc.eps, static_cast<__half*>(w_folded), bias_folded);
     else
         launch_k(bn_fold_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const __nv_bfloat16*>(w), K, p->g.c_out, gamma, beta, running_mean,
                  running_var, p->desc.eps, static_cast<__nv_bfloat16*>(w_folded), bias_folded);
@@ -671,16 +683,16 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
         return NB_OK;
     }
     const bool tc_dg = dx && !p->stem && p->tc.dgrad;  // the finalize kernel also rearranges the filter for the tensor-core dgrad
-    NB_TRY((run_bwd_elementwise<__half, __nv_bfloat16, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st,
-                                                             tc_dg ? w : nullptr, tc_dg ? ws + p->off_wt : nullptr, tc_dg ? &p->tc.wtp : nullptr)));
+    NB_TRY(NB_WITH_AT(p, run_bwd_elementwise<__half, AT, true>(p, g, y_saved, save_mean, save_invstd, gamma, beta, dgamma, dbeta, dy_out, part, coef, st,
+                                                               tc_dg ? w : nullptr, tc_dg ? ws + p->off_wt : nullptr, tc_dg ? &p->tc.wtp : nullptr)));
     if (!dx) return NB_OK;
     if (p->stem) {
         SiteTimer tm(p, SITE_DGRAD, st);
         {
             const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
             const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-            launch_k(stem_dgrad_tiled_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dy_out), static_cast<const __nv_bfloat16*>(w),
-                     static_cast<__nv_bfloat16*>(dx), p->g);
+            NB_WITH_AT(p, launch_k(stem_dgrad_tiled_kernel<48, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dy_out), static_cast<const AT*>(w),
+                                   static_cast<AT*>(dx), p->g));
         }
         return launch_ok("stem_dgrad");
     }
@@ -692,7 +704,7 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         return NB_OK;
     }
-    return run_simt_dgrad<__nv_bfloat16>(p, dy_out, w, dx, st);
+    return NB_WITH_AT(p, run_simt_dgrad<AT>(p, dy_out, w, dx, st));
 }
 
 nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const void* dout, void* dx, float* dw, float* dbias, void* workspace,
@@ -709,7 +721,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
         if (dbias) {  // column sums of dout: the statistics kernels with only the raw sum requested
             float* part = reinterpret_cast<float*>(ws + p->off_bpart);
             if (is_f32(p)) NB_TRY(run_stats_partial<float>(p, dout, part, st));
-            else NB_TRY(run_stats_partial<__nv_bfloat16>(p, dout, part, st));
+            else NB_TRY(NB_WITH_AT(p, run_stats_partial<AT>(p, dout, part, st)));
             NB_TRY(run_finalize(p, part, p->ew.blocks_stats, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, dbias, nullptr, st));
         }
         if (dx) {
@@ -719,8 +731,8 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
                 SiteTimer tm(p, SITE_DGRAD, st);
                 const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
                 const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-                launch_k(stem_dgrad_tiled_kernel<48>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(w),
-                         static_cast<__nv_bfloat16*>(dx), p->g);
+                NB_WITH_AT(p, launch_k(stem_dgrad_tiled_kernel<48, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dout), static_cast<const AT*>(w),
+                                       static_cast<AT*>(dx), p->g));
                 NB_LAUNCH_OK("stem_dgrad");
             } else if (p->tc.dgrad) {
                 SiteTimer tm(p, SITE_DGRAD, st);
@@ -729,7 +741,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
                 g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
                 if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
             } else {
-                NB_TRY(run_simt_dgrad<__nv_bfloat16>(p, dout, w, dx, st));
+                NB_TRY(NB_WITH_AT(p, run_simt_dgrad<AT>(p, dout, w, dx, st)));
             }
         }
     }
@@ -750,8 +762,8 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
         {
             SiteTimer tm(p, SITE_WGRAD, st);
             const long long per = (p->g.m + p->stem_blocks - 1) / p->stem_blocks;
-            launch_k(stem_wgrad_mma_kernel<48>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),
-                                                                 partial, p->g, per);
+            NB_WITH_AT(p, launch_k(stem_wgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(dy), partial,
+                                   p->g, per));
             NB_LAUNCH_OK("stem_wgrad");
         }
         const size_t elems = (size_t)p->g.c_out * p->g.kdim;
@@ -767,7 +779,7 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         return NB_OK;
     }
-    return run_simt_wgrad<__nv_bfloat16>(p, x, dy, dw, partial, st);
+    return NB_WITH_AT(p, run_simt_wgrad<AT>(p, x, dy, dw, partial, st));
 }
 
 }  // extern "C"
@@ -939,6 +951,8 @@ nb_status nb_sgd_plan_create(const nb_sgd_tensor* t, int32_t count, int device, 
         if (t[i].numel <= 0) return fail(NB_ERR_INVALID_ARG, "tensor %d: numel must be positive", i);
         if (t[i].group < 0 || t[i].group >= NB_SGD_GROUPS) return fail(NB_ERR_INVALID_ARG, "tensor %d: group %d out of range", i, t[i].group);
         if (!t[i].grad || !t[i].param || !t[i].momentum) return fail(NB_ERR_INVALID_ARG, "tensor %d: grad, param and momentum must not be NULL", i);
+        if (t[i].copy_dtype != 0 && t[i].copy_dtype != NB_DTYPE_BF16 && t[i].copy_dtype != NB_DTYPE_F16)
+            return fail(NB_ERR_INVALID_ARG, "tensor %d: copy_dtype %d is neither bf16 nor fp16", i, t[i].copy_dtype);
         const uintptr_t bits = reinterpret_cast<uintptr_t>(t[i].grad) | reinterpret_cast<uintptr_t>(t[i].param) |
                                reinterpret_cast<uintptr_t>(t[i].momentum) | reinterpret_cast<uintptr_t>(t[i].param_bf16);
         if (bits & 15u) return fail(NB_ERR_ALIGNMENT, "tensor %d: a pointer is not 16-byte aligned", i);

@@ -119,7 +119,8 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
         const float* g = t_.grad + ch.start;
         float* p = t_.param + ch.start;
         float* b = t_.momentum + ch.start;
-        __nv_bfloat16* lp = t_.param_bf16 ? static_cast<__nv_bfloat16*>(t_.param_bf16) + ch.start : nullptr;
+        __nv_bfloat16* lp = t_.param_bf16 ? static_cast<__nv_bfloat16*>(t_.param_bf16) + ch.start : nullptr;  // (or __half: same size)
+        const bool lp_f16 = t_.copy_dtype == NB_DTYPE_F16;
         const int n4 = ch.len >> 2;
         // all loads of the chunk first (up to 3 x SGD_VPT vectors in flight per thread), then the arithmetic and the stores
         float4 gv[SGD_VPT], pv[SGD_VPT], bv[SGD_VPT];
@@ -143,10 +144,16 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
             reinterpret_cast<float4*>(p)[i] = pv[k];
             reinterpret_cast<float4*>(b)[i] = bv[k];
             if (lp) {
-                const __nv_bfloat162 lo = __floats2bfloat162_rn(pv[k].x, pv[k].y), hi = __floats2bfloat162_rn(pv[k].z, pv[k].w);
                 uint2 o;
-                o.x = *reinterpret_cast<const uint32_t*>(&lo);
-                o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                if (lp_f16) {
+                    const __half a0 = from_f32<__half>(pv[k].x), a1 = from_f32<__half>(pv[k].y), a2 = from_f32<__half>(pv[k].z), a3 = from_f32<__half>(pv[k].w);
+                    o.x = (uint32_t)__half_as_ushort(a0) | ((uint32_t)__half_as_ushort(a1) << 16);
+                    o.y = (uint32_t)__half_as_ushort(a2) | ((uint32_t)__half_as_ushort(a3) << 16);
+                } else {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(pv[k].x, pv[k].y), hi = __floats2bfloat162_rn(pv[k].z, pv[k].w);
+                    o.x = *reinterpret_cast<const uint32_t*>(&lo);
+                    o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                }
                 reinterpret_cast<uint2*>(lp)[i] = o;
             }
         }
@@ -155,7 +162,10 @@ __global__ void __launch_bounds__(SGD_THREADS) sgd_update_kernel(const uint8_t* 
             sgd_one(g[i], pv, bv, coef, lr, wd, mom, first);
             p[i] = pv;
             b[i] = bv;
-            if (lp) lp[i] = __float2bfloat16_rn(pv);
+            if (lp) {
+                if (lp_f16) reinterpret_cast<__half*>(lp)[i] = from_f32<__half>(pv);
+                else lp[i] = __float2bfloat16_rn(pv);
+            }
         }
     }
 }

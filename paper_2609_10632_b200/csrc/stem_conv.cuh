@@ -15,8 +15,14 @@ constexpr int STEM_CIN = 3, STEM_K = 3, STEM_TAPS = 9, STEM_KDIM = 27;
 // pixels x COUT channels with K padded to 32.  The filter fragments stay in registers for the whole kernel; a thread
 // gathers the 2 x 8 input values of its fragment rows with 2-byte loads (the 3 x 3 x 3 patch of a pixel is three runs of 9
 // contiguous values, L1-resident across neighbouring pixels) and writes its accumulator pairs as fp16.
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+template <typename T> __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1);
+template <> __device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+template <> __device__ __forceinline__ void mma_16816<__half>(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -27,8 +33,9 @@ struct StemEpi {
     int act;
 };
 // EPI = false: y = the convolution output in fp16 (training forward).  EPI = true: OutT = bf16 activations, see StemEpi.
-template <int COUT, typename OutT = __half, bool EPI = false>
-__global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+// InT = the 16-bit type of x and w (bf16, or IEEE fp16).
+template <int COUT, typename OutT = __half, bool EPI = false, typename InT = __nv_bfloat16>
+__global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const InT* __restrict__ x, const InT* __restrict__ w,
                                                              OutT* __restrict__ y, Geom g, StemEpi ep) {
     pdl_launch_dependents();
     pdl_wait();
@@ -109,8 +116,8 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) {
             acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
-            mma_bf16_16816(acc[nb], a[0], bfrag[0][nb][0], bfrag[0][nb][1]);
-            mma_bf16_16816(acc[nb], a[1], bfrag[1][nb][0], bfrag[1][nb][1]);
+            mma_16816<InT>(acc[nb], a[0], bfrag[0][nb][0], bfrag[0][nb][1]);
+            mma_16816<InT>(acc[nb], a[1], bfrag[1][nb][0], bfrag[1][nb][1]);
         }
         // accumulator registers: c0, c1 = (row g, columns 2t, 2t+1), c2, c3 = (row g+8, same columns).  The 16 x COUT tile is one
         // contiguous run of the output, so it is staged in shared memory and written with coalesced 16-byte stores.
@@ -146,13 +153,16 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const __nv_bfloat16
 // against 175 us on the 16 x 640 x 640 stem).
 // With pixel (2i+a, 2j+b): (0,0) <- dy[i][j] w11;  (0,1) <- dy[i][j+1] w10 + dy[i][j] w12;  (1,0) <- dy[i+1][j] w01 + dy[i][j] w21;
 // (1,1) <- dy[i+1][j+1] w00 + dy[i+1][j] w02 + dy[i][j+1] w20 + dy[i][j] w22   (w_rt = filter tap (r,t); H and W even).
-template <int COUT>
-__global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ w,
-                                                               __nv_bfloat16* __restrict__ dx, Geom g) {
+template <typename T> __device__ __forceinline__ uint32_t stem_pack2(float a, float b) {
+    const T lo = from_f32<T>(a), hi = from_f32<T>(b);
+    return (uint32_t)(*reinterpret_cast<const unsigned short*>(&lo)) | ((uint32_t)(*reinterpret_cast<const unsigned short*>(&hi)) << 16);
+}
+template <int COUT, typename T = __nv_bfloat16>
+__global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const T* __restrict__ dy, const T* __restrict__ w, T* __restrict__ dx, Geom g) {
     pdl_launch_dependents();
     pdl_wait();
     __shared__ __align__(16) float ws[COUT][28];  // ws[c'][tap*3 + c]
-    for (int e = threadIdx.x; e < COUT * STEM_KDIM; e += blockDim.x) ws[e / STEM_KDIM][e % STEM_KDIM] = __bfloat162float(w[e]);
+    for (int e = threadIdx.x; e < COUT * STEM_KDIM; e += blockDim.x) ws[e / STEM_KDIM][e % STEM_KDIM] = to_f32(w[e]);
     __syncthreads();
     const int npair = (g.wo + 1) / 2;
     const long long total = (long long)g.n * g.ho * npair;
@@ -163,28 +173,28 @@ __global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const __nv_bfloat
         const int i = (int)(t1 % g.ho), n = (int)(t1 / g.ho);
         const int j = 2 * jp;
         const bool row1 = i + 1 < g.ho, col1 = j + 1 < g.wo, col2 = j + 2 < g.wo;
-        const __nv_bfloat16* r0 = dy + (((size_t)n * g.ho + i) * g.wo + j) * COUT;
-        const __nv_bfloat16* r1 = r0 + (size_t)g.wo * COUT;
+        const T* r0 = dy + (((size_t)n * g.ho + i) * g.wo + j) * COUT;
+        const T* r1 = r0 + (size_t)g.wo * COUT;
         float acc[2][4][3];  // [row a][column 0..3 of the 4 produced][channel]
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = 0.f;
-        Vec16<__nv_bfloat16> zero;
+        Vec16<T> zero;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) zero.v[e] = __float2bfloat16_rn(0.f);
+        for (int e = 0; e < 8; ++e) zero.v[e] = from_f32<T>(0.f);
 #pragma unroll 1
         for (int c0 = 0; c0 < COUT; c0 += 8) {
-            const Vec16<__nv_bfloat16> v00 = ld16(r0 + c0);
-            const Vec16<__nv_bfloat16> v01 = col1 ? ld16(r0 + COUT + c0) : zero;
-            const Vec16<__nv_bfloat16> v02 = col2 ? ld16(r0 + 2 * COUT + c0) : zero;
-            const Vec16<__nv_bfloat16> v10 = row1 ? ld16(r1 + c0) : zero;
-            const Vec16<__nv_bfloat16> v11 = (row1 && col1) ? ld16(r1 + COUT + c0) : zero;
-            const Vec16<__nv_bfloat16> v12 = (row1 && col2) ? ld16(r1 + 2 * COUT + c0) : zero;
+            const Vec16<T> v00 = ld16(r0 + c0);
+            const Vec16<T> v01 = col1 ? ld16(r0 + COUT + c0) : zero;
+            const Vec16<T> v02 = col2 ? ld16(r0 + 2 * COUT + c0) : zero;
+            const Vec16<T> v10 = row1 ? ld16(r1 + c0) : zero;
+            const Vec16<T> v11 = (row1 && col1) ? ld16(r1 + COUT + c0) : zero;
+            const Vec16<T> v12 = (row1 && col2) ? ld16(r1 + 2 * COUT + c0) : zero;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const float d00 = __bfloat162float(v00.v[e]), d01 = __bfloat162float(v01.v[e]), d02 = __bfloat162float(v02.v[e]);
-                const float d10 = __bfloat162float(v10.v[e]), d11 = __bfloat162float(v11.v[e]), d12 = __bfloat162float(v12.v[e]);
+                const float d00 = to_f32(v00.v[e]), d01 = to_f32(v01.v[e]), d02 = to_f32(v02.v[e]);
+                const float d10 = to_f32(v10.v[e]), d11 = to_f32(v11.v[e]), d12 = to_f32(v12.v[e]);
                 float wv[28];
 #pragma unroll
                 for (int q = 0; q < 7; ++q) *reinterpret_cast<float4*>(wv + 4 * q) = *reinterpret_cast<const float4*>(&ws[c0 + e][4 * q]);
@@ -207,15 +217,15 @@ __global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const __nv_bfloat
         // rows 2i and 2i+1, columns 4jp .. 4jp+3 (the last two only when dy column j+1 exists): 12 bf16 = 24 bytes per row, 8-byte aligned
 #pragma unroll
         for (int a = 0; a < 2; ++a) {
-            __nv_bfloat16* o = dx + (((size_t)n * g.h + 2 * i + a) * g.w + 4 * (size_t)jp) * 3;
-            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(o);
-            o2[0] = __floats2bfloat162_rn(acc[a][0][0], acc[a][0][1]);
-            o2[1] = __floats2bfloat162_rn(acc[a][0][2], acc[a][1][0]);
-            o2[2] = __floats2bfloat162_rn(acc[a][1][1], acc[a][1][2]);
+            T* o = dx + (((size_t)n * g.h + 2 * i + a) * g.w + 4 * (size_t)jp) * 3;
+            uint32_t* o2 = reinterpret_cast<uint32_t*>(o);
+            o2[0] = stem_pack2<T>(acc[a][0][0], acc[a][0][1]);
+            o2[1] = stem_pack2<T>(acc[a][0][2], acc[a][1][0]);
+            o2[2] = stem_pack2<T>(acc[a][1][1], acc[a][1][2]);
             if (col1) {
-                o2[3] = __floats2bfloat162_rn(acc[a][2][0], acc[a][2][1]);
-                o2[4] = __floats2bfloat162_rn(acc[a][2][2], acc[a][3][0]);
-                o2[5] = __floats2bfloat162_rn(acc[a][3][1], acc[a][3][2]);
+                o2[3] = stem_pack2<T>(acc[a][2][0], acc[a][2][1]);
+                o2[4] = stem_pack2<T>(acc[a][2][2], acc[a][3][0]);
+                o2[5] = stem_pack2<T>(acc[a][3][1], acc[a][3][2]);
             }
         }
     }
@@ -230,14 +240,14 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
 }
-template <int COUT>
-__global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
+template <int COUT, typename T = __nv_bfloat16>
+__global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const T* __restrict__ x, const T* __restrict__ dy,
                                                              float* __restrict__ partial, Geom g, long long pix_per_block) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 16 == 0, "whole m-blocks");
     constexpr int MB = COUT / 16, NBK = 4;  // accumulator blocks: MB x 16 channels by NBK x 8 filter positions (27 padded to 32)
-    __shared__ __align__(16) __nv_bfloat16 dys[4][16 * COUT];
+    __shared__ __align__(16) T dys[4][16 * COUT];
     __shared__ float red[4][COUT][33];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
@@ -257,17 +267,17 @@ __global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const __nv_bfloat16
         for (int b = 0; b < NBK; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = acc[a][b][3] = 0.f;
     const long long m_begin = (long long)blockIdx.x * pix_per_block;
     const long long m_end = (m_begin + pix_per_block < g.m) ? m_begin + pix_per_block : g.m;
-    __nv_bfloat16* st = dys[warp];
+    T* st = dys[warp];
     for (long long m0 = m_begin + warp * 16; m0 < m_end; m0 += 64) {
         const int np = (int)((m_end - m0 < 16) ? (m_end - m0) : 16);  // pixels of this tile inside the block's range
         // stage dy[m0 .. m0+15][:] (zeros past the range)
         for (int v = lane; v < 16 * COUT / 8; v += 32) {
-            Vec16<__nv_bfloat16> q;
+            Vec16<T> q;
             if (v * 8 < np * COUT) {
                 q = ld16(dy + (size_t)m0 * COUT + v * 8);
             } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) q.v[i] = __float2bfloat16_rn(0.f);
+                for (int i = 0; i < 8; ++i) q.v[i] = from_f32<T>(0.f);
             }
             st16(st + v * 8, q);
         }
@@ -305,7 +315,7 @@ __global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const __nv_bfloat16
             const int mi = lane >> 3, mr = lane & 7;
             ldmatrix_x4_trans(afr, st + (mr + (mi >> 1) * 8) * COUT + mb * 16 + (mi & 1) * 8);
 #pragma unroll
-            for (int nb = 0; nb < NBK; ++nb) mma_bf16_16816(acc[mb][nb], afr, bfr[nb][0], bfr[nb][1]);
+            for (int nb = 0; nb < NBK; ++nb) mma_16816<T>(acc[mb][nb], afr, bfr[nb][0], bfr[nb][1]);
         }
         __syncwarp();  // before the next tile overwrites the staged rows
     }

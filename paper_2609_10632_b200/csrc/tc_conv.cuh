@@ -1076,6 +1076,7 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
 
 struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
+    bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
     int fprop_parts = 0;
     size_t wt_bytes = 0;
     size_t wgrad_partial_bytes = 0;
@@ -1393,7 +1394,20 @@ template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmS
 inline const char* tc_last_error() { return tcdetail::err().c_str(); }
 
 // Decide which convolutions of this shape run on the tensor-core kernels and size their scratch.
-inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&) {
+inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int sm_count);
+inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&, bool f16 = false) {
+    const nb_status st = tc_plan_init_impl(tc, g, enable, sm_count);
+    tc->f16 = f16;
+    if (st == NB_OK && f16) {  // A and B formats of the instruction descriptors: bits 7 and 10 set = bf16, clear = f16
+        const uint32_t fmt = (1u << 7) | (1u << 10);
+        tc->fp.prm.idesc &= ~fmt;
+        tc->inf.prm.idesc &= ~fmt;
+        tc->dg.prm.idesc &= ~fmt;
+        tc->wg.idesc &= ~fmt;
+    }
+    return st;
+}
+inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int sm_count) {
     using namespace tcdetail;
     *tc = TcPlan();
     tc->sm_count = sm_count;
@@ -1655,6 +1669,7 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
     S.prm.variant = 0;
     S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
     tc->launches += 1;
+    if (tc->f16) return S.cfg.cg2 ? launch_igemm_impl<__half, false, true, false, 1>(S, st) : launch_igemm_impl<__half, false, false, false, 1>(S, st);
     return S.cfg.cg2 ? launch_igemm_impl<__nv_bfloat16, false, true, false, 1>(S, st) : launch_igemm_impl<__nv_bfloat16, false, false, false, 1>(S, st);
 }
 
@@ -1690,7 +1705,7 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         S.out_ptr = dx;
     }
     S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
-    nb_status r = launch_igemm<__nv_bfloat16, false>(S, st);
+    nb_status r = tc->f16 ? launch_igemm<__half, false>(S, st) : launch_igemm<__nv_bfloat16, false>(S, st);
     if (r != NB_OK) return r;
     tc->launches += 1;
     return NB_OK;

@@ -110,6 +110,9 @@ def test_sgd_plan_rejects_bad_lists_before_any_cuda_call(lib):
     assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
     assert "group" in nb.nb_last_error()
     arr[0].group = 0
+    arr[0].copy_dtype = 7
+    assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_INVALID_ARG
+    arr[0].copy_dtype = nb.NB_DTYPE_F16
     arr[0].grad = 0x1004
     assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_ALIGNMENT
     assert ctypes.sizeof(nb.nb_sgd_tensor) == 48 and ctypes.sizeof(nb.nb_sgd_hyper) == 40 and ctypes.sizeof(nb.nb_scaler_hyper) == 20

@@ -183,3 +183,19 @@ def test_loss_scaled_steps_skip_on_overflow_and_follow_the_scaler_dynamics():
                 parity.check(f"param[{i}]", st.p[i].double().cpu().numpy(), st.h_params[i], "f32")
                 parity.check(f"momentum[{i}]", st.m[i].double().cpu().numpy(), st.h_bufs[i], "f32")
     assert scale == 1024.0  # 1024 -> 512 (skip) -> 1024 (two good steps) -> 512 (skip) -> 1024 (two good steps)
+
+
+def test_fp16_working_copy():
+    import torch
+
+    st = State([5000, 4097], [0, 0], cfg_id=36)
+    st.lp = [torch.empty(n, dtype=torch.float16, device=st.p[0].device) for n in st.sizes]
+    st.plan = st.nb.SgdPlan(zip(st.g, st.p, st.m, st.lp, st.groups))
+    st.plan.upload(st.ws)
+    _, grads = wl.make_optimizer_inputs(st.sizes, 36, 0, 0.1)
+    for d, h in zip(st.g, grads):
+        d.copy_(torch.from_numpy(h))
+    st.plan.step(st.ws, LR, WD, MOM, MAX_NORM, first_step=True)
+    torch.cuda.synchronize()
+    for p, lp in zip(st.p, st.lp):
+        assert torch.equal(lp, p.to(torch.float16))

@@ -19,7 +19,7 @@ def _run_block(shape, mode, cfg_id, layer_id=0, affine="init", flags=0, need_dx=
     from paper_2609_10632_b200 import binding as nb
     from paper_2609_10632_b200.block import CbsBlock
 
-    bf16 = mode == nb.NB_MODE_BF16_TC
+    bf16 = mode != nb.NB_MODE_F32_REF  # the seeded 16-bit inputs are bf16-representable, hence also exact in fp16
     inp = wl.make_inputs(shape, cfg_id, layer_id, bf16=bf16, affine=affine)
     blk = CbsBlock(shape, mode=mode, eps=EPS, momentum=momentum, flags=flags, need_dx=need_dx, running_stats=running)
     blk.upload(inp)
@@ -79,6 +79,57 @@ def test_block_matches_oracle(shape, mode):
     inp, blk, out = _run_block(shape, mode, cfg_id=11, layer_id=SMALL_SHAPES.index(shape), affine="random")
     ref = _oracle(inp)
     _compare(out, ref, mode)
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES, ids=lambda s: s.name)
+def test_block_matches_oracle_in_fp16_mode(shape):
+    """NB_MODE_F16_TC (the paper's own 16-bit format, Sec. 3.2): the same kernels with fp16 operands and outputs.  fp16 keeps
+    three more significant bits than bf16, so the bf16 bars hold with room; and the results must really be fp16-accurate:
+    a good deal closer to the oracle than the bf16 mode can be."""
+    from paper_2609_10632_b200 import binding as nb
+
+    inp, blk, out = _run_block(shape, nb.NB_MODE_F16_TC, cfg_id=11, layer_id=SMALL_SHAPES.index(shape), affine="random")
+    rep = _compare(out, _oracle(inp), 0)
+    assert rep["a"][0] < 1.2e-3  # bf16 rounding alone is about 1.7e-3 relative L2
+    if shape.c_in % 16 == 0 and shape.c_out % 16 == 0:
+        assert blk.plan.paths["fprop"] == 1 and blk.plan.paths["wgrad"] == 1  # (a 1x1 stride-2 data gradient stays on the CUDA cores)
+
+
+def test_fp16_mode_inference_calls_match_oracle():
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    shape = SMALL_SHAPES[8]
+    inp = wl.make_inputs(shape, 18, 0, bf16=True, affine="random")
+    rm, rv, bias = wl.make_eval_stats(shape, 18, 0)
+    blk = CbsBlock_f16(shape)
+    blk.upload(inp)
+    dev = blk.dev
+    up = lambda a: torch.from_numpy(a).to(dev)
+    out = torch.empty_like(blk.a)
+    ws = torch.empty(max(blk.plan.infer_bytes, blk.plan.bwd_bytes, 256), dtype=torch.uint8, device=dev)
+    assert blk.plan.infer_fused
+    nb.nb_conv_bn_silu_infer(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, up(rm), up(rv), out, ws)
+    torch.cuda.synchronize()
+    parity.check("a_eval", out.double().cpu().numpy(), oracle.cbs_infer(inp.x, inp.w, inp.gamma, inp.beta, rm, rv, shape.stride, EPS), "bf16")
+    nb.nb_conv_bias_act(blk.plan, blk.x, blk.w, up(bias), 0, out, ws)
+    dx, dw, db = torch.empty_like(blk.x), torch.empty_like(blk.dw), torch.empty(shape.c_out, dtype=torch.float32, device=dev)
+    nb.nb_conv_bias_bwd(blk.plan, blk.x, blk.w, blk.g, dx, dw, db, ws)
+    torch.cuda.synchronize()
+    blk.poll()
+    parity.check("out", out.double().cpu().numpy(), oracle.conv_bias_act(inp.x, inp.w, bias, shape.stride), "bf16")
+    rdx, rdw, rdb = oracle.conv_bias_bwd(inp.x, inp.w, inp.g, shape.stride)
+    parity.check("dx", dx.double().cpu().numpy(), rdx, "bf16")
+    parity.check("dw", dw.double().cpu().numpy(), rdw, "bf16")
+    parity.check("dbias", db.double().cpu().numpy(), rdb, "bf16")
+
+
+def CbsBlock_f16(shape):
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    return CbsBlock(shape, mode=nb.NB_MODE_F16_TC, eps=EPS)
 
 
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[0], SMALL_SHAPES[7], SMALL_SHAPES[9]], ids=lambda s: s.name)
