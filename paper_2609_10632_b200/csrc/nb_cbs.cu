@@ -72,6 +72,7 @@ struct nb_cbs_plan_s {
     int wg_splits;   // split-K slices of the CUDA-core wgrad
     long long wg_chunk;
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
+    bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or NB_FUSE_FINALIZE=0 at plan creation)
     bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
     int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
@@ -195,7 +196,7 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
                               float* coef, cudaStream_t st, const void* w = nullptr, void* wt = nullptr, const WtParams* wtp = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
-    const bool fuse = !(p->desc.flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+    const bool fuse = p->fuse_finalize;
     WtParams none;
     if (!wtp) memset(&none, 0, sizeof none);
     {
@@ -321,6 +322,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->g = g;
     p->device = device;
     p->sm_count = prop.multiProcessorCount;
+    p->fuse_finalize = !(d->flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
 
     EwCfg& e = p->ew;
     e.vec = vec;
@@ -537,7 +539,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
         // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
-        const bool fuse = !(p->desc.flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+        const bool fuse = p->fuse_finalize;
         const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
         const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);

@@ -1077,6 +1077,7 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
 struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
     bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
+    bool tma_store = true;  // epilogues store through TMA where the layout allows (NB_TC_TMA_STORE=0 at plan creation: coalesced stores instead)
     int fprop_parts = 0;
     size_t wt_bytes = 0;
     size_t wgrad_partial_bytes = 0;
@@ -1398,6 +1399,7 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
 inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&, bool f16 = false) {
     const nb_status st = tc_plan_init_impl(tc, g, enable, sm_count);
     tc->f16 = f16;
+    tc->tma_store = !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0);
     if (st == NB_OK && f16) {  // A and B formats of the instruction descriptors: bits 7 and 10 set = bf16, clear = f16
         const uint32_t fmt = (1u << 7) | (1u << 10);
         tc->fp.prm.idesc &= ~fmt;
@@ -1618,7 +1620,7 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
-    S.prm.tma_store = (!S.cfg.halo && !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0)) ? 1 : 0;
+    S.prm.tma_store = (!S.cfg.halo && tc->tma_store) ? 1 : 0;
     if (S.prm.tma_store && S.out_ptr != y) {
         if (!encode_out_maps(S.prm, S.cfg, y, g.m)) return NB_ERR_CUDA;
         S.out_ptr = y;
@@ -1699,7 +1701,7 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         }
         S.a_ptr = dy; S.b_ptr = wt;
     }
-    S.prm.tma_store = (g.stride == 1 && !S.cfg.halo && !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0)) ? 1 : 0;
+    S.prm.tma_store = (g.stride == 1 && !S.cfg.halo && tc->tma_store) ? 1 : 0;
     if (S.prm.tma_store && S.out_ptr != dx) {
         if (!encode_out_maps(S.prm, S.cfg, dx, (long long)g.n * g.h * g.w)) return NB_ERR_CUDA;
         S.out_ptr = dx;
