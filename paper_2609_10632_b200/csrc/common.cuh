@@ -21,7 +21,7 @@ struct Geom {
 // each pair is zero whenever no kernel of the plan is running.  (A fused split-K reduce behind such a barrier at the
 // tail of the wgrad kernel was measured 0.13 ms per step slower than the separate reduce kernel, whose many small
 // blocks hide the load latency better than 148 resident CTAs can.)
-enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_BAR_FWD = 8, ST_BAR_BWD = 10, ST_WORDS = 16 };
+enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_BAR_FWD = 8, ST_BAR_BWD = 10, ST_BAR_FWD2 = 12, ST_WORDS = 16 };
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }

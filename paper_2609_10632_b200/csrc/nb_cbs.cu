@@ -522,7 +522,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     float* shift = reinterpret_cast<float*>(ws + p->off_shift);
     float* part = reinterpret_cast<float*>(ws + p->off_fpart);
     int nparts = p->ew.blocks_stats;
-    bool finalized = false;
+    bool finalized = false, applied = false;
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
@@ -541,7 +541,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
         const bool fuse = p->fuse_finalize;
         const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
-        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr);
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, a_out, &applied);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
@@ -552,6 +552,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     }
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
+    if (applied) return NB_OK;  // the forward kernel kept its accumulators in TMEM and wrote the activations itself
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
     return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st));
 }

@@ -47,6 +47,10 @@ struct IgemmParams {
     int tma_store;
     int out_w[3];
     CUtensorMap tmOut[3];
+    // Resident variant (RES): every accumulator of the launch stays in TMEM until the statistics are final; after a second
+    // grid barrier the CTA reads its accumulators again, applies scale, shift and SiLU and stores the activations
+    // through tmOut2 (maps over the activation tensor, same boxes as tmOut): the separate normalise + SiLU pass is gone.
+    CUtensorMap tmOut2[3];
     // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
     // b, b + gridDim.x, ...: sums the per-CTA partials in fp64 and writes mean, invstd, scale, shift and the running
     // statistics, which saves the separate finalize launch between this kernel and the apply pass.
@@ -194,6 +198,16 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
     ptx::tmem_ld_wait();
     release();
     if (EPI) {
+        if (EPI == 2) {  // the value the training path stores as y and normalises: the accumulator rounded to fp16 (saturating)
+#pragma unroll
+            for (int j = 0; j < NP; j += 2) {
+                uint32_t v;
+                asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(v) : "f"(__uint_as_float(r[j + 1])), "f"(__uint_as_float(r[j])));
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v));
+                r[j] = __float_as_uint(f.x);
+                r[j + 1] = __float_as_uint(f.y);
+            }
+        }
         if (act) {
 #pragma unroll
             for (int j = 0; j < NP; j += 2) {
@@ -269,9 +283,12 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 // are computed and discarded.
 // EPI = 1: the epilogue applies a per-channel scale and shift (evaluation-mode BN or a bias) and optionally SiLU to the
 // accumulators, so the kernel writes the block's final activations (no statistics, no second pass); TMA stores only.
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0>
+// RES = 1 (forward with statistics only): no CTA has more tiles than accumulator sets, so after the finalize and a second
+// grid barrier every CTA applies BN + SiLU to its accumulators, which are still in TMEM, and writes the activations.
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0>
 __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
     static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
+    static_assert(!RES || (STATS && !HALO && !EPI), "the resident variant is the forward kernel with statistics");
     static_assert(!EPI || (!STATS && !HALO), "the fused per-channel epilogue is a forward-only variant without statistics");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1027,6 +1044,44 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 }
                 epi2_bar_sync();  // every warp is past its reads of the partial sums
                 if (et == 0) grid_depart(ctr, (int)gridDim.x);
+                if (RES) {
+                    // ---- second barrier: every channel's scale and shift is in global memory; then the second pass
+                    int* ctr2 = p.status + ST_BAR_FWD2;
+                    if (et == 0) *fin_ok = (*fin_ok && grid_arrive_wait(ctr2, (int)gridDim.x)) ? 1 : 0;
+                    epi2_bar_sync();
+                    if (*fin_ok) {
+                        float2* coef = reinterpret_cast<float2*>(wstat);  // the channel sums are flushed: reuse their space
+                        for (int c = et; c < p.ldo; c += 256) coef[c] = make_float2(__ldcg(p.fin_scale + c), __ldcg(p.fin_shift + c));
+                        epi2_bar_sync();
+                        int acc2 = 0;
+                        auto no_release = []() {};
+                        for (int tile = worker; tile < total_tiles; tile += nworkers, ++acc2) {
+                            const int lt = tile % p.tiles_per_class;
+                            const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
+                            for (int h = 0; h < mh; ++h) {
+                                const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
+                                const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc2 * mh + h) * p.acc_stride) + (uint32_t)c_lo;
+                                for (int cb = 0; cb < ncol; cb += cw) {
+                                    const int npass = (ncol - cb < cw) ? ncol - cb : cw;
+                                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut2[0] : npass == p.out_w[1] ? &p.tmOut2[1] : &p.tmOut2[2];
+                                    const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
+                                    const uint32_t ta = taddr + (uint32_t)cb;
+                                    int sat2 = 0;
+                                    if (npass == 64) epi_pass_tma<__nv_bfloat16, false, 64, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
+                                    else if (npass == 48) epi_pass_tma<__nv_bfloat16, false, 48, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
+                                    else if (npass == 32) epi_pass_tma<__nv_bfloat16, false, 32, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
+                                    else epi_pass_tma<__nv_bfloat16, false, 16, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
+                                }
+                            }
+                        }
+                        if (store_pending && lane == 0) ptx::tma_store_wait_read<0>();
+                    } else if (et == 0 && atomicCAS(p.status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
+                        p.status[ST_WHERE] = 22;
+                        p.status[ST_DETAIL] = (int)blockIdx.x;
+                    }
+                    epi2_bar_sync();
+                    if (et == 0) grid_depart(ctr2, (int)gridDim.x);
+                }
             }
         }
 #ifdef NB_TC_DEBUG_TIMING
@@ -1077,6 +1132,8 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
 struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
     bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
+    bool fp_resident = false;  // forward: every CTA keeps all its accumulators in TMEM (tiles per CTA <= accumulator sets): BN + SiLU applied in the same kernel
+    const void* res_out_ptr = nullptr;
     bool tma_store = true;  // epilogues store through TMA where the layout allows (NB_TC_TMA_STORE=0 at plan creation: coalesced stores instead)
     int fprop_parts = 0;
     size_t wt_bytes = 0;
@@ -1365,20 +1422,20 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
     return true;
 }
 
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     // the attribute belongs to the (function, device) pair: one bit per device ordinal that already has it
     static std::atomic<unsigned long long> attr_set{0};
     int dev = 0;
     cudaGetDevice(&dev);
     const unsigned long long bit = 1ull << (dev & 63);
     if (!(attr_set.load(std::memory_order_acquire) & bit)) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
         attr_set.fetch_or(bit, std::memory_order_release);
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
@@ -1400,6 +1457,14 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
     const nb_status st = tc_plan_init_impl(tc, g, enable, sm_count);
     tc->f16 = f16;
     tc->tma_store = !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0);
+    // Measured on the detector's layers: 41 of the 77 qualify, and the step gets 0.2 ms SLOWER (the second pass runs on the
+    // eight epilogue warps of each CTA behind one more grid barrier, where the separate pass is a 4 us kernel of 444
+    // blocks), so the variant is chosen only on request (NB_TC_RESIDENT=1 at plan creation).
+    if (st == NB_OK && tc->fprop && !tc->fp.cfg.halo && tc->tma_store && !f16 && getenv("NB_TC_RESIDENT") && atoi(getenv("NB_TC_RESIDENT")) == 1) {
+        const IgemmCfg& c = tc->fp.cfg;
+        const long long tiles = (long long)c.m_tiles * c.n_tiles, workers = c.cg2 ? c.grid / 2 : c.grid;
+        tc->fp_resident = (tiles + workers - 1) / workers <= c.acc_bufs;
+    }
     if (st == NB_OK && f16) {  // A and B formats of the instruction descriptors: bits 7 and 10 set = bf16, clear = f16
         const uint32_t fmt = (1u << 7) | (1u << 10);
         tc->fp.prm.idesc &= ~fmt;
@@ -1603,10 +1668,13 @@ struct FwdFinalize {  // inputs and outputs of the BatchNorm finalize that the f
     const float *gamma, *beta;
     float *mean, *invstd, *scale, *shift, *rmean, *rvar;
 };
+// a_out / applied: with the fused finalize on a plan whose accumulators all stay resident (tc->fp_resident) the kernel also
+// writes the activations a = SiLU(y*scale + shift) and *applied is set: the caller then skips its normalise + SiLU pass.
 inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st,
-                          const FwdFinalize* fin) {
+                          const FwdFinalize* fin, void* a_out = nullptr, bool* applied = nullptr) {
     using namespace tcdetail;
     TcGemmSlot& S = tc->fp;
+    if (applied) *applied = false;
     if (S.a_ptr != x || S.b_ptr != w) {
         const int up = g.pad - (g.k - 1);
         if (S.cfg.halo) {
@@ -1637,6 +1705,16 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
     if (const char* e = getenv("NB_TC_DBG_PTR")) S.prm.dbg = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
 #endif
     tc->launches += 1;
+    if (fin && a_out && applied && tc->fp_resident && S.prm.tma_store) {
+        if (tc->res_out_ptr != a_out) {  // the same boxes as the y maps, over the activation tensor
+            IgemmParams tmp = S.prm;
+            if (!encode_out_maps(tmp, S.cfg, a_out, g.m)) return NB_ERR_CUDA;
+            for (int i = 0; i < 3; ++i) S.prm.tmOut2[i] = tmp.tmOut[i];
+            tc->res_out_ptr = a_out;
+        }
+        *applied = true;
+        return S.cfg.cg2 ? launch_igemm_impl<__half, true, true, false, 0, 1>(S, st) : launch_igemm_impl<__half, true, false, false, 0, 1>(S, st);
+    }
     return launch_igemm<__half, true>(S, st);
 }
 

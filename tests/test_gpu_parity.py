@@ -204,6 +204,28 @@ def test_weight_gradient_on_a_second_stream_overlaps_the_next_layers():
         _compare(b.download(), _oracle(inp), 0)
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[0], SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[9], SMALL_SHAPES[11], SMALL_SHAPES[12]], ids=lambda s: s.name)
+def test_resident_forward_variant_is_bitwise_the_default_path(shape, monkeypatch):
+    """NB_TC_RESIDENT=1: the forward kernel keeps its accumulators in TMEM across the finalize, applies BN + SiLU itself
+    behind a second grid barrier and the separate pass is skipped.  Off by default (measured slower); it must stay
+    correct: against the oracle, and bit for bit equal to the default two-kernel path (it rounds the accumulators to fp16
+    before normalising them, exactly as the stored convolution output is)."""
+    from paper_2609_10632_b200 import binding as nb
+
+    inp, blk0, out0 = _run_block(shape, 0, cfg_id=19, affine="random")
+    l0 = nb.nb_cbs_launch_count()
+    blk0.forward()
+    default_launches = nb.nb_cbs_launch_count() - l0
+    monkeypatch.setenv("NB_TC_RESIDENT", "1")
+    inp, blk1, out1 = _run_block(shape, 0, cfg_id=19, affine="random")
+    l0 = nb.nb_cbs_launch_count()
+    blk1.forward()
+    assert nb.nb_cbs_launch_count() - l0 == default_launches - 1  # the normalise + SiLU kernel is gone
+    _compare(out1, _oracle(inp), 0)
+    for name in ("a", "y", "mean", "invstd", "dx", "dw"):
+        np.testing.assert_array_equal(out1[name], out0[name])
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[11], S(3, 9, 11, 32, 16, 3, 1), S(2, 24, 24, 96, 192, 3, 1)],
                          ids=lambda s: s.name)
 def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
