@@ -212,6 +212,8 @@ def test_resident_forward_variant_is_bitwise_the_default_path(shape, monkeypatch
     before normalising them, exactly as the stored convolution output is)."""
     from paper_2609_10632_b200 import binding as nb
 
+    for name in ("NB_FUSE_FINALIZE", "NB_TC_TMA_STORE", "NB_TC_HALO"):  # the variant needs the fused finalize and TMA stores
+        monkeypatch.delenv(name, raising=False)
     inp, blk0, out0 = _run_block(shape, 0, cfg_id=19, affine="random")
     l0 = nb.nb_cbs_launch_count()
     blk0.forward()
