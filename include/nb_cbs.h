@@ -116,6 +116,16 @@ nb_status nb_cbs_out_shape(nb_cbs_plan plan, int32_t* ho, int32_t* wo);
  * do not overlap on the device; it must be 256-byte aligned. */
 nb_status nb_cbs_workspace_bytes(nb_cbs_plan plan, size_t* fwd_bytes, size_t* bwd_bytes);
 
+/* Channel-slice operands for chained blocks (split / concat without copies): declare that, in the three TRAINING calls
+ * of this plan, the input x, the output a_out and the upstream gradient g are channel slices of wider NHWC tensors:
+ * the pointer passed to the call addresses the slice's first channel and consecutive pixels are ld_* elements apart
+ * (0 = dense; otherwise at least the channel count and a multiple of 8 elements -- 4 in F32 mode -- so that slices stay
+ * 16-byte aligned).  x is read with this pitch by the forward and the weight-gradient call, a_out is written with ld_a,
+ * g is read with ld_g by the data-gradient call; every other tensor (y, dy, dx, dw, ...) stays dense.
+ * NB_ERR_UNSUPPORTED if ld_x is given and the plan's forward or weight gradient does not run on the tensor-core kernels
+ * (their TMA descriptors carry the pitch).  The evaluation-mode, plain and host-buffer calls refuse a pitched plan. */
+nb_status nb_cbs_plan_set_pitches(nb_cbs_plan plan, int64_t ld_x, int64_t ld_a, int64_t ld_g);
+
 /* Which implementation each convolution of this plan runs on: writes three ints (fprop, dgrad, wgrad),
  * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel, 2 = the tap-reuse variant of the tensor-core kernel
  * (3x3 stride-1 layers only; an experiment that is chosen only when the environment variable NB_TC_HALO is 1

@@ -28,7 +28,7 @@ EXPORTS = (
     "nb_conv_bn_silu_step_host", "nb_cbs_launch_count", "nb_cbs_profile_enable", "nb_cbs_profile_site_name",
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step", "nb_sgd_clip_nesterov_step_scaled",
-    "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd",
+    "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd", "nb_cbs_plan_set_pitches",
 )
 
 
@@ -80,6 +80,7 @@ def load() -> ctypes.CDLL:
         lib.nb_cbs_out_shape.argtypes = [V, POINTER(c_int32), POINTER(c_int32)]
         lib.nb_cbs_workspace_bytes.argtypes = [V, POINTER(c_size_t), POINTER(c_size_t)]
         lib.nb_cbs_plan_paths.argtypes = [V, POINTER(c_int32)]
+        lib.nb_cbs_plan_set_pitches.argtypes = [V, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64]
         lib.nb_cbs_poll_status.argtypes = [V, V]
         lib.nb_conv_bn_silu_fwd.argtypes = [V, V, V, FP, FP, FP, FP, V, FP, FP, V, V, c_size_t, V]
         lib.nb_bn_stats.argtypes = [V, V, c_int32, FP, FP, FP, FP, V, c_size_t, V]
@@ -178,6 +179,10 @@ class Plan:
         ib, fused = c_size_t(), c_int32()
         _check(load().nb_cbs_infer_workspace_bytes(self.handle, byref(ib), byref(fused)))
         self.infer_bytes, self.infer_fused = ib.value, bool(fused.value)
+
+    def set_pitches(self, ld_x=0, ld_a=0, ld_g=0):
+        """x, a_out, g of the training calls are channel slices with these row pitches in elements (0 = dense)."""
+        _check(load().nb_cbs_plan_set_pitches(self.handle, int(ld_x), int(ld_a), int(ld_g)))
 
     @classmethod
     def for_shape(cls, s, **kw):

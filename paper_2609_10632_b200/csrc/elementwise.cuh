@@ -159,10 +159,10 @@ template <int V> __device__ __forceinline__ void load_params(const float* __rest
 }
 
 // ------------------------------------------------------------------ a = SiLU(y*scale + shift)  (ACT = false: no SiLU)
-template <typename YT, typename AT, bool FAST, bool ACT = true>
+template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
                                                              long long total_vecs, int C, const float* __restrict__ scale,
-                                                             const float* __restrict__ shift) {
+                                                             const float* __restrict__ shift, long long ld_a) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -172,7 +172,13 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
     load_params<V>(scale, cg, sc);
     load_params<V>(shift, cg, sh);
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+    // a may be a channel slice of a wider tensor: row pitch ld_a elements (the stride is a whole number of rows, so the
+    // output offset advances by a constant)
+    const int cgs = C / V;
+    const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    long long oa = PITCHED ? (v0 / cgs) * ld_a + (long long)cg * V : v0 * V;  // (dense: the flat offset, no division)
+    const long long oa_step = PITCHED ? (stride / cgs) * ld_a : stride * V;
+    for (long long v = v0; v < total_vecs; v += stride, oa += oa_step) {
         if (v + 2 * stride < total_vecs) asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));  // see the reduce kernel
         const Vec16<YT> q = ld16(y + v * V);
         Vec16<AT> o;
@@ -181,7 +187,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
             const float z = fmaf(to_f32(q.v[i]), sc[i], sh[i]);
             o.v[i] = from_f32<AT>(ACT ? z * sigmoid_f<FAST>(z) : z);
         }
-        st16(a + v * V, o);
+        st16(a + oa, o);
     }
 }
 
@@ -271,7 +277,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
                                                                   long long total_vecs, int C, const float* __restrict__ mean,
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
                                                                   const float* __restrict__ beta, float* __restrict__ partials, BwdFused fb,
-                                                                  WtParams wtp) {
+                                                                  WtParams wtp, long long ld_g) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -306,15 +312,19 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
         }
     }
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long v = (long long)blockIdx.x * blockDim.x + tid; v < total_vecs; v += stride) {
+    // g may be a channel slice of a wider tensor (row pitch ld_g elements); the stride is a whole number of rows
+    const long long v0 = (long long)blockIdx.x * blockDim.x + tid;
+    long long og = (v0 / cgs) * ld_g + (long long)cg * V;
+    const long long og_step = (stride / cgs) * ld_g;
+    for (long long v = v0; v < total_vecs; v += stride, og += og_step) {
         // ask L2 for the lines this thread reads two iterations from now: more DRAM requests in flight without holding
         // registers (measured on 157 MB tensors: 93 -> 79 us; no effect on tensors that already sit in L2)
         if (v + 2 * stride < total_vecs) {
             asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + (v + 2 * stride) * V));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + og + 2 * og_step));
         }
         const Vec16<YT> qy = ld16(y + v * V);
-        const Vec16<AT> qg = ld16(g + v * V);
+        const Vec16<AT> qg = ld16(g + og);
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const float yv = to_f32(qy.v[i]);
@@ -392,7 +402,7 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __res
 template <typename YT, typename AT, bool FAST>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
-                                                              const float* __restrict__ coef) {
+                                                              const float* __restrict__ coef, long long ld_g) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -403,13 +413,17 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
     load_params<V>(coef + 2 * C, cg, p1);
     load_params<V>(coef + 3 * C, cg, p0);
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total_vecs; v += stride) {
+    const int cgs = C / V;
+    const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    long long og = (v0 / cgs) * ld_g + (long long)cg * V;  // g may be a channel slice (row pitch ld_g), see the reduce kernel
+    const long long og_step = (stride / cgs) * ld_g;
+    for (long long v = v0; v < total_vecs; v += stride, og += og_step) {
         if (v + 2 * stride < total_vecs) {  // L2 prefetch two iterations ahead (see the reduce kernel)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + (v + 2 * stride) * V));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g + og + 2 * og_step));
         }
         const Vec16<YT> qy = ld16(y + v * V);
-        const Vec16<AT> qg = ld16(g + v * V);
+        const Vec16<AT> qg = ld16(g + og);
         Vec16<AT> o;
 #pragma unroll
         for (int i = 0; i < V; ++i) {

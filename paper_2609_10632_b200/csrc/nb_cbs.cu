@@ -72,6 +72,8 @@ struct nb_cbs_plan_s {
     int wg_splits;   // split-K slices of the CUDA-core wgrad
     long long wg_chunk;
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
+    long long ld_a = 0, ld_g = 0;  // row pitch (elements) of a_out in the forward call and of g in the backward call (set by nb_cbs_plan_set_pitches; default c_out)
+    bool pitched = false;
     bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or NB_FUSE_FINALIZE=0 at plan creation)
     bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
     int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
@@ -182,11 +184,15 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
 }
 
 template <typename YT, typename AT, bool FAST, bool ACT = true>
-nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st) {
+nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st, long long ld_a = 0) {
     const EwCfg& e = p->ew;
     SiteTimer tm(p, SITE_APPLY, st);
-    launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs,
-                                                                       p->g.c_out, scale, shift);
+    if (ld_a)
+        launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, true>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
+                 e.total_vecs, p->g.c_out, scale, shift, ld_a);
+    else
+        launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, false>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
+                 e.total_vecs, p->g.c_out, scale, shift, (long long)p->g.c_out);
     return launch_ok("bn_silu_apply");
 }
 
@@ -210,7 +216,8 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
             fb.w = static_cast<const __nv_bfloat16*>(w); fb.wt = wtp ? static_cast<__nv_bfloat16*>(wt) : nullptr;
         }
         launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
-            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none);
+            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none,
+            p->ld_g ? p->ld_g : (long long)C);
         NB_LAUNCH_OK("bn_silu_bwd_reduce");
     }
     if (!fuse) {
@@ -227,7 +234,7 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
     launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
-                                                                        static_cast<AT*>(dy), e.total_vecs, C, coef);
+                                                                        static_cast<AT*>(dy), e.total_vecs, C, coef, p->ld_g ? p->ld_g : (long long)C);
     return launch_ok("bn_silu_bwd_dy");
 }
 
@@ -450,6 +457,26 @@ nb_status nb_cbs_workspace_bytes(nb_cbs_plan p, size_t* fwd, size_t* bwd) {
     return NB_OK;
 }
 
+nb_status nb_cbs_plan_set_pitches(nb_cbs_plan p, int64_t ld_x, int64_t ld_a, int64_t ld_g) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    const int vec = is_f32(p) ? 4 : 8;
+    auto bad = [&](int64_t ld, int channels) { return ld != 0 && (ld < channels || ld % vec != 0); };
+    if (bad(ld_x, p->g.c_in) || bad(ld_a, p->g.c_out) || bad(ld_g, p->g.c_out))
+        return fail(NB_ERR_INVALID_ARG, "a pitch must be 0 (dense) or at least the channel count and a multiple of %d elements", vec);
+    if (ld_x != 0 && ld_x != p->g.c_in && (is_f32(p) || p->stem || !p->tc.fprop || !p->tc.wgrad || p->tc.fp.cfg.halo))
+        return fail(NB_ERR_UNSUPPORTED, "an input pitch needs the tensor-core forward and weight-gradient kernels (this plan runs them elsewhere)");
+    p->tc.ld_x = (ld_x == p->g.c_in) ? 0 : ld_x;
+    p->ld_a = (ld_a == p->g.c_out) ? 0 : ld_a;
+    p->ld_g = (ld_g == p->g.c_out) ? 0 : ld_g;
+    p->pitched = p->tc.ld_x || p->ld_a || p->ld_g;
+    // tensor maps cached for the previous layout are stale
+    p->tc.fp.a_ptr = nullptr;
+    p->tc.inf.a_ptr = nullptr;
+    p->tc.wg_a_ptr = nullptr;
+    return NB_OK;
+}
+
 nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
     g_err.clear();
     if (!p || !paths3) return fail(NB_ERR_INVALID_ARG, "NULL argument");
@@ -541,7 +568,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
         const bool fuse = p->fuse_finalize;
         const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
-        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, a_out, &applied);
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, p->ld_a ? nullptr : a_out, &applied);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
@@ -553,8 +580,8 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
     if (applied) return NB_OK;  // the forward kernel kept its accumulators in TMEM and wrote the activations itself
-    if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st);
-    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st));
+    if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st, p->ld_a);
+    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a));
 }
 
 namespace {
@@ -609,6 +636,7 @@ nb_status nb_conv_bn_silu_infer(nb_cbs_plan p, const void* x, const void* w, con
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta); NB_CHECK_PTR(running_mean); NB_CHECK_PTR(running_var);
     NB_CHECK_PTR(a_out);
+    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
     DeviceGuard on_device(p->device);
     return run_infer(p, x, w, gamma, beta, running_mean, running_var, 1, a_out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
@@ -620,6 +648,7 @@ nb_status nb_conv_bias_act(nb_cbs_plan p, const void* x, const void* w, const fl
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(bias, true); NB_CHECK_PTR(out);
     if (act != 0 && act != 1) return fail(NB_ERR_INVALID_ARG, "act must be 0 (none) or 1 (SiLU), got %d", act);
+    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
     DeviceGuard on_device(p->device);
     return run_infer(p, x, w, nullptr, bias, nullptr, nullptr, act, out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
@@ -716,6 +745,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(dout); NB_CHECK_PTR(dw); NB_CHECK_PTR(dx, true); NB_CHECK_PTR(dbias, true);
     if (dx) NB_CHECK_PTR(w);
+    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
     {
         DeviceGuard on_device(p->device);
@@ -904,6 +934,7 @@ nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const voi
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     if (!host_x || !host_w || !host_gamma || !host_beta || !host_g || !host_a || !host_dw || !host_dgamma || !host_dbeta)
         return fail(NB_ERR_INVALID_ARG, "a required host pointer is NULL");
+    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: the host-buffer step works on dense tensors");
     const StepLayout L = step_layout(p);
     NB_TRY(check_ws(device_scratch, scratch_bytes, L.total));
     DeviceGuard on_device(p->device);

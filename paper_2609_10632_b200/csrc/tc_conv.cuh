@@ -1132,6 +1132,7 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
 struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
     bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
+    long long ld_x = 0;        // row pitch (elements) of the input activation when it is a channel slice of a wider tensor (0 = dense)
     bool fp_resident = false;  // forward: every CTA keeps all its accumulators in TMEM (tiles per CTA <= accumulator sets): BN + SiLU applied in the same kernel
     const void* res_out_ptr = nullptr;
     bool tma_store = true;  // epilogues store through TMA where the layout allows (NB_TC_TMA_STORE=0 at plan creation: coalesced stores instead)
@@ -1372,11 +1373,13 @@ inline void fill_halo_taps(IgemmParams& P) {
 }
 
 // im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
-inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W, int C, int lo, int up, int ts, int KC, int pixels = TC_BM) {
+// ld = pixel pitch in elements (0: dense, = C); channels past C read as zeros whatever lies behind them in memory.
+inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W, int C, int lo, int up, int ts, int KC, int pixels = TC_BM, long long ld = 0) {
     DriverFns& d = driver();
     if (!d.im2col) { err() = "cuTensorMapEncodeIm2col is not available from the driver"; return false; }
+    const cuuint64_t pitch = (cuuint64_t)(ld ? ld : C);
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
-    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint64_t strides[3] = {pitch * 2, (cuuint64_t)W * pitch * 2, (cuuint64_t)H * W * pitch * 2};
     int lower[2] = {lo, lo}, upper[2] = {up, up};
     cuuint32_t estr[4] = {1, (cuuint32_t)ts, (cuuint32_t)ts, 1};
     CUresult r = d.im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower, upper, (cuuint32_t)KC, (cuuint32_t)pixels, estr,
@@ -1386,11 +1389,11 @@ inline bool encode_im2col(CUtensorMap* m, const void* base, int N, int H, int W,
 }
 
 // tiled map over a bf16 matrix [rows][cols] (cols contiguous), box = KC columns x box_rows rows.
-inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, long long cols, int KC, int box_rows) {
+inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, long long cols, int KC, int box_rows, long long ld = 0) {
     DriverFns& d = driver();
     if (!d.tiled) { err() = "cuTensorMapEncodeTiled is not available from the driver"; return false; }
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint64_t strides[1] = {(cuuint64_t)(ld ? ld : cols) * 2};
     cuuint32_t box[2] = {(cuuint32_t)KC, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = d.tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -1681,8 +1684,8 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
             // traversal over the padded raster: window start from -1 to W (one past each edge), tap offsets always zero
             if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -1, 1, 1, 64, S.cfg.box_pix)) return NB_ERR_CUDA;
         } else if (S.prm.a_tiled) {
-            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
-        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh)) {
+            if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh, tc->ld_x)) return NB_ERR_CUDA;
+        } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh, tc->ld_x)) {
             return NB_ERR_CUDA;
         }
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
@@ -1796,7 +1799,7 @@ inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* 
     WgradParams& P = tc->wg;
     if (tc->wg_a_ptr != x || tc->wg_b_ptr != dy) {
         const int up = g.pad - (g.k - 1);
-        if (!encode_im2col(&P.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, 64, P.KP)) return NB_ERR_CUDA;
+        if (!encode_im2col(&P.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, 64, P.KP, tc->ld_x)) return NB_ERR_CUDA;
         if (!encode_tiled_2d(&P.tmB, dy, g.m, g.c_out, 64, P.KP)) return NB_ERR_CUDA;
         tc->wg_a_ptr = x; tc->wg_b_ptr = dy;
     }

@@ -204,6 +204,58 @@ def test_weight_gradient_on_a_second_stream_overlaps_the_next_layers():
         _compare(b.download(), _oracle(inp), 0)
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[9], SMALL_SHAPES[12], SMALL_SHAPES[3]], ids=lambda s: s.name)
+def test_channel_slice_operands_give_bitwise_the_dense_results(shape):
+    """nb_cbs_plan_set_pitches: x, a_out and g as channel slices of wider tensors (what a chained network's split and
+    concat buffers are).  Results must equal the dense run bit for bit (the kernels do the same arithmetic on the same
+    values, only addresses change), match the oracle, and nothing outside the output slice may be written."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    inp, dense, want = _run_block(shape, 0, cfg_id=20, affine="random")
+    tc_x = dense.plan.paths["fprop"] == 1 and dense.plan.paths["wgrad"] == 1
+    blk = CbsBlock(shape, eps=EPS)
+    blk.upload(inp)
+    dev, s = blk.dev, shape
+    ldx, lda, ldg = (s.c_in + 24 if tc_x else s.c_in), s.c_out + 40, s.c_out + 8
+    offx, offa, offg = (16 if tc_x else 0), 24, 8
+    if not tc_x:
+        with pytest.raises(nb.NbError) as e:
+            blk.plan.set_pitches(ld_x=s.c_in + 8)
+        assert e.value.status == nb.NB_ERR_UNSUPPORTED
+    blk.plan.set_pitches(ld_x=ldx, ld_a=lda, ld_g=ldg)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    X = torch.randn(s.n, s.h, s.w, ldx, generator=gen, device=dev).to(torch.bfloat16)
+    A = torch.randn(s.n, s.ho, s.wo, lda, generator=gen, device=dev).to(torch.bfloat16)
+    G = torch.randn(s.n, s.ho, s.wo, ldg, generator=gen, device=dev).to(torch.bfloat16)
+    X[..., offx:offx + s.c_in] = blk.x
+    G[..., offg:offg + s.c_out] = blk.g
+    A0 = A.clone()
+    at = lambda t, c: t.data_ptr() + c * t.element_size()
+    nb.nb_conv_bn_silu_fwd(blk.plan, at(X, offx), blk.w, blk.gamma, blk.beta, None, None, blk.y, blk.mean, blk.invstd, at(A, offa), blk.ws)
+    nb.nb_conv_bn_silu_bwd_data(blk.plan, at(G, offg), blk.y, blk.mean, blk.invstd, blk.gamma, blk.beta, blk.w, blk.dx, blk.dgamma, blk.dbeta, blk.dy, blk.ws)
+    nb.nb_conv_bn_silu_bwd_weight(blk.plan, at(X, offx), blk.dy, blk.dw, blk.ws)
+    torch.cuda.synchronize()
+    blk.poll()
+    blk.a.copy_(A[..., offa:offa + s.c_out])
+    got = blk.download()
+    for name in ("a", "y", "dy", "dx", "dw", "dgamma", "dbeta", "mean", "invstd"):
+        np.testing.assert_array_equal(got[name], want[name], err_msg=name)
+    _compare(got, _oracle(inp), 0)
+    assert torch.equal(A[..., :offa], A0[..., :offa]) and torch.equal(A[..., offa + s.c_out:], A0[..., offa + s.c_out:])
+    # the other calls refuse a pitched plan; clearing the pitches brings them back
+    ws = torch.empty(max(blk.plan.infer_bytes, 256), dtype=torch.uint8, device=dev)
+    with pytest.raises(nb.NbError) as e:
+        nb.nb_conv_bias_act(blk.plan, blk.x, blk.w, None, 0, blk.a, ws)
+    assert e.value.status == nb.NB_ERR_UNSUPPORTED
+    blk.plan.set_pitches()
+    nb.nb_conv_bias_act(blk.plan, blk.x, blk.w, None, 0, blk.a, ws)
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[0], SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[9], SMALL_SHAPES[11], SMALL_SHAPES[12]], ids=lambda s: s.name)
 def test_resident_forward_variant_is_bitwise_the_default_path(shape, monkeypatch):
     """NB_TC_RESIDENT=1: the forward kernel keeps its accumulators in TMEM across the finalize, applies BN + SiLU itself
