@@ -551,8 +551,7 @@ def run_detector_chain(args, dev, local, peaks, step_flops_value):
 
     ops, layers, outs, plain = wl.detector_graph(16, 640, plain_head=True)  # up to the six raw head outputs
     run = GraphRunner(ops, layers, outs, device=local, plain_layers=plain)
-    for i, b in enumerate(run.blocks):
-        b.fill_random(seed=7000 + i)  # (fills the block's own scratch x / g as well; the chained buffers are set below)
+    run.fill_parameters(seed=7000)
     for pl in run.plain:
         pl["w"].normal_(0.0, 0.05)
         pl["bias"].normal_(0.0, 0.5)

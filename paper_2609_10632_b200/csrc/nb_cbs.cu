@@ -461,7 +461,7 @@ nb_status nb_cbs_plan_set_pitches(nb_cbs_plan p, int64_t ld_x, int64_t ld_a, int
     g_err.clear();
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     const int vec = is_f32(p) ? 4 : 8;
-    auto bad = [&](int64_t ld, int channels) { return ld != 0 && (ld < channels || ld % vec != 0); };
+    auto bad = [&](int64_t ld, int channels) { return ld != 0 && ld != channels && (ld < channels || ld % vec != 0); };  // 0 or the channel count: dense
     if (bad(ld_x, p->g.c_in) || bad(ld_a, p->g.c_out) || bad(ld_g, p->g.c_out))
         return fail(NB_ERR_INVALID_ARG, "a pitch must be 0 (dense) or at least the channel count and a multiple of %d elements", vec);
     if (ld_x != 0 && ld_x != p->g.c_in && (is_f32(p) || p->stem || !p->tc.fprop || !p->tc.wgrad || p->tc.fp.cfg.halo))

@@ -239,7 +239,7 @@ def test_detector_dataflow_matches_graph_oracle():
     from paper_2609_10632_b200.detector import GraphRunner
 
     ops, layers, outs, plain = wl.detector_graph(2, 256, plain_head=True)  # up to the six raw head outputs
-    run = GraphRunner(ops, layers, outs, eps=EPS, plain_layers=plain)
+    run = GraphRunner(ops, layers, outs, eps=EPS, plain_layers=plain)  # channel-slice views: split / concat without copies
     pparams = []
     for j, pl in enumerate(run.plain):
         w = wl.make_inputs(plain[j], 54, j, bf16=True).w
@@ -302,8 +302,7 @@ def test_chained_detector_in_the_benchmarks_launch_configuration_is_bitwise_the_
     run = GraphRunner(ops, layers, outs, eps=EPS)
     gen = torch.Generator(device=run.dev)
     gen.manual_seed(7)
-    for i, b in enumerate(run.blocks):
-        b.fill_random(seed=100 + i)
+    run.fill_parameters(seed=100)
     img = torch.rand(run.shape["img"], generator=gen, device=run.dev).to(torch.bfloat16)
     gout = {n: torch.randn(run.shape[n], generator=gen, device=run.dev).to(torch.bfloat16) for n in outs}
 
@@ -347,3 +346,45 @@ def test_chained_detector_in_the_benchmarks_launch_configuration_is_bitwise_the_
     for b, (dw, dgamma, dbeta) in zip(run.blocks, want):
         assert torch.equal(b.dw, dw) and torch.equal(b.dgamma, dgamma) and torch.equal(b.dbeta, dbeta), b.shape.name
     assert torch.equal(run.grad["img"], want_dimg)
+
+
+def test_views_and_copies_give_the_same_bits():
+    """GraphRunner(views=True) places tensors inside concatenation buffers and hands channel slices to the calls;
+    views=False copies.  Same arithmetic on the same values: every forward tensor and every gradient must agree bit for
+    bit, and the views must save most of the glue launches."""
+    import torch
+
+    from paper_2609_10632_b200.detector import GraphRunner
+
+    ops, layers, outs, plain = wl.detector_graph(2, 128, plain_head=True)
+    runs = [GraphRunner(ops, layers, outs, eps=EPS, plain_layers=plain, views=v) for v in (True, False)]
+    gen = torch.Generator(device=runs[0].dev)
+    gen.manual_seed(11)
+    img = torch.rand(runs[0].shape["img"], generator=gen, device=runs[0].dev).to(torch.bfloat16)
+    gout = {n: torch.randn(runs[0].shape[n], generator=gen, device=runs[0].dev).to(torch.bfloat16) for n in outs}
+    for r in runs:
+        r.fill_parameters(seed=200)
+        for j, pl in enumerate(r.plain):
+            g2 = torch.Generator(device=r.dev)
+            g2.manual_seed(300 + j)
+            pl["w"].copy_(torch.randn(pl["w"].shape, generator=g2, device=r.dev) * 0.05)
+            pl["bias"].copy_(torch.randn(pl["bias"].shape, generator=g2, device=r.dev) * 0.5)
+        r.buf["img"].copy_(img)
+        for n in outs:
+            r.grad[n].copy_(gout[n])
+        r.forward()
+        r.backward()
+    torch.cuda.synchronize()
+    a, b = runs
+    a.poll()
+    b.poll()
+    for name in a.buf:
+        assert torch.equal(a.buf[name], b.buf[name]), name
+    assert torch.equal(a.grad["img"], b.grad["img"])
+    for x, y in zip(a.blocks, b.blocks):
+        assert torch.equal(x.dw, y.dw) and torch.equal(x.dgamma, y.dgamma) and torch.equal(x.dbeta, y.dbeta), x.shape.name
+    for x, y in zip(a.plain, b.plain):
+        assert torch.equal(x["dw"], y["dw"]) and torch.equal(x["dbias"], y["dbias"])
+    va, vb = sum(a.glue_launches()), sum(b.glue_launches())
+    print("glue launches with views", a.glue_launches(), "with copies", b.glue_launches(), "placed", len(a.placed), "slice views", len(a.slice_view))
+    assert va < 0.6 * vb
