@@ -272,7 +272,7 @@ struct BwdFused {
     const __nv_bfloat16* w;  // filter and its rearranged copy for the data-gradient GEMM (wt = NULL: nothing to rearrange)
     __nv_bfloat16* wt;
 };
-template <typename YT, typename AT, bool FAST>
+template <typename YT, typename AT, bool FAST, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                                   long long total_vecs, int C, const float* __restrict__ mean,
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
@@ -314,8 +314,8 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
     const long long stride = (long long)gridDim.x * blockDim.x;
     // g may be a channel slice of a wider tensor (row pitch ld_g elements); the stride is a whole number of rows
     const long long v0 = (long long)blockIdx.x * blockDim.x + tid;
-    long long og = (v0 / cgs) * ld_g + (long long)cg * V;
-    const long long og_step = (stride / cgs) * ld_g;
+    long long og = PITCHED ? (v0 / cgs) * ld_g + (long long)cg * V : v0 * V;  // (dense: the flat offset)
+    const long long og_step = PITCHED ? (stride / cgs) * ld_g : stride * V;
     for (long long v = v0; v < total_vecs; v += stride, og += og_step) {
         // ask L2 for the lines this thread reads two iterations from now: more DRAM requests in flight without holding
         // registers (measured on 157 MB tensors: 93 -> 79 us; no effect on tensors that already sit in L2)
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __res
 }
 
 // ------------------------------------------------------------------ dy = a*dz - p1*y + p0
-template <typename YT, typename AT, bool FAST>
+template <typename YT, typename AT, bool FAST, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
                                                               const float* __restrict__ coef, long long ld_g) {
@@ -415,8 +415,8 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
     const long long stride = (long long)gridDim.x * blockDim.x;
     const int cgs = C / V;
     const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    long long og = (v0 / cgs) * ld_g + (long long)cg * V;  // g may be a channel slice (row pitch ld_g), see the reduce kernel
-    const long long og_step = (stride / cgs) * ld_g;
+    long long og = PITCHED ? (v0 / cgs) * ld_g + (long long)cg * V : v0 * V;  // g may be a channel slice (row pitch ld_g), see the reduce kernel
+    const long long og_step = PITCHED ? (stride / cgs) * ld_g : stride * V;
     for (long long v = v0; v < total_vecs; v += stride, og += og_step) {
         if (v + 2 * stride < total_vecs) {  // L2 prefetch two iterations ahead (see the reduce kernel)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));

@@ -215,9 +215,12 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
             fb.dgamma = dgamma; fb.dbeta = dbeta; fb.coef = coef;
             fb.w = static_cast<const __nv_bfloat16*>(w); fb.wt = wtp ? static_cast<__nv_bfloat16*>(wt) : nullptr;
         }
-        launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
-            static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none,
-            p->ld_g ? p->ld_g : (long long)C);
+        if (p->ld_g)
+            launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST, true>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
+                static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none, p->ld_g);
+        else
+            launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST, false>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
+                static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none, (long long)C);
         NB_LAUNCH_OK("bn_silu_bwd_reduce");
     }
     if (!fuse) {
@@ -233,8 +236,12 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
-    launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
-                                                                        static_cast<AT*>(dy), e.total_vecs, C, coef, p->ld_g ? p->ld_g : (long long)C);
+    if (p->ld_g)
+        launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST, true>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
+                 static_cast<AT*>(dy), e.total_vecs, C, coef, p->ld_g);
+    else
+        launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST, false>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
+                 static_cast<AT*>(dy), e.total_vecs, C, coef, (long long)C);
     return launch_ok("bn_silu_bwd_dy");
 }
 

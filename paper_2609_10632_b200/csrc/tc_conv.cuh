@@ -49,8 +49,8 @@ struct IgemmParams {
     CUtensorMap tmOut[3];
     // Resident variant (RES): every accumulator of the launch stays in TMEM until the statistics are final; after a second
     // grid barrier the CTA reads its accumulators again, applies scale, shift and SiLU and stores the activations
-    // through tmOut2 (maps over the activation tensor, same boxes as tmOut): the separate normalise + SiLU pass is gone.
-    CUtensorMap tmOut2[3];
+    // through maps over the activation tensor with the same boxes as tmOut.  Those maps sit in tmB[1..3], which a forward
+    // launch (one class) does not use: the parameter block of every launch stays as small as it was.
     // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
     // b, b + gridDim.x, ...: sums the per-CTA partials in fp64 and writes mean, invstd, scale, shift and the running
     // statistics, which saves the separate finalize launch between this kernel and the apply pass.
@@ -1063,7 +1063,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                                 const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc2 * mh + h) * p.acc_stride) + (uint32_t)c_lo;
                                 for (int cb = 0; cb < ncol; cb += cw) {
                                     const int npass = (ncol - cb < cw) ? ncol - cb : cw;
-                                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut2[0] : npass == p.out_w[1] ? &p.tmOut2[1] : &p.tmOut2[2];
+                                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmB[1] : npass == p.out_w[1] ? &p.tmB[2] : &p.tmB[3];
                                     const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
                                     const uint32_t ta = taddr + (uint32_t)cb;
                                     int sat2 = 0;
@@ -1712,7 +1712,7 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (tc->res_out_ptr != a_out) {  // the same boxes as the y maps, over the activation tensor
             IgemmParams tmp = S.prm;
             if (!encode_out_maps(tmp, S.cfg, a_out, g.m)) return NB_ERR_CUDA;
-            for (int i = 0; i < 3; ++i) S.prm.tmOut2[i] = tmp.tmOut[i];
+            for (int i = 0; i < 3; ++i) S.prm.tmB[1 + i] = tmp.tmOut[i];
             tc->res_out_ptr = a_out;
         }
         *applied = true;
