@@ -32,7 +32,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or needs_build():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp, os.path.join(CSRC, "nb_cbs.cu")]
+        units = sorted(glob.glob(os.path.join(CSRC, "*.cu")))  # nb_cbs.cu (blocks), nb_glue.cu, nb_sgd.cu
+        cmd = [nvcc] + NVCC_FLAGS + ["--threads", str(len(units))] + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + units
         subprocess.check_call(cmd)
         os.replace(tmp, LIB)
     return LIB

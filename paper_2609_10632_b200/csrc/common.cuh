@@ -209,7 +209,7 @@ __device__ __forceinline__ void wt_transform_blocks(const __nv_bfloat16* __restr
         __syncthreads();
     }
 }
-__global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
+static __global__ void dgrad_weight_transform_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, WtParams P) {
     pdl_launch_dependents();
     pdl_wait();
     wt_transform_blocks(w, wt, P, (int)blockIdx.x, (int)gridDim.x);

@@ -1,5 +1,6 @@
 // C ABI of the Conv -> BN(train) -> SiLU block library (see include/nb_cbs.h): plans, validation, workspace
 // carving and kernel dispatch.  No device memory is allocated here except the plan's status block.
+// (The optimiser step of include/nb_sgd.h lives in nb_sgd.cu, the glue calls of include/nb_glue.h in nb_glue.cu.)
 #include "../../include/nb_cbs.h"
 
 #include <algorithm>
@@ -17,12 +18,12 @@
 #include "simt_conv.cuh"
 #include "stem_conv.cuh"
 #include "tc_conv.cuh"
-#include "sgd.cuh"
-#include "glue.cuh"
+#include "api_common.cuh"
 
 using namespace nbcbs;
+using namespace nbapi;
 
-namespace {
+namespace nbapi {  // shared with the other translation units of the library (api_common.cuh)
 
 thread_local std::string g_err;
 
@@ -36,15 +37,11 @@ nb_status fail(nb_status code, const char* fmt, ...) {
     return code;
 }
 
-#define NB_CUDA_CHECK(expr)                                                                         \
-    do {                                                                                            \
-        cudaError_t e__ = (expr);                                                                   \
-        if (e__ != cudaSuccess) return fail(NB_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
-    } while (0)
-
-inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
 std::atomic<unsigned long long> g_launches{0};  // kernels launched by this library in this process
+
+}  // namespace nbapi
+
+namespace {
 
 enum Site { SITE_FPROP = 0, SITE_STATS, SITE_FINALIZE, SITE_APPLY, SITE_BWD_REDUCE, SITE_BWD_FINALIZE, SITE_BWD_DY,
             SITE_WTRANSFORM, SITE_DGRAD, SITE_WGRAD, SITE_SPLITK_REDUCE, SITE_INFER, SITE_EVAL_COEF, SITE_FOLD, SITE_COUNT };
@@ -108,13 +105,6 @@ nb_status check_ptr(const void* p, const char* name, bool nullable = false) {
         if (s__ != NB_OK) return s__;                          \
     } while (0)
 
-nb_status check_ws(const void* ws, size_t have, size_t need) {
-    if (need == 0) return NB_OK;
-    if (!ws) return fail(NB_ERR_WORKSPACE, "workspace is NULL (%zu bytes needed)", need);
-    if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(NB_ERR_WORKSPACE, "workspace is not 256-byte aligned");
-    if (have < need) return fail(NB_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", have, need);
-    return NB_OK;
-}
 
 // Brackets one kernel site with events when the plan is in profiling mode (diagnostic; synchronises the stream).
 struct SiteTimer {
@@ -135,34 +125,6 @@ struct SiteTimer {
     }
 };
 
-// Makes the plan's device current for the duration of a compute call and restores the caller's device afterwards.
-struct DeviceGuard {
-    int prev = -1;
-    bool switched = false;
-    explicit DeviceGuard(int device) {
-        if (cudaGetDevice(&prev) == cudaSuccess && prev != device) switched = cudaSetDevice(device) == cudaSuccess;
-    }
-    ~DeviceGuard() {
-        if (switched) cudaSetDevice(prev);
-    }
-};
-
-nb_status launch_ok(const char* what) {
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(NB_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
-    return NB_OK;
-}
-#define NB_LAUNCH_OK(what)                    \
-    do {                                      \
-        nb_status s__ = launch_ok(what);      \
-        if (s__ != NB_OK) return s__;         \
-    } while (0)
-#define NB_TRY(expr)                          \
-    do {                                      \
-        nb_status s__ = (expr);               \
-        if (s__ != NB_OK) return s__;         \
-    } while (0)
 
 // ---------------------------------------------------------------- elementwise launch helpers
 template <typename YT> nb_status run_stats_partial(nb_cbs_plan_s* p, const void* y, float* partials, cudaStream_t st) {
@@ -972,275 +934,3 @@ nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const voi
 
 }  // extern "C"
 
-// ---------------------------------------------------------------- fused optimiser step (include/nb_sgd.h)
-struct nb_sgd_plan_s {
-    int device = 0;
-    SgdHeader h;
-    std::vector<uint8_t> image;  // header + tensor list + chunk table, as they sit at the start of the workspace
-};
-
-extern "C" {
-
-nb_status nb_sgd_plan_create(const nb_sgd_tensor* t, int32_t count, int device, nb_sgd_plan* out) {
-    g_err.clear();
-    if (!out) return fail(NB_ERR_INVALID_ARG, "out_plan is NULL");
-    *out = nullptr;
-    if (!t) return fail(NB_ERR_INVALID_ARG, "host_tensors is NULL");
-    if (count <= 0) return fail(NB_ERR_INVALID_ARG, "count must be positive, got %d", count);
-    long long nchunks = 0;
-    for (int i = 0; i < count; ++i) {
-        if (t[i].numel <= 0) return fail(NB_ERR_INVALID_ARG, "tensor %d: numel must be positive", i);
-        if (t[i].group < 0 || t[i].group >= NB_SGD_GROUPS) return fail(NB_ERR_INVALID_ARG, "tensor %d: group %d out of range", i, t[i].group);
-        if (!t[i].grad || !t[i].param || !t[i].momentum) return fail(NB_ERR_INVALID_ARG, "tensor %d: grad, param and momentum must not be NULL", i);
-        if (t[i].copy_dtype != 0 && t[i].copy_dtype != NB_DTYPE_BF16 && t[i].copy_dtype != NB_DTYPE_F16)
-            return fail(NB_ERR_INVALID_ARG, "tensor %d: copy_dtype %d is neither bf16 nor fp16", i, t[i].copy_dtype);
-        const uintptr_t bits = reinterpret_cast<uintptr_t>(t[i].grad) | reinterpret_cast<uintptr_t>(t[i].param) |
-                               reinterpret_cast<uintptr_t>(t[i].momentum) | reinterpret_cast<uintptr_t>(t[i].param_bf16);
-        if (bits & 15u) return fail(NB_ERR_ALIGNMENT, "tensor %d: a pointer is not 16-byte aligned", i);
-        nchunks += (t[i].numel + SGD_CHUNK - 1) / SGD_CHUNK;
-    }
-    if (nchunks > 0x7fffffffLL) return fail(NB_ERR_UNSUPPORTED, "too many elements for one tensor list");
-    int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(NB_ERR_CUDA, "cannot query device %d", device);
-    }
-    nb_sgd_plan_s* p = new (std::nothrow) nb_sgd_plan_s;
-    if (!p) return fail(NB_ERR_INTERNAL, "out of host memory");
-    p->device = device;
-    SgdHeader& h = p->h;
-    memset(&h, 0, sizeof h);
-    h.magic = SGD_MAGIC;
-    h.count = count;
-    h.nchunks = (int32_t)nchunks;
-    h.grid = (int32_t)std::min<long long>(nchunks, std::min<long long>(SGD_MAX_BLOCKS, (long long)std::max(sms, 1) * 8));
-    size_t off = 256;
-    h.off_tensors = off; off = align_up(off + (size_t)count * sizeof(nb_sgd_tensor), 256);
-    h.off_chunks = off; off = align_up(off + (size_t)nchunks * sizeof(SgdChunk), 256);
-    h.off_partials = off; off = align_up(off + (size_t)SGD_MAX_BLOCKS * sizeof(double), 256);
-    h.total_bytes = off;
-    p->image.assign((size_t)h.off_partials, 0);
-    memcpy(p->image.data(), &h, sizeof h);
-    memcpy(p->image.data() + h.off_tensors, t, (size_t)count * sizeof(nb_sgd_tensor));
-    SgdChunk* c = reinterpret_cast<SgdChunk*>(p->image.data() + h.off_chunks);  // chunk i goes to block i % grid
-    for (int i = 0; i < count; ++i)
-        for (int64_t s = 0; s < t[i].numel; s += SGD_CHUNK, ++c) {
-            c->tensor = i;
-            c->start = s;
-            c->len = (int32_t)std::min<int64_t>(SGD_CHUNK, t[i].numel - s);
-        }
-    *out = p;
-    return NB_OK;
-}
-
-nb_status nb_sgd_plan_destroy(nb_sgd_plan p) {
-    g_err.clear();
-    delete p;
-    return NB_OK;
-}
-
-nb_status nb_sgd_workspace_bytes(nb_sgd_plan p, size_t* bytes) {
-    g_err.clear();
-    if (!p || !bytes) return fail(NB_ERR_INVALID_ARG, "NULL argument");
-    *bytes = (size_t)p->h.total_bytes;
-    return NB_OK;
-}
-
-nb_status nb_sgd_upload(nb_sgd_plan p, void* workspace, size_t workspace_bytes, void* stream) {
-    g_err.clear();
-    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
-    NB_TRY(check_ws(workspace, workspace_bytes, (size_t)p->h.total_bytes));
-    DeviceGuard on_device(p->device);
-    // the source is the plan's own host image, which lives as long as the plan
-    NB_CUDA_CHECK(cudaMemcpyAsync(workspace, p->image.data(), p->image.size(), cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
-    return NB_OK;
-}
-
-namespace {
-nb_status sgd_step_impl(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc, nb_loss_scaler* state,
-                        float* total_norm, void* stream);
-}
-nb_status nb_sgd_clip_nesterov_step(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, float* total_norm,
-                                    void* stream) {
-    g_err.clear();
-    return sgd_step_impl(p, workspace, workspace_bytes, hyper, nullptr, nullptr, total_norm, stream);
-}
-
-nb_status nb_sgd_clip_nesterov_step_scaled(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc,
-                                           nb_loss_scaler* state, float* total_norm, void* stream) {
-    g_err.clear();
-    if (!sc || !state) return fail(NB_ERR_INVALID_ARG, "scaler and state must not be NULL");
-    if (sc->struct_size != sizeof(nb_scaler_hyper)) return fail(NB_ERR_INVALID_ARG, "nb_scaler_hyper.struct_size is %u, expected %zu", sc->struct_size, sizeof(nb_scaler_hyper));
-    if (reinterpret_cast<uintptr_t>(state) & 15u) return fail(NB_ERR_ALIGNMENT, "state is not 16-byte aligned");
-    if (!(sc->growth_factor > 0.f) || !(sc->backoff_factor > 0.f) || sc->growth_interval < 1) return fail(NB_ERR_INVALID_ARG, "scaler factors must be positive, growth_interval >= 1");
-    return sgd_step_impl(p, workspace, workspace_bytes, hyper, sc, state, total_norm, stream);
-}
-
-}  // extern "C"
-
-namespace {
-nb_status sgd_step_impl(nb_sgd_plan p, void* workspace, size_t workspace_bytes, const nb_sgd_hyper* hyper, const nb_scaler_hyper* sc, nb_loss_scaler* state,
-                        float* total_norm, void* stream) {
-    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
-    if (!hyper) return fail(NB_ERR_INVALID_ARG, "hyper is NULL");
-    if (hyper->struct_size != sizeof(nb_sgd_hyper))
-        return fail(NB_ERR_INVALID_ARG, "nb_sgd_hyper.struct_size is %u, expected %zu", hyper->struct_size, sizeof(nb_sgd_hyper));
-    NB_TRY(check_ws(workspace, workspace_bytes, (size_t)p->h.total_bytes));
-    if (reinterpret_cast<uintptr_t>(total_norm) & 3u) return fail(NB_ERR_ALIGNMENT, "total_norm is not 4-byte aligned");
-    DeviceGuard on_device(p->device);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    SgdScalars s;
-    s.momentum = hyper->momentum; s.max_norm = hyper->max_norm; s.first_step = hyper->first_step;
-    s.scaler = state;
-    for (int i = 0; i < NB_SGD_GROUPS; ++i) { s.lr[i] = hyper->lr[i]; s.wd[i] = hyper->weight_decay[i]; }
-    const uint8_t* ws = static_cast<const uint8_t*>(workspace);
-    launch_k(sgd_sqnorm_kernel, dim3((unsigned)p->h.grid), dim3(SGD_THREADS), 0, st, 1, ws);
-    NB_LAUNCH_OK("sgd_sqnorm");
-    launch_k(sgd_update_kernel, dim3((unsigned)p->h.grid), dim3(SGD_THREADS), 0, st, 1, ws, s, total_norm);
-    NB_LAUNCH_OK("sgd_update");
-    if (state) {
-        launch_k(sgd_scaler_kernel, dim3(1), dim3(32), 0, st, 1, ws, state, sc->growth_factor, sc->backoff_factor, sc->floor_scale, (int)sc->growth_interval);
-        NB_LAUNCH_OK("sgd_scaler");
-    }
-    return NB_OK;
-}
-}  // namespace
-
-// ---------------------------------------------------------------- glue between chained blocks (include/nb_glue.h)
-namespace {
-template <typename T>
-nb_status run_slice_add(void* out, long long ld_out, const void* a, long long ld_a, const void* b, long long ld_b, long long rows, int channels,
-                        int accumulate, cudaStream_t st) {
-    constexpr int V = 16 / (int)sizeof(T);
-    const bool vec = channels % V == 0 && ld_out % V == 0 && ld_a % V == 0 && (!b || ld_b % V == 0) &&
-                     !((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) & 15u);
-    const long long total = rows * (vec ? channels / V : channels);
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 16));
-    const bool small = total + 256LL * blocks < (1LL << 32);  // indices (one grid stride past the end included) fit 32 bits
-#define NB_SLICE_LAUNCH(VECF, IDX)                                                                                                         \
-    launch_k(slice_add_kernel<T, VECF, IDX>, dim3(blocks), dim3(256), 0, st, 1, static_cast<T*>(out), ld_out, static_cast<const T*>(a), ld_a, \
-             static_cast<const T*>(b), ld_b, rows, channels, accumulate)
-    if (vec && small) NB_SLICE_LAUNCH(true, unsigned);
-    else if (vec) NB_SLICE_LAUNCH(true, long long);
-    else if (small) NB_SLICE_LAUNCH(false, unsigned);
-    else NB_SLICE_LAUNCH(false, long long);
-#undef NB_SLICE_LAUNCH
-    return launch_ok("slice_add");
-}
-}  // namespace
-
-extern "C" nb_status nb_slice_add(int32_t dtype, int64_t rows, int32_t channels, void* out, int64_t ld_out, const void* a, int64_t ld_a,
-                                  const void* b, int64_t ld_b, int32_t accumulate, void* stream) {
-    g_err.clear();
-    if (!out || !a) return fail(NB_ERR_INVALID_ARG, "out and a must not be NULL");
-    if (rows <= 0 || channels <= 0) return fail(NB_ERR_INVALID_ARG, "rows and channels must be positive");
-    if (ld_out < channels || ld_a < channels || (b && ld_b < channels)) return fail(NB_ERR_INVALID_ARG, "a row pitch is smaller than the channel count");
-    const size_t es = dtype == NB_DTYPE_F32 ? 4 : 2;
-    if ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) & (es - 1))
-        return fail(NB_ERR_ALIGNMENT, "a pointer is not aligned to its element size");
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    switch (dtype) {
-        case NB_DTYPE_F32: return run_slice_add<float>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
-        case NB_DTYPE_BF16: return run_slice_add<__nv_bfloat16>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
-        case NB_DTYPE_F16: return run_slice_add<__half>(out, ld_out, a, ld_a, b, ld_b, rows, channels, accumulate != 0, st);
-        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-    }
-}
-
-namespace {
-unsigned glue_blocks(long long total) {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    return (unsigned)std::max<long long>(1, std::min<long long>((total + 255) / 256, (long long)sms * 8));
-}
-nb_status check_nhwc(int32_t n, int32_t h, int32_t w, int32_t c) {
-    if (n <= 0 || h <= 0 || w <= 0 || c <= 0) return fail(NB_ERR_INVALID_ARG, "extents must be positive");
-    return NB_OK;
-}
-template <typename T>
-nb_status run_maxpool_fwd(const void* x, void* y, uint8_t* idx, int n, int h, int w, int c, cudaStream_t st) {
-    const bool vec = sizeof(T) == 2 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u);
-    if (vec) {
-        const long long total = (long long)n * h * w * (c / 8);
-        launch_k(maxpool5_fwd_kernel<T, 8>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
-    } else {
-        const long long total = (long long)n * h * w * c;
-        launch_k(maxpool5_fwd_kernel<T, 1>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
-    }
-    return launch_ok("maxpool5_fwd");
-}
-}  // namespace
-
-extern "C" {
-
-nb_status nb_maxpool5_fwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* x, void* y, uint8_t* idx, void* stream) {
-    g_err.clear();
-    if (!x || !y) return fail(NB_ERR_INVALID_ARG, "x and y must not be NULL");
-    NB_TRY(check_nhwc(n, h, w, c));
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    switch (dtype) {
-        case NB_DTYPE_F32: return run_maxpool_fwd<float>(x, y, idx, n, h, w, c, st);
-        case NB_DTYPE_BF16: return run_maxpool_fwd<__nv_bfloat16>(x, y, idx, n, h, w, c, st);
-        case NB_DTYPE_F16: return run_maxpool_fwd<__half>(x, y, idx, n, h, w, c, st);
-        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-    }
-}
-
-nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* g, const uint8_t* idx, void* dx, int32_t accumulate,
-                          void* stream) {
-    g_err.clear();
-    if (!g || !idx || !dx) return fail(NB_ERR_INVALID_ARG, "g, idx and dx must not be NULL");
-    NB_TRY(check_nhwc(n, h, w, c));
-    if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 &&
-                     !((reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(dx)) & 15u) && !(reinterpret_cast<uintptr_t>(idx) & 7u);
-    const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
-#define NB_POOLB(T)                                                                                                                               \
-    do {                                                                                                                                          \
-        if (vec) launch_k(maxpool5_bwd_kernel<T, 8>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0); \
-        else launch_k(maxpool5_bwd_kernel<T, 1>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0);     \
-    } while (0)
-    switch (dtype) {
-        case NB_DTYPE_F32: NB_POOLB(float); break;
-        case NB_DTYPE_BF16: NB_POOLB(__nv_bfloat16); break;
-        case NB_DTYPE_F16: NB_POOLB(__half); break;
-        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-    }
-#undef NB_POOLB
-    return launch_ok("maxpool5_bwd");
-}
-
-nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* src, void* dst, int32_t backward, int32_t accumulate,
-                       void* stream) {
-    g_err.clear();
-    if (!src || !dst) return fail(NB_ERR_INVALID_ARG, "src and dst must not be NULL");
-    NB_TRY(check_nhwc(n, h, w, c));
-    if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u);
-    const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
-#define NB_UPS1(T, BW, VV) launch_k(upsample2_kernel<T, BW, VV>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0)
-#define NB_UPS(T)                                   \
-    do {                                            \
-        if (backward && vec) NB_UPS1(T, true, 8);   \
-        else if (backward) NB_UPS1(T, true, 1);     \
-        else if (vec) NB_UPS1(T, false, 8);         \
-        else NB_UPS1(T, false, 1);                  \
-    } while (0)
-    switch (dtype) {
-        case NB_DTYPE_F32: NB_UPS(float); break;
-        case NB_DTYPE_BF16: NB_UPS(__nv_bfloat16); break;
-        case NB_DTYPE_F16: NB_UPS(__half); break;
-        default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-    }
-#undef NB_UPS
-#undef NB_UPS1
-    return launch_ok("upsample2");
-}
-
-}  // extern "C"
