@@ -36,8 +36,55 @@ template <> __device__ __forceinline__ __half from_f32<__half>(float v) {
     return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
 }
 
+// Two fp32 values per instruction (fma / mul / add .f32x2 of sm_100): each half is the IEEE round-to-nearest result of the
+// scalar operation, so a loop written with these gives the same bits as its scalar form with half the arithmetic issue slots.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tadd.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+
+// Elements 2j and 2j+1 of a vector as fp32, and back (round to nearest; fp16 saturates like from_f32<__half>).
+template <typename T> __device__ __forceinline__ float2 pair_to_f32(const T* v);
+template <> __device__ __forceinline__ float2 pair_to_f32<float>(const float* v) { return make_float2(v[0], v[1]); }
+template <> __device__ __forceinline__ float2 pair_to_f32<__nv_bfloat16>(const __nv_bfloat16* v) {
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(v));
+}
+template <> __device__ __forceinline__ float2 pair_to_f32<__half>(const __half* v) { return __half22float2(*reinterpret_cast<const __half2*>(v)); }
+template <typename T> __device__ __forceinline__ void pair_from_f32(T* v, float2 f);
+template <> __device__ __forceinline__ void pair_from_f32<float>(float* v, float2 f) {
+    v[0] = f.x;
+    v[1] = f.y;
+}
+template <> __device__ __forceinline__ void pair_from_f32<__nv_bfloat16>(__nv_bfloat16* v, float2 f) {
+    *reinterpret_cast<__nv_bfloat162*>(v) = __float22bfloat162_rn(f);
+}
+template <> __device__ __forceinline__ void pair_from_f32<__half>(__half* v, float2 f) {
+    f.x = fminf(fmaxf(f.x, -65504.f), 65504.f);
+    f.y = fminf(fmaxf(f.y, -65504.f), 65504.f);
+    *reinterpret_cast<__half2*>(v) = __float22half2_rn(f);
+}
+
 // 16-byte vector of VT elements (8 x 16-bit or 4 x fp32).
-template <typename T> struct Vec16 {
+template <typename T> struct __align__(16) Vec16 {
     static constexpr int N = 16 / sizeof(T);
     T v[N];
 };

@@ -21,6 +21,25 @@ template <bool FAST> __device__ __forceinline__ float sigmoid_f(float z) {
     }
 }
 
+// The same for two values at once, and dz = g * s * (1 + z*(1 - s)) with s = sigmoid(z) (the derivative of SiLU times g);
+// the operations and their order are those of the scalar expressions the passes used to spell out, so the bits agree.
+template <bool FAST> __device__ __forceinline__ float2 sigmoid2(float2 z) {
+    if (FAST) {
+        const float2 hz = mul2(splat2(0.5f), z);
+        float2 t;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(t.x) : "f"(hz.x));
+        asm("tanh.approx.f32 %0, %1;" : "=f"(t.y) : "f"(hz.y));
+        return fma2(splat2(0.5f), t, splat2(0.5f));
+    } else {
+        return make_float2(sigmoid_f<false>(z.x), sigmoid_f<false>(z.y));
+    }
+}
+template <bool FAST> __device__ __forceinline__ float2 silu_bwd_dz2(float2 z, float2 g) {
+    const float2 s = sigmoid2<FAST>(z);
+    const float2 oms = fma2(s, splat2(-1.f), splat2(1.f));  // 1 - s, exactly
+    return mul2(mul2(g, s), fma2(z, oms, splat2(1.f)));
+}
+
 // ------------------------------------------------------------------ per-channel sum and sum of squares
 // partials layout: [gridDim.x][2][C]; blockDim.x = (C/V) * R.
 template <typename YT>
@@ -158,6 +177,16 @@ template <int V> __device__ __forceinline__ void load_params(const float* __rest
     }
 }
 
+template <int V> __device__ __forceinline__ void load_params(const float* __restrict__ p, int cg, float2 (&out)[V / 2]) {  // as pairs
+    const float4* q = reinterpret_cast<const float4*>(p + (size_t)cg * V);
+#pragma unroll
+    for (int i = 0; i < V / 4; ++i) {
+        const float4 t = q[i];
+        out[2 * i] = make_float2(t.x, t.y);
+        out[2 * i + 1] = make_float2(t.z, t.w);
+    }
+}
+
 // ------------------------------------------------------------------ a = SiLU(y*scale + shift)  (ACT = false: no SiLU)
 template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
@@ -168,7 +197,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "y and a must have the same element size");
     const int cg = threadIdx.x % (C / V);
-    float sc[V], sh[V];
+    float2 sc[V / 2], sh[V / 2];
     load_params<V>(scale, cg, sc);
     load_params<V>(shift, cg, sh);
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -183,9 +212,9 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
         const Vec16<YT> q = ld16(y + v * V);
         Vec16<AT> o;
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            const float z = fmaf(to_f32(q.v[i]), sc[i], sh[i]);
-            o.v[i] = from_f32<AT>(ACT ? z * sigmoid_f<FAST>(z) : z);
+        for (int j = 0; j < V / 2; ++j) {
+            const float2 z = fma2(pair_to_f32(q.v + 2 * j), sc[j], sh[j]);
+            pair_from_f32(o.v + 2 * j, ACT ? mul2(z, sigmoid2<FAST>(z)) : z);
         }
         st16(a + oa, o);
     }
@@ -297,7 +326,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
             if (t < wt_tiles) wt_tile_load_async(fb.w, wtp, wt_tile_decode(wtp, t), wtile[k]);
         }
     }
-    float a[V], b[V], sb[V], sy[V];
+    float2 a[V / 2], b[V / 2], sb[V / 2], sy[V / 2];
     {
         float mu[V], is[V], ga[V], be[V];
         load_params<V>(mean, cg, mu);
@@ -305,10 +334,10 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
         load_params<V>(gamma, cg, ga);
         load_params<V>(beta, cg, be);
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            a[i] = ga[i] * is[i];
-            b[i] = fmaf(-mu[i], a[i], be[i]);
-            sb[i] = sy[i] = 0.f;
+        for (int j = 0; j < V / 2; ++j) {
+            a[j] = make_float2(ga[2 * j] * is[2 * j], ga[2 * j + 1] * is[2 * j + 1]);
+            b[j] = make_float2(fmaf(-mu[2 * j], a[j].x, be[2 * j]), fmaf(-mu[2 * j + 1], a[j].y, be[2 * j + 1]));
+            sb[j] = sy[j] = splat2(0.f);
         }
     }
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -326,19 +355,17 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
         const Vec16<YT> qy = ld16(y + v * V);
         const Vec16<AT> qg = ld16(g + og);
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            const float yv = to_f32(qy.v[i]);
-            const float z = fmaf(yv, a[i], b[i]);
-            const float s = sigmoid_f<FAST>(z);
-            const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
-            sb[i] += dz;
-            sy[i] = fmaf(dz, yv, sy[i]);
+        for (int j = 0; j < V / 2; ++j) {
+            const float2 yv = pair_to_f32(qy.v + 2 * j);
+            const float2 dz = silu_bwd_dz2<FAST>(fma2(yv, a[j], b[j]), pair_to_f32(qg.v + 2 * j));
+            sb[j] = add2(sb[j], dz);
+            sy[j] = fma2(dz, yv, sy[j]);
         }
     }
     const int R = blockDim.x / cgs;
     for (int pass = 0; pass < 2; ++pass) {
 #pragma unroll
-        for (int i = 0; i < V; ++i) red[tid * V + i] = pass ? sy[i] : sb[i];
+        for (int j = 0; j < V / 2; ++j) *reinterpret_cast<float2*>(&red[tid * V + 2 * j]) = pass ? sy[j] : sb[j];
         __syncthreads();
         for (int c = tid; c < C; c += blockDim.x) {
             const int gq = c / V, e = c % V;
@@ -407,11 +434,13 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
     const int cg = threadIdx.x % (C / V);
-    float a[V], b[V], p1[V], p0[V];
+    float2 a[V / 2], b[V / 2], np1[V / 2], p0[V / 2];
     load_params<V>(coef, cg, a);
     load_params<V>(coef + C, cg, b);
-    load_params<V>(coef + 2 * C, cg, p1);
+    load_params<V>(coef + 2 * C, cg, np1);
     load_params<V>(coef + 3 * C, cg, p0);
+#pragma unroll
+    for (int j = 0; j < V / 2; ++j) np1[j] = make_float2(-np1[j].x, -np1[j].y);
     const long long stride = (long long)gridDim.x * blockDim.x;
     const int cgs = C / V;
     const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -426,12 +455,10 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
         const Vec16<AT> qg = ld16(g + og);
         Vec16<AT> o;
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            const float yv = to_f32(qy.v[i]);
-            const float z = fmaf(yv, a[i], b[i]);
-            const float s = sigmoid_f<FAST>(z);
-            const float dz = to_f32(qg.v[i]) * s * fmaf(z, 1.f - s, 1.f);
-            o.v[i] = from_f32<AT>(fmaf(a[i], dz, fmaf(-p1[i], yv, p0[i])));
+        for (int j = 0; j < V / 2; ++j) {
+            const float2 yv = pair_to_f32(qy.v + 2 * j);
+            const float2 dz = silu_bwd_dz2<FAST>(fma2(yv, a[j], b[j]), pair_to_f32(qg.v + 2 * j));
+            pair_from_f32(o.v + 2 * j, fma2(a[j], dz, fma2(np1[j], yv, p0[j])));
         }
         st16(dy + v * V, o);
     }

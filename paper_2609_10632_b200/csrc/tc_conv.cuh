@@ -186,7 +186,7 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
 // hands the 32 x NP piece to TMA, and with STATS the warp adds the piece's per-channel sums of the rounded values to its
 // running sums (a lane owns two adjacent channels).  Everything is unrolled on NP: constant offsets, no predicates.
 // With EPI the accumulators first become act(acc*scale + shift) with the pass's per-channel (scale, shift) pairs read
-// from shared memory (`coef`, the same address in every lane: a broadcast).
+// from shared memory (`coef`, the same address in every lane: a broadcast; per channel pair scale, scale, shift, shift).
 template <typename OutT, bool STATS, int NP, int EPI, class Release>
 __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int lane, bool& store_pending, int& sat, const CUtensorMap* tm, int col,
                                              int grow, float* stat_s, float* stat_q, const float2* coef, int act, Release release) {
@@ -212,16 +212,18 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 #pragma unroll
             for (int j = 0; j < NP; j += 2) {
                 const float4 cf = *reinterpret_cast<const float4*>(coef + j);
-                const float z0 = fmaf(__uint_as_float(r[j]), cf.x, cf.y), z1 = fmaf(__uint_as_float(r[j + 1]), cf.z, cf.w);
-                r[j] = __float_as_uint(z0 * sigmoid_f<true>(z0));
-                r[j + 1] = __float_as_uint(z1 * sigmoid_f<true>(z1));
+                const float2 z = fma2(make_float2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), make_float2(cf.x, cf.y), make_float2(cf.z, cf.w));
+                const float2 o = mul2(z, sigmoid2<true>(z));
+                r[j] = __float_as_uint(o.x);
+                r[j + 1] = __float_as_uint(o.y);
             }
         } else {
 #pragma unroll
             for (int j = 0; j < NP; j += 2) {
                 const float4 cf = *reinterpret_cast<const float4*>(coef + j);
-                r[j] = __float_as_uint(fmaf(__uint_as_float(r[j]), cf.x, cf.y));
-                r[j + 1] = __float_as_uint(fmaf(__uint_as_float(r[j + 1]), cf.z, cf.w));
+                const float2 z = fma2(make_float2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), make_float2(cf.x, cf.y), make_float2(cf.z, cf.w));
+                r[j] = __float_as_uint(z.x);
+                r[j + 1] = __float_as_uint(z.y);
             }
         }
     }
@@ -257,10 +259,10 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
             for (int rr = 0; rr < 32; rr += 2) {
                 const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(base + rr * PITCH + (SWZ ? (cj ^ (rr & 7)) : cj) * 16));
                 const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(base + (rr + 1) * PITCH + (SWZ ? (cj ^ ((rr + 1) & 7)) : cj) * 16));
-                sa.x += f0.x; sa.y += f0.y;
-                sb.x += f1.x; sb.y += f1.y;
-                qa.x = fmaf(f0.x, f0.x, qa.x); qa.y = fmaf(f0.y, f0.y, qa.y);
-                qb.x = fmaf(f1.x, f1.x, qb.x); qb.y = fmaf(f1.y, f1.y, qb.y);
+                sa = add2(sa, f0);  // packed fp32 pairs: the same sums in half the issue slots
+                sb = add2(sb, f1);
+                qa = fma2(f0, f0, qa);
+                qb = fma2(f1, f1, qb);
             }
             float2* ps = reinterpret_cast<float2*>(stat_s + 2 * lane);
             float2* pq = reinterpret_cast<float2*>(stat_q + 2 * lane);
@@ -364,11 +366,12 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     pdl_wait();  // everything above touched only shared memory, TMEM and kernel parameters
     if (EPI) {
         // per-channel coefficients of the fused epilogue, in fp64 like the training-mode finalize
-        float2* coef = reinterpret_cast<float2*>(wstat);
+        // (stored per channel pair as scale, scale, shift, shift: the operands of the packed fp32 multiply-add)
         for (int c = threadIdx.x; c < p.ldo; c += IG_THREADS) {
             double sc, sh;
             bn_eval_coef(p.fin_gamma, p.fin_beta, p.fin_rmean, p.fin_rvar, p.fin_eps, c, sc, sh);
-            coef[c] = make_float2((float)sc, (float)sh);
+            wstat[4 * (c >> 1) + (c & 1)] = (float)sc;
+            wstat[4 * (c >> 1) + 2 + (c & 1)] = (float)sh;
         }
         __syncthreads();
     }
@@ -1051,7 +1054,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     epi2_bar_sync();
                     if (*fin_ok) {
                         float2* coef = reinterpret_cast<float2*>(wstat);  // the channel sums are flushed: reuse their space
-                        for (int c = et; c < p.ldo; c += 256) coef[c] = make_float2(__ldcg(p.fin_scale + c), __ldcg(p.fin_shift + c));
+                        for (int c = et; c < p.ldo; c += 256) {  // per channel pair: scale, scale, shift, shift
+                            wstat[4 * (c >> 1) + (c & 1)] = __ldcg(p.fin_scale + c);
+                            wstat[4 * (c >> 1) + 2 + (c & 1)] = __ldcg(p.fin_shift + c);
+                        }
                         epi2_bar_sync();
                         int acc2 = 0;
                         auto no_release = []() {};
