@@ -30,8 +30,8 @@ struct IgemmParams {
     int ts;           // traversal stride (input pixels per grid step)
     int lo_w, lo_h;   // input coordinate of grid position 0 for tap offset 0
     // A launch covers up to four "classes" that share A, the tiling and the output tensor but have their own filter
-    // matrix, tap list and output offset (the four output-parity classes of a stride-2 data gradient); tiles are
-    // numbered class by class, classes with more taps first.
+    // matrix, tap list and output offset (the four output-parity classes of a stride-2 data gradient); for the order of
+    // the tiles see igemm_tile_class.
     int nclasses, tiles_per_class;
     int cls_ntaps[4], cls_oa[4], cls_ob[4];
     int Ca, KC, kc_per_tap;
@@ -82,6 +82,23 @@ struct IgemmParams {
     long long npos;            // N*(H+2)*(W+2)
     uint32_t tap_off16[9];     // start of tap t inside the slab, in 16-byte units
 };
+
+// Tile number -> (class, tile within the class).  Default order: class by class, classes with more taps first.  With
+// variant bit 64 (set for the four parity classes of a stride-2 data gradient) the four classes of one [m][n] tile are
+// neighbours in the order, so the dy rows they share are fetched from DRAM once and found in L2 three times instead of being
+// streamed once per class; the class of position r is rotated by the round of the persistent loop so that a worker
+// (whose tile numbers are nworkers apart) still cycles through heavy and light classes.
+__device__ __forceinline__ void igemm_tile_class(const IgemmParams& p, int tile, int nworkers, int& cls, int& lt) {
+    if (p.variant & 64) {
+        const int r = tile & 3;
+        const int round = (tile - r) / nworkers;
+        cls = (r + ((nworkers & 1) ? 0 : round)) & 3;
+        lt = tile >> 2;
+    } else {
+        cls = tile / p.tiles_per_class;
+        lt = tile - cls * p.tiles_per_class;
+    }
+}
 
 #ifdef NB_TC_DEBUG_TIMING
 #define NB_DBG_T0() const long long dbg_t0__ = clock64()
@@ -493,9 +510,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             // pairs: loads of both CTAs are counted on the rank-0 CTA's full barriers (the MMA issuer waits there)
             const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB);
             const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
-            const int tpc = p.tiles_per_class;
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                const int cls = tile / tpc, lt = tile - cls * tpc;
+                int cls, lt;
+                igemm_tile_class(p, tile, nworkers, cls, lt);
                 const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
                 const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
                 const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
@@ -678,10 +695,12 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, p.sbo, p.umma_swizzle);
             const uint32_t empty_u32 = ptx::smem_u32(empty);
             uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
-            const int tpc = p.tiles_per_class, kc_per_tap = p.kc_per_tap;
+            const int kc_per_tap = p.kc_per_tap;
             const uint32_t tfull_u32 = ptx::smem_u32(tfull);
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                const int kblocks = p.cls_ntaps[tile / tpc] * kc_per_tap;
+                int cls_mma, lt_mma;
+                igemm_tile_class(p, tile, nworkers, cls_mma, lt_mma);
+                const int kblocks = p.cls_ntaps[cls_mma] * kc_per_tap;
                 {
                     NB_DBG_T0();
                     if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
@@ -778,7 +797,8 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
 #endif
         const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
         for (int tile = worker; tile < total_tiles; tile += nworkers) {
-            const int cls = tile / p.tiles_per_class, lt = tile - cls * p.tiles_per_class;
+            int cls, lt;
+            igemm_tile_class(p, tile, nworkers, cls, lt);
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
             NB_DBG_T0();
             bool ok = true;
@@ -1578,6 +1598,7 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
             fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
             if (c.halo) fill_halo_taps(P);
             P.nclasses = ncls; P.tiles_per_class = c.m_tiles * c.n_tiles;
+            if (ncls == 4 && !(getenv("NB_TC_CLS_INTERLEAVE") && atoi(getenv("NB_TC_CLS_INTERLEAVE")) == 0)) P.variant |= 64;  // see igemm_tile_class
             P.ldo = g.c_in;
             W.nclasses = ncls;
             tc->wt_bytes = off * 2;
