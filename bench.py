@@ -710,7 +710,7 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
         hin, hout = host[s.key]
         h2d += sum(t.numel() * t.element_size() for t in hin.values())
         d2h += sum(t.numel() * t.element_size() for t in hout.values())
-    # Three streams, each with its own device scratch, take the layers round-robin: while one layer computes, the next
+    # Several streams (--e2e-streams, default 6), each with its own device scratch, take the layers in turn: while one layer computes, the next
     # layer's inputs arrive over PCIe and the previous layer's results leave (the two copy directions run concurrently).
     # Kernels of different layers may then share the GPU, so the plans of this arm are created with NB_CBS_FLAG_SHARED_GPU
     # (separate finalize kernels instead of in-kernel grid barriers).

@@ -1541,7 +1541,7 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
         }
     }
     // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four output-parity
-    // classes, heaviest (four taps) first so that the static round-robin tile order approximates longest-first
+    // classes, numbered heaviest (four taps) first; the order in which their tiles are visited is igemm_tile_class's
     if (g.c_in % 16 == 0 && g.c_out % 16 == 0 && (g.stride == 1 || (g.k == 3 && even))) {
         WtParams& W = tc->wtp;
         memset(&W, 0, sizeof W);
