@@ -313,7 +313,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = sA + (HALO ? (size_t)p.a_slots * p.slab_bytes : (size_t)p.stages * p.a_stage_bytes);
-    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
+    // Weights-stationary mode (variant bit 128, non-halo): the CTA's share of the whole filter stays in shared memory
+    // (p.a_slots groups of kpb k-blocks, fetched once, in the order of this CTA's K loop); the stage ring then holds A only.
+    const bool bres = !HALO && (p.variant & 128);
+    uint8_t* stg = sB + (size_t)(bres ? p.a_slots : p.stages) * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
     const int cw = p.stage_cw;  // columns per staging pass (<= 64)
     const int pitch = cw * 2 + 16;
     float* wstat = reinterpret_cast<float*>(stg + (size_t)2 * TC_BM * pitch);  // per team [4 warps][2][its columns of every n-tile]: warp-private channel sums
@@ -339,7 +342,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, HALO ? 1 : 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
+            ptx::mbar_init(full + s, (HALO || bres) ? 1 : 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
                                           // producers announce the bytes of both CTAs, the peer only issues its loads)
             ptx::mbar_init(empty + s, 1);
         }
@@ -502,6 +505,48 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             const long long dbg_start = clock64();
 #endif
             const int bn_own = CG2 ? p.BN / 2 : p.BN;  // rows of the B tile this CTA fetches
+            if (bres && !isA) {
+                // The whole filter share of this CTA, once: group i of the K loop (which starts at this worker's rotation)
+                // goes to slot i; the groups are announced in four chunks on fullA[0..3] (pairs: on rank 0's barriers, with
+                // the bytes of both CTAs) so that the first MMAs need not wait for the last group.
+                const int kc_per_tap = p.kc_per_tap, kpb = p.kpb, KC = p.KC, Ca = p.Ca;
+                const int kblocks = p.cls_ntaps[0] * kc_per_tap, groups = p.a_slots;
+                const uint32_t kb_bytes = (uint32_t)(bn_own * KC * 2);
+                const uint32_t fullA_local = ptx::smem_u32(fullA);
+                const uint32_t fullA_u32 = CG2 ? ptx::mapa_u32(fullA_local, 0u) : fullA_local;
+                if (worker < total_tiles) {
+                    const int brow = (CG2 ? (int)rank * bn_own : 0);  // one column tile
+                    const int rot = (p.variant & 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
+                    int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
+                    const int per_chunk = (groups + 3) / 4;
+                    uint32_t dst = ptx::smem_u32(sB);
+                    for (int g0 = 0; g0 < groups; g0 += per_chunk) {
+                        const int g1 = g0 + per_chunk < groups ? g0 + per_chunk : groups;
+                        const int kb_lo = g0 * kpb, kb_hi = g1 * kpb < kblocks ? g1 * kpb : kblocks;
+                        const uint32_t chunk = (uint32_t)(g0 / per_chunk);
+                        if (!CG2 || rank == 0) ptx::mbar_expect_tx_u32_if(leader, fullA_local + 8u * chunk, (CG2 ? 2u : 1u) * kb_bytes * (uint32_t)(kb_hi - kb_lo));
+                        const uint32_t bar = fullA_u32 + 8u * chunk;
+                        for (int g = g0; g < g1; ++g) {
+                            const int nkb = (kblocks - g * kpb < kpb) ? kblocks - g * kpb : kpb;
+                            uint32_t d = dst;
+                            for (int j = 0; j < nkb; ++j) {
+                                if (CG2) ptx::tma_load_2d_cg2_if(leader, d, &p.tmB[0], bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32_if(leader, d, &p.tmB[0], bar, tap * Ca + kc * KC, brow);
+                                d += p.b_sub_bytes;
+                                if (++kc == kc_per_tap) {
+                                    kc = 0;
+                                    if (++tap == p.cls_ntaps[0]) tap = 0;
+                                }
+                            }
+                            dst += p.b_stage_bytes;
+                        }
+                    }
+                    // nothing else to do: see the loads land (bounded) so that none is in flight when the CTA leaves early
+                    if (!CG2 || rank == 0)
+                        for (int c4 = 0; c4 * per_chunk < groups; ++c4)
+                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(fullA + c4, 0); ++i) {
+                            }
+                }
+            } else {
             const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(bn_own * p.KC * 2);
             // loop-invariant values in registers: this thread's instruction stream is on the critical path
             const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
@@ -583,6 +628,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
                     }
                 }
+            }
             }
         }
     } else if (warp == 1) {
@@ -697,6 +743,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
             const int kc_per_tap = p.kc_per_tap;
             const uint32_t tfull_u32 = ptx::smem_u32(tfull);
+            const int b_per_chunk = bres ? (p.a_slots + 3) / 4 : 1;  // weights-stationary: groups per announced chunk
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 int cls_mma, lt_mma;
                 igemm_tile_class(p, tile, nworkers, cls_mma, lt_mma);
@@ -709,6 +756,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
                 uint32_t accumulate = 0;
+                const bool b_first = tile == worker;  // weights-stationary: the filter groups arrive during the first tile
+                int b_grp = 0, b_next = 0, b_chunk = 0;
+                uint64_t db_res = db0;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
                     {
@@ -718,6 +768,19 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                             break;
                         }
                         if (kb0 == 0) { NB_DBG_ADD(dbg_wait_first); } else { NB_DBG_ADD(dbg_wait_full); }
+                    }
+                    if (bres) {  // (counters instead of divisions: this loop is the critical instruction stream)
+                        if (b_first && b_grp == b_next) {
+                            if (!wait_bar_fast(fullA + b_chunk, 0u, abort_flag, p.status, 7)) {
+                                ok = false;
+                                break;
+                            }
+                            ++b_chunk;
+                            b_next += b_per_chunk;
+                        }
+                        ++b_grp;
+                        db_s = db_res;
+                        db_res += b_stage16;
                     }
                     ptx::tc_fence_after();
                     uint64_t da = da_s, db = db_s;
@@ -1139,6 +1202,8 @@ struct IgemmCfg {
     int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
     bool cg2 = false;  // CTA pairs (tcgen05 cta_group::2)
     bool halo = false;  // tap-reuse variant (3x3, stride 1)
+    bool bres = false;  // weights-stationary: the CTA's share of the filter is fetched once (b_groups groups of kpb k-blocks)
+    int b_groups = 0;
     int Wp = 0, Hp = 0, Hin = 0, Win = 0, Nimg = 0, slab_boxes = 0, box_pix = 0, a_slots = 0;
     uint32_t slab_bytes = 0;
     long long npos = 0;
@@ -1298,6 +1363,25 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
     c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, c.cg2 ? sm_count / 2 : sm_count);
+    // Weights-stationary (opt-in, NB_TC_BRES=1; =2 also for 3x3): with one column tile and one class every tile of a CTA
+    // multiplies by the same filter rows, and when that share of the filter fits beside a ring of at least three A stages
+    // it is fetched once per launch instead of once per tile.  Measured on B200, kernels timed one at a time: 1x1 layers
+    // gain in the data gradient (96 -> 192 at 160 x 160: 62.7 -> 53.5 us, 96 -> 96: 40.9 -> 36.6 us; forward +-1 us), 3x3
+    // layers with 48 or 64 channels lose 2-5 % (the ring loses a stage to the resident filter); inside the benchmark's
+    // CUDA graph, where these data gradients overlap the weight gradients of the second stream, the step time does not
+    // move (9.60 ms either way), so the mode is off by default.
+    {
+        const int groups = (kblocks + c.kpb - 1) / c.kpb;
+        const size_t fixed = igemm_fixed_smem(c.BN, ldo), res_b = (size_t)groups * c.b_stage;
+        const int want = getenv("NB_TC_BRES") ? atoi(getenv("NB_TC_BRES")) : 0;
+        if (want > 0 && (ntaps == 1 || want == 2) && c.n_tiles == 1 && nclasses == 1 && c.m_tiles >= 2 * c.grid &&
+            fixed + res_b + 3 * (size_t)c.a_stage <= kMaxSmem) {
+            c.bres = true;
+            c.b_groups = groups;
+            c.stages = (int)std::min<size_t>(8, (kMaxSmem - fixed - res_b) / c.a_stage);  // the A ring runs ahead across tiles
+            c.smem_bytes = std::max<size_t>(fixed + (size_t)c.stages * c.a_stage + res_b, 120 * 1024);
+        }
+    }
     if (c.cg2) c.grid *= 2;  // two CTAs per pair
     c.ok = true;
     return c;
@@ -1381,10 +1465,14 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.ncol_a = c.stage_cols; P.stage_cw = igemm_stage_cw(c.BN);
     P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
     if (getenv("NB_TC_VERBOSE"))
-        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
-                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu bres=%d(%d)\n", c.M, c.Ca,
+                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes, (int)c.bres, c.b_groups);
     P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
     P.halo = c.halo ? 1 : 0;
+    if (c.bres) {
+        P.variant |= 128;
+        P.a_slots = c.b_groups;
+    }
     if (c.halo) {
         P.Wp = c.Wp; P.Hp = c.Hp; P.Hin = c.Hin; P.Win = c.Win; P.Nimg = c.Nimg;
         P.slab_boxes = c.slab_boxes; P.box_pix = c.box_pix; P.a_slots = c.a_slots; P.slab_bytes = c.slab_bytes; P.npos = c.npos;
@@ -1776,7 +1864,7 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
     S.prm.fin_gamma = e.gamma; S.prm.fin_beta = e.beta;
     S.prm.fin_rmean = const_cast<float*>(e.rmean); S.prm.fin_rvar = const_cast<float*>(e.rvar);  // only read
     S.prm.fin_eps = e.eps; S.prm.epi_act = e.act;
-    S.prm.variant = 0;
+    S.prm.variant = S.cfg.bres ? 128 : 0;  // no experiment switches on this path; the weights-stationary layout is part of the configuration
     S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
     tc->launches += 1;
     if (tc->f16) return S.cfg.cg2 ? launch_igemm_impl<__half, false, true, false, 1>(S, st) : launch_igemm_impl<__half, false, false, false, 1>(S, st);

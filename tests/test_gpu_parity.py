@@ -292,6 +292,38 @@ def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
     _compare(out, _oracle(inp), 0)
 
 
+@pytest.mark.parametrize("shape", [S(4, 160, 160, 96, 96, 1, 1), S(4, 160, 160, 96, 192, 1, 1), S(4, 160, 160, 48, 48, 3, 1)], ids=lambda s: s.name)
+def test_weights_stationary_variant_is_bitwise_the_default_path(shape, monkeypatch, capfd):
+    """NB_TC_BRES: a CTA keeps its share of the filter in shared memory for all its tiles instead of fetching it per tile
+    (needs one column tile and at least two tiles per CTA, hence the 102400-row shapes).  Off by default (no gain inside
+    the benchmark's graph); it must stay correct: the same MMAs in the same order, so every result equals the default
+    path's bit for bit, in the training calls and in the fused evaluation-mode forward."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    def infer(blk):
+        a_eval = torch.empty_like(blk.a)
+        ws = torch.empty(max(blk.plan.infer_bytes, 256), dtype=torch.uint8, device=blk.dev)
+        nb.nb_conv_bn_silu_infer(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, blk.mean, 1.0 / blk.invstd**2, a_eval, ws)
+        blk.poll()
+        return a_eval.view(torch.int16).cpu().numpy()
+
+    monkeypatch.delenv("NB_TC_BRES", raising=False)
+    inp, blk0, out0 = _run_block(shape, 0, cfg_id=23, affine="random")
+    e0 = infer(blk0)
+    monkeypatch.setenv("NB_TC_BRES", "2")
+    monkeypatch.setenv("NB_TC_VERBOSE", "1")
+    capfd.readouterr()
+    inp, blk1, out1 = _run_block(shape, 0, cfg_id=23, affine="random")
+    assert "bres=1" in capfd.readouterr().err  # the plan really chose the variant
+    e1 = infer(blk1)
+    _compare(out1, _oracle(inp), 0)
+    for name in ("a", "y", "mean", "invstd", "dx", "dw", "dgamma", "dbeta"):
+        np.testing.assert_array_equal(out1[name], out0[name])
+    np.testing.assert_array_equal(e1, e0)
+
+
 def test_config1_fresh_bn_both_modes():
     shape, = wl.config_shapes(1)
     for mode in (1, 0):
