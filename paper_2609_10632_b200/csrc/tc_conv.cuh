@@ -88,8 +88,13 @@ struct IgemmParams {
 // neighbours in the order, so the dy rows they share are fetched from DRAM once and found in L2 three times instead of being
 // streamed once per class; the class of position r is rotated by the round of the persistent loop so that a worker
 // (whose tile numbers are nworkers apart) still cycles through heavy and light classes.
-__device__ __forceinline__ void igemm_tile_class(const IgemmParams& p, int tile, int nworkers, int& cls, int& lt) {
-    if (p.variant & 64) {
+// CLS4 = the launch has the four classes (a template parameter: every other launch has one class and pays nothing for
+// the decoding, which sits in the producer, MMA and epilogue loops).
+template <bool CLS4> __device__ __forceinline__ void igemm_tile_class(const IgemmParams& p, int tile, int nworkers, int& cls, int& lt) {
+    if (!CLS4) {
+        cls = 0;
+        lt = tile;
+    } else if (p.variant & 64) {
         const int r = tile & 3;
         const int round = (tile - r) / nworkers;
         cls = (r + ((nworkers & 1) ? 0 : round)) & 3;
@@ -304,8 +309,10 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 // accumulators, so the kernel writes the block's final activations (no statistics, no second pass); TMA stores only.
 // RES = 1 (forward with statistics only): no CTA has more tiles than accumulator sets, so after the finalize and a second
 // grid barrier every CTA applies BN + SiLU to its accumulators, which are still in TMEM, and writes the activations.
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0>
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0, bool BRES = false, bool CLS4 = false>
 __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
+    static_assert(!CLS4 || (!HALO && !STATS && !EPI && !RES && !BRES), "four classes: the stride-2 data gradient only");
+    static_assert(!BRES || (!HALO && !STATS && !EPI && !RES), "the weights-stationary variant is instantiated for the data gradient only");
     static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
     static_assert(!RES || (STATS && !HALO && !EPI), "the resident variant is the forward kernel with statistics");
     static_assert(!EPI || (!STATS && !HALO), "the fused per-channel epilogue is a forward-only variant without statistics");
@@ -313,9 +320,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = sA + (HALO ? (size_t)p.a_slots * p.slab_bytes : (size_t)p.stages * p.a_stage_bytes);
-    // Weights-stationary mode (variant bit 128, non-halo): the CTA's share of the whole filter stays in shared memory
-    // (p.a_slots groups of kpb k-blocks, fetched once, in the order of this CTA's K loop); the stage ring then holds A only.
-    const bool bres = !HALO && (p.variant & 128);
+    // Weights-stationary variant (BRES; a template parameter because the same switch as a run-time flag cost every launch
+    // of this kernel about 1 %): the CTA's share of the whole filter stays in shared memory (p.a_slots groups of kpb
+    // k-blocks, fetched once, in the order of this CTA's K loop); the stage ring then holds A only.
+    constexpr bool bres = BRES;
     uint8_t* stg = sB + (size_t)(bres ? p.a_slots : p.stages) * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
     const int cw = p.stage_cw;  // columns per staging pass (<= 64)
     const int pitch = cw * 2 + 16;
@@ -557,7 +565,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 int cls, lt;
-                igemm_tile_class(p, tile, nworkers, cls, lt);
+                igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
                 const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
                 const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
                 const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
@@ -746,7 +754,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             const int b_per_chunk = bres ? (p.a_slots + 3) / 4 : 1;  // weights-stationary: groups per announced chunk
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 int cls_mma, lt_mma;
-                igemm_tile_class(p, tile, nworkers, cls_mma, lt_mma);
+                igemm_tile_class<CLS4>(p, tile, nworkers, cls_mma, lt_mma);
                 const int kblocks = p.cls_ntaps[cls_mma] * kc_per_tap;
                 {
                     NB_DBG_T0();
@@ -861,7 +869,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
         for (int tile = worker; tile < total_tiles; tile += nworkers) {
             int cls, lt;
-            igemm_tile_class(p, tile, nworkers, cls, lt);
+            igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
             NB_DBG_T0();
             bool ok = true;
@@ -1300,7 +1308,7 @@ inline int igemm_stage_cw(int BN) {
 inline size_t igemm_fixed_smem(int BN, int ldo) {
     return 1024 /*alignment slack*/ + (size_t)2 * TC_BM * (igemm_stage_cw(BN) * 2 + 16) + (size_t)8 * ldo * 4 + 512;
 }
-inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses) {
+inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses, bool allow_bres = false) {
     IgemmCfg c;
     c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
     if (Ca % 16 || rowsB % 16 || M < 1) return c;
@@ -1363,8 +1371,8 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
     c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, c.cg2 ? sm_count / 2 : sm_count);
-    // Weights-stationary (opt-in, NB_TC_BRES=1; =2 also for 3x3): with one column tile and one class every tile of a CTA
-    // multiplies by the same filter rows, and when that share of the filter fits beside a ring of at least three A stages
+    // Weights-stationary (data gradient only; opt-in, NB_TC_BRES=1; =2 also for 3x3): with one column tile and one class
+    // every tile of a CTA multiplies by the same filter rows, and when that share of the filter fits beside a ring of at least three A stages
     // it is fetched once per launch instead of once per tile.  Measured on B200, kernels timed one at a time: 1x1 layers
     // gain in the data gradient (96 -> 192 at 160 x 160: 62.7 -> 53.5 us, 96 -> 96: 40.9 -> 36.6 us; forward +-1 us), 3x3
     // layers with 48 or 64 channels lose 2-5 % (the ring loses a stage to the resident filter); inside the benchmark's
@@ -1374,7 +1382,7 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
         const int groups = (kblocks + c.kpb - 1) / c.kpb;
         const size_t fixed = igemm_fixed_smem(c.BN, ldo), res_b = (size_t)groups * c.b_stage;
         const int want = getenv("NB_TC_BRES") ? atoi(getenv("NB_TC_BRES")) : 0;
-        if (want > 0 && (ntaps == 1 || want == 2) && c.n_tiles == 1 && nclasses == 1 && c.m_tiles >= 2 * c.grid &&
+        if (allow_bres && want > 0 && (ntaps == 1 || want == 2) && c.n_tiles == 1 && nclasses == 1 && c.m_tiles >= 2 * c.grid &&
             fixed + res_b + 3 * (size_t)c.a_stage <= kMaxSmem) {
             c.bres = true;
             c.b_groups = groups;
@@ -1469,10 +1477,7 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
                 c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes, (int)c.bres, c.b_groups);
     P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
     P.halo = c.halo ? 1 : 0;
-    if (c.bres) {
-        P.variant |= 128;
-        P.a_slots = c.b_groups;
-    }
+    if (c.bres) P.a_slots = c.b_groups;
     if (c.halo) {
         P.Wp = c.Wp; P.Hp = c.Hp; P.Hin = c.Hin; P.Win = c.Win; P.Nimg = c.Nimg;
         P.slab_boxes = c.slab_boxes; P.box_pix = c.box_pix; P.a_slots = c.a_slots; P.slab_bytes = c.slab_bytes; P.npos = c.npos;
@@ -1539,20 +1544,20 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
     return true;
 }
 
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0, bool BRES = false, bool CLS4 = false> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     // the attribute belongs to the (function, device) pair: one bit per device ordinal that already has it
     static std::atomic<unsigned long long> attr_set{0};
     int dev = 0;
     cudaGetDevice(&dev);
     const unsigned long long bit = 1ull << (dev & 63);
     if (!(attr_set.load(std::memory_order_acquire) & bit)) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES, BRES, CLS4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
             return NB_ERR_CUDA;
         }
         attr_set.fetch_or(bit, std::memory_order_release);
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES, BRES, CLS4>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
@@ -1561,6 +1566,10 @@ template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES =
 }
 template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
     if (s.cfg.halo) return launch_igemm_impl<OutT, STATS, true, true>(s, st);
+    if constexpr (!STATS) {  // the data gradient: the only launch with four classes or the weights-stationary configuration
+        if (s.prm.nclasses == 4) return s.cfg.cg2 ? launch_igemm_impl<OutT, false, true, false, 0, 0, false, true>(s, st) : launch_igemm_impl<OutT, false, false, false, 0, 0, false, true>(s, st);
+        if (s.cfg.bres) return s.cfg.cg2 ? launch_igemm_impl<OutT, false, true, false, 0, 0, true>(s, st) : launch_igemm_impl<OutT, false, false, false, 0, 0, true>(s, st);
+    }
     return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true, false>(s, st) : launch_igemm_impl<OutT, STATS, false, false>(s, st);
 }
 
@@ -1680,7 +1689,7 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
         }
         IgemmCfg c;
         if (g.k == 3 && g.stride == 1 && g.pad == 1) c = halo_configure(g.n, g.h, g.w, g.c_out, g.c_in, g.c_in, sm_count);
-        if (!c.ok) c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls);
+        if (!c.ok) c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls, true);
         if (c.ok) {
             tc->dg.cfg = c;
             fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
@@ -1864,7 +1873,7 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
     S.prm.fin_gamma = e.gamma; S.prm.fin_beta = e.beta;
     S.prm.fin_rmean = const_cast<float*>(e.rmean); S.prm.fin_rvar = const_cast<float*>(e.rvar);  // only read
     S.prm.fin_eps = e.eps; S.prm.epi_act = e.act;
-    S.prm.variant = S.cfg.bres ? 128 : 0;  // no experiment switches on this path; the weights-stationary layout is part of the configuration
+    S.prm.variant = 0;  // no experiment switches on this path
     S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
     tc->launches += 1;
     if (tc->f16) return S.cfg.cg2 ? launch_igemm_impl<__half, false, true, false, 1>(S, st) : launch_igemm_impl<__half, false, false, false, 1>(S, st);

@@ -294,10 +294,10 @@ def test_tap_reuse_variant_matches_oracle(shape, monkeypatch):
 
 @pytest.mark.parametrize("shape", [S(4, 160, 160, 96, 96, 1, 1), S(4, 160, 160, 96, 192, 1, 1), S(4, 160, 160, 48, 48, 3, 1)], ids=lambda s: s.name)
 def test_weights_stationary_variant_is_bitwise_the_default_path(shape, monkeypatch, capfd):
-    """NB_TC_BRES: a CTA keeps its share of the filter in shared memory for all its tiles instead of fetching it per tile
-    (needs one column tile and at least two tiles per CTA, hence the 102400-row shapes).  Off by default (no gain inside
-    the benchmark's graph); it must stay correct: the same MMAs in the same order, so every result equals the default
-    path's bit for bit, in the training calls and in the fused evaluation-mode forward."""
+    """NB_TC_BRES: in the data gradient a CTA keeps its share of the filter in shared memory for all its tiles instead of
+    fetching it per tile (needs one column tile and at least two tiles per CTA, hence the 102400-row shapes).  Off by
+    default (no gain inside the benchmark's graph); it must stay correct: the same MMAs in the same order, so every
+    result equals the default path's bit for bit (the other calls of such a plan, checked too, do not use the variant)."""
     import torch
 
     from paper_2609_10632_b200 import binding as nb
