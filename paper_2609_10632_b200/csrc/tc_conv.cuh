@@ -21,6 +21,14 @@
 
 namespace nbcbs {
 
+// Timing-experiment switches (bits 4..32 of IgemmParams::variant: parts of the kernel are left out and the results are
+// wrong) are compiled in only with -DNB_TC_EXPERIMENTS; a normal build does not test them in its loops.
+#ifdef NB_TC_EXPERIMENTS
+#define NB_TC_SWITCH(p, bits) ((p).variant & (bits))
+#else
+#define NB_TC_SWITCH(p, bits) 0
+#endif
+
 // ------------------------------------------------------------------------------------------ kernel parameters
 struct IgemmParams {
     CUtensorMap tmA;     // im2col map over the activation [N][Hs][Ws][Ca]
@@ -524,7 +532,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 const uint32_t fullA_u32 = CG2 ? ptx::mapa_u32(fullA_local, 0u) : fullA_local;
                 if (worker < total_tiles) {
                     const int brow = (CG2 ? (int)rank * bn_own : 0);  // one column tile
-                    const int rot = (p.variant & 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
+                    const int rot = NB_TC_SWITCH(p, 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
                     int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
                     const int per_chunk = (groups + 3) / 4;
                     uint32_t dst = ptx::smem_u32(sB);
@@ -582,7 +590,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // each CTA starts its K loop at a different k-block so that the CTAs do not all ask L2 for the same
                 // filter lines at the same moment
                 const int ntaps_c = p.cls_ntaps[cls];
-                const int rot = (p.variant & 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
+                const int rot = NB_TC_SWITCH(p, 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
                 int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
@@ -880,7 +888,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             ok = epi2_bar_and(ok);
             if (!ok) break;
             ptx::tc_fence_after();
-            if ((p.variant & 8) || ncol == 0) {
+            if (NB_TC_SWITCH(p, 8) || ncol == 0) {
                 ptx::tc_fence_before();
                 if (CG2) {
                     __syncwarp();
@@ -910,7 +918,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // The team's columns go through the staging buffer in passes of at most cw (<= 64) columns.
                 for (int cb = 0; cb < ncol; cb += cw) {
                 const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
-                if (tma_out && !(p.variant & (16 | 32))) {
+                if (tma_out && !NB_TC_SWITCH(p, (16 | 32))) {
                     const bool last = h == mh - 1 && cb + cw >= ncol;  // last TMEM read of this tile: the accumulator set becomes free
                     auto release = [&]() {
                         if (last) {
@@ -1005,7 +1013,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     __syncwarp();  // every warp only reads back the 32 rows it staged itself
                 }
                 NB_DBG_PHASE(dbg_pack);
-                if (STATS && !(p.variant & 16)) {
+                if (STATS && !NB_TC_SWITCH(p, 16)) {
                     // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
                     // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends.
                     // A lane owns two adjacent channels (a pass has at most 64), two rows per step for independent chains.
@@ -1035,7 +1043,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
                 // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
                 // output offset of row r, the others fetch it by shuffle
-                if (!tma_out && !(p.variant & 32)) {
+                if (!tma_out && !NB_TC_SWITCH(p, 32)) {
                     const int cpr = npass / 8;  // 16-byte pieces per staged row (<= 8)
                     long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
                     if (HALO) {
