@@ -39,12 +39,12 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # of the cfg5 workload) from the ncu capture summarised in profiles/launch_list_cfg5_step.md (warm caches, as in a real
 # step: most layers' tensors stay in the 126 MB L2, so the traffic is well below the algorithmic bytes).
 NCU_DRAM_BYTES_PER_LAUNCH_CFG5 = {
-    "conv_fprop": (807 + 1283 + 39 + 657 + 645 + 148) * 1e6 / 77,
-    "conv_dgrad": (625 + 26 + 155 + 1182 + 498 + 65) * 1e6 / 77,
-    "conv_wgrad": (2252 + 185 + 1405 + 18) * 1e6 / 77,
-    "bn_silu_apply": (445 + 773) * 1e6 / 77,
-    "bn_silu_bwd_reduce": (1986 + 909) * 1e6 / 77,
-    "bn_silu_bwd_dy": (1084 + 801) * 1e6 / 77,
+    "conv_fprop": (2129 + 1439) * 1e6 / 77,
+    "conv_dgrad": (576 + 1708) * 1e6 / 77,
+    "conv_wgrad": (2434 + 1458) * 1e6 / 77,
+    "bn_silu_apply": (440 + 770) * 1e6 / 77,
+    "bn_silu_bwd_reduce": (1989 + 906) * 1e6 / 77,
+    "bn_silu_bwd_dy": (1090 + 794) * 1e6 / 77,
 }
 
 
