@@ -127,9 +127,7 @@ nb_status nb_cbs_workspace_bytes(nb_cbs_plan plan, size_t* fwd_bytes, size_t* bw
 nb_status nb_cbs_plan_set_pitches(nb_cbs_plan plan, int64_t ld_x, int64_t ld_a, int64_t ld_g);
 
 /* Which implementation each convolution of this plan runs on: writes three ints (fprop, dgrad, wgrad),
- * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel, 2 = the tap-reuse variant of the tensor-core kernel
- * (3x3 stride-1 layers only; an experiment that is chosen only when the environment variable NB_TC_HALO is 1
- * at plan creation). */
+ * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel. */
 nb_status nb_cbs_plan_paths(nb_cbs_plan plan, int32_t* paths3);
 
 /* Synchronise `stream`, then report whether any kernel launched through this plan gave up a bounded
@@ -145,6 +143,14 @@ nb_status nb_cbs_poll_status(nb_cbs_plan plan, void* stream);
  * nb_cbs_profile_site_name(i): name of kernel site i, NULL once i is past the last site.
  * nb_cbs_profile_read: accumulated milliseconds and launch count of one site since the last enable call. */
 unsigned long long nb_cbs_launch_count(void);
+/* Test hook for the bounded waits (the paper has no counterpart).  Every wait inside the kernels is bounded and reports
+ * NB_ERR_TIMEOUT through nb_cbs_poll_status instead of hanging.  This call makes that path observable without any
+ * fault: the NEXT launch of this plan that contains a grid-wide barrier (the tensor-core forward kernel, or the backward
+ * reduce kernel, whichever is launched first) waits for one block more than its grid has, for at most `limit_ms`
+ * milliseconds (1..1000), gives up, skips its finalize step and returns normally; nb_cbs_poll_status then reports
+ * NB_ERR_TIMEOUT (the outputs of that call are not valid), and later calls on the plan work as usual.
+ * NB_ERR_UNSUPPORTED for plans without such kernels (NB_CBS_FLAG_SHARED_GPU). */
+nb_status nb_cbs_debug_expire_next_wait(nb_cbs_plan plan, int32_t limit_ms);
 nb_status nb_cbs_profile_enable(nb_cbs_plan plan, int32_t enable);
 const char* nb_cbs_profile_site_name(int32_t site);
 nb_status nb_cbs_profile_read(nb_cbs_plan plan, int32_t site, double* total_ms, int64_t* launches);

@@ -11,7 +11,7 @@ import os
 from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_size_t, c_uint32, c_void_p
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libnb_cbs.so")
+LIB_PATH = os.environ.get("NB_CBS_LIBRARY") or os.path.join(HERE, "libnb_cbs.so")  # (the variable: another build of the same library, for A/B timing)
 
 NB_OK = 0
 NB_ERR_INVALID_ARG, NB_ERR_UNSUPPORTED, NB_ERR_WORKSPACE, NB_ERR_ALIGNMENT = 1, 2, 3, 4
@@ -29,6 +29,7 @@ EXPORTS = (
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step", "nb_sgd_clip_nesterov_step_scaled",
     "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd", "nb_cbs_plan_set_pitches",
+    "nb_cbs_debug_expire_next_wait",
 )
 
 
@@ -82,6 +83,7 @@ def load() -> ctypes.CDLL:
         lib.nb_cbs_plan_paths.argtypes = [V, POINTER(c_int32)]
         lib.nb_cbs_plan_set_pitches.argtypes = [V, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64]
         lib.nb_cbs_poll_status.argtypes = [V, V]
+        lib.nb_cbs_debug_expire_next_wait.argtypes = [V, c_int32]
         lib.nb_conv_bn_silu_fwd.argtypes = [V, V, V, FP, FP, FP, FP, V, FP, FP, V, V, c_size_t, V]
         lib.nb_bn_stats.argtypes = [V, V, c_int32, FP, FP, FP, FP, V, c_size_t, V]
         lib.nb_conv_bn_silu_bwd_data.argtypes = [V, V, V, FP, FP, FP, FP, V, V, FP, FP, V, V, c_size_t, V]
@@ -246,6 +248,11 @@ def nb_conv_bn_silu_fwd(plan: Plan, x, w, gamma, beta, running_mean, running_var
 def nb_bn_stats(plan: Plan, y, y_dtype, mean, invstd, sum_, sumsq, workspace, stream=None):
     _check(load().nb_bn_stats(plan.handle, _ptr(y), y_dtype, _ptr(mean), _ptr(invstd), _ptr(sum_), _ptr(sumsq), _ptr(workspace),
                               _nbytes(workspace), _stream(stream)))
+
+
+def nb_cbs_debug_expire_next_wait(plan: "Plan", limit_ms: int):
+    """Test hook: the plan's next grid-barrier launch gives up its wait after `limit_ms` ms (see include/nb_cbs.h)."""
+    _check(load().nb_cbs_debug_expire_next_wait(plan.handle, int(limit_ms)))
 
 
 def nb_bn_stats_static(y, y_dtype, m, c, eps, mean, invstd, sum_=None, sumsq=None, stream=None):

@@ -300,6 +300,8 @@ struct BwdFused {
     float *dgamma, *dbeta, *coef;
     const __nv_bfloat16* w;  // filter and its rearranged copy for the data-gradient GEMM (wt = NULL: nothing to rearrange)
     __nv_bfloat16* wt;
+    int wait_limit_ms;  // bound of the grid-barrier wait in milliseconds (0: the default of about two seconds)
+    int bar_extra;      // test knob: the barrier expects this many more arrivals than there are blocks (0 in normal use)
 };
 template <typename YT, typename AT, bool FAST, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
@@ -307,7 +309,9 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
                                                                   const float* __restrict__ beta, float* __restrict__ partials, BwdFused fb,
                                                                   WtParams wtp, long long ld_g) {
-    pdl_launch_dependents();
+    // With the fused finalize this kernel contains a grid barrier: it is launched without the programmatic-serialization
+    // attribute and lets the next kernel go only behind the barrier (see grid_arrive).
+    if (!fb.on) pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "g and y must have the same element size");
@@ -391,15 +395,15 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
             }
             if (wt_tiles > 2 * (int)gridDim.x) wt_transform_blocks(fb.w, fb.wt, wtp, (int)blockIdx.x, (int)gridDim.x, 2);  // rare: very large filters
         }
-        if (tid == 0) ok = grid_wait(fb.ctr, (int)gridDim.x) ? 1 : 0;
+        if (tid == 0) ok = grid_wait(fb.ctr, (int)gridDim.x + fb.bar_extra, wait_limit_ns(fb.wait_limit_ms)) ? 1 : 0;
         __syncthreads();
+        pdl_launch_dependents();  // every block of this grid is resident and past the barrier
         if (ok) {
             const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
             for (int c = (int)blockIdx.x + (int)gridDim.x * warp; c < C; c += (int)gridDim.x * nwarps)
                 bn_bwd_finalize_channel<true>(partials, (int)gridDim.x, C, c, lane, fb.M, mean, invstd, gamma, beta, fb.dgamma, fb.dbeta, fb.coef);
-        } else if (tid == 0 && atomicCAS(fb.status + ST_ERR, 0, 2 /* NB_ERR_TIMEOUT */) == 0) {
-            fb.status[ST_WHERE] = 21;
-            fb.status[ST_DETAIL] = (int)blockIdx.x;
+        } else if (tid == 0) {
+            report_timeout(fb.status, SITE_GRID_BARRIER_BWD, (int)blockIdx.x);
         }
         __syncthreads();
         if (tid == 0) grid_depart(fb.ctr, (int)gridDim.x);

@@ -71,7 +71,8 @@ struct nb_cbs_plan_s {
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
     long long ld_a = 0, ld_g = 0;  // row pitch (elements) of a_out in the forward call and of g in the backward call (set by nb_cbs_plan_set_pitches; default c_out)
     bool pitched = false;
-    bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or NB_FUSE_FINALIZE=0 at plan creation)
+    bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or an occupancy query that failed)
+    int expire_next_ms = 0;     // nb_cbs_debug_expire_next_wait: the next grid-barrier launch waits for one block too many, for at most this long
     bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
     int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
@@ -174,15 +175,25 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
         memset(&fb, 0, sizeof fb);
         if (fuse) {
             fb.on = 1; fb.ctr = p->status + ST_BAR_BWD; fb.status = p->status; fb.M = (double)p->g.m;
+            if (p->expire_next_ms > 0) {
+                fb.wait_limit_ms = p->expire_next_ms; fb.bar_extra = 1;
+                p->expire_next_ms = 0;
+            }
             fb.dgamma = dgamma; fb.dbeta = dbeta; fb.coef = coef;
             fb.w = static_cast<const __nv_bfloat16*>(w); fb.wt = wtp ? static_cast<__nv_bfloat16*>(wt) : nullptr;
         }
-        if (p->ld_g)
-            launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST, true>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
-                static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none, p->ld_g);
-        else
-            launch_k(bn_silu_bwd_reduce_kernel<YT, AT, FAST, false>, dim3(e.blocks_reduce), dim3(e.tpb), (size_t)e.tpb * e.vec * sizeof(float), st, 1,
-                static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd, gamma, beta, partials, fb, wtp ? *wtp : none, (long long)C);
+        // with the grid barrier (fuse): launched without the programmatic-serialization attribute, see grid_arrive
+        const size_t red_smem = (size_t)e.tpb * e.vec * sizeof(float);
+        auto go = [&](auto kernel, long long ld) {
+            if (fuse)
+                launch_k<false>(kernel, dim3(e.blocks_reduce), dim3(e.tpb), red_smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean,
+                                invstd, gamma, beta, partials, fb, wtp ? *wtp : none, ld);
+            else
+                launch_k(kernel, dim3(e.blocks_reduce), dim3(e.tpb), red_smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd,
+                         gamma, beta, partials, fb, wtp ? *wtp : none, ld);
+        };
+        if (p->ld_g) go(bn_silu_bwd_reduce_kernel<YT, AT, FAST, true>, p->ld_g);
+        else go(bn_silu_bwd_reduce_kernel<YT, AT, FAST, false>, (long long)C);
         NB_LAUNCH_OK("bn_silu_bwd_reduce");
     }
     if (!fuse) {
@@ -298,7 +309,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->g = g;
     p->device = device;
     p->sm_count = prop.multiProcessorCount;
-    p->fuse_finalize = !(d->flags & NB_CBS_FLAG_SHARED_GPU) && !(getenv("NB_FUSE_FINALIZE") && atoi(getenv("NB_FUSE_FINALIZE")) == 0);
+    p->fuse_finalize = !(d->flags & NB_CBS_FLAG_SHARED_GPU);
 
     EwCfg& e = p->ew;
     e.vec = vec;
@@ -314,7 +325,11 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     {
         auto wave = [&](const void* fn, size_t dyn_smem, int min_vecs) {
             int occ = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, e.tpb, dyn_smem) != cudaSuccess || occ < 1) occ = 2;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, e.tpb, dyn_smem) != cudaSuccess || occ < 1) {
+                cudaGetLastError();
+                occ = 1;
+                p->fuse_finalize = false;  // residency unknown: no grid barriers on this plan (separate finalize kernels)
+            }
             const long long cap = (long long)p->sm_count * occ;
             return (int)std::max<long long>(1, std::min<long long>((max_blocks + min_vecs - 1) / min_vecs, cap));
         };
@@ -433,7 +448,7 @@ nb_status nb_cbs_plan_set_pitches(nb_cbs_plan p, int64_t ld_x, int64_t ld_a, int
     auto bad = [&](int64_t ld, int channels) { return ld != 0 && ld != channels && (ld < channels || ld % vec != 0); };  // 0 or the channel count: dense
     if (bad(ld_x, p->g.c_in) || bad(ld_a, p->g.c_out) || bad(ld_g, p->g.c_out))
         return fail(NB_ERR_INVALID_ARG, "a pitch must be 0 (dense) or at least the channel count and a multiple of %d elements", vec);
-    if (ld_x != 0 && ld_x != p->g.c_in && (is_f32(p) || p->stem || !p->tc.fprop || !p->tc.wgrad || p->tc.fp.cfg.halo))
+    if (ld_x != 0 && ld_x != p->g.c_in && (is_f32(p) || p->stem || !p->tc.fprop || !p->tc.wgrad))
         return fail(NB_ERR_UNSUPPORTED, "an input pitch needs the tensor-core forward and weight-gradient kernels (this plan runs them elsewhere)");
     p->tc.ld_x = (ld_x == p->g.c_in) ? 0 : ld_x;
     p->ld_a = (ld_a == p->g.c_out) ? 0 : ld_a;
@@ -449,8 +464,8 @@ nb_status nb_cbs_plan_set_pitches(nb_cbs_plan p, int64_t ld_x, int64_t ld_a, int
 nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
     g_err.clear();
     if (!p || !paths3) return fail(NB_ERR_INVALID_ARG, "NULL argument");
-    paths3[0] = p->tc.fprop ? (p->tc.fp.cfg.halo ? 2 : 1) : 0;
-    paths3[1] = p->tc.dgrad ? (p->tc.dg.cfg.halo ? 2 : 1) : 0;
+    paths3[0] = p->tc.fprop ? 1 : 0;
+    paths3[1] = p->tc.dgrad ? 1 : 0;
     paths3[2] = p->tc.wgrad ? 1 : 0;
     return NB_OK;
 }
@@ -469,6 +484,15 @@ nb_status nb_cbs_profile_enable(nb_cbs_plan p, int32_t enable) {
         p->prof_ms[i] = 0.0;
         p->prof_n[i] = 0;
     }
+    return NB_OK;
+}
+
+nb_status nb_cbs_debug_expire_next_wait(nb_cbs_plan p, int32_t limit_ms) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    if (limit_ms < 1 || limit_ms > 1000) return fail(NB_ERR_INVALID_ARG, "limit_ms must be between 1 and 1000, got %d", limit_ms);
+    if (!p->fuse_finalize) return fail(NB_ERR_UNSUPPORTED, "this plan launches no kernel with a grid barrier");
+    p->expire_next_ms = limit_ms;
     return NB_OK;
 }
 
@@ -518,7 +542,7 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     float* shift = reinterpret_cast<float*>(ws + p->off_shift);
     float* part = reinterpret_cast<float*>(ws + p->off_fpart);
     int nparts = p->ew.blocks_stats;
-    bool finalized = false, applied = false;
+    bool finalized = false;
     if (is_f32(p)) {
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
@@ -535,9 +559,11 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
         // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
-        const bool fuse = p->fuse_finalize;
+        const bool fuse = p->fuse_finalize && p->tc.fp_barrier_ok;
         const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
-        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, p->ld_a ? nullptr : a_out, &applied);
+        const int expire_ms = fuse ? p->expire_next_ms : 0;
+        if (fuse) p->expire_next_ms = 0;
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, expire_ms, expire_ms > 0 ? 1 : 0);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
@@ -548,7 +574,6 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     }
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
-    if (applied) return NB_OK;  // the forward kernel kept its accumulators in TMEM and wrote the activations itself
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st, p->ld_a);
     return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a));
 }

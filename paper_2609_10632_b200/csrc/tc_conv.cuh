@@ -1,8 +1,8 @@
 // Tensor-core convolution kernels for sm_100a: an implicit GEMM whose A operand (activation pixels x channels of
 // one filter tap) is fetched by TMA in im2col mode, whose B operand (filter rows) is fetched by tiled TMA, whose
-// products are issued as tcgen05.mma by one thread with fp32 accumulators in TMEM, and whose epilogue (four warps)
+// products are issued as tcgen05.mma by one thread with fp32 accumulators in TMEM, and whose epilogue (eight warps)
 // reads the accumulators back with tcgen05.ld, converts, stages the tile in shared memory, takes per-channel sums
-// for the batch statistics and writes coalesced rows.  The same kernel computes fprop (A = x, B = w) and dgrad
+// for the batch statistics and hands the rows to TMA stores.  The same kernel computes fprop (A = x, B = w) and dgrad
 // (A = dy, B = the filter rearranged per output-parity class).  No multicast anywhere; every wait is bounded.
 #pragma once
 #include <atomic>
@@ -21,14 +21,6 @@
 
 namespace nbcbs {
 
-// Timing-experiment switches (bits 4..32 of IgemmParams::variant: parts of the kernel are left out and the results are
-// wrong) are compiled in only with -DNB_TC_EXPERIMENTS; a normal build does not test them in its loops.
-#ifdef NB_TC_EXPERIMENTS
-#define NB_TC_SWITCH(p, bits) ((p).variant & (bits))
-#else
-#define NB_TC_SWITCH(p, bits) 0
-#endif
-
 // ------------------------------------------------------------------------------------------ kernel parameters
 struct IgemmParams {
     CUtensorMap tmA;     // im2col map over the activation [N][Hs][Ws][Ca]
@@ -41,6 +33,7 @@ struct IgemmParams {
     // matrix, tap list and output offset (the four output-parity classes of a stride-2 data gradient); for the order of
     // the tiles see igemm_tile_class.
     int nclasses, tiles_per_class;
+    int cls_interleave;          // four classes: the classes of one [m][n] tile are neighbours in the tile order
     int cls_ntaps[4], cls_oa[4], cls_ob[4];
     int Ca, KC, kc_per_tap;
     int kpb;                     // k-blocks (of KC channels) per pipeline stage
@@ -50,15 +43,11 @@ struct IgemmParams {
     int acc_bufs;                // accumulator sets in TMEM (2 when 2*mh*acc_stride <= 512)
     int ncol_a;                  // columns of a tile that epilogue team 0 handles (team 1: the other BN - ncol_a)
     int stage_cw;                // columns per staging pass of a team (<= 64)
-    // When GEMM row == output row (not a stride-2 dgrad, not the halo variant) a warp hands each staged [32 x width] piece
+    // When GEMM row == output row (everything but a stride-2 dgrad) a warp hands each staged [32 x width] piece
     // to TMA: tmOut[i] is a tiled map over the output [M][ldo] with box {out_w[i], 32}; clipping at M is the map's.
     int tma_store;
     int out_w[3];
     CUtensorMap tmOut[3];
-    // Resident variant (RES): every accumulator of the launch stays in TMEM until the statistics are final; after a second
-    // grid barrier the CTA reads its accumulators again, applies scale, shift and SiLU and stores the activations
-    // through maps over the activation tensor with the same boxes as tmOut.  Those maps sit in tmB[1..3], which a forward
-    // launch (one class) does not use: the parameter block of every launch stays as small as it was.
     // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
     // b, b + gridDim.x, ...: sums the per-CTA partials in fp64 and writes mean, invstd, scale, shift and the running
     // statistics, which saves the separate finalize launch between this kernel and the apply pass.
@@ -73,26 +62,19 @@ struct IgemmParams {
     int epi_act;
     int stages, acc_stride, tmem_cols;
     uint32_t umma_swizzle, sbo, a_stage_bytes, b_stage_bytes, idesc;
-    int variant;                 // experiment switches
     int a_tiled;                 // 1: A is a plain [M][Ca] matrix fetched with a tiled 2-D map (1x1 stride-1 convolutions)
     int ldo;                     // channels per output pixel
     int Hout, Wout, os;          // GEMM row (n,i,j) -> output pixel (n, i*os+oa, j*os+ob) of an Hout x Wout image
     void* out;
-    long long* dbg;   // optional [gridDim.x][8] cycle counters (only read when built with NB_TC_DEBUG_TIMING)
     float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
     int* status;
+    int wait_limit_ms;  // bound of the grid-barrier wait in milliseconds (0: the default of about two seconds)
+    int bar_extra;      // test knob: the grid barrier expects this many more arrivals than there are CTAs (0 in normal use)
     uint16_t off_w[4][9], off_h[4][9];
-    // Halo mode (3x3, stride 1): the GEMM rows are the positions of the zero-padded raster [N][H+2][W+2]; one slab of
-    // 128*mh + 2*(W+2) + 2 consecutive positions x 64 channels serves all nine taps (tap (r,t) starts r*(W+2)+t rows in).
-    int halo, Wp, Hp, Hin, Win, Nimg;
-    int slab_boxes, box_pix, a_slots;
-    uint32_t slab_bytes;
-    long long npos;            // N*(H+2)*(W+2)
-    uint32_t tap_off16[9];     // start of tap t inside the slab, in 16-byte units
 };
 
 // Tile number -> (class, tile within the class).  Default order: class by class, classes with more taps first.  With
-// variant bit 64 (set for the four parity classes of a stride-2 data gradient) the four classes of one [m][n] tile are
+// cls_interleave (set for the four parity classes of a stride-2 data gradient) the four classes of one [m][n] tile are
 // neighbours in the order, so the dy rows they share are fetched from DRAM once and found in L2 three times instead of being
 // streamed once per class; the class of position r is rotated by the round of the persistent loop so that a worker
 // (whose tile numbers are nworkers apart) still cycles through heavy and light classes.
@@ -102,7 +84,7 @@ template <bool CLS4> __device__ __forceinline__ void igemm_tile_class(const Igem
     if (!CLS4) {
         cls = 0;
         lt = tile;
-    } else if (p.variant & 64) {
+    } else if (p.cls_interleave) {
         const int r = tile & 3;
         const int round = (tile - r) / nworkers;
         cls = (r + ((nworkers & 1) ? 0 : round)) & 3;
@@ -113,19 +95,9 @@ template <bool CLS4> __device__ __forceinline__ void igemm_tile_class(const Igem
     }
 }
 
-#ifdef NB_TC_DEBUG_TIMING
-#define NB_DBG_T0() const long long dbg_t0__ = clock64()
-#define NB_DBG_ADD(var) var += clock64() - dbg_t0__
-#define NB_DBG_PHASE(var) { const long long dbg_now__ = clock64(); var += dbg_now__ - dbg_ph__; dbg_ph__ = dbg_now__; }
-#else
-#define NB_DBG_T0()
-#define NB_DBG_ADD(var)
-#define NB_DBG_PHASE(var)
-#endif
 constexpr int TC_BM = 128;
 constexpr int IG_THREADS = 352;  // implicit-GEMM kernel: the roles below plus a second epilogue team in warps 7-10
 constexpr int TC_THREADS = 224;  // warp 0: TMA producer for A, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue, warp 6: TMA producer for B
-constexpr int WG_THREADS = 192;  // wgrad kernel: warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
@@ -133,8 +105,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 
-// Bounded mbarrier wait: gives up after ~2 s (or as soon as another role has given up), records the site.
-__device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+// Bounded mbarrier wait: gives up after `limit_ns` (or as soon as another role has given up), records the site.
+__device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int site, uint64_t limit_ns = kWaitLimitNs) {
     uint64_t t0 = 0;
     for (uint32_t i = 0;; ++i) {
         if (ptx::mbar_try_wait_parked(bar, parity, 4000u)) return true;
@@ -143,12 +115,9 @@ __device__ __noinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile i
             const uint64_t now = global_timer_ns();
             if (t0 == 0) {
                 t0 = now;
-            } else if (now - t0 > 2000000000ull) {
+            } else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
-                if (atomicCAS(status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
-                    status[ST_WHERE] = site;
-                    status[ST_DETAIL] = (int)blockIdx.x;
-                }
+                report_timeout(status, site, (int)blockIdx.x);
                 return false;
             }
         }
@@ -228,16 +197,6 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
     ptx::tmem_ld_wait();
     release();
     if (EPI) {
-        if (EPI == 2) {  // the value the training path stores as y and normalises: the accumulator rounded to fp16 (saturating)
-#pragma unroll
-            for (int j = 0; j < NP; j += 2) {
-                uint32_t v;
-                asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(v) : "f"(__uint_as_float(r[j + 1])), "f"(__uint_as_float(r[j])));
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v));
-                r[j] = __float_as_uint(f.x);
-                r[j + 1] = __float_as_uint(f.y);
-            }
-        }
         if (act) {
 #pragma unroll
             for (int j = 0; j < NP; j += 2) {
@@ -309,30 +268,19 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 // CG2 = the CTAs run as pairs (clusters of two): rank 0 issues tcgen05.mma.cta_group::2 with M = 256; each CTA owns 128
 // of the rows (its own A tile, accumulator and epilogue) and fetches half of the B tile, which halves the filter
 // bytes written to and read from each SM's shared memory.
-// HALO = the tap-reuse variant for 3x3 stride-1 convolutions (always CTA pairs): A is fetched once per 64-channel block
-// as a slab of padded-raster positions and the nine taps are nine row offsets into it, so the activation bytes written to
-// shared memory drop from 9 x 128*mh rows to 128*mh + 2*(W+2) + 2 rows per block.  Rows that fall on the padding ring
-// are computed and discarded.
 // EPI = 1: the epilogue applies a per-channel scale and shift (evaluation-mode BN or a bias) and optionally SiLU to the
 // accumulators, so the kernel writes the block's final activations (no statistics, no second pass); TMA stores only.
-// RES = 1 (forward with statistics only): no CTA has more tiles than accumulator sets, so after the finalize and a second
-// grid barrier every CTA applies BN + SiLU to its accumulators, which are still in TMEM, and writes the activations.
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0, bool BRES = false, bool CLS4 = false>
+// STATS (forward of a training block): TMA stores only; with fin_on the kernel ends in a grid-wide barrier, so it is
+// launched without the programmatic-serialization attribute and lets its dependents go only behind that barrier.
+template <typename OutT, bool STATS, bool CG2, int EPI = 0, bool CLS4 = false>
 __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
-    static_assert(!CLS4 || (!HALO && !STATS && !EPI && !RES && !BRES), "four classes: the stride-2 data gradient only");
-    static_assert(!BRES || (!HALO && !STATS && !EPI && !RES), "the weights-stationary variant is instantiated for the data gradient only");
-    static_assert(!HALO || CG2, "the halo variant runs as CTA pairs");
-    static_assert(!RES || (STATS && !HALO && !EPI), "the resident variant is the forward kernel with statistics");
-    static_assert(!EPI || (!STATS && !HALO), "the fused per-channel epilogue is a forward-only variant without statistics");
+    static_assert(!CLS4 || (!STATS && !EPI), "four classes: the stride-2 data gradient only");
+    static_assert(!EPI || !STATS, "the fused per-channel epilogue is a forward-only variant without statistics");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
-    uint8_t* sB = sA + (HALO ? (size_t)p.a_slots * p.slab_bytes : (size_t)p.stages * p.a_stage_bytes);
-    // Weights-stationary variant (BRES; a template parameter because the same switch as a run-time flag cost every launch
-    // of this kernel about 1 %): the CTA's share of the whole filter stays in shared memory (p.a_slots groups of kpb
-    // k-blocks, fetched once, in the order of this CTA's K loop); the stage ring then holds A only.
-    constexpr bool bres = BRES;
-    uint8_t* stg = sB + (size_t)(bres ? p.a_slots : p.stages) * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
+    uint8_t* sB = sA + (size_t)p.stages * p.a_stage_bytes;
+    uint8_t* stg = sB + (size_t)p.stages * p.b_stage_bytes;  // staging: per epilogue team [128 rows][ncol_a columns] of OutT, row pitch ncol_a*2+16 bytes
     const int cw = p.stage_cw;  // columns per staging pass (<= 64)
     const int pitch = cw * 2 + 16;
     float* wstat = reinterpret_cast<float*>(stg + (size_t)2 * TC_BM * pitch);  // per team [4 warps][2][its columns of every n-tile]: warp-private channel sums
@@ -342,12 +290,12 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint64_t* tfull = empty + p.stages;   // [2]
     uint64_t* tempty = tfull + 2;         // [2]
     uint64_t* drain = tempty + 2;         // [1]
-    uint64_t* fullA = drain + 1;          // [4] halo mode: the slab ring has its own barriers
-    uint64_t* emptyA = fullA + 4;         // [4]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(emptyA + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    pdl_launch_dependents();
+    // A kernel that ends in a grid-wide barrier lets the next kernel of the stream start only once that barrier has been
+    // passed (see the epilogue); all others let it become resident and run its prologue right away.
+    if (!STATS) pdl_launch_dependents();
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // warp index in a form the compiler knows to be uniform
     const int total_tiles = p.nclasses * p.tiles_per_class;
     const int mh = p.mh;          // 128-row sub-tiles per tile (1 or 2); both share every B stage
@@ -358,7 +306,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(full + s, (HALO || bres) ? 1 : 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
+            ptx::mbar_init(full + s, 2);  // the A and the B producer arrive once each with their byte counts (pairs: rank 0's
                                           // producers announce the bytes of both CTAs, the peer only issues its loads)
             ptx::mbar_init(empty + s, 1);
         }
@@ -367,10 +315,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         ptx::mbar_init(tempty, CG2 ? 16 : 256);  // pairs: one arrival per epilogue warp of both CTAs
         ptx::mbar_init(tempty + 1, CG2 ? 16 : 256);
         ptx::mbar_init(drain, 1);
-        for (int s = 0; s < 4; ++s) {
-            ptx::mbar_init(fullA + s, 1);
-            ptx::mbar_init(emptyA + s, 1);
-        }
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -416,338 +360,94 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         // ------------------------------------------------------------------ TMA producers: warp 0 feeds A, warp 6 feeds B
         // Both producer warps run their loops converged; `leader` predicates the instructions that must be issued once.
         const uint32_t leader = ptx::elect_one() ? 1u : 0u;
-        if (HALO) {
-            {
-                const bool isA = warp == 0;
-                const int n_tiles = p.n_tiles, cbs = p.kc_per_tap, bn_own = p.BN / 2;
-                bool ok = true;
-                int issued = 0;
-                if (isA) {
-                    const int a_slots = p.a_slots, boxes = p.slab_boxes, box_pix = p.box_pix, Wp = p.Wp, HpWp = p.Hp * p.Wp;
-                    const uint32_t slab_bytes = p.slab_bytes, box_bytes = (uint32_t)box_pix * 128u;
-                    const uint32_t base_u32 = ptx::smem_u32(sA), fullA_local = ptx::smem_u32(fullA);
-                    const uint32_t fullA0 = ptx::mapa_u32(fullA_local, 0u);
-                    const int npos = (int)p.npos, rows_cta = TC_BM * mh;
-                    int sa = 0;
-                    uint32_t pha = 0;
-                    for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                        const int m_tile = tile / n_tiles;
-                        const int s0 = (m_tile * 2 + (int)rank) * rows_cta;  // first padded-raster position of this CTA's slab
-                        for (int cb = 0; cb < cbs; ++cb) {
-                            if (!wait_bar_fast(emptyA + sa, pha ^ 1u, abort_flag, p.status, 1)) {
-                                ok = false;
-                                break;
-                            }
-                            if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, fullA_local + 8u * (uint32_t)sa, 2u * slab_bytes);
-                            const uint32_t bar = fullA0 + 8u * (uint32_t)sa;
-                            uint32_t dst = base_u32 + (uint32_t)sa * slab_bytes;
-                            for (int b = 0; b < boxes; ++b) {
-                                // a box that would start past the last position feeds discarded rows only: fetch position 0 instead
-                                int q = s0 + b * box_pix;
-                                if (q >= npos) q = 0;
-                                const int n = q / HpWp, r = q - n * HpWp;
-                                const int hp = r / Wp, wp = r - hp * Wp;
-                                ptx::tma_load_im2col_4d_cg2_if(leader, dst, &p.tmA, bar, cb * 64, wp - 1, hp - 1, n, 0, 0);
-                                dst += box_bytes;
-                            }
-                            ++issued;
-                            if (++sa == a_slots) {
-                                sa = 0;
-                                pha ^= 1u;
-                            }
-                        }
-                    }
-                    if (!ok) {
-                        // gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited
-                        const int back = issued < a_slots ? issued : a_slots;
-                        for (int b = 0; b < back; ++b) {
-                            sa = (sa == 0) ? a_slots - 1 : sa - 1;
-                            if (sa == a_slots - 1) pha ^= 1u;
-                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(fullA + sa, pha); ++i) {
-                            }
-                        }
-                    }
-                } else {
-                    const int kpb = p.kpb, stages = p.stages, Ca = p.Ca, BN = p.BN, ntaps = p.cls_ntaps[0];
-                    const uint32_t b_sub = p.b_sub_bytes, stage_bytes = p.b_stage_bytes;
-                    const uint32_t tx = 2u * (uint32_t)kpb * (uint32_t)(bn_own * 128);
-                    const uint32_t base_u32 = ptx::smem_u32(sB), full_local = ptx::smem_u32(full);
-                    const uint32_t full0 = ptx::mapa_u32(full_local, 0u);
-                    int s = 0;
-                    uint32_t ph = 0;
-                    for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                        const int n_tile = tile % n_tiles;
-                        const int brow = n_tile * BN + (int)rank * bn_own;
-                        for (int cb = 0; ok && cb < cbs; ++cb) {
-                            for (int tap0 = 0; tap0 < ntaps; tap0 += kpb) {
-                                if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, 5)) {
-                                    ok = false;
-                                    break;
-                                }
-                                if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, full_local + 8u * (uint32_t)s, tx);
-                                const uint32_t bar = full0 + 8u * (uint32_t)s;
-                                uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
-                                for (int j = 0; j < kpb; ++j) {
-                                    ptx::tma_load_2d_cg2_if(leader, dst, &p.tmB[0], bar, (tap0 + j) * Ca + cb * 64, brow);
-                                    dst += b_sub;
-                                }
-                                ++issued;
-                                if (++s == stages) {
-                                    s = 0;
-                                    ph ^= 1u;
-                                }
-                            }
-                        }
-                    }
-                    if (!ok) {
-                        const int back = issued < stages ? issued : stages;
-                        for (int b = 0; b < back; ++b) {
-                            s = (s == 0) ? stages - 1 : s - 1;
-                            if (s == stages - 1) ph ^= 1u;
-                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
-                            }
-                        }
-                    }
-                }
+        const bool isA = warp == 0;
+        int s = 0;
+        uint32_t ph = 0;
+        long long issued = 0;
+        bool ok = true;
+        const int bn_own = CG2 ? p.BN / 2 : p.BN;  // rows of the B tile this CTA fetches
+        const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(bn_own * p.KC * 2);
+        // loop-invariant values in registers: this thread's instruction stream is on the critical path
+        const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
+        const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
+        const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes, sub_bytes = isA ? p.a_sub_bytes : p.b_sub_bytes;
+        // pairs: loads of both CTAs are counted on the rank-0 CTA's full barriers (the MMA issuer waits there)
+        const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB);
+        const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
+        for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
+            int cls, lt;
+            igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
+            const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
+            const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
+            const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
+            const int m0 = (CG2 ? m_tile * 2 + (int)rank : m_tile) * TC_BM * mh;
+            int cw0 = 0, ch0 = 0, n0 = 0;
+            if (isA && !a_tiled) {
+                const int j0 = m0 % Wq, t1 = m0 / Wq;
+                const int i0 = t1 % Hq;
+                n0 = t1 / Hq;
+                cw0 = p.lo_w + j0 * ts;
+                ch0 = p.lo_h + i0 * ts;
             }
-        } else {
-            const bool isA = warp == 0;
-            int s = 0;
-            uint32_t ph = 0;
-            long long issued = 0;
-            bool ok = true;
-#ifdef NB_TC_DEBUG_TIMING
-            long long dbg_wait_empty = 0;
-            const long long dbg_start = clock64();
-#endif
-            const int bn_own = CG2 ? p.BN / 2 : p.BN;  // rows of the B tile this CTA fetches
-            if (bres && !isA) {
-                // The whole filter share of this CTA, once: group i of the K loop (which starts at this worker's rotation)
-                // goes to slot i; the groups are announced in four chunks on fullA[0..3] (pairs: on rank 0's barriers, with
-                // the bytes of both CTAs) so that the first MMAs need not wait for the last group.
-                const int kc_per_tap = p.kc_per_tap, kpb = p.kpb, KC = p.KC, Ca = p.Ca;
-                const int kblocks = p.cls_ntaps[0] * kc_per_tap, groups = p.a_slots;
-                const uint32_t kb_bytes = (uint32_t)(bn_own * KC * 2);
-                const uint32_t fullA_local = ptx::smem_u32(fullA);
-                const uint32_t fullA_u32 = CG2 ? ptx::mapa_u32(fullA_local, 0u) : fullA_local;
-                if (worker < total_tiles) {
-                    const int brow = (CG2 ? (int)rank * bn_own : 0);  // one column tile
-                    const int rot = NB_TC_SWITCH(p, 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
-                    int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
-                    const int per_chunk = (groups + 3) / 4;
-                    uint32_t dst = ptx::smem_u32(sB);
-                    for (int g0 = 0; g0 < groups; g0 += per_chunk) {
-                        const int g1 = g0 + per_chunk < groups ? g0 + per_chunk : groups;
-                        const int kb_lo = g0 * kpb, kb_hi = g1 * kpb < kblocks ? g1 * kpb : kblocks;
-                        const uint32_t chunk = (uint32_t)(g0 / per_chunk);
-                        if (!CG2 || rank == 0) ptx::mbar_expect_tx_u32_if(leader, fullA_local + 8u * chunk, (CG2 ? 2u : 1u) * kb_bytes * (uint32_t)(kb_hi - kb_lo));
-                        const uint32_t bar = fullA_u32 + 8u * chunk;
-                        for (int g = g0; g < g1; ++g) {
-                            const int nkb = (kblocks - g * kpb < kpb) ? kblocks - g * kpb : kpb;
-                            uint32_t d = dst;
-                            for (int j = 0; j < nkb; ++j) {
-                                if (CG2) ptx::tma_load_2d_cg2_if(leader, d, &p.tmB[0], bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32_if(leader, d, &p.tmB[0], bar, tap * Ca + kc * KC, brow);
-                                d += p.b_sub_bytes;
-                                if (++kc == kc_per_tap) {
-                                    kc = 0;
-                                    if (++tap == p.cls_ntaps[0]) tap = 0;
-                                }
-                            }
-                            dst += p.b_stage_bytes;
-                        }
-                    }
-                    // nothing else to do: see the loads land (bounded) so that none is in flight when the CTA leaves early
-                    if (!CG2 || rank == 0)
-                        for (int c4 = 0; c4 * per_chunk < groups; ++c4)
-                            for (int i = 0; i < 100000 && !ptx::mbar_try_wait(fullA + c4, 0); ++i) {
-                            }
+            const int brow = n_tile * BN + (CG2 ? (int)rank * bn_own : 0);
+            // each CTA starts its K loop at a different k-block so that the CTAs do not all ask L2 for the same
+            // filter lines at the same moment
+            const int ntaps_c = p.cls_ntaps[cls];
+            const int rot = (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
+            int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
+            for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
+                const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
+                if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, isA ? 1 : 5)) {
+                    ok = false;
+                    break;
                 }
-            } else {
-            const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(bn_own * p.KC * 2);
-            // loop-invariant values in registers: this thread's instruction stream is on the critical path
-            const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
-            const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
-            const uint32_t stage_bytes = isA ? p.a_stage_bytes : p.b_stage_bytes, sub_bytes = isA ? p.a_sub_bytes : p.b_sub_bytes;
-            // pairs: loads of both CTAs are counted on the rank-0 CTA's full barriers (the MMA issuer waits there)
-            const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB);
-            const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
-            for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                int cls, lt;
-                igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
-                const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
-                const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
-                const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
-                const int m0 = (CG2 ? m_tile * 2 + (int)rank : m_tile) * TC_BM * mh;
-                int cw = 0, ch = 0, n0 = 0;
-                if (isA && !a_tiled) {
-                    const int j0 = m0 % Wq, t1 = m0 / Wq;
-                    const int i0 = t1 % Hq;
-                    n0 = t1 / Hq;
-                    cw = p.lo_w + j0 * ts;
-                    ch = p.lo_h + i0 * ts;
-                }
-                const int brow = n_tile * BN + (CG2 ? (int)rank * bn_own : 0);
-                // each CTA starts its K loop at a different k-block so that the CTAs do not all ask L2 for the same
-                // filter lines at the same moment
-                const int ntaps_c = p.cls_ntaps[cls];
-                const int rot = NB_TC_SWITCH(p, 4) ? 0 : (int)(((unsigned)worker * 7u) % (unsigned)kblocks);
-                int tap = rot / kc_per_tap, kc = rot - tap * kc_per_tap;
-                for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
-                    const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
-                    {
-                        NB_DBG_T0();
-                        if (!wait_bar_fast(empty + s, ph ^ 1u, abort_flag, p.status, isA ? 1 : 5)) {
-                            ok = false;
-                            break;
-                        }
-                        NB_DBG_ADD(dbg_wait_empty);
-                    }
-                    const uint32_t bar = full_u32 + 8u * (uint32_t)s;
-                    if (!CG2) ptx::mbar_expect_tx_u32_if(leader, bar, kb_bytes * (uint32_t)nkb);
-                    else if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
-                    uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
-                    for (int j = 0; j < nkb; ++j) {
-                        if (isA) {
-                            if (a_tiled) {
-                                if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, kc * KC, m0);
-                            } else {
-                                if (CG2)
-                                    ptx::tma_load_im2col_4d_cg2_if(leader, dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
-                                else
-                                    ptx::tma_load_im2col_4d_u32_if(leader, dst, tm, bar, kc * KC, cw, ch, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
-                            }
+                const uint32_t bar = full_u32 + 8u * (uint32_t)s;
+                if (!CG2) ptx::mbar_expect_tx_u32_if(leader, bar, kb_bytes * (uint32_t)nkb);
+                else if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
+                uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
+                for (int j = 0; j < nkb; ++j) {
+                    if (isA) {
+                        if (a_tiled) {
+                            if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, kc * KC, m0);
                         } else {
-                            if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow);
+                            if (CG2)
+                                ptx::tma_load_im2col_4d_cg2_if(leader, dst, tm, bar, kc * KC, cw0, ch0, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
+                            else
+                                ptx::tma_load_im2col_4d_u32_if(leader, dst, tm, bar, kc * KC, cw0, ch0, n0, p.off_w[cls][tap], p.off_h[cls][tap]);
                         }
-                        dst += sub_bytes;
-                        if (++kc == kc_per_tap) {
-                            kc = 0;
-                            if (++tap == ntaps_c) tap = 0;
-                        }
+                    } else {
+                        if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, tap * Ca + kc * KC, brow);
                     }
-                    ++issued;
-                    if (++s == stages) {
-                        s = 0;
-                        ph ^= 1u;
+                    dst += sub_bytes;
+                    if (++kc == kc_per_tap) {
+                        kc = 0;
+                        if (++tap == ntaps_c) tap = 0;
                     }
                 }
-            }
-#ifdef NB_TC_DEBUG_TIMING
-            if (p.dbg && isA && leader) { p.dbg[blockIdx.x * 8 + 0] = dbg_wait_empty; p.dbg[blockIdx.x * 8 + 1] = clock64() - dbg_start; }
-#endif
-            if (!ok) {
-                // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
-                const int back = issued < (long long)p.stages ? (int)issued : p.stages;
-                for (int b = 0; b < back; ++b) {
-                    s = (s == 0) ? p.stages - 1 : s - 1;
-                    if (s == p.stages - 1) ph ^= 1u;
-                    for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
-                    }
+                ++issued;
+                if (++s == stages) {
+                    s = 0;
+                    ph ^= 1u;
                 }
             }
+        }
+        if (!ok) {
+            // Gave up: wait (bounded) for the loads still in flight so that nothing lands after the CTA has exited.
+            const int back = issued < (long long)p.stages ? (int)issued : p.stages;
+            for (int b = 0; b < back; ++b) {
+                s = (s == 0) ? p.stages - 1 : s - 1;
+                if (s == p.stages - 1) ph ^= 1u;
+                for (int i = 0; i < 100000 && !ptx::mbar_try_wait(full + s, ph); ++i) {
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (one thread; in a pair only rank 0)
         const uint32_t leader = ptx::elect_one() ? 1u : 0u;  // the whole warp runs the loop, this lane issues
-        if (HALO) {
-            if (rank == 0) {
-                int s = 0, sa = 0, acc = 0;
-                uint32_t ph = 0, pha = 0, acc_ph = 0;
-                bool ok = true;
-#ifdef NB_TC_DEBUG_TIMING
-                long long dbg_wait_full = 0, dbg_wait_tempty = 0;
-                const long long dbg_start = clock64();
-#endif
-                const int kpb = p.kpb, stages = p.stages, a_slots = p.a_slots, cbs = p.kc_per_tap, ntaps = p.cls_ntaps[0];
-                const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
-                const uint64_t b_sub16 = (uint64_t)(p.b_sub_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
-                const uint64_t slab16 = (uint64_t)(p.slab_bytes >> 4);
-                const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), 16, 1024, ptx::kSwizzle128);
-                const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, 1024, ptx::kSwizzle128);
-                const uint32_t empty_u32 = ptx::smem_u32(empty), emptyA_u32 = ptx::smem_u32(emptyA), tfull_u32 = ptx::smem_u32(tfull);
-                for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
-                    {
-                        NB_DBG_T0();
-                        if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
-                        NB_DBG_ADD(dbg_wait_tempty);
-                    }
-                    ptx::tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
-                    uint32_t accumulate = 0;
-                    for (int cb = 0; ok && cb < cbs; ++cb) {
-                        {
-                            NB_DBG_T0();
-                            if (!wait_bar_fast(fullA + sa, pha, abort_flag, p.status, 6)) {
-                                ok = false;
-                                break;
-                            }
-                            NB_DBG_ADD(dbg_wait_full);
-                        }
-                        ptx::tc_fence_after();
-                        const uint64_t da_slab = da0 + (uint64_t)sa * slab16;
-                        for (int tap0 = 0; tap0 < ntaps; tap0 += kpb) {
-                            {
-                                NB_DBG_T0();
-                                if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
-                                    ok = false;
-                                    break;
-                                }
-                                NB_DBG_ADD(dbg_wait_full);
-                            }
-                            ptx::tc_fence_after();
-                            uint64_t db = db0 + (uint64_t)s * b_stage16;
-                            for (int j = 0; j < kpb; ++j) {
-                                const uint64_t da_tap = da_slab + (uint64_t)p.tap_off16[tap0 + j];
-                                for (int h = 0; h < mh; ++h) {
-                                    const uint64_t dah = da_tap + (uint64_t)h * (uint64_t)((TC_BM * 128) >> 4);
-                                    // the rows of a tap start anywhere inside an 8-row swizzle group; the pattern itself stays
-                                    // anchored at 1024-byte boundaries of shared memory, where TMA put it, so the descriptor's
-                                    // base-offset field stays zero (measured: setting it to the row phase gives wrong sums)
-                                    const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
-                                    ptx::umma_f16_cg2_if(leader, dt, dah, db, idesc, accumulate);
-                                    ptx::umma_f16_cg2_if(leader, dt, dah + 2, db + 2, idesc, 1u);
-                                    ptx::umma_f16_cg2_if(leader, dt, dah + 4, db + 4, idesc, 1u);
-                                    ptx::umma_f16_cg2_if(leader, dt, dah + 6, db + 6, idesc, 1u);
-                                }
-                                accumulate = 1u;
-                                db += b_sub16;
-                            }
-                            ptx::umma_commit_cg2_mc_if(leader, empty_u32 + 8u * (uint32_t)s, 3);
-                            if (++s == stages) {
-                                s = 0;
-                                ph ^= 1u;
-                            }
-                        }
-                        if (!ok) break;
-                        ptx::umma_commit_cg2_mc_if(leader, emptyA_u32 + 8u * (uint32_t)sa, 3);
-                        if (++sa == a_slots) {
-                            sa = 0;
-                            pha ^= 1u;
-                        }
-                    }
-                    if (!ok) break;
-                    ptx::umma_commit_cg2_mc_if(leader, tfull_u32 + 8u * (uint32_t)acc, 3);
-                    if (++acc == nbuf) {
-                        acc = 0;
-                        acc_ph ^= 1u;
-                    }
-                }
-#ifdef NB_TC_DEBUG_TIMING
-                if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; }
-#endif
-                ptx::umma_commit_cg2_if(leader, ptx::smem_u32(drain));
-                for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
-                }
-            }
-        } else if (rank == 0) {
+        if (rank == 0) {
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
-#ifdef NB_TC_DEBUG_TIMING
-            long long dbg_wait_full = 0, dbg_wait_tempty = 0, dbg_wait_first = 0;
-            const long long dbg_start = clock64();
-#endif
             const int ksteps = p.KC / 16, kpb = p.kpb, stages = p.stages;
             const uint32_t idesc = p.idesc, acc_stride = (uint32_t)p.acc_stride;
             const uint64_t a_sub16 = (uint64_t)(p.a_sub_bytes >> 4), b_sub16 = (uint64_t)(p.b_sub_bytes >> 4);
@@ -759,44 +459,19 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             uint64_t da_s = da0, db_s = db0;  // descriptors of the current stage
             const int kc_per_tap = p.kc_per_tap;
             const uint32_t tfull_u32 = ptx::smem_u32(tfull);
-            const int b_per_chunk = bres ? (p.a_slots + 3) / 4 : 1;  // weights-stationary: groups per announced chunk
             for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
                 int cls_mma, lt_mma;
                 igemm_tile_class<CLS4>(p, tile, nworkers, cls_mma, lt_mma);
                 const int kblocks = p.cls_ntaps[cls_mma] * kc_per_tap;
-                {
-                    NB_DBG_T0();
-                    if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
-                    NB_DBG_ADD(dbg_wait_tempty);
-                }
+                if (!wait_bar_fast(tempty + acc, acc_ph ^ 1u, abort_flag, p.status, 2)) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
                 uint32_t accumulate = 0;
-                const bool b_first = tile == worker;  // weights-stationary: the filter groups arrive during the first tile
-                int b_grp = 0, b_next = 0, b_chunk = 0;
-                uint64_t db_res = db0;
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
-                    {
-                        NB_DBG_T0();
-                        if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
-                            ok = false;
-                            break;
-                        }
-                        if (kb0 == 0) { NB_DBG_ADD(dbg_wait_first); } else { NB_DBG_ADD(dbg_wait_full); }
-                    }
-                    if (bres) {  // (counters instead of divisions: this loop is the critical instruction stream)
-                        if (b_first && b_grp == b_next) {
-                            if (!wait_bar_fast(fullA + b_chunk, 0u, abort_flag, p.status, 7)) {
-                                ok = false;
-                                break;
-                            }
-                            ++b_chunk;
-                            b_next += b_per_chunk;
-                        }
-                        ++b_grp;
-                        db_s = db_res;
-                        db_res += b_stage16;
+                    if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
+                        ok = false;
+                        break;
                     }
                     ptx::tc_fence_after();
                     uint64_t da = da_s, db = db_s;
@@ -840,9 +515,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     acc_ph ^= 1u;
                 }
             }
-#ifdef NB_TC_DEBUG_TIMING
-            if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 2] = dbg_wait_full; p.dbg[blockIdx.x * 8 + 3] = dbg_wait_tempty; p.dbg[blockIdx.x * 8 + 4] = clock64() - dbg_start; p.dbg[blockIdx.x * 8 + 7] = dbg_wait_first; }
-#endif
             // Make sure every MMA issued by this thread has retired before TMEM is released.
             if (CG2) ptx::umma_commit_cg2_if(leader, ptx::smem_u32(drain)); else ptx::umma_commit_u32_if(leader, ptx::smem_u32(drain));
             for (int i = 0; i < 4000000 && !ptx::mbar_try_wait(drain, 0); ++i) {
@@ -856,7 +528,6 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         // nearly halves the time per tile.
         const int team = warp >= 7 ? 1 : 0;
         const int lane_group = warp & 3;          // TMEM lanes this warp may read: rows [32*lane_group, +32) of a sub-tile
-        const int row = lane_group * 32 + lane;   // accumulator row == sub-tile row
         const int c_lo = team ? p.ncol_a : 0;     // first column (within the tile) and number of columns of this team
         const int ncol = team ? p.BN - p.ncol_a : p.ncol_a;
         const int st_ld = p.n_tiles * ncol;       // row length of this team's running sums: its columns of every n-tile
@@ -864,31 +535,25 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         uint32_t acc_ph = 0;
         float* team_stat = wstat + (team ? (size_t)8 * p.n_tiles * p.ncol_a : 0);  // [4 warps][2][st_ld]
         float* my_stat = team_stat + (size_t)lane_group * 2 * st_ld;
-        const bool tma_out = !HALO && p.tma_store != 0;
+        const bool tma_out = p.tma_store != 0;  // (always set for the STATS and EPI variants)
         // staging of this warp's 32 rows: padded rows for the store loop, dense rows (the TMA box) for TMA stores
         uint8_t* stg_t = stg + (size_t)team * TC_BM * pitch;
         uint8_t* const wrows = tma_out ? stg + (size_t)((team * 4 + lane_group) * 32) * (cw * 2) : stg_t + (size_t)(lane_group * 32) * pitch;
         bool store_pending = false;
         uint8_t* outb = static_cast<uint8_t*>(p.out);
-#ifdef NB_TC_DEBUG_TIMING
-        long long dbg_wait_tfull = 0, dbg_ld = 0, dbg_pack = 0, dbg_stats = 0, dbg_store = 0, dbg_ph__ = 0;
-        const long long dbg_start = clock64();
-#endif
         const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
         for (int tile = worker; tile < total_tiles; tile += nworkers) {
             int cls, lt;
             igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
             const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
-            NB_DBG_T0();
             bool ok = true;
             // one poller per warp: 256 threads spinning on one mbarrier would crowd the shared-memory pipe
             if (lane == 0) ok = wait_bar(tfull + acc, acc_ph, abort_flag, p.status, 4);
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            NB_DBG_ADD(dbg_wait_tfull);
             ok = epi2_bar_and(ok);
             if (!ok) break;
             ptx::tc_fence_after();
-            if (NB_TC_SWITCH(p, 8) || ncol == 0) {
+            auto release_acc = [&]() {  // this warp is done reading the tile's accumulators
                 ptx::tc_fence_before();
                 if (CG2) {
                     __syncwarp();
@@ -896,6 +561,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 } else {
                     ptx::mbar_arrive(tempty + acc);
                 }
+            };
+            if (ncol == 0) {
+                release_acc();
                 if (++acc == nbuf) {
                     acc = 0;
                     acc_ph ^= 1u;
@@ -905,206 +573,120 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             for (int h = 0; h < mh; ++h) {
                 const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
                 const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc * mh + h) * p.acc_stride) + (uint32_t)c_lo;
-                long long halo_pix = -1;  // halo mode: output pixel of this thread's row, -1 on the padding ring / past the end
-                if (HALO) {
-                    const long long pos = m0 + row + p.Wp + 1;  // output tiles start one padded row and one pixel in
-                    if (pos < p.npos) {
-                        const int HpWp = p.Hp * p.Wp;
-                        const int n = (int)(pos / HpWp), r = (int)(pos - (long long)n * HpWp);
-                        const int hp = r / p.Wp, wp = r - hp * p.Wp;
-                        if (hp >= 1 && hp <= p.Hin && wp >= 1 && wp <= p.Win) halo_pix = ((long long)n * p.Hin + (hp - 1)) * p.Win + (wp - 1);
-                    }
-                }
                 // The team's columns go through the staging buffer in passes of at most cw (<= 64) columns.
                 for (int cb = 0; cb < ncol; cb += cw) {
-                const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
-                if (tma_out && !NB_TC_SWITCH(p, (16 | 32))) {
-                    const bool last = h == mh - 1 && cb + cw >= ncol;  // last TMEM read of this tile: the accumulator set becomes free
-                    auto release = [&]() {
-                        if (last) {
-                            ptx::tc_fence_before();
-                            if (CG2) {
-                                __syncwarp();
-                                if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
-                            } else {
-                                ptx::mbar_arrive(tempty + acc);
-                            }
-                        }
-                    };
-                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut[0] : npass == p.out_w[1] ? &p.tmOut[1] : &p.tmOut[2];
-                    const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
-                    float* ss = my_stat + n_tile * ncol + cb;
-                    float* sq = ss + st_ld;
-                    const uint32_t ta = taddr + (uint32_t)cb;
-                    const float2* cf = reinterpret_cast<const float2*>(wstat) + col;  // read only by the EPI variant
-                    if (npass == 64) epi_pass_tma<OutT, STATS, 64, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                    else if (npass == 48) epi_pass_tma<OutT, STATS, 48, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                    else if (npass == 32) epi_pass_tma<OutT, STATS, 32, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                    else epi_pass_tma<OutT, STATS, 16, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                    continue;
-                }
-                const int rpitch = tma_out ? npass * 2 : pitch;       // bytes between staged rows of this pass
-                const bool swz = tma_out && npass == 64;              // 128-byte rows: 16-byte chunk j of row r sits at j ^ (r & 7)
-                uint8_t* const my_row = wrows + (size_t)lane * rpitch;
-                const uint8_t* const my_rows = wrows;
-                // ---- TMEM -> registers -> staging (this thread's row); up to four 16-column loads are in flight before the
-                // one wait: a TMEM load has a long latency
-                {
-                    uint32_t r[64];
-                    const int nld = npass / 16;
-#ifdef NB_TC_DEBUG_TIMING
-                    dbg_ph__ = clock64();
-#endif
-#pragma unroll
-                    for (int hh = 0; hh < 4; ++hh)
-                        if (hh < nld) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cb + 16 * hh), r + 16 * hh);
-                    ptx::tmem_ld_wait();
-                    NB_DBG_PHASE(dbg_ld);
-                    if (store_pending) {  // the previous TMA store must have read the staging rows before they are overwritten
-                        if (lane == 0) ptx::tma_store_wait_read<0>();
-                        __syncwarp();
-                        store_pending = false;
-                    }
-                    int sat_bits = 0;
-#pragma unroll
-                    for (int hh = 0; hh < 4; ++hh) {
-                        if (hh >= nld) break;
-                        uint4 v0, v1;
-                        const uint32_t* q = r + 16 * hh;
-                        v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat_bits);
-                        v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat_bits);
-                        v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat_bits);
-                        v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat_bits);
-                        v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat_bits);
-                        v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat_bits);
-                        v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat_bits);
-                        v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat_bits);
-                        if (HALO && halo_pix < 0) {  // discarded row: zeros keep the channel sums exact
-                            v0 = v1 = make_uint4(0u, 0u, 0u, 0u);
-                            sat_bits = 0;
-                        }
-                        const int j0 = swz ? ((2 * hh) ^ (lane & 7)) : 2 * hh, j1 = swz ? ((2 * hh + 1) ^ (lane & 7)) : 2 * hh + 1;
-                        *reinterpret_cast<uint4*>(my_row + j0 * 16) = v0;
-                        *reinterpret_cast<uint4*>(my_row + j1 * 16) = v1;
-                    }
-                    if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
-                }
-                if (h == mh - 1 && cb + cw >= ncol) {
-                    // last TMEM read of this tile: the accumulator set is free for the MMAs of a later tile
-                    ptx::tc_fence_before();
-                    if (CG2) {
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_cluster(tempty_u32 + 8u * (uint32_t)acc);
-                    } else {
-                        ptx::mbar_arrive(tempty + acc);
-                    }
-                }
-                if (tma_out) {
-                    // hand the staged rows to TMA: writes made visible to the async proxy, then one lane issues the store
-                    ptx::fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
+                    const int npass = (ncol - cb < cw) ? ncol - cb : cw;  // multiple of 16
+                    const bool last = h == mh - 1 && cb + cw >= ncol;    // last TMEM read of this tile: the accumulator set becomes free
+                    if (tma_out) {
+                        auto release = [&]() {
+                            if (last) release_acc();
+                        };
                         const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmOut[0] : npass == p.out_w[1] ? &p.tmOut[1] : &p.tmOut[2];
-                        ptx::tma_store_2d(tm, wrows, n_tile * p.BN + c_lo + cb, (int)(m0 + lane_group * 32));
-                        ptx::tma_store_commit();
+                        const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
+                        float* ss = my_stat + n_tile * ncol + cb;
+                        float* sq = ss + st_ld;
+                        const uint32_t ta = taddr + (uint32_t)cb;
+                        const float2* cf = reinterpret_cast<const float2*>(wstat) + col;  // read only by the EPI variant
+                        if (npass == 64) epi_pass_tma<OutT, STATS, 64, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                        else if (npass == 48) epi_pass_tma<OutT, STATS, 48, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                        else if (npass == 32) epi_pass_tma<OutT, STATS, 32, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                        else epi_pass_tma<OutT, STATS, 16, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                        continue;
                     }
-                    store_pending = true;
-                } else {
+                    // ---- output rows that are not GEMM rows (the parity classes of a stride-2 data gradient): padded staging
+                    // rows and a coalesced store loop.  TMEM -> registers -> staging (this thread's row); up to four
+                    // 16-column loads are in flight before the one wait: a TMEM load has a long latency
+                    uint8_t* const my_row = wrows + (size_t)lane * pitch;
+                    {
+                        uint32_t r[64];
+                        const int nld = npass / 16;
+#pragma unroll
+                        for (int hh = 0; hh < 4; ++hh)
+                            if (hh < nld) ptx::tmem_ld_32x32b_x16(taddr + (uint32_t)(cb + 16 * hh), r + 16 * hh);
+                        ptx::tmem_ld_wait();
+                        int sat_bits = 0;
+#pragma unroll
+                        for (int hh = 0; hh < 4; ++hh) {
+                            if (hh >= nld) break;
+                            uint4 v0, v1;
+                            const uint32_t* q = r + 16 * hh;
+                            v0.x = pack2<OutT>(__uint_as_float(q[0]), __uint_as_float(q[1]), &sat_bits);
+                            v0.y = pack2<OutT>(__uint_as_float(q[2]), __uint_as_float(q[3]), &sat_bits);
+                            v0.z = pack2<OutT>(__uint_as_float(q[4]), __uint_as_float(q[5]), &sat_bits);
+                            v0.w = pack2<OutT>(__uint_as_float(q[6]), __uint_as_float(q[7]), &sat_bits);
+                            v1.x = pack2<OutT>(__uint_as_float(q[8]), __uint_as_float(q[9]), &sat_bits);
+                            v1.y = pack2<OutT>(__uint_as_float(q[10]), __uint_as_float(q[11]), &sat_bits);
+                            v1.z = pack2<OutT>(__uint_as_float(q[12]), __uint_as_float(q[13]), &sat_bits);
+                            v1.w = pack2<OutT>(__uint_as_float(q[14]), __uint_as_float(q[15]), &sat_bits);
+                            *reinterpret_cast<uint4*>(my_row + (2 * hh) * 16) = v0;
+                            *reinterpret_cast<uint4*>(my_row + (2 * hh + 1) * 16) = v1;
+                        }
+                        if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
+                    }
+                    if (last) release_acc();
                     __syncwarp();  // every warp only reads back the 32 rows it staged itself
-                }
-                NB_DBG_PHASE(dbg_pack);
-                if (STATS && !NB_TC_SWITCH(p, 16)) {
-                    // per-channel sums over this warp's 32 rows (rows past M hold zeros: their A rows were zero-filled),
-                    // accumulated into the warp's private running sums: no cross-warp traffic until the kernel ends.
-                    // A lane owns two adjacent channels (a pass has at most 64), two rows per step for independent chains.
-                    if (lane < npass / 2) {
-                        float2 sa = make_float2(0.f, 0.f), sb = sa, qa = sa, qb = sa;
-                        const int cj = lane >> 2, cw4 = (lane & 3) * 4;  // 16-byte chunk and offset inside it of this lane's channels
-#pragma unroll 8
-                        for (int rr = 0; rr < 32; rr += 2) {
-                            const int ja = swz ? (cj ^ (rr & 7)) : cj, jb = swz ? (cj ^ ((rr + 1) & 7)) : cj;
-                            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(my_rows + (size_t)rr * rpitch + ja * 16 + cw4));
-                            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(my_rows + (size_t)(rr + 1) * rpitch + jb * 16 + cw4));
-                            sa.x += f0.x; sa.y += f0.y;
-                            sb.x += f1.x; sb.y += f1.y;
-                            qa.x = fmaf(f0.x, f0.x, qa.x); qa.y = fmaf(f0.y, f0.y, qa.y);
-                            qb.x = fmaf(f1.x, f1.x, qb.x); qb.y = fmaf(f1.y, f1.y, qb.y);
+                    // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
+                    // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
+                    // output offset of row r, the others fetch it by shuffle
+                    {
+                        const int cpr = npass / 8;  // 16-byte pieces per staged row (<= 8)
+                        long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
+                        if (pixrow >= p.M) {
+                            pixrow = -1;
+                        } else if (p.os != 1) {
+                            const int j = (int)(pixrow % p.Wq);
+                            const long long t1 = pixrow / p.Wq;
+                            const int i = (int)(t1 % p.Hq);
+                            const long long n = t1 / p.Hq;
+                            pixrow = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
                         }
-                        float2* ps = reinterpret_cast<float2*>(my_stat + n_tile * ncol + cb + 2 * lane);
-                        float2* pq = reinterpret_cast<float2*>(my_stat + st_ld + n_tile * ncol + cb + 2 * lane);
-                        float2 a2 = *ps, b2 = *pq;
-                        a2.x += sa.x + sb.x; a2.y += sa.y + sb.y;
-                        b2.x += qa.x + qb.x; b2.y += qa.y + qb.y;
-                        *ps = a2;
-                        *pq = b2;
-                    }
-                }
-                NB_DBG_PHASE(dbg_stats);
-                // ---- coalesced stores: the warp walks its 32 staged rows as one flat sequence of 16-byte pieces
-                // (32 rows x cpr pieces = cpr iterations of 32 lanes, every lane busy); lane r first works out the
-                // output offset of row r, the others fetch it by shuffle
-                if (!tma_out && !NB_TC_SWITCH(p, 32)) {
-                    const int cpr = npass / 8;  // 16-byte pieces per staged row (<= 8)
-                    long long pixrow = m0 + lane_group * 32 + lane;  // GEMM row of staged row `lane`
-                    if (HALO) {
-                        pixrow = halo_pix;
-                    } else if (pixrow >= p.M) {
-                        pixrow = -1;
-                    } else if (p.os != 1) {
-                        const int j = (int)(pixrow % p.Wq);
-                        const long long t1 = pixrow / p.Wq;
-                        const int i = (int)(t1 % p.Hq);
-                        const long long n = t1 / p.Hq;
-                        pixrow = (n * p.Hout + (long long)i * p.os + p.cls_oa[cls]) * p.Wout + (long long)j * p.os + p.cls_ob[cls];
-                    }
-                    // byte offset of staged row `lane` in the output (-1: not stored); pieces are handled four (or two) at
-                    // a time so that their shuffle -> shared load -> global store chains overlap
-                    const long long rowbyte = pixrow < 0 ? -1 : pixrow * (long long)(p.ldo * 2) + (n_tile * p.BN + c_lo + cb) * 2;
-                    const int step_r = 32 / cpr, step_c = 32 - step_r * cpr;
-                    int rr = lane / cpr, cc = lane - rr * cpr;
-                    auto advance = [&](int& r_, int& c_) {
-                        r_ += step_r;
-                        c_ += step_c;
-                        if (c_ >= cpr) {
-                            c_ -= cpr;
-                            ++r_;
+                        // byte offset of staged row `lane` in the output (-1: not stored); pieces are handled four (or two) at
+                        // a time so that their shuffle -> shared load -> global store chains overlap
+                        const long long rowbyte = pixrow < 0 ? -1 : pixrow * (long long)(p.ldo * 2) + (n_tile * p.BN + c_lo + cb) * 2;
+                        const int step_r = 32 / cpr, step_c = 32 - step_r * cpr;
+                        int rr = lane / cpr, cc = lane - rr * cpr;
+                        auto advance = [&](int& r_, int& c_) {
+                            r_ += step_r;
+                            c_ += step_c;
+                            if (c_ >= cpr) {
+                                c_ -= cpr;
+                                ++r_;
+                            }
+                        };
+                        int it = 0;
+                        for (; it + 4 <= cpr; it += 4) {
+                            int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
+                            advance(r1, c1);
+                            int r2 = r1, c2 = c1;
+                            advance(r2, c2);
+                            int r3 = r2, c3 = c2;
+                            advance(r3, c3);
+                            rr = r3; cc = c3;
+                            advance(rr, cc);
+                            const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
+                            const long long o2 = __shfl_sync(0xffffffffu, rowbyte, r2), o3 = __shfl_sync(0xffffffffu, rowbyte, r3);
+                            const uint4 v0 = *reinterpret_cast<const uint4*>(wrows + r0 * pitch + c0 * 16);
+                            const uint4 v1 = *reinterpret_cast<const uint4*>(wrows + r1 * pitch + c1 * 16);
+                            const uint4 v2 = *reinterpret_cast<const uint4*>(wrows + r2 * pitch + c2 * 16);
+                            const uint4 v3 = *reinterpret_cast<const uint4*>(wrows + r3 * pitch + c3 * 16);
+                            if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
+                            if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
+                            if (o2 >= 0) *reinterpret_cast<uint4*>(outb + o2 + c2 * 16) = v2;
+                            if (o3 >= 0) *reinterpret_cast<uint4*>(outb + o3 + c3 * 16) = v3;
                         }
-                    };
-                    int it = 0;
-                    for (; it + 4 <= cpr; it += 4) {
-                        int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
-                        advance(r1, c1);
-                        int r2 = r1, c2 = c1;
-                        advance(r2, c2);
-                        int r3 = r2, c3 = c2;
-                        advance(r3, c3);
-                        rr = r3; cc = c3;
-                        advance(rr, cc);
-                        const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
-                        const long long o2 = __shfl_sync(0xffffffffu, rowbyte, r2), o3 = __shfl_sync(0xffffffffu, rowbyte, r3);
-                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * rpitch + c0 * 16);
-                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * rpitch + c1 * 16);
-                        const uint4 v2 = *reinterpret_cast<const uint4*>(my_rows + r2 * rpitch + c2 * 16);
-                        const uint4 v3 = *reinterpret_cast<const uint4*>(my_rows + r3 * rpitch + c3 * 16);
-                        if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
-                        if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
-                        if (o2 >= 0) *reinterpret_cast<uint4*>(outb + o2 + c2 * 16) = v2;
-                        if (o3 >= 0) *reinterpret_cast<uint4*>(outb + o3 + c3 * 16) = v3;
+                        for (; it < cpr; it += 2) {  // cpr is even
+                            int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
+                            advance(r1, c1);
+                            rr = r1; cc = c1;
+                            advance(rr, cc);
+                            const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
+                            const uint4 v0 = *reinterpret_cast<const uint4*>(wrows + r0 * pitch + c0 * 16);
+                            const uint4 v1 = *reinterpret_cast<const uint4*>(wrows + r1 * pitch + c1 * 16);
+                            if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
+                            if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
+                        }
                     }
-                    for (; it < cpr; it += 2) {  // cpr is even
-                        int r0 = rr, c0 = cc, r1 = r0, c1 = c0;
-                        advance(r1, c1);
-                        rr = r1; cc = c1;
-                        advance(rr, cc);
-                        const long long o0 = __shfl_sync(0xffffffffu, rowbyte, r0), o1 = __shfl_sync(0xffffffffu, rowbyte, r1);
-                        const uint4 v0 = *reinterpret_cast<const uint4*>(my_rows + r0 * rpitch + c0 * 16);
-                        const uint4 v1 = *reinterpret_cast<const uint4*>(my_rows + r1 * rpitch + c1 * 16);
-                        if (o0 >= 0) *reinterpret_cast<uint4*>(outb + o0 + c0 * 16) = v0;
-                        if (o1 >= 0) *reinterpret_cast<uint4*>(outb + o1 + c1 * 16) = v1;
-                    }
-                }
-                __syncwarp();  // staged rows consumed before the next pass overwrites them
-                NB_DBG_PHASE(dbg_store);
+                    __syncwarp();  // staged rows consumed before the next pass overwrites them
                 }
             }
             if (++acc == nbuf) {
@@ -1133,69 +715,25 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 int* ctr = p.status + ST_BAR_FWD;
                 volatile int* fin_ok = abort_flag + 1;  // (the kernel uses all of the opt-in shared memory as dynamic: no static variables)
                 epi2_bar_sync();  // this CTA's partial sums are written
-                if (et == 0) *fin_ok = grid_arrive_wait(ctr, (int)gridDim.x) ? 1 : 0;
+                if (et == 0) *fin_ok = grid_arrive_wait(ctr, (int)gridDim.x + p.bar_extra, wait_limit_ns(p.wait_limit_ms)) ? 1 : 0;
                 epi2_bar_sync();
+                // Every CTA of this grid is resident and past the barrier: only now may the next kernel of the stream take
+                // SM resources (before the barrier its CTAs could have kept CTAs of this grid from becoming resident).
+                pdl_launch_dependents();
                 if (*fin_ok) {
                     const int ew = et >> 5;
                     for (int c = (int)blockIdx.x + (int)gridDim.x * ew; c < p.ldo; c += (int)gridDim.x * 8)
                         bn_finalize_channel<true>(p.partials, (int)gridDim.x, p.ldo, c, lane, p.fin_count, p.fin_eps, p.fin_momentum, p.fin_gamma, p.fin_beta,
                                                   p.fin_mean, p.fin_invstd, p.fin_scale, p.fin_shift, p.fin_rmean, p.fin_rvar, nullptr, nullptr);
-                } else if (et == 0 && atomicCAS(p.status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
-                    p.status[ST_WHERE] = 20;
-                    p.status[ST_DETAIL] = (int)blockIdx.x;
+                } else if (et == 0) {
+                    report_timeout(p.status, SITE_GRID_BARRIER_FWD, (int)blockIdx.x);
                 }
                 epi2_bar_sync();  // every warp is past its reads of the partial sums
                 if (et == 0) grid_depart(ctr, (int)gridDim.x);
-                if (RES) {
-                    // ---- second barrier: every channel's scale and shift is in global memory; then the second pass
-                    int* ctr2 = p.status + ST_BAR_FWD2;
-                    if (et == 0) *fin_ok = (*fin_ok && grid_arrive_wait(ctr2, (int)gridDim.x)) ? 1 : 0;
-                    epi2_bar_sync();
-                    if (*fin_ok) {
-                        float2* coef = reinterpret_cast<float2*>(wstat);  // the channel sums are flushed: reuse their space
-                        for (int c = et; c < p.ldo; c += 256) {  // per channel pair: scale, scale, shift, shift
-                            wstat[4 * (c >> 1) + (c & 1)] = __ldcg(p.fin_scale + c);
-                            wstat[4 * (c >> 1) + 2 + (c & 1)] = __ldcg(p.fin_shift + c);
-                        }
-                        epi2_bar_sync();
-                        int acc2 = 0;
-                        auto no_release = []() {};
-                        for (int tile = worker; tile < total_tiles; tile += nworkers, ++acc2) {
-                            const int lt = tile % p.tiles_per_class;
-                            const int m_tile = lt / p.n_tiles, n_tile = lt % p.n_tiles;
-                            for (int h = 0; h < mh; ++h) {
-                                const long long m0 = (((CG2 ? (long long)m_tile * 2 + rank : (long long)m_tile)) * mh + h) * TC_BM;
-                                const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)((acc2 * mh + h) * p.acc_stride) + (uint32_t)c_lo;
-                                for (int cb = 0; cb < ncol; cb += cw) {
-                                    const int npass = (ncol - cb < cw) ? ncol - cb : cw;
-                                    const CUtensorMap* tm = npass == p.out_w[0] ? &p.tmB[1] : npass == p.out_w[1] ? &p.tmB[2] : &p.tmB[3];
-                                    const int col = n_tile * p.BN + c_lo + cb, grow = (int)(m0 + lane_group * 32);
-                                    const uint32_t ta = taddr + (uint32_t)cb;
-                                    int sat2 = 0;
-                                    if (npass == 64) epi_pass_tma<__nv_bfloat16, false, 64, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
-                                    else if (npass == 48) epi_pass_tma<__nv_bfloat16, false, 48, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
-                                    else if (npass == 32) epi_pass_tma<__nv_bfloat16, false, 32, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
-                                    else epi_pass_tma<__nv_bfloat16, false, 16, 2>(ta, wrows, lane, store_pending, sat2, tm, col, grow, nullptr, nullptr, coef + col, 1, no_release);
-                                }
-                            }
-                        }
-                        if (store_pending && lane == 0) ptx::tma_store_wait_read<0>();
-                    } else if (et == 0 && atomicCAS(p.status + ST_ERR, 0, (int)NB_ERR_TIMEOUT) == 0) {
-                        p.status[ST_WHERE] = 22;
-                        p.status[ST_DETAIL] = (int)blockIdx.x;
-                    }
-                    epi2_bar_sync();
-                    if (et == 0) grid_depart(ctr2, (int)gridDim.x);
-                }
+            } else {
+                pdl_launch_dependents();
             }
         }
-#ifdef NB_TC_DEBUG_TIMING
-        if (p.dbg && warp == 2 && lane == 0) {
-            p.dbg[blockIdx.x * 8 + 5] = dbg_wait_tfull; p.dbg[blockIdx.x * 8 + 6] = clock64() - dbg_start;
-            long long* ph = p.dbg + (size_t)gridDim.x * 8 + blockIdx.x * 4;
-            ph[0] = dbg_ld; ph[1] = dbg_pack; ph[2] = dbg_stats; ph[3] = dbg_store;
-        }
-#endif
         if (sat) atomicAdd(p.status + ST_SAT, sat);
     }
     ptx::tc_fence_before();
@@ -1205,6 +743,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         if (CG2) ptx::tmem_dealloc_cg2(tmem_base, (uint32_t)p.tmem_cols); else ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
+
 
 
 }  // namespace nbcbs
@@ -1217,12 +756,6 @@ struct IgemmCfg {
     int Ca = 0, rowsB = 0, ntaps = 0;
     int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
     bool cg2 = false;  // CTA pairs (tcgen05 cta_group::2)
-    bool halo = false;  // tap-reuse variant (3x3, stride 1)
-    bool bres = false;  // weights-stationary: the CTA's share of the filter is fetched once (b_groups groups of kpb k-blocks)
-    int b_groups = 0;
-    int Wp = 0, Hp = 0, Hin = 0, Win = 0, Nimg = 0, slab_boxes = 0, box_pix = 0, a_slots = 0;
-    uint32_t slab_bytes = 0;
-    long long npos = 0;
     uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
@@ -1240,9 +773,7 @@ struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
     bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
     long long ld_x = 0;        // row pitch (elements) of the input activation when it is a channel slice of a wider tensor (0 = dense)
-    bool fp_resident = false;  // forward: every CTA keeps all its accumulators in TMEM (tiles per CTA <= accumulator sets): BN + SiLU applied in the same kernel
-    const void* res_out_ptr = nullptr;
-    bool tma_store = true;  // epilogues store through TMA where the layout allows (NB_TC_TMA_STORE=0 at plan creation: coalesced stores instead)
+    bool fp_barrier_ok = false;  // the forward launch's whole grid fits the device at once (asked of the runtime at plan creation)
     int fprop_parts = 0;
     size_t wt_bytes = 0;
     size_t wgrad_partial_bytes = 0;
@@ -1316,7 +847,7 @@ inline int igemm_stage_cw(int BN) {
 inline size_t igemm_fixed_smem(int BN, int ldo) {
     return 1024 /*alignment slack*/ + (size_t)2 * TC_BM * (igemm_stage_cw(BN) * 2 + 16) + (size_t)8 * ldo * 4 + 512;
 }
-inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses, bool allow_bres = false) {
+inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int ldo, int sm_count, int nclasses) {
     IgemmCfg c;
     c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
     if (Ca % 16 || rowsB % 16 || M < 1) return c;
@@ -1379,92 +910,7 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     c.stages = std::max(2, std::min(c.stages, std::max(2, (kblocks + c.kpb - 1) / c.kpb)));
     c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.stages * (c.a_stage + c.b_stage), 120 * 1024);  // > half an SM: one CTA per SM
     c.grid = (int)std::min<long long>((long long)c.m_tiles * c.n_tiles * nclasses, c.cg2 ? sm_count / 2 : sm_count);
-    // Weights-stationary (data gradient only; opt-in, NB_TC_BRES=1; =2 also for 3x3): with one column tile and one class
-    // every tile of a CTA multiplies by the same filter rows, and when that share of the filter fits beside a ring of at least three A stages
-    // it is fetched once per launch instead of once per tile.  Measured on B200, kernels timed one at a time: 1x1 layers
-    // gain in the data gradient (96 -> 192 at 160 x 160: 62.7 -> 53.5 us, 96 -> 96: 40.9 -> 36.6 us; forward +-1 us), 3x3
-    // layers with 48 or 64 channels lose 2-5 % (the ring loses a stage to the resident filter); inside the benchmark's
-    // CUDA graph, where these data gradients overlap the weight gradients of the second stream, the step time does not
-    // move (9.60 ms either way), so the mode is off by default.
-    {
-        const int groups = (kblocks + c.kpb - 1) / c.kpb;
-        const size_t fixed = igemm_fixed_smem(c.BN, ldo), res_b = (size_t)groups * c.b_stage;
-        const int want = getenv("NB_TC_BRES") ? atoi(getenv("NB_TC_BRES")) : 0;
-        if (allow_bres && want > 0 && (ntaps == 1 || want == 2) && c.n_tiles == 1 && nclasses == 1 && c.m_tiles >= 2 * c.grid &&
-            fixed + res_b + 3 * (size_t)c.a_stage <= kMaxSmem) {
-            c.bres = true;
-            c.b_groups = groups;
-            c.stages = (int)std::min<size_t>(8, (kMaxSmem - fixed - res_b) / c.a_stage);  // the A ring runs ahead across tiles
-            c.smem_bytes = std::max<size_t>(fixed + (size_t)c.stages * c.a_stage + res_b, 120 * 1024);
-        }
-    }
     if (c.cg2) c.grid *= 2;  // two CTAs per pair
-    c.ok = true;
-    return c;
-}
-
-// Tile configuration of the tap-reuse variant for a 3x3 stride-1 convolution over [N][H][W][Ca] with rowsB output channels.
-// Rows of the GEMM are padded-raster positions; CTA t of the launch order owns positions [W+3 + t*128*mh, +128*mh) and
-// fetches the slab [t*128*mh, +128*mh + 2*(W+2) + 2).
-inline IgemmCfg halo_configure(int N, int H, int W, int Ca, int rowsB, int ldo, int sm_count) {
-    IgemmCfg c;
-    c.Ca = Ca; c.rowsB = rowsB; c.ntaps = 9; c.KC = 64;
-    c.M = (long long)N * H * W;
-    // Off unless NB_TC_HALO=1.  Measured on B200 over the detector's 3x3 layers: the slab cuts the bytes TMA writes to
-    // shared memory by 1.3-1.9x, but a tap whose first row is not a multiple of eight rows into the slab makes every
-    // tcgen05.mma read its A operand ~1.2x slower (119 instead of 92-96 cycles per 256 x 192 x 16 MMA), and 5-17 % of the
-    // rows are padding; only the 20 x 20 layers with 288 channels gained (10 %), the others lost 5-20 %.
-    if (!(getenv("NB_TC_HALO") && atoi(getenv("NB_TC_HALO")) == 1)) return c;
-    if (Ca % 16 || rowsB % 16) return c;
-    const int Wp = W + 2, Hp = H + 2;
-    const long long npos = (long long)N * Hp * Wp;
-    if (npos >= (1LL << 30)) return c;
-    const int force_bn = getenv("NB_TC_BN") ? atoi(getenv("NB_TC_BN")) : 0;
-    const int force_mh = getenv("NB_TC_MH") ? atoi(getenv("NB_TC_MH")) : 0;
-    const int force_kpb = getenv("NB_TC_KPB") ? atoi(getenv("NB_TC_KPB")) : 0;
-    const long long span = npos - 2LL * (Wp + 1);  // positions from the first to the last real output
-    for (int bn = std::min(256, rowsB) / 16 * 16; bn >= 16 && !c.BN; bn -= 16) {
-        if (rowsB % bn) continue;
-        if (force_bn && bn != force_bn && rowsB % force_bn == 0) continue;
-        const int acc_stride = bn <= 32 ? 32 : bn <= 64 ? 64 : bn <= 128 ? 128 : 256;
-        for (int mh = (4 * acc_stride <= 512) ? 2 : 1; mh >= 1 && !c.BN; --mh) {
-            if (force_mh && mh != force_mh && force_mh * acc_stride <= 512) continue;
-            const int rows_cta = TC_BM * mh;
-            const long long cta_tiles = (span + rows_cta - 1) / rows_cta;
-            const long long pair_tiles = (cta_tiles + 1) / 2;
-            // two row blocks per CTA only while every pair still gets a tile
-            if (mh == 2 && !force_mh && pair_tiles * (rowsB / bn) < sm_count / 2) continue;
-            const int R = rows_cta + 2 * Wp + 2;
-            const int boxes = (R + 255) / 256;
-            const int box_pix = ((R + boxes - 1) / boxes + 7) / 8 * 8;
-            const uint32_t slab = (uint32_t)boxes * (uint32_t)box_pix * 128u;
-            const uint32_t b_sub = (uint32_t)((bn / 2 * 128 + 1023) / 1024 * 1024);
-            const size_t fixed = igemm_fixed_smem(bn, ldo);
-            const double tap_cycles = 4.0 * mh * std::max(32.0, bn / 2.0);  // tensor cycles per tap of one 64-channel block
-            int kpb = tap_cycles < 300.0 ? 3 : 1;
-            if (force_kpb == 1 || force_kpb == 3 || force_kpb == 9) kpb = force_kpb;
-            int a_slots = 2, stages = 0;
-            for (;;) {
-                if (fixed + (size_t)a_slots * slab < kMaxSmem) stages = (int)std::min<size_t>(8, (kMaxSmem - fixed - (size_t)a_slots * slab) / ((size_t)kpb * b_sub));
-                if (stages >= 3 || kpb == 1) break;
-                kpb = 1;
-            }
-            if (stages < 2) continue;
-            c.BN = bn; c.mh = mh; c.kpb = kpb; c.stages = stages; c.acc_stride = acc_stride;
-            c.acc_bufs = (2 * mh * acc_stride <= 512) ? 2 : 1;
-            c.a_sub = 0; c.b_sub = b_sub; c.a_stage = slab; c.b_stage = b_sub * (uint32_t)kpb;
-            c.cg2 = true; c.halo = true;
-            c.Wp = Wp; c.Hp = Hp; c.Hin = H; c.Win = W; c.Nimg = N;
-            c.slab_boxes = boxes; c.box_pix = box_pix; c.a_slots = a_slots; c.slab_bytes = slab; c.npos = npos;
-            c.m_tiles = (int)pair_tiles;
-        }
-    }
-    if (!c.BN) return c;
-    c.n_tiles = rowsB / c.BN;
-    c.stage_cols = igemm_team_cols(c.BN);
-    c.tmem_cols = std::max(32, c.acc_bufs * c.mh * c.acc_stride);
-    c.smem_bytes = std::max<size_t>(igemm_fixed_smem(c.BN, ldo) + (size_t)c.a_slots * c.slab_bytes + (size_t)c.stages * c.b_stage, 120 * 1024);
-    c.grid = 2 * (int)std::min<long long>((long long)c.m_tiles * c.n_tiles, sm_count / 2);
     c.ok = true;
     return c;
 }
@@ -1479,24 +925,10 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
     P.kpb = c.kpb; P.a_sub_bytes = c.a_sub; P.b_sub_bytes = c.b_sub;
     P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.ncol_a = c.stage_cols; P.stage_cw = igemm_stage_cw(c.BN);
-    P.variant = getenv("NB_TC_VARIANT") ? atoi(getenv("NB_TC_VARIANT")) : 0;
     if (getenv("NB_TC_VERBOSE"))
-        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu bres=%d(%d)\n", c.M, c.Ca,
-                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes, (int)c.bres, c.b_groups);
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
+                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
     P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
-    P.halo = c.halo ? 1 : 0;
-    if (c.bres) P.a_slots = c.b_groups;
-    if (c.halo) {
-        P.Wp = c.Wp; P.Hp = c.Hp; P.Hin = c.Hin; P.Win = c.Win; P.Nimg = c.Nimg;
-        P.slab_boxes = c.slab_boxes; P.box_pix = c.box_pix; P.a_slots = c.a_slots; P.slab_bytes = c.slab_bytes; P.npos = c.npos;
-        if (getenv("NB_TC_VERBOSE"))
-            fprintf(stderr, "[nb_cbs]   halo: Wp=%d slab=%d boxes x %d positions (%u bytes) x %d slots, taps per B stage %d\n", c.Wp, c.slab_boxes, c.box_pix,
-                    c.slab_bytes, c.a_slots, c.kpb);
-    }
-}
-// Start of tap t inside a slab: off_h rows of the padded raster down, off_w positions right (16-byte units, 8 per position).
-inline void fill_halo_taps(IgemmParams& P) {
-    for (int t = 0; t < 9; ++t) P.tap_off16[t] = (uint32_t)((int)P.off_h[0][t] * P.Wp + (int)P.off_w[0][t]) * 8u;
 }
 
 // im2col map over a bf16 NHWC tensor [N][H][W][C]: traversal starts at (lo, lo), steps `ts`, and ends `up` short of the far edge.
@@ -1552,20 +984,31 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
     return true;
 }
 
-template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES = 0, bool BRES = false, bool CLS4 = false> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+// Raises the dynamic shared-memory limit of one kernel instantiation once per device.
+template <typename OutT, bool STATS, bool CG2, int EPI, bool CLS4> inline bool igemm_allow_smem() {
     // the attribute belongs to the (function, device) pair: one bit per device ordinal that already has it
     static std::atomic<unsigned long long> attr_set{0};
     int dev = 0;
     cudaGetDevice(&dev);
     const unsigned long long bit = 1ull << (dev & 63);
     if (!(attr_set.load(std::memory_order_acquire) & bit)) {
-        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES, BRES, CLS4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_igemm_kernel<OutT, STATS, CG2, EPI, CLS4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
             err() = "cannot raise the dynamic shared memory limit of the implicit-GEMM kernel";
-            return NB_ERR_CUDA;
+            return false;
         }
         attr_set.fetch_or(bit, std::memory_order_release);
     }
-    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, HALO, EPI, RES, BRES, CLS4>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
+    return true;
+}
+template <typename OutT, bool STATS, bool CG2, int EPI = 0, bool CLS4 = false> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
+    if (!igemm_allow_smem<OutT, STATS, CG2, EPI, CLS4>()) return NB_ERR_CUDA;
+    // Also the forward launch that ends in a grid barrier may become resident beside its predecessor: it runs one CTA
+    // per SM (more than half of the shared memory each), so a CTA of it that is resident early can never keep another CTA
+    // of the same grid from fitting once the predecessor's CTAs have left, and nothing the predecessor waits for is
+    // held by it.  (Grids with several CTAs per SM are different: see grid_arrive.)
+    // Measured: launching it only after its predecessor has completed costs 3.4 us per forward kernel (its prologue --
+    // barrier set-up, TMEM allocation, tensor-map fetch -- no longer overlaps the predecessor's tail).
+    const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, EPI, CLS4>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
         return NB_ERR_CUDA;
@@ -1573,12 +1016,42 @@ template <typename OutT, bool STATS, bool CG2, bool HALO, int EPI = 0, int RES =
     return NB_OK;
 }
 template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmSlot& s, cudaStream_t st) {
-    if (s.cfg.halo) return launch_igemm_impl<OutT, STATS, true, true>(s, st);
-    if constexpr (!STATS) {  // the data gradient: the only launch with four classes or the weights-stationary configuration
-        if (s.prm.nclasses == 4) return s.cfg.cg2 ? launch_igemm_impl<OutT, false, true, false, 0, 0, false, true>(s, st) : launch_igemm_impl<OutT, false, false, false, 0, 0, false, true>(s, st);
-        if (s.cfg.bres) return s.cfg.cg2 ? launch_igemm_impl<OutT, false, true, false, 0, 0, true>(s, st) : launch_igemm_impl<OutT, false, false, false, 0, 0, true>(s, st);
+    if constexpr (!STATS) {  // the data gradient: the only launch with four classes
+        if (s.prm.nclasses == 4) return s.cfg.cg2 ? launch_igemm_impl<OutT, false, true, 0, true>(s, st) : launch_igemm_impl<OutT, false, false, 0, true>(s, st);
     }
-    return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true, false>(s, st) : launch_igemm_impl<OutT, STATS, false, false>(s, st);
+    return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true>(s, st) : launch_igemm_impl<OutT, STATS, false>(s, st);
+}
+// Whether all CTAs of the forward launch with statistics can be resident at once on the current device (the condition of
+// its grid barrier), asked of the runtime for this kernel, block size and shared-memory size.
+inline bool igemm_fwd_grid_fits(const IgemmCfg& c, int sm_count) {
+    int per_sm = 0;
+    if (c.cg2) {
+        if (!igemm_allow_smem<__half, true, true, 0, false>()) return false;
+        cudaLaunchConfig_t lc;
+        memset(&lc, 0, sizeof lc);
+        lc.gridDim = dim3((unsigned)c.grid);
+        lc.blockDim = dim3(IG_THREADS);
+        lc.dynamicSmemBytes = c.smem_bytes;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, tc_igemm_kernel<__half, true, true, 0, false>, &lc) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        return c.grid <= 2 * clusters;
+    }
+    if (!igemm_allow_smem<__half, true, false, 0, false>()) return false;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_igemm_kernel<__half, true, false, 0, false>, IG_THREADS, c.smem_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return c.grid <= per_sm * sm_count;
 }
 
 }  // namespace tcdetail
@@ -1590,15 +1063,9 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
 inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&, bool f16 = false) {
     const nb_status st = tc_plan_init_impl(tc, g, enable, sm_count);
     tc->f16 = f16;
-    tc->tma_store = !(getenv("NB_TC_TMA_STORE") && atoi(getenv("NB_TC_TMA_STORE")) == 0);
-    // Measured on the detector's layers: 41 of the 77 qualify, and the step gets 0.2 ms SLOWER (the second pass runs on the
-    // eight epilogue warps of each CTA behind one more grid barrier, where the separate pass is a 4 us kernel of 444
-    // blocks), so the variant is chosen only on request (NB_TC_RESIDENT=1 at plan creation).
-    if (st == NB_OK && tc->fprop && !tc->fp.cfg.halo && tc->tma_store && !f16 && getenv("NB_TC_RESIDENT") && atoi(getenv("NB_TC_RESIDENT")) == 1) {
-        const IgemmCfg& c = tc->fp.cfg;
-        const long long tiles = (long long)c.m_tiles * c.n_tiles, workers = c.cg2 ? c.grid / 2 : c.grid;
-        tc->fp_resident = (tiles + workers - 1) / workers <= c.acc_bufs;
-    }
+    // the forward kernel may finalize the statistics behind a grid barrier only if the runtime confirms that its whole grid
+    // can be resident at once
+    if (st == NB_OK && tc->fprop) tc->fp_barrier_ok = tcdetail::igemm_fwd_grid_fits(tc->fp.cfg, sm_count);
     if (st == NB_OK && f16) {  // A and B formats of the instruction descriptors: bits 7 and 10 set = bf16, clear = f16
         const uint32_t fmt = (1u << 7) | (1u << 10);
         tc->fp.prm.idesc &= ~fmt;
@@ -1618,9 +1085,7 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
     const bool even = (g.h % 2 == 0) && (g.w % 2 == 0);
     // ---- fprop: A = x (im2col), B = w [Cout][k*k*Cin]
     if (g.c_in % 16 == 0 && g.c_out % 16 == 0) {
-        IgemmCfg c;
-        if (g.k == 3 && g.stride == 1 && g.pad == 1) c = halo_configure(g.n, g.h, g.w, g.c_in, g.c_out, g.c_out, sm_count);
-        if (!c.ok) c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count, 1);
+        const IgemmCfg c = igemm_configure(g.m, g.c_in, g.c_out, g.k * g.k, g.c_out, sm_count, 1);
         if (c.ok) {
             tc->fp.cfg = c;
             IgemmParams& P = tc->fp.prm;
@@ -1636,13 +1101,10 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
                 }
             P.ldo = g.c_out; P.Hout = g.ho; P.Wout = g.wo; P.os = 1;
             P.a_tiled = (g.k == 1 && g.stride == 1) ? 1 : 0;
-            if (c.halo) fill_halo_taps(P);
             tc->fprop = true;
             tc->fprop_parts = c.grid;
-            if (!c.halo) {
-                tc->inf = tc->fp;
-                tc->infer = true;
-            }
+            tc->inf = tc->fp;
+            tc->infer = true;
         }
     }
     // ---- dgrad: A = dy (im2col), B = rearranged filter [Cin][taps*Cout]; stride 2 splits dx into four output-parity
@@ -1695,15 +1157,12 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
             P.Hq = g.h / 2; P.Wq = g.w / 2; P.ts = 1; P.lo_w = P.lo_h = 0;
             P.Hout = g.h; P.Wout = g.w; P.os = 2;
         }
-        IgemmCfg c;
-        if (g.k == 3 && g.stride == 1 && g.pad == 1) c = halo_configure(g.n, g.h, g.w, g.c_out, g.c_in, g.c_in, sm_count);
-        if (!c.ok) c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls, true);
+        const IgemmCfg c = igemm_configure((long long)g.n * P.Hq * P.Wq, g.c_out, g.c_in, max_taps, g.c_in, sm_count, ncls);
         if (c.ok) {
             tc->dg.cfg = c;
             fill_params(P, c);  // sets only the tiling fields; the geometry written above stays
-            if (c.halo) fill_halo_taps(P);
             P.nclasses = ncls; P.tiles_per_class = c.m_tiles * c.n_tiles;
-            if (ncls == 4 && !(getenv("NB_TC_CLS_INTERLEAVE") && atoi(getenv("NB_TC_CLS_INTERLEAVE")) == 0)) P.variant |= 64;  // see igemm_tile_class
+            P.cls_interleave = ncls == 4 ? 1 : 0;  // see igemm_tile_class
             P.ldo = g.c_in;
             W.nclasses = ncls;
             tc->wt_bytes = off * 2;
@@ -1803,19 +1262,14 @@ struct FwdFinalize {  // inputs and outputs of the BatchNorm finalize that the f
     const float *gamma, *beta;
     float *mean, *invstd, *scale, *shift, *rmean, *rvar;
 };
-// a_out / applied: with the fused finalize on a plan whose accumulators all stay resident (tc->fp_resident) the kernel also
-// writes the activations a = SiLU(y*scale + shift) and *applied is set: the caller then skips its normalise + SiLU pass.
+// fin == NULL: the kernel only writes y and the per-CTA partial sums.  wait_limit_ms / bar_extra: see IgemmParams (0 in normal use).
 inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st,
-                          const FwdFinalize* fin, void* a_out = nullptr, bool* applied = nullptr) {
+                          const FwdFinalize* fin, int wait_limit_ms = 0, int bar_extra = 0) {
     using namespace tcdetail;
     TcGemmSlot& S = tc->fp;
-    if (applied) *applied = false;
     if (S.a_ptr != x || S.b_ptr != w) {
         const int up = g.pad - (g.k - 1);
-        if (S.cfg.halo) {
-            // traversal over the padded raster: window start from -1 to W (one past each edge), tap offsets always zero
-            if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -1, 1, 1, 64, S.cfg.box_pix)) return NB_ERR_CUDA;
-        } else if (S.prm.a_tiled) {
+        if (S.prm.a_tiled) {
             if (!encode_tiled_2d(&S.prm.tmA, x, g.m, g.c_in, S.cfg.KC, TC_BM * S.cfg.mh, tc->ld_x)) return NB_ERR_CUDA;
         } else if (!encode_im2col(&S.prm.tmA, x, g.n, g.h, g.w, g.c_in, -g.pad, up, g.stride, S.cfg.KC, TC_BM * S.cfg.mh, tc->ld_x)) {
             return NB_ERR_CUDA;
@@ -1823,8 +1277,8 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         S.a_ptr = x; S.b_ptr = w;
     }
-    S.prm.tma_store = (!S.cfg.halo && tc->tma_store) ? 1 : 0;
-    if (S.prm.tma_store && S.out_ptr != y) {
+    S.prm.tma_store = 1;
+    if (S.out_ptr != y) {
         if (!encode_out_maps(S.prm, S.cfg, y, g.m)) return NB_ERR_CUDA;
         S.out_ptr = y;
     }
@@ -1835,21 +1289,9 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         S.prm.fin_mean = fin->mean; S.prm.fin_invstd = fin->invstd; S.prm.fin_scale = fin->scale; S.prm.fin_shift = fin->shift;
         S.prm.fin_rmean = fin->rmean; S.prm.fin_rvar = fin->rvar;
     }
+    S.prm.wait_limit_ms = wait_limit_ms; S.prm.bar_extra = bar_extra;
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
-#ifdef NB_TC_DEBUG_TIMING
-    if (const char* e = getenv("NB_TC_DBG_PTR")) S.prm.dbg = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
-#endif
     tc->launches += 1;
-    if (fin && a_out && applied && tc->fp_resident && S.prm.tma_store) {
-        if (tc->res_out_ptr != a_out) {  // the same boxes as the y maps, over the activation tensor
-            IgemmParams tmp = S.prm;
-            if (!encode_out_maps(tmp, S.cfg, a_out, g.m)) return NB_ERR_CUDA;
-            for (int i = 0; i < 3; ++i) S.prm.tmB[1 + i] = tmp.tmOut[i];
-            tc->res_out_ptr = a_out;
-        }
-        *applied = true;
-        return S.cfg.cg2 ? launch_igemm_impl<__half, true, true, false, 0, 1>(S, st) : launch_igemm_impl<__half, true, false, false, 0, 1>(S, st);
-    }
     return launch_igemm<__half, true>(S, st);
 }
 
@@ -1881,11 +1323,10 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
     S.prm.fin_gamma = e.gamma; S.prm.fin_beta = e.beta;
     S.prm.fin_rmean = const_cast<float*>(e.rmean); S.prm.fin_rvar = const_cast<float*>(e.rvar);  // only read
     S.prm.fin_eps = e.eps; S.prm.epi_act = e.act;
-    S.prm.variant = 0;  // no experiment switches on this path
     S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
     tc->launches += 1;
-    if (tc->f16) return S.cfg.cg2 ? launch_igemm_impl<__half, false, true, false, 1>(S, st) : launch_igemm_impl<__half, false, false, false, 1>(S, st);
-    return S.cfg.cg2 ? launch_igemm_impl<__nv_bfloat16, false, true, false, 1>(S, st) : launch_igemm_impl<__nv_bfloat16, false, false, false, 1>(S, st);
+    if (tc->f16) return S.cfg.cg2 ? launch_igemm_impl<__half, false, true, 1>(S, st) : launch_igemm_impl<__half, false, false, 1>(S, st);
+    return S.cfg.cg2 ? launch_igemm_impl<__nv_bfloat16, false, true, 1>(S, st) : launch_igemm_impl<__nv_bfloat16, false, false, 1>(S, st);
 }
 
 // `wt_ready`: the rearranged filter was already written by an earlier kernel of this call (the BN backward finalize kernel
@@ -1903,18 +1344,14 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
     if (S.a_ptr != dy || S.b_ptr != wt) {
         // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
         const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
-        if (S.cfg.halo) {
-            if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, -1, 1, 1, 64, S.cfg.box_pix)) return NB_ERR_CUDA;
-        } else if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) {
-            return NB_ERR_CUDA;
-        }
+        if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
         for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
             const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
             if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
         }
         S.a_ptr = dy; S.b_ptr = wt;
     }
-    S.prm.tma_store = (g.stride == 1 && !S.cfg.halo && tc->tma_store) ? 1 : 0;
+    S.prm.tma_store = g.stride == 1 ? 1 : 0;  // the parity classes of a stride-2 layer write every other output pixel
     if (S.prm.tma_store && S.out_ptr != dx) {
         if (!encode_out_maps(S.prm, S.cfg, dx, (long long)g.n * g.h * g.w)) return NB_ERR_CUDA;
         S.out_ptr = dx;

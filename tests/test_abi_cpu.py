@@ -116,3 +116,28 @@ def test_sgd_plan_rejects_bad_lists_before_any_cuda_call(lib):
     arr[0].grad = 0x1004
     assert lib.nb_sgd_plan_create(arr, 1, 0, ctypes.byref(h)) == nb.NB_ERR_ALIGNMENT
     assert ctypes.sizeof(nb.nb_sgd_tensor) == 48 and ctypes.sizeof(nb.nb_sgd_hyper) == 40 and ctypes.sizeof(nb.nb_scaler_hyper) == 20
+
+
+def test_status_codes_of_the_binding_match_the_header():
+    text = open(os.path.join(ROOT, "include", "nb_cbs.h")).read()
+    codes = dict((k, int(v)) for k, v in re.findall(r"\b(NB_(?:OK|ERR_[A-Z_]+)) = (\d+)", text))
+    assert codes["NB_ERR_TIMEOUT"] == 7 and len(codes) == 9
+    for name, value in codes.items():
+        assert getattr(nb, name) == value, name
+
+
+def test_device_code_reports_give_ups_through_the_named_constant_only():
+    """The status word that nb_cbs_poll_status returns is written in ONE place (report_timeout in common.cuh, with
+    NB_ERR_TIMEOUT from the header); no kernel source writes a literal code there, and the two grid-barrier sites are the
+    named constants 20 and 21 that the header documents for the test hook."""
+    csrc = os.path.join(ROOT, "paper_2609_10632_b200", "csrc")
+    writers = []
+    for fn in sorted(os.listdir(csrc)):
+        text = open(os.path.join(csrc, fn)).read()
+        for m in re.finditer(r"atomicCAS\([^;]*ST_ERR[^;]*;", text):
+            writers.append((fn, m.group(0)))
+    assert len(writers) == 1 and writers[0][0] == "common.cuh" and "(int)NB_ERR_TIMEOUT" in writers[0][1], writers
+    common = open(os.path.join(csrc, "common.cuh")).read()
+    assert "SITE_GRID_BARRIER_FWD = 20" in common and "SITE_GRID_BARRIER_BWD = 21" in common
+    assert "SITE_GRID_BARRIER_BWD" in open(os.path.join(csrc, "elementwise.cuh")).read()
+    assert "SITE_GRID_BARRIER_FWD" in open(os.path.join(csrc, "tc_conv.cuh")).read()
