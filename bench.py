@@ -35,17 +35,33 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the 77 launches of a site in one step
-# of the cfg5 workload) from the ncu capture summarised in profiles/launch_list_cfg5_step.md (warm caches, as in a real
-# step: most layers' tensors stay in the 126 MB L2, so the traffic is well below the algorithmic bytes).
-NCU_DRAM_BYTES_PER_LAUNCH_CFG5 = {
-    "conv_fprop": (2129 + 1439) * 1e6 / 77,
-    "conv_dgrad": (576 + 1708) * 1e6 / 77,
-    "conv_wgrad": (2434 + 1458) * 1e6 / 77,
-    "bn_silu_apply": (440 + 770) * 1e6 / 77,
-    "bn_silu_bwd_reduce": (1989 + 906) * 1e6 / 77,
-    "bn_silu_bwd_dy": (1090 + 794) * 1e6 / 77,
+# DRAM traffic of one launch divided by its algorithmic bytes, measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum) on SINGLE-kernel captures of small cases whose tensors exceed L2: benchmark configuration 3 for
+# the three GEMM kernels, configuration 2 (157 MB tensors) for the elementwise passes.  roofline.traffic of a full-size
+# launch is this ratio times the launch's algorithmic bytes (traffic grows in proportion to the tensor sizes).
+NCU_TRAFFIC_OVER_ALGORITHMIC = {
+    "conv_fprop": 1.03, "conv_dgrad": 1.02, "conv_wgrad": 1.9,  # the weight gradient also writes and re-reads its split-K partial tiles
+    "bn_silu_apply": 1.00, "bn_silu_bwd_reduce": 1.00, "bn_silu_bwd_dy": 1.00,
 }
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def spread(ms_list):
+    """mean / median / min of per-step device times (milliseconds)."""
+    v = sorted(ms_list)
+    n = len(v)
+    med = v[n // 2] if n % 2 else 0.5 * (v[n // 2 - 1] + v[n // 2])
+    return {"mean": sum(v) / n, "median": med, "min": v[0], "max": v[-1], "steps": n}
 
 
 def write_per_layer(path, blocks, per_shape, peaks):
@@ -231,7 +247,7 @@ def run_reference(args):
         "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs_all) / len(secs_all), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "note": "fp64 CPU oracle on a bounded sample per step; ms_per_step is the sample's time"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "cpu": cpu_model(), "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -276,6 +292,8 @@ def main():
     ap.add_argument("--force-simt", action="store_true", help="run the convolutions on the CUDA-core kernels")
     ap.add_argument("--no-wgrad-stream", action="store_true", help="queue the weight gradients on the main stream instead of a second stream")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph of one step")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the additional sustained region in seconds of device time (0 = skip)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration figures (cfg2, cfg3, cfg4a, cfg4b)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -368,21 +386,41 @@ def main():
     barrier()
     stream = torch.cuda.current_stream()
     l0 = nb.nb_cbs_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # Exactly --steps steps between two events; an event after every step gives the spread (mean / median / min).
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with ClockSampler(local) as clocks:
-        ev0.record(stream)
-        for _ in range(args.steps):
+        marks[0].record(stream)
+        for i in range(args.steps):
             run_step()
-        ev1.record(stream)
+            marks[i + 1].record(stream)
         barrier()
     launches = launches_per_step * args.steps if launches_per_step is not None else nb.nb_cbs_launch_count() - l0
     for b in blocks:
         b.poll()
-    ms_total = ev0.elapsed_time(ev1)
+    ms_total = marks[0].elapsed_time(marks[-1])
+    per_step = spread([marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)])
     ms_total = max_over_ranks(ms_total, dist, dev)
     ms_step = ms_total / args.steps
     value = whole_job_value(world, flops, ms_step)
     peaks = load_peaks()
+    # The same step for at least --sustain-seconds of device time (default 2 s), with its own clock record: the timed
+    # region above lasts a fraction of a second at boost clock, this one shows what a long run settles at.
+    sustained = None
+    if args.sustain_seconds > 0:
+        n_sus = max(args.steps, int(args.sustain_seconds * 1e3 / ms_step) + 1)
+        smarks = [torch.cuda.Event(enable_timing=True) for _ in range(n_sus + 1)]
+        barrier()
+        with ClockSampler(local) as sclocks:
+            smarks[0].record(stream)
+            for i in range(n_sus):
+                run_step()
+                smarks[i + 1].record(stream)
+            barrier()
+        for b in blocks:
+            b.poll()
+        sus_ms = max_over_ranks(smarks[0].elapsed_time(smarks[-1]), dist, dev)
+        sustained = spread([smarks[i].elapsed_time(smarks[i + 1]) for i in range(n_sus)]) | {
+            "ms_per_step": sus_ms / n_sus, "value": whole_job_value(world, flops, sus_ms / n_sus), "unit": UNIT, "seconds": sus_ms * 1e-3, "clocks": sclocks.summary()}
 
     # ---------------- instrumented pass: per-site device times (events around every launch; calls wait for each kernel)
     roofline, kernels = None, {}
@@ -436,9 +474,11 @@ def main():
         else:
             roofline = {"kernel": top, "bound": "hbm", "achieved": a["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        roofline["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH_CFG5.get(top) if args.workload == "cfg5" else None
-        roofline["traffic_note"] = ("bytes per launch, average of the site's launches in one step, from the committed ncu launch list "
-                                    "(profiles/launch_list_cfg5_step.md); algorithmic bytes per launch: %.3g" % (a["bytes"] / a["launches"]))
+        ratio = NCU_TRAFFIC_OVER_ALGORITHMIC.get(top)
+        roofline["traffic"] = ratio * a["bytes"] / a["launches"] if ratio else None
+        roofline["traffic_note"] = ("DRAM bytes per launch = algorithmic bytes per launch (%.3g, average over the site's launches of one step) x %s, the "
+                                    "ratio ncu measured on a single-kernel capture of a small case of the same kernel; inside a step most layers' "
+                                    "tensors are found in the 126 MB L2, so the real traffic is lower" % (a["bytes"] / a["launches"], ratio))
         roofline["peak_source"] = peaks["source"] + (" (burst figure: kernels timed one at a time)" if roofline["bound"] == "tensor" else "")
         roofline["avg_launch_ms"] = a["ms"] / a["launches"]
         roofline["share_of_step"] = a["ms"] / tot_ms
@@ -463,10 +503,15 @@ def main():
     if not args.no_e2e:
         e2e = run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops)
 
+    # ---------------- the other benchmark configurations, one by one (cfg2 stem, cfg3, cfg4a, cfg4b)
+    cfgs = None
+    if not args.no_configs and args.workload == "cfg5" and not args.f16:
+        cfgs = run_configs(args, dev, local, peaks, ws, wgrad_ws)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, secs, fl, cores, desc = time_oracle(layers, args.cpu_budget)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": f"{desc}; {secs:.1f} s"}
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "cpu": cpu_model(), "kind": "oracle", "sample": f"{desc}; {secs:.1f} s"}
 
     if rank == 0:
         paths = {"fprop": 0, "dgrad": 0, "wgrad": 0}
@@ -475,7 +520,7 @@ def main():
                 paths[k] += b.plan.paths[k]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16" if args.f16 else "bf16", "data": "synthetic",
+            "ms_per_step": ms_step, "ms_per_step_spread": per_step, "sustained": sustained, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16" if args.f16 else "bf16", "data": "synthetic",
             "config": {
                 "workload": f"{args.workload}: {len(layers)} Conv-BN-SiLU layers, batch {layers[0].n}, fwd + bwd_data + bwd_weight per layer "
                             f"(stem data gradient included), each layer on its own tensors",
@@ -485,11 +530,73 @@ def main():
                 "frac_of_measured_sustained_bf16_peak": value / world / peaks["bf16_tflops_sustained"],
             },
             "clocks": clocks.summary(), "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
-            "kernels": kernels, "eval_forward": eval_fwd, "optimizer_step": opt_step, "detector_chain": chain,
+            "kernels": kernels, "configs": cfgs, "eval_forward": eval_fwd, "optimizer_step": opt_step, "detector_chain": chain,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_configs(args, dev, local, peaks, ws, wgrad_ws):
+    """Benchmark configurations 2, 3, 4a and 4b on their own: one training step of that layer as a CUDA-graph replay (weight
+    gradient on the main stream: a single layer has nothing to overlap it with), repeated with an L2 flush between
+    replays left out on purpose for cfg2 / cfg3, whose tensors (157 MB / 79 MB each) exceed L2 anyway; per kernel site
+    the device time of an instrumented pass and what it means against the measured peaks."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200 import workloads as wl
+    from paper_2609_10632_b200.block import CbsBlock
+
+    out = {}
+    shapes = [("cfg2", wl.config_shapes(2)[0]), ("cfg3", wl.config_shapes(3)[0])] + list(zip(("cfg4a", "cfg4b"), wl.config_shapes(4)))
+    for name, s in shapes:
+        blk = CbsBlock(s, device=local)
+        blk.fill_random(seed=4000)
+        for _ in range(3):
+            blk.step()
+        torch.cuda.synchronize()
+        blk.poll()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            blk.step()
+        n = 100
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        marks[0].record()
+        for i in range(n):
+            graph.replay()
+            marks[i + 1].record()
+        torch.cuda.synchronize()
+        blk.poll()
+        sp = spread([marks[i].elapsed_time(marks[i + 1]) for i in range(n)])
+        fl = 3 * s.gemm_flops
+        rec = {"shape": [s.n, s.h, s.w, s.c_in, s.c_out, s.k, s.stride], "ms_per_step": sp["mean"], "ms_median": sp["median"], "ms_min": sp["min"],
+               "tflops": fl / (sp["mean"] * 1e-3) / 1e12, "frac_of_measured_bf16_peak": fl / (sp["mean"] * 1e-3) / 1e12 / peaks["bf16_tflops"], "kernels": {}}
+        nb.nb_cbs_profile_enable(blk.plan, True)
+        for _ in range(5):
+            blk.step()
+        torch.cuda.synchronize()
+        for site, (ms, cnt) in nb.nb_cbs_profile_read(blk.plan).items():
+            if cnt == 0:
+                continue
+            f, by = site_work(site, s)
+            us = ms / cnt * 1e3
+            k = {"us": us}
+            if site in ("conv_fprop", "conv_dgrad", "conv_wgrad"):
+                k["tflops"] = f / (us * 1e-6) / 1e12
+                k["frac_of_measured_bf16_peak"] = k["tflops"] / peaks["bf16_tflops"]
+            elif by:
+                k["gbs"] = by / (us * 1e-6) / 1e9
+                k["frac_of_measured_hbm_peak"] = k["gbs"] / peaks["hbm_gbs"]
+            rec["kernels"][site] = k
+        nb.nb_cbs_profile_enable(blk.plan, False)
+        out[name] = rec
+        del blk, graph
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_eval_forward(args, blocks, dev, fwd_flops, peaks, kernels):
@@ -744,7 +851,7 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
                 e.record(st)
                 main.wait_event(e)
 
-    steps = max(1, min(args.steps, 3))
+    steps = max(1, min(args.steps, 20))  # (the main arm's step count, up to 20: a step moves 7.3 GB over PCIe)
     fork()
     one()
     join()
