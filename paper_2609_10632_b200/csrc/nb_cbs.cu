@@ -384,8 +384,8 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
 
     p->stem = d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
               g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0 && g.m < (1LL << 31) && (long long)g.n * g.h * g.w * 3 < (1LL << 31);
-    p->stem_blocks = (int)std::min<long long>((g.m + 255) / 256, (long long)p->sm_count * 8);
-    p->nparts = std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts);
+    p->stem_blocks = (int)std::min<long long>(stem_num_strips(g), (long long)p->sm_count * 4);  // grid of the three first-layer kernels: one wave of four resident blocks per SM
+    p->nparts = std::max(std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts), p->stem ? p->stem_blocks : 0);
     const size_t C = (size_t)g.c_out;
     size_t off = 0;
     p->off_scale = off; off = align_up(off + C * 4, 256);
@@ -547,14 +547,12 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         NB_TRY((run_simt_fprop<float, float>(p, x, w, y_saved, st)));
         NB_TRY(run_stats_partial<float>(p, y_saved, part, st));
     } else if (p->stem) {
-        {
-            SiteTimer tm(p, SITE_FPROP, st);
-            const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
-            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
-                                   static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}));
-            NB_LAUNCH_OK("stem_fprop");
-        }
-        NB_TRY(run_stats_partial<__half>(p, y_saved, part, st));
+        // the first layer's kernel sums the statistics of the values it stores itself (one partial slice per block)
+        SiteTimer tm(p, SITE_FPROP, st);
+        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
+                               static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}, part));
+        NB_LAUNCH_OK("stem_fprop");
+        nparts = p->stem_blocks;
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
@@ -593,9 +591,8 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
     }
     if (!is_f32(p) && p->stem) {  // the first layer's own kernel applies the coefficients and the activation itself
         SiteTimer tm(p, SITE_INFER, st);
-        const int blocks = (int)std::min<long long>((p->g.m + 63) / 64, (long long)p->sm_count * 16);
-        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(w),
-                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}));
+        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(w),
+                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}, static_cast<float*>(nullptr)));
         return launch_ok("stem_fprop (fused epilogue)");
     }
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
@@ -714,12 +711,8 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     if (!dx) return NB_OK;
     if (p->stem) {
         SiteTimer tm(p, SITE_DGRAD, st);
-        {
-            const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
-            const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-            NB_WITH_AT(p, launch_k(stem_dgrad_tiled_kernel<48, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dy_out), static_cast<const AT*>(w),
-                                   static_cast<AT*>(dx), p->g));
-        }
+        NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dy_out), static_cast<const AT*>(w),
+                               static_cast<AT*>(dx), p->g));
         return launch_ok("stem_dgrad");
     }
     if (p->tc.dgrad) {
@@ -756,9 +749,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
                 NB_TRY(run_simt_dgrad<float>(p, dout, w, dx, st));
             } else if (p->stem) {
                 SiteTimer tm(p, SITE_DGRAD, st);
-                const long long total = (long long)p->g.n * p->g.ho * ((p->g.wo + 1) / 2);
-                const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)p->sm_count * 16);
-                NB_WITH_AT(p, launch_k(stem_dgrad_tiled_kernel<48, AT>, dim3(blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dout), static_cast<const AT*>(w),
+                NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dout), static_cast<const AT*>(w),
                                        static_cast<AT*>(dx), p->g));
                 NB_LAUNCH_OK("stem_dgrad");
             } else if (p->tc.dgrad) {
@@ -788,9 +779,8 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     if (p->stem) {
         {
             SiteTimer tm(p, SITE_WGRAD, st);
-            const long long per = (p->g.m + p->stem_blocks - 1) / p->stem_blocks;
             NB_WITH_AT(p, launch_k(stem_wgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(dy), partial,
-                                   p->g, per));
+                                   p->g));
             NB_LAUNCH_OK("stem_wgrad");
         }
         const size_t elems = (size_t)p->g.c_out * p->g.kdim;

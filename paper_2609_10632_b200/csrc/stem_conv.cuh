@@ -1,20 +1,22 @@
-// Kernels for the network's first layer: 3 input channels, 3x3, stride 2, pad 1.
-// A 3-channel bf16 pixel is 6 bytes, which no TMA descriptor can address (strides must be multiples of 16 bytes), and
-// K = 27 is far too short for the tcgen05 pipeline: the forward and the weight gradient run on warp-level mma.sync tiles of
-// 16 pixels, the data gradient (3 output channels) on register-tiled CUDA-core FMAs.  COUT is a template parameter
-// (48 for the detector's stem).
+// Kernels for the network's first layer: 3 input channels, 3x3, stride 2, pad 1, even H and W.
+// A 3-channel 16-bit pixel is 6 bytes, which no TMA descriptor can address (strides must be multiples of 16 bytes), and
+// K = 27 is far too short for the tcgen05 pipeline, so all three convolutions run on warp-level mma.sync tiles
+// (m16n8k16, fp32 accumulation).  All three are HBM-bound by design (157 MB of y / dy against 39 MB of x / dx at batch
+// 16, 640 x 640): every global access is a coalesced 16-byte (or 4-byte) vector; the 3 x 3 x 3 patches are never gathered
+// from global memory but cut out of input rows staged in shared memory.
+// Work unit of every kernel: a STRIP of up to 64 consecutive output pixels of one output row (16 per warp).
+// COUT is a template parameter (48 for the detector's stem).
 #pragma once
 #include "common.cuh"
 
 namespace nbcbs {
 
 constexpr int STEM_CIN = 3, STEM_K = 3, STEM_TAPS = 9, STEM_KDIM = 27;
+constexpr int STEM_TQ = 64;                                   // output pixels per strip
+constexpr int STEM_ROW_ELEMS = (2 * STEM_TQ + 1) * STEM_CIN;  // input values of one staged row: columns 2*q0-1 .. 2*q0+2*TQ-1
+constexpr int STEM_XCHUNKS = (STEM_ROW_ELEMS + 7 + 7) / 8;    // 16-byte chunks per staged row incl. the alignment shift (<= 7)
+constexpr int STEM_XPITCH = STEM_XCHUNKS * 8;
 
-// ---- tensor-core forward for the stem.  K = 27 is far too short for the tcgen05 pipeline (and a 6-byte pixel cannot be
-// fetched by TMA), so this kernel uses warp-level mma.sync (m16n8k16, bf16 -> fp32): a warp computes 16 consecutive output
-// pixels x COUT channels with K padded to 32.  The filter fragments stay in registers for the whole kernel; a thread
-// gathers the 2 x 8 input values of its fragment rows with 2-byte loads (the 3 x 3 x 3 patch of a pixel is three runs of 9
-// contiguous values, L1-resident across neighbouring pixels) and writes its accumulator pairs as fp16.
 template <typename T> __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1);
 template <> __device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
@@ -26,27 +28,112 @@ template <> __device__ __forceinline__ void mma_16816<__half>(float (&d)[4], con
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_row) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+
+// Strip number -> image n, output row p, first output column q0.
+struct StemStrip {
+    int n, p, q0;
+};
+__device__ __forceinline__ StemStrip stem_strip(long long t, const Geom& g, int strips_per_row) {
+    // (32-bit divisions: the plan admits fewer than 2^31 output pixels; 64-bit ones cost about a hundred instructions each,
+    // and these kernels are bound by instruction issue)
+    StemStrip s;
+    const unsigned tt = (unsigned)t, t1 = tt / (unsigned)strips_per_row;
+    s.q0 = (int)(tt - t1 * (unsigned)strips_per_row) * STEM_TQ;
+    s.n = (int)(t1 / (unsigned)g.ho);
+    s.p = (int)(t1 - (unsigned)s.n * (unsigned)g.ho);
+    return s;
+}
+__host__ __device__ inline long long stem_num_strips(const Geom& g) { return (long long)g.n * g.ho * ((g.wo + STEM_TQ - 1) / STEM_TQ); }
+
+// 16-byte asynchronous copy global -> shared; bytes past `src_bytes` (0..16) are written as zeros.
+__device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_pending() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }  // at most N groups still in flight
+
+// The three input rows 2p-1, 2p, 2p+1 of a strip, columns 2*q0-1 .. 2*q0+2*TQ-1, are staged in shared memory as aligned
+// 16-byte chunks of the flat tensor: element k of staged row r -- input column 2*q0-1 + k/3, channel k%3 -- is
+// xrow[r][shift[r] + k].  Row -1 (p = 0) is written as zeros; column -1 (q0 = 0) holds whatever precedes the row in memory
+// and is masked when the fragments of the strip's first pixel are built; values past the image's last column belong to output pixels that do not
+// exist and are never used.  The copies are asynchronous (cp.async) and run several strips ahead of the arithmetic (a ring
+// of NS buffers, NS - 1 strips in flight per block): with one strip in flight the kernels were bound by memory latency
+// (bytes in flight per SM x 148 / latency was far below the HBM rate), not by bandwidth.  `total` = number of elements of x.
+__device__ __forceinline__ int stem_row_start(const Geom& g, const StemStrip& s, int r, int& shift) {
+    // (int arithmetic: the plan admits fewer than 2^31 input elements)
+    const int e0 = ((s.n * g.h + (2 * s.p - 1 + r)) * g.w + (2 * s.q0 - 1)) * 3;  // negative only inside the padding
+    const int a0 = e0 >= 0 ? (e0 & ~7) : -((-e0 + 7) & ~7);
+    shift = e0 - a0;
+    return a0;
+}
+__device__ __forceinline__ void stem_stage_rows_async(const unsigned short* __restrict__ x, const Geom& g, int total, const StemStrip& s,
+                                                      unsigned short (*xrow)[STEM_XPITCH]) {
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        int sh;
+        const int a0 = stem_row_start(g, s, r, sh);
+        const bool row_ok = 2 * s.p - 1 + r >= 0;
+        for (int ci = threadIdx.x; ci < STEM_XCHUNKS; ci += blockDim.x) {
+            const int start = a0 + 8 * ci;
+            int bytes = 0;  // a chunk before the tensor's start (a0 < 0: only padding lies there), in row -1 or past the end: zeros
+            if (row_ok && start >= 0 && start < total) bytes = total - start >= 8 ? 16 : (total - start) * 2;
+            cp_async16_zfill(&xrow[r][8 * ci], bytes ? x + start : x, bytes);
+        }
+    }
+}
+
+// Two fp32 values rounded to a pair of 16-bit values (fp16 saturates at the largest finite value), and back.
+template <typename T> __device__ __forceinline__ uint32_t stem_pack2(float2 v);
+template <> __device__ __forceinline__ uint32_t stem_pack2<__half>(float2 v) {
+    uint32_t r;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(v.y), "f"(v.x));
+    return r;
+}
+template <> __device__ __forceinline__ uint32_t stem_pack2<__nv_bfloat16>(float2 v) {
+    const __nv_bfloat162 b = __float22bfloat162_rn(v);
+    return *reinterpret_cast<const uint32_t*>(&b);
+}
+template <typename T> __device__ __forceinline__ float2 stem_unpack2(uint32_t v);
+template <> __device__ __forceinline__ float2 stem_unpack2<__half>(uint32_t v) { return __half22float2(*reinterpret_cast<const __half2*>(&v)); }
+template <> __device__ __forceinline__ float2 stem_unpack2<__nv_bfloat16>(uint32_t v) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v)); }
+
 // Per-channel epilogue of the evaluation-mode / plain forward: out = act(acc*scale_c + shift_c), coefficients as bn_eval_coef.
 struct StemEpi {
     const float *gamma, *beta, *rmean, *rvar;
     float eps;
     int act;
 };
-// EPI = false: y = the convolution output in fp16 (training forward).  EPI = true: OutT = bf16 activations, see StemEpi.
+// Forward.  A warp computes 16 output pixels x COUT channels with K padded to 32 (two k-steps); the filter fragments stay
+// in registers for the whole kernel; the A fragments are read from the staged rows (2-byte shared-memory loads: the nine
+// values of one filter row of a pixel are contiguous there).  The 16 x COUT output tile is one contiguous run: staged and
+// written with 16-byte stores.
+// EPI = false: y = the convolution output in fp16 (training forward), and with `partials` != NULL the block also writes the
+// per-channel sum and sum of squares of the ROUNDED values it stored to partials[blockIdx.x][2][COUT] (batch statistics
+// without a second pass over y; fixed order, bitwise reproducible).  EPI = true: OutT = activations, see StemEpi.
 // InT = the 16-bit type of x and w (bf16, or IEEE fp16).
 template <int COUT, typename OutT = __half, bool EPI = false, typename InT = __nv_bfloat16>
-__global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const InT* __restrict__ x, const InT* __restrict__ w,
-                                                             OutT* __restrict__ y, Geom g, StemEpi ep) {
+__global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __restrict__ x, const InT* __restrict__ w, OutT* __restrict__ y, Geom g,
+                                                                StemEpi ep, float* __restrict__ partials) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 8 == 0, "whole n-blocks");
     constexpr int NB = COUT / 8;
-    const int lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
     const unsigned short* wsrc = reinterpret_cast<const unsigned short*>(w);
-    // the eight K indices of this lane's A / B fragment elements: k-step s, register half j, element e
-    int koff[8];   // element offset of K index k inside the input relative to the patch origin, or -1 for the padding (k >= 27)
-    int kr[8], kt[8];  // filter row and column of k (bounds checks)
+    // the eight K indices of this lane's A fragment elements: k-step s2, register half j, element e -> filter row and offset
+    // inside the nine contiguous values of that row (-1: the padding k >= 27)
+    // (a padding index k >= 27 meets a zero filter value: it reads the patch's centre, a value the pixel depends on anyway)
+    int krow[8], koff[8];    // filter row of k, and its offset in the staged rows relative to the pixel's first element
+    unsigned left_mask = 0;  // bit i: element i lies in the patch's left column (zero padding for the image's first column)
     uint32_t bfrag[2][NB][2];
 #pragma unroll
     for (int s2 = 0; s2 < 2; ++s2)
@@ -55,10 +142,9 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const InT* __restri
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int k = s2 * 16 + j * 8 + tq * 2 + e, i = s2 * 4 + j * 2 + e;
-                const int r = k / 9, kp = k - r * 9;
-                kr[i] = r;
-                kt[i] = kp / 3;
-                koff[i] = k < STEM_KDIM ? r * g.w * 3 + kp : -1;
+                krow[i] = k < STEM_KDIM ? k / 9 : 1;
+                koff[i] = krow[i] * STEM_XPITCH + (k < STEM_KDIM ? k % 9 : 3);
+                if (k < STEM_KDIM && k % 9 < 3) left_mask |= 1u << i;
             }
 #pragma unroll
     for (int s2 = 0; s2 < 2; ++s2)
@@ -83,243 +169,372 @@ __global__ void __launch_bounds__(128) stem_fprop_mma_kernel(const InT* __restri
                 esh[nb][e] = (float)sh;
             }
     }
+    float2 ssum[EPI ? 1 : NB], ssq[EPI ? 1 : NB];  // running channel sums of this lane's two columns per n-block over its rows
+    if (!EPI) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) ssum[nb] = ssq[nb] = make_float2(0.f, 0.f);
+    }
+    constexpr int NS = 4;  // ring of staged strips
+    __shared__ __align__(16) unsigned short xrow[NS][3][STEM_XPITCH];
     __shared__ __align__(16) OutT stage[4][16 * COUT];
-    const long long ntiles = (g.m + 15) / 16;
-    const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
-    for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < ntiles; tile += wstride) {
-        const long long m0 = tile * 16;
-        uint32_t a[2][4];
+    const int total = g.n * g.h * g.w * 3;
+    const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
+    const long long nstrips = stem_num_strips(g);
+    StemStrip ahead[NS - 1];  // the strips whose rows are in flight, decoded once
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {  // fragment rows gq and gq + 8
-            const long long m = m0 + gq + half * 8;
-            const bool row_ok = m < g.m;
-            const unsigned mm = row_ok ? (unsigned)m : 0u;  // the stem has fewer than 2^31 output pixels: 32-bit divisions
-            const unsigned t1 = mm / (unsigned)g.wo;
-            const int q = (int)(mm - t1 * (unsigned)g.wo);
-            const int n = (int)(t1 / (unsigned)g.ho), p = (int)(t1 - (unsigned)n * (unsigned)g.ho);
-            const int h0 = 2 * p - 1, w0 = 2 * q - 1;
-            const long long origin = (((long long)n * g.h + h0) * g.w + w0) * 3;  // may point before the image; only used when in bounds
-            unsigned short v[8];
+    for (int k = 0; k < NS - 1; ++k) {  // (one group per strip, empty when the block has no such strip)
+        const long long tk = blockIdx.x + (long long)k * gridDim.x;
+        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
+        if (tk < nstrips) stem_stage_rows_async(xs, g, total, ahead[k], xrow[k]);
+        cp_async_commit();
+    }
+    int buf = 0;
+    for (long long t = blockIdx.x; t < nstrips; t += gridDim.x, buf = (buf + 1) % NS) {
+        const StemStrip s = ahead[0];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int h = h0 + kr[i], ww = w0 + kt[i];
-                const bool ok = row_ok && koff[i] >= 0 && h >= 0 && h < g.h && ww >= 0 && ww < g.w;
-                v[i] = ok ? xs[origin + koff[i]] : (unsigned short)0;
+        for (int k = 0; k + 1 < NS - 1; ++k) ahead[k] = ahead[k + 1];
+        cp_async_wait_pending<NS - 2>();
+        __syncthreads();  // this strip's rows have landed; the buffer refilled below (the previous strip's) has been consumed
+        const long long tn = t + (long long)(NS - 1) * gridDim.x;
+        if (tn < nstrips) {
+            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
+            stem_stage_rows_async(xs, g, total, ahead[NS - 2], xrow[(buf + NS - 1) % NS]);
+        }
+        cp_async_commit();
+        const int qw = s.q0 + warp * 16;  // first output column of this warp's 16 pixels
+        if (qw < g.wo) {
+            int sh[3], addr[8];
+#pragma unroll
+            for (int r = 0; r < 3; ++r) stem_row_start(g, s, r, sh[r]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) addr[i] = koff[i] + (krow[i] == 0 ? sh[0] : krow[i] == 1 ? sh[1] : sh[2]);
+            const unsigned short* xr = &xrow[buf][0][0] + 6 * (warp * 16 + gq);
+            uint32_t a[2][4];
+            bool row_ok[2];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {  // fragment rows gq and gq + 8
+                row_ok[half] = qw + gq + half * 8 < g.wo;  // (pixels past the row's end compute on defined staged values and are dropped below)
+                unsigned short v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = xr[addr[i] + 48 * half];
+                if (half == 0 && qw + gq == 0) {  // the image's first column: its left neighbours are zero padding
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if ((left_mask >> i) & 1u) v[i] = 0;
+                }
+                // registers of m16n8k16 A: a0 = (row g, k 2t..2t+1), a1 = (row g+8, same k), a2 = (row g, k 2t+8..), a3 = (row g+8, k 2t+8..)
+                a[0][half] = (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+                a[0][2 + half] = (uint32_t)v[2] | ((uint32_t)v[3] << 16);
+                a[1][half] = (uint32_t)v[4] | ((uint32_t)v[5] << 16);
+                a[1][2 + half] = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
             }
-            // registers of m16n8k16 A: a0 = (row g, k 2t..2t+1), a1 = (row g+8, same k), a2 = (row g, k 2t+8..), a3 = (row g+8, k 2t+8..)
-            a[0][half] = (uint32_t)v[0] | ((uint32_t)v[1] << 16);
-            a[0][2 + half] = (uint32_t)v[2] | ((uint32_t)v[3] << 16);
-            a[1][half] = (uint32_t)v[4] | ((uint32_t)v[5] << 16);
-            a[1][2 + half] = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
-        }
-        float acc[NB][4];
-#pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-            acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
-            mma_16816<InT>(acc[nb], a[0], bfrag[0][nb][0], bfrag[0][nb][1]);
-            mma_16816<InT>(acc[nb], a[1], bfrag[1][nb][0], bfrag[1][nb][1]);
-        }
-        // accumulator registers: c0, c1 = (row g, columns 2t, 2t+1), c2, c3 = (row g+8, same columns).  The 16 x COUT tile is one
-        // contiguous run of the output, so it is staged in shared memory and written with coalesced 16-byte stores.
-        OutT* st = stage[threadIdx.x >> 5];
-#pragma unroll
-        for (int half = 0; half < 2; ++half)
+            float acc[NB][4];
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
-                float v0 = acc[nb][2 * half], v1 = acc[nb][2 * half + 1];
-                if (EPI) {
-                    v0 = fmaf(v0, esc[nb][0], esh[nb][0]);
-                    v1 = fmaf(v1, esc[nb][1], esh[nb][1]);
-                    if (ep.act) {
-                        v0 *= sigmoid_f<true>(v0);
-                        v1 *= sigmoid_f<true>(v1);
+                acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
+                mma_16816<InT>(acc[nb], a[0], bfrag[0][nb][0], bfrag[0][nb][1]);
+                mma_16816<InT>(acc[nb], a[1], bfrag[1][nb][0], bfrag[1][nb][1]);
+            }
+            // accumulator registers: c0, c1 = (row g, columns 2t, 2t+1), c2, c3 = (row g+8, same columns)
+            OutT* st = stage[warp];
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) {
+                    float2 v = make_float2(acc[nb][2 * half], acc[nb][2 * half + 1]);
+                    if (EPI) {
+                        v.x = fmaf(v.x, esc[nb][0], esh[nb][0]);
+                        v.y = fmaf(v.y, esc[nb][1], esh[nb][1]);
+                        if (ep.act) v = mul2(v, sigmoid2<true>(v));
+                    }
+                    const uint32_t pk = stem_pack2<OutT>(v);  // the two rounded values: one 4-byte store
+                    *reinterpret_cast<uint32_t*>(st + (gq + half * 8) * COUT + nb * 8 + tq * 2) = pk;
+                    if (!EPI && row_ok[half]) {
+                        const float2 r = stem_unpack2<OutT>(pk);
+                        ssum[nb] = add2(ssum[nb], r);
+                        ssq[nb] = fma2(r, r, ssq[nb]);
                     }
                 }
-                OutT* dst = st + (gq + half * 8) * COUT + nb * 8 + tq * 2;
-                dst[0] = from_f32<OutT>(v0);
-                dst[1] = from_f32<OutT>(v1);
-            }
-        __syncwarp();
-        const long long rows_left = g.m - m0;
-        const int nvec = (int)(rows_left >= 16 ? 16 : rows_left) * COUT / 8;  // 16-byte pieces of the tile that exist
-        for (int v = lane; v < nvec; v += 32) st16(y + (size_t)m0 * COUT + v * 8, ld16(st + v * 8));
-        __syncwarp();
+            __syncwarp();
+            const long long m0 = ((long long)s.n * g.ho + s.p) * g.wo + qw;
+            const int rows = g.wo - qw < 16 ? g.wo - qw : 16;
+            const int nvec = rows * COUT / 8;  // 16-byte pieces of the tile that exist
+            for (int v = lane; v < nvec; v += 32) st16(y + (size_t)m0 * COUT + v * 8, ld16(st + v * 8));
+            __syncwarp();
+        }
     }
-}
-
-// Data gradient, register-tiled: a thread produces the 2 x 4 input pixels (rows 2i, 2i+1, columns 4jp .. 4jp+3) that the
-// six dy pixels (rows i, i+1, columns 2jp .. 2jp+2) feed, so one broadcast read of a channel's 27 filter values serves
-// 54 FMAs (a one-pair-per-thread version read three float4 per nine FMAs and was bound by shared-memory reads: 246 us
-// against 175 us on the 16 x 640 x 640 stem).
-// With pixel (2i+a, 2j+b): (0,0) <- dy[i][j] w11;  (0,1) <- dy[i][j+1] w10 + dy[i][j] w12;  (1,0) <- dy[i+1][j] w01 + dy[i][j] w21;
-// (1,1) <- dy[i+1][j+1] w00 + dy[i+1][j] w02 + dy[i][j+1] w20 + dy[i][j] w22   (w_rt = filter tap (r,t); H and W even).
-template <typename T> __device__ __forceinline__ uint32_t stem_pack2(float a, float b) {
-    const T lo = from_f32<T>(a), hi = from_f32<T>(b);
-    return (uint32_t)(*reinterpret_cast<const unsigned short*>(&lo)) | ((uint32_t)(*reinterpret_cast<const unsigned short*>(&hi)) << 16);
-}
-template <int COUT, typename T = __nv_bfloat16>
-__global__ void __launch_bounds__(128) stem_dgrad_tiled_kernel(const T* __restrict__ dy, const T* __restrict__ w, T* __restrict__ dx, Geom g) {
-    pdl_launch_dependents();
-    pdl_wait();
-    __shared__ __align__(16) float ws[COUT][28];  // ws[c'][tap*3 + c]
-    for (int e = threadIdx.x; e < COUT * STEM_KDIM; e += blockDim.x) ws[e / STEM_KDIM][e % STEM_KDIM] = to_f32(w[e]);
-    __syncthreads();
-    const int npair = (g.wo + 1) / 2;
-    const long long total = (long long)g.n * g.ho * npair;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += stride) {
-        const int jp = (int)(idx % npair);
-        const long long t1 = idx / npair;
-        const int i = (int)(t1 % g.ho), n = (int)(t1 / g.ho);
-        const int j = 2 * jp;
-        const bool row1 = i + 1 < g.ho, col1 = j + 1 < g.wo, col2 = j + 2 < g.wo;
-        const T* r0 = dy + (((size_t)n * g.ho + i) * g.wo + j) * COUT;
-        const T* r1 = r0 + (size_t)g.wo * COUT;
-        float acc[2][4][3];  // [row a][column 0..3 of the 4 produced][channel]
+    if (!EPI && partials) {
+        // lanes with the same tq hold the same columns for different rows: add over gq (fixed butterfly), then over the warps
+        __shared__ float wsum[4][2][COUT];
+        __syncthreads();
 #pragma unroll
-        for (int a = 0; a < 2; ++a)
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = 0.f;
-        Vec16<T> zero;
+            for (int e = 0; e < 2; ++e) {
+                float sv = e ? ssum[nb].y : ssum[nb].x, qv = e ? ssq[nb].y : ssq[nb].x;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) zero.v[e] = from_f32<T>(0.f);
-#pragma unroll 1
-        for (int c0 = 0; c0 < COUT; c0 += 8) {
-            const Vec16<T> v00 = ld16(r0 + c0);
-            const Vec16<T> v01 = col1 ? ld16(r0 + COUT + c0) : zero;
-            const Vec16<T> v02 = col2 ? ld16(r0 + 2 * COUT + c0) : zero;
-            const Vec16<T> v10 = row1 ? ld16(r1 + c0) : zero;
-            const Vec16<T> v11 = (row1 && col1) ? ld16(r1 + COUT + c0) : zero;
-            const Vec16<T> v12 = (row1 && col2) ? ld16(r1 + 2 * COUT + c0) : zero;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float d00 = to_f32(v00.v[e]), d01 = to_f32(v01.v[e]), d02 = to_f32(v02.v[e]);
-                const float d10 = to_f32(v10.v[e]), d11 = to_f32(v11.v[e]), d12 = to_f32(v12.v[e]);
-                float wv[28];
-#pragma unroll
-                for (int q = 0; q < 7; ++q) *reinterpret_cast<float4*>(wv + 4 * q) = *reinterpret_cast<const float4*>(&ws[c0 + e][4 * q]);
-#pragma unroll
-                for (int c = 0; c < 3; ++c) {
-                    const float w00 = wv[0 + c], w01 = wv[3 + c], w02 = wv[6 + c], w10 = wv[9 + c], w11 = wv[12 + c], w12 = wv[15 + c];
-                    const float w20 = wv[18 + c], w21 = wv[21 + c], w22 = wv[24 + c];
-                    // first 2 x 2 group (dy column j), second (dy column j+1)
-                    acc[0][0][c] = fmaf(d00, w11, acc[0][0][c]);
-                    acc[0][1][c] = fmaf(d01, w10, fmaf(d00, w12, acc[0][1][c]));
-                    acc[1][0][c] = fmaf(d10, w01, fmaf(d00, w21, acc[1][0][c]));
-                    acc[1][1][c] = fmaf(d11, w00, fmaf(d10, w02, fmaf(d01, w20, fmaf(d00, w22, acc[1][1][c]))));
-                    acc[0][2][c] = fmaf(d01, w11, acc[0][2][c]);
-                    acc[0][3][c] = fmaf(d02, w10, fmaf(d01, w12, acc[0][3][c]));
-                    acc[1][2][c] = fmaf(d11, w01, fmaf(d01, w21, acc[1][2][c]));
-                    acc[1][3][c] = fmaf(d12, w00, fmaf(d11, w02, fmaf(d02, w20, fmaf(d01, w22, acc[1][3][c]))));
+                for (int o = 4; o < 32; o <<= 1) {
+                    sv += __shfl_xor_sync(0xffffffffu, sv, o);
+                    qv += __shfl_xor_sync(0xffffffffu, qv, o);
+                }
+                if (gq == 0) {
+                    wsum[warp][0][nb * 8 + tq * 2 + e] = sv;
+                    wsum[warp][1][nb * 8 + tq * 2 + e] = qv;
                 }
             }
-        }
-        // rows 2i and 2i+1, columns 4jp .. 4jp+3 (the last two only when dy column j+1 exists): 12 bf16 = 24 bytes per row, 8-byte aligned
-#pragma unroll
-        for (int a = 0; a < 2; ++a) {
-            T* o = dx + (((size_t)n * g.h + 2 * i + a) * g.w + 4 * (size_t)jp) * 3;
-            uint32_t* o2 = reinterpret_cast<uint32_t*>(o);
-            o2[0] = stem_pack2<T>(acc[a][0][0], acc[a][0][1]);
-            o2[1] = stem_pack2<T>(acc[a][0][2], acc[a][1][0]);
-            o2[2] = stem_pack2<T>(acc[a][1][1], acc[a][1][2]);
-            if (col1) {
-                o2[3] = stem_pack2<T>(acc[a][2][0], acc[a][2][1]);
-                o2[4] = stem_pack2<T>(acc[a][2][2], acc[a][3][0]);
-                o2[5] = stem_pack2<T>(acc[a][3][1], acc[a][3][2]);
-            }
+        __syncthreads();
+        for (int e = threadIdx.x; e < 2 * COUT; e += blockDim.x) {
+            const int which = e / COUT, c = e - which * COUT;
+            partials[(size_t)blockIdx.x * 2 * COUT + e] = ((wsum[0][which][c] + wsum[1][which][c]) + wsum[2][which][c]) + wsum[3][which][c];
         }
     }
 }
 
-// ---- tensor-core weight gradient for the stem: dw[c'][k] = sum over pixels of dy[pixel][c'] * patch[pixel][k] as
-// mma.sync tiles of 16 pixels (the reduction index): A = dy^T (the 16 x COUT piece of dy is one contiguous run: staged in
-// shared memory with 16-byte loads and read back transposed with ldmatrix), B = the pixels' patch values (gathered like
-// in the forward kernel).  A block sums its pixel range; its four warps are combined in a fixed order into the block's
-// slice of `partial` [gridDim.x][COUT][27].
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
-    const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_row);
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
-}
+// Data gradient as mma.sync tiles.  For dy position (i, j) the four input pixels (2i+a, 2j+b) receive
+//   (0,0) <- dy[i][j] w11;  (0,1) <- dy[i][j+1] w10 + dy[i][j] w12;  (1,0) <- dy[i+1][j] w01 + dy[i][j] w21;
+//   (1,1) <- dy[i+1][j+1] w00 + dy[i+1][j] w02 + dy[i][j+1] w20 + dy[i][j] w22        (w_rt = filter tap (r,t)),
+// i.e. per parity class a GEMM [16 positions x COUT] x [COUT x 3] per tap with the dy tile shifted by (0|1, 0|1): 27 MMAs
+// (N padded from 3 to 8) per 16 positions.  A block stages rows i and i+1 of a 64-position strip (plus one column) in
+// shared memory with 16-byte loads (pixel pitch 112 bytes: conflict-free ldmatrix), the 27 filter fragments stay in
+// registers, and the 2 x 32 output pixels of a warp are staged and written as 4-byte words (coalesced).
+constexpr int STEM_DYPITCH = 56;  // elements per staged dy pixel (48 channels + padding)
 template <int COUT, typename T = __nv_bfloat16>
-__global__ void __launch_bounds__(128) stem_wgrad_mma_kernel(const T* __restrict__ x, const T* __restrict__ dy,
-                                                             float* __restrict__ partial, Geom g, long long pix_per_block) {
+__global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restrict__ dy, const T* __restrict__ w, T* __restrict__ dx, Geom g) {
+    pdl_launch_dependents();
+    pdl_wait();
+    static_assert(COUT % 16 == 0 && COUT + 8 <= STEM_DYPITCH, "whole k-steps; pitch holds a pixel");
+    constexpr int KS = COUT / 16;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
+    const unsigned short* wsrc = reinterpret_cast<const unsigned short*>(w);
+    // B fragments: for tap (r,t) and k-step ks, element (k = channel c', n = input channel c): w[c'][r][t][c]; n >= 3 is padding
+    uint32_t bfrag[STEM_TAPS][KS][2];
+#pragma unroll
+    for (int tap = 0; tap < STEM_TAPS; ++tap)
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int c0 = ks * 16 + j * 8 + tq * 2;
+                const uint32_t lo = gq < 3 ? wsrc[c0 * STEM_KDIM + tap * 3 + gq] : 0u, hi = gq < 3 ? wsrc[(c0 + 1) * STEM_KDIM + tap * 3 + gq] : 0u;
+                bfrag[tap][ks][j] = lo | (hi << 16);
+            }
+    constexpr int NS = 3;  // ring of staged strips
+    __shared__ __align__(16) T dys[NS][2][(STEM_TQ + 1) * STEM_DYPITCH];  // [buffer][row i / i+1][pixel][channel]
+    __shared__ __align__(16) T outs[4][2][32 * 3];
+    const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
+    const long long nstrips = stem_num_strips(g);
+    constexpr int VPP = COUT / 8;  // 16-byte vectors per pixel
+    // asynchronous staging of dy[i..i+1][q0 .. q0+64][:] (zeros past the last row / column)
+    auto stage_async = [&](const StemStrip& s, T(*dst)[(STEM_TQ + 1) * STEM_DYPITCH]) {
+        // a row's 65 pixels are one contiguous run of 65 * VPP vectors in global memory; in shared memory pixels are
+        // STEM_DYPITCH apart
+        const T* row0 = dy + (((size_t)s.n * g.ho + s.p) * g.wo + s.q0) * COUT;
+        const int npx = g.wo - s.q0;  // pixels of the row from q0 on
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const bool row_ok = s.p + r < g.ho;
+            const T* src = row0 + (size_t)r * g.wo * COUT;
+            for (int u = threadIdx.x; u < (STEM_TQ + 1) * VPP; u += blockDim.x) {
+                const int px = u / VPP;
+                const bool ok = row_ok && px < npx;
+                cp_async16_zfill(&dst[r][u * 8 + px * (STEM_DYPITCH - COUT)], ok ? src + u * 8 : dy, ok ? 16 : 0);
+            }
+        }
+    };
+    StemStrip ahead[NS - 1];  // the strips whose rows are in flight, decoded once (p = dy row i, q0 = first dy column)
+#pragma unroll
+    for (int k = 0; k < NS - 1; ++k) {
+        const long long tk = blockIdx.x + (long long)k * gridDim.x;
+        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
+        if (tk < nstrips) stage_async(ahead[k], dys[k]);
+        cp_async_commit();
+    }
+    int buf = 0;
+    for (long long t = blockIdx.x; t < nstrips; t += gridDim.x, buf = (buf + 1) % NS) {
+        const StemStrip s = ahead[0];
+#pragma unroll
+        for (int k = 0; k + 1 < NS - 1; ++k) ahead[k] = ahead[k + 1];
+        cp_async_wait_pending<NS - 2>();
+        __syncthreads();  // this strip's rows have landed; the buffer refilled below has been consumed
+        const long long tn = t + (long long)(NS - 1) * gridDim.x;
+        if (tn < nstrips) {
+            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
+            stage_async(ahead[NS - 2], dys[(buf + NS - 1) % NS]);
+        }
+        cp_async_commit();
+        const int jw = s.q0 + warp * 16;  // first dy column of this warp's 16 positions
+        if (jw < g.wo) {
+            float acc[4][4];  // parity class a*2+b
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.f;
+            const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: matrix and row this lane addresses
+            const T* d0 = dys[buf][0];
+            const T* d1 = dys[buf][1];
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t a00[4], a01[4], a10[4], a11[4];  // dy tile shifted by (di, dj)
+                const int px = warp * 16 + mr + (mi & 1) * 8, ko = ks * 16 + (mi >> 1) * 8;
+                ldmatrix_x4(a00, &d0[px * STEM_DYPITCH + ko]);
+                ldmatrix_x4(a01, &d0[(px + 1) * STEM_DYPITCH + ko]);
+                ldmatrix_x4(a10, &d1[px * STEM_DYPITCH + ko]);
+                ldmatrix_x4(a11, &d1[(px + 1) * STEM_DYPITCH + ko]);
+                // tap index = r*3 + t
+                mma_16816<T>(acc[0], a00, bfrag[4][ks][0], bfrag[4][ks][1]);  // (0,0): w11
+                mma_16816<T>(acc[1], a01, bfrag[3][ks][0], bfrag[3][ks][1]);  // (0,1): dy[i][j+1] w10
+                mma_16816<T>(acc[1], a00, bfrag[5][ks][0], bfrag[5][ks][1]);  //        dy[i][j]   w12
+                mma_16816<T>(acc[2], a10, bfrag[1][ks][0], bfrag[1][ks][1]);  // (1,0): dy[i+1][j] w01
+                mma_16816<T>(acc[2], a00, bfrag[7][ks][0], bfrag[7][ks][1]);  //        dy[i][j]   w21
+                mma_16816<T>(acc[3], a11, bfrag[0][ks][0], bfrag[0][ks][1]);  // (1,1): dy[i+1][j+1] w00
+                mma_16816<T>(acc[3], a10, bfrag[2][ks][0], bfrag[2][ks][1]);  //        dy[i+1][j]   w02
+                mma_16816<T>(acc[3], a01, bfrag[6][ks][0], bfrag[6][ks][1]);  //        dy[i][j+1]   w20
+                mma_16816<T>(acc[3], a00, bfrag[8][ks][0], bfrag[8][ks][1]);  //        dy[i][j]     w22
+            }
+            // accumulator registers: c0, c1 = (position gq, channels 2tq, 2tq+1), c2, c3 = (position gq+8, same): channels 0..2 exist
+            T(*o)[32 * 3] = outs[warp];
+            if (tq < 2) {
+#pragma unroll
+                for (int a = 0; a < 2; ++a)
+#pragma unroll
+                    for (int b = 0; b < 2; ++b)
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int pos = gq + half * 8;
+                            T* dst = &o[a][(2 * pos + b) * 3 + tq * 2];
+                            dst[0] = from_f32<T>(acc[a * 2 + b][2 * half]);
+                            if (tq == 0) dst[1] = from_f32<T>(acc[a * 2 + b][2 * half + 1]);
+                        }
+            }
+            __syncwarp();
+            const int npos = g.wo - jw < 16 ? g.wo - jw : 16;
+            const int nwords = npos * 3;  // 4-byte words per output row segment (2*npos pixels x 3 channels x 2 bytes)
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+                uint32_t* dst = reinterpret_cast<uint32_t*>(dx + (((size_t)s.n * g.h + 2 * s.p + a) * g.w + 2 * (size_t)jw) * 3);
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(o[a]);
+                for (int v = lane; v < nwords; v += 32) dst[v] = src[v];
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// Weight gradient: dw[c'][k] = sum over pixels of dy[pixel][c'] * patch[pixel][k] as mma.sync tiles of 16 pixels (the
+// reduction index): A = dy^T (the 16 x COUT piece of dy is one contiguous run: staged in shared memory with 16-byte loads
+// and read back transposed with ldmatrix), B = the pixels' patch values cut out of the staged input rows.  A block sums
+// the strips it is dealt; its four warps are combined in a fixed order into the block's slice of `partial`
+// [gridDim.x][COUT][27].
+template <int COUT, typename T = __nv_bfloat16>
+__global__ void __launch_bounds__(128, 4) stem_wgrad_mma_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, Geom g) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 16 == 0, "whole m-blocks");
     constexpr int MB = COUT / 16, NBK = 4;  // accumulator blocks: MB x 16 channels by NBK x 8 filter positions (27 padded to 32)
-    __shared__ __align__(16) T dys[4][16 * COUT];
-    __shared__ float red[4][COUT][33];
+    constexpr int NS = 4;  // ring of staged strips
+    struct Ring {
+        unsigned short xrow[NS][3][STEM_XPITCH];
+        T dys[NS][STEM_TQ * COUT];  // the strip's 64 x COUT piece of dy (one contiguous run), per buffer
+    };
+    typedef float Red[COUT][33];
+    constexpr size_t kRaw = sizeof(Ring) > 4 * sizeof(Red) ? sizeof(Ring) : 4 * sizeof(Red);
+    __shared__ __align__(16) unsigned char raw[kRaw];  // the ring while strips are processed, then the four warps' sums
+    Ring& ring = *reinterpret_cast<Ring*>(raw);
+    Red* red = reinterpret_cast<Red*>(raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
-    // B fragment element (k = pixel 2t.., n = 8*nb + g): filter position n of the pixel's patch
-    int koff[NBK], kr[NBK], kt[NBK];
+    // B fragment element (k = pixel 2t.., n = 8*nb + g): filter position n of the pixel's patch -> filter row, offset in the row
+    // (positions n >= 27 are accumulator columns that are never stored: they read the patch's centre)
+    int krow[NBK], koff[NBK];
+    unsigned left_mask = 0;  // bit nb: the position lies in the patch's left column (zero padding for the image's first column)
 #pragma unroll
     for (int nb = 0; nb < NBK; ++nb) {
-        const int k = nb * 8 + gq, r = k / 9, kp = k - r * 9;
-        kr[nb] = r;
-        kt[nb] = kp / 3;
-        koff[nb] = k < STEM_KDIM ? r * g.w * 3 + kp : -1;
+        const int k = nb * 8 + gq;
+        krow[nb] = k < STEM_KDIM ? k / 9 : 1;
+        koff[nb] = krow[nb] * STEM_XPITCH + (k < STEM_KDIM ? k % 9 : 3);
+        if (k < STEM_KDIM && k % 9 < 3) left_mask |= 1u << nb;
     }
     float acc[MB][NBK][4];
 #pragma unroll
     for (int a = 0; a < MB; ++a)
 #pragma unroll
         for (int b = 0; b < NBK; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = acc[a][b][3] = 0.f;
-    const long long m_begin = (long long)blockIdx.x * pix_per_block;
-    const long long m_end = (m_begin + pix_per_block < g.m) ? m_begin + pix_per_block : g.m;
-    T* st = dys[warp];
-    for (long long m0 = m_begin + warp * 16; m0 < m_end; m0 += 64) {
-        const int np = (int)((m_end - m0 < 16) ? (m_end - m0) : 16);  // pixels of this tile inside the block's range
-        // stage dy[m0 .. m0+15][:] (zeros past the range)
-        for (int v = lane; v < 16 * COUT / 8; v += 32) {
-            Vec16<T> q;
-            if (v * 8 < np * COUT) {
-                q = ld16(dy + (size_t)m0 * COUT + v * 8);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) q.v[i] = from_f32<T>(0.f);
-            }
-            st16(st + v * 8, q);
+    const int total = g.n * g.h * g.w * 3;
+    const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
+    const long long nstrips = stem_num_strips(g);
+    // asynchronous staging of a strip: the three input rows and dy[strip][:] (zeros past the row's end: those pixels then
+    // contribute nothing)
+    auto stage_async = [&](const StemStrip& s, int b) {
+        stem_stage_rows_async(xs, g, total, s, ring.xrow[b]);
+        const size_t m0 = ((size_t)s.n * g.ho + s.p) * g.wo + s.q0;
+        const int np = g.wo - s.q0 < STEM_TQ ? g.wo - s.q0 : STEM_TQ;
+        for (int v = threadIdx.x; v < STEM_TQ * COUT / 8; v += blockDim.x) {
+            const bool ok = v * 8 < np * COUT;
+            cp_async16_zfill(&ring.dys[b][v * 8], ok ? dy + m0 * COUT + v * 8 : dy, ok ? 16 : 0);
         }
-        // B fragments: four pixels of the tile (2t, 2t+1, 2t+8, 2t+9) x NBK filter positions
-        uint32_t bfr[NBK][2];
-        unsigned short v4[4][NBK];
+    };
+    StemStrip ahead[NS - 1];  // the strips whose data are in flight, decoded once
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int pl = tq * 2 + (j & 1) + (j >> 1) * 8;
-            const bool row_ok = pl < np;
-            const unsigned mm = row_ok ? (unsigned)(m0 + pl) : 0u;
-            const unsigned t1 = mm / (unsigned)g.wo;
-            const int q = (int)(mm - t1 * (unsigned)g.wo);
-            const int n = (int)(t1 / (unsigned)g.ho), p = (int)(t1 - (unsigned)n * (unsigned)g.ho);
-            const int h0 = 2 * p - 1, w0 = 2 * q - 1;
-            const long long origin = (((long long)n * g.h + h0) * g.w + w0) * 3;
+    for (int k = 0; k < NS - 1; ++k) {
+        const long long tk = blockIdx.x + (long long)k * gridDim.x;
+        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
+        if (tk < nstrips) stage_async(ahead[k], k);
+        cp_async_commit();
+    }
+    int buf = 0;
+    for (long long t = blockIdx.x; t < nstrips; t += gridDim.x, buf = (buf + 1) % NS) {
+        const StemStrip s = ahead[0];
+#pragma unroll
+        for (int k = 0; k + 1 < NS - 1; ++k) ahead[k] = ahead[k + 1];
+        cp_async_wait_pending<NS - 2>();
+        __syncthreads();
+        const long long tn = t + (long long)(NS - 1) * gridDim.x;
+        if (tn < nstrips) {
+            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
+            stage_async(ahead[NS - 2], (buf + NS - 1) % NS);
+        }
+        cp_async_commit();
+        const int qw = s.q0 + warp * 16;
+        if (qw < g.wo) {
+            int sh[3], addr[NBK];
+#pragma unroll
+            for (int r = 0; r < 3; ++r) stem_row_start(g, s, r, sh[r]);
+#pragma unroll
+            for (int nb = 0; nb < NBK; ++nb) addr[nb] = koff[nb] + (krow[nb] == 0 ? sh[0] : krow[nb] == 1 ? sh[1] : sh[2]);
+            const unsigned short* xr = &ring.xrow[buf][0][0] + 6 * (warp * 16 + tq * 2);
+            const T* st = &ring.dys[buf][warp * 16 * COUT];
+            // B fragments: four pixels of the tile (2t, 2t+1, 2t+8, 2t+9) x NBK filter positions.  (Pixels past the row's
+            // end meet zero dy rows, so whatever defined values they read contribute nothing.)
+            uint32_t bfr[NBK][2];
+            unsigned short v4[4][NBK];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) v4[j][nb] = xr[addr[nb] + 6 * ((j & 1) + (j >> 1) * 8)];
+            }
+            if (qw + tq == 0) {  // the image's first column (pixel j = 0 of this lane): its left neighbours are zero padding
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb)
+                    if ((left_mask >> nb) & 1u) v4[0][nb] = 0;
+            }
 #pragma unroll
             for (int nb = 0; nb < NBK; ++nb) {
-                const int h = h0 + kr[nb], ww = w0 + kt[nb];
-                const bool ok = row_ok && koff[nb] >= 0 && h >= 0 && h < g.h && ww >= 0 && ww < g.w;
-                v4[j][nb] = ok ? xs[origin + koff[nb]] : (unsigned short)0;
+                bfr[nb][0] = (uint32_t)v4[0][nb] | ((uint32_t)v4[1][nb] << 16);
+                bfr[nb][1] = (uint32_t)v4[2][nb] | ((uint32_t)v4[3][nb] << 16);
+            }
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                // A = dy^T: matrix i of the x4 load is [8 pixels][8 channels] of the staged tile, read transposed:
+                // i = 0: pixels 0-7, channels 16mb+0..7 (a0), 1: pixels 0-7, channels +8 (a1), 2: pixels 8-15, channels +0 (a2), 3: pixels 8-15, +8 (a3)
+                uint32_t afr[4];
+                const int mi = lane >> 3, mr = lane & 7;
+                ldmatrix_x4_trans(afr, st + (mr + (mi >> 1) * 8) * COUT + mb * 16 + (mi & 1) * 8);
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) mma_16816<T>(acc[mb][nb], afr, bfr[nb][0], bfr[nb][1]);
             }
         }
-#pragma unroll
-        for (int nb = 0; nb < NBK; ++nb) {
-            bfr[nb][0] = (uint32_t)v4[0][nb] | ((uint32_t)v4[1][nb] << 16);
-            bfr[nb][1] = (uint32_t)v4[2][nb] | ((uint32_t)v4[3][nb] << 16);
-        }
-        __syncwarp();  // the staged dy rows are complete
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-            // A = dy^T: matrix i of the x4 load is [8 pixels][8 channels] of the staged tile, read transposed:
-            // i = 0: pixels 0-7, channels 16mb+0..7 (a0), 1: pixels 0-7, channels +8 (a1), 2: pixels 8-15, channels +0 (a2), 3: pixels 8-15, +8 (a3)
-            uint32_t afr[4];
-            const int mi = lane >> 3, mr = lane & 7;
-            ldmatrix_x4_trans(afr, st + (mr + (mi >> 1) * 8) * COUT + mb * 16 + (mi & 1) * 8);
-#pragma unroll
-            for (int nb = 0; nb < NBK; ++nb) mma_16816<T>(acc[mb][nb], afr, bfr[nb][0], bfr[nb][1]);
-        }
-        __syncwarp();  // before the next tile overwrites the staged rows
     }
     // accumulator registers: c0, c1 = (channel 16mb+g, positions 8nb+2t, +1), c2, c3 = (channel 16mb+g+8, same positions)
+    cp_async_wait_pending<0>();
+    __syncthreads();  // every warp is done with the ring: its space now holds the warps' sums
 #pragma unroll
     for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
