@@ -129,10 +129,13 @@ __device__ __forceinline__ void bn_finalize_channel(const float* __restrict__ pa
     double s, q;
     warp_sum_partials2<L2>(partials, nparts, C, c, lane, s, q);
     if (lane == 0) {
-        const double mu = s / M;
-        double var = q / M - mu * mu;
+        // (this chain sits on the critical path of the forward kernel's tail: one reciprocal serves all divisions by M,
+        // and the inverse square root is the library's, accurate to within two units in the last place of fp64)
+        const double inv_m = 1.0 / M;
+        const double mu = s * inv_m;
+        double var = q * inv_m - mu * mu;
         if (var < 0.0) var = 0.0;
-        const double is = 1.0 / sqrt(var + (double)eps);
+        const double is = rsqrt(var + (double)eps);
         if (mean) mean[c] = (float)mu;
         if (invstd) invstd[c] = (float)is;
         if (scale) {
@@ -275,15 +278,16 @@ __device__ __forceinline__ void bn_bwd_finalize_channel(const float* __restrict_
     warp_sum_partials2<L2>(partials, nparts, C, c, lane, s0, s1);
     if (lane == 0) {
         const double mu = (double)mu_f, is = (double)is_f;
+        const double inv_m = 1.0 / M;
         const double dg = is * (s1 - mu * s0);
         const double a = (double)ga * is;
-        const double p1 = a * is * dg / M;
+        const double p1 = a * is * dg * inv_m;
         dbeta[c] = (float)s0;
         dgamma[c] = (float)dg;
         coef[c] = (float)a;
         coef[C + c] = (float)((double)be - mu * a);
         coef[2 * C + c] = (float)p1;
-        coef[3 * C + c] = (float)(p1 * mu - a * s0 / M);
+        coef[3 * C + c] = (float)(p1 * mu - a * s0 * inv_m);
     }
 }
 

@@ -343,8 +343,11 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     if (CG2) ptx::cluster_sync_all(); else __syncthreads();  // barriers of both CTAs are initialised before any remote arrive
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();  // everything above touched only shared memory, TMEM and kernel parameters
+    // Everything above touched only shared memory, TMEM and kernel parameters.  Each role waits for the previous kernel
+    // (griddepcontrol.wait) itself, as late as it can: the producers after they have read their parameters, right before
+    // the first load; the epilogue warps before their first access to global memory; the MMA issuer touches none.
     if (EPI) {
+        pdl_wait();
         // per-channel coefficients of the fused epilogue, in fp64 like the training-mode finalize
         // (stored per channel pair as scale, scale, shift, shift: the operands of the packed fp32 multiply-add)
         for (int c = threadIdx.x; c < p.ldo; c += IG_THREADS) {
@@ -374,6 +377,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         // pairs: loads of both CTAs are counted on the rank-0 CTA's full barriers (the MMA issuer waits there)
         const uint32_t base_u32 = ptx::smem_u32(isA ? sA : sB);
         const uint32_t full_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(full), 0u) : ptx::smem_u32(full);
+        pdl_wait();
         for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
             int cls, lt;
             igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
@@ -542,6 +546,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         bool store_pending = false;
         uint8_t* outb = static_cast<uint8_t*>(p.out);
         const uint32_t tempty_u32 = CG2 ? ptx::mapa_u32(ptx::smem_u32(tempty), 0u) : 0u;  // the issuer's barriers (rank 0)
+        pdl_wait();
         for (int tile = worker; tile < total_tiles; tile += nworkers) {
             int cls, lt;
             igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
@@ -872,8 +877,8 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
         // and writes only half of B in shared memory.  Measured per layer on B200: 3x3 layers with at least 96 reduction
         // channels gain 5-15 %; 1x1 layers (one k-block group per tile, epilogue-bound) lose 5-10 % to the extra
         // cluster synchronisation, as do 3x3 layers with one k-block per tap and the stride-2 data gradients (1-4 taps
-        // per parity class) below 384 channels.
-        const bool pair_pays = ntaps > 1 && Ca >= 96 && (nclasses == 1 || Ca >= 384);
+        // per parity class) below 384 channels; 1x1 layers with 960 and more input channels gain 1.5-2 us again.
+        const bool pair_pays = (ntaps > 1 && Ca >= 96 && (nclasses == 1 || Ca >= 384)) || (ntaps == 1 && Ca >= 960);
         const bool cg2 = bn % 32 == 0 && (getenv("NB_TC_CG2") ? atoi(getenv("NB_TC_CG2")) != 0 : pair_pays);
         int mh = 1;
         if (4 * acc_stride <= 512) {
