@@ -126,6 +126,23 @@ nb_status nb_cbs_workspace_bytes(nb_cbs_plan plan, size_t* fwd_bytes, size_t* bw
  * (their TMA descriptors carry the pitch).  The evaluation-mode, plain and host-buffer calls refuse a pitched plan. */
 nb_status nb_cbs_plan_set_pitches(nb_cbs_plan plan, int64_t ld_x, int64_t ld_a, int64_t ld_g);
 
+/* Residual connection performed by the block that feeds it (the bottlenecks of the detector's C2f units, Sec. 6): with
+ * res != NULL, nb_conv_bn_silu_fwd of this plan writes a_out = SiLU(z) + res, where res is a tensor of a_out's shape and
+ * type, dense or a channel slice with pixels ld_res elements apart (0 = dense); the sum is formed in fp32 and rounded
+ * once.  Everything the backward calls need (y_saved, mean, invstd) is unchanged: the gradient of the sum is the
+ * gradient of both summands.  res must stay valid while calls of the plan may run; NULL restores the plain block.
+ * The evaluation-mode, plain and host-buffer calls refuse such a plan. */
+nb_status nb_cbs_plan_set_fwd_residual(nb_cbs_plan plan, const void* res, int64_t ld_res);
+
+/* Gradient accumulation at fan-out without a separate pass: declare that, in nb_conv_bn_silu_bwd_data of this plan, dx is
+ * a channel slice of a wider NHWC tensor (pointer = the slice's first channel, pixels ld_dx elements apart; 0 = dense) and,
+ * with accumulate = 1, that the data gradient is ADDED to what dx holds instead of overwriting it (a tensor with several
+ * consumers receives the sum of their gradients, Sec. 6 dataflow; each addition rounds once to the 16-bit type, exactly as
+ * a separate accumulation pass would).  The epilogue then issues TMA reductions instead of TMA stores.
+ * NB_ERR_UNSUPPORTED unless the plan's data gradient runs on the tensor-core kernel of a stride-1 layer; ld_dx at least
+ * c_in and a multiple of 8 elements.  (0, 0) restores the default.  The plain and host-buffer calls refuse such a plan. */
+nb_status nb_cbs_plan_set_dx_target(nb_cbs_plan plan, int64_t ld_dx, int32_t accumulate);
+
 /* Which implementation each convolution of this plan runs on: writes three ints (fprop, dgrad, wgrad),
  * 1 = tcgen05 tensor-core kernel, 0 = CUDA-core kernel. */
 nb_status nb_cbs_plan_paths(nb_cbs_plan plan, int32_t* paths3);

@@ -191,10 +191,12 @@ template <int V> __device__ __forceinline__ void load_params(const float* __rest
 }
 
 // ------------------------------------------------------------------ a = SiLU(y*scale + shift)  (ACT = false: no SiLU)
-template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false>
+// RES: a = SiLU(...) + res with res a (possibly pitched) tensor of the output's type -- the residual connection of a
+// bottleneck performed by the block that feeds it; the sum is formed in fp32 and rounded once.
+template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false, bool RES = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
                                                              long long total_vecs, int C, const float* __restrict__ scale,
-                                                             const float* __restrict__ shift, long long ld_a) {
+                                                             const float* __restrict__ shift, long long ld_a, const AT* __restrict__ res, long long ld_r) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -210,14 +212,19 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
     const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     long long oa = PITCHED ? (v0 / cgs) * ld_a + (long long)cg * V : v0 * V;  // (dense: the flat offset, no division)
     const long long oa_step = PITCHED ? (stride / cgs) * ld_a : stride * V;
-    for (long long v = v0; v < total_vecs; v += stride, oa += oa_step) {
+    long long orr = RES ? (v0 / cgs) * ld_r + (long long)cg * V : 0;
+    const long long or_step = RES ? (stride / cgs) * ld_r : 0;
+    for (long long v = v0; v < total_vecs; v += stride, oa += oa_step, orr += or_step) {
         if (v + 2 * stride < total_vecs) asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));  // see the reduce kernel
         const Vec16<YT> q = ld16(y + v * V);
-        Vec16<AT> o;
+        Vec16<AT> o, r;
+        if (RES) r = ld16(res + orr);
 #pragma unroll
         for (int j = 0; j < V / 2; ++j) {
             const float2 z = fma2(pair_to_f32(q.v + 2 * j), sc[j], sh[j]);
-            pair_from_f32(o.v + 2 * j, ACT ? mul2(z, sigmoid2<FAST>(z)) : z);
+            float2 out = ACT ? mul2(z, sigmoid2<FAST>(z)) : z;
+            if (RES) out = add2(out, pair_to_f32(r.v + 2 * j));
+            pair_from_f32(o.v + 2 * j, out);
         }
         st16(a + oa, o);
     }

@@ -70,6 +70,10 @@ struct nb_cbs_plan_s {
     long long wg_chunk;
     TcPlan tc;       // tensor-core kernel choices (all disabled when unsupported or forced off)
     long long ld_a = 0, ld_g = 0;  // row pitch (elements) of a_out in the forward call and of g in the backward call (set by nb_cbs_plan_set_pitches; default c_out)
+    const void* fwd_res = nullptr;  // residual added to the forward call's output (nb_cbs_plan_set_fwd_residual) and its row pitch
+    long long ld_res = 0;
+    long long ld_dx = 0;           // row pitch of dx in the data-gradient call and whether dx is added to (nb_cbs_plan_set_dx_target)
+    bool dx_accumulate = false;
     bool pitched = false;
     bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or an occupancy query that failed)
     int expire_next_ms = 0;     // nb_cbs_debug_expire_next_wait: the next grid-barrier launch waits for one block too many, for at most this long
@@ -146,16 +150,26 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
     return launch_ok("bn_finalize");
 }
 
+// res != NULL (training forward with SiLU only): a = SiLU(...) + res, res with row pitch ld_res elements.
 template <typename YT, typename AT, bool FAST, bool ACT = true>
-nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st, long long ld_a = 0) {
+nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st, long long ld_a = 0,
+                    const void* res = nullptr, long long ld_res = 0) {
     const EwCfg& e = p->ew;
+    const int C = p->g.c_out;
     SiteTimer tm(p, SITE_APPLY, st);
+    if constexpr (ACT) {
+        if (res) {
+            launch_k(bn_silu_apply_kernel<YT, AT, FAST, true, true, true>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
+                     e.total_vecs, C, scale, shift, ld_a ? ld_a : (long long)C, static_cast<const AT*>(res), ld_res ? ld_res : (long long)C);
+            return launch_ok("bn_silu_apply (+ residual)");
+        }
+    }
     if (ld_a)
         launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, true>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
-                 e.total_vecs, p->g.c_out, scale, shift, ld_a);
+                 e.total_vecs, C, scale, shift, ld_a, static_cast<const AT*>(nullptr), 0LL);
     else
         launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, false>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
-                 e.total_vecs, p->g.c_out, scale, shift, (long long)p->g.c_out);
+                 e.total_vecs, C, scale, shift, (long long)C, static_cast<const AT*>(nullptr), 0LL);
     return launch_ok("bn_silu_apply");
 }
 
@@ -461,6 +475,32 @@ nb_status nb_cbs_plan_set_pitches(nb_cbs_plan p, int64_t ld_x, int64_t ld_a, int
     return NB_OK;
 }
 
+nb_status nb_cbs_plan_set_fwd_residual(nb_cbs_plan p, const void* res, int64_t ld_res) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(res, true);
+    const int vec = is_f32(p) ? 4 : 8;
+    if (ld_res == p->g.c_out) ld_res = 0;
+    if (res && ld_res != 0 && (ld_res < p->g.c_out || ld_res % vec != 0))
+        return fail(NB_ERR_INVALID_ARG, "ld_res must be 0 (dense) or at least c_out and a multiple of %d elements", vec);
+    p->fwd_res = res;
+    p->ld_res = res ? ld_res : 0;
+    return NB_OK;
+}
+
+nb_status nb_cbs_plan_set_dx_target(nb_cbs_plan p, int64_t ld_dx, int32_t accumulate) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    if (accumulate != 0 && accumulate != 1) return fail(NB_ERR_INVALID_ARG, "accumulate must be 0 or 1, got %d", accumulate);
+    if (ld_dx == p->g.c_in) ld_dx = 0;
+    if (ld_dx != 0 && (ld_dx < p->g.c_in || ld_dx % 8 != 0)) return fail(NB_ERR_INVALID_ARG, "ld_dx must be 0 (dense) or at least c_in and a multiple of 8 elements");
+    if ((ld_dx != 0 || accumulate) && (is_f32(p) || p->stem || !p->tc.dgrad || p->g.stride != 1))
+        return fail(NB_ERR_UNSUPPORTED, "a pitched or accumulating dx needs the tensor-core data gradient of a stride-1 layer (its epilogue stores through TMA)");
+    p->ld_dx = ld_dx;
+    p->dx_accumulate = accumulate != 0;
+    return NB_OK;
+}
+
 nb_status nb_cbs_plan_paths(nb_cbs_plan p, int32_t* paths3) {
     g_err.clear();
     if (!p || !paths3) return fail(NB_ERR_INVALID_ARG, "NULL argument");
@@ -572,8 +612,8 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     }
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
-    if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st, p->ld_a);
-    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a));
+    if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st, p->ld_a, p->fwd_res, p->ld_res);
+    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a, p->fwd_res, p->ld_res));
 }
 
 namespace {
@@ -627,7 +667,7 @@ nb_status nb_conv_bn_silu_infer(nb_cbs_plan p, const void* x, const void* w, con
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(gamma); NB_CHECK_PTR(beta); NB_CHECK_PTR(running_mean); NB_CHECK_PTR(running_var);
     NB_CHECK_PTR(a_out);
-    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
+    if (p->pitched || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches or a residual set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
     DeviceGuard on_device(p->device);
     return run_infer(p, x, w, gamma, beta, running_mean, running_var, 1, a_out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
@@ -639,7 +679,7 @@ nb_status nb_conv_bias_act(nb_cbs_plan p, const void* x, const void* w, const fl
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(w); NB_CHECK_PTR(bias, true); NB_CHECK_PTR(out);
     if (act != 0 && act != 1) return fail(NB_ERR_INVALID_ARG, "act must be 0 (none) or 1 (SiLU), got %d", act);
-    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
+    if (p->pitched || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches or a residual set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->infer_bytes));
     DeviceGuard on_device(p->device);
     return run_infer(p, x, w, nullptr, bias, nullptr, nullptr, act, out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
@@ -718,7 +758,7 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     if (p->tc.dgrad) {
         SiteTimer tm(p, SITE_DGRAD, st);
         const long long l0 = p->tc.launches;
-        const nb_status ts = tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st, true);
+        const nb_status ts = tc_dgrad(&p->tc, p->g, dy_out, w, dx, ws + p->off_wt, p->status, st, true, p->ld_dx, p->dx_accumulate);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         return NB_OK;
@@ -732,7 +772,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(dout); NB_CHECK_PTR(dw); NB_CHECK_PTR(dx, true); NB_CHECK_PTR(dbias, true);
     if (dx) NB_CHECK_PTR(w);
-    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: only the three training calls honour them");
+    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
     {
         DeviceGuard on_device(p->device);
@@ -918,7 +958,7 @@ nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const voi
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     if (!host_x || !host_w || !host_gamma || !host_beta || !host_g || !host_a || !host_dw || !host_dgamma || !host_dbeta)
         return fail(NB_ERR_INVALID_ARG, "a required host pointer is NULL");
-    if (p->pitched) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches set: the host-buffer step works on dense tensors");
+    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: the host-buffer step works on dense tensors");
     const StepLayout L = step_layout(p);
     NB_TRY(check_ws(device_scratch, scratch_bytes, L.total));
     DeviceGuard on_device(p->device);

@@ -46,6 +46,7 @@ struct IgemmParams {
     // When GEMM row == output row (everything but a stride-2 dgrad) a warp hands each staged [32 x width] piece
     // to TMA: tmOut[i] is a tiled map over the output [M][ldo] with box {out_w[i], 32}; clipping at M is the map's.
     int tma_store;
+    int out_accumulate;  // the TMA stores are reductions: the tile is added to what the output tensor holds (data gradient into a shared gradient buffer)
     int out_w[3];
     CUtensorMap tmOut[3];
     // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
@@ -188,7 +189,7 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, 
 // from shared memory (`coef`, the same address in every lane: a broadcast; per channel pair scale, scale, shift, shift).
 template <typename OutT, bool STATS, int NP, int EPI, class Release>
 __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int lane, bool& store_pending, int& sat, const CUtensorMap* tm, int col,
-                                             int grow, float* stat_s, float* stat_q, const float2* coef, int act, Release release) {
+                                             int grow, float* stat_s, float* stat_q, const float2* coef, int act, bool accumulate, Release release) {
     constexpr bool SWZ = NP == 64;
     constexpr int PITCH = NP * 2;
     uint32_t r[NP];
@@ -235,7 +236,7 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
     ptx::fence_async_smem();  // writes visible to the async proxy before the store is issued
     __syncwarp();
     if (lane == 0) {
-        ptx::tma_store_2d(tm, wrows, col, grow);
+        if (accumulate) ptx::tma_reduce_add_2d(tm, wrows, col, grow); else ptx::tma_store_2d(tm, wrows, col, grow);
         ptx::tma_store_commit();
     }
     store_pending = true;
@@ -540,6 +541,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         float* team_stat = wstat + (team ? (size_t)8 * p.n_tiles * p.ncol_a : 0);  // [4 warps][2][st_ld]
         float* my_stat = team_stat + (size_t)lane_group * 2 * st_ld;
         const bool tma_out = p.tma_store != 0;  // (always set for the STATS and EPI variants)
+        const bool acc_out = !STATS && !EPI && p.out_accumulate != 0;
         // staging of this warp's 32 rows: padded rows for the store loop, dense rows (the TMA box) for TMA stores
         uint8_t* stg_t = stg + (size_t)team * TC_BM * pitch;
         uint8_t* const wrows = tma_out ? stg + (size_t)((team * 4 + lane_group) * 32) * (cw * 2) : stg_t + (size_t)(lane_group * 32) * pitch;
@@ -592,10 +594,10 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                         float* sq = ss + st_ld;
                         const uint32_t ta = taddr + (uint32_t)cb;
                         const float2* cf = reinterpret_cast<const float2*>(wstat) + col;  // read only by the EPI variant
-                        if (npass == 64) epi_pass_tma<OutT, STATS, 64, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                        else if (npass == 48) epi_pass_tma<OutT, STATS, 48, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                        else if (npass == 32) epi_pass_tma<OutT, STATS, 32, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
-                        else epi_pass_tma<OutT, STATS, 16, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, release);
+                        if (npass == 64) epi_pass_tma<OutT, STATS, 64, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, acc_out, release);
+                        else if (npass == 48) epi_pass_tma<OutT, STATS, 48, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, acc_out, release);
+                        else if (npass == 32) epi_pass_tma<OutT, STATS, 32, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, acc_out, release);
+                        else epi_pass_tma<OutT, STATS, 16, EPI>(ta, wrows, lane, store_pending, sat, tm, col, grow, ss, sq, cf, p.epi_act, acc_out, release);
                         continue;
                     }
                     // ---- output rows that are not GEMM rows (the parity classes of a stride-2 data gradient): padded staging
@@ -772,6 +774,7 @@ struct TcGemmSlot {  // one launch: configuration plus the tensor maps encoded f
     const void* a_ptr = nullptr;
     const void* b_ptr = nullptr;
     const void* out_ptr = nullptr;
+    long long out_ld = 0;  // row pitch the output maps were encoded with
 };
 
 struct TcPlan {
@@ -967,7 +970,9 @@ inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, lo
 }
 
 // Tiled maps over the output matrix [rows][ldo] (16-bit elements) for the epilogue's TMA stores: one per distinct pass width.
-inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long long rows) {
+// ld = row pitch in elements when the output is a channel slice of a wider tensor (0: dense); f16: the elements are IEEE
+// fp16 (it matters only for reductions: a store moves bits).
+inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long long rows, long long ld = 0, bool f16 = false) {
     DriverFns& d = driver();
     const int na = c.stage_cols, nb = c.BN - c.stage_cols, cw = P.stage_cw;
     const int cand[3] = {cw, na % cw, nb % cw};  // full passes, team 0's last pass, team 1's last pass
@@ -977,10 +982,10 @@ inline bool encode_out_maps(IgemmParams& P, const IgemmCfg& c, void* out, long l
         const int wv = cand[i];
         if (wv == 0 || (n > 0 && P.out_w[0] == wv) || (n > 1 && P.out_w[1] == wv)) continue;
         cuuint64_t dims[2] = {(cuuint64_t)P.ldo, (cuuint64_t)rows};
-        cuuint64_t strides[1] = {(cuuint64_t)P.ldo * 2};
+        cuuint64_t strides[1] = {(cuuint64_t)(ld ? ld : P.ldo) * 2};
         cuuint32_t box[2] = {(cuuint32_t)wv, 32};
         cuuint32_t estr[2] = {1, 1};
-        CUresult r = d.tiled(&P.tmOut[n], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        CUresult r = d.tiled(&P.tmOut[n], f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              wv == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeTiled (output) failed with code " + std::to_string((int)r); return false; }
@@ -1336,7 +1341,10 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
 
 // `wt_ready`: the rearranged filter was already written by an earlier kernel of this call (the BN backward finalize kernel
 // carries that work in extra blocks, where it costs nothing: the GPU is almost empty while the finalize chain runs).
-inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void* w, void* dx, void* wt, int* status, cudaStream_t st, bool wt_ready) {
+// ld_dx / accumulate (stride-1 layers only, whose epilogue goes through TMA): dx is a channel slice with row pitch ld_dx
+// elements (0: dense) and the result is added to what it holds instead of overwriting it.
+inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void* w, void* dx, void* wt, int* status, cudaStream_t st, bool wt_ready,
+                          long long ld_dx = 0, bool accumulate = false) {
     using namespace tcdetail;
     if (!wt_ready) {
         const size_t total = tc->wt_bytes / 2;
@@ -1357,10 +1365,16 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         S.a_ptr = dy; S.b_ptr = wt;
     }
     S.prm.tma_store = g.stride == 1 ? 1 : 0;  // the parity classes of a stride-2 layer write every other output pixel
-    if (S.prm.tma_store && S.out_ptr != dx) {
-        if (!encode_out_maps(S.prm, S.cfg, dx, (long long)g.n * g.h * g.w)) return NB_ERR_CUDA;
-        S.out_ptr = dx;
+    if (!S.prm.tma_store && (ld_dx || accumulate)) {
+        err() = "a pitched or accumulating data gradient needs the TMA-store epilogue (stride-1 layers)";
+        return NB_ERR_UNSUPPORTED;
     }
+    if (S.prm.tma_store && (S.out_ptr != dx || S.out_ld != ld_dx)) {
+        if (!encode_out_maps(S.prm, S.cfg, dx, (long long)g.n * g.h * g.w, ld_dx, tc->f16)) return NB_ERR_CUDA;
+        S.out_ptr = dx;
+        S.out_ld = ld_dx;
+    }
+    S.prm.out_accumulate = accumulate ? 1 : 0;
     S.prm.out = dx; S.prm.partials = nullptr; S.prm.status = status;
     nb_status r = tc->f16 ? launch_igemm<__half, false>(S, st) : launch_igemm<__nv_bfloat16, false>(S, st);
     if (r != NB_OK) return r;

@@ -28,10 +28,15 @@ _PITCH_IN = ("slice", "add", "concat")  # glue ops that read pitched operands (b
 
 
 class GraphRunner:
-    def __init__(self, ops, layers, outputs, eps=1e-3, device=0, plain_layers=None, views=True):
+    def __init__(self, ops, layers, outputs, eps=1e-3, device=0, plain_layers=None, views=True, direct_dx=True, fuse_residual=True):
         """plain_layers: shapes of the plain convolutions (bias, no BN, no activation) that "plain" ops refer to; their
         parameters and gradients live in self.plain[k] (dict with plan, w, bias, dw, dbias, dx, ws).
-        views=False: every tensor dense, split / concat by copies (the reference behaviour of the views)."""
+        views=False: every tensor dense, split / concat by copies (the reference behaviour of the views).
+        direct_dx=False: every block writes its data gradient to a buffer of its own and a glue launch adds it to the
+        input's gradient (the reference behaviour of nb_cbs_plan_set_dx_target).
+        fuse_residual=False: every residual add is a glue launch of its own (the reference behaviour of
+        nb_cbs_plan_set_fwd_residual, up to one rounding: the fused add rounds the sum once, the separate one rounds the
+        block's output first)."""
         self.ops, self.layers, self.outputs = ops, layers, list(outputs)
         self.dev = torch.device("cuda", device)
         self.plain, self.idx = [], {}
@@ -42,6 +47,16 @@ class GraphRunner:
         for i, o in enumerate(ops):
             for pos, name in enumerate(o["ins"]):
                 cons.setdefault(name, []).append((i, o, pos))
+        # ---- residual adds "out = shortcut + v" whose v is a block's output with no other consumer: that block performs the
+        # add itself (its normalise + SiLU pass adds the shortcut), v and out are one tensor, and so are their gradients
+        self.fused_v = {}  # name of v -> the add op
+        if fuse_residual:
+            for o in ops:
+                if o["op"] == "add":
+                    v = o["ins"][1]
+                    if v in prod and prod[v][1]["op"] == "cbs" and len(cons[v]) == 1 and v not in self.outputs and o["ins"][0] != v:
+                        self.fused_v[v] = o
+        self.fused_adds = {id(o) for o in self.fused_v.values()}
         # ---- shapes, blocks, plain convolutions
         s0 = layers[0]
         shape = self.shape = {"img": (s0.n, s0.h, s0.w, s0.c_in)}
@@ -125,6 +140,8 @@ class GraphRunner:
 
         for o in ops:
             out, kind, c = o["out"], o["op"], shape[o["out"]][3]
+            if out in self.fused_v:
+                continue  # lives in the add's output tensor (set when that op is reached)
             if out in placed:
                 cat, off = placed[out]
                 buf[out] = cat_storage(cat)[..., off:off + c]
@@ -138,6 +155,8 @@ class GraphRunner:
                 buf[out] = new(shape[out])
             if kind == "maxpool":
                 self.idx[out] = new(shape[out], torch.uint8)
+            if id(o) in self.fused_adds:
+                buf[o["ins"][1]] = buf[out]
         # ---- gradients
         grad = self.grad = {}
         self.owned = []
@@ -148,7 +167,9 @@ class GraphRunner:
             c = shape[name][3]
             po = prod.get(name, (None, {"op": "input"}))[1]
             cs = cons.get(name, [])
-            if name in placed:
+            if name in self.fused_v:
+                g = grad_of(self.fused_v[name]["out"])
+            elif name in placed:
                 cat, off = placed[name]
                 g = grad_of(cat)[..., off:off + c]
             elif po["op"] == "slice" and name in slice_view:
@@ -173,6 +194,9 @@ class GraphRunner:
             blk, s = self.blocks[o["layer"]], layers[o["layer"]]
             blk.x, blk.a, blk.g = buf[o["ins"][0]], buf[o["out"]], grad[o["out"]]
             blk.plan.set_pitches(ld_x=blk.x.stride(-2), ld_a=blk.a.stride(-2), ld_g=blk.g.stride(-2))
+            if o["out"] in self.fused_v:
+                blk.res = buf[self.fused_v[o["out"]]["ins"][0]]
+                blk.plan.set_fwd_residual(blk.res, blk.res.stride(-2))
         # ---- which contributions overwrite and which add: walk the backward order once over the OWNED buffers
         def root(name):  # (owned tensor whose buffer holds this gradient, channel offset in it) or (None, 0)
             po = prod.get(name, (None, {"op": "input"}))[1]
@@ -211,11 +235,29 @@ class GraphRunner:
                 self.zeroed.append(name)
                 for key in pending.get(name, []):
                     self.acc[key] = True
+        # ---- a block whose input's gradient lives in a buffer other than its own dx writes (or adds) there itself: its data
+        # gradient kernel stores through TMA into the channel slice, as a reduction when other consumers contributed before
+        self.direct_dx = set()
+        if direct_dx:
+            for oi, o in enumerate(ops):
+                if o["op"] != "cbs":
+                    continue
+                blk, target = self.blocks[o["layer"]], grad[o["ins"][0]]
+                if target is blk.dx:
+                    continue
+                try:
+                    blk.plan.set_dx_target(ld_dx=target.stride(-2), accumulate=self.acc[(oi, 0)])
+                except nb.NbError:
+                    continue  # (stride-2 layers and layers off the tensor-core path keep the glue launch)
+                blk.dx = target
+                self.direct_dx.add(oi)
 
     # ------------------------------------------------------------------ helpers
     def _implicit(self, o, pos):
         """True when op o's backward contribution to its input `pos` needs no work: a slice view, a placed concat input."""
         src = o["ins"][pos]
+        if o["op"] == "add" and id(o) in self.fused_adds:
+            return pos == 1  # the block's output IS the sum: its gradient is the sum's gradient
         if o["op"] == "slice":
             return o["out"] in self.slice_view
         if o["op"] == "concat":
@@ -250,8 +292,9 @@ class GraphRunner:
                     self._sadd(B[out], B[ins[0]][..., o["c0"]:o["c1"]], rows, c_out, stream=stream)
                     n_glue += 1
             elif kind == "add":
-                self._sadd(B[out], B[ins[0]], rows, c_out, b=B[ins[1]], stream=stream)
-                n_glue += 1
+                if id(o) not in self.fused_adds:
+                    self._sadd(B[out], B[ins[0]], rows, c_out, b=B[ins[1]], stream=stream)
+                    n_glue += 1
             elif kind == "concat":
                 c0 = 0
                 for name in ins:
@@ -306,8 +349,9 @@ class GraphRunner:
                     n_glue += 1
             elif kind == "add":
                 for pos, src in enumerate(ins):
-                    self._sadd(G[src], G[out], self._rows(out), c_out, accumulate=self.acc[(oi, pos)], stream=stream)
-                    n_glue += 1
+                    if not self._implicit(o, pos):
+                        self._sadd(G[src], G[out], self._rows(out), c_out, accumulate=self.acc[(oi, pos)], stream=stream)
+                        n_glue += 1
             elif kind == "concat":
                 c0 = 0
                 for pos, src in enumerate(ins):

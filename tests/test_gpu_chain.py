@@ -279,7 +279,7 @@ def test_detector_dataflow_matches_graph_oracle():
         assert e <= 2 * y + 5e-3, (name, e, y)
 
     for name in T0:
-        if name != "img":
+        if name != "img" and name not in run.fused_v:  # (the output of a block that adds its shortcut itself exists only as the sum)
             held(name, f64(run.buf[name]), T0[name], T1[name])
     held("d img", f64(run.grad["img"]), G0["img"], G1["img"])
     for k, blk in enumerate(run.blocks):
@@ -325,8 +325,12 @@ def test_detector_stage_by_stage_against_the_oracle_on_the_gpus_own_inputs(batch
         run.grad[name].copy_(torch.from_numpy(wl.round_to_bf16(rng.standard_normal(run.shape[name], dtype=np.float32))).to(torch.bfloat16))
     # With channel-slice views the gradient of a tensor placed inside a concatenation buffer lives in the consuming block's
     # dx buffer, where later contributions are added in place: keep each block's own dx as it was right after its call.
-    for blk in run.blocks:
-        def keep_dx(stream=None, _call=blk.backward_data, _blk=blk):
+    # A block that adds its data gradient straight into a shared gradient buffer (nb_cbs_plan_set_dx_target): keep the
+    # buffer as it was before the call too.
+    adds = {o["layer"] for oi, o in enumerate(ops) if o["op"] == "cbs" and oi in run.direct_dx and run.acc[(oi, 0)]}
+    for k, blk in enumerate(run.blocks):
+        def keep_dx(stream=None, _call=blk.backward_data, _blk=blk, _adds=k in adds):
+            _blk.dx_before = _blk.dx.clone() if _adds else None
             _call(stream)
             _blk.dx_own = _blk.dx.clone()
         blk.backward_data = keep_dx
@@ -372,7 +376,10 @@ def test_detector_stage_by_stage_against_the_oracle_on_the_gpus_own_inputs(batch
             k = o["layer"]
             blk, prm, st = run.blocks[k], params[k], layers[k].stride
             f = oracle.cbs_fwd(x, prm.w, prm.gamma, prm.beta, st, EPS)
-            bar("a", out, f64(B[out]), f.a)
+            if out in run.fused_v:  # the block adds the bottleneck's shortcut itself: its output tensor is the sum
+                bar("a + shortcut", out, f64(B[out]), f.a + f64(B[run.fused_v[out]["ins"][0]]))
+            else:
+                bar("a", out, f64(B[out]), f.a)
             bar("y", out, f64(blk.y), f.y)
             parity.check_stats(f64(blk.mean), f64(blk.invstd), f.y, EPS, "bf16")
             # backward stages, each from the GPU's own inputs of that stage
@@ -382,8 +389,13 @@ def test_detector_stage_by_stage_against_the_oracle_on_the_gpus_own_inputs(batch
             bar("dgamma", out, f64(blk.dgamma), dgamma)
             bar("dbeta", out, f64(blk.dbeta), dbeta)
             bar("dw", out, f64(blk.dw), oracle.conv_wgrad(x, dy_gpu, layers[k].k, st))
-            bar("dx", out, f64(blk.dx_own), oracle.conv_dgrad(dy_gpu, prm.w, x.shape, st))
-            give(ins[0], f64(blk.dx_own))
+            want_dx = oracle.conv_dgrad(dy_gpu, prm.w, x.shape, st)
+            if blk.dx_before is None:
+                bar("dx", out, f64(blk.dx_own), want_dx)
+                give(ins[0], f64(blk.dx_own))
+            else:  # the buffer after the call = what it held before + this block's data gradient (one rounding)
+                bar("dx (added)", out, f64(blk.dx_own), f64(blk.dx_before) + want_dx)
+                give(ins[0], f64(blk.dx_own) - f64(blk.dx_before))
         elif kind == "plain":
             k = o["layer"]
             pl, (w, bias) = run.plain[k], pparams[k]
@@ -397,9 +409,10 @@ def test_detector_stage_by_stage_against_the_oracle_on_the_gpus_own_inputs(batch
             same(out, f64(B[out]), x[..., o["c0"]:o["c1"]])
             give(ins[0], f64(G[out]), o["c0"])
         elif kind == "add":
-            same(out, f64(B[out]), chain.round_bf16(x + f64(B[ins[1]])))
             give(ins[0], f64(G[out]))
-            give(ins[1], f64(G[out]))
+            if ins[1] not in run.fused_v:  # (a fused add was checked with the block that performs it)
+                same(out, f64(B[out]), chain.round_bf16(x + f64(B[ins[1]])))
+                give(ins[1], f64(G[out]))
         elif kind == "concat":
             same(out, f64(B[out]), np.concatenate([f64(B[i]) for i in ins], axis=-1))
             # (the concatenation's own gradient is the consuming block's dx before anything was added into it)

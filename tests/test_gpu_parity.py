@@ -255,6 +255,91 @@ def test_channel_slice_operands_give_bitwise_the_dense_results(shape):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[8], SMALL_SHAPES[12], SMALL_SHAPES[11]], ids=lambda s: s.name)
+def test_data_gradient_into_a_pitched_and_accumulating_target(shape):
+    """nb_cbs_plan_set_dx_target: the data gradient written straight into a channel slice of a wider gradient buffer, and
+    ADDED to what the slice holds (TMA reductions in the epilogue), as a tensor with several consumers needs.  Overwriting
+    must give the dense run's bits; accumulating must give round(old + dx) -- one rounding to bf16 per element, what a
+    separate accumulation pass gives -- and nothing outside the slice may change.  Layers without the TMA epilogue refuse."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    inp, dense, want = _run_block(shape, 0, cfg_id=21, affine="random")
+    assert dense.plan.paths["dgrad"] == 1
+    blk = CbsBlock(shape, eps=EPS)
+    blk.upload(inp)
+    blk.step()
+    s, dev = shape, blk.dev
+    ld, off = s.c_in + 24, 16
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(9)
+    wide = torch.randn(s.n, s.h, s.w, ld, generator=gen, device=dev).to(torch.bfloat16)
+    before = wide.clone()
+    view = wide[..., off:off + s.c_in]
+
+    def bwd(dx):
+        nb.nb_conv_bn_silu_bwd_data(blk.plan, blk.g, blk.y, blk.mean, blk.invstd, blk.gamma, blk.beta, blk.w, dx, blk.dgamma, blk.dbeta, blk.dy, blk.ws)
+        torch.cuda.synchronize()
+        blk.poll()
+
+    blk.plan.set_dx_target(ld_dx=ld, accumulate=False)
+    bwd(view.data_ptr())
+    assert torch.equal(view, dense.dx)
+    assert torch.equal(wide[..., :off], before[..., :off]) and torch.equal(wide[..., off + s.c_in:], before[..., off + s.c_in:])
+    wide.copy_(before)
+    blk.plan.set_dx_target(ld_dx=ld, accumulate=True)
+    bwd(view.data_ptr())
+    expect = (before[..., off:off + s.c_in].float() + dense.dx.float()).to(torch.bfloat16)
+    assert torch.equal(view, expect)
+    assert torch.equal(wide[..., :off], before[..., :off]) and torch.equal(wide[..., off + s.c_in:], before[..., off + s.c_in:])
+    blk.plan.set_dx_target()  # back to a dense, overwritten dx
+    bwd(blk.dx)
+    assert torch.equal(blk.dx, dense.dx)
+    strided = CbsBlock(SMALL_SHAPES[9], eps=EPS)  # stride 2: its epilogue does not go through TMA
+    with pytest.raises(nb.NbError) as e:
+        strided.plan.set_dx_target(accumulate=True)
+    assert e.value.status == nb.NB_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[12], SMALL_SHAPES[3]], ids=lambda s: s.name)
+@pytest.mark.parametrize("mode", [0, 1], ids=["bf16", "f32"])
+def test_forward_with_a_residual_adds_it_once(shape, mode):
+    """nb_cbs_plan_set_fwd_residual: a_out = SiLU(z) + res in the normalise + SiLU pass (res dense or a channel slice), the
+    sum rounded once; against the oracle's block output plus the same residual, at the block's own bars; the saved
+    tensors are those of the plain block, bit for bit."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+
+    inp, blk, plain = _run_block(shape, mode, cfg_id=22, affine="random")
+    ref = _oracle(inp)
+    s, dev = shape, blk.dev
+    dt = blk.a.dtype
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(3)
+    for ld, off in ((0, 0), (s.c_out + 16, 8)):
+        wide = torch.randn(s.n, s.ho, s.wo, ld or s.c_out, generator=gen, device=dev).to(dt)
+        res = wide[..., off:off + s.c_out]
+        blk.plan.set_fwd_residual(res, res.stride(-2))
+        blk.forward()
+        torch.cuda.synchronize()
+        blk.poll()
+        got = blk.a.double().cpu().numpy()
+        parity.check("a + res", got, ref.a + res.double().cpu().numpy(), "bf16" if mode == 0 else "f32")
+        np.testing.assert_array_equal(blk.y.double().cpu().numpy(), plain["y"])
+        np.testing.assert_array_equal(blk.mean.double().cpu().numpy(), plain["mean"])
+    ws = torch.empty(max(blk.plan.infer_bytes, 256), dtype=torch.uint8, device=dev)
+    with pytest.raises(nb.NbError) as e:
+        nb.nb_conv_bias_act(blk.plan, blk.x, blk.w, None, 0, blk.a, ws)
+    assert e.value.status == nb.NB_ERR_UNSUPPORTED
+    blk.plan.set_fwd_residual(None)
+    blk.forward()
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(blk.a.double().cpu().numpy(), plain["a"])
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_plan_stays_usable():
     """Every wait inside the kernels has a limit; a wait that runs out makes the kernel skip the step behind it, drain and
     return, and nb_cbs_poll_status reports NB_ERR_TIMEOUT with the site.  No fault, trap or hang is involved: the test
