@@ -25,6 +25,11 @@ namespace nbcbs {
 struct IgemmParams {
     CUtensorMap tmA;     // im2col map over the activation [N][Hs][Ws][Ca]
     CUtensorMap tmB[4];  // per class: tiled map over the filter matrix [rowsB][ntaps*Ca], K contiguous
+    // Ca mod 64 in (0, 32]: the last k-block of every tap is 32 channels wide, fetched through these maps (same tensors,
+    // boxes of 32 channels in the 64-byte swizzle) and multiplied by two MMAs instead of four.
+    int tail32;
+    CUtensorMap tmA_t;
+    CUtensorMap tmB_t[4];
     long long M;      // rows of the GEMM: n * Hq * Wq
     int Hq, Wq;       // traversal grid per image
     int ts;           // traversal stride (input pixels per grid step)
@@ -371,6 +376,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         bool ok = true;
         const int bn_own = CG2 ? p.BN / 2 : p.BN;  // rows of the B tile this CTA fetches
         const uint32_t kb_bytes = isA ? (uint32_t)(TC_BM * mh * p.KC * 2) : (uint32_t)(bn_own * p.KC * 2);
+        const int kc_tail = p.tail32 ? p.kc_per_tap - 1 : -1;  // index of the 32-channel k-block inside a tap (-1: none)
         // loop-invariant values in registers: this thread's instruction stream is on the critical path
         const int kpb = p.kpb, stages = p.stages, KC = p.KC, kc_per_tap = p.kc_per_tap, Ca = p.Ca, BN = p.BN, n_tiles = p.n_tiles;
         const int Wq = p.Wq, Hq = p.Hq, ts = p.ts, a_tiled = p.a_tiled;
@@ -382,7 +388,8 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
         for (int tile = worker; ok && tile < total_tiles; tile += nworkers) {
             int cls, lt;
             igemm_tile_class<CLS4>(p, tile, nworkers, cls, lt);
-            const CUtensorMap* tm = isA ? &p.tmA : &p.tmB[cls];
+            const CUtensorMap* tm_full = isA ? &p.tmA : &p.tmB[cls];
+            const CUtensorMap* tm_tail = isA ? &p.tmA_t : &p.tmB_t[cls];
             const int kblocks = p.cls_ntaps[cls] * kc_per_tap;
             const int m_tile = lt / n_tiles, n_tile = lt - m_tile * n_tiles;
             const int m0 = (CG2 ? m_tile * 2 + (int)rank : m_tile) * TC_BM * mh;
@@ -407,10 +414,19 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     break;
                 }
                 const uint32_t bar = full_u32 + 8u * (uint32_t)s;
-                if (!CG2) ptx::mbar_expect_tx_u32_if(leader, bar, kb_bytes * (uint32_t)nkb);
-                else if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * kb_bytes * (uint32_t)nkb);
+                uint32_t tx_bytes = kb_bytes * (uint32_t)nkb;
+                if (kc_tail >= 0) {  // a 32-channel k-block brings half the bytes
+                    int kq = kc;
+                    for (int j = 0; j < nkb; ++j) {
+                        if (kq == kc_tail) tx_bytes -= kb_bytes >> 1;
+                        if (++kq == kc_per_tap) kq = 0;
+                    }
+                }
+                if (!CG2) ptx::mbar_expect_tx_u32_if(leader, bar, tx_bytes);
+                else if (rank == 0) ptx::mbar_expect_tx_u32_if(leader, ptx::smem_u32(full) + 8u * (uint32_t)s, 2u * tx_bytes);
                 uint32_t dst = base_u32 + (uint32_t)s * stage_bytes;
                 for (int j = 0; j < nkb; ++j) {
+                    const CUtensorMap* tm = kc == kc_tail ? tm_tail : tm_full;
                     if (isA) {
                         if (a_tiled) {
                             if (CG2) ptx::tma_load_2d_cg2_if(leader, dst, tm, bar, kc * KC, m0); else ptx::tma_load_2d_u32_if(leader, dst, tm, bar, kc * KC, m0);
@@ -458,6 +474,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
             const uint64_t a_sub16 = (uint64_t)(p.a_sub_bytes >> 4), b_sub16 = (uint64_t)(p.b_sub_bytes >> 4);
             const uint64_t a_stage16 = (uint64_t)(p.a_stage_bytes >> 4), b_stage16 = (uint64_t)(p.b_stage_bytes >> 4);
             const uint64_t a_half16 = (uint64_t)((TC_BM * p.KC * 2) >> 4);  // second 128-row sub-tile inside a k-block of A
+            // 32-channel k-block: rows of 64 bytes in the 64-byte swizzle; same start address, other stride and swizzle fields
+            const uint64_t tail_flip = ptx::make_smem_desc(0u, 16, p.sbo, p.umma_swizzle) ^ ptx::make_smem_desc(0u, 16, p.sbo >> 1, (uint32_t)ptx::kSwizzle64);
+            const int kc_tail = p.tail32 ? p.kc_per_tap - 1 : -1;
             const uint64_t da0 = ptx::make_smem_desc(ptx::smem_u32(sA), 16, p.sbo, p.umma_swizzle);
             const uint64_t db0 = ptx::make_smem_desc(ptx::smem_u32(sB), 16, p.sbo, p.umma_swizzle);
             const uint32_t empty_u32 = ptx::smem_u32(empty);
@@ -472,6 +491,7 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * mh) * acc_stride;
                 uint32_t accumulate = 0;
+                int kc = (int)(((unsigned)worker * 7u) % (unsigned)kblocks) % kc_per_tap;  // the producers' starting k-block
                 for (int kb0 = 0; kb0 < kblocks; kb0 += kpb) {
                     const int nkb = (kblocks - kb0 < kpb) ? kblocks - kb0 : kpb;
                     if (!wait_bar_fast(full + s, ph, abort_flag, p.status, 3)) {
@@ -481,10 +501,21 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                     ptx::tc_fence_after();
                     uint64_t da = da_s, db = db_s;
                     for (int j = 0; j < nkb; ++j) {
+                        const bool tail = kc == kc_tail;
+                        if (++kc == kc_per_tap) kc = 0;
                         for (int h = 0; h < mh; ++h) {
                             const uint64_t dah = da + (uint64_t)h * a_half16;
                             const uint32_t dt = d_tmem + (uint32_t)h * acc_stride;
-                            if (CG2) {
+                            if (tail) {
+                                const uint64_t dat = (da + (uint64_t)h * (a_half16 >> 1)) ^ tail_flip, dbt = db ^ tail_flip;
+                                if (CG2) {
+                                    ptx::umma_f16_cg2_if(leader, dt, dat, dbt, idesc, accumulate);
+                                    ptx::umma_f16_cg2_if(leader, dt, dat + 2, dbt + 2, idesc, 1u);
+                                } else {
+                                    ptx::umma_f16_if(leader, dt, dat, dbt, idesc, accumulate);
+                                    ptx::umma_f16_if(leader, dt, dat + 2, dbt + 2, idesc, 1u);
+                                }
+                            } else if (CG2) {
                                 ptx::umma_f16_cg2_if(leader, dt, dah, db, idesc, accumulate);
                                 ptx::umma_f16_cg2_if(leader, dt, dah + 2, db + 2, idesc, 1u);
                                 ptx::umma_f16_cg2_if(leader, dt, dah + 4, db + 4, idesc, 1u);
@@ -763,6 +794,7 @@ struct IgemmCfg {
     int Ca = 0, rowsB = 0, ntaps = 0;
     int KC = 0, BN = 0, n_tiles = 0, m_tiles = 0, stages = 0, acc_stride = 0, tmem_cols = 0, grid = 0, kpb = 1, mh = 1, acc_bufs = 2, stage_cols = 0;
     bool cg2 = false;  // CTA pairs (tcgen05 cta_group::2)
+    bool tail32 = false;  // the last k-block of every tap is 32 channels wide
     uint32_t a_stage = 0, b_stage = 0, a_sub = 0, b_sub = 0;
     size_t smem_bytes = 0;
     long long M = 0;
@@ -859,10 +891,13 @@ inline IgemmCfg igemm_configure(long long M, int Ca, int rowsB, int ntaps, int l
     IgemmCfg c;
     c.Ca = Ca; c.rowsB = rowsB; c.ntaps = ntaps; c.M = M;
     if (Ca % 16 || rowsB % 16 || M < 1) return c;
-    // Always 64-channel k-blocks in the 128-byte swizzle (the narrower swizzles make tcgen05.mma 1.6-2.1x slower per
+    // 64-channel k-blocks in the 128-byte swizzle (the narrower swizzles make tcgen05.mma 1.6-2.1x slower per
     // instruction); when Ca is not a multiple of 64 the last k-block of every tap reads past the channel extent and
     // TMA fills A with zeros there (whatever finite filter values B holds at those positions are multiplied by zero).
+    // When at most 32 channels are left for that last k-block it is fetched 32 channels wide in the 64-byte swizzle:
+    // two slower MMAs instead of four, and half the bytes written to and read from shared memory.
     c.KC = 64;
+    c.tail32 = Ca % 64 != 0 && Ca % 64 <= 32 && (getenv("NB_TC_TAIL") ? atoi(getenv("NB_TC_TAIL")) != 0 : true);
     const int kblocks = ntaps * ((Ca + c.KC - 1) / c.KC);
     const int force_bn = getenv("NB_TC_BN") ? atoi(getenv("NB_TC_BN")) : 0;
     const int force_kpb = getenv("NB_TC_KPB") ? atoi(getenv("NB_TC_KPB")) : 0;
@@ -932,10 +967,11 @@ inline void fill_params(IgemmParams& P, const IgemmCfg& c) {
     P.sbo = (uint32_t)(8 * c.KC * 2);
     P.a_stage_bytes = c.a_stage; P.b_stage_bytes = c.b_stage;
     P.kpb = c.kpb; P.a_sub_bytes = c.a_sub; P.b_sub_bytes = c.b_sub;
+    P.tail32 = c.tail32 ? 1 : 0;
     P.mh = c.mh; P.acc_bufs = c.acc_bufs; P.ncol_a = c.stage_cols; P.stage_cw = igemm_stage_cw(c.BN);
     if (getenv("NB_TC_VERBOSE"))
-        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
-                c.rowsB, c.ntaps, c.mh, (int)c.cg2, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
+        fprintf(stderr, "[nb_cbs] igemm M=%lld Ca=%d rowsB=%d taps=%d: mh=%d cg2=%d tail32=%d BN=%d kpb=%d stages=%d accbufs=%d tiles=%dx%d grid=%d smem=%zu\n", c.M, c.Ca,
+                c.rowsB, c.ntaps, c.mh, (int)c.cg2, (int)c.tail32, c.BN, c.kpb, c.stages, c.acc_bufs, c.m_tiles, c.n_tiles, c.grid, c.smem_bytes);
     P.idesc = ptx::make_idesc_bf16(c.cg2 ? 2 * TC_BM : TC_BM, c.BN, 0, 0);
 }
 
@@ -1285,6 +1321,14 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
             return NB_ERR_CUDA;
         }
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+        if (S.cfg.tail32) {
+            if (S.prm.a_tiled) {
+                if (!encode_tiled_2d(&S.prm.tmA_t, x, g.m, g.c_in, 32, TC_BM * S.cfg.mh, tc->ld_x)) return NB_ERR_CUDA;
+            } else if (!encode_im2col(&S.prm.tmA_t, x, g.n, g.h, g.w, g.c_in, -g.pad, g.pad - (g.k - 1), g.stride, 32, TC_BM * S.cfg.mh, tc->ld_x)) {
+                return NB_ERR_CUDA;
+            }
+            if (!encode_tiled_2d(&S.prm.tmB_t[0], w, g.c_out, (long long)g.kdim, 32, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+        }
         S.a_ptr = x; S.b_ptr = w;
     }
     S.prm.tma_store = 1;
@@ -1322,6 +1366,14 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
             return NB_ERR_CUDA;
         }
         if (!encode_tiled_2d(&S.prm.tmB[0], w, g.c_out, (long long)g.kdim, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+        if (S.cfg.tail32) {
+            if (S.prm.a_tiled) {
+                if (!encode_tiled_2d(&S.prm.tmA_t, x, g.m, g.c_in, 32, TC_BM * S.cfg.mh, 0)) return NB_ERR_CUDA;
+            } else if (!encode_im2col(&S.prm.tmA_t, x, g.n, g.h, g.w, g.c_in, -g.pad, g.pad - (g.k - 1), g.stride, 32, TC_BM * S.cfg.mh, 0)) {
+                return NB_ERR_CUDA;
+            }
+            if (!encode_tiled_2d(&S.prm.tmB_t[0], w, g.c_out, (long long)g.kdim, 32, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+        }
         S.a_ptr = x; S.b_ptr = w;
     }
     S.prm.tma_store = 1;  // the fused epilogue exists only on the TMA-store path
@@ -1358,9 +1410,12 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
         // stride 1: window start runs over [-(k-1-P), W-1-(k-1-P)], i.e. W positions; stride-2 classes: over [0, Wo-1]
         const int lo = g.stride == 1 ? -(g.k - 1 - g.pad) : 0;
         if (!encode_im2col(&S.prm.tmA, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, S.cfg.KC, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
+        if (S.cfg.tail32 && !encode_im2col(&S.prm.tmA_t, dy, g.n, g.ho, g.wo, g.c_out, lo, lo, 1, 32, TC_BM * S.cfg.mh)) return NB_ERR_CUDA;
         for (int cls = 0; cls < tc->wtp.nclasses; ++cls) {
             const __nv_bfloat16* wcls = static_cast<const __nv_bfloat16*>(wt) + tc->wtp.cls[cls].offset;
             if (!encode_tiled_2d(&S.prm.tmB[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, S.cfg.KC, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN)) return NB_ERR_CUDA;
+            if (S.cfg.tail32 && !encode_tiled_2d(&S.prm.tmB_t[cls], wcls, g.c_in, (long long)tc->wtp.cls[cls].ntaps * g.c_out, 32, S.cfg.cg2 ? S.cfg.BN / 2 : S.cfg.BN))
+                return NB_ERR_CUDA;
         }
         S.a_ptr = dy; S.b_ptr = wt;
     }

@@ -67,6 +67,8 @@ SMALL_SHAPES = [
     S(1, 64, 64, 3, 48, 3, 2, True),  # stem-like
     S(2, 20, 20, 576, 64, 3, 1),
     S(2, 20, 20, 288, 288, 1, 1),
+    S(2, 36, 36, 48, 96, 3, 2),     # data gradient: four parity classes over 96 channels (64 + a 32-channel k-block per tap)
+    S(2, 24, 24, 80, 160, 3, 1),    # 80 = 64 + 16: the 32-channel k-block is half zero fill; 160 = 2 x 64 + 32
 ]
 
 
