@@ -836,13 +836,14 @@ def run_e2e(args, layers, blocks, flags, local, dev, dist, world, flops):
         d2h += sum(t.numel() * t.element_size() for t in hout.values())
     # Several streams (--e2e-streams, default 6), each with its own device scratch, take the layers in turn: while one layer computes, the next
     # layer's inputs arrive over PCIe and the previous layer's results leave (the two copy directions run concurrently).
-    # Kernels of different layers may then share the GPU, so the plans of this arm are created with NB_CBS_FLAG_SHARED_GPU
-    # (separate finalize kernels instead of in-kernel grid barriers).
+    # Layers of the same shape share a plan and may then be in flight on different streams at once, so the plans of this arm
+    # are created with NB_CBS_FLAG_SEPARATE_FINALIZE: all scratch of a call then lies in the workspace it was given (a default
+    # plan sums its statistics in accumulators of its own, which only one call at a time may use).
     nstreams = max(1, args.e2e_streams)
     plans = {}
     for b in blocks:
         if b.shape.key not in plans:
-            plans[b.shape.key] = nb.Plan.for_shape(b.shape, flags=flags | (nb.NB_CBS_FLAG_SHARED_GPU if nstreams > 1 else 0), device=local)
+            plans[b.shape.key] = nb.Plan.for_shape(b.shape, flags=flags | (nb.NB_CBS_FLAG_SEPARATE_FINALIZE if nstreams > 1 else 0), device=local)
     scratches = [torch.empty(scratch_bytes, dtype=torch.uint8, device=dev) for _ in range(nstreams)]
     main = torch.cuda.current_stream()
     streams = [main] if nstreams == 1 else [torch.cuda.Stream(device=dev) for _ in range(nstreams)]

@@ -33,10 +33,13 @@
  * and return without synchronising; they make the plan's device current while they run and restore the
  * caller's current device before returning (`stream` must belong to the plan's device).  Outputs are
  * overwritten, never accumulated into.  Calls on one plan must not run concurrently, neither on the host
- * (they share the plan's cached tensor maps) nor on the device (its status block and the workspace).
- * One exception on the device: nb_conv_bn_silu_bwd_weight uses no grid barrier and of the status block only
- * its atomic error words, so on a stream of its own, with a workspace of its own and ordered after the call
- * that produced dy, it may overlap any other call of this or another plan (default flags included).
+ * (they share the plan's cached tensor maps) nor on the device (its status block, the accumulators in which a
+ * default plan sums the BatchNorm statistics, and the workspace).  Two exceptions on the device:
+ * nb_conv_bn_silu_bwd_weight uses of the plan only the atomic error words of the status block, so on a stream of
+ * its own, with a workspace of its own and ordered after the call that produced dy, it may overlap any other
+ * call of this or another plan; and a plan created with NB_CBS_FLAG_SEPARATE_FINALIZE keeps all scratch of a
+ * call in the workspace that call was given, so its calls may overlap on different streams when their
+ * workspaces differ.  Calls of DIFFERENT plans may always overlap: no kernel waits for another block or kernel.
  * On invalid arguments nothing is launched and a non-zero status is returned; nb_last_error()
  * then describes the problem.
  */
@@ -71,13 +74,16 @@ typedef enum { NB_MODE_BF16_TC = 0, NB_MODE_F32_REF = 1, NB_MODE_F16_TC = 2 } nb
 /* nb_cbs_desc.flags */
 #define NB_CBS_FLAG_FORCE_SIMT 1u /* BF16 mode: run the three convolutions on the CUDA-core kernels
                                      (same arithmetic contract; for testing and as a cross-check) */
-#define NB_CBS_FLAG_SHARED_GPU 2u /* kernels of this plan may run at the same time as other kernels (other streams,
-                                     other processes).  By default the forward kernel and the backward reduce kernel
-                                     finish the BatchNorm statistics themselves behind a grid-wide barrier, which needs
-                                     all of their blocks resident at once: two such kernels that each hold half of the
-                                     GPU would wait for each other until the bounded waits give up (NB_ERR_TIMEOUT).
-                                     With this flag the finalize steps run as separate small kernels instead
-                                     (same results, a few microseconds more per call). */
+#define NB_CBS_FLAG_SEPARATE_FINALIZE 2u /* the BatchNorm statistics are finished by separate small kernels that add
+                                     per-block partial sums in a fixed order, so that they come out bit-identical from
+                                     run to run (a few microseconds more per call).  By default the kernels that sum
+                                     (the tensor-core forward convolution, the backward reduce pass) add their block
+                                     sums to fp64 accumulators with atomics and the pass that follows derives its
+                                     coefficients from the totals: the same values, except that a total may differ
+                                     in its last fp64 bit with the order of the additions (seen in an fp32 result
+                                     only if the total sits within 2^-50 of a rounding boundary).  No kernel of either
+                                     kind waits for another block or kernel, so calls of different plans may share
+                                     the GPU (other streams, other processes) with or without this flag. */
 
 typedef struct nb_cbs_desc {
     uint32_t struct_size; /* = sizeof(nb_cbs_desc) */
@@ -160,14 +166,6 @@ nb_status nb_cbs_poll_status(nb_cbs_plan plan, void* stream);
  * nb_cbs_profile_site_name(i): name of kernel site i, NULL once i is past the last site.
  * nb_cbs_profile_read: accumulated milliseconds and launch count of one site since the last enable call. */
 unsigned long long nb_cbs_launch_count(void);
-/* Test hook for the bounded waits (the paper has no counterpart).  Every wait inside the kernels is bounded and reports
- * NB_ERR_TIMEOUT through nb_cbs_poll_status instead of hanging.  This call makes that path observable without any
- * fault: the NEXT launch of this plan that contains a grid-wide barrier (the tensor-core forward kernel, or the backward
- * reduce kernel, whichever is launched first) waits for one block more than its grid has, for at most `limit_ms`
- * milliseconds (1..1000), gives up, skips its finalize step and returns normally; nb_cbs_poll_status then reports
- * NB_ERR_TIMEOUT (the outputs of that call are not valid), and later calls on the plan work as usual.
- * NB_ERR_UNSUPPORTED for plans without such kernels (NB_CBS_FLAG_SHARED_GPU). */
-nb_status nb_cbs_debug_expire_next_wait(nb_cbs_plan plan, int32_t limit_ms);
 nb_status nb_cbs_profile_enable(nb_cbs_plan plan, int32_t enable);
 const char* nb_cbs_profile_site_name(int32_t site);
 nb_status nb_cbs_profile_read(nb_cbs_plan plan, int32_t site, double* total_ms, int64_t* launches);

@@ -19,7 +19,7 @@ NB_ERR_CUDA, NB_ERR_ARCH, NB_ERR_TIMEOUT, NB_ERR_INTERNAL = 5, 6, 7, 8
 NB_DTYPE_F32, NB_DTYPE_BF16, NB_DTYPE_F16 = 0, 1, 2
 NB_MODE_BF16_TC, NB_MODE_F32_REF, NB_MODE_F16_TC = 0, 1, 2
 NB_CBS_FLAG_FORCE_SIMT = 1
-NB_CBS_FLAG_SHARED_GPU = 2
+NB_CBS_FLAG_SEPARATE_FINALIZE = 2
 
 EXPORTS = (
     "nb_abi_version", "nb_last_error", "nb_cbs_plan_create", "nb_cbs_plan_destroy", "nb_cbs_out_shape",
@@ -29,7 +29,7 @@ EXPORTS = (
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step", "nb_sgd_clip_nesterov_step_scaled",
     "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd", "nb_cbs_plan_set_pitches",
-    "nb_cbs_debug_expire_next_wait", "nb_cbs_plan_set_dx_target", "nb_cbs_plan_set_fwd_residual",
+    "nb_cbs_plan_set_dx_target", "nb_cbs_plan_set_fwd_residual",
 )
 
 
@@ -85,7 +85,6 @@ def load() -> ctypes.CDLL:
         lib.nb_cbs_poll_status.argtypes = [V, V]
         lib.nb_cbs_plan_set_dx_target.argtypes = [V, ctypes.c_int64, c_int32]
         lib.nb_cbs_plan_set_fwd_residual.argtypes = [V, V, ctypes.c_int64]
-        lib.nb_cbs_debug_expire_next_wait.argtypes = [V, c_int32]
         lib.nb_conv_bn_silu_fwd.argtypes = [V, V, V, FP, FP, FP, FP, V, FP, FP, V, V, c_size_t, V]
         lib.nb_bn_stats.argtypes = [V, V, c_int32, FP, FP, FP, FP, V, c_size_t, V]
         lib.nb_conv_bn_silu_bwd_data.argtypes = [V, V, V, FP, FP, FP, FP, V, V, FP, FP, V, V, c_size_t, V]
@@ -258,11 +257,6 @@ def nb_conv_bn_silu_fwd(plan: Plan, x, w, gamma, beta, running_mean, running_var
 def nb_bn_stats(plan: Plan, y, y_dtype, mean, invstd, sum_, sumsq, workspace, stream=None):
     _check(load().nb_bn_stats(plan.handle, _ptr(y), y_dtype, _ptr(mean), _ptr(invstd), _ptr(sum_), _ptr(sumsq), _ptr(workspace),
                               _nbytes(workspace), _stream(stream)))
-
-
-def nb_cbs_debug_expire_next_wait(plan: "Plan", limit_ms: int):
-    """Test hook: the plan's next grid-barrier launch gives up its wait after `limit_ms` ms (see include/nb_cbs.h)."""
-    _check(load().nb_cbs_debug_expire_next_wait(plan.handle, int(limit_ms)))
 
 
 def nb_bn_stats_static(y, y_dtype, m, c, eps, mean, invstd, sum_=None, sumsq=None, stream=None):

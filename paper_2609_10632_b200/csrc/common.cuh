@@ -19,21 +19,15 @@ struct Geom {
 };
 
 // Device status block owned by a plan (ints): [0] error code, [1] where, [2] detail, [3] fp16 saturation count.
-// Words 8-11 are two arrive/depart counter pairs of the in-kernel grid barriers (forward finalize, backward finalize);
-// each pair is zero whenever no kernel of the plan is running.  (A fused split-K reduce behind such a barrier at the
-// tail of the wgrad kernel was measured 0.13 ms per step slower than the separate reduce kernel, whose many small
-// blocks hide the load latency better than 148 resident CTAs can.)
-enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_BAR_FWD = 8, ST_BAR_BWD = 10, ST_WORDS = 16 };
+// Words 8 and 10 count the blocks of the normalise + SiLU pass / the dy pass that have read the fp64 channel
+// accumulators (see ChanAcc); each is zero whenever no kernel of the plan is running.
+enum { ST_ERR = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_SAT = 3, ST_READERS_FWD = 8, ST_READERS_BWD = 10, ST_WORDS = 16 };
 // Sites that a give-up is reported from (ST_WHERE): 1-5 the roles of the implicit-GEMM kernel (A producer, accumulator
-// free, operands ready, accumulator ready, B producer), 11-15 the same roles of the weight-gradient kernel, 20 the
-// forward kernel's grid barrier, 21 the backward reduce kernel's grid barrier.
-enum { SITE_GRID_BARRIER_FWD = 20, SITE_GRID_BARRIER_BWD = 21 };
+// free, operands ready, accumulator ready, B producer), 11-15 the same roles of the weight-gradient kernel.
 
-// Every wait in the library is bounded: about two seconds by default, or what a launch was told (in milliseconds).
+// Every wait in the library (all of them waits of a CTA on its own mbarriers: no kernel waits for another CTA's or
+// another kernel's flag) is bounded: about two seconds.
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-__host__ __device__ __forceinline__ unsigned long long wait_limit_ns(int limit_ms) {
-    return limit_ms > 0 ? (unsigned long long)limit_ms * 1000000ull : kWaitLimitNs;
-}
 
 // Records a give-up in a plan's status block (first one wins): error code, site, detail.
 __device__ __forceinline__ void report_timeout(int* status, int site, int detail) {
@@ -126,58 +120,12 @@ template <typename T> __device__ __forceinline__ void st16_stream(T* p, const Ve
     __stcs(reinterpret_cast<uint4*>(p), *reinterpret_cast<const uint4*>(&r));
 }
 
-// Grid-wide barrier for kernels whose CTAs are all resident at once (grids of at most one wave, nothing the CTAs wait for
-// runs behind them).  ctr[0] counts arrivals, ctr[1] departures; the last CTA to leave zeroes both, so the pair is ready
-// for the next launch.  All calls are made by ONE thread of the CTA, bracketed by CTA-level barriers; data written before
-// grid_arrive_wait by any CTA may be read (from L2: __ldcg) after it.  The wait is bounded (`limit_ns`): false = gave up.
-// `expected` is the number of arrivals waited for (the grid size; a test may ask for one more so that the wait runs out),
-// grid_depart always counts the CTAs that really exist.
-// Rules for kernels that use it:
-// (a) griddepcontrol.launch_dependents is issued only after the barrier has been passed, so no CTA of the NEXT kernel
-//     takes SM resources while CTAs of this grid still wait for a slot (with the trigger at the kernel's start the next
-//     kernel's CTAs could become resident, park at griddepcontrol.wait, and keep the last CTAs of this grid out);
-// (b) a grid with SEVERAL CTAs per SM is launched without the programmatic-serialization attribute, so none of its CTAs
-//     becomes resident beside CTAs of the previous kernel: a CTA placed in the middle of an SM's register file while
-//     other CTAs still hold the rest stays there until the barrier, and the space that is free afterwards can be too
-//     fragmented for the grid's last CTAs although the occupancy query counted them in (observed once with a grid sized
-//     to the last register; such grids also leave part of the register file free).  A grid with ONE CTA per SM cannot do
-//     that to itself and may start early;
-// (c) the grid is at most what the occupancy query of that kernel returns, else the plan uses separate finalize kernels.
-__device__ __forceinline__ void grid_arrive(int* ctr) {
-    __threadfence();
-    atomicAdd(ctr, 1);
-}
-__device__ __forceinline__ bool grid_wait(int* ctr, int expected, unsigned long long limit_ns = kWaitLimitNs) {
-    unsigned long long t0 = 0;
-    for (unsigned i = 0;; ++i) {
-        int v;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-        if (v >= expected) return true;
-        if ((i & 255u) == 255u) {
-            unsigned long long now;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) return false;
-        }
-    }
-}
-__device__ __forceinline__ bool grid_arrive_wait(int* ctr, int expected, unsigned long long limit_ns = kWaitLimitNs) {
-    grid_arrive(ctr);
-    return grid_wait(ctr, expected, limit_ns);
-}
-__device__ __forceinline__ void grid_depart(int* ctr, int nblocks) {
-    if (atomicAdd(ctr + 1, 1) == nblocks - 1) {
-        ctr[1] = 0;
-        ctr[0] = 0;
-        __threadfence();
-    }
-}
-
-// Programmatic dependent launch.  A kernel without a grid barrier starts with pdl_launch_dependents() and executes
-// pdl_wait() before its first access to global memory: the next kernel in the stream may then become resident and run its
-// prologue (barrier set-up, TMEM allocation, descriptor prefetch) while this one drains, and still sees all of its results.
-// Because every kernel waits before it finishes, completion of the previous kernel implies completion of all earlier ones.
-// Kernels with a grid barrier: see the rules above grid_arrive.
+// Programmatic dependent launch.  Every kernel starts with pdl_launch_dependents() and executes pdl_wait() before its
+// first access to global memory: the next kernel in the stream may then become resident and run its prologue (barrier
+// set-up, TMEM allocation, descriptor prefetch) while this one drains, and still sees all of its results.  Because every
+// kernel waits before it finishes, completion of the previous kernel implies completion of all earlier ones.  This is
+// safe because no block of any kernel waits for another block: a resident block of the next kernel can delay blocks of
+// this one, never stop them.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -187,9 +135,7 @@ inline bool pdl_enabled() {
 }
 
 // Launches `kernel` on `st` with the programmatic-serialization attribute (and a cluster of `cluster_x` CTAs when > 1).
-// EARLY = false (kernels that contain a grid barrier): without that attribute, i.e. the kernel starts only when its
-// predecessor in the stream has completed.
-template <bool EARLY = true, typename... KArgs, typename... Args>
+template <typename... KArgs, typename... Args>
 inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x, Args&&... args) {
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof lc);
@@ -199,7 +145,7 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     lc.stream = st;
     cudaLaunchAttribute at[2];
     unsigned n = 0;
-    if (EARLY && pdl_enabled()) {
+    if (pdl_enabled()) {
         at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         at[n].val.programmaticStreamSerializationAllowed = 1;
         ++n;

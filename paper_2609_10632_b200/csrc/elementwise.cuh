@@ -190,21 +190,147 @@ template <int V> __device__ __forceinline__ void load_params(const float* __rest
     }
 }
 
+// ------------------------------------------------------------------ per-channel sums kept in fp64 accumulators
+// The kernel that produces per-channel sums (the convolution's epilogue, the backward reduce pass) adds every block's
+// fp32 partial sums to `acc` with fp64 atomics, and every block of the kernel that consumes them (the normalise + SiLU
+// pass, the dy pass) reads the totals and derives its coefficients itself.  No block waits for another one: the
+// producer needs neither a grid-wide barrier nor a resident grid, and the only ordering is the kernel boundary.
+// acc holds `copies` sets of [2][C] doubles (block b adds to set b mod copies, so the cache lines of one set are not
+// the target of every block at once).  The sets are zero when the producer starts: the last block of the consumer to
+// have read them (counted in *readers) zeroes them again.  Adding a few hundred fp32 values in fp64 is exact unless
+// their magnitudes differ by more than 2^29, so the totals do not depend on the order in which the atomics land.
+struct ChanAcc {
+    double* acc;   // NULL: the consumer reads coefficients that a finalize kernel has written
+    int* readers;
+    int copies;
+};
+__device__ __forceinline__ void chan_acc_add(const ChanAcc& ca, int C, int which, int c, float v) {
+    atomicAdd(ca.acc + ((size_t)((int)blockIdx.x % ca.copies) * 2 + which) * C + c, (double)v);
+}
+// totals of channels c and c + 1 (c even) of both sums; read from L2, where the atomics were performed, with the loads
+// of four sets in flight at a time (the consuming pass starts with this latency)
+__device__ __forceinline__ void chan_acc_total2(const ChanAcc& ca, int C, int c, double2& t0, double2& t1) {
+    t0 = t1 = make_double2(0.0, 0.0);
+    const size_t set = (size_t)2 * C;
+    const double* base = ca.acc + c;
+    int k = 0;
+    for (; k + 4 <= ca.copies; k += 4) {
+        double2 a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            a[i] = __ldcg(reinterpret_cast<const double2*>(base + (k + i) * set));
+            b[i] = __ldcg(reinterpret_cast<const double2*>(base + (k + i) * set + C));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            t0.x += a[i].x; t0.y += a[i].y;
+            t1.x += b[i].x; t1.y += b[i].y;
+        }
+    }
+    for (; k < ca.copies; ++k) {
+        const double2 a = __ldcg(reinterpret_cast<const double2*>(base + k * set)), b = __ldcg(reinterpret_cast<const double2*>(base + k * set + C));
+        t0.x += a.x; t0.y += a.y;
+        t1.x += b.x; t1.y += b.y;
+    }
+}
+// One thread per block, after the block's reads of acc (and a block-level barrier): returns the number of blocks that
+// had read before this one.  The value is needed only at the end of the kernel.  No fence: the block's reads have
+// delivered their values (they were used before the barrier), and the zeroes are written only by the block that sees
+// every other block's increment.
+__device__ __forceinline__ int chan_acc_reader_arrive(const ChanAcc& ca) { return atomicAdd(ca.readers, 1); }
+// All threads of the block, `last` block-uniform: the last reader leaves the sets and the counter zeroed.
+__device__ __forceinline__ void chan_acc_reset_if(const ChanAcc& ca, int C, bool last) {
+    if (!last) return;
+    const int n = ca.copies * 2 * C;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) ca.acc[i] = 0.0;
+    if (threadIdx.x == 0) *ca.readers = 0;
+}
+
+// 1/sqrt(v) for v well inside the fp32 range: the fp32 approximation refined by one Newton step in fp64 (relative error
+// below 2^-44, i.e. exact once rounded to fp32 but for values within 2^-20 units in the last place of a rounding
+// boundary).  The library's fp64 rsqrt is a chain three times as long, and every block of the consuming pass waits for it.
+__device__ __forceinline__ double rsqrt_refined(double v) {
+    const float vf = (float)v;
+    if (!(vf > 1e-30f && vf < 1e30f)) return rsqrt(v);
+    const double r = (double)rsqrtf(vf);
+    const double e = fma(-(v * r), r, 1.0);
+    return fma(0.5 * r, e, r);
+}
+
+// What a block of the normalise + SiLU pass needs to turn the totals (sum y, sum y^2) into scale and shift; block 0
+// also writes the batch statistics and updates the running ones (the same fp64 chain as bn_finalize_channel).
+struct FwdFin {
+    double inv_m, unbias;  // 1/M and M/(M-1)
+    float eps, momentum;
+    const float *gamma, *beta;
+    float *mean, *invstd, *rmean, *rvar;
+};
+__device__ __forceinline__ void fwd_coef_from_acc(const ChanAcc& ca, const FwdFin& f, int C, float* s_coef /*[2][C] shared*/) {
+    const bool writer = blockIdx.x == 0;
+    // two channels per thread and round (kept rolled: the fp64 chains must not crowd the registers of the streaming loop)
+#pragma unroll 1
+    for (int c = 2 * (int)threadIdx.x; c < C; c += 2 * (int)blockDim.x) {
+        const float2 ga = *reinterpret_cast<const float2*>(f.gamma + c), be = *reinterpret_cast<const float2*>(f.beta + c);
+        double2 s, q;
+        chan_acc_total2(ca, C, c, s, q);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const double mu = (j ? s.y : s.x) * f.inv_m;
+            double var = (j ? q.y : q.x) * f.inv_m - mu * mu;
+            if (var < 0.0) var = 0.0;
+            const double is = rsqrt_refined(var + (double)f.eps);
+            const double sc = (double)(j ? ga.y : ga.x) * is;
+            s_coef[c + j] = (float)sc;
+            s_coef[C + c + j] = (float)((double)(j ? be.y : be.x) - mu * sc);
+            if (writer) {
+                f.mean[c + j] = (float)mu;
+                f.invstd[c + j] = (float)is;
+                if (f.rmean) {
+                    f.rmean[c + j] = (float)((1.0 - (double)f.momentum) * (double)f.rmean[c + j] + (double)f.momentum * mu);
+                    f.rvar[c + j] = (float)((1.0 - (double)f.momentum) * (double)f.rvar[c + j] + (double)f.momentum * var * f.unbias);
+                }
+            }
+        }
+    }
+}
+template <int V> __device__ __forceinline__ void load_params_shared(const float* s, int cg, float2 (&out)[V / 2]) {
+    const float4* q = reinterpret_cast<const float4*>(s + (size_t)cg * V);
+#pragma unroll
+    for (int i = 0; i < V / 4; ++i) {
+        const float4 t = q[i];
+        out[2 * i] = make_float2(t.x, t.y);
+        out[2 * i + 1] = make_float2(t.z, t.w);
+    }
+}
+
 // ------------------------------------------------------------------ a = SiLU(y*scale + shift)  (ACT = false: no SiLU)
 // RES: a = SiLU(...) + res with res a (possibly pitched) tensor of the output's type -- the residual connection of a
 // bottleneck performed by the block that feeds it; the sum is formed in fp32 and rounded once.
-template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false, bool RES = false>
+// FIN: scale and shift are derived here from the totals in `ca` (dynamic shared memory: 2*C floats); else they are read.
+template <typename YT, typename AT, bool FAST, bool ACT = true, bool PITCHED = false, bool RES = false, bool FIN = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restrict__ y, AT* __restrict__ a,
                                                              long long total_vecs, int C, const float* __restrict__ scale,
-                                                             const float* __restrict__ shift, long long ld_a, const AT* __restrict__ res, long long ld_r) {
+                                                             const float* __restrict__ shift, long long ld_a, const AT* __restrict__ res, long long ld_r,
+                                                             ChanAcc ca, FwdFin fin) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "y and a must have the same element size");
     const int cg = threadIdx.x % (C / V);
     float2 sc[V / 2], sh[V / 2];
-    load_params<V>(scale, cg, sc);
-    load_params<V>(shift, cg, sh);
+    extern __shared__ __align__(16) float s_coef[];
+    __shared__ int s_last;
+    int readers_before = 0;
+    if (FIN) {
+        fwd_coef_from_acc(ca, fin, C, s_coef);
+        __syncthreads();
+        if (threadIdx.x == 0) readers_before = chan_acc_reader_arrive(ca);
+        load_params_shared<V>(s_coef, cg, sc);
+        load_params_shared<V>(s_coef + C, cg, sh);
+    } else {
+        load_params<V>(scale, cg, sc);
+        load_params<V>(shift, cg, sh);
+    }
     const long long stride = (long long)gridDim.x * blockDim.x;
     // a may be a channel slice of a wider tensor: row pitch ld_a elements (the stride is a whole number of rows, so the
     // output offset advances by a constant)
@@ -227,6 +353,11 @@ __global__ void __launch_bounds__(288, 3) bn_silu_apply_kernel(const YT* __restr
             pair_from_f32(o.v + 2 * j, out);
         }
         st16(a + oa, o);
+    }
+    if (FIN) {
+        if (threadIdx.x == 0) s_last = readers_before == (int)gridDim.x - 1;
+        __syncthreads();
+        chan_acc_reset_if(ca, C, s_last != 0);
     }
 }
 
@@ -302,17 +433,13 @@ __device__ __forceinline__ void bn_bwd_finalize_channel(const float* __restrict_
 // z = y*a + b with a = gamma*invstd, b = beta - mean*a (recomputed here from the saved statistics).  The second
 // sum is taken against y itself; sum dz*xhat = invstd*(sum dz*y - mean*sum dz) is formed in fp64 by the finalize
 // kernel, so this pass needs only two per-channel values per element.
-// What the reduce kernel needs to finalize by itself (on = 0: it only writes the partial sums).
+// Extras of the reduce kernel: with acc.acc != NULL the block sums go to the fp64 accumulators (and `partials` is not
+// written); w / wt: filter and its rearranged copy for the data-gradient GEMM (wt = NULL: nothing to rearrange), work
+// that the blocks of this kernel carry along because the memory latency of a few filter tiles costs them nothing.
 struct BwdFused {
-    int on;
-    int* ctr;     // arrive/depart counters of the grid barrier
-    int* status;  // the plan's status block
-    double M;
-    float *dgamma, *dbeta, *coef;
-    const __nv_bfloat16* w;  // filter and its rearranged copy for the data-gradient GEMM (wt = NULL: nothing to rearrange)
+    ChanAcc acc;
+    const __nv_bfloat16* w;
     __nv_bfloat16* wt;
-    int wait_limit_ms;  // bound of the grid-barrier wait in milliseconds (0: the default of about two seconds)
-    int bar_extra;      // test knob: the barrier expects this many more arrivals than there are blocks (0 in normal use)
 };
 template <typename YT, typename AT, bool FAST, bool PITCHED = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
@@ -320,9 +447,7 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
                                                                   const float* __restrict__ invstd, const float* __restrict__ gamma,
                                                                   const float* __restrict__ beta, float* __restrict__ partials, BwdFused fb,
                                                                   WtParams wtp, long long ld_g) {
-    // With the fused finalize this kernel contains a grid barrier: it is launched without the programmatic-serialization
-    // attribute and lets the next kernel go only behind the barrier (see grid_arrive).
-    if (!fb.on) pdl_launch_dependents();
+    pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
     static_assert(V == Vec16<AT>::N, "g and y must have the same element size");
@@ -330,10 +455,10 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
     const int tid = threadIdx.x;
     const int cgs = C / V;
     const int cg = tid % cgs;
-    // Fused mode: the first two filter tiles of this block (for the data-gradient GEMM's rearranged filter) are requested
-    // now with cp.async and written back after the streaming loop, so their memory latency costs nothing.
+    // The first two filter tiles of this block (for the data-gradient GEMM's rearranged filter) are requested now with
+    // cp.async and written back after the streaming loop, so their memory latency costs nothing.
     __shared__ __align__(16) WtTileBuf wtile[2];
-    const int wt_tiles = (fb.on && fb.wt) ? wt_num_tiles(wtp) : 0;
+    const int wt_tiles = fb.wt ? wt_num_tiles(wtp) : 0;
     if (wt_tiles > 0) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
@@ -386,38 +511,21 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_reduce_kernel(const AT* __
             const int gq = c / V, e = c % V;
             float acc = 0.f;
             for (int r = 0; r < R; ++r) acc += red[(r * cgs + gq) * V + e];
-            partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;  // pass 0: sum dz, pass 1: sum dz*y
+            // pass 0: sum dz, pass 1: sum dz*y
+            if (fb.acc.acc) chan_acc_add(fb.acc, C, pass, c, acc);
+            else partials[((size_t)blockIdx.x * 2 + pass) * C + c] = acc;
         }
         __syncthreads();
     }
-    if (fb.on) {
-        // Fused finalize: the grid is one wave of resident blocks, so a grid-wide barrier is safe.  Between arriving and
-        // waiting the block writes back its filter tiles; afterwards block b finalizes channels b, b + gridDim.x, ...
-        // with one warp per channel.
-        __shared__ int ok;
-        if (tid == 0) grid_arrive(fb.ctr);
-        if (wt_tiles > 0) {
-            wt_async_wait();
-            __syncthreads();
+    if (wt_tiles > 0) {
+        wt_async_wait();
+        __syncthreads();
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const int t = (int)blockIdx.x + k * (int)gridDim.x;
-                if (t < wt_tiles) wt_tile_store(fb.wt, wtp, wt_tile_decode(wtp, t), wtile[k]);
-            }
-            if (wt_tiles > 2 * (int)gridDim.x) wt_transform_blocks(fb.w, fb.wt, wtp, (int)blockIdx.x, (int)gridDim.x, 2);  // rare: very large filters
+        for (int k = 0; k < 2; ++k) {
+            const int t = (int)blockIdx.x + k * (int)gridDim.x;
+            if (t < wt_tiles) wt_tile_store(fb.wt, wtp, wt_tile_decode(wtp, t), wtile[k]);
         }
-        if (tid == 0) ok = grid_wait(fb.ctr, (int)gridDim.x + fb.bar_extra, wait_limit_ns(fb.wait_limit_ms)) ? 1 : 0;
-        __syncthreads();
-        pdl_launch_dependents();  // every block of this grid is resident and past the barrier
-        if (ok) {
-            const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-            for (int c = (int)blockIdx.x + (int)gridDim.x * warp; c < C; c += (int)gridDim.x * nwarps)
-                bn_bwd_finalize_channel<true>(partials, (int)gridDim.x, C, c, lane, fb.M, mean, invstd, gamma, beta, fb.dgamma, fb.dbeta, fb.coef);
-        } else if (tid == 0) {
-            report_timeout(fb.status, SITE_GRID_BARRIER_BWD, (int)blockIdx.x);
-        }
-        __syncthreads();
-        if (tid == 0) grid_depart(fb.ctr, (int)gridDim.x);
+        if (wt_tiles > 2 * (int)gridDim.x) wt_transform_blocks(fb.w, fb.wt, wtp, (int)blockIdx.x, (int)gridDim.x, 2);  // rare: very large filters
     }
 }
 
@@ -441,19 +549,66 @@ __global__ void __launch_bounds__(256) bn_bwd_finalize_kernel(const float* __res
 }
 
 // ------------------------------------------------------------------ dy = a*dz - p1*y + p0
-template <typename YT, typename AT, bool FAST, bool PITCHED = false>
+// What a block of the dy pass needs to turn the totals (sum dz, sum dz*y) into its four coefficients; block 0 also
+// writes dgamma and dbeta (the same fp64 chain as bn_bwd_finalize_channel).
+struct BwdFin {
+    double inv_m;
+    const float *mean, *invstd, *gamma, *beta;
+    float *dgamma, *dbeta;
+};
+__device__ __forceinline__ void bwd_coef_from_acc(const ChanAcc& ca, const BwdFin& f, int C, float* s_coef /*[4][C] shared*/) {
+    const bool writer = blockIdx.x == 0;
+#pragma unroll 1
+    for (int c = 2 * (int)threadIdx.x; c < C; c += 2 * (int)blockDim.x) {  // two channels per thread and round, see fwd_coef_from_acc
+        const float2 mu_f = *reinterpret_cast<const float2*>(f.mean + c), is_f = *reinterpret_cast<const float2*>(f.invstd + c);
+        const float2 ga = *reinterpret_cast<const float2*>(f.gamma + c), be = *reinterpret_cast<const float2*>(f.beta + c);
+        double2 t0, t1;
+        chan_acc_total2(ca, C, c, t0, t1);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const double mu = (double)(j ? mu_f.y : mu_f.x), is = (double)(j ? is_f.y : is_f.x);
+            const double s0 = j ? t0.y : t0.x, s1 = j ? t1.y : t1.x;
+            const double dg = is * (s1 - mu * s0);
+            const double a = (double)(j ? ga.y : ga.x) * is;
+            const double p1 = a * is * dg * f.inv_m;
+            s_coef[c + j] = (float)a;
+            s_coef[C + c + j] = (float)((double)(j ? be.y : be.x) - mu * a);
+            s_coef[2 * C + c + j] = (float)p1;
+            s_coef[3 * C + c + j] = (float)(p1 * mu - a * s0 * f.inv_m);
+            if (writer) {
+                f.dbeta[c + j] = (float)s0;
+                f.dgamma[c + j] = (float)dg;
+            }
+        }
+    }
+}
+// FIN: the coefficients are derived here from the totals in `ca` (dynamic shared memory: 4*C floats); else read from coef.
+template <typename YT, typename AT, bool FAST, bool PITCHED = false, bool FIN = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
-                                                              const float* __restrict__ coef, long long ld_g) {
+                                                              const float* __restrict__ coef, long long ld_g, ChanAcc ca, BwdFin fin) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
     const int cg = threadIdx.x % (C / V);
     float2 a[V / 2], b[V / 2], np1[V / 2], p0[V / 2];
-    load_params<V>(coef, cg, a);
-    load_params<V>(coef + C, cg, b);
-    load_params<V>(coef + 2 * C, cg, np1);
-    load_params<V>(coef + 3 * C, cg, p0);
+    extern __shared__ __align__(16) float s_coef[];
+    __shared__ int s_last;
+    int readers_before = 0;
+    if (FIN) {
+        bwd_coef_from_acc(ca, fin, C, s_coef);
+        __syncthreads();
+        if (threadIdx.x == 0) readers_before = chan_acc_reader_arrive(ca);
+        load_params_shared<V>(s_coef, cg, a);
+        load_params_shared<V>(s_coef + C, cg, b);
+        load_params_shared<V>(s_coef + 2 * C, cg, np1);
+        load_params_shared<V>(s_coef + 3 * C, cg, p0);
+    } else {
+        load_params<V>(coef, cg, a);
+        load_params<V>(coef + C, cg, b);
+        load_params<V>(coef + 2 * C, cg, np1);
+        load_params<V>(coef + 3 * C, cg, p0);
+    }
 #pragma unroll
     for (int j = 0; j < V / 2; ++j) np1[j] = make_float2(-np1[j].x, -np1[j].y);
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -476,6 +631,11 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
             pair_from_f32(o.v + 2 * j, fma2(a[j], dz, fma2(np1[j], yv, p0[j])));
         }
         st16(dy + v * V, o);
+    }
+    if (FIN) {
+        if (threadIdx.x == 0) s_last = readers_before == (int)gridDim.x - 1;
+        __syncthreads();
+        chan_acc_reset_if(ca, C, s_last != 0);
     }
 }
 

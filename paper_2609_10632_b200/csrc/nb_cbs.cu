@@ -11,6 +11,7 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "common.cuh"
@@ -58,6 +59,9 @@ struct EwCfg {  // launch geometry of the [M][C] passes
 
 }  // namespace
 
+constexpr size_t kStatusBytes = 256;  // ST_WORDS ints, padded so that what follows in the same allocation is 256-byte aligned
+static_assert(ST_WORDS * sizeof(int) <= kStatusBytes, "status block");
+
 struct nb_cbs_plan_s {
     nb_cbs_desc desc;
     Geom g;
@@ -75,8 +79,11 @@ struct nb_cbs_plan_s {
     long long ld_dx = 0;           // row pitch of dx in the data-gradient call and whether dx is added to (nb_cbs_plan_set_dx_target)
     bool dx_accumulate = false;
     bool pitched = false;
-    bool fuse_finalize = true;  // BN finalizes behind in-kernel grid barriers (off: NB_CBS_FLAG_SHARED_GPU, or an occupancy query that failed)
-    int expire_next_ms = 0;     // nb_cbs_debug_expire_next_wait: the next grid-barrier launch waits for one block too many, for at most this long
+    // Channel sums go to fp64 accumulators that the consuming pass turns into coefficients itself (ChanAcc); off
+    // (NB_CBS_FLAG_SEPARATE_FINALIZE, fp32 mode): per-block partial sums and separate finalize kernels.
+    bool fuse_finalize = true;
+    double* acc = nullptr;      // device: [acc_copies_f][2][C] forward sums, then [acc_copies_b][2][C] backward sums; zero between calls
+    int acc_copies_f = 0, acc_copies_b = 0;
     bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
     int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
@@ -151,25 +158,35 @@ nb_status run_finalize(nb_cbs_plan_s* p, const float* partials, int nparts, cons
 }
 
 // res != NULL (training forward with SiLU only): a = SiLU(...) + res, res with row pitch ld_res elements.
+// fin != NULL (training forward with SiLU only): scale and shift are derived inside the kernel from the plan's forward accumulators.
 template <typename YT, typename AT, bool FAST, bool ACT = true>
 nb_status run_apply(nb_cbs_plan_s* p, const void* y, void* a, const float* scale, const float* shift, cudaStream_t st, long long ld_a = 0,
-                    const void* res = nullptr, long long ld_res = 0) {
+                    const void* res = nullptr, long long ld_res = 0, const FwdFin* fin = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
     SiteTimer tm(p, SITE_APPLY, st);
+    const ChanAcc none{nullptr, nullptr, 1};
+    const FwdFin nofin{};
+    auto go = [&](auto kernel, const ChanAcc& ca, const FwdFin& f, size_t smem) {
+        launch_k(kernel, dim3(e.blocks_apply), dim3(e.tpb), smem, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a), e.total_vecs, C, scale, shift,
+                 ld_a ? ld_a : (long long)C, static_cast<const AT*>(res), ld_res ? ld_res : (long long)C, ca, f);
+    };
     if constexpr (ACT) {
+        if (fin) {
+            const ChanAcc ca{p->acc, p->status + ST_READERS_FWD, p->acc_copies_f};
+            const size_t smem = (size_t)2 * C * sizeof(float);
+            if (res) go(bn_silu_apply_kernel<YT, AT, FAST, true, true, true, true>, ca, *fin, smem);
+            else if (ld_a) go(bn_silu_apply_kernel<YT, AT, FAST, true, true, false, true>, ca, *fin, smem);
+            else go(bn_silu_apply_kernel<YT, AT, FAST, true, false, false, true>, ca, *fin, smem);
+            return launch_ok("bn_silu_apply (statistics from the accumulators)");
+        }
         if (res) {
-            launch_k(bn_silu_apply_kernel<YT, AT, FAST, true, true, true>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
-                     e.total_vecs, C, scale, shift, ld_a ? ld_a : (long long)C, static_cast<const AT*>(res), ld_res ? ld_res : (long long)C);
+            go(bn_silu_apply_kernel<YT, AT, FAST, true, true, true>, none, nofin, 0);
             return launch_ok("bn_silu_apply (+ residual)");
         }
     }
-    if (ld_a)
-        launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, true>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
-                 e.total_vecs, C, scale, shift, ld_a, static_cast<const AT*>(nullptr), 0LL);
-    else
-        launch_k(bn_silu_apply_kernel<YT, AT, FAST, ACT, false>, dim3(e.blocks_apply), dim3(e.tpb), 0, st, 1, static_cast<const YT*>(y), static_cast<AT*>(a),
-                 e.total_vecs, C, scale, shift, (long long)C, static_cast<const AT*>(nullptr), 0LL);
+    if (ld_a) go(bn_silu_apply_kernel<YT, AT, FAST, ACT, true>, none, nofin, 0);
+    else go(bn_silu_apply_kernel<YT, AT, FAST, ACT, false>, none, nofin, 0);
     return launch_ok("bn_silu_apply");
 }
 
@@ -179,32 +196,23 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
                               float* coef, cudaStream_t st, const void* w = nullptr, void* wt = nullptr, const WtParams* wtp = nullptr) {
     const EwCfg& e = p->ew;
     const int C = p->g.c_out;
-    const bool fuse = p->fuse_finalize;
+    const bool fuse = p->fuse_finalize && !std::is_same<YT, float>::value;
     WtParams none;
     if (!wtp) memset(&none, 0, sizeof none);
+    const ChanAcc ca{fuse ? p->acc + (size_t)p->acc_copies_f * 2 * C : nullptr, p->status + ST_READERS_BWD, p->acc_copies_b};
     {
-        // one wave of resident blocks: the kernel finalizes behind a grid-wide barrier and rearranges the dgrad filter meanwhile
+        // sums of dz and dz*y per channel (into the accumulators, or as per-block partial sums); the blocks also rearrange the dgrad filter
         SiteTimer tm(p, SITE_BWD_REDUCE, st);
         BwdFused fb;
         memset(&fb, 0, sizeof fb);
+        fb.acc = ca;
         if (fuse) {
-            fb.on = 1; fb.ctr = p->status + ST_BAR_BWD; fb.status = p->status; fb.M = (double)p->g.m;
-            if (p->expire_next_ms > 0) {
-                fb.wait_limit_ms = p->expire_next_ms; fb.bar_extra = 1;
-                p->expire_next_ms = 0;
-            }
-            fb.dgamma = dgamma; fb.dbeta = dbeta; fb.coef = coef;
             fb.w = static_cast<const __nv_bfloat16*>(w); fb.wt = wtp ? static_cast<__nv_bfloat16*>(wt) : nullptr;
         }
-        // with the grid barrier (fuse): launched without the programmatic-serialization attribute, see grid_arrive
         const size_t red_smem = (size_t)e.tpb * e.vec * sizeof(float);
         auto go = [&](auto kernel, long long ld) {
-            if (fuse)
-                launch_k<false>(kernel, dim3(e.blocks_reduce), dim3(e.tpb), red_smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean,
-                                invstd, gamma, beta, partials, fb, wtp ? *wtp : none, ld);
-            else
-                launch_k(kernel, dim3(e.blocks_reduce), dim3(e.tpb), red_smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd,
-                         gamma, beta, partials, fb, wtp ? *wtp : none, ld);
+            launch_k(kernel, dim3(e.blocks_reduce), dim3(e.tpb), red_smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), e.total_vecs, C, mean, invstd,
+                     gamma, beta, partials, fb, wtp ? *wtp : none, ld);
         };
         if (p->ld_g) go(bn_silu_bwd_reduce_kernel<YT, AT, FAST, true>, p->ld_g);
         else go(bn_silu_bwd_reduce_kernel<YT, AT, FAST, false>, (long long)C);
@@ -223,12 +231,19 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
         NB_LAUNCH_OK("bn_bwd_finalize");
     }
     SiteTimer tm(p, SITE_BWD_DY, st);
-    if (p->ld_g)
-        launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST, true>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
-                 static_cast<AT*>(dy), e.total_vecs, C, coef, p->ld_g);
-    else
-        launch_k(bn_silu_bwd_dy_kernel<YT, AT, FAST, false>, dim3(e.blocks_dy), dim3(e.tpb), 0, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y),
-                 static_cast<AT*>(dy), e.total_vecs, C, coef, (long long)C);
+    const BwdFin bf{1.0 / (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta};
+    auto go_dy = [&](auto kernel, size_t smem) {
+        launch_k(kernel, dim3(e.blocks_dy), dim3(e.tpb), smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), static_cast<AT*>(dy), e.total_vecs, C, coef,
+                 p->ld_g ? p->ld_g : (long long)C, ca, bf);
+    };
+    const size_t coef_smem = (size_t)4 * C * sizeof(float);
+    if (fuse) {
+        if (p->ld_g) go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, true, true>, coef_smem);
+        else go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, false, true>, coef_smem);
+    } else {
+        if (p->ld_g) go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, true, false>, 0);
+        else go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, false, false>, 0);
+    }
     return launch_ok("bn_silu_bwd_dy");
 }
 
@@ -323,7 +338,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->g = g;
     p->device = device;
     p->sm_count = prop.multiProcessorCount;
-    p->fuse_finalize = !(d->flags & NB_CBS_FLAG_SHARED_GPU);
+    p->fuse_finalize = !(d->flags & NB_CBS_FLAG_SEPARATE_FINALIZE) && d->mode != NB_MODE_F32_REF;
 
     EwCfg& e = p->ew;
     e.vec = vec;
@@ -342,12 +357,13 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, e.tpb, dyn_smem) != cudaSuccess || occ < 1) {
                 cudaGetLastError();
                 occ = 1;
-                p->fuse_finalize = false;  // residency unknown: no grid barriers on this plan (separate finalize kernels)
             }
             const long long cap = (long long)p->sm_count * occ;
             return (int)std::max<long long>(1, std::min<long long>((max_blocks + min_vecs - 1) / min_vecs, cap));
         };
         const size_t red_smem = (size_t)e.tpb * vec * sizeof(float);
+        // the passes that derive their coefficients from the accumulators keep them in dynamic shared memory
+        const size_t apply_smem = p->fuse_finalize ? (size_t)2 * g.c_out * sizeof(float) : 0, dy_smem = p->fuse_finalize ? (size_t)4 * g.c_out * sizeof(float) : 0;
         if (d->mode == NB_MODE_F32_REF) {
             e.blocks_stats = wave((const void*)bn_stats_partial_kernel<float>, red_smem, 8);
             e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<float, float, false>, red_smem, 8);
@@ -356,13 +372,13 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
         } else if (d->mode == NB_MODE_F16_TC) {
             e.blocks_stats = wave((const void*)bn_stats_partial_kernel<__half>, red_smem, 8);
             e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<__half, __half, true>, red_smem, 8);
-            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __half, true>, 0, 4);
-            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __half, true>, 0, 4);
+            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __half, true, true, false, false, true>, apply_smem, 4);
+            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __half, true, false, true>, dy_smem, 4);
         } else {
             e.blocks_stats = wave((const void*)bn_stats_partial_kernel<__half>, red_smem, 8);
             e.blocks_reduce = wave((const void*)bn_silu_bwd_reduce_kernel<__half, __nv_bfloat16, true>, red_smem, 8);
-            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __nv_bfloat16, true>, 0, 4);
-            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __nv_bfloat16, true>, 0, 4);
+            e.blocks_apply = wave((const void*)bn_silu_apply_kernel<__half, __nv_bfloat16, true, true, false, false, true>, apply_smem, 4);
+            e.blocks_dy = wave((const void*)bn_silu_bwd_dy_kernel<__half, __nv_bfloat16, true, false, true>, dy_smem, 4);
         }
         e.blocks_map = std::max(e.blocks_apply, e.blocks_dy);
     }
@@ -383,8 +399,20 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     int cur = 0;
     NB_CUDA_CHECK(cudaGetDevice(&cur));
     cudaError_t ce = cudaSetDevice(device);
-    if (ce == cudaSuccess) ce = cudaMalloc(&p->status, ST_WORDS * sizeof(int));
-    if (ce == cudaSuccess) ce = cudaMemset(p->status, 0, ST_WORDS * sizeof(int));
+    // one allocation: the status words, then (256-byte aligned) the fp64 channel accumulators
+    {
+        auto copies = [](const char* name, int dflt) {
+            const char* v = getenv(name);
+            const int k = v ? atoi(v) : dflt;
+            return k < 1 ? 1 : k > 16 ? 16 : k;
+        };
+        p->acc_copies_f = p->fuse_finalize ? copies("NB_ACC_COPIES_FWD", 2) : 0;
+        p->acc_copies_b = p->fuse_finalize ? copies("NB_ACC_COPIES_BWD", 4) : 0;
+    }
+    const size_t acc_bytes = (size_t)(p->acc_copies_f + p->acc_copies_b) * 2 * g.c_out * sizeof(double);
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->status, kStatusBytes + acc_bytes);
+    if (ce == cudaSuccess) ce = cudaMemset(p->status, 0, kStatusBytes + acc_bytes);
+    if (ce == cudaSuccess && acc_bytes) p->acc = reinterpret_cast<double*>(reinterpret_cast<char*>(p->status) + kStatusBytes);
     nb_status tcs = NB_OK;
     if (ce == cudaSuccess)
         tcs = tc_plan_init(&p->tc, g, d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT), p->sm_count, prop, d->mode == NB_MODE_F16_TC);
@@ -527,15 +555,6 @@ nb_status nb_cbs_profile_enable(nb_cbs_plan p, int32_t enable) {
     return NB_OK;
 }
 
-nb_status nb_cbs_debug_expire_next_wait(nb_cbs_plan p, int32_t limit_ms) {
-    g_err.clear();
-    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
-    if (limit_ms < 1 || limit_ms > 1000) return fail(NB_ERR_INVALID_ARG, "limit_ms must be between 1 and 1000, got %d", limit_ms);
-    if (!p->fuse_finalize) return fail(NB_ERR_UNSUPPORTED, "this plan launches no kernel with a grid barrier");
-    p->expire_next_ms = limit_ms;
-    return NB_OK;
-}
-
 const char* nb_cbs_profile_site_name(int32_t site) { return (site >= 0 && site < SITE_COUNT) ? kSiteNames[site] : nullptr; }
 
 nb_status nb_cbs_profile_read(nb_cbs_plan p, int32_t site, double* total_ms, int64_t* launches) {
@@ -555,6 +574,8 @@ nb_status nb_cbs_poll_status(nb_cbs_plan p, void* stream) {
     NB_CUDA_CHECK(cudaStreamSynchronize(st));
     NB_CUDA_CHECK(cudaMemcpy(host, p->status, sizeof host, cudaMemcpyDeviceToHost));
     NB_CUDA_CHECK(cudaMemset(p->status, 0, sizeof host));
+    if (host[ST_ERR] != 0 && p->acc)  // a kernel that gave up may have left sums behind: the next call must find zeros
+        NB_CUDA_CHECK(cudaMemset(p->acc, 0, (size_t)(p->acc_copies_f + p->acc_copies_b) * 2 * p->g.c_out * sizeof(double)));
     if (host[ST_ERR] != 0)
         return fail((nb_status)host[ST_ERR], "device status: error %d at site %d (detail %d)", host[ST_ERR], host[ST_WHERE], host[ST_DETAIL]);
     if (host[ST_SAT] != 0) {
@@ -596,12 +617,10 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
-        // writes y (fp16) and the partial sums and, after a grid-wide barrier, finalizes the statistics itself
-        const bool fuse = p->fuse_finalize && p->tc.fp_barrier_ok;
-        const FwdFinalize fin{p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var};
-        const int expire_ms = fuse ? p->expire_next_ms : 0;
-        if (fuse) p->expire_next_ms = 0;
-        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, fuse ? &fin : nullptr, expire_ms, expire_ms > 0 ? 1 : 0);
+        // writes y (fp16) and adds its channel sums to the accumulators (or writes them as per-CTA partial sums)
+        const bool fuse = p->fuse_finalize;
+        const ChanAcc ca{fuse ? p->acc : nullptr, nullptr, fuse ? p->acc_copies_f : 1};
+        const nb_status ts = tc_fprop(&p->tc, p->g, x, w, y_saved, part, p->status, st, ca);
         g_launches.fetch_add((unsigned long long)(p->tc.launches - l0), std::memory_order_relaxed);
         if (ts != NB_OK) return fail(ts, "%s", tc_last_error());
         nparts = p->tc.fprop_parts;
@@ -613,7 +632,10 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     if (!finalized)
         NB_TRY(run_finalize(p, part, nparts, gamma, beta, save_mean, save_invstd, scale, shift, running_mean, running_var, nullptr, nullptr, st));
     if (is_f32(p)) return run_apply<float, float, false>(p, y_saved, a_out, scale, shift, st, p->ld_a, p->fwd_res, p->ld_res);
-    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a, p->fwd_res, p->ld_res));
+    // after the tensor-core kernel the pass derives mean, invstd, scale and shift from the accumulators itself
+    const double M = (double)p->g.m;
+    const FwdFin fin{1.0 / M, M / (M - 1.0), p->desc.eps, p->desc.momentum, gamma, beta, save_mean, save_invstd, running_mean, running_var};
+    return NB_WITH_AT(p, run_apply<__half, AT, true>(p, y_saved, a_out, scale, shift, st, p->ld_a, p->fwd_res, p->ld_res, finalized ? &fin : nullptr));
 }
 
 namespace {

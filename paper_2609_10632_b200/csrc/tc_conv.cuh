@@ -54,14 +54,12 @@ struct IgemmParams {
     int out_accumulate;  // the TMA stores are reductions: the tile is added to what the output tensor holds (data gradient into a shared gradient buffer)
     int out_w[3];
     CUtensorMap tmOut[3];
-    // Fused BatchNorm finalize (statistics variant, fin_on != 0): after a grid-wide barrier CTA b finalizes channels
-    // b, b + gridDim.x, ...: sums the per-CTA partials in fp64 and writes mean, invstd, scale, shift and the running
-    // statistics, which saves the separate finalize launch between this kernel and the apply pass.
-    int fin_on;
-    float fin_eps, fin_momentum;
-    double fin_count;
-    const float *fin_gamma, *fin_beta;
-    float *fin_mean, *fin_invstd, *fin_scale, *fin_shift, *fin_rmean, *fin_rvar;
+    // Statistics variant: with acc.acc != NULL every CTA adds its channel sums to the plan's fp64 accumulators (the
+    // normalise + SiLU pass derives mean, invstd, scale and shift from them, see ChanAcc); else it writes them to
+    // `partials` for a separate finalize kernel.
+    ChanAcc acc;
+    float fin_eps;
+    const float *fin_gamma, *fin_beta, *fin_rmean, *fin_rvar;
     // Fused per-channel epilogue (EPI variant: evaluation-mode BN or a bias, then optionally SiLU, applied to the fp32
     // accumulators before they are rounded): out = act(acc*scale_c + shift_c).  The CTA derives the coefficients itself
     // from fin_gamma / fin_beta / fin_rmean / fin_rvar / fin_eps (gamma NULL: scale 1; rmean NULL: shift = beta or 0).
@@ -74,8 +72,6 @@ struct IgemmParams {
     void* out;
     float* partials;  // [gridDim.x][2][ldo] per-CTA channel sums and sums of squares (statistics variant only)
     int* status;
-    int wait_limit_ms;  // bound of the grid-barrier wait in milliseconds (0: the default of about two seconds)
-    int bar_extra;      // test knob: the grid barrier expects this many more arrivals than there are CTAs (0 in normal use)
     uint16_t off_w[4][9], off_h[4][9];
 };
 
@@ -276,8 +272,7 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
 // bytes written to and read from each SM's shared memory.
 // EPI = 1: the epilogue applies a per-channel scale and shift (evaluation-mode BN or a bias) and optionally SiLU to the
 // accumulators, so the kernel writes the block's final activations (no statistics, no second pass); TMA stores only.
-// STATS (forward of a training block): TMA stores only; with fin_on the kernel ends in a grid-wide barrier, so it is
-// launched without the programmatic-serialization attribute and lets its dependents go only behind that barrier.
+// STATS (forward of a training block): TMA stores only; the epilogue also sums every channel's values and squares.
 template <typename OutT, bool STATS, bool CG2, int EPI = 0, bool CLS4 = false>
 __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_constant__ IgemmParams p) {
     static_assert(!CLS4 || (!STATS && !EPI), "four classes: the stride-2 data gradient only");
@@ -299,9 +294,8 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    // A kernel that ends in a grid-wide barrier lets the next kernel of the stream start only once that barrier has been
-    // passed (see the epilogue); all others let it become resident and run its prologue right away.
-    if (!STATS) pdl_launch_dependents();
+    // the next kernel of the stream may become resident and run its prologue right away
+    pdl_launch_dependents();
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // warp index in a form the compiler knows to be uniform
     const int total_tiles = p.nclasses * p.tiles_per_class;
     const int mh = p.mh;          // 128-row sub-tiles per tile (1 or 2); both share every B stage
@@ -747,29 +741,9 @@ __global__ void __launch_bounds__(IG_THREADS, 1) tc_igemm_kernel(const __grid_co
                 const int tm = cc >= p.ncol_a ? 1 : 0;
                 const int ld = p.n_tiles * (tm ? ncb : p.ncol_a);
                 const float* base = wstat + (tm ? (size_t)8 * p.n_tiles * p.ncol_a : 0) + (size_t)which * ld + nt * (tm ? ncb : p.ncol_a) + (cc - (tm ? p.ncol_a : 0));
-                dst[e] = ((base[0] + base[2 * ld]) + base[4 * ld]) + base[6 * ld];
-            }
-            if (p.fin_on) {
-                int* ctr = p.status + ST_BAR_FWD;
-                volatile int* fin_ok = abort_flag + 1;  // (the kernel uses all of the opt-in shared memory as dynamic: no static variables)
-                epi2_bar_sync();  // this CTA's partial sums are written
-                if (et == 0) *fin_ok = grid_arrive_wait(ctr, (int)gridDim.x + p.bar_extra, wait_limit_ns(p.wait_limit_ms)) ? 1 : 0;
-                epi2_bar_sync();
-                // Every CTA of this grid is resident and past the barrier: only now may the next kernel of the stream take
-                // SM resources (before the barrier its CTAs could have kept CTAs of this grid from becoming resident).
-                pdl_launch_dependents();
-                if (*fin_ok) {
-                    const int ew = et >> 5;
-                    for (int c = (int)blockIdx.x + (int)gridDim.x * ew; c < p.ldo; c += (int)gridDim.x * 8)
-                        bn_finalize_channel<true>(p.partials, (int)gridDim.x, p.ldo, c, lane, p.fin_count, p.fin_eps, p.fin_momentum, p.fin_gamma, p.fin_beta,
-                                                  p.fin_mean, p.fin_invstd, p.fin_scale, p.fin_shift, p.fin_rmean, p.fin_rvar, nullptr, nullptr);
-                } else if (et == 0) {
-                    report_timeout(p.status, SITE_GRID_BARRIER_FWD, (int)blockIdx.x);
-                }
-                epi2_bar_sync();  // every warp is past its reads of the partial sums
-                if (et == 0) grid_depart(ctr, (int)gridDim.x);
-            } else {
-                pdl_launch_dependents();
+                const float v = ((base[0] + base[2 * ld]) + base[4 * ld]) + base[6 * ld];
+                if (p.acc.acc) chan_acc_add(p.acc, p.ldo, which, c, v);
+                else dst[e] = v;
             }
         }
         if (sat) atomicAdd(p.status + ST_SAT, sat);
@@ -813,7 +787,6 @@ struct TcPlan {
     bool fprop = false, dgrad = false, wgrad = false;
     bool f16 = false;  // operands and 16-bit outputs are IEEE fp16 instead of bf16 (same kernels, other instruction-descriptor formats)
     long long ld_x = 0;        // row pitch (elements) of the input activation when it is a channel slice of a wider tensor (0 = dense)
-    bool fp_barrier_ok = false;  // the forward launch's whole grid fits the device at once (asked of the runtime at plan creation)
     int fprop_parts = 0;
     size_t wt_bytes = 0;
     size_t wgrad_partial_bytes = 0;
@@ -1048,12 +1021,8 @@ template <typename OutT, bool STATS, bool CG2, int EPI, bool CLS4> inline bool i
 }
 template <typename OutT, bool STATS, bool CG2, int EPI = 0, bool CLS4 = false> inline nb_status launch_igemm_impl(const TcGemmSlot& s, cudaStream_t st) {
     if (!igemm_allow_smem<OutT, STATS, CG2, EPI, CLS4>()) return NB_ERR_CUDA;
-    // Also the forward launch that ends in a grid barrier may become resident beside its predecessor: it runs one CTA
-    // per SM (more than half of the shared memory each), so a CTA of it that is resident early can never keep another CTA
-    // of the same grid from fitting once the predecessor's CTAs have left, and nothing the predecessor waits for is
-    // held by it.  (Grids with several CTAs per SM are different: see grid_arrive.)
-    // Measured: launching it only after its predecessor has completed costs 3.4 us per forward kernel (its prologue --
-    // barrier set-up, TMEM allocation, tensor-map fetch -- no longer overlaps the predecessor's tail).
+    // (Measured: launching a kernel only after its predecessor has completed costs 3.4 us per launch: its prologue --
+    // barrier set-up, TMEM allocation, tensor-map fetch -- no longer overlaps the predecessor's tail.)
     const cudaError_t e = launch_k(tc_igemm_kernel<OutT, STATS, CG2, EPI, CLS4>, dim3((unsigned)s.cfg.grid), dim3(IG_THREADS), s.cfg.smem_bytes, st, CG2 ? 2 : 1, s.prm);
     if (e != cudaSuccess) {
         err() = std::string("launch of tc_igemm_kernel failed: ") + cudaGetErrorString(e);
@@ -1067,39 +1036,6 @@ template <typename OutT, bool STATS> inline nb_status launch_igemm(const TcGemmS
     }
     return s.cfg.cg2 ? launch_igemm_impl<OutT, STATS, true>(s, st) : launch_igemm_impl<OutT, STATS, false>(s, st);
 }
-// Whether all CTAs of the forward launch with statistics can be resident at once on the current device (the condition of
-// its grid barrier), asked of the runtime for this kernel, block size and shared-memory size.
-inline bool igemm_fwd_grid_fits(const IgemmCfg& c, int sm_count) {
-    int per_sm = 0;
-    if (c.cg2) {
-        if (!igemm_allow_smem<__half, true, true, 0, false>()) return false;
-        cudaLaunchConfig_t lc;
-        memset(&lc, 0, sizeof lc);
-        lc.gridDim = dim3((unsigned)c.grid);
-        lc.blockDim = dim3(IG_THREADS);
-        lc.dynamicSmemBytes = c.smem_bytes;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = 2;
-        at[0].val.clusterDim.y = 1;
-        at[0].val.clusterDim.z = 1;
-        lc.attrs = at;
-        lc.numAttrs = 1;
-        int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, tc_igemm_kernel<__half, true, true, 0, false>, &lc) != cudaSuccess) {
-            cudaGetLastError();
-            return false;
-        }
-        return c.grid <= 2 * clusters;
-    }
-    if (!igemm_allow_smem<__half, true, false, 0, false>()) return false;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_igemm_kernel<__half, true, false, 0, false>, IG_THREADS, c.smem_bytes) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
-    return c.grid <= per_sm * sm_count;
-}
-
 }  // namespace tcdetail
 
 inline const char* tc_last_error() { return tcdetail::err().c_str(); }
@@ -1109,9 +1045,6 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
 inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_count, const cudaDeviceProp&, bool f16 = false) {
     const nb_status st = tc_plan_init_impl(tc, g, enable, sm_count);
     tc->f16 = f16;
-    // the forward kernel may finalize the statistics behind a grid barrier only if the runtime confirms that its whole grid
-    // can be resident at once
-    if (st == NB_OK && tc->fprop) tc->fp_barrier_ok = tcdetail::igemm_fwd_grid_fits(tc->fp.cfg, sm_count);
     if (st == NB_OK && f16) {  // A and B formats of the instruction descriptors: bits 7 and 10 set = bf16, clear = f16
         const uint32_t fmt = (1u << 7) | (1u << 10);
         tc->fp.prm.idesc &= ~fmt;
@@ -1303,14 +1236,9 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
     return NB_OK;
 }
 
-struct FwdFinalize {  // inputs and outputs of the BatchNorm finalize that the forward kernel performs itself
-    float eps, momentum;
-    const float *gamma, *beta;
-    float *mean, *invstd, *scale, *shift, *rmean, *rvar;
-};
-// fin == NULL: the kernel only writes y and the per-CTA partial sums.  wait_limit_ms / bar_extra: see IgemmParams (0 in normal use).
+// acc.acc != NULL: the kernel adds its channel sums to the fp64 accumulators; else it writes per-CTA partial sums.
 inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* w, void* y, float* partials, int* status, cudaStream_t st,
-                          const FwdFinalize* fin, int wait_limit_ms = 0, int bar_extra = 0) {
+                          const ChanAcc& acc) {
     using namespace tcdetail;
     TcGemmSlot& S = tc->fp;
     if (S.a_ptr != x || S.b_ptr != w) {
@@ -1336,14 +1264,7 @@ inline nb_status tc_fprop(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (!encode_out_maps(S.prm, S.cfg, y, g.m)) return NB_ERR_CUDA;
         S.out_ptr = y;
     }
-    S.prm.fin_on = fin ? 1 : 0;
-    if (fin) {
-        S.prm.fin_eps = fin->eps; S.prm.fin_momentum = fin->momentum; S.prm.fin_count = (double)g.m;
-        S.prm.fin_gamma = fin->gamma; S.prm.fin_beta = fin->beta;
-        S.prm.fin_mean = fin->mean; S.prm.fin_invstd = fin->invstd; S.prm.fin_scale = fin->scale; S.prm.fin_shift = fin->shift;
-        S.prm.fin_rmean = fin->rmean; S.prm.fin_rvar = fin->rvar;
-    }
-    S.prm.wait_limit_ms = wait_limit_ms; S.prm.bar_extra = bar_extra;
+    S.prm.acc = acc;
     S.prm.out = y; S.prm.partials = partials; S.prm.status = status;
     tc->launches += 1;
     return launch_igemm<__half, true>(S, st);
@@ -1381,9 +1302,9 @@ inline nb_status tc_infer(TcPlan* tc, const Geom& g, const void* x, const void* 
         if (!encode_out_maps(S.prm, S.cfg, out, g.m)) return NB_ERR_CUDA;
         S.out_ptr = out;
     }
-    S.prm.fin_on = 0;
+    S.prm.acc = ChanAcc{nullptr, nullptr, 1};
     S.prm.fin_gamma = e.gamma; S.prm.fin_beta = e.beta;
-    S.prm.fin_rmean = const_cast<float*>(e.rmean); S.prm.fin_rvar = const_cast<float*>(e.rvar);  // only read
+    S.prm.fin_rmean = e.rmean; S.prm.fin_rvar = e.rvar;
     S.prm.fin_eps = e.eps; S.prm.epi_act = e.act;
     S.prm.out = out; S.prm.partials = nullptr; S.prm.status = status;
     tc->launches += 1;
