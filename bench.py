@@ -42,7 +42,7 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # a full-size launch is this ratio times the launch's algorithmic bytes (traffic grows in proportion to the tensor sizes).
 NCU_TRAFFIC_OVER_ALGORITHMIC = {
     "conv_fprop": 0.75, "conv_dgrad": 0.76, "conv_wgrad": 1.03,
-    "bn_silu_apply": 0.84, "bn_silu_bwd_reduce": 1.01, "bn_silu_bwd_dy": 0.91,
+    "bn_silu_apply": 0.86, "bn_silu_bwd_reduce": 1.01, "bn_silu_bwd_dy": 0.92,
 }
 
 
