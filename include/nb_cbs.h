@@ -53,7 +53,8 @@
 extern "C" {
 #endif
 
-#define NB_CBS_ABI_VERSION 2u /* 2: adds the evaluation-mode / plain calls (additive) */
+#define NB_CBS_ABI_VERSION 3u /* 2: adds the evaluation-mode / plain calls (additive); 3: flag 2 is NB_CBS_FLAG_SEPARATE_FINALIZE,
+                                  the grid-barrier test hook is gone with the barriers */
 
 typedef int32_t nb_status;
 enum {
@@ -254,7 +255,9 @@ nb_status nb_bn_fold(nb_cbs_plan plan, const void* w, const float* gamma, const 
  *   Limits: c <= 1024 channels, c % 8 == 0 for NB_DTYPE_F16, c % 4 == 0 for NB_DTYPE_F32, m >= 2; anything beyond
  *   returns NB_ERR_UNSUPPORTED (or NB_ERR_INVALID_ARG) with a message and launches nothing.
  *   It runs on the CURRENT device.  The first call on each device looks up the array's device address (one
- *   cudaGetSymbolAddress); make that first call before any stream capture begins.
+ *   cudaGetSymbolAddress); make that first call before any stream capture begins.  The address is cached per
+ *   device for the life of the process: after a cudaDeviceReset of that device it is stale, and this entry point
+ *   must not be used again in that process.
  *   It calls no cudaMalloc / cudaFree and no allocating library routine.
  *   Every call on a device shares the one array, which keeps the previous call's contents; each call overwrites
  *   every entry it later reads, so nothing needs clearing -- but two calls whose kernels overlap on the GPU
