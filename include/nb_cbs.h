@@ -141,6 +141,15 @@ nb_status nb_cbs_plan_set_pitches(nb_cbs_plan plan, int64_t ld_x, int64_t ld_a, 
  * The evaluation-mode, plain and host-buffer calls refuse such a plan. */
 nb_status nb_cbs_plan_set_fwd_residual(nb_cbs_plan plan, const void* res, int64_t ld_res);
 
+/* Backward counterpart of nb_cbs_plan_set_fwd_residual: the gradient that reaches the sum a_out = SiLU(z) + res is the
+ * gradient of both summands, so with gres != NULL nb_conv_bn_silu_bwd_data of this plan also hands its incoming
+ * gradient g to the shortcut: gres (a tensor of g's shape and type, dense or a channel slice with pixels ld_gres
+ * elements apart; 0 = dense) receives gres + g when accumulate = 1 (fp32 sum rounded once to the 16-bit type, exactly
+ * as a separate accumulation pass would) or a copy of g when accumulate = 0.  The dy pass, which reads g anyway, does
+ * it.  gres must not overlap g, dy or dx, and must stay valid while calls of the plan may run; NULL switches it off.
+ * NB_ERR_UNSUPPORTED in fp32 mode and for NB_CBS_FLAG_SEPARATE_FINALIZE plans.  The host-buffer call refuses such a plan. */
+nb_status nb_cbs_plan_set_bwd_residual(nb_cbs_plan plan, void* gres, int64_t ld_gres, int32_t accumulate);
+
 /* Gradient accumulation at fan-out without a separate pass: declare that, in nb_conv_bn_silu_bwd_data of this plan, dx is
  * a channel slice of a wider NHWC tensor (pointer = the slice's first channel, pixels ld_dx elements apart; 0 = dense) and,
  * with accumulate = 1, that the data gradient is ADDED to what dx holds instead of overwriting it (a tensor with several

@@ -29,7 +29,7 @@ EXPORTS = (
     "nb_cbs_profile_read", "nb_bn_stats_static", "nb_cbs_infer_workspace_bytes", "nb_conv_bn_silu_infer", "nb_conv_bias_act",
     "nb_bn_fold", "nb_sgd_plan_create", "nb_sgd_plan_destroy", "nb_sgd_workspace_bytes", "nb_sgd_upload", "nb_sgd_clip_nesterov_step", "nb_sgd_clip_nesterov_step_scaled",
     "nb_slice_add", "nb_maxpool5_fwd", "nb_maxpool5_bwd", "nb_upsample2", "nb_conv_bias_bwd", "nb_cbs_plan_set_pitches",
-    "nb_cbs_plan_set_dx_target", "nb_cbs_plan_set_fwd_residual",
+    "nb_cbs_plan_set_dx_target", "nb_cbs_plan_set_fwd_residual", "nb_cbs_plan_set_bwd_residual",
 )
 
 
@@ -85,6 +85,7 @@ def load() -> ctypes.CDLL:
         lib.nb_cbs_poll_status.argtypes = [V, V]
         lib.nb_cbs_plan_set_dx_target.argtypes = [V, ctypes.c_int64, c_int32]
         lib.nb_cbs_plan_set_fwd_residual.argtypes = [V, V, ctypes.c_int64]
+        lib.nb_cbs_plan_set_bwd_residual.argtypes = [V, V, ctypes.c_int64, c_int32]
         lib.nb_conv_bn_silu_fwd.argtypes = [V, V, V, FP, FP, FP, FP, V, FP, FP, V, V, c_size_t, V]
         lib.nb_bn_stats.argtypes = [V, V, c_int32, FP, FP, FP, FP, V, c_size_t, V]
         lib.nb_conv_bn_silu_bwd_data.argtypes = [V, V, V, FP, FP, FP, FP, V, V, FP, FP, V, V, c_size_t, V]
@@ -190,6 +191,10 @@ class Plan:
     def set_fwd_residual(self, res=None, ld_res=0):
         """The forward call adds `res` (a tensor of the output's shape; row pitch ld_res elements, 0 = dense) to its output."""
         _check(load().nb_cbs_plan_set_fwd_residual(self.handle, _ptr(res), int(ld_res)))
+
+    def set_bwd_residual(self, gres=None, ld_gres=0, accumulate=True):
+        """The data-gradient call also adds (accumulate) or copies its incoming gradient g into `gres` (row pitch ld_gres, 0 = dense)."""
+        _check(load().nb_cbs_plan_set_bwd_residual(self.handle, _ptr(gres), int(ld_gres), 1 if accumulate else 0))
 
     def set_dx_target(self, ld_dx=0, accumulate=False):
         """dx of the data-gradient call is a channel slice with this row pitch (0 = dense) and is added to, not overwritten."""

@@ -583,10 +583,14 @@ __device__ __forceinline__ void bwd_coef_from_acc(const ChanAcc& ca, const BwdFi
     }
 }
 // FIN: the coefficients are derived here from the totals in `ca` (dynamic shared memory: 4*C floats); else read from coef.
-template <typename YT, typename AT, bool FAST, bool PITCHED = false, bool FIN = false>
+// GRES: the incoming gradient g is also the gradient of a residual connection's shortcut: the pass adds it to (or, with
+// gres_add = 0, copies it into) `gres`, a tensor of g's shape with pixels ld_gres elements apart -- the backward
+// counterpart of the RES form of the normalise + SiLU pass (fp32 sum, rounded once, like a separate accumulation pass).
+template <typename YT, typename AT, bool FAST, bool PITCHED = false, bool FIN = false, bool GRES = false>
 __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __restrict__ g, const YT* __restrict__ y,
                                                               AT* __restrict__ dy, long long total_vecs, int C,
-                                                              const float* __restrict__ coef, long long ld_g, ChanAcc ca, BwdFin fin) {
+                                                              const float* __restrict__ coef, long long ld_g, ChanAcc ca, BwdFin fin,
+                                                              AT* __restrict__ gres, long long ld_gres, int gres_add) {
     pdl_launch_dependents();
     pdl_wait();
     constexpr int V = Vec16<YT>::N;
@@ -616,13 +620,24 @@ __global__ void __launch_bounds__(288, 3) bn_silu_bwd_dy_kernel(const AT* __rest
     const long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     long long og = PITCHED ? (v0 / cgs) * ld_g + (long long)cg * V : v0 * V;  // g may be a channel slice (row pitch ld_g), see the reduce kernel
     const long long og_step = PITCHED ? (stride / cgs) * ld_g : stride * V;
-    for (long long v = v0; v < total_vecs; v += stride, og += og_step) {
+    long long ogr = GRES ? (v0 / cgs) * ld_gres + (long long)cg * V : 0;
+    const long long ogr_step = GRES ? (stride / cgs) * ld_gres : 0;
+    for (long long v = v0; v < total_vecs; v += stride, og += og_step, ogr += ogr_step) {
         if (v + 2 * stride < total_vecs) {  // L2 prefetch two iterations ahead (see the reduce kernel)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(y + (v + 2 * stride) * V));
             asm volatile("prefetch.global.L2 [%0];" ::"l"(g + og + 2 * og_step));
         }
         const Vec16<YT> qy = ld16(y + v * V);
         const Vec16<AT> qg = ld16(g + og);
+        if (GRES) {
+            Vec16<AT> r = qg;
+            if (gres_add) {
+                const Vec16<AT> old = ld16(gres + ogr);
+#pragma unroll
+                for (int j = 0; j < V / 2; ++j) pair_from_f32(r.v + 2 * j, add2(pair_to_f32(old.v + 2 * j), pair_to_f32(qg.v + 2 * j)));
+            }
+            st16(gres + ogr, r);
+        }
         Vec16<AT> o;
 #pragma unroll
         for (int j = 0; j < V / 2; ++j) {

@@ -76,6 +76,9 @@ struct nb_cbs_plan_s {
     long long ld_a = 0, ld_g = 0;  // row pitch (elements) of a_out in the forward call and of g in the backward call (set by nb_cbs_plan_set_pitches; default c_out)
     const void* fwd_res = nullptr;  // residual added to the forward call's output (nb_cbs_plan_set_fwd_residual) and its row pitch
     long long ld_res = 0;
+    void* bwd_gres = nullptr;       // tensor that the data-gradient call adds (or copies) its incoming gradient to (nb_cbs_plan_set_bwd_residual)
+    long long ld_gres = 0;
+    bool gres_add = true;
     long long ld_dx = 0;           // row pitch of dx in the data-gradient call and whether dx is added to (nb_cbs_plan_set_dx_target)
     bool dx_accumulate = false;
     bool pitched = false;
@@ -234,10 +237,13 @@ nb_status run_bwd_elementwise(nb_cbs_plan_s* p, const void* g, const void* y, co
     const BwdFin bf{1.0 / (double)p->g.m, mean, invstd, gamma, beta, dgamma, dbeta};
     auto go_dy = [&](auto kernel, size_t smem) {
         launch_k(kernel, dim3(e.blocks_dy), dim3(e.tpb), smem, st, 1, static_cast<const AT*>(g), static_cast<const YT*>(y), static_cast<AT*>(dy), e.total_vecs, C, coef,
-                 p->ld_g ? p->ld_g : (long long)C, ca, bf);
+                 p->ld_g ? p->ld_g : (long long)C, ca, bf, static_cast<AT*>(p->bwd_gres), p->ld_gres ? p->ld_gres : (long long)C, p->gres_add ? 1 : 0);
     };
     const size_t coef_smem = (size_t)4 * C * sizeof(float);
-    if (fuse) {
+    if (fuse && p->bwd_gres) {  // (the setter admits this only on plans that take this path)
+        if (p->ld_g) go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, true, true, true>, coef_smem);
+        else go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, false, true, true>, coef_smem);
+    } else if (fuse) {
         if (p->ld_g) go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, true, true>, coef_smem);
         else go_dy(bn_silu_bwd_dy_kernel<YT, AT, FAST, false, true>, coef_smem);
     } else {
@@ -513,6 +519,22 @@ nb_status nb_cbs_plan_set_fwd_residual(nb_cbs_plan p, const void* res, int64_t l
         return fail(NB_ERR_INVALID_ARG, "ld_res must be 0 (dense) or at least c_out and a multiple of %d elements", vec);
     p->fwd_res = res;
     p->ld_res = res ? ld_res : 0;
+    return NB_OK;
+}
+
+nb_status nb_cbs_plan_set_bwd_residual(nb_cbs_plan p, void* gres, int64_t ld_gres, int32_t accumulate) {
+    g_err.clear();
+    if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
+    NB_CHECK_PTR(gres, true);
+    if (accumulate != 0 && accumulate != 1) return fail(NB_ERR_INVALID_ARG, "accumulate must be 0 or 1, got %d", accumulate);
+    if (ld_gres == p->g.c_out) ld_gres = 0;
+    if (gres && ld_gres != 0 && (ld_gres < p->g.c_out || ld_gres % 8 != 0))
+        return fail(NB_ERR_INVALID_ARG, "ld_gres must be 0 (dense) or at least c_out and a multiple of 8 elements");
+    if (gres && !p->fuse_finalize)
+        return fail(NB_ERR_UNSUPPORTED, "the shortcut's gradient rides in the dy pass of the default 16-bit plans only (not fp32 mode, not NB_CBS_FLAG_SEPARATE_FINALIZE)");
+    p->bwd_gres = gres;
+    p->ld_gres = gres ? ld_gres : 0;
+    p->gres_add = accumulate != 0;
     return NB_OK;
 }
 
@@ -794,7 +816,7 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     NB_CHECK_PTR(x); NB_CHECK_PTR(dout); NB_CHECK_PTR(dw); NB_CHECK_PTR(dx, true); NB_CHECK_PTR(dbias, true);
     if (dx) NB_CHECK_PTR(w);
-    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: only the three training calls honour them");
+    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res || p->bwd_gres) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: only the three training calls honour them");
     NB_TRY(check_ws(workspace, workspace_bytes, p->bwd_bytes));
     {
         DeviceGuard on_device(p->device);
@@ -980,7 +1002,7 @@ nb_status nb_conv_bn_silu_step_host(nb_cbs_plan p, const void* host_x, const voi
     if (!p) return fail(NB_ERR_INVALID_ARG, "plan is NULL");
     if (!host_x || !host_w || !host_gamma || !host_beta || !host_g || !host_a || !host_dw || !host_dgamma || !host_dbeta)
         return fail(NB_ERR_INVALID_ARG, "a required host pointer is NULL");
-    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: the host-buffer step works on dense tensors");
+    if (p->pitched || p->ld_dx || p->dx_accumulate || p->fwd_res || p->bwd_gres) return fail(NB_ERR_UNSUPPORTED, "the plan has row pitches, a dx target or a residual set: the host-buffer step works on dense tensors");
     const StepLayout L = step_layout(p);
     NB_TRY(check_ws(device_scratch, scratch_bytes, L.total));
     DeviceGuard on_device(p->device);

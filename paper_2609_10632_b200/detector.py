@@ -28,7 +28,8 @@ _PITCH_IN = ("slice", "add", "concat")  # glue ops that read pitched operands (b
 
 
 class GraphRunner:
-    def __init__(self, ops, layers, outputs, eps=1e-3, device=0, plain_layers=None, views=True, direct_dx=True, fuse_residual=True):
+    def __init__(self, ops, layers, outputs, eps=1e-3, device=0, plain_layers=None, views=True, direct_dx=True, fuse_residual=True,
+                 fuse_shortcut_grad=True):
         """plain_layers: shapes of the plain convolutions (bias, no BN, no activation) that "plain" ops refer to; their
         parameters and gradients live in self.plain[k] (dict with plan, w, bias, dw, dbias, dx, ws).
         views=False: every tensor dense, split / concat by copies (the reference behaviour of the views).
@@ -36,7 +37,9 @@ class GraphRunner:
         input's gradient (the reference behaviour of nb_cbs_plan_set_dx_target).
         fuse_residual=False: every residual add is a glue launch of its own (the reference behaviour of
         nb_cbs_plan_set_fwd_residual, up to one rounding: the fused add rounds the sum once, the separate one rounds the
-        block's output first)."""
+        block's output first).
+        fuse_shortcut_grad=False: the shortcut's share of a fused residual add's gradient is a glue launch of its own (the
+        reference behaviour of nb_cbs_plan_set_bwd_residual)."""
         self.ops, self.layers, self.outputs = ops, layers, list(outputs)
         self.dev = torch.device("cuda", device)
         self.plain, self.idx = [], {}
@@ -251,6 +254,24 @@ class GraphRunner:
                     continue  # (stride-2 layers and layers off the tensor-core path keep the glue launch)
                 blk.dx = target
                 self.direct_dx.add(oi)
+        # ---- the shortcut's share of a fused residual add's gradient: the block that performs the add also hands its
+        # incoming gradient (the sum's gradient) to the shortcut's gradient buffer, inside its dy pass
+        self.shortcut_by_block = {}  # index of the add op -> the block that does its backward
+        if fuse_shortcut_grad:
+            for oi, o in enumerate(ops):
+                if o["op"] != "add" or id(o) not in self.fused_adds:
+                    continue
+                vi, vo = prod[o["ins"][1]]
+                if any(vi < i < oi for i, _, _ in cons[o["ins"][0]]):
+                    continue  # another contribution to the same gradient would change places with this one
+                blk = self.blocks[vo["layer"]]
+                gres = grad[o["ins"][0]]
+                try:
+                    blk.plan.set_bwd_residual(gres, gres.stride(-2), accumulate=self.acc[(oi, 0)])
+                except nb.NbError:
+                    continue
+                blk.gres = gres
+                self.shortcut_by_block[oi] = blk
 
     # ------------------------------------------------------------------ helpers
     def _implicit(self, o, pos):
@@ -349,7 +370,7 @@ class GraphRunner:
                     n_glue += 1
             elif kind == "add":
                 for pos, src in enumerate(ins):
-                    if not self._implicit(o, pos):
+                    if not self._implicit(o, pos) and not (pos == 0 and oi in self.shortcut_by_block):
                         self._sadd(G[src], G[out], self._rows(out), c_out, accumulate=self.acc[(oi, pos)], stream=stream)
                         n_glue += 1
             elif kind == "concat":

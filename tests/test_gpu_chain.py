@@ -541,3 +541,41 @@ def test_views_and_copies_give_the_same_bits():
     va, vb = sum(a.glue_launches()), sum(b.glue_launches())
     print("glue launches with views", a.glue_launches(), "with copies", b.glue_launches(), "placed", len(a.placed), "slice views", len(a.slice_view))
     assert va < 0.6 * vb
+
+
+def test_the_shortcut_gradient_inside_the_dy_pass_gives_the_same_bits():
+    """GraphRunner(fuse_shortcut_grad=True) lets the block that performs a residual add also hand the sum's gradient to the
+    shortcut (nb_cbs_plan_set_bwd_residual) instead of a glue launch per bottleneck: same additions in the same order, so
+    every gradient agrees bit for bit, with twelve launches fewer."""
+    import torch
+
+    from paper_2609_10632_b200.detector import GraphRunner
+
+    ops, layers, outs, plain = wl.detector_graph(2, 128, plain_head=True)
+    runs = [GraphRunner(ops, layers, outs, eps=EPS, plain_layers=plain, fuse_shortcut_grad=f) for f in (True, False)]
+    gen = torch.Generator(device=runs[0].dev)
+    gen.manual_seed(13)
+    img = torch.rand(runs[0].shape["img"], generator=gen, device=runs[0].dev).to(torch.bfloat16)
+    gout = {n: torch.randn(runs[0].shape[n], generator=gen, device=runs[0].dev).to(torch.bfloat16) for n in outs}
+    for r in runs:
+        r.fill_parameters(seed=210)
+        for j, pl in enumerate(r.plain):
+            g2 = torch.Generator(device=r.dev)
+            g2.manual_seed(310 + j)
+            pl["w"].copy_(torch.randn(pl["w"].shape, generator=g2, device=r.dev) * 0.05)
+            pl["bias"].copy_(torch.randn(pl["bias"].shape, generator=g2, device=r.dev) * 0.5)
+        r.buf["img"].copy_(img)
+        for n in outs:
+            r.grad[n].copy_(gout[n])
+        r.forward()
+        r.backward()
+    torch.cuda.synchronize()
+    a, b = runs
+    a.poll()
+    b.poll()
+    assert len(a.shortcut_by_block) == 12 and not b.shortcut_by_block
+    assert torch.equal(a.grad["img"], b.grad["img"])
+    for x, y in zip(a.blocks, b.blocks):
+        assert torch.equal(x.dw, y.dw) and torch.equal(x.dgamma, y.dgamma) and torch.equal(x.dbeta, y.dbeta), x.shape.name
+    assert sum(a.glue_launches()) == sum(b.glue_launches()) - 12
+

@@ -354,6 +354,47 @@ def test_forward_with_a_residual_adds_it_once(shape, mode):
     np.testing.assert_array_equal(blk.a.double().cpu().numpy(), plain["a"])
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[9], SMALL_SHAPES[5]], ids=lambda s: s.name)
+def test_backward_hands_the_gradient_to_the_shortcut(shape):
+    """nb_cbs_plan_set_bwd_residual: the data-gradient call also adds (or copies) its incoming gradient g into the
+    shortcut's gradient tensor (dense or a channel slice), inside its dy pass.  The sum is the fp32 sum of the two 16-bit
+    values rounded once -- checked exactly --, everything else the call writes is what the plain call writes, bit for
+    bit, and the plans that cannot do it say so."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    inp, blk, plain = _run_block(shape, 0, cfg_id=23, affine="random")
+    s, dev = shape, blk.dev
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    for ld, off, accumulate in ((0, 0, True), (s.c_out + 24, 16, True), (s.c_out + 8, 8, False)):
+        wide = torch.randn(s.n, s.ho, s.wo, ld or s.c_out, generator=gen, device=dev).to(torch.bfloat16)
+        before = wide.clone()
+        gres = wide[..., off:off + s.c_out]
+        blk.plan.set_bwd_residual(gres, gres.stride(-2), accumulate=accumulate)
+        blk.backward_data()
+        torch.cuda.synchronize()
+        blk.poll()
+        old = before[..., off:off + s.c_out]
+        want = (old.float() + blk.g.float()).to(torch.bfloat16) if accumulate else blk.g
+        assert torch.equal(gres, want)
+        untouched = torch.ones(wide.shape[-1], dtype=torch.bool, device=dev)
+        untouched[off:off + s.c_out] = False
+        assert torch.equal(wide[..., untouched], before[..., untouched])  # the channels beside the slice
+        for k in ("dx", "dy", "dgamma", "dbeta"):
+            np.testing.assert_array_equal(getattr(blk, k).double().cpu().numpy(), plain[k], err_msg=k)
+    blk.plan.set_bwd_residual(None)
+    blk.backward_data()
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(blk.dy.double().cpu().numpy(), plain["dy"])
+    fixed = CbsBlock(shape, eps=EPS, flags=nb.NB_CBS_FLAG_SEPARATE_FINALIZE)
+    with pytest.raises(nb.NbError) as e:
+        fixed.plan.set_bwd_residual(blk.g, 0)
+    assert e.value.status == nb.NB_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[9], SMALL_SHAPES[12], SMALL_SHAPES[13]], ids=lambda s: s.name)
 def test_channel_accumulators_are_clean_between_calls(shape):
     """The default plans sum the BatchNorm statistics with fp64 atomics into accumulators that the plan owns, and the last
