@@ -54,7 +54,7 @@ extern "C" {
 #endif
 
 #define NB_CBS_ABI_VERSION 3u /* 2: adds the evaluation-mode / plain calls (additive); 3: flag 2 is NB_CBS_FLAG_SEPARATE_FINALIZE,
-                                  the grid-barrier test hook is gone with the barriers */
+                                  the grid-barrier test hook is gone with the barriers, nb_cbs_plan_set_bwd_residual is new */
 
 typedef int32_t nb_status;
 enum {
