@@ -43,9 +43,11 @@ nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_
 
 /* Nearest-neighbour 2x upsampling of [n][h][w][c] (the extents of the SMALL tensor):
  *   backward == 0: dst[n][2i+a][2j+b][c] = src[n][i][j][c]                       (src small, dst large)
- *   backward != 0: dst[n][i][j][c] = [dst +] sum_{a,b} src[n][2i+a][2j+b][c]      (src large, dst small) */
+ *   backward != 0: dst[n][i][j][c] = [dst +] sum_{a,b} src[n][2i+a][2j+b][c]      (src large, dst small)
+ * ld_small / ld_large: elements between consecutive pixels of the small / the large tensor (0 = dense, else >= c): either
+ * may be a channel slice of a wider tensor, e.g. the large one a part of the concatenation buffer it feeds. */
 nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* src, void* dst,
-                       int32_t backward, int32_t accumulate, void* stream);
+                       int32_t backward, int32_t accumulate, int64_t ld_small, int64_t ld_large, void* stream);
 
 #ifdef __cplusplus
 }

@@ -107,7 +107,7 @@ def load() -> ctypes.CDLL:
         lib.nb_slice_add.argtypes = [c_int32, ctypes.c_int64, c_int32, V, ctypes.c_int64, V, ctypes.c_int64, V, ctypes.c_int64, c_int32, V]
         lib.nb_maxpool5_fwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, V]
         lib.nb_maxpool5_bwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, c_int32, V]
-        lib.nb_upsample2.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, c_int32, c_int32, V]
+        lib.nb_upsample2.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, c_int32, c_int32, ctypes.c_int64, ctypes.c_int64, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
         lib.nb_cbs_profile_enable.argtypes = [V, c_int32]
@@ -322,9 +322,10 @@ def nb_maxpool5_bwd(dtype, n, h, w, c, g, idx, dx, accumulate=False, stream=None
     _check(load().nb_maxpool5_bwd(int(dtype), n, h, w, c, _ptr(g), _ptr(idx), _ptr(dx), 1 if accumulate else 0, _stream(stream)))
 
 
-def nb_upsample2(dtype, n, h, w, c, src, dst, backward=False, accumulate=False, stream=None):
-    """(n, h, w, c) are the extents of the SMALL tensor."""
-    _check(load().nb_upsample2(int(dtype), n, h, w, c, _ptr(src), _ptr(dst), 1 if backward else 0, 1 if accumulate else 0, _stream(stream)))
+def nb_upsample2(dtype, n, h, w, c, src, dst, backward=False, accumulate=False, ld_small=0, ld_large=0, stream=None):
+    """2x nearest-neighbour upsampling (or its gradient); n, h, w, c and ld_small describe the SMALL tensor, ld_large the large one (pixel pitches, 0 = dense)."""
+    _check(load().nb_upsample2(int(dtype), n, h, w, c, _ptr(src), _ptr(dst), 1 if backward else 0, 1 if accumulate else 0, int(ld_small), int(ld_large),
+                               _stream(stream)))
 
 
 class SgdPlan:

@@ -167,12 +167,13 @@ __global__ void __launch_bounds__(256) maxpool5_bwd_kernel(const T* __restrict__
 // dx[n][h][w][c] = sum of the four g (BWD = true; fp32 sum, one rounding; accumulate adds to dx).  x / dx is [N][H][W][C];
 // one thread per V channels of a small-tensor pixel (V = 8: 16-byte accesses, or 1).
 template <typename T, bool BWD, int V>
-__global__ void __launch_bounds__(256) upsample2_kernel(const T* __restrict__ src, T* __restrict__ dst, int N, int H, int W, int C, int accumulate) {
+__global__ void __launch_bounds__(256) upsample2_kernel(const T* __restrict__ src, T* __restrict__ dst, int N, int H, int W, int C, int accumulate,
+                                                        long long ld_s /* pixel pitch of the small tensor */, long long ld_l /* of the large one */) {
     pdl_launch_dependents();
     pdl_wait();
     const unsigned cv = (unsigned)(C / V);
     const long long total = (long long)N * H * W * cv;
-    const long long row2 = 2LL * W * C;
+    const long long row2 = 2LL * W * ld_l, nx = ld_l;  // one row down / one pixel to the right in the large tensor
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const unsigned pix = (unsigned)(i / cv);
         const int c = (int)((unsigned)(i - (long long)pix * cv)) * V;
@@ -180,11 +181,11 @@ __global__ void __launch_bounds__(256) upsample2_kernel(const T* __restrict__ sr
         const int w = (int)(pix - t1 * (unsigned)W);
         const unsigned n = t1 / (unsigned)H;
         const int h = (int)(t1 - n * (unsigned)H);
-        const long long os = (long long)pix * C + c;                                              // in the small tensor
-        const long long o = (((long long)n * 2 * H + 2 * h) * 2 * W + 2 * w) * (long long)C + c;  // (2h, 2w) in the large tensor
+        const long long os = (long long)pix * ld_s + c;                                   // in the small tensor
+        const long long o = (((long long)n * 2 * H + 2 * h) * 2 * W + 2 * w) * ld_l + c;  // (2h, 2w) in the large tensor
         if (V == 8) {
             if (BWD) {
-                const Vec16<T> a0 = ld16(src + o), a1 = ld16(src + o + C), a2 = ld16(src + o + row2), a3 = ld16(src + o + row2 + C);
+                const Vec16<T> a0 = ld16(src + o), a1 = ld16(src + o + nx), a2 = ld16(src + o + row2), a3 = ld16(src + o + row2 + nx);
                 Vec16<T> old, res;
                 if (accumulate) old = ld16(dst + os);
 #pragma unroll
@@ -197,20 +198,20 @@ __global__ void __launch_bounds__(256) upsample2_kernel(const T* __restrict__ sr
             } else {
                 const Vec16<T> v = ld16(src + os);
                 st16(dst + o, v);
-                st16(dst + o + C, v);
+                st16(dst + o + nx, v);
                 st16(dst + o + row2, v);
-                st16(dst + o + row2 + C, v);
+                st16(dst + o + row2 + nx, v);
             }
         } else if (BWD) {
-            float sum = (to_f32(src[o]) + to_f32(src[o + C])) + (to_f32(src[o + row2]) + to_f32(src[o + row2 + C]));
+            float sum = (to_f32(src[o]) + to_f32(src[o + nx])) + (to_f32(src[o + row2]) + to_f32(src[o + row2 + nx]));
             if (accumulate) sum += to_f32(dst[os]);
             dst[os] = from_f32<T>(sum);
         } else {
             const T v = src[os];
             dst[o] = v;
-            dst[o + C] = v;
+            dst[o + nx] = v;
             dst[o + row2] = v;
-            dst[o + row2 + C] = v;
+            dst[o + row2 + nx] = v;
         }
     }
 }

@@ -122,15 +122,18 @@ nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_
 }
 
 nb_status nb_upsample2(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* src, void* dst, int32_t backward, int32_t accumulate,
-                       void* stream) {
+                       int64_t ld_small, int64_t ld_large, void* stream) {
     g_err.clear();
     if (!src || !dst) return fail(NB_ERR_INVALID_ARG, "src and dst must not be NULL");
     NB_TRY(check_nhwc(n, h, w, c));
+    if (ld_small == 0) ld_small = c;
+    if (ld_large == 0) ld_large = c;
+    if (ld_small < c || ld_large < c) return fail(NB_ERR_INVALID_ARG, "a pixel pitch must be 0 (dense) or at least c");
     if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u);
+    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 && ld_small % 8 == 0 && ld_large % 8 == 0 && !((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u);
     const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
-#define NB_UPS1(T, BW, VV) launch_k(upsample2_kernel<T, BW, VV>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0)
+#define NB_UPS1(T, BW, VV) launch_k(upsample2_kernel<T, BW, VV>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(src), static_cast<T*>(dst), n, h, w, c, accumulate != 0, (long long)ld_small, (long long)ld_large)
 #define NB_UPS(T)                                   \
     do {                                            \
         if (backward && vec) NB_UPS1(T, true, 8);   \

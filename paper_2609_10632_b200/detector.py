@@ -24,7 +24,7 @@ import torch
 from . import binding as nb
 from .block import CbsBlock
 
-_PITCH_IN = ("slice", "add", "concat")  # glue ops that read pitched operands (blocks do when their plan says so)
+_PITCH_IN = ("slice", "add", "concat", "upsample")  # glue ops that read pitched operands (blocks do when their plan says so)
 
 
 class GraphRunner:
@@ -110,7 +110,7 @@ class GraphRunner:
                 while k < len(ins):
                     t = ins[k]
                     _, po = prod.get(t, (None, {"op": "input"}))
-                    if po["op"] in ("cbs", "add") and t not in placed and t not in self.outputs and others_ok(t, o):
+                    if po["op"] in ("cbs", "add", "upsample") and t not in placed and t not in self.outputs and others_ok(t, o):
                         placed[t] = (o["out"], off)
                     elif po["op"] == "slice" and t in slice_view and po["c0"] == 0:
                         src = po["ins"][0]  # consecutive slices of one tensor that together are that tensor: place the tensor
@@ -330,7 +330,7 @@ class GraphRunner:
                 n_glue += 1
             elif kind == "upsample":
                 n, h, w, c = self.shape[ins[0]]
-                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], stream=stream)
+                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], ld_small=B[ins[0]].stride(-2), ld_large=B[out].stride(-2), stream=stream)
                 n_glue += 1
         self.glue_fwd = n_glue
 
@@ -387,7 +387,8 @@ class GraphRunner:
                 n_glue += 1
             elif kind == "upsample":
                 n, h, w, c = self.shape[ins[0]]
-                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, G[out], G[ins[0]], backward=True, accumulate=self.acc[(oi, 0)], stream=stream)
+                nb.nb_upsample2(nb.NB_DTYPE_BF16, n, h, w, c, G[out], G[ins[0]], backward=True, accumulate=self.acc[(oi, 0)], ld_small=G[ins[0]].stride(-2),
+                                ld_large=G[out].stride(-2), stream=stream)
                 n_glue += 1
         self.glue_bwd = n_glue
 

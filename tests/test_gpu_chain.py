@@ -163,6 +163,18 @@ def test_upsample2_forward_and_adjoint(dtype_name):
         assert torch.equal(dx, torch.from_numpy(ref).to(dt).to(dev))
     else:
         np.testing.assert_allclose(dx.double().cpu().numpy(), ref, rtol=1e-6, atol=2e-6)  # three fp32 additions with cancellation
+    # channel slices of wider tensors on both sides (pixel pitches): the same values, nothing beside the slices touched
+    ws = torch.full((n, h, w, c + 8), 7.0, dtype=dt, device=dev)
+    wl_ = torch.full((n, 2 * h, 2 * w, c + 16), 9.0, dtype=dt, device=dev)
+    xs, yl = ws[..., 4:4 + c], wl_[..., 8:8 + c]
+    xs.copy_(x)
+    nb.nb_upsample2(code, n, h, w, c, xs, yl, ld_small=xs.stride(-2), ld_large=yl.stride(-2))
+    torch.cuda.synchronize()
+    assert torch.equal(yl, y) and bool((wl_[..., :8] == 9).all()) and bool((wl_[..., 8 + c:] == 9).all())
+    yl.copy_(g)
+    nb.nb_upsample2(code, n, h, w, c, yl, xs, backward=True, ld_small=xs.stride(-2), ld_large=yl.stride(-2))
+    torch.cuda.synchronize()
+    assert torch.equal(xs, dx) and bool((ws[..., :4] == 7).all()) and bool((ws[..., 4 + c:] == 7).all())
 
 
 def test_sppf_unit_matches_chained_oracle():
