@@ -32,14 +32,17 @@ nb_status nb_slice_add(int32_t dtype /* nb_dtype */, int64_t rows, int32_t chann
 /* 5x5 max-pool, stride 1, padding 2 over x [n][h][w][c] (the detector's SPPF unit chains three of them); padding never
  * wins.  idx (may be NULL; one byte per element, same shape) receives r*5 + t of the FIRST maximum of each window in
  * row-major order (r, t = 0..4 from the window's corner at (p-2, q-2)): the record the backward call needs.
- * 16-byte accesses for 16-bit types when c % 8 == 0 and x, y are 16-byte aligned. */
+ * ld_x / ld_y: elements between consecutive pixels of x / y (0 = dense, else >= c): either may be a channel slice of a
+ * wider tensor (the SPPF concatenation buffer holds the pools side by side); idx is always dense.
+ * 16-byte accesses for 16-bit types when c and the pitches are multiples of 8 and x, y are 16-byte aligned. */
 nb_status nb_maxpool5_fwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* x, void* y, uint8_t* idx,
-                          void* stream);
+                          int64_t ld_x, int64_t ld_y, void* stream);
 
 /* Gradient of nb_maxpool5_fwd: dx[n][i][j][c] = [dx +] sum of g over the windows whose recorded maximum is (i, j)
- * (fp32 sum in a fixed order, one rounding; accumulate != 0 adds to dx for tensors with several consumers). */
+ * (fp32 sum in a fixed order, one rounding; accumulate != 0 adds to dx for tensors with several consumers).
+ * ld_g / ld_dx: pixel pitches of g and dx as above. */
 nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* g, const uint8_t* idx,
-                          void* dx, int32_t accumulate, void* stream);
+                          void* dx, int32_t accumulate, int64_t ld_g, int64_t ld_dx, void* stream);
 
 /* Nearest-neighbour 2x upsampling of [n][h][w][c] (the extents of the SMALL tensor):
  *   backward == 0: dst[n][2i+a][2j+b][c] = src[n][i][j][c]                       (src small, dst large)

@@ -105,8 +105,8 @@ def load() -> ctypes.CDLL:
         lib.nb_sgd_clip_nesterov_step.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), FP, V]
         lib.nb_sgd_clip_nesterov_step_scaled.argtypes = [V, V, c_size_t, POINTER(nb_sgd_hyper), POINTER(nb_scaler_hyper), V, FP, V]
         lib.nb_slice_add.argtypes = [c_int32, ctypes.c_int64, c_int32, V, ctypes.c_int64, V, ctypes.c_int64, V, ctypes.c_int64, c_int32, V]
-        lib.nb_maxpool5_fwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, V]
-        lib.nb_maxpool5_bwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, c_int32, V]
+        lib.nb_maxpool5_fwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, ctypes.c_int64, ctypes.c_int64, V]
+        lib.nb_maxpool5_bwd.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, V, c_int32, ctypes.c_int64, ctypes.c_int64, V]
         lib.nb_upsample2.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, V, V, c_int32, c_int32, ctypes.c_int64, ctypes.c_int64, V]
         lib.nb_cbs_launch_count.argtypes = []
         lib.nb_cbs_launch_count.restype = ctypes.c_ulonglong
@@ -314,12 +314,12 @@ def nb_slice_add(dtype, rows, channels, out, ld_out, a, ld_a, b=None, ld_b=0, ac
                                1 if accumulate else 0, _stream(stream)))
 
 
-def nb_maxpool5_fwd(dtype, n, h, w, c, x, y, idx=None, stream=None):
-    _check(load().nb_maxpool5_fwd(int(dtype), n, h, w, c, _ptr(x), _ptr(y), _ptr(idx), _stream(stream)))
+def nb_maxpool5_fwd(dtype, n, h, w, c, x, y, idx=None, stream=None, ld_x=0, ld_y=0):
+    _check(load().nb_maxpool5_fwd(int(dtype), n, h, w, c, _ptr(x), _ptr(y), _ptr(idx), int(ld_x), int(ld_y), _stream(stream)))
 
 
-def nb_maxpool5_bwd(dtype, n, h, w, c, g, idx, dx, accumulate=False, stream=None):
-    _check(load().nb_maxpool5_bwd(int(dtype), n, h, w, c, _ptr(g), _ptr(idx), _ptr(dx), 1 if accumulate else 0, _stream(stream)))
+def nb_maxpool5_bwd(dtype, n, h, w, c, g, idx, dx, accumulate=False, stream=None, ld_g=0, ld_dx=0):
+    _check(load().nb_maxpool5_bwd(int(dtype), n, h, w, c, _ptr(g), _ptr(idx), _ptr(dx), 1 if accumulate else 0, int(ld_g), int(ld_dx), _stream(stream)))
 
 
 def nb_upsample2(dtype, n, h, w, c, src, dst, backward=False, accumulate=False, ld_small=0, ld_large=0, stream=None):

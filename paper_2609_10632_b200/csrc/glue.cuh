@@ -53,7 +53,8 @@ namespace nbcbs {
 // vector of an output pixel, or per element when C % 8 != 0.  idx (optional, one byte per element) = r*5 + t of the FIRST
 // maximum of the window in row-major order: comparisons are strict, elements outside the image never win.
 template <typename T, int V>
-__global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, uint8_t* __restrict__ idx, int N, int H, int W, int C) {
+__global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, uint8_t* __restrict__ idx, int N, int H, int W, int C,
+                                                           long long ld_x, long long ld_y /* pixel pitches of x and y; idx is dense */) {
     pdl_launch_dependents();
     pdl_wait();
     const int cv = C / V;
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__
             for (int t = 0; t < 5; ++t) {
                 const int w = q - 2 + t;
                 if (w < 0 || w >= W) continue;
-                const T* src = x + (((n * H + h) * W + w) * (long long)C + c);
+                const T* src = x + (((n * H + h) * W + w) * ld_x + c);
                 T v[V];
                 if (V == 8) *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(src); else v[0] = src[0];
 #pragma unroll
@@ -91,10 +92,11 @@ __global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__
                 }
             }
         }
-        const long long o = ((n * H + p) * W + q) * (long long)C + c;
+        const long long pixo = (n * H + p) * W + q;
+        const long long o = pixo * (long long)C + c, oy = pixo * ld_y + c;
 #pragma unroll
         for (int k = 0; k < V; ++k) {
-            y[o + k] = from_f32<T>(best[k]);  // the maximum of stored values is itself a stored value: exact
+            y[oy + k] = from_f32<T>(best[k]);  // the maximum of stored values is itself a stored value: exact
             if (idx) idx[o + k] = (uint8_t)bi[k];
         }
     }
@@ -105,7 +107,7 @@ __global__ void __launch_bounds__(256) maxpool5_fwd_kernel(const T* __restrict__
 // V channels of an input pixel (V = 8 with 16-byte loads of g and 8-byte loads of the recorded positions, or 1).
 template <typename T, int V>
 __global__ void __launch_bounds__(256) maxpool5_bwd_kernel(const T* __restrict__ g, const uint8_t* __restrict__ idx, T* __restrict__ dx, int N, int H, int W,
-                                                           int C, int accumulate) {
+                                                           int C, int accumulate, long long ld_g, long long ld_dx /* pixel pitches of g and dx; idx is dense */) {
     pdl_launch_dependents();
     pdl_wait();
     const unsigned cv = (unsigned)(C / V);
@@ -126,7 +128,8 @@ __global__ void __launch_bounds__(256) maxpool5_bwd_kernel(const T* __restrict__
             for (int t = 4; t >= 0; --t) {
                 const int q = w + 2 - t;
                 if (q < 0 || q >= W) continue;
-                const long long o = (((long long)n * H + p) * W + q) * (long long)C + c;
+                const long long pixo = ((long long)n * H + p) * W + q;
+                const long long o = pixo * (long long)C + c, og = pixo * ld_g + c;
                 const int code = r * 5 + t;
                 if (V == 8) {
                     const uint2 ib = *reinterpret_cast<const uint2*>(idx + o);
@@ -134,18 +137,18 @@ __global__ void __launch_bounds__(256) maxpool5_bwd_kernel(const T* __restrict__
                     if (((ib.x ^ pat) & 0xffu) && ((ib.x ^ pat) & 0xff00u) && ((ib.x ^ pat) & 0xff0000u) && ((ib.x ^ pat) & 0xff000000u) &&
                         ((ib.y ^ pat) & 0xffu) && ((ib.y ^ pat) & 0xff00u) && ((ib.y ^ pat) & 0xff0000u) && ((ib.y ^ pat) & 0xff000000u))
                         continue;  // none of the eight channels of this window points here
-                    const Vec16<T> gv = ld16(g + o);
+                    const Vec16<T> gv = ld16(g + og);
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         const uint32_t byte = ((k < 4 ? ib.x : ib.y) >> (8 * (k & 3))) & 0xffu;
                         if (byte == (uint32_t)code) s[k] += to_f32(gv.v[k]);
                     }
                 } else if (idx[o] == code) {
-                    s[0] += to_f32(g[o]);
+                    s[0] += to_f32(g[og]);
                 }
             }
         }
-        const long long oi = (long long)pix * C + c;
+        const long long oi = (long long)pix * ld_dx + c;
         if (V == 8) {
             Vec16<T> res;
             if (accumulate) {

@@ -68,14 +68,14 @@ nb_status check_nhwc(int32_t n, int32_t h, int32_t w, int32_t c) {
     return NB_OK;
 }
 template <typename T>
-nb_status run_maxpool_fwd(const void* x, void* y, uint8_t* idx, int n, int h, int w, int c, cudaStream_t st) {
-    const bool vec = sizeof(T) == 2 && c % 8 == 0 && !((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u);
+nb_status run_maxpool_fwd(const void* x, void* y, uint8_t* idx, int n, int h, int w, int c, long long ld_x, long long ld_y, cudaStream_t st) {
+    const bool vec = sizeof(T) == 2 && c % 8 == 0 && ld_x % 8 == 0 && ld_y % 8 == 0 && !((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u);
     if (vec) {
         const long long total = (long long)n * h * w * (c / 8);
-        launch_k(maxpool5_fwd_kernel<T, 8>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
+        launch_k(maxpool5_fwd_kernel<T, 8>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c, ld_x, ld_y);
     } else {
         const long long total = (long long)n * h * w * c;
-        launch_k(maxpool5_fwd_kernel<T, 1>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c);
+        launch_k(maxpool5_fwd_kernel<T, 1>, dim3(glue_blocks(total)), dim3(256), 0, st, 1, static_cast<const T*>(x), static_cast<T*>(y), idx, n, h, w, c, ld_x, ld_y);
     }
     return launch_ok("maxpool5_fwd");
 }
@@ -83,33 +83,40 @@ nb_status run_maxpool_fwd(const void* x, void* y, uint8_t* idx, int n, int h, in
 
 extern "C" {
 
-nb_status nb_maxpool5_fwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* x, void* y, uint8_t* idx, void* stream) {
+nb_status nb_maxpool5_fwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* x, void* y, uint8_t* idx, int64_t ld_x, int64_t ld_y,
+                          void* stream) {
     g_err.clear();
     if (!x || !y) return fail(NB_ERR_INVALID_ARG, "x and y must not be NULL");
     NB_TRY(check_nhwc(n, h, w, c));
+    if (ld_x == 0) ld_x = c;
+    if (ld_y == 0) ld_y = c;
+    if (ld_x < c || ld_y < c) return fail(NB_ERR_INVALID_ARG, "a pixel pitch must be 0 (dense) or at least c");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (dtype) {
-        case NB_DTYPE_F32: return run_maxpool_fwd<float>(x, y, idx, n, h, w, c, st);
-        case NB_DTYPE_BF16: return run_maxpool_fwd<__nv_bfloat16>(x, y, idx, n, h, w, c, st);
-        case NB_DTYPE_F16: return run_maxpool_fwd<__half>(x, y, idx, n, h, w, c, st);
+        case NB_DTYPE_F32: return run_maxpool_fwd<float>(x, y, idx, n, h, w, c, (long long)ld_x, (long long)ld_y, st);
+        case NB_DTYPE_BF16: return run_maxpool_fwd<__nv_bfloat16>(x, y, idx, n, h, w, c, (long long)ld_x, (long long)ld_y, st);
+        case NB_DTYPE_F16: return run_maxpool_fwd<__half>(x, y, idx, n, h, w, c, (long long)ld_x, (long long)ld_y, st);
         default: return fail(NB_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     }
 }
 
 nb_status nb_maxpool5_bwd(int32_t dtype, int32_t n, int32_t h, int32_t w, int32_t c, const void* g, const uint8_t* idx, void* dx, int32_t accumulate,
-                          void* stream) {
+                          int64_t ld_g, int64_t ld_dx, void* stream) {
     g_err.clear();
     if (!g || !idx || !dx) return fail(NB_ERR_INVALID_ARG, "g, idx and dx must not be NULL");
     NB_TRY(check_nhwc(n, h, w, c));
+    if (ld_g == 0) ld_g = c;
+    if (ld_dx == 0) ld_dx = c;
+    if (ld_g < c || ld_dx < c) return fail(NB_ERR_INVALID_ARG, "a pixel pitch must be 0 (dense) or at least c");
     if ((long long)n * h * w >= (1LL << 32)) return fail(NB_ERR_UNSUPPORTED, "more than 2^32 pixels");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 &&
+    const bool vec = dtype != NB_DTYPE_F32 && c % 8 == 0 && ld_g % 8 == 0 && ld_dx % 8 == 0 &&
                      !((reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(dx)) & 15u) && !(reinterpret_cast<uintptr_t>(idx) & 7u);
     const unsigned blocks = glue_blocks((long long)n * h * w * (vec ? c / 8 : c));
 #define NB_POOLB(T)                                                                                                                               \
     do {                                                                                                                                          \
-        if (vec) launch_k(maxpool5_bwd_kernel<T, 8>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0); \
-        else launch_k(maxpool5_bwd_kernel<T, 1>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0);     \
+        if (vec) launch_k(maxpool5_bwd_kernel<T, 8>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0, (long long)ld_g, (long long)ld_dx); \
+        else launch_k(maxpool5_bwd_kernel<T, 1>, dim3(blocks), dim3(256), 0, st, 1, static_cast<const T*>(g), idx, static_cast<T*>(dx), n, h, w, c, accumulate != 0, (long long)ld_g, (long long)ld_dx);     \
     } while (0)
     switch (dtype) {
         case NB_DTYPE_F32: NB_POOLB(float); break;

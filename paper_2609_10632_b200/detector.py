@@ -24,7 +24,7 @@ import torch
 from . import binding as nb
 from .block import CbsBlock
 
-_PITCH_IN = ("slice", "add", "concat", "upsample")  # glue ops that read pitched operands (blocks do when their plan says so)
+_PITCH_IN = ("slice", "add", "concat", "upsample", "maxpool")  # glue ops that read pitched operands (blocks do when their plan says so)
 
 
 class GraphRunner:
@@ -110,7 +110,7 @@ class GraphRunner:
                 while k < len(ins):
                     t = ins[k]
                     _, po = prod.get(t, (None, {"op": "input"}))
-                    if po["op"] in ("cbs", "add", "upsample") and t not in placed and t not in self.outputs and others_ok(t, o):
+                    if po["op"] in ("cbs", "add", "upsample", "maxpool") and t not in placed and t not in self.outputs and others_ok(t, o):
                         placed[t] = (o["out"], off)
                     elif po["op"] == "slice" and t in slice_view and po["c0"] == 0:
                         src = po["ins"][0]  # consecutive slices of one tensor that together are that tensor: place the tensor
@@ -326,7 +326,7 @@ class GraphRunner:
                     c0 += c
             elif kind == "maxpool":
                 n, h, w, c = self.shape[out]
-                nb.nb_maxpool5_fwd(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], self.idx[out], stream)
+                nb.nb_maxpool5_fwd(nb.NB_DTYPE_BF16, n, h, w, c, B[ins[0]], B[out], self.idx[out], stream, ld_x=B[ins[0]].stride(-2), ld_y=B[out].stride(-2))
                 n_glue += 1
             elif kind == "upsample":
                 n, h, w, c = self.shape[ins[0]]
@@ -383,7 +383,8 @@ class GraphRunner:
                     c0 += c
             elif kind == "maxpool":
                 n, h, w, c = self.shape[out]
-                nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, G[out], self.idx[out], G[ins[0]], self.acc[(oi, 0)], stream)
+                nb.nb_maxpool5_bwd(nb.NB_DTYPE_BF16, n, h, w, c, G[out], self.idx[out], G[ins[0]], self.acc[(oi, 0)], stream, ld_g=G[out].stride(-2),
+                                   ld_dx=G[ins[0]].stride(-2))
                 n_glue += 1
             elif kind == "upsample":
                 n, h, w, c = self.shape[ins[0]]

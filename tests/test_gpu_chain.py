@@ -134,10 +134,24 @@ def test_maxpool5_forward_backward(dtype_name, n, h, w, c):
     # 16-bit terms add exactly in fp32, so those results are one rounding away from the exact sum
     atol = 25 * ulp * float(np.abs(g.double().numpy()).max()) * 5 if dtype_name == "float32" else ulp * 1e-3
     np.testing.assert_allclose(dx.double().cpu().numpy(), ref_dx, rtol=ulp, atol=atol)
+    dx1 = dx.clone()
     # accumulate: dx += the same gradient again
     nb.nb_maxpool5_bwd(code, n, h, w, c, gd, idx, dx, accumulate=True)
     torch.cuda.synchronize()
     np.testing.assert_allclose(dx.double().cpu().numpy(), 2 * ref_dx, rtol=4 * ulp, atol=2 * atol)
+    # every tensor a channel slice of a wider one (pixel pitches): the same bits, nothing beside the slices touched
+    pad = 8 if c % 8 == 0 else 3
+    wx, wy = torch.full((n, h, w, c + pad), 3.0, dtype=dt, device=dev), torch.full((n, h, w, c + 2 * pad), 5.0, dtype=dt, device=dev)
+    xs, ys = wx[..., pad:], wy[..., pad:pad + c]
+    xs.copy_(xd)
+    idx2 = torch.empty_like(idx)
+    nb.nb_maxpool5_fwd(code, n, h, w, c, xs, ys, idx2, ld_x=xs.stride(-2), ld_y=ys.stride(-2))
+    torch.cuda.synchronize()
+    assert torch.equal(ys, y) and torch.equal(idx2, idx) and bool((wy[..., :pad] == 5).all()) and bool((wy[..., pad + c:] == 5).all())
+    ys.copy_(gd)
+    nb.nb_maxpool5_bwd(code, n, h, w, c, ys, idx, xs, ld_g=ys.stride(-2), ld_dx=xs.stride(-2))
+    torch.cuda.synchronize()
+    assert torch.equal(xs, dx1) and bool((wx[..., :pad] == 3).all())
 
 
 @pytest.mark.parametrize("dtype_name", ["bfloat16", "float32"])
