@@ -632,10 +632,13 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
     } else if (p->stem) {
         // the first layer's kernel sums the statistics of the values it stores itself (one partial slice per block)
         SiteTimer tm(p, SITE_FPROP, st);
+        const bool fuse = p->fuse_finalize;  // sums into the plan's accumulators; the normalise + SiLU pass finalizes
         NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
-                               static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}, part));
+                               static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}, fuse ? static_cast<float*>(nullptr) : part,
+                               fuse ? p->acc : static_cast<double*>(nullptr), fuse ? p->acc_copies_f : 1));
         NB_LAUNCH_OK("stem_fprop");
         nparts = p->stem_blocks;
+        finalized = fuse;
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
         const long long l0 = p->tc.launches;
@@ -676,7 +679,8 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
     if (!is_f32(p) && p->stem) {  // the first layer's own kernel applies the coefficients and the activation itself
         SiteTimer tm(p, SITE_INFER, st);
         NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(w),
-                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}, static_cast<float*>(nullptr)));
+                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}, static_cast<float*>(nullptr),
+                               static_cast<double*>(nullptr), 1));
         return launch_ok("stem_fprop (fused epilogue)");
     }
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);

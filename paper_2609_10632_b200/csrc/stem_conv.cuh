@@ -116,12 +116,13 @@ struct StemEpi {
 // values of one filter row of a pixel are contiguous there).  The 16 x COUT output tile is one contiguous run: staged and
 // written with 16-byte stores.
 // EPI = false: y = the convolution output in fp16 (training forward), and with `partials` != NULL the block also writes the
-// per-channel sum and sum of squares of the ROUNDED values it stored to partials[blockIdx.x][2][COUT] (batch statistics
+// per-channel sum and sum of squares of the ROUNDED values it stored to partials[blockIdx.x][2][COUT], or with `acc` != NULL
+// adds them to accumulator set blockIdx.x mod acc_copies of [acc_copies][2][COUT] doubles (batch statistics
 // without a second pass over y; fixed order, bitwise reproducible).  EPI = true: OutT = activations, see StemEpi.
 // InT = the 16-bit type of x and w (bf16, or IEEE fp16).
 template <int COUT, typename OutT = __half, bool EPI = false, typename InT = __nv_bfloat16>
 __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __restrict__ x, const InT* __restrict__ w, OutT* __restrict__ y, Geom g,
-                                                                StemEpi ep, float* __restrict__ partials) {
+                                                                StemEpi ep, float* __restrict__ partials, double* __restrict__ acc, int acc_copies) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 8 == 0, "whole n-blocks");
@@ -263,7 +264,7 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
             __syncwarp();
         }
     }
-    if (!EPI && partials) {
+    if (!EPI && (partials || acc)) {
         // lanes with the same tq hold the same columns for different rows: add over gq (fixed butterfly), then over the warps
         __shared__ float wsum[4][2][COUT];
         __syncthreads();
@@ -285,7 +286,9 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
         __syncthreads();
         for (int e = threadIdx.x; e < 2 * COUT; e += blockDim.x) {
             const int which = e / COUT, c = e - which * COUT;
-            partials[(size_t)blockIdx.x * 2 * COUT + e] = ((wsum[0][which][c] + wsum[1][which][c]) + wsum[2][which][c]) + wsum[3][which][c];
+            const float v = ((wsum[0][which][c] + wsum[1][which][c]) + wsum[2][which][c]) + wsum[3][which][c];
+            if (acc) atomicAdd(acc + ((size_t)((int)blockIdx.x % acc_copies) * 2 + which) * COUT + c, (double)v);  // the plan's fp64 accumulators (see ChanAcc)
+            else partials[(size_t)blockIdx.x * 2 * COUT + e] = v;
         }
     }
 }
