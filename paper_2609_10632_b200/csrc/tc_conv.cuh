@@ -177,7 +177,7 @@ template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, fl
 template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b, int* sat) {
     uint32_t v;
     asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(v) : "f"(b), "f"(a));
-    *sat |= (int)((v & 0x7fff7fffu) + 0x04010401u);
+    if (sat) *sat |= (int)((v & 0x7fff7fffu) + 0x04010401u);  // (sat is a compile-time NULL where the caller tracks saturation otherwise)
     return v;
 }
 
@@ -224,13 +224,15 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
     }
     uint8_t* const my_row = wrows + lane * PITCH;
     int sat_bits = 0;
+    // (With STATS a saturated value is recognised below from the sums of squares, which costs nothing per element.)
+    int* const sat_track = STATS ? nullptr : &sat_bits;
 #pragma unroll
     for (int j = 0; j < NP / 8; ++j) {
         uint4 v;
-        v.x = pack2<OutT>(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]), &sat_bits);
-        v.y = pack2<OutT>(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]), &sat_bits);
-        v.z = pack2<OutT>(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]), &sat_bits);
-        v.w = pack2<OutT>(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]), &sat_bits);
+        v.x = pack2<OutT>(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]), sat_track);
+        v.y = pack2<OutT>(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]), sat_track);
+        v.z = pack2<OutT>(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]), sat_track);
+        v.w = pack2<OutT>(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]), sat_track);
         *reinterpret_cast<uint4*>(my_row + (SWZ ? (j ^ (lane & 7)) : j) * 16) = v;
     }
     if (sat_bits & (int)0x80008000u) ++sat;  // this thread's row segment of the pass held a saturated value
@@ -255,6 +257,10 @@ __device__ __forceinline__ void epi_pass_tma(uint32_t taddr, uint8_t* wrows, int
                 qa = fma2(f0, f0, qa);
                 qb = fma2(f1, f1, qb);
             }
+            // a stored +-65504 puts at least 65504^2 into its channel's sum of squares over these 32 rows; nothing else
+            // does unless the 32 values average above 11585, i.e. sit within a factor of six of the fp16 range
+            const float qx = qa.x + qb.x, qy = qa.y + qb.y;
+            if (fmaxf(qx, qy) >= 4290774016.f) ++sat;
             float2* ps = reinterpret_cast<float2*>(stat_s + 2 * lane);
             float2* pq = reinterpret_cast<float2*>(stat_q + 2 * lane);
             float2 a2 = *ps, b2 = *pq;

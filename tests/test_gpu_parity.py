@@ -354,6 +354,23 @@ def test_forward_with_a_residual_adds_it_once(shape, mode):
     np.testing.assert_array_equal(blk.a.double().cpu().numpy(), plain["a"])
 
 
+@pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[12]], ids=lambda s: s.name)
+def test_saturated_fp16_stores_of_the_convolution_output_are_reported(shape):
+    """The saved convolution output is fp16 (Sec. 3.2): a value beyond +-65504 is stored as +-65504 and the call says so
+    through nb_cbs_poll_status (still NB_OK).  One input pixel made huge saturates the outputs around it and nothing else
+    is reported when the inputs are ordinary."""
+    import torch
+
+    inp, blk, out = _run_block(shape, 0, cfg_id=24, affine="random")
+    assert "saturated" not in blk.poll()
+    blk.x[0, shape.h // 2, shape.w // 2, :] = 3.0e4
+    blk.w.fill_(1.0)
+    blk.forward()
+    msg = blk.poll()
+    assert "saturated" in msg, msg
+    assert float(blk.y.abs().max()) == 65504.0 and bool(torch.isfinite(blk.y.float()).all())
+
+
 @pytest.mark.parametrize("shape", [SMALL_SHAPES[7], SMALL_SHAPES[9], SMALL_SHAPES[5]], ids=lambda s: s.name)
 def test_backward_hands_the_gradient_to_the_shortcut(shape):
     """nb_cbs_plan_set_bwd_residual: the data-gradient call also adds (or copies) its incoming gradient g into the
