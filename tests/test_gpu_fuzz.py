@@ -1,0 +1,101 @@
+"""Seeded random layer shapes through every call of the block against the fp64 oracle.
+
+The hand-picked shapes of test_gpu_parity.py aim at the tile boundaries known to the author; this file draws shapes
+without knowing them: 96 layers with 1-3 images of 2..69 x 2..69 pixels, 8..384 channels on either side, 1x1 and 3x3,
+stride 1 and 2, at least 32 output pixels.  Each goes through the training step (forward, data gradient, weight
+gradient), the inference call and the bias-head calls (forward and backward), in bf16 and in fp16 operand mode, at the
+bars of the hand-picked shapes.
+
+One reading, for the data gradient of a 1x1 stride-2 layer only: three of four input pixels receive no gradient.  They
+must be exactly zero, and the per-element bar is taken relative to the rms of the pixels that do receive one (the zeros
+would halve the rms and with it the bar, which is defined for a dense tensor)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_10632_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-3
+CHANNELS_IN = [8, 16, 24, 32, 40, 48, 64, 80, 96, 112, 128, 144, 160, 192, 224, 256, 288, 320, 384]
+CHANNELS_OUT = [8, 16, 24, 32, 48, 64, 80, 96, 128, 144, 160, 192, 256, 288, 320, 384]
+
+
+def _draw(rs):
+    while True:
+        n, h, w = int(rs.randint(1, 4)), int(rs.randint(2, 70)), int(rs.randint(2, 70))
+        k, s = int(rs.choice([1, 3])), int(rs.choice([1, 2]))
+        ci, co = int(rs.choice(CHANNELS_IN)), int(rs.choice(CHANNELS_OUT))
+        m = n * oracle.out_extent(h, k, s) * oracle.out_extent(w, k, s)
+        if m < 32 or m * k * k * ci * co > 1.5e9:
+            continue
+        return wl.ConvShape(f"r{n}x{h}x{w}x{ci}->{co}k{k}s{s}", n, h, w, ci, co, k, s, False)
+
+
+def _shapes(seed, count):
+    rs = np.random.RandomState(seed)
+    return [_draw(rs) for _ in range(count)]
+
+
+def _check_dx(name, got, ref, shape):
+    if shape.k == 1 and shape.stride == 2:
+        hit = np.zeros(ref.shape, dtype=bool)
+        hit[:, ::2, ::2, :] = True
+        assert not got[~hit].any() and not ref[~hit].any(), f"{name}: a pixel outside the stride-2 grid received a gradient"
+        sel = lambda t: t[:, ::2, ::2, :]
+        parity.check(name, sel(got), sel(ref), "bf16")
+    else:
+        parity.check(name, got, ref, "bf16")
+
+
+@pytest.mark.parametrize("mode_name,seed", [("bf16", 101), ("fp16", 202)])
+def test_random_shapes_match_oracle(mode_name, seed):
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    mode = nb.NB_MODE_BF16_TC if mode_name == "bf16" else nb.NB_MODE_F16_TC
+    paths = set()
+    for i, shape in enumerate(_shapes(seed, 48)):
+        inp = wl.make_inputs(shape, 31, i, bf16=True, affine="random")
+        blk = CbsBlock(shape, mode=mode, eps=EPS)
+        blk.upload(inp)
+        blk.step()
+        blk.poll()
+        out = blk.download()
+        ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, shape.stride, EPS)
+        try:
+            parity.check_stats(out["mean"], out["invstd"], ref.y, EPS, "bf16")
+            for name in ("a", "dgamma", "dbeta", "dw", "y", "dy"):
+                parity.check(name, out[name], getattr(ref, name), "bf16")
+            _check_dx("dx", out["dx"], ref.dx, shape)
+
+            rm, rv, bias = wl.make_eval_stats(shape, 31, i)
+            up = lambda a: torch.from_numpy(a).to(blk.dev)
+            o = torch.empty_like(blk.a)
+            ws = torch.empty(max(blk.plan.infer_bytes, blk.plan.bwd_bytes, 256), dtype=torch.uint8, device=blk.dev)
+            nb.nb_conv_bn_silu_infer(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, up(rm), up(rv), o, ws)
+            torch.cuda.synchronize()
+            want = oracle.cbs_infer(inp.x, inp.w, inp.gamma, inp.beta, rm, rv, shape.stride, EPS)
+            parity.check("a_eval", o.double().cpu().numpy(), want, "bf16")
+
+            nb.nb_conv_bias_act(blk.plan, blk.x, blk.w, up(bias), 0, o, ws)
+            dx, dw = torch.empty_like(blk.x), torch.empty_like(blk.dw)
+            db = torch.empty(shape.c_out, dtype=torch.float32, device=blk.dev)
+            nb.nb_conv_bias_bwd(blk.plan, blk.x, blk.w, blk.g, dx, dw, db, ws)
+            torch.cuda.synchronize()
+            blk.poll()
+            parity.check("head out", o.double().cpu().numpy(), oracle.conv_bias_act(inp.x, inp.w, bias, shape.stride), "bf16")
+            rdx, rdw, rdb = oracle.conv_bias_bwd(inp.x, inp.w, inp.g, shape.stride)
+            _check_dx("head dx", dx.double().cpu().numpy(), rdx, shape)
+            parity.check("head dw", dw.double().cpu().numpy(), rdw, "bf16")
+            parity.check("head dbias", db.double().cpu().numpy(), rdb, "bf16")
+        except AssertionError as e:
+            raise AssertionError(f"{shape.name} (shape {i} of seed {seed}, paths {blk.plan.paths}): {e}") from None
+        paths.add((blk.plan.paths["fprop"], blk.plan.paths["dgrad"], blk.plan.paths["wgrad"]))
+    # the draw reaches the tensor-core kernels, the CUDA-core fallback and the mixed case (tensor-core forward and weight
+    # gradient beside a CUDA-core data gradient)
+    assert {(1, 1, 1), (0, 0, 0), (1, 0, 1)} <= paths, paths
