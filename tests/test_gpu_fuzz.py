@@ -1,4 +1,5 @@
-"""Seeded random layer shapes through every call of the block against the fp64 oracle.
+"""Seeded random layer shapes through every call of the block against the fp64 oracle, and through the options of a
+chained network against the dense run.
 
 The hand-picked shapes of test_gpu_parity.py aim at the tile boundaries known to the author; this file draws shapes
 without knowing them: 96 layers with 1-3 images of 2..69 x 2..69 pixels, 8..384 channels on either side, 1x1 and 3x3,
@@ -99,3 +100,97 @@ def test_random_shapes_match_oracle(mode_name, seed):
     # the draw reaches the tensor-core kernels, the CUDA-core fallback and the mixed case (tensor-core forward and weight
     # gradient beside a CUDA-core data gradient)
     assert {(1, 1, 1), (0, 0, 0), (1, 0, 1)} <= paths, paths
+
+
+def test_random_shapes_with_every_chain_option_give_the_dense_bits():
+    """The options a chained network uses (x, a_out and g as channel slices of wider tensors; a residual added in the
+    forward pass; the incoming gradient handed to the shortcut; the data gradient written or added into a slice of a
+    wider buffer) switched on in random combinations with random pitches and offsets on 64 random shapes.  None of them
+    changes the arithmetic, so everything the calls write equals the dense run's bits; the sums are the fp32 sum of two
+    16-bit values rounded once (checked exactly); the block output with a residual is held to the oracle's bars; and
+    nothing beside a slice may change.  A plan that cannot take an option says NB_ERR_UNSUPPORTED and runs without it."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    rs = np.random.RandomState(303)
+    used = dict(x_pitch=0, res=0, gres=0, dx_target=0, dx_add=0)
+    for i in range(64):
+        s = _draw(rs)
+        inp = wl.make_inputs(s, 33, i, bf16=True, affine="random")
+        dense = CbsBlock(s, eps=EPS)
+        dense.upload(inp)
+        dense.step()
+        dense.poll()
+        blk = CbsBlock(s, eps=EPS)
+        blk.upload(inp)
+        dev = blk.dev
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(303000 + i)
+        pad = lambda: 8 * int(rs.randint(0, 6))
+        off = {k: pad() for k in "xagrqd"}
+        ld = {k: (s.c_in if k in "xd" else s.c_out) + off[k] + pad() for k in "xagrqd"}
+        try:
+            blk.plan.set_pitches(ld_x=ld["x"], ld_a=ld["a"], ld_g=ld["g"])
+            used["x_pitch"] += 1
+        except nb.NbError as e:  # the CUDA-core forward reads a dense x
+            assert e.status == nb.NB_ERR_UNSUPPORTED
+            off["x"], ld["x"] = 0, s.c_in
+            blk.plan.set_pitches(ld_x=0, ld_a=ld["a"], ld_g=ld["g"])
+        mk = lambda h, w, c: torch.randn(s.n, h, w, c, generator=gen, device=dev).to(torch.bfloat16)
+        X, D = mk(s.h, s.w, ld["x"]), mk(s.h, s.w, ld["d"])
+        A, G, R, Q = (mk(s.ho, s.wo, ld[k]) for k in "agrq")
+        cut = lambda t, k: t[..., off[k]:off[k] + (s.c_in if k in "xd" else s.c_out)]
+        cut(X, "x").copy_(blk.x)
+        cut(G, "g").copy_(blk.g)
+        A0, Q0, D0 = A.clone(), Q.clone(), D.clone()
+        with_res, with_gres, gres_add = rs.rand() < 0.6, rs.rand() < 0.6, bool(rs.rand() < 0.5)
+        dx_target, dx_add = rs.rand() < 0.7, bool(rs.rand() < 0.5)
+        if with_res:
+            blk.plan.set_fwd_residual(cut(R, "r"), ld["r"])
+            used["res"] += 1
+        if with_gres:
+            blk.plan.set_bwd_residual(cut(Q, "q"), ld["q"], accumulate=gres_add)
+            used["gres"] += 1
+        if dx_target:
+            try:
+                blk.plan.set_dx_target(ld_dx=ld["d"], accumulate=dx_add)
+                used["dx_target"] += 1
+                used["dx_add"] += dx_add
+            except nb.NbError as e:  # only the bulk-store epilogue of the stride-1 tensor-core data gradient can
+                assert e.status == nb.NB_ERR_UNSUPPORTED
+                dx_target = False
+        first = lambda t, k: t.data_ptr() + off[k] * t.element_size()
+        nb.nb_conv_bn_silu_fwd(blk.plan, first(X, "x"), blk.w, blk.gamma, blk.beta, None, None, blk.y, blk.mean, blk.invstd, first(A, "a"), blk.ws)
+        nb.nb_conv_bn_silu_bwd_data(blk.plan, first(G, "g"), blk.y, blk.mean, blk.invstd, blk.gamma, blk.beta, blk.w,
+                                    first(D, "d") if dx_target else blk.dx, blk.dgamma, blk.dbeta, blk.dy, blk.ws)
+        nb.nb_conv_bn_silu_bwd_weight(blk.plan, first(X, "x"), blk.dy, blk.dw, blk.ws)
+        torch.cuda.synchronize()
+        blk.poll()
+
+        def beside_untouched(t, t0, k):
+            c = s.c_in if k in "xd" else s.c_out
+            return torch.equal(t[..., :off[k]], t0[..., :off[k]]) and torch.equal(t[..., off[k] + c:], t0[..., off[k] + c:])
+
+        add16 = lambda old, new: (old.float() + new.float()).to(torch.bfloat16)
+        what = f"{s.name} (shape {i}; paths {blk.plan.paths}; res {with_res}, gres {with_gres}/{gres_add}, dx target {dx_target}/{dx_add}; ld {ld}, off {off})"
+        assert beside_untouched(A, A0, "a"), what
+        if with_res:
+            ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, EPS, need_dx=False)
+            parity.check(what + ": a + res", cut(A, "a").double().cpu().numpy(), ref.a + cut(R, "r").double().cpu().numpy(), "bf16")
+        else:
+            assert torch.equal(cut(A, "a"), dense.a), what
+        for name in ("y", "dy", "dw", "dgamma", "dbeta", "mean", "invstd"):
+            assert torch.equal(getattr(blk, name), getattr(dense, name)), (what, name)
+        if dx_target:
+            assert beside_untouched(D, D0, "d"), what
+            assert torch.equal(cut(D, "d"), add16(cut(D0, "d"), dense.dx) if dx_add else dense.dx), what
+        else:
+            assert torch.equal(blk.dx, dense.dx) and torch.equal(D, D0), what
+        if with_gres:
+            assert beside_untouched(Q, Q0, "q"), what
+            assert torch.equal(cut(Q, "q"), add16(cut(Q0, "q"), blk.g) if gres_add else blk.g), what
+        else:
+            assert torch.equal(Q, Q0), what
+    assert min(used.values()) >= 4, used
