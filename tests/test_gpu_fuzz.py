@@ -194,3 +194,89 @@ def test_random_shapes_with_every_chain_option_give_the_dense_bits():
         else:
             assert torch.equal(Q, Q0), what
     assert min(used.values()) >= 4, used
+
+
+def test_random_shapes_through_the_glue_calls_and_the_plan_free_statistics():
+    """The wiring calls of a chained network (5x5 max-pool, 2x upsampling, slice add) forward and backward on 80 random
+    extents (1-3 images of 1..39 x 1..39 pixels, 8..392 channels), both 16-bit types, every operand a randomly placed
+    channel slice of a wider tensor or dense, against the chain oracle's definitions; and the plan-free statistics call on
+    random matrices against the fp64 moments of the tensor it read."""
+    import torch
+
+    from oracle import chain as och
+    from paper_2609_10632_b200 import binding as nb
+
+    rs = np.random.RandomState(404)
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(404)
+
+    def wide(n, h, w, c, dt):
+        off = 8 * int(rs.randint(0, 5))
+        ld = c + off + 8 * int(rs.randint(0, 5))
+        if rs.rand() < 0.3:
+            off, ld = 0, c
+        return torch.randn(n, h, w, ld, generator=gen, device=dev).to(dt), off, ld
+
+    first = lambda t, off: t.data_ptr() + off * t.element_size()
+    f64 = lambda t: t.double().cpu().numpy()
+
+    def beside_untouched(t, t0, off, c):
+        return torch.equal(t[..., :off], t0[..., :off]) and torch.equal(t[..., off + c:], t0[..., off + c:])
+
+    for i in range(80):
+        n, h, w, c = int(rs.randint(1, 4)), int(rs.randint(1, 40)), int(rs.randint(1, 40)), 8 * int(rs.randint(1, 50))
+        dtn = int(rs.choice([nb.NB_DTYPE_BF16, nb.NB_DTYPE_F16]))
+        dt, ulp = (torch.bfloat16, 2.0**-8) if dtn == nb.NB_DTYPE_BF16 else (torch.float16, 2.0**-10)
+        what = f"draw {i}: {n} x {h} x {w} x {c}, dtype {dtn}"
+
+        X, ox, lx = wide(n, h, w, c, dt)
+        Y, oy, ly = wide(n, h, w, c, dt)
+        Y0 = Y.clone()
+        idx = torch.empty(n, h, w, c, dtype=torch.uint8, device=dev)
+        nb.nb_maxpool5_fwd(dtn, n, h, w, c, first(X, ox), first(Y, oy), idx, ld_x=lx, ld_y=ly)
+        ref_y, _ = och.maxpool5(f64(X[..., ox:ox + c]))
+        assert np.array_equal(f64(Y[..., oy:oy + c]), ref_y) and beside_untouched(Y, Y0, oy, c), what + ": max-pool"
+        G, og, lg = wide(n, h, w, c, dt)
+        DX, od, ldd = wide(n, h, w, c, dt)
+        DX0, add = DX.clone(), bool(rs.rand() < 0.5)
+        nb.nb_maxpool5_bwd(dtn, n, h, w, c, first(G, og), idx, first(DX, od), accumulate=add, ld_g=lg, ld_dx=ldd)
+        torch.cuda.synchronize()
+        # equal maxima may be routed to either position: the gradient is checked from the positions the kernel recorded
+        want = och.maxpool5_bwd(f64(G[..., og:og + c]), idx.cpu().numpy()) + (f64(DX0[..., od:od + c]) if add else 0.0)
+        assert np.abs(f64(DX[..., od:od + c]) - want).max() <= ulp * max(1.0, np.abs(want).max()), what + ": max-pool gradient"
+        assert beside_untouched(DX, DX0, od, c), what + ": max-pool gradient"
+
+        S, os_, ls = wide(n, h, w, c, dt)
+        L, ol, ll = wide(n, 2 * h, 2 * w, c, dt)
+        L0 = L.clone()
+        nb.nb_upsample2(dtn, n, h, w, c, first(S, os_), first(L, ol), ld_small=ls, ld_large=ll)
+        torch.cuda.synchronize()
+        assert np.array_equal(f64(L[..., ol:ol + c]), och.upsample2(f64(S[..., os_:os_ + c]))) and beside_untouched(L, L0, ol, c), what + ": upsampling"
+        S0, add = S.clone(), bool(rs.rand() < 0.5)
+        nb.nb_upsample2(dtn, n, h, w, c, first(L, ol), first(S, os_), backward=True, accumulate=add, ld_small=ls, ld_large=ll)
+        torch.cuda.synchronize()
+        want = och.upsample2_bwd(f64(L[..., ol:ol + c])) + (f64(S0[..., os_:os_ + c]) if add else 0.0)
+        assert np.abs(f64(S[..., os_:os_ + c]) - want).max() <= ulp * max(1.0, np.abs(want).max()), what + ": upsampling gradient"
+        assert beside_untouched(S, S0, os_, c), what + ": upsampling gradient"
+
+        A, oa, la = wide(n, h, w, c, dt)
+        B, ob, lb = wide(n, h, w, c, dt)
+        O, oo, lo = wide(n, h, w, c, dt)
+        O0, with_b, add = O.clone(), bool(rs.rand() < 0.6), bool(rs.rand() < 0.5)
+        nb.nb_slice_add(dtn, n * h * w, c, first(O, oo), lo, first(A, oa), la, first(B, ob) if with_b else None, lb if with_b else 0, accumulate=add)
+        torch.cuda.synchronize()
+        want = A[..., oa:oa + c].float() + (B[..., ob:ob + c].float() if with_b else 0.0) + (O0[..., oo:oo + c].float() if add else 0.0)
+        assert torch.equal(O[..., oo:oo + c], want.to(dt)) and beside_untouched(O, O0, oo, c), what + ": slice add"
+
+        m, cc = int(rs.randint(2, 5000)), 8 * int(rs.randint(1, 73))
+        sdt = int(rs.choice([nb.NB_DTYPE_F16, nb.NB_DTYPE_F32]))
+        y = torch.randn(m, cc, generator=gen, device=dev) * float(rs.uniform(0.5, 3)) + float(rs.uniform(-2, 2))
+        y = y.to(torch.float16 if sdt == nb.NB_DTYPE_F16 else torch.float32)
+        mean, invstd = torch.empty(cc, device=dev), torch.empty(cc, device=dev)
+        nb.nb_bn_stats_static(y, sdt, m, cc, EPS, mean, invstd)
+        torch.cuda.synchronize()
+        ref_mean, ref_var = f64(y).mean(0), f64(y).var(0)
+        ref_invstd = 1.0 / np.sqrt(ref_var + EPS)
+        assert (np.abs(f64(mean) - ref_mean) <= 2e-6 * np.sqrt(ref_mean**2 + ref_var) + 1e-7).all(), f"{what}: mean of {m} x {cc}"
+        assert (np.abs(f64(invstd) - ref_invstd) / ref_invstd <= 1e-6 * (1 + ref_mean**2 / (ref_var + EPS)) + 2e-6).all(), f"{what}: invstd of {m} x {cc}"
