@@ -89,6 +89,9 @@ struct nb_cbs_plan_s {
     int acc_copies_f = 0, acc_copies_b = 0;
     bool stem = false;       // 3-channel 3x3 stride-2 first layer: dedicated direct kernels
     int stem_blocks = 0;     // blocks (= partial slices) of the stem wgrad kernel
+    bool stem_wide = false;  // the stem forward kernel takes 320-pixel strips (wide images)
+    int stem_fprop_blocks = 0;  // its grid (= its partial slices)
+    int stem_wgrad_blocks = 0;  // grid (= partial slices) of the stem weight-gradient kernel (128-pixel strips on wide images)
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     double prof_ms[SITE_COUNT] = {};
@@ -433,6 +436,23 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->stem = d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
               g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0 && g.m < (1LL << 31) && (long long)g.n * g.h * g.w * 3 < (1LL << 31);
     p->stem_blocks = (int)std::min<long long>(stem_num_strips(g), (long long)p->sm_count * 4);  // grid of the three first-layer kernels: one wave of four resident blocks per SM
+    p->stem_wide = g.wo >= STEM_TQ_WIDE / 2;  // (a strip of a narrower row would leave most of its tile slots empty)
+    if (const char* e2 = getenv("NB_STEM_WIDE")) p->stem_wide = atoi(e2) != 0;
+    p->stem_fprop_blocks = p->stem_wide ? (int)std::min<long long>(stem_num_strips(g, STEM_TQ_WIDE), (long long)p->sm_count * 4) : p->stem_blocks;
+    p->stem_wgrad_blocks = p->stem_wide ? (int)std::min<long long>(stem_num_strips(g, STEM_TQ_WGRAD), (long long)p->sm_count * 4) : p->stem_blocks;
+    if (p->stem && p->stem_wide) {  // (more than the 48 KB a kernel gets without asking)
+        DeviceGuard on_device(p->device);
+        cudaError_t ae = cudaFuncSetAttribute(stem_wgrad_mma_kernel<48, __nv_bfloat16, STEM_TQ_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)stem_wgrad_smem_bytes<48, __nv_bfloat16, STEM_TQ_WGRAD>());
+        if (ae == cudaSuccess)
+            ae = cudaFuncSetAttribute(stem_wgrad_mma_kernel<48, __half, STEM_TQ_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)stem_wgrad_smem_bytes<48, __half, STEM_TQ_WGRAD>());
+        if (ae != cudaSuccess) {
+            p->stem_wide = false;
+            p->stem_fprop_blocks = p->stem_wgrad_blocks = p->stem_blocks;
+            (void)cudaGetLastError();
+        }
+    }
     p->nparts = std::max(std::max(std::max(e.blocks_reduce, e.blocks_stats), p->tc.fprop_parts), p->stem ? p->stem_blocks : 0);
     const size_t C = (size_t)g.c_out;
     size_t off = 0;
@@ -633,11 +653,17 @@ nb_status nb_conv_bn_silu_fwd(nb_cbs_plan p, const void* x, const void* w, const
         // the first layer's kernel sums the statistics of the values it stores itself (one partial slice per block)
         SiteTimer tm(p, SITE_FPROP, st);
         const bool fuse = p->fuse_finalize;  // sums into the plan's accumulators; the normalise + SiLU pass finalizes
-        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
-                               static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{}, fuse ? static_cast<float*>(nullptr) : part,
-                               fuse ? p->acc : static_cast<double*>(nullptr), fuse ? p->acc_copies_f : 1));
+        if (p->stem_wide) {
+            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT, STEM_TQ_WIDE>, dim3(p->stem_fprop_blocks), dim3(128), 0, st, 1,
+                                   static_cast<const AT*>(x), static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{},
+                                   fuse ? static_cast<float*>(nullptr) : part, fuse ? p->acc : static_cast<double*>(nullptr), fuse ? p->acc_copies_f : 1));
+        } else {
+            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, __half, false, AT, STEM_TQ>, dim3(p->stem_fprop_blocks), dim3(128), 0, st, 1,
+                                   static_cast<const AT*>(x), static_cast<const AT*>(w), static_cast<__half*>(y_saved), p->g, StemEpi{},
+                                   fuse ? static_cast<float*>(nullptr) : part, fuse ? p->acc : static_cast<double*>(nullptr), fuse ? p->acc_copies_f : 1));
+        }
         NB_LAUNCH_OK("stem_fprop");
-        nparts = p->stem_blocks;
+        nparts = p->stem_fprop_blocks;
         finalized = fuse;
     } else if (p->tc.fprop) {
         SiteTimer tm(p, SITE_FPROP, st);
@@ -678,9 +704,15 @@ nb_status run_infer(nb_cbs_plan_s* p, const void* x, const void* w, const float*
     }
     if (!is_f32(p) && p->stem) {  // the first layer's own kernel applies the coefficients and the activation itself
         SiteTimer tm(p, SITE_INFER, st);
-        NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(w),
-                               static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act}, static_cast<float*>(nullptr),
-                               static_cast<double*>(nullptr), 1));
+        if (p->stem_wide) {
+            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT, STEM_TQ_WIDE>, dim3(p->stem_fprop_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
+                                   static_cast<const AT*>(w), static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act},
+                                   static_cast<float*>(nullptr), static_cast<double*>(nullptr), 1));
+        } else {
+            NB_WITH_AT(p, launch_k(stem_fprop_mma_kernel<48, AT, true, AT, STEM_TQ>, dim3(p->stem_fprop_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x),
+                                   static_cast<const AT*>(w), static_cast<AT*>(out), p->g, StemEpi{gamma, beta, rmean, rvar, p->desc.eps, act},
+                                   static_cast<float*>(nullptr), static_cast<double*>(nullptr), 1));
+        }
         return launch_ok("stem_fprop (fused epilogue)");
     }
     float* scale = reinterpret_cast<float*>(ws + p->off_scale);
@@ -867,13 +899,18 @@ nb_status nb_conv_bn_silu_bwd_weight(nb_cbs_plan p, const void* x, const void* d
     if (p->stem) {
         {
             SiteTimer tm(p, SITE_WGRAD, st);
-            NB_WITH_AT(p, launch_k(stem_wgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(x), static_cast<const AT*>(dy), partial,
-                                   p->g));
+            if (p->stem_wide) {
+                NB_WITH_AT(p, launch_k(stem_wgrad_mma_kernel<48, AT, STEM_TQ_WGRAD>, dim3(p->stem_wgrad_blocks), dim3(128),
+                                       stem_wgrad_smem_bytes<48, AT, STEM_TQ_WGRAD>(), st, 1, static_cast<const AT*>(x), static_cast<const AT*>(dy), partial, p->g));
+            } else {
+                NB_WITH_AT(p, launch_k(stem_wgrad_mma_kernel<48, AT, STEM_TQ>, dim3(p->stem_wgrad_blocks), dim3(128), stem_wgrad_smem_bytes<48, AT, STEM_TQ>(), st, 1,
+                                       static_cast<const AT*>(x), static_cast<const AT*>(dy), partial, p->g));
+            }
             NB_LAUNCH_OK("stem_wgrad");
         }
         const size_t elems = (size_t)p->g.c_out * p->g.kdim;
         SiteTimer tm(p, SITE_SPLITK_REDUCE, st);
-        launch_k(splitk_reduce_tall_kernel, dim3((unsigned)((elems + 31) / 32)), dim3(1024), 0, st, 1, partial, p->stem_blocks, elems, dw);
+        launch_k(splitk_reduce_tall_kernel, dim3((unsigned)((elems + 31) / 32)), dim3(1024), 0, st, 1, partial, p->stem_wgrad_blocks, elems, dw);
         return launch_ok("splitk_reduce");
     }
     if (p->tc.wgrad) {

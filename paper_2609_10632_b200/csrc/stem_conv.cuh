@@ -4,7 +4,8 @@
 // (m16n8k16, fp32 accumulation).  All three are HBM-bound by design (157 MB of y / dy against 39 MB of x / dx at batch
 // 16, 640 x 640): every global access is a coalesced 16-byte (or 4-byte) vector; the 3 x 3 x 3 patches are never gathered
 // from global memory but cut out of input rows staged in shared memory.
-// Work unit of every kernel: a STRIP of up to 64 consecutive output pixels of one output row (16 per warp).
+// Work unit of every kernel: a STRIP of up to 64 consecutive output pixels of one output row (16 per warp); the forward
+// kernel takes strips of up to 320 pixels on wide images (five tiles per warp).
 // COUT is a template parameter (48 for the detector's stem).
 #pragma once
 #include "common.cuh"
@@ -12,9 +13,12 @@
 namespace nbcbs {
 
 constexpr int STEM_CIN = 3, STEM_K = 3, STEM_TAPS = 9, STEM_KDIM = 27;
-constexpr int STEM_TQ = 64;                                   // output pixels per strip
-constexpr int STEM_ROW_ELEMS = (2 * STEM_TQ + 1) * STEM_CIN;  // input values of one staged row: columns 2*q0-1 .. 2*q0+2*TQ-1
-constexpr int STEM_XCHUNKS = (STEM_ROW_ELEMS + 7 + 7) / 8;    // 16-byte chunks per staged row incl. the alignment shift (<= 7)
+constexpr int STEM_TQ = 64;        // output pixels per strip (data and weight gradient; forward of narrow images)
+constexpr int STEM_TQ_WIDE = 320;  // the forward kernel's strip on wide images: per-strip work is shared by 20 tiles instead of 4
+__host__ __device__ constexpr int stem_xchunks(int tq) {  // 16-byte chunks per staged input row: columns 2*q0-1 .. 2*q0+2*tq-1, plus the alignment shift (<= 7)
+    return ((2 * tq + 1) * STEM_CIN + 7 + 7) / 8;
+}
+constexpr int STEM_XCHUNKS = stem_xchunks(STEM_TQ);
 constexpr int STEM_XPITCH = STEM_XCHUNKS * 8;
 
 template <typename T> __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1);
@@ -37,21 +41,52 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
 }
 
-// Strip number -> image n, output row p, first output column q0.
+// Strip number -> image n, output row p, first output column q0.  `sh` is filled by the kernels that stage input rows:
+// the alignment shifts of the strip's three staged rows, 3 bits each (see stem_stage_rows_async).
 struct StemStrip {
-    int n, p, q0;
+    int n, p, q0, sh;
 };
-__device__ __forceinline__ StemStrip stem_strip(long long t, const Geom& g, int strips_per_row) {
+template <int TQ = STEM_TQ> __device__ __forceinline__ StemStrip stem_strip(long long t, const Geom& g, int strips_per_row) {
     // (32-bit divisions: the plan admits fewer than 2^31 output pixels; 64-bit ones cost about a hundred instructions each,
     // and these kernels are bound by instruction issue)
     StemStrip s;
     const unsigned tt = (unsigned)t, t1 = tt / (unsigned)strips_per_row;
-    s.q0 = (int)(tt - t1 * (unsigned)strips_per_row) * STEM_TQ;
+    s.q0 = (int)(tt - t1 * (unsigned)strips_per_row) * TQ;
     s.n = (int)(t1 / (unsigned)g.ho);
     s.p = (int)(t1 - (unsigned)s.n * (unsigned)g.ho);
+    s.sh = 0;
     return s;
 }
-__host__ __device__ inline long long stem_num_strips(const Geom& g) { return (long long)g.n * g.ho * ((g.wo + STEM_TQ - 1) / STEM_TQ); }
+// A block visits strips blockIdx.x, + gridDim.x, + 2 gridDim.x, ...: the stride is decomposed once (two divisions), and
+// every further strip follows from the one before it by additions and two carries.
+struct StemWalk {
+    int dq0, dp, dn, row_len, ho;  // stride in first-column units / rows / images; strips_per_row * strip width; output rows
+};
+template <int TQ = STEM_TQ> __device__ __forceinline__ StemWalk stem_walk(const Geom& g, int strips_per_row) {
+    StemWalk k;
+    const unsigned d = gridDim.x, d1 = d / (unsigned)strips_per_row;
+    k.dq0 = (int)(d - d1 * (unsigned)strips_per_row) * TQ;
+    k.dn = (int)(d1 / (unsigned)g.ho);
+    k.dp = (int)(d1 - (unsigned)k.dn * (unsigned)g.ho);
+    k.row_len = strips_per_row * TQ;
+    k.ho = g.ho;
+    return k;
+}
+__device__ __forceinline__ StemStrip stem_advance(StemStrip s, const StemWalk& k) {
+    s.q0 += k.dq0;
+    if (s.q0 >= k.row_len) {
+        s.q0 -= k.row_len;
+        ++s.p;
+    }
+    s.p += k.dp;  // (p < ho, dp < ho and one carry: a single subtraction brings it back into range)
+    if (s.p >= k.ho) {
+        s.p -= k.ho;
+        ++s.n;
+    }
+    s.n += k.dn;
+    return s;
+}
+__host__ __device__ inline long long stem_num_strips(const Geom& g, int tq = STEM_TQ) { return (long long)g.n * g.ho * ((g.wo + tq - 1) / tq); }
 
 // 16-byte asynchronous copy global -> shared; bytes past `src_bytes` (0..16) are written as zeros.
 __device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, int src_bytes) {
@@ -68,26 +103,34 @@ template <int N> __device__ __forceinline__ void cp_async_wait_pending() { asm v
 // of NS buffers, NS - 1 strips in flight per block): with one strip in flight the kernels were bound by memory latency
 // (bytes in flight per SM x 148 / latency was far below the HBM rate), not by bandwidth.  `total` = number of elements of x.
 __device__ __forceinline__ int stem_row_start(const Geom& g, const StemStrip& s, int r, int& shift) {
-    // (int arithmetic: the plan admits fewer than 2^31 input elements)
-    const int e0 = ((s.n * g.h + (2 * s.p - 1 + r)) * g.w + (2 * s.q0 - 1)) * 3;  // negative only inside the padding
-    const int a0 = e0 >= 0 ? (e0 & ~7) : -((-e0 + 7) & ~7);
-    shift = e0 - a0;
-    return a0;
+    // (int arithmetic: the plan admits fewer than 2^31 input elements; e0 is negative only inside the padding, and in two's
+    // complement the masks below round towards minus infinity there too)
+    const int e0 = ((s.n * g.h + (2 * s.p - 1 + r)) * g.w + (2 * s.q0 - 1)) * 3;
+    shift = e0 & 7;
+    return e0 & ~7;
 }
-__device__ __forceinline__ void stem_stage_rows_async(const unsigned short* __restrict__ x, const Geom& g, int total, const StemStrip& s,
-                                                      unsigned short (*xrow)[STEM_XPITCH]) {
+// WHOLE = false stages only what the strip's own pixels read (a wide strip of a narrower row); what lies behind in the buffer
+// is then stale, which only a kernel whose tiles' rows are independent of one another may ignore.
+template <int TQ = STEM_TQ, bool WHOLE = true>
+__device__ __forceinline__ int stem_stage_rows_async(const unsigned short* __restrict__ x, const Geom& g, int total, const StemStrip& s,
+                                                     unsigned short (*xrow)[stem_xchunks(TQ) * 8]) {
+    int shifts = 0;  // returned: the three rows' shifts, 3 bits each
+    const int width = g.wo - s.q0 < TQ ? g.wo - s.q0 : TQ;  // output pixels the strip really has
 #pragma unroll
     for (int r = 0; r < 3; ++r) {
         int sh;
         const int a0 = stem_row_start(g, s, r, sh);
+        shifts |= sh << (3 * r);
         const bool row_ok = 2 * s.p - 1 + r >= 0;
-        for (int ci = threadIdx.x; ci < STEM_XCHUNKS; ci += blockDim.x) {
+        const int nchunks = WHOLE ? stem_xchunks(TQ) : ((2 * width + 1) * STEM_CIN + sh + 7) >> 3;
+        for (int ci = threadIdx.x; ci < nchunks; ci += blockDim.x) {
             const int start = a0 + 8 * ci;
             int bytes = 0;  // a chunk before the tensor's start (a0 < 0: only padding lies there), in row -1 or past the end: zeros
             if (row_ok && start >= 0 && start < total) bytes = total - start >= 8 ? 16 : (total - start) * 2;
             cp_async16_zfill(&xrow[r][8 * ci], bytes ? x + start : x, bytes);
         }
     }
+    return shifts;
 }
 
 // Two fp32 values rounded to a pair of 16-bit values (fp16 saturates at the largest finite value), and back.
@@ -120,13 +163,14 @@ struct StemEpi {
 // adds them to accumulator set blockIdx.x mod acc_copies of [acc_copies][2][COUT] doubles (batch statistics
 // without a second pass over y; fixed order, bitwise reproducible).  EPI = true: OutT = activations, see StemEpi.
 // InT = the 16-bit type of x and w (bf16, or IEEE fp16).
-template <int COUT, typename OutT = __half, bool EPI = false, typename InT = __nv_bfloat16>
+template <int COUT, typename OutT = __half, bool EPI = false, typename InT = __nv_bfloat16, int TQ = STEM_TQ>
 __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __restrict__ x, const InT* __restrict__ w, OutT* __restrict__ y, Geom g,
                                                                 StemEpi ep, float* __restrict__ partials, double* __restrict__ acc, int acc_copies) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 8 == 0, "whole n-blocks");
-    constexpr int NB = COUT / 8;
+    static_assert(TQ % 64 == 0, "whole 16-pixel tiles for each of the four warps");
+    constexpr int NB = COUT / 8, XPITCH = stem_xchunks(TQ) * 8;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
     const unsigned short* xs = reinterpret_cast<const unsigned short*>(x);
     const unsigned short* wsrc = reinterpret_cast<const unsigned short*>(w);
@@ -144,7 +188,7 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
             for (int e = 0; e < 2; ++e) {
                 const int k = s2 * 16 + j * 8 + tq * 2 + e, i = s2 * 4 + j * 2 + e;
                 krow[i] = k < STEM_KDIM ? k / 9 : 1;
-                koff[i] = krow[i] * STEM_XPITCH + (k < STEM_KDIM ? k % 9 : 3);
+                koff[i] = krow[i] * XPITCH + (k < STEM_KDIM ? k % 9 : 3);
                 if (k < STEM_KDIM && k % 9 < 3) left_mask |= 1u << i;
             }
 #pragma unroll
@@ -175,18 +219,19 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) ssum[nb] = ssq[nb] = make_float2(0.f, 0.f);
     }
-    constexpr int NS = 4;  // ring of staged strips
-    __shared__ __align__(16) unsigned short xrow[NS][3][STEM_XPITCH];
+    constexpr int NS = TQ == STEM_TQ ? 4 : 3;  // ring of staged strips
+    __shared__ __align__(16) unsigned short xrow[NS][3][XPITCH];
     __shared__ __align__(16) OutT stage[4][16 * COUT];
     const int total = g.n * g.h * g.w * 3;
-    const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
-    const long long nstrips = stem_num_strips(g);
+    const int strips_per_row = (g.wo + TQ - 1) / TQ;
+    const long long nstrips = stem_num_strips(g, TQ);
+    const StemWalk walk = stem_walk<TQ>(g, strips_per_row);
     StemStrip ahead[NS - 1];  // the strips whose rows are in flight, decoded once
 #pragma unroll
     for (int k = 0; k < NS - 1; ++k) {  // (one group per strip, empty when the block has no such strip)
         const long long tk = blockIdx.x + (long long)k * gridDim.x;
-        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
-        if (tk < nstrips) stem_stage_rows_async(xs, g, total, ahead[k], xrow[k]);
+        ahead[k] = k == 0 ? stem_strip<TQ>(tk < nstrips ? tk : 0, g, strips_per_row) : stem_advance(ahead[k > 0 ? k - 1 : 0], walk);
+        if (tk < nstrips) ahead[k].sh = stem_stage_rows_async<TQ, TQ == STEM_TQ>(xs, g, total, ahead[k], xrow[k]);
         cp_async_commit();
     }
     int buf = 0;
@@ -197,24 +242,31 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
         cp_async_wait_pending<NS - 2>();
         __syncthreads();  // this strip's rows have landed; the buffer refilled below (the previous strip's) has been consumed
         const long long tn = t + (long long)(NS - 1) * gridDim.x;
-        if (tn < nstrips) {
-            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
-            stem_stage_rows_async(xs, g, total, ahead[NS - 2], xrow[(buf + NS - 1) % NS]);
+        if (tn < nstrips) {  // (then strip tn - gridDim.x, which ahead[NS - 2] still holds, was decoded too)
+            ahead[NS - 2] = stem_advance(ahead[NS - 2], walk);
+            ahead[NS - 2].sh = stem_stage_rows_async<TQ, TQ == STEM_TQ>(xs, g, total, ahead[NS - 2], xrow[(buf + NS - 1) % NS]);
         }
         cp_async_commit();
-        const int qw = s.q0 + warp * 16;  // first output column of this warp's 16 pixels
-        if (qw < g.wo) {
-            int sh[3], addr[8];
+        // per strip: where this lane's eight fragment elements sit in the staged rows, relative to a pixel's first element
+        int addr[8];
+        {
+            int sh[3];
 #pragma unroll
-            for (int r = 0; r < 3; ++r) stem_row_start(g, s, r, sh[r]);
+            for (int r = 0; r < 3; ++r) sh[r] = (s.sh >> (3 * r)) & 7;
 #pragma unroll
             for (int i = 0; i < 8; ++i) addr[i] = koff[i] + (krow[i] == 0 ? sh[0] : krow[i] == 1 ? sh[1] : sh[2]);
-            const unsigned short* xr = &xrow[buf][0][0] + 6 * (warp * 16 + gq);
+        }
+        const long long mrow = ((long long)s.n * g.ho + s.p) * g.wo;  // first output pixel of the strip's row
+#pragma unroll 1
+        for (int tile = warp; tile < TQ / 16; tile += 4) {  // (one tile per warp with 64-pixel strips)
+            const int qw = s.q0 + tile * 16;  // first output column of this tile's 16 pixels
+            if (qw >= g.wo) break;
+            const unsigned short* xr = &xrow[buf][0][0] + 6 * (tile * 16 + gq);
             uint32_t a[2][4];
             bool row_ok[2];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {  // fragment rows gq and gq + 8
-                row_ok[half] = qw + gq + half * 8 < g.wo;  // (pixels past the row's end compute on defined staged values and are dropped below)
+                row_ok[half] = qw + gq + half * 8 < g.wo;  // (pixels past the row's end compute on whatever the buffer holds there and are dropped below)
                 unsigned short v[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) v[i] = xr[addr[i] + 48 * half];
@@ -257,10 +309,10 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
                     }
                 }
             __syncwarp();
-            const long long m0 = ((long long)s.n * g.ho + s.p) * g.wo + qw;
             const int rows = g.wo - qw < 16 ? g.wo - qw : 16;
             const int nvec = rows * COUT / 8;  // 16-byte pieces of the tile that exist
-            for (int v = lane; v < nvec; v += 32) st16(y + (size_t)m0 * COUT + v * 8, ld16(st + v * 8));
+            OutT* yt = y + (size_t)(mrow + qw) * COUT;
+            for (int v = lane; v < nvec; v += 32) st16(yt + v * 8, ld16(st + v * 8));
             __syncwarp();
         }
     }
@@ -327,28 +379,37 @@ __global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restr
     const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
     const long long nstrips = stem_num_strips(g);
     constexpr int VPP = COUT / 8;  // 16-byte vectors per pixel
-    // asynchronous staging of dy[i..i+1][q0 .. q0+64][:] (zeros past the last row / column)
+    // asynchronous staging of dy[i..i+1][q0 .. q0+64][:] (zeros past the last row / column).  A row's 65 pixels are one
+    // contiguous run of 65 * VPP vectors in global memory; in shared memory pixels are STEM_DYPITCH apart.  A thread copies
+    // vector `vec` of pixels px0, px0 + PXSTEP, ...: both addresses advance by constants (no division per copy).
+    constexpr int PXSTEP = 128 / VPP, PXITER = (STEM_TQ + 1 + PXSTEP - 1) / PXSTEP;
+    const int px0 = threadIdx.x / VPP, vec = threadIdx.x - px0 * VPP;
+    const bool stager = px0 < PXSTEP;  // (128 threads = PXSTEP whole pixels and a remainder that stays idle)
     auto stage_async = [&](const StemStrip& s, T(*dst)[(STEM_TQ + 1) * STEM_DYPITCH]) {
-        // a row's 65 pixels are one contiguous run of 65 * VPP vectors in global memory; in shared memory pixels are
-        // STEM_DYPITCH apart
-        const T* row0 = dy + (((size_t)s.n * g.ho + s.p) * g.wo + s.q0) * COUT;
+        if (!stager) return;
+        const T* row0 = dy + (((size_t)s.n * g.ho + s.p) * g.wo + s.q0 + px0) * COUT + vec * 8;
         const int npx = g.wo - s.q0;  // pixels of the row from q0 on
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const bool row_ok = s.p + r < g.ho;
             const T* src = row0 + (size_t)r * g.wo * COUT;
-            for (int u = threadIdx.x; u < (STEM_TQ + 1) * VPP; u += blockDim.x) {
-                const int px = u / VPP;
-                const bool ok = row_ok && px < npx;
-                cp_async16_zfill(&dst[r][u * 8 + px * (STEM_DYPITCH - COUT)], ok ? src + u * 8 : dy, ok ? 16 : 0);
+            T* d = &dst[r][px0 * STEM_DYPITCH + vec * 8];
+#pragma unroll
+            for (int it = 0; it < PXITER; ++it) {
+                const int px = px0 + it * PXSTEP;
+                if (px <= STEM_TQ) {
+                    const bool ok = row_ok && px < npx;
+                    cp_async16_zfill(d + it * PXSTEP * STEM_DYPITCH, ok ? src + it * PXSTEP * COUT : dy, ok ? 16 : 0);
+                }
             }
         }
     };
+    const StemWalk walk = stem_walk(g, strips_per_row);
     StemStrip ahead[NS - 1];  // the strips whose rows are in flight, decoded once (p = dy row i, q0 = first dy column)
 #pragma unroll
     for (int k = 0; k < NS - 1; ++k) {
         const long long tk = blockIdx.x + (long long)k * gridDim.x;
-        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
+        ahead[k] = k == 0 ? stem_strip(tk < nstrips ? tk : 0, g, strips_per_row) : stem_advance(ahead[k > 0 ? k - 1 : 0], walk);
         if (tk < nstrips) stage_async(ahead[k], dys[k]);
         cp_async_commit();
     }
@@ -360,8 +421,8 @@ __global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restr
         cp_async_wait_pending<NS - 2>();
         __syncthreads();  // this strip's rows have landed; the buffer refilled below has been consumed
         const long long tn = t + (long long)(NS - 1) * gridDim.x;
-        if (tn < nstrips) {
-            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
+        if (tn < nstrips) {  // (then strip tn - gridDim.x, which ahead[NS - 2] still holds, was decoded too)
+            ahead[NS - 2] = stem_advance(ahead[NS - 2], walk);
             stage_async(ahead[NS - 2], dys[(buf + NS - 1) % NS]);
         }
         cp_async_commit();
@@ -426,20 +487,29 @@ __global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restr
 // and read back transposed with ldmatrix), B = the pixels' patch values cut out of the staged input rows.  A block sums
 // the strips it is dealt; its four warps are combined in a fixed order into the block's slice of `partial`
 // [gridDim.x][COUT][27].
-template <int COUT, typename T = __nv_bfloat16>
+// TQ = strip width: STEM_TQ, or STEM_TQ_WGRAD on wide images (two tiles per warp and strip: the per-strip work -- staging
+// loops, strip arithmetic, one block-wide barrier -- is shared by twice as many tiles).  Dynamic shared memory:
+// stem_wgrad_smem_bytes<COUT, T, TQ>().
+constexpr int STEM_TQ_WGRAD = 128;
+template <int COUT, typename T, int TQ> struct StemWgradRing {
+    static constexpr int NS = TQ == STEM_TQ ? 4 : 3;  // ring of staged strips
+    unsigned short xrow[NS][3][stem_xchunks(TQ) * 8];
+    T dys[NS][TQ * COUT];  // the strip's TQ x COUT piece of dy (one contiguous run), per buffer
+};
+template <int COUT, typename T, int TQ> constexpr size_t stem_wgrad_smem_bytes() {
+    return sizeof(StemWgradRing<COUT, T, TQ>) > 4 * sizeof(float[COUT][33]) ? sizeof(StemWgradRing<COUT, T, TQ>) : 4 * sizeof(float[COUT][33]);
+}
+template <int COUT, typename T = __nv_bfloat16, int TQ = STEM_TQ>
 __global__ void __launch_bounds__(128, 4) stem_wgrad_mma_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, Geom g) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 16 == 0, "whole m-blocks");
+    static_assert(TQ % 64 == 0, "whole 16-pixel tiles for each of the four warps");
     constexpr int MB = COUT / 16, NBK = 4;  // accumulator blocks: MB x 16 channels by NBK x 8 filter positions (27 padded to 32)
-    constexpr int NS = 4;  // ring of staged strips
-    struct Ring {
-        unsigned short xrow[NS][3][STEM_XPITCH];
-        T dys[NS][STEM_TQ * COUT];  // the strip's 64 x COUT piece of dy (one contiguous run), per buffer
-    };
+    typedef StemWgradRing<COUT, T, TQ> Ring;
+    constexpr int NS = Ring::NS, XPITCH = stem_xchunks(TQ) * 8;
     typedef float Red[COUT][33];
-    constexpr size_t kRaw = sizeof(Ring) > 4 * sizeof(Red) ? sizeof(Ring) : 4 * sizeof(Red);
-    __shared__ __align__(16) unsigned char raw[kRaw];  // the ring while strips are processed, then the four warps' sums
+    extern __shared__ __align__(16) unsigned char raw[];  // the ring while strips are processed, then the four warps' sums
     Ring& ring = *reinterpret_cast<Ring*>(raw);
     Red* red = reinterpret_cast<Red*>(raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
@@ -452,7 +522,7 @@ __global__ void __launch_bounds__(128, 4) stem_wgrad_mma_kernel(const T* __restr
     for (int nb = 0; nb < NBK; ++nb) {
         const int k = nb * 8 + gq;
         krow[nb] = k < STEM_KDIM ? k / 9 : 1;
-        koff[nb] = krow[nb] * STEM_XPITCH + (k < STEM_KDIM ? k % 9 : 3);
+        koff[nb] = krow[nb] * XPITCH + (k < STEM_KDIM ? k % 9 : 3);
         if (k < STEM_KDIM && k % 9 < 3) left_mask |= 1u << nb;
     }
     float acc[MB][NBK][4];
@@ -461,25 +531,29 @@ __global__ void __launch_bounds__(128, 4) stem_wgrad_mma_kernel(const T* __restr
 #pragma unroll
         for (int b = 0; b < NBK; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = acc[a][b][3] = 0.f;
     const int total = g.n * g.h * g.w * 3;
-    const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
-    const long long nstrips = stem_num_strips(g);
+    const int strips_per_row = (g.wo + TQ - 1) / TQ;
+    const long long nstrips = stem_num_strips(g, TQ);
     // asynchronous staging of a strip: the three input rows and dy[strip][:] (zeros past the row's end: those pixels then
     // contribute nothing)
-    auto stage_async = [&](const StemStrip& s, int b) {
-        stem_stage_rows_async(xs, g, total, s, ring.xrow[b]);
-        const size_t m0 = ((size_t)s.n * g.ho + s.p) * g.wo + s.q0;
-        const int np = g.wo - s.q0 < STEM_TQ ? g.wo - s.q0 : STEM_TQ;
-        for (int v = threadIdx.x; v < STEM_TQ * COUT / 8; v += blockDim.x) {
-            const bool ok = v * 8 < np * COUT;
-            cp_async16_zfill(&ring.dys[b][v * 8], ok ? dy + m0 * COUT + v * 8 : dy, ok ? 16 : 0);
+    auto stage_async = [&](const StemStrip& s, int b) -> int {
+        const int shifts = stem_stage_rows_async<TQ, true>(xs, g, total, s, ring.xrow[b]);  // (whole: pixels past the row's end must read defined values)
+        const T* src = dy + (((size_t)s.n * g.ho + s.p) * g.wo + s.q0) * COUT;
+        const int nv = (g.wo - s.q0 < TQ ? g.wo - s.q0 : TQ) * (COUT / 8);  // 16-byte vectors of dy that exist
+#pragma unroll
+        for (int it = 0; it < TQ * COUT / 8 / 128; ++it) {
+            const int v = threadIdx.x + it * 128;
+            const bool ok = v < nv;
+            cp_async16_zfill(&ring.dys[b][v * 8], ok ? src + v * 8 : dy, ok ? 16 : 0);
         }
+        return shifts;
     };
+    const StemWalk walk = stem_walk<TQ>(g, strips_per_row);
     StemStrip ahead[NS - 1];  // the strips whose data are in flight, decoded once
 #pragma unroll
     for (int k = 0; k < NS - 1; ++k) {
         const long long tk = blockIdx.x + (long long)k * gridDim.x;
-        ahead[k] = stem_strip(tk < nstrips ? tk : 0, g, strips_per_row);
-        if (tk < nstrips) stage_async(ahead[k], k);
+        ahead[k] = k == 0 ? stem_strip<TQ>(tk < nstrips ? tk : 0, g, strips_per_row) : stem_advance(ahead[k > 0 ? k - 1 : 0], walk);
+        if (tk < nstrips) ahead[k].sh = stage_async(ahead[k], k);
         cp_async_commit();
     }
     int buf = 0;
@@ -490,20 +564,25 @@ __global__ void __launch_bounds__(128, 4) stem_wgrad_mma_kernel(const T* __restr
         cp_async_wait_pending<NS - 2>();
         __syncthreads();
         const long long tn = t + (long long)(NS - 1) * gridDim.x;
-        if (tn < nstrips) {
-            ahead[NS - 2] = stem_strip(tn, g, strips_per_row);
-            stage_async(ahead[NS - 2], (buf + NS - 1) % NS);
+        if (tn < nstrips) {  // (then strip tn - gridDim.x, which ahead[NS - 2] still holds, was decoded too)
+            ahead[NS - 2] = stem_advance(ahead[NS - 2], walk);
+            ahead[NS - 2].sh = stage_async(ahead[NS - 2], (buf + NS - 1) % NS);
         }
         cp_async_commit();
-        const int qw = s.q0 + warp * 16;
-        if (qw < g.wo) {
-            int sh[3], addr[NBK];
+        int addr[NBK];  // per strip: where this lane's filter positions sit in the staged rows, relative to a pixel's first element
+        {
+            int sh[3];
 #pragma unroll
-            for (int r = 0; r < 3; ++r) stem_row_start(g, s, r, sh[r]);
+            for (int r = 0; r < 3; ++r) sh[r] = (s.sh >> (3 * r)) & 7;
 #pragma unroll
             for (int nb = 0; nb < NBK; ++nb) addr[nb] = koff[nb] + (krow[nb] == 0 ? sh[0] : krow[nb] == 1 ? sh[1] : sh[2]);
-            const unsigned short* xr = &ring.xrow[buf][0][0] + 6 * (warp * 16 + tq * 2);
-            const T* st = &ring.dys[buf][warp * 16 * COUT];
+        }
+#pragma unroll 1
+        for (int tile = warp; tile < TQ / 16; tile += 4) {  // (one tile per warp with 64-pixel strips)
+            const int qw = s.q0 + tile * 16;
+            if (qw >= g.wo) break;
+            const unsigned short* xr = &ring.xrow[buf][0][0] + 6 * (tile * 16 + tq * 2);
+            const T* st = &ring.dys[buf][tile * 16 * COUT];
             // B fragments: four pixels of the tile (2t, 2t+1, 2t+8, 2t+9) x NBK filter positions.  (Pixels past the row's
             // end meet zero dy rows, so whatever defined values they read contribute nothing.)
             uint32_t bfr[NBK][2];

@@ -280,3 +280,45 @@ def test_random_shapes_through_the_glue_calls_and_the_plan_free_statistics():
         ref_invstd = 1.0 / np.sqrt(ref_var + EPS)
         assert (np.abs(f64(mean) - ref_mean) <= 2e-6 * np.sqrt(ref_mean**2 + ref_var) + 1e-7).all(), f"{what}: mean of {m} x {cc}"
         assert (np.abs(f64(invstd) - ref_invstd) / ref_invstd <= 1e-6 * (1 + ref_mean**2 / (ref_var + EPS)) + 2e-6).all(), f"{what}: invstd of {m} x {cc}"
+
+
+@pytest.mark.parametrize("strips", ["by_width", "wide", "narrow"])
+def test_random_first_layer_shapes_match_oracle(strips, monkeypatch):
+    """The network's first layer (3 -> 48 channels, 3x3, stride 2) has kernels of its own, which cut every output row into
+    strips: 320 pixels (forward) and 128 pixels (weight gradient) on rows of at least 160 output pixels, 64 otherwise.  30
+    random images per form (1-2 images, 2..78 x 2..838 pixels, even; bf16 and fp16 operands) through the training step
+    and the inference call, with the form chosen by the width as in production and with either form forced on every
+    width (NB_STEM_WIDE), so that ragged last strips, rows narrower than a strip and rows of several strips all occur."""
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    if strips != "by_width":
+        monkeypatch.setenv("NB_STEM_WIDE", "1" if strips == "wide" else "0")
+    rs = np.random.RandomState({"by_width": 505, "wide": 606, "narrow": 707}[strips])
+    for i in range(30):
+        n, h = int(rs.randint(1, 3)), 2 * int(rs.randint(1, 40))
+        w = 2 * int(rs.randint(150, 340)) if rs.rand() < 0.3 else 2 * int(rs.randint(1, 420))
+        mode = int(rs.choice([nb.NB_MODE_BF16_TC, nb.NB_MODE_F16_TC]))
+        shape = wl.ConvShape(f"first{n}x{h}x{w}", n, h, w, 3, 48, 3, 2, True)
+        inp = wl.make_inputs(shape, 35, i, bf16=True, affine="random")
+        blk = CbsBlock(shape, mode=mode, eps=EPS)
+        blk.upload(inp)
+        blk.step()
+        blk.poll()
+        out = blk.download()
+        ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, 2, EPS)
+        try:
+            parity.check_stats(out["mean"], out["invstd"], ref.y, EPS, "bf16")
+            for name in ("a", "dgamma", "dbeta", "dw", "dx", "y", "dy"):
+                parity.check(name, out[name], getattr(ref, name), "bf16")
+            rm, rv, _ = wl.make_eval_stats(shape, 35, i)
+            up = lambda a: torch.from_numpy(a).to(blk.dev)
+            o = torch.empty_like(blk.a)
+            ws = torch.empty(max(blk.plan.infer_bytes, blk.plan.bwd_bytes, 256), dtype=torch.uint8, device=blk.dev)
+            nb.nb_conv_bn_silu_infer(blk.plan, blk.x, blk.w, blk.gamma, blk.beta, up(rm), up(rv), o, ws)
+            torch.cuda.synchronize()
+            parity.check("a_eval", o.double().cpu().numpy(), oracle.cbs_infer(inp.x, inp.w, inp.gamma, inp.beta, rm, rv, 2, EPS), "bf16")
+        except AssertionError as e:
+            raise AssertionError(f"{shape.name} (draw {i}, mode {mode}, strips {strips}): {e}") from None
