@@ -92,6 +92,8 @@ struct nb_cbs_plan_s {
     bool stem_wide = false;  // the stem forward kernel takes 320-pixel strips (wide images)
     int stem_fprop_blocks = 0;  // its grid (= its partial slices)
     int stem_wgrad_blocks = 0;  // grid (= partial slices) of the stem weight-gradient kernel (128-pixel strips on wide images)
+    int stem_dgrad_blocks = 0;  // grid of the stem data-gradient kernel (at most one wave of five resident blocks per SM unless the bands alone are more)
+    int stem_dgrad_rows = 0;    // output row pairs per block
     bool profiling = false;  // when set, every kernel site is bracketed by events and the call waits for it
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     double prof_ms[SITE_COUNT] = {};
@@ -436,6 +438,7 @@ nb_status nb_cbs_plan_create(const nb_cbs_desc* d, int device, nb_cbs_plan* out)
     p->stem = d->mode != NB_MODE_F32_REF && !(d->flags & NB_CBS_FLAG_FORCE_SIMT) && g.c_in == 3 && g.k == 3 && g.stride == 2 &&
               g.c_out == 48 && g.h % 2 == 0 && g.w % 2 == 0 && g.m < (1LL << 31) && (long long)g.n * g.h * g.w * 3 < (1LL << 31);
     p->stem_blocks = (int)std::min<long long>(stem_num_strips(g), (long long)p->sm_count * 4);  // grid of the three first-layer kernels: one wave of four resident blocks per SM
+    p->stem_dgrad_blocks = stem_dgrad_grid(g, p->sm_count * 5, &p->stem_dgrad_rows);
     p->stem_wide = g.wo >= STEM_TQ_WIDE / 2;  // (a strip of a narrower row would leave most of its tile slots empty)
     if (const char* e2 = getenv("NB_STEM_WIDE")) p->stem_wide = atoi(e2) != 0;
     p->stem_fprop_blocks = p->stem_wide ? (int)std::min<long long>(stem_num_strips(g, STEM_TQ_WIDE), (long long)p->sm_count * 4) : p->stem_blocks;
@@ -831,8 +834,8 @@ nb_status nb_conv_bn_silu_bwd_data(nb_cbs_plan p, const void* g, const void* y_s
     if (!dx) return NB_OK;
     if (p->stem) {
         SiteTimer tm(p, SITE_DGRAD, st);
-        NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dy_out), static_cast<const AT*>(w),
-                               static_cast<AT*>(dx), p->g));
+        NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_dgrad_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dy_out), static_cast<const AT*>(w),
+                               static_cast<AT*>(dx), p->g, p->stem_dgrad_rows));
         return launch_ok("stem_dgrad");
     }
     if (p->tc.dgrad) {
@@ -869,8 +872,8 @@ nb_status nb_conv_bias_bwd(nb_cbs_plan p, const void* x, const void* w, const vo
                 NB_TRY(run_simt_dgrad<float>(p, dout, w, dx, st));
             } else if (p->stem) {
                 SiteTimer tm(p, SITE_DGRAD, st);
-                NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dout), static_cast<const AT*>(w),
-                                       static_cast<AT*>(dx), p->g));
+                NB_WITH_AT(p, launch_k(stem_dgrad_mma_kernel<48, AT>, dim3(p->stem_dgrad_blocks), dim3(128), 0, st, 1, static_cast<const AT*>(dout), static_cast<const AT*>(w),
+                                       static_cast<AT*>(dx), p->g, p->stem_dgrad_rows));
                 NB_LAUNCH_OK("stem_dgrad");
             } else if (p->tc.dgrad) {
                 SiteTimer tm(p, SITE_DGRAD, st);

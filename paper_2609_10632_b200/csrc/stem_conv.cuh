@@ -348,52 +348,81 @@ __global__ void __launch_bounds__(128, 4) stem_fprop_mma_kernel(const InT* __res
 // Data gradient as mma.sync tiles.  For dy position (i, j) the four input pixels (2i+a, 2j+b) receive
 //   (0,0) <- dy[i][j] w11;  (0,1) <- dy[i][j+1] w10 + dy[i][j] w12;  (1,0) <- dy[i+1][j] w01 + dy[i][j] w21;
 //   (1,1) <- dy[i+1][j+1] w00 + dy[i+1][j] w02 + dy[i][j+1] w20 + dy[i][j] w22        (w_rt = filter tap (r,t)),
-// i.e. per parity class a GEMM [16 positions x COUT] x [COUT x 3] per tap with the dy tile shifted by (0|1, 0|1): 27 MMAs
-// (N padded from 3 to 8) per 16 positions.  A block stages rows i and i+1 of a 64-position strip (plus one column) in
-// shared memory with 16-byte loads (pixel pitch 112 bytes: conflict-free ldmatrix), the 27 filter fragments stay in
-// registers, and the 2 x 32 output pixels of a warp are staged and written as 4-byte words (coalesced).
+// i.e. per parity class a GEMM [16 positions x COUT] x [COUT x 3] per tap with the dy tile shifted by (0|1, 0|1).  An MMA
+// has eight output columns and a tap fills three, so two taps that read the same shifted tile share an MMA: columns 0-2
+// belong to a class of output row parity 0, columns 3-5 to the class of parity 1 with the same column parity.  Two
+// accumulators (column parity 0 and 1) and six MMAs per 16 channels of dy instead of four accumulators and nine:
+//   parity b = 0:  dy[i][j] x [w11 | w21],  dy[i+1][j] x [0 | w01]
+//   parity b = 1:  dy[i][j] x [w12 | w22],  dy[i][j+1] x [w10 | w20],  dy[i+1][j] x [0 | w02],  dy[i+1][j+1] x [0 | w00].
+// A block stages rows i and i+1 of a 64-position strip (plus one column) in shared memory with 16-byte loads (pixel
+// pitch 112 bytes: conflict-free ldmatrix), the 18 filter fragments stay in registers, and the 2 x 32 output pixels of a
+// warp are staged and written as 4-byte words (coalesced).  Five blocks are resident per SM (96 registers, a ring of four
+// staged rows of 7.3 KB per block).  Grid: stem_dgrad_grid().
 constexpr int STEM_DYPITCH = 56;  // elements per staged dy pixel (48 channels + padding)
+// Blocks and rows per block of the data-gradient kernel: the bands (image x 64-column strip) are cut into as many row
+// segments as keep the grid within one wave of `slots` resident blocks; more bands than slots: whole bands, several waves.
+inline int stem_dgrad_grid(const Geom& g, int slots, int* seg_rows) {
+    const long long bands = (long long)g.n * ((g.wo + STEM_TQ - 1) / STEM_TQ);
+    const long long segs_wanted = bands < slots ? slots / bands : 1;
+    *seg_rows = (int)((g.ho + segs_wanted - 1) / segs_wanted);
+    const long long segs = (g.ho + *seg_rows - 1) / *seg_rows;
+    return (int)(bands * segs);
+}
 template <int COUT, typename T = __nv_bfloat16>
-__global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restrict__ dy, const T* __restrict__ w, T* __restrict__ dx, Geom g) {
+__global__ void __launch_bounds__(128, 5) stem_dgrad_mma_kernel(const T* __restrict__ dy, const T* __restrict__ w, T* __restrict__ dx, Geom g, int seg_rows) {
     pdl_launch_dependents();
     pdl_wait();
     static_assert(COUT % 16 == 0 && COUT + 8 <= STEM_DYPITCH, "whole k-steps; pitch holds a pixel");
     constexpr int KS = COUT / 16;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gq = lane >> 2, tq = lane & 3;
     const unsigned short* wsrc = reinterpret_cast<const unsigned short*>(w);
-    // B fragments: for tap (r,t) and k-step ks, element (k = channel c', n = input channel c): w[c'][r][t][c]; n >= 3 is padding
-    uint32_t bfrag[STEM_TAPS][KS][2];
+    // B fragments of the six MMAs: element (k = channel c' of dy, n = output column gq): columns 0-2 take filter tap
+    // pair[m][0], columns 3-5 tap pair[m][1] (tap = r*3 + t; -1: zeros), input channel gq % 3; columns 6, 7 are padding
+    constexpr int kPair[6][2] = {{4, 7}, {-1, 1}, {5, 8}, {3, 6}, {-1, 2}, {-1, 0}};
+    uint32_t bfrag[6][KS][2];
+    {
+        const int slot = gq >= 3 ? 1 : 0, ch = gq - 3 * slot;
 #pragma unroll
-    for (int tap = 0; tap < STEM_TAPS; ++tap)
+        for (int m = 0; m < 6; ++m) {
+            const int tap = gq < 6 ? (slot ? kPair[m][1] : kPair[m][0]) : -1;
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks)
+            for (int ks = 0; ks < KS; ++ks)
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int c0 = ks * 16 + j * 8 + tq * 2;
-                const uint32_t lo = gq < 3 ? wsrc[c0 * STEM_KDIM + tap * 3 + gq] : 0u, hi = gq < 3 ? wsrc[(c0 + 1) * STEM_KDIM + tap * 3 + gq] : 0u;
-                bfrag[tap][ks][j] = lo | (hi << 16);
-            }
-    constexpr int NS = 3;  // ring of staged strips
-    __shared__ __align__(16) T dys[NS][2][(STEM_TQ + 1) * STEM_DYPITCH];  // [buffer][row i / i+1][pixel][channel]
+                for (int j = 0; j < 2; ++j) {
+                    const int c0 = ks * 16 + j * 8 + tq * 2;
+                    const uint32_t lo = tap >= 0 ? wsrc[c0 * STEM_KDIM + tap * 3 + ch] : 0u, hi = tap >= 0 ? wsrc[(c0 + 1) * STEM_KDIM + tap * 3 + ch] : 0u;
+                    bfrag[m][ks][j] = lo | (hi << 16);
+                }
+        }
+    }
+    // Work unit of a block: output row pairs [p_lo, p_hi) of one 64-column band of one image.  Consecutive strips of a band
+    // share a dy row, so the block keeps a ring of single rows and every dy row travels to the SM once per band instead of
+    // twice; the strip arithmetic is one addition.
+    constexpr int NR = 4;  // ring of staged dy rows: two in use, two on their way
+    __shared__ __align__(16) T dyrow[NR][(STEM_TQ + 1) * STEM_DYPITCH];  // [buffer][pixel][channel]
     __shared__ __align__(16) T outs[4][2][32 * 3];
     const int strips_per_row = (g.wo + STEM_TQ - 1) / STEM_TQ;
-    const long long nstrips = stem_num_strips(g);
+    const int bands = g.n * strips_per_row;
+    const int seg = (int)blockIdx.x / bands, band = (int)blockIdx.x - seg * bands;  // (neighbouring blocks: neighbouring bands of the same rows)
+    StemStrip s;
+    s.n = band / strips_per_row;
+    s.q0 = (band - s.n * strips_per_row) * STEM_TQ;
+    s.sh = 0;
+    const int p_lo = seg * seg_rows, p_hi = p_lo + seg_rows < g.ho ? p_lo + seg_rows : g.ho;
     constexpr int VPP = COUT / 8;  // 16-byte vectors per pixel
-    // asynchronous staging of dy[i..i+1][q0 .. q0+64][:] (zeros past the last row / column).  A row's 65 pixels are one
+    // asynchronous staging of dy[row][q0 .. q0+64][:] (zeros past the last row / column).  A row's 65 pixels are one
     // contiguous run of 65 * VPP vectors in global memory; in shared memory pixels are STEM_DYPITCH apart.  A thread copies
     // vector `vec` of pixels px0, px0 + PXSTEP, ...: both addresses advance by constants (no division per copy).
     constexpr int PXSTEP = 128 / VPP, PXITER = (STEM_TQ + 1 + PXSTEP - 1) / PXSTEP;
     const int px0 = threadIdx.x / VPP, vec = threadIdx.x - px0 * VPP;
     const bool stager = px0 < PXSTEP;  // (128 threads = PXSTEP whole pixels and a remainder that stays idle)
-    auto stage_async = [&](const StemStrip& s, T(*dst)[(STEM_TQ + 1) * STEM_DYPITCH]) {
-        if (!stager) return;
-        const T* row0 = dy + (((size_t)s.n * g.ho + s.p) * g.wo + s.q0 + px0) * COUT + vec * 8;
-        const int npx = g.wo - s.q0;  // pixels of the row from q0 on
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const bool row_ok = s.p + r < g.ho;
-            const T* src = row0 + (size_t)r * g.wo * COUT;
-            T* d = &dst[r][px0 * STEM_DYPITCH + vec * 8];
+    const int npx = g.wo - s.q0;       // pixels of a row from q0 on
+    const T* const col0 = dy + ((size_t)s.n * g.ho * g.wo + s.q0 + px0) * COUT + vec * 8;
+    auto stage_row_async = [&](int row) {  // rows beyond p_hi are not needed by this block: an empty group
+        if (stager && row <= p_hi) {
+            const bool row_ok = row < g.ho;
+            const T* src = col0 + (size_t)row * g.wo * COUT;
+            T* d = &dyrow[row & (NR - 1)][px0 * STEM_DYPITCH + vec * 8];
 #pragma unroll
             for (int it = 0; it < PXITER; ++it) {
                 const int px = px0 + it * PXSTEP;
@@ -403,37 +432,24 @@ __global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restr
                 }
             }
         }
+        cp_async_commit();
     };
-    const StemWalk walk = stem_walk(g, strips_per_row);
-    StemStrip ahead[NS - 1];  // the strips whose rows are in flight, decoded once (p = dy row i, q0 = first dy column)
-#pragma unroll
-    for (int k = 0; k < NS - 1; ++k) {
-        const long long tk = blockIdx.x + (long long)k * gridDim.x;
-        ahead[k] = k == 0 ? stem_strip(tk < nstrips ? tk : 0, g, strips_per_row) : stem_advance(ahead[k > 0 ? k - 1 : 0], walk);
-        if (tk < nstrips) stage_async(ahead[k], dys[k]);
-        cp_async_commit();
-    }
-    int buf = 0;
-    for (long long t = blockIdx.x; t < nstrips; t += gridDim.x, buf = (buf + 1) % NS) {
-        const StemStrip s = ahead[0];
-#pragma unroll
-        for (int k = 0; k + 1 < NS - 1; ++k) ahead[k] = ahead[k + 1];
-        cp_async_wait_pending<NS - 2>();
-        __syncthreads();  // this strip's rows have landed; the buffer refilled below has been consumed
-        const long long tn = t + (long long)(NS - 1) * gridDim.x;
-        if (tn < nstrips) {  // (then strip tn - gridDim.x, which ahead[NS - 2] still holds, was decoded too)
-            ahead[NS - 2] = stem_advance(ahead[NS - 2], walk);
-            stage_async(ahead[NS - 2], dys[(buf + NS - 1) % NS]);
-        }
-        cp_async_commit();
+    stage_row_async(p_lo);
+    stage_row_async(p_lo + 1);
+    stage_row_async(p_lo + 2);
+    for (s.p = p_lo; s.p < p_hi; ++s.p) {
+        cp_async_wait_pending<1>();  // all groups but the newest: rows p and p + 1 have landed
+        __syncthreads();             // ... for every thread, and the buffer refilled below (row p - 1's) has been consumed
+        stage_row_async(s.p + 3);
+        const int buf = s.p & (NR - 1), buf1 = (s.p + 1) & (NR - 1);
         const int jw = s.q0 + warp * 16;  // first dy column of this warp's 16 positions
         if (jw < g.wo) {
-            float acc[4][4];  // parity class a*2+b
+            float acc[2][4];  // column parity b: columns 0-2 = row parity 0, columns 3-5 = row parity 1
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.f;
+            for (int c = 0; c < 2; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.f;
             const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: matrix and row this lane addresses
-            const T* d0 = dys[buf][0];
-            const T* d1 = dys[buf][1];
+            const T* d0 = dyrow[buf];
+            const T* d1 = dyrow[buf1];
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 uint32_t a00[4], a01[4], a10[4], a11[4];  // dy tile shifted by (di, dj)
@@ -442,31 +458,25 @@ __global__ void __launch_bounds__(128, 4) stem_dgrad_mma_kernel(const T* __restr
                 ldmatrix_x4(a01, &d0[(px + 1) * STEM_DYPITCH + ko]);
                 ldmatrix_x4(a10, &d1[px * STEM_DYPITCH + ko]);
                 ldmatrix_x4(a11, &d1[(px + 1) * STEM_DYPITCH + ko]);
-                // tap index = r*3 + t
-                mma_16816<T>(acc[0], a00, bfrag[4][ks][0], bfrag[4][ks][1]);  // (0,0): w11
-                mma_16816<T>(acc[1], a01, bfrag[3][ks][0], bfrag[3][ks][1]);  // (0,1): dy[i][j+1] w10
-                mma_16816<T>(acc[1], a00, bfrag[5][ks][0], bfrag[5][ks][1]);  //        dy[i][j]   w12
-                mma_16816<T>(acc[2], a10, bfrag[1][ks][0], bfrag[1][ks][1]);  // (1,0): dy[i+1][j] w01
-                mma_16816<T>(acc[2], a00, bfrag[7][ks][0], bfrag[7][ks][1]);  //        dy[i][j]   w21
-                mma_16816<T>(acc[3], a11, bfrag[0][ks][0], bfrag[0][ks][1]);  // (1,1): dy[i+1][j+1] w00
-                mma_16816<T>(acc[3], a10, bfrag[2][ks][0], bfrag[2][ks][1]);  //        dy[i+1][j]   w02
-                mma_16816<T>(acc[3], a01, bfrag[6][ks][0], bfrag[6][ks][1]);  //        dy[i][j+1]   w20
-                mma_16816<T>(acc[3], a00, bfrag[8][ks][0], bfrag[8][ks][1]);  //        dy[i][j]     w22
+                mma_16816<T>(acc[0], a00, bfrag[0][ks][0], bfrag[0][ks][1]);  // b = 0: dy[i][j]     x [w11 | w21]
+                mma_16816<T>(acc[1], a00, bfrag[2][ks][0], bfrag[2][ks][1]);  // b = 1: dy[i][j]     x [w12 | w22]
+                mma_16816<T>(acc[0], a10, bfrag[1][ks][0], bfrag[1][ks][1]);  // b = 0: dy[i+1][j]   x [ 0  | w01]
+                mma_16816<T>(acc[1], a01, bfrag[3][ks][0], bfrag[3][ks][1]);  // b = 1: dy[i][j+1]   x [w10 | w20]
+                mma_16816<T>(acc[1], a10, bfrag[4][ks][0], bfrag[4][ks][1]);  //        dy[i+1][j]   x [ 0  | w02]
+                mma_16816<T>(acc[1], a11, bfrag[5][ks][0], bfrag[5][ks][1]);  //        dy[i+1][j+1] x [ 0  | w00]
             }
-            // accumulator registers: c0, c1 = (position gq, channels 2tq, 2tq+1), c2, c3 = (position gq+8, same): channels 0..2 exist
+            // accumulator registers: c0, c1 = (position gq, columns 2tq, 2tq+1), c2, c3 = (position gq+8, same columns);
+            // column c < 6 = row parity c / 3, input channel c % 3
             T(*o)[32 * 3] = outs[warp];
-            if (tq < 2) {
+            if (tq < 3) {
 #pragma unroll
-                for (int a = 0; a < 2; ++a)
+                for (int e = 0; e < 2; ++e) {
+                    const int col = 2 * tq + e, a = col >= 3 ? 1 : 0, ch = col - 3 * a;
 #pragma unroll
                     for (int b = 0; b < 2; ++b)
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const int pos = gq + half * 8;
-                            T* dst = &o[a][(2 * pos + b) * 3 + tq * 2];
-                            dst[0] = from_f32<T>(acc[a * 2 + b][2 * half]);
-                            if (tq == 0) dst[1] = from_f32<T>(acc[a * 2 + b][2 * half + 1]);
-                        }
+                        for (int half = 0; half < 2; ++half) o[a][(2 * (gq + half * 8) + b) * 3 + ch] = from_f32<T>(acc[b][2 * half + e]);
+                }
             }
             __syncwarp();
             const int npos = g.wo - jw < 16 ? g.wo - jw : 16;
