@@ -322,3 +322,43 @@ def test_random_first_layer_shapes_match_oracle(strips, monkeypatch):
             parity.check("a_eval", o.double().cpu().numpy(), oracle.cbs_infer(inp.x, inp.w, inp.gamma, inp.beta, rm, rv, 2, EPS), "bf16")
         except AssertionError as e:
             raise AssertionError(f"{shape.name} (draw {i}, mode {mode}, strips {strips}): {e}") from None
+
+
+def test_random_shapes_on_the_other_paths_match_oracle():
+    """The paths beside the default one on 60 random shapes, one of the three per shape: the fp32 reference mode (CUDA-core
+    kernels, fp32 tensors; bar 1e-5), the CUDA-core kernels forced in bf16 mode, and the fixed-order statistics kernels
+    (NB_CBS_FLAG_SEPARATE_FINALIZE) under the tensor-core convolutions."""
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    rs = np.random.RandomState(808)
+    seen = set()
+    for i in range(60):
+        s = _draw(rs)
+        which = int(rs.randint(0, 3))
+        if which == 0 and s.c_out % 4:
+            continue  # (fp32 mode reads the channels as 16-byte vectors)
+        mode, flags = [(nb.NB_MODE_F32_REF, 0), (nb.NB_MODE_BF16_TC, nb.NB_CBS_FLAG_FORCE_SIMT), (nb.NB_MODE_BF16_TC, nb.NB_CBS_FLAG_SEPARATE_FINALIZE)][which]
+        inp = wl.make_inputs(s, 37, i, bf16=(which != 0), affine="random")
+        blk = CbsBlock(s, mode=mode, eps=EPS, flags=flags)
+        blk.upload(inp)
+        blk.step()
+        blk.poll()
+        out = blk.download()
+        ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, s.stride, EPS)
+        tag = "f32" if which == 0 else "bf16"
+        try:
+            parity.check_stats(out["mean"], out["invstd"], ref.y, EPS, tag)
+            for name in ("a", "dgamma", "dbeta", "dw", "y", "dy"):
+                parity.check(name, out[name], getattr(ref, name), tag)
+            if s.k == 1 and s.stride == 2:  # (see _check_dx; fp32 mode has only the relative L2 bar)
+                assert not out["dx"][:, 1::2].any() and not out["dx"][:, :, 1::2].any()
+                parity.check("dx", out["dx"][:, ::2, ::2, :], ref.dx[:, ::2, ::2, :], tag)
+            else:
+                parity.check("dx", out["dx"], ref.dx, tag)
+        except AssertionError as e:
+            raise AssertionError(f"{s.name} (draw {i}, path {which}, {blk.plan.paths}): {e}") from None
+        if which == 1:
+            assert blk.plan.paths == {"fprop": 0, "dgrad": 0, "wgrad": 0}
+        seen.add(which)
+    assert seen == {0, 1, 2}
