@@ -279,6 +279,12 @@ __device__ __forceinline__ void tma_load_2d_u32_if(uint32_t issue, uint32_t dst,
                  "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1)
                  : "memory");
 }
+// Tiled 4-D load (no multicast): coordinates innermost first; a coordinate outside the tensor reads zeros.
+__device__ __forceinline__ void tma_load_4d_u32_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(NB_PRED_OPEN "@q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2, {%4, %5, %6, %7}], [%3];\n\t}\n" ::"r"(issue),
+                 "r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_load_im2col_4d_u32_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, uint32_t bar, int c, int w, int h, int n,
                                                           uint16_t off_w, uint16_t off_h) {
     asm volatile(NB_PRED_OPEN

@@ -809,6 +809,11 @@ struct TcPlan {
     size_t wg_smem = 0;
     const void* wg_a_ptr = nullptr;
     const void* wg_b_ptr = nullptr;
+    // 3x3 stride-1 layers with an image width that is a multiple of 16: the row-tile form (tc_wgrad_rows_kernel)
+    bool wgrad_rows = false;
+    WgradRowsParams wr;
+    int wr_grid = 0;
+    size_t wr_smem = 0;
 };
 
 namespace tcdetail {
@@ -984,6 +989,21 @@ inline bool encode_tiled_2d(CUtensorMap* m, const void* base, long long rows, lo
     return true;
 }
 
+// tiled map over a bf16 NHWC tensor [N][H][W][C] (pixel pitch ld elements, 0 = dense): box = KC channels x box_w columns of one row.
+inline bool encode_tiled_nhwc(CUtensorMap* m, const void* base, int N, int H, int W, int C, int KC, int box_w, long long ld = 0) {
+    DriverFns& d = driver();
+    if (!d.tiled) { err() = "cuTensorMapEncodeTiled is not available from the driver"; return false; }
+    const cuuint64_t pitch = (cuuint64_t)(ld ? ld : C);
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[3] = {pitch * 2, (cuuint64_t)W * pitch * 2, (cuuint64_t)H * W * pitch * 2};
+    cuuint32_t box[4] = {(cuuint32_t)KC, (cuuint32_t)box_w, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = d.tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         tma_swizzle_for(KC), CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { err() = "cuTensorMapEncodeTiled (NHWC) failed with code " + std::to_string((int)r); return false; }
+    return true;
+}
+
 // Tiled maps over the output matrix [rows][ldo] (16-bit elements) for the epilogue's TMA stores: one per distinct pass width.
 // ld = row pitch in elements when the output is a channel slice of a wider tensor (0: dense); f16: the elements are IEEE
 // fp16 (it matters only for reductions: a store moves bits).
@@ -1057,6 +1077,7 @@ inline nb_status tc_plan_init(TcPlan* tc, const Geom& g, bool enable, int sm_cou
         tc->inf.prm.idesc &= ~fmt;
         tc->dg.prm.idesc &= ~fmt;
         tc->wg.idesc &= ~fmt;
+        tc->wr.idesc &= ~fmt;
     }
     return st;
 }
@@ -1235,6 +1256,55 @@ inline nb_status tc_plan_init_impl(TcPlan* tc, const Geom& g, bool enable, int s
         tc->wg_grid = tiles * P.splits;
         tc->wgrad_partial_bytes = P.splits > 1 ? (size_t)P.splits * g.c_out * g.kdim * 4 : 0;
         tc->wgrad = true;
+        // the row-tile form: 3x3, stride 1, pad 1, image width a multiple of 16 (a stage is one output row: whole K = 16 steps)
+        // (layers with more than 128 output columns per tile are not bound by x traffic in the other kernel: measured equal)
+        const bool rows_wanted = getenv("NB_WG_ROWS") ? atoi(getenv("NB_WG_ROWS")) != 0 : P.acc_stride <= 128;
+        if (g.k == 3 && g.stride == 1 && g.pad == 1 && g.w % 16 == 0 && g.w + 2 <= 256 && g.wo == g.w && g.ho == g.h && rows_wanted) {
+            WgradRowsParams& R = tc->wr;
+            memset(&R, 0, sizeof R);
+            R.W = g.w; R.H = g.h; R.rows_total = g.n * g.h;
+            R.c_in = g.c_in; R.c_out = g.c_out; R.kdim = g.kdim;
+            R.cblk = (g.c_in + 63) / 64;
+            R.ksteps = g.w / 16;
+            R.blocks_total = 9 * R.cblk;
+            R.BN = P.BN; R.n_tiles = P.n_tiles; R.nblkB = P.nblkB; R.acc_stride = P.acc_stride;
+            const int max_acc = std::min(8, 512 / R.acc_stride);
+            const int total_acc = (R.blocks_total + 1) / 2;
+            R.m_tiles = (total_acc + max_acc - 1) / max_acc;
+            const int acc_per_tile = (total_acc + R.m_tiles - 1) / R.m_tiles;
+            R.blocks_per_tile = 2 * acc_per_tile;
+            R.m_tiles = (R.blocks_total + R.blocks_per_tile - 1) / R.blocks_per_tile;
+            int cols = acc_per_tile * R.acc_stride;
+            R.tmem_cols = 32;
+            while (R.tmem_cols < cols) R.tmem_cols *= 2;
+            int max_boxes = 1;  // (r, channel block) boxes that a tile's blocks read
+            for (int t = 0; t < R.m_tiles; ++t) {
+                const int tb0 = t * R.blocks_per_tile, tb1 = std::min(R.blocks_total, tb0 + R.blocks_per_tile);
+                max_boxes = std::max(max_boxes, (tb1 - 1) / 3 - tb0 / 3 + 1);
+            }
+            R.a_box_bytes = (uint32_t)((g.w + 2 + 7) / 8 * 8 * 128);
+            R.b_box_bytes = (uint32_t)(g.w * 128);
+            R.a_stage_bytes = (uint32_t)max_boxes * R.a_box_bytes;
+            R.b_stage_bytes = (uint32_t)R.nblkB * R.b_box_bytes;
+            R.stages = (int)std::min<size_t>(8, (kMaxSmem - 2048) / (R.a_stage_bytes + R.b_stage_bytes));
+            const int tiles = R.m_tiles * R.n_tiles;
+            int splits = std::max(1, sm_count / tiles);
+            if (getenv("NB_WG_ROWS_SPLITS")) splits = std::max(1, atoi(getenv("NB_WG_ROWS_SPLITS")) / tiles);
+            splits = std::min(splits, std::max(1, R.rows_total / 4));
+            R.rows_per_split = (R.rows_total + splits - 1) / splits;
+            R.splits = (R.rows_total + R.rows_per_split - 1) / R.rows_per_split;
+            R.stages = std::max(2, std::min(R.stages, std::max(2, R.rows_per_split)));
+            R.idesc = ptx::make_idesc_bf16(128, R.BN, 1, 1);
+            if (R.stages >= 2 && (size_t)2 * (R.a_stage_bytes + R.b_stage_bytes) + 2048 <= kMaxSmem) {
+                tc->wgrad_rows = true;
+                tc->wr_smem = std::max<size_t>(2048 + (size_t)R.stages * (R.a_stage_bytes + R.b_stage_bytes), 120 * 1024);
+                tc->wr_grid = tiles * R.splits;
+                tc->wgrad_partial_bytes = std::max(tc->wgrad_partial_bytes, R.splits > 1 ? (size_t)R.splits * g.c_out * g.kdim * 4 : (size_t)0);
+                if (getenv("NB_TC_VERBOSE"))
+                    fprintf(stderr, "[nb_cbs] wgrad by rows W=%d Cin=%d Cout=%d: %d blocks, %d per tile (%d accumulators), tiles=%dx%d splits=%d (%d rows each) stages=%d smem=%zu\n",
+                            g.w, g.c_in, g.c_out, R.blocks_total, R.blocks_per_tile, acc_per_tile, R.m_tiles, R.n_tiles, R.splits, R.rows_per_split, R.stages, tc->wr_smem);
+            }
+        }
         if (getenv("NB_TC_VERBOSE"))
             fprintf(stderr, "[nb_cbs] wgrad M=%lld Cin=%d Cout=%d k=%d: BN=%d mh=%d KP=%d stages=%d tiles=%dx%d splits=%d (chunks/split %d) grid=%d\n", (long long)g.m,
                     g.c_in, g.c_out, g.k, P.BN, P.mh, P.KP, P.stages, P.m_tiles, P.n_tiles, P.splits, P.chunks_per_split, tc->wg_grid);
@@ -1366,6 +1436,44 @@ inline nb_status tc_dgrad(TcPlan* tc, const Geom& g, const void* dy, const void*
 
 inline nb_status tc_wgrad(TcPlan* tc, const Geom& g, const void* x, const void* dy, float* dw, float* partial, int* status, cudaStream_t st) {
     using namespace tcdetail;
+    if (tc->wgrad_rows) {
+        WgradRowsParams& R = tc->wr;
+        if (tc->wg_a_ptr != x || tc->wg_b_ptr != dy) {
+            if (!encode_tiled_nhwc(&R.tmA, x, g.n, g.h, g.w, g.c_in, 64, g.w + 2, tc->ld_x)) return NB_ERR_CUDA;
+            if (!encode_tiled_2d(&R.tmB, dy, g.m, g.c_out, 64, g.w)) return NB_ERR_CUDA;
+            tc->wg_a_ptr = x; tc->wg_b_ptr = dy;
+        }
+        R.out = R.splits > 1 ? partial : dw;
+        R.status = status;
+        static std::atomic<unsigned long long> rows_attr_set{0};  // one bit per device ordinal (see launch_igemm_impl)
+        int dev = 0;
+        cudaGetDevice(&dev);
+        const unsigned long long bit = 1ull << (dev & 63);
+        if (!(rows_attr_set.load(std::memory_order_acquire) & bit)) {
+            if (cudaFuncSetAttribute(tc_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) != cudaSuccess) {
+                err() = "cannot raise the dynamic shared memory limit of the row-tile wgrad kernel";
+                return NB_ERR_CUDA;
+            }
+            rows_attr_set.fetch_or(bit, std::memory_order_release);
+        }
+        launch_k(tc_wgrad_rows_kernel, dim3(tc->wr_grid), dim3(TC_THREADS), tc->wr_smem, st, 1, R);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { err() = std::string("launch of tc_wgrad_rows_kernel failed: ") + cudaGetErrorString(e); return NB_ERR_CUDA; }
+        tc->launches += 1;
+        if (R.splits > 1) {
+            const size_t elems = (size_t)g.c_out * g.kdim;
+            static const int tall_from = getenv("NB_WG_TALL") ? atoi(getenv("NB_WG_TALL")) : 96;
+            if (R.splits >= tall_from) {  // many slices: 32 threads share an element's slices (same fp64 sum, fixed order)
+                launch_k(splitk_reduce_tall_kernel, dim3((unsigned)((elems + 31) / 32)), dim3(1024), 0, st, 1, partial, R.splits, elems, dw);
+            } else {
+                const int blocks = (int)std::min<size_t>((elems / 4 + 127) / 128 + 1, (size_t)tc->sm_count * 8);
+                launch_k(splitk_reduce_kernel, dim3(blocks), dim3(128), 0, st, 1, partial, R.splits, elems, dw);
+            }
+            if (cudaGetLastError() != cudaSuccess) { err() = "launch of splitk_reduce_kernel failed"; return NB_ERR_CUDA; }
+            tc->launches += 1;
+        }
+        return NB_OK;
+    }
     WgradParams& P = tc->wg;
     if (tc->wg_a_ptr != x || tc->wg_b_ptr != dy) {
         const int up = g.pad - (g.k - 1);

@@ -362,3 +362,58 @@ def test_random_shapes_on_the_other_paths_match_oracle():
             assert blk.plan.paths == {"fprop": 0, "dgrad": 0, "wgrad": 0}
         seen.add(which)
     assert seen == {0, 1, 2}
+
+
+def test_random_shapes_of_the_row_tile_weight_gradient_match_oracle():
+    """3x3 stride-1 layers whose width is a multiple of 16 take their weight gradient from a kernel of its own (a stage is
+    one output row; the three taps of a filter row read one staged input row at three start addresses).  40 random
+    shapes of that kind (1-3 images, 1..39 rows, widths 16..80, 16..384 channels on either side, bf16 and fp16 operands),
+    with the form chosen by the plan and with it forced on (NB_WG_ROWS=1: also where the plan prefers the other kernel),
+    against the oracle; and on a pitched x, which must give the dense run's bits."""
+    import os
+
+    import torch
+
+    from paper_2609_10632_b200 import binding as nb
+    from paper_2609_10632_b200.block import CbsBlock
+
+    channels = [16, 32, 48, 64, 80, 96, 128, 160, 192, 256, 288, 384]
+    rs = np.random.RandomState(909)
+    old = os.environ.get("NB_WG_ROWS")
+    try:
+        for i in range(40):
+            n, h, w = int(rs.randint(1, 4)), int(rs.randint(1, 40)), 16 * int(rs.randint(1, 6))
+            ci, co = int(rs.choice(channels)), int(rs.choice(channels))
+            if n * h * w * 9 * ci * co > 2e9:
+                continue
+            if i % 2:
+                os.environ["NB_WG_ROWS"] = "1"
+            else:
+                os.environ.pop("NB_WG_ROWS", None)
+            mode = int(rs.choice([nb.NB_MODE_BF16_TC, nb.NB_MODE_F16_TC]))
+            s = wl.ConvShape(f"rows{n}x{h}x{w}x{ci}->{co}", n, h, w, ci, co, 3, 1, False)
+            inp = wl.make_inputs(s, 39, i, bf16=True, affine="random")
+            blk = CbsBlock(s, mode=mode, eps=EPS)
+            blk.upload(inp)
+            blk.step()
+            blk.poll()
+            ref = oracle.cbs_fwd_bwd(inp.x, inp.w, inp.gamma, inp.beta, inp.g, 1, EPS, need_dx=False)
+            what = f"{s.name} (draw {i}, mode {mode}, forced {i % 2})"
+            parity.check(what + ": dw", blk.dw.double().cpu().numpy(), ref.dw, "bf16")
+            # x as a channel slice of a wider tensor: the same bits
+            ld, off = ci + 24, 8
+            wide = torch.randn(n, h, w, ld, device=blk.dev).to(blk.x.dtype)
+            wide[..., off:off + ci] = blk.x
+            pitched = CbsBlock(s, mode=mode, eps=EPS)
+            pitched.upload(inp)
+            pitched.plan.set_pitches(ld_x=ld)
+            dw2 = torch.empty_like(blk.dw)
+            nb.nb_conv_bn_silu_bwd_weight(pitched.plan, wide.data_ptr() + off * wide.element_size(), blk.dy, dw2, pitched.ws)
+            torch.cuda.synchronize()
+            pitched.poll()
+            assert torch.equal(dw2, blk.dw), what + ": pitched x"
+    finally:
+        if old is None:
+            os.environ.pop("NB_WG_ROWS", None)
+        else:
+            os.environ["NB_WG_ROWS"] = old
